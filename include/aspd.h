@@ -1,0 +1,228 @@
+/*
+ * aspd.h -- C ABI of the B200 (sm_100a) branch-isolated attention library.
+ *
+ * The library implements one step of one attention layer of ASPD's Hybrid Decoding
+ * Engine (Section 3.3 of the paper) under the model-side rules of Section 3.2
+ * (Eq. 1-4): during a parallel segment every branch decodes its next token against the
+ * shared prefix KV plus its own branch's KV only, all branches sharing position IDs per
+ * timestep; when the segment ends, serial decoding continues over the merged cache,
+ * which is reused as it lies (nothing is copied or re-encoded).
+ *
+ * Conventions
+ *   - "host"/"device" on every pointer says where the memory lives.  The caller owns
+ *     every buffer it passes; buffers must stay valid until the stream has passed the
+ *     call.  The library owns only plans.
+ *   - Every function returns 0 (ASPD_OK) or a negative aspd_status_t; nothing throws,
+ *     aborts or synchronises the device unless stated.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Token order: the new tokens of a step are ordered request-major, then branch, then
+ *     token inside the branch.  q, out, k_new, v_new and pos all use that order.
+ *   - Layouts: q, out [n_new][n_q_heads][head_dim]; k_new, v_new [n_new][n_kv_heads]
+ *     [head_dim]; element type per aspd_shape_t.dtype.  The K and V pools are
+ *     [n_pool_pages][n_kv_heads] tiles of page_size x head_dim elements each
+ *     (aspd_pool_bytes gives the size); the order of elements INSIDE a tile is private to
+ *     the library -- read tokens back with aspd_debug_read_token.
+ *   - Positions are 0-based.  Query head h uses KV head h / (n_q_heads / n_kv_heads).
+ *     RoPE pairs element i with i + head_dim/2 and uses inv_freq[i] = theta^(-2i/head_dim)
+ *     (the paper leaves the encoding open; this is the rotate-half convention of the
+ *     models it fine-tunes).
+ */
+#ifndef ASPD_H_
+#define ASPD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ASPD_OK = 0,
+  ASPD_ERR_INVALID_ARG = -1,    /* null pointer, negative count, wrong mode              */
+  ASPD_ERR_BAD_DESCRIPTOR = -2, /* overlapping regions, slot beyond the page table, ...  */
+  ASPD_ERR_UNSUPPORTED = -3,    /* head_dim / page_size / dtype outside what is built     */
+  ASPD_ERR_CUDA = -4,           /* a CUDA runtime call or a launch failed                 */
+  ASPD_ERR_TIMEOUT = -5,        /* a bounded device-side wait ran out (see aspd_plan_status) */
+  ASPD_ERR_NOMEM = -6,          /* host or device allocation failed at plan creation      */
+  ASPD_ERR_TOO_LARGE = -7       /* a size exceeds a stated maximum                        */
+} aspd_status_t;
+
+enum { ASPD_MODE_BRANCH = 0, ASPD_MODE_SERIAL = 1 };
+enum { ASPD_DTYPE_F32 = 0, ASPD_DTYPE_BF16 = 1 };
+enum { ASPD_KERNEL_AUTO = 0, ASPD_KERNEL_GENERIC = 1, ASPD_KERNEL_MMA = 2 };
+
+/* One request (host memory).  Logical slot s of the request lives in physical page
+ * page_ids[page_begin + s / page_size], row s % page_size. */
+typedef struct {
+  int32_t prefix_len;   /* P: shared main-branch tokens at logical slots [0, P)            */
+  int32_t n_branches;   /* N >= 0                                                           */
+  int32_t branch_begin; /* first entry of this request in the branch array                  */
+  int32_t page_begin;   /* first entry of this request in page_ids[]                        */
+  int32_t n_pages;      /* length of this request's page table                              */
+  int32_t tail_off;     /* first logical slot of the main-branch tokens written after the
+                           segment closed (page-aligned); used by serial mode              */
+  int32_t tail_len;     /* their number, including the token appended this step            */
+} aspd_request_t;
+
+/* One parallel branch (host memory). */
+typedef struct {
+  int32_t kv_off;    /* first logical slot of the branch (page-aligned)                     */
+  int32_t kv_len;    /* tokens of the branch in the cache AFTER this step's append          */
+  int32_t pos_start; /* position ID of the branch's first token; Eq. 4 gives prefix_len     */
+  int32_t q_len;     /* query tokens this step = the LAST q_len tokens (0: finished branch) */
+} aspd_branch_t;
+
+typedef struct {
+  int32_t n_q_heads, n_kv_heads;
+  int32_t head_dim;  /* 64 or 128 */
+  int32_t page_size; /* tokens per page: 16 (8, 32 also accepted by the generic kernel) */
+  int32_t dtype;     /* ASPD_DTYPE_* : element type of q, out, k_new, v_new and the pools */
+  float rope_theta;
+  float sm_scale;    /* Eq. 1's 1/sqrt(d_k), as a parameter */
+} aspd_shape_t;
+
+/* Optional knobs of plan creation (NULL = all automatic). */
+typedef struct {
+  int32_t kernel;       /* ASPD_KERNEL_* */
+  int32_t chunk_tokens; /* keys per split-K work item (multiple of page_size); 0 = auto   */
+  int32_t n_ctas;       /* size of the persistent grid; 0 = auto                           */
+  int32_t host_only;    /* 1: build the work list on the host only (no CUDA call at all);
+                           such a plan serves aspd_plan_info / aspd_plan_items only        */
+} aspd_tuning_t;
+
+/* One split-K work item of a plan, as aspd_plan_items reports it. */
+typedef struct {
+  int32_t q_tok0;     /* first new token (step order) of the item's row block               */
+  int32_t n_q_tok;    /* tokens in the block; rows = n_q_tok * (n_q_heads / n_kv_heads)     */
+  int32_t kv_head;
+  int32_t page0;      /* index into page_ids[] of the chunk's first page                    */
+  int32_t n_keys;     /* keys of the chunk, starting at row 0 of page0                      */
+  int32_t causal0;    /* token i of the block sees chunk key j iff j <= causal0 + i         */
+  int32_t part_slot;  /* which of the token's partial results this item writes              */
+  int32_t request;
+} aspd_item_t;
+
+typedef struct {
+  int32_t n_new;            /* new tokens (= query tokens) of the step                      */
+  int32_t n_items;          /* split-K work items                                           */
+  int32_t n_partials;       /* partial (m, l, O) records per query head, summed over tokens */
+  int32_t kernel;           /* ASPD_KERNEL_* actually chosen                                */
+  int32_t chunk_tokens;
+  int32_t n_ctas;
+  int64_t workspace_bytes;  /* device memory the plan holds                                 */
+  int64_t kv_tokens_read;   /* cached tokens the step must read (each once)                 */
+  int64_t algorithmic_bytes;/* K+V of those tokens + q in + out + appended K/V              */
+} aspd_plan_info_t;
+
+typedef struct aspd_plan aspd_plan_t;
+
+const char* aspd_strerror(int status);
+
+/* Bytes of one pool (K or V) with n_pages pages; 0 if the shape is unsupported. */
+size_t aspd_pool_bytes(const aspd_shape_t* shape, int64_t n_pages);
+
+/* Number of new tokens of a step: sum of q_len (branch mode) or n_req (serial mode). */
+int aspd_count_new_tokens(const aspd_request_t* req /*host*/, const aspd_branch_t* br /*host*/,
+                          int n_req, int mode);
+
+/*
+ * Position ID and logical slot of every new token (Eq. 4; Section 3.3: positions grow by
+ * one per token inside a branch, and the first serial token after a segment takes its index
+ * in the complete sequence).  Pure host integer code, no CUDA.
+ *   branch mode: i-th query of a branch -> pos_start + kv_len - q_len + i,
+ *                slot kv_off + kv_len - q_len + i
+ *   serial mode: prefix_len + sum of kv_len + tail_len - 1, slot tail_off + tail_len - 1
+ * pos_out, slot_out, req_out: host arrays of aspd_count_new_tokens entries (req_out may be NULL).
+ */
+int aspd_positions(const aspd_request_t* req, const aspd_branch_t* br, int n_req, int mode,
+                   int32_t* pos_out, int32_t* slot_out, int32_t* req_out);
+
+/*
+ * Mask membership as integers (Eq. 2-3 in descriptor form): vis_out[t * n_slots + s] = 1 iff
+ * new token t may attend logical slot s of its own request.  Host only, for tests.
+ */
+int aspd_visible_slots(const aspd_request_t* req, const aspd_branch_t* br, int n_req, int mode,
+                       int n_slots, uint8_t* vis_out /*host*/);
+
+/*
+ * Validate the descriptors and build the step's plan: new-token table, query RoPE table,
+ * split-K work list over (request, KV head, key chunk), partial-result workspace.  One plan
+ * serves every layer of the step.  All device allocation of the library happens here
+ * (unless tuning->host_only); copies are enqueued on `stream`.
+ *   page_ids      host, concatenated page tables
+ *   n_pool_pages  pages in each pool; every page id must be < n_pool_pages and unique
+ *   q_pos         host, optional (NULL = derive as aspd_positions does): RoPE position of
+ *                 each new token's query
+ * Errors: ASPD_ERR_BAD_DESCRIPTOR for overlapping or out-of-table regions, unaligned kv_off /
+ * tail_off, q_len > kv_len, serial mode with tail_len < 1, duplicate or out-of-pool page ids.
+ */
+int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const aspd_branch_t* br,
+                     const int32_t* page_ids, int n_req, int64_t n_pool_pages, int mode,
+                     const int32_t* q_pos, const aspd_tuning_t* tuning, void* stream,
+                     aspd_plan_t** plan_out);
+int aspd_plan_destroy(aspd_plan_t* plan);
+int aspd_plan_info(const aspd_plan_t* plan, aspd_plan_info_t* info /*host*/);
+/* Copy up to max_items work items to `items` (host); returns the number of items. */
+int aspd_plan_items(const aspd_plan_t* plan, aspd_item_t* items, int max_items);
+/* Device status word of the plan (synchronises `stream`): ASPD_OK, or the first error a
+ * kernel recorded (ASPD_ERR_TIMEOUT from a bounded wait, ASPD_ERR_BAD_DESCRIPTOR from a
+ * bounds check). */
+int aspd_plan_status(aspd_plan_t* plan, void* stream);
+
+/*
+ * a3: K' = RoPE(k_new, pos), V' = v_new, written into the paged cache at the slots the plan
+ * derived from the descriptors (Section 3.3: KV of parallel tokens joins the one shared
+ * cache).  pos: device int32[n_new], caller-given position IDs (aspd_positions for ASPD;
+ * other values implement position-ID variants).  RoPE in fp32 with the angle reduced in
+ * fp64; bf16 stores round to nearest even.
+ */
+int aspd_kv_append(aspd_plan_t* plan, const void* k_new /*device*/, const void* v_new /*device*/,
+                   const int32_t* pos /*device*/, void* k_pool /*device*/, void* v_pool /*device*/,
+                   void* stream);
+
+/*
+ * a4-a7: parallel-mode attention (Eq. 1 under the mask of Eq. 2-3).  Query i of branch b
+ * attends the prefix [0, P) and tokens 0 .. kv_len - q_len + i of its own branch; the prefix
+ * is read once per KV head for all branches' query heads.  Split-K partials are merged by
+ * log-sum-exp.  The plan must have been created in ASPD_MODE_BRANCH.  q is raw (un-rotated).
+ */
+int aspd_branch_attn(aspd_plan_t* plan, const void* q /*device*/, const void* k_pool /*device*/,
+                     const void* v_pool /*device*/, void* out /*device*/, void* stream);
+
+/*
+ * a9: serial-mode attention after the segment closed: one query per request attends the
+ * prefix, every token of every branch and the tail up to itself (the main branch sees the
+ * whole history, Section 3.2).  The plan must have been created in ASPD_MODE_SERIAL.
+ */
+int aspd_serial_attn(aspd_plan_t* plan, const void* q /*device*/, const void* k_pool /*device*/,
+                     const void* v_pool /*device*/, void* out /*device*/, void* stream);
+
+/*
+ * The two halves of either attention call, for callers (and profilers) that want them
+ * apart: a4-a6, the split-K pass that leaves one un-normalised (max, sum, O) record per work
+ * item and query row in the plan's workspace; and a7, the log-sum-exp merge of a token's
+ * records into `out`.  aspd_branch_attn / aspd_serial_attn are exactly these two in sequence.
+ */
+int aspd_attn_partials(aspd_plan_t* plan, const void* q /*device*/, const void* k_pool /*device*/,
+                       const void* v_pool /*device*/, void* stream);
+int aspd_attn_combine(aspd_plan_t* plan, void* out /*device*/, void* stream);
+
+/*
+ * The whole step (a3-a7 or a3 + a9, by the plan's mode) from HOST buffers: copies q, k_new,
+ * v_new, pos to staging memory the plan owns, runs append + attention, copies out back, all
+ * on `stream`, then synchronises it.  The pools stay on the device (they are the state).
+ */
+int aspd_step_host(aspd_plan_t* plan, const void* q /*host*/, const void* k_new /*host*/,
+                   const void* v_new /*host*/, const int32_t* pos /*host*/, void* k_pool /*device*/,
+                   void* v_pool /*device*/, void* out /*host*/, void* stream);
+
+/* Read one cached token (physical page, row, KV head) back as head_dim floats (host).
+ * Synchronises `stream`.  For tests. */
+int aspd_debug_read_token(const aspd_shape_t* shape, const void* pool /*device*/, int64_t page,
+                          int row, int kv_head, float* out /*host*/, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASPD_H_ */

@@ -1,0 +1,250 @@
+"""Thin Python binding of the C ABI in ``include/aspd.h`` (argument marshalling only).
+
+Every step of the path runs in the CUDA library; nothing here computes.  Descriptors are
+given as a dict of int32 numpy arrays (struct of arrays, the form the workload generator
+emits) and packed into the C structs.  Device buffers are torch tensors (or anything with
+``data_ptr()``), host buffers numpy arrays.  There is no CPU fallback: if the library is
+missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, Optional
+
+import numpy as np
+
+from . import build as _build
+
+MODE_BRANCH, MODE_SERIAL = 0, 1
+DTYPE_F32, DTYPE_BF16 = 0, 1
+KERNEL_AUTO, KERNEL_GENERIC, KERNEL_MMA = 0, 1, 2
+
+REQUEST_DTYPE = np.dtype([(n, np.int32) for n in
+                          ("prefix_len", "n_branches", "branch_begin", "page_begin", "n_pages", "tail_off", "tail_len")])
+BRANCH_DTYPE = np.dtype([(n, np.int32) for n in ("kv_off", "kv_len", "pos_start", "q_len")])
+ITEM_DTYPE = np.dtype([(n, np.int32) for n in
+                       ("q_tok0", "n_q_tok", "kv_head", "page0", "n_keys", "causal0", "part_slot", "request")])
+
+
+class Shape(ctypes.Structure):
+    _fields_ = [("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+                ("page_size", ctypes.c_int32), ("dtype", ctypes.c_int32), ("rope_theta", ctypes.c_float),
+                ("sm_scale", ctypes.c_float)]
+
+
+class Tuning(ctypes.Structure):
+    _fields_ = [("kernel", ctypes.c_int32), ("chunk_tokens", ctypes.c_int32), ("n_ctas", ctypes.c_int32),
+                ("host_only", ctypes.c_int32)]
+
+
+class PlanInfo(ctypes.Structure):
+    _fields_ = [("n_new", ctypes.c_int32), ("n_items", ctypes.c_int32), ("n_partials", ctypes.c_int32),
+                ("kernel", ctypes.c_int32), ("chunk_tokens", ctypes.c_int32), ("n_ctas", ctypes.c_int32),
+                ("workspace_bytes", ctypes.c_int64), ("kv_tokens_read", ctypes.c_int64),
+                ("algorithmic_bytes", ctypes.c_int64)]
+
+
+class AspdError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {strerror(status)} ({status})")
+
+
+EXPORTS = ("aspd_strerror", "aspd_pool_bytes", "aspd_count_new_tokens", "aspd_positions", "aspd_visible_slots",
+           "aspd_plan_create", "aspd_plan_destroy", "aspd_plan_info", "aspd_plan_items", "aspd_plan_status",
+           "aspd_kv_append", "aspd_branch_attn", "aspd_serial_attn", "aspd_attn_partials", "aspd_attn_combine",
+           "aspd_step_host", "aspd_debug_read_token")
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library (building it first if the sources are newer).  Fails loudly."""
+    global _lib
+    if _lib is None:
+        path = _build.build()
+        L = ctypes.CDLL(path)
+        L.aspd_strerror.restype = ctypes.c_char_p
+        L.aspd_strerror.argtypes = [ctypes.c_int]
+        L.aspd_pool_bytes.restype = ctypes.c_size_t
+        L.aspd_pool_bytes.argtypes = [ctypes.c_void_p, ctypes.c_int64]
+        vp, ci = ctypes.c_void_p, ctypes.c_int
+        L.aspd_count_new_tokens.argtypes = [vp, vp, ci, ci]
+        L.aspd_positions.argtypes = [vp, vp, ci, ci, vp, vp, vp]
+        L.aspd_visible_slots.argtypes = [vp, vp, ci, ci, ci, vp]
+        L.aspd_plan_create.argtypes = [vp, vp, vp, vp, ci, ctypes.c_int64, ci, vp, vp, vp, vp]
+        L.aspd_plan_destroy.argtypes = [vp]
+        L.aspd_plan_info.argtypes = [vp, vp]
+        L.aspd_plan_items.argtypes = [vp, vp, ci]
+        L.aspd_plan_status.argtypes = [vp, vp]
+        L.aspd_kv_append.argtypes = [vp] * 7
+        L.aspd_branch_attn.argtypes = [vp] * 6
+        L.aspd_serial_attn.argtypes = [vp] * 6
+        L.aspd_attn_partials.argtypes = [vp] * 5
+        L.aspd_attn_combine.argtypes = [vp] * 3
+        L.aspd_step_host.argtypes = [vp] * 9
+        L.aspd_debug_read_token.argtypes = [vp, vp, ctypes.c_int64, ci, ci, vp, vp]
+        for name in EXPORTS:
+            if name not in ("aspd_strerror", "aspd_pool_bytes"):
+                getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def strerror(status: int) -> str:
+    return lib().aspd_strerror(int(status)).decode()
+
+
+def _check(rc: int, where: str) -> int:
+    if rc < 0:
+        raise AspdError(rc, where)
+    return rc
+
+
+def _ptr(x) -> Optional[int]:
+    if x is None:
+        return None
+    if isinstance(x, np.ndarray):
+        assert x.flags.c_contiguous
+        return x.ctypes.data
+    return x.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream if torch.cuda.is_available() else None
+    return getattr(stream, "cuda_stream", stream)
+
+
+def make_shape(n_q_heads, n_kv_heads, head_dim, page_size, dtype, rope_theta, sm_scale) -> Shape:
+    code = {"f32": DTYPE_F32, "bf16": DTYPE_BF16}.get(dtype, dtype)
+    return Shape(n_q_heads, n_kv_heads, head_dim, page_size, code, rope_theta, sm_scale)
+
+
+def pack_descriptors(desc: Dict[str, np.ndarray]):
+    """dict of int32 arrays -> (aspd_request_t[], aspd_branch_t[], page_ids) numpy arrays.
+
+    A missing ``br_pos_start`` is filled with the request's prefix length, the paper's
+    shared position-ID rule (Eq. 4: stage_start)."""
+    n_req = len(desc["prefix_len"])
+    req = np.zeros(n_req, dtype=REQUEST_DTYPE)
+    for name in REQUEST_DTYPE.names:
+        req[name] = desc[name]
+    n_br = len(desc["br_kv_off"])
+    br = np.zeros(n_br, dtype=BRANCH_DTYPE)
+    br["kv_off"], br["kv_len"], br["q_len"] = desc["br_kv_off"], desc["br_kv_len"], desc["br_q_len"]
+    if "br_pos_start" in desc:
+        br["pos_start"] = desc["br_pos_start"]
+    else:
+        for r in range(n_req):
+            b0 = int(req["branch_begin"][r])
+            br["pos_start"][b0:b0 + int(req["n_branches"][r])] = req["prefix_len"][r]
+    pages = np.ascontiguousarray(desc["page_ids"], dtype=np.int32)
+    return req, br, pages
+
+
+def pool_bytes(shape: Shape, n_pages: int) -> int:
+    return int(lib().aspd_pool_bytes(ctypes.addressof(shape), n_pages))
+
+
+def count_new_tokens(desc, mode: int) -> int:
+    req, br, _ = pack_descriptors(desc)
+    return _check(lib().aspd_count_new_tokens(_ptr(req), _ptr(br), len(req), mode), "aspd_count_new_tokens")
+
+
+def positions(desc, mode: int):
+    """(pos, slot, request) int32 arrays of the step's new tokens (host integer code in the library)."""
+    req, br, _ = pack_descriptors(desc)
+    n = _check(lib().aspd_count_new_tokens(_ptr(req), _ptr(br), len(req), mode), "aspd_count_new_tokens")
+    pos, slot, rq = (np.zeros(max(n, 1), dtype=np.int32) for _ in range(3))
+    _check(lib().aspd_positions(_ptr(req), _ptr(br), len(req), mode, _ptr(pos), _ptr(slot), _ptr(rq)), "aspd_positions")
+    return pos[:n], slot[:n], rq[:n]
+
+
+def visible_slots(desc, mode: int, n_slots: int) -> np.ndarray:
+    req, br, _ = pack_descriptors(desc)
+    n = _check(lib().aspd_count_new_tokens(_ptr(req), _ptr(br), len(req), mode), "aspd_count_new_tokens")
+    vis = np.zeros((max(n, 1), n_slots), dtype=np.uint8)
+    _check(lib().aspd_visible_slots(_ptr(req), _ptr(br), len(req), mode, n_slots, _ptr(vis)), "aspd_visible_slots")
+    return vis[:n]
+
+
+class Plan:
+    """Owner of an ``aspd_plan_t`` (see ``aspd_plan_create``)."""
+
+    def __init__(self, shape: Shape, desc, n_pool_pages: int, mode: int, q_pos=None, kernel: int = KERNEL_AUTO,
+                 chunk_tokens: int = 0, n_ctas: int = 0, host_only: bool = False, stream=None):
+        self.shape, self.mode = shape, mode
+        req, br, pages = pack_descriptors(desc)
+        tune = Tuning(kernel, chunk_tokens, n_ctas, 1 if host_only else 0)
+        qp = None if q_pos is None else np.ascontiguousarray(q_pos, dtype=np.int32)
+        handle = ctypes.c_void_p()
+        self._h = None
+        _check(lib().aspd_plan_create(ctypes.addressof(shape), _ptr(req), _ptr(br), _ptr(pages), len(req), n_pool_pages,
+                                      mode, _ptr(qp), ctypes.addressof(tune), None if host_only else _stream(stream),
+                                      ctypes.addressof(handle)), "aspd_plan_create")
+        self._h = handle
+        self.info = PlanInfo()
+        _check(lib().aspd_plan_info(self._h, ctypes.addressof(self.info)), "aspd_plan_info")
+        self.n_new = self.info.n_new
+
+    def items(self) -> np.ndarray:
+        items = np.zeros(max(self.info.n_items, 1), dtype=ITEM_DTYPE)
+        _check(lib().aspd_plan_items(self._h, _ptr(items), self.info.n_items), "aspd_plan_items")
+        return items[: self.info.n_items]
+
+    def status(self, stream=None) -> int:
+        return lib().aspd_plan_status(self._h, _stream(stream))
+
+    def destroy(self):
+        if self._h is not None:
+            lib().aspd_plan_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def kv_append(plan: Plan, k_new, v_new, pos, k_pool, v_pool, stream=None) -> None:
+    _check(lib().aspd_kv_append(plan._h, _ptr(k_new), _ptr(v_new), _ptr(pos), _ptr(k_pool), _ptr(v_pool), _stream(stream)),
+           "aspd_kv_append")
+
+
+def branch_attn(plan: Plan, q, k_pool, v_pool, out, stream=None) -> None:
+    _check(lib().aspd_branch_attn(plan._h, _ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(out), _stream(stream)),
+           "aspd_branch_attn")
+
+
+def serial_attn(plan: Plan, q, k_pool, v_pool, out, stream=None) -> None:
+    _check(lib().aspd_serial_attn(plan._h, _ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(out), _stream(stream)),
+           "aspd_serial_attn")
+
+
+def attn_partials(plan: Plan, q, k_pool, v_pool, stream=None) -> None:
+    _check(lib().aspd_attn_partials(plan._h, _ptr(q), _ptr(k_pool), _ptr(v_pool), _stream(stream)), "aspd_attn_partials")
+
+
+def attn_combine(plan: Plan, out, stream=None) -> None:
+    _check(lib().aspd_attn_combine(plan._h, _ptr(out), _stream(stream)), "aspd_attn_combine")
+
+
+def step_host(plan: Plan, q, k_new, v_new, pos, k_pool, v_pool, out, stream=None) -> None:
+    """Whole step from host (numpy / pinned torch CPU) buffers; ``out`` is a host buffer."""
+    _check(lib().aspd_step_host(plan._h, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(pos), _ptr(k_pool), _ptr(v_pool),
+                                _ptr(out), _stream(stream)), "aspd_step_host")
+
+
+def debug_read_token(shape: Shape, pool, page: int, row: int, kv_head: int, stream=None) -> np.ndarray:
+    out = np.zeros(shape.head_dim, dtype=np.float32)
+    _check(lib().aspd_debug_read_token(ctypes.addressof(shape), _ptr(pool), page, row, kv_head, _ptr(out), _stream(stream)),
+           "aspd_debug_read_token")
+    return out

@@ -1,0 +1,221 @@
+// Small kernels: RoPE + paged append (a3), the generic CUDA-core attention kernel (any
+// supported dtype / head_dim / page_size), the log-sum-exp combine (a7) and a debug reader.
+#include "aspd_internal.cuh"
+
+namespace aspd {
+
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+
+template <typename T> __device__ inline float to_f32(T x);
+template <> __device__ inline float to_f32<float>(float x) { return x; }
+template <> __device__ inline float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ inline T from_f32(float x);
+template <> __device__ inline float from_f32<float>(float x) { return x; }
+template <> __device__ inline __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// ------------------------------------------------------------------------------- append
+// One block per (new token, KV head); thread i rotates the pair (i, i + d/2).
+template <typename T>
+__global__ void append_kernel(const T* __restrict__ k_new, const T* __restrict__ v_new, const int32_t* __restrict__ pos,
+                              const int32_t* __restrict__ tok_page, const int32_t* __restrict__ tok_row,
+                              const double* __restrict__ inv_freq, T* __restrict__ k_pool, T* __restrict__ v_pool,
+                              int n_kv_heads, int head_dim, int page_size) {
+  const int t = blockIdx.x / n_kv_heads, h = blockIdx.x % n_kv_heads, i = threadIdx.x, half = head_dim / 2;
+  if (i >= half) return;
+  // angle reduced to [-pi, pi] in fp64, then fp32 sincos: the error stays near 1e-7 rad
+  // however large the position is
+  double a = (double)pos[t] * inv_freq[i];
+  a -= rint(a * 0.15915494309189535) * 6.283185307179586;
+  float sn, cs;
+  sincosf((float)a, &sn, &cs);
+  const size_t src = ((size_t)t * n_kv_heads + h) * head_dim;
+  const float x0 = to_f32(k_new[src + i]), x1 = to_f32(k_new[src + i + half]);
+  const float y0 = x0 * cs - x1 * sn, y1 = x1 * cs + x0 * sn;
+  const size_t tile = ((size_t)tok_page[t] * n_kv_heads + h) * tile_bytes(page_size, head_dim, sizeof(T));
+  const int row = tok_row[t];
+  const uint32_t o0 = tile_offset(row, i * sizeof(T), page_size), o1 = tile_offset(row, (i + half) * sizeof(T), page_size);
+  char* kp = reinterpret_cast<char*>(k_pool) + tile;
+  char* vp = reinterpret_cast<char*>(v_pool) + tile;
+  *reinterpret_cast<T*>(kp + o0) = from_f32<T>(y0);
+  *reinterpret_cast<T*>(kp + o1) = from_f32<T>(y1);
+  *reinterpret_cast<T*>(vp + o0) = v_new[src + i];
+  *reinterpret_cast<T*>(vp + o1) = v_new[src + i + half];
+}
+
+// ------------------------------------------------------------------- generic attention
+// One block per work item, one warp per query row at a time.  Lane j scores key j of each
+// group of 32 keys (a full dot product against the rotated, pre-scaled query held in shared
+// memory); the weighted V sum is taken with each lane owning D/32 output elements.
+template <typename T, int D>
+__global__ void __launch_bounds__(128) attn_generic_kernel(PlanDevice pd, const T* __restrict__ q,
+                                                           const T* __restrict__ k_pool, const T* __restrict__ v_pool,
+                                                           int n_q_heads, int n_kv_heads, int page_size, float scale_log2) {
+  constexpr int EPL = D / 32;                 // output elements per lane
+  constexpr int EPC = 16 / (int)sizeof(T);    // elements per 16-byte chunk
+  __shared__ float q_s[4][D];
+  const DeviceItem it = pd.items[blockIdx.x];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = n_q_heads / n_kv_heads, n_rows = it.n_q_tok * G;
+  const size_t tb = tile_bytes(page_size, D, sizeof(T));
+  for (int r = warp; r < n_rows; r += 4) {
+    const int tl = r / G, g = r % G, tok = it.q_tok0 + tl, hq = it.kv_head * G + g;
+    // rotate the query at its own position (table built on the host in fp64), fold in the scale
+    const T* qrow = q + ((size_t)tok * n_q_heads + hq) * D;
+    for (int i = lane; i < D / 2; i += 32) {
+      const float2 cs = pd.q_cs[(size_t)tok * (D / 2) + i];
+      const float x0 = to_f32(qrow[i]), x1 = to_f32(qrow[i + D / 2]);
+      q_s[warp][i] = (x0 * cs.x - x1 * cs.y) * scale_log2;
+      q_s[warp][i + D / 2] = (x1 * cs.x + x0 * cs.y) * scale_log2;
+    }
+    __syncwarp();
+    long lim = (long)it.causal0 + tl + 1;
+    const int limit = (int)(lim < 0 ? 0 : (lim > it.n_keys ? it.n_keys : lim));
+    float m = -INFINITY, l = 0.f, acc[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+    for (int base = 0; base < limit; base += 32) {
+      const int j = base + lane;
+      float s = -INFINITY;
+      if (j < limit) {
+        const int page = pd.page_ids[it.page0 + j / page_size], row = j % page_size;
+        const char* tile = reinterpret_cast<const char*>(k_pool) + ((size_t)page * n_kv_heads + it.kv_head) * tb;
+        float dot = 0.f;
+#pragma unroll 4
+        for (int c = 0; c < D / EPC; ++c) {
+          const uint4 raw = *reinterpret_cast<const uint4*>(tile + tile_offset(row, c * 16, page_size));
+          const T* e8 = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+          for (int e = 0; e < EPC; ++e) dot = fmaf(q_s[warp][c * EPC + e], to_f32(e8[e]), dot);
+        }
+        s = dot;
+      }
+      float mx = s;
+#pragma unroll
+      for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      const float m_new = fmaxf(m, mx);
+      const float p = j < limit ? exp2f(s - m_new) : 0.f;
+      const float alpha = exp2f(m - m_new);           // m = -inf on the first group: alpha = 0
+      float ps = p;
+#pragma unroll
+      for (int o = 16; o; o >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
+      l = l * alpha + ps;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) acc[e] *= alpha;
+      const int cnt = min(32, limit - base);
+      for (int jj = 0; jj < cnt; ++jj) {
+        const float pj = __shfl_sync(0xffffffffu, p, jj);
+        const int key = base + jj;
+        const int page = pd.page_ids[it.page0 + key / page_size], row = key % page_size;
+        const char* tile = reinterpret_cast<const char*>(v_pool) + ((size_t)page * n_kv_heads + it.kv_head) * tb;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+          const T v = *reinterpret_cast<const T*>(tile + tile_offset(row, (lane * EPL + e) * sizeof(T), page_size));
+          acc[e] = fmaf(pj, to_f32(v), acc[e]);
+        }
+      }
+      m = m_new;
+    }
+    const size_t rec = (size_t)(pd.part_base[tok] + it.part_slot) * n_q_heads + hq;
+    if (lane == 0) pd.ws_ml[rec] = make_float2(m, l);
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) pd.ws_o[rec * D + lane * EPL + e] = acc[e];
+    __syncwarp();
+  }
+}
+
+// ------------------------------------------------------------------------------ combine
+// One warp per (new token, query head): merge the token's partial records.
+template <typename T>
+__global__ void combine_kernel(PlanDevice pd, T* __restrict__ out, int n_new, int n_q_heads, int head_dim) {
+  const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (w >= n_new * n_q_heads) return;
+  const int tok = w / n_q_heads, hq = w % n_q_heads;
+  const int p0 = pd.part_base[tok], p1 = pd.part_base[tok + 1];
+  float M = -INFINITY;
+  for (int p = p0; p < p1; ++p) M = fmaxf(M, pd.ws_ml[(size_t)p * n_q_heads + hq].x);
+  float L = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
+  const int epl = head_dim / 32;
+  for (int p = p0; p < p1; ++p) {
+    const size_t rec = (size_t)p * n_q_heads + hq;
+    const float2 ml = pd.ws_ml[rec];
+    if (ml.y == 0.f) continue;                        // a chunk with no visible key
+    const float w8 = exp2f(ml.x - M);
+    L += ml.y * w8;
+    for (int e = 0; e < epl; ++e) acc[e] = fmaf(pd.ws_o[rec * head_dim + lane * epl + e], w8, acc[e]);
+  }
+  const float inv = 1.f / L;
+  for (int e = 0; e < epl; ++e) out[((size_t)tok * n_q_heads + hq) * head_dim + lane * epl + e] = from_f32<T>(acc[e] * inv);
+}
+
+template <typename T>
+__global__ void read_token_kernel(const T* pool, size_t tile, int row, int page_size, float* out) {
+  const int e = threadIdx.x;
+  out[e] = to_f32(*reinterpret_cast<const T*>(reinterpret_cast<const char*>(pool) + tile + tile_offset(row, e * sizeof(T), page_size)));
+}
+
+inline int check_launch() { return cudaGetLastError() == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA; }
+
+}  // namespace
+
+int launch_append(const aspd_plan* p, const void* k_new, const void* v_new, const int32_t* pos, void* k_pool,
+                  void* v_pool, cudaStream_t s) {
+  const aspd_shape_t& sh = p->shape;
+  const dim3 grid(p->n_new * sh.n_kv_heads), block(sh.head_dim / 2);
+  if (sh.dtype == ASPD_DTYPE_BF16)
+    append_kernel<__nv_bfloat16><<<grid, block, 0, s>>>((const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, pos,
+                                                        p->dev.tok_page, p->dev.tok_row, p->dev.inv_freq,
+                                                        (__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool, sh.n_kv_heads,
+                                                        sh.head_dim, sh.page_size);
+  else
+    append_kernel<float><<<grid, block, 0, s>>>((const float*)k_new, (const float*)v_new, pos, p->dev.tok_page,
+                                                p->dev.tok_row, p->dev.inv_freq, (float*)k_pool, (float*)v_pool,
+                                                sh.n_kv_heads, sh.head_dim, sh.page_size);
+  return check_launch();
+}
+
+int launch_attn_generic(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, cudaStream_t s) {
+  const aspd_shape_t& sh = p->shape;
+  if (p->n_items == 0) return ASPD_OK;
+  const float sc = sh.sm_scale * kLog2e;
+  const dim3 grid(p->n_items), block(128);
+#define ASPD_GEN(T, D)                                                                                         \
+  attn_generic_kernel<T, D><<<grid, block, 0, s>>>(p->dev, (const T*)q, (const T*)k_pool, (const T*)v_pool,    \
+                                                   sh.n_q_heads, sh.n_kv_heads, sh.page_size, sc)
+  if (sh.dtype == ASPD_DTYPE_BF16 && sh.head_dim == 128) ASPD_GEN(__nv_bfloat16, 128);
+  else if (sh.dtype == ASPD_DTYPE_BF16) ASPD_GEN(__nv_bfloat16, 64);
+  else if (sh.head_dim == 128) ASPD_GEN(float, 128);
+  else ASPD_GEN(float, 64);
+#undef ASPD_GEN
+  return check_launch();
+}
+
+int launch_combine(const aspd_plan* p, void* out, cudaStream_t s) {
+  const aspd_shape_t& sh = p->shape;
+  const int warps = p->n_new * sh.n_q_heads;
+  const dim3 block(128), grid((warps + 3) / 4);
+  if (sh.dtype == ASPD_DTYPE_BF16)
+    combine_kernel<__nv_bfloat16><<<grid, block, 0, s>>>(p->dev, (__nv_bfloat16*)out, p->n_new, sh.n_q_heads, sh.head_dim);
+  else
+    combine_kernel<float><<<grid, block, 0, s>>>(p->dev, (float*)out, p->n_new, sh.n_q_heads, sh.head_dim);
+  return check_launch();
+}
+
+int launch_read_token(const aspd_shape_t* sh, const void* pool, int64_t page, int row, int kv_head, float* out_dev,
+                      cudaStream_t s) {
+  const int es = esize_of(sh->dtype);
+  const size_t tile = ((size_t)page * sh->n_kv_heads + kv_head) * tile_bytes(sh->page_size, sh->head_dim, es);
+  if (sh->dtype == ASPD_DTYPE_BF16)
+    read_token_kernel<__nv_bfloat16><<<1, sh->head_dim, 0, s>>>((const __nv_bfloat16*)pool, tile, row, sh->page_size, out_dev);
+  else
+    read_token_kernel<float><<<1, sh->head_dim, 0, s>>>((const float*)pool, tile, row, sh->page_size, out_dev);
+  return check_launch();
+}
+
+// Until the tensor-core kernel exists the MMA selection falls back to the generic GPU kernel.
+int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, cudaStream_t s) {
+  return launch_attn_generic(p, q, k_pool, v_pool, s);
+}
+
+}  // namespace aspd

@@ -1,0 +1,517 @@
+// Host side of the library: descriptor validation, position IDs and slots (integer rules of
+// Eq. 4 and Section 3.3), the split-K work list, plan life cycle and the C entry points.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "aspd_internal.cuh"
+
+using namespace aspd;
+
+namespace {
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int check_shape(const aspd_shape_t* s) {
+  if (!s) return ASPD_ERR_INVALID_ARG;
+  if (s->n_q_heads <= 0 || s->n_kv_heads <= 0 || s->n_q_heads % s->n_kv_heads) return ASPD_ERR_INVALID_ARG;
+  if (s->head_dim != 64 && s->head_dim != 128) return ASPD_ERR_UNSUPPORTED;
+  if (s->dtype != ASPD_DTYPE_F32 && s->dtype != ASPD_DTYPE_BF16) return ASPD_ERR_UNSUPPORTED;
+  if (s->page_size != 8 && s->page_size != 16 && s->page_size != 32) return ASPD_ERR_UNSUPPORTED;
+  if (s->n_q_heads / s->n_kv_heads > kMaxRowsPerItem) return ASPD_ERR_UNSUPPORTED;
+  if (!(s->rope_theta > 0.f) || !(s->sm_scale > 0.f)) return ASPD_ERR_INVALID_ARG;
+  return ASPD_OK;
+}
+
+// Structural checks that need no page table: counts, q_len <= kv_len, tail in serial mode.
+int check_counts(const aspd_request_t* req, const aspd_branch_t* br, int n_req, int mode) {
+  if (n_req < 0 || (n_req > 0 && !req)) return ASPD_ERR_INVALID_ARG;
+  if (mode != ASPD_MODE_BRANCH && mode != ASPD_MODE_SERIAL) return ASPD_ERR_INVALID_ARG;
+  for (int r = 0; r < n_req; ++r) {
+    const aspd_request_t& q = req[r];
+    if (q.prefix_len < 0 || q.n_branches < 0 || q.branch_begin < 0 || q.tail_len < 0 || q.tail_off < 0)
+      return ASPD_ERR_BAD_DESCRIPTOR;
+    if (q.n_branches > 0 && !br) return ASPD_ERR_INVALID_ARG;
+    for (int b = 0; b < q.n_branches; ++b) {
+      const aspd_branch_t& x = br[q.branch_begin + b];
+      if (x.kv_off < 0 || x.kv_len < 0 || x.q_len < 0 || x.q_len > x.kv_len || x.pos_start < 0)
+        return ASPD_ERR_BAD_DESCRIPTOR;
+    }
+    if (mode == ASPD_MODE_SERIAL && q.tail_len < 1) return ASPD_ERR_BAD_DESCRIPTOR;
+  }
+  return ASPD_OK;
+}
+
+struct Region { int lo, hi; };
+
+// Regions inside the page table, page alignment, overlap, page ids.
+int check_layout(const aspd_shape_t* s, const aspd_request_t* req, const aspd_branch_t* br, const int32_t* page_ids,
+                 int n_req, int64_t n_pool_pages, int mode) {
+  if (n_req > 0 && !page_ids) return ASPD_ERR_INVALID_ARG;
+  if (n_pool_pages < 0) return ASPD_ERR_INVALID_ARG;
+  std::vector<uint8_t> used((size_t)n_pool_pages, 0);
+  std::vector<Region> regs;
+  for (int r = 0; r < n_req; ++r) {
+    const aspd_request_t& q = req[r];
+    if (q.page_begin < 0 || q.n_pages < 0) return ASPD_ERR_BAD_DESCRIPTOR;
+    const long cap = (long)q.n_pages * s->page_size;
+    regs.clear();
+    regs.push_back({0, q.prefix_len});
+    for (int b = 0; b < q.n_branches; ++b) {
+      const aspd_branch_t& x = br[q.branch_begin + b];
+      if (x.kv_off % s->page_size) return ASPD_ERR_BAD_DESCRIPTOR;
+      regs.push_back({x.kv_off, x.kv_off + x.kv_len});
+    }
+    if (mode == ASPD_MODE_SERIAL || q.tail_len > 0) {
+      if (q.tail_off % s->page_size) return ASPD_ERR_BAD_DESCRIPTOR;
+      regs.push_back({q.tail_off, q.tail_off + q.tail_len});
+    }
+    for (const Region& g : regs)
+      if (g.hi > cap) return ASPD_ERR_BAD_DESCRIPTOR;
+    std::vector<Region> sorted;
+    for (const Region& g : regs)
+      if (g.hi > g.lo) sorted.push_back(g);
+    std::sort(sorted.begin(), sorted.end(), [](const Region& a, const Region& b) { return a.lo < b.lo; });
+    for (size_t i = 1; i < sorted.size(); ++i)
+      if (sorted[i].lo < sorted[i - 1].hi) return ASPD_ERR_BAD_DESCRIPTOR;
+    for (int p = 0; p < q.n_pages; ++p) {
+      int32_t id = page_ids[q.page_begin + p];
+      if (id < 0 || id >= n_pool_pages) return ASPD_ERR_BAD_DESCRIPTOR;
+      if (used[id]) return ASPD_ERR_BAD_DESCRIPTOR;
+      used[id] = 1;
+    }
+  }
+  return ASPD_OK;
+}
+
+struct Segment { int key0, n_keys, causal0, tok0, n_tok, slot0; };
+
+}  // namespace
+
+extern "C" {
+
+const char* aspd_strerror(int status) {
+  switch (status) {
+    case ASPD_OK: return "ok";
+    case ASPD_ERR_INVALID_ARG: return "invalid argument";
+    case ASPD_ERR_BAD_DESCRIPTOR: return "bad descriptor (overlap, out-of-table slot, alignment, q_len > kv_len or page id)";
+    case ASPD_ERR_UNSUPPORTED: return "unsupported shape (head_dim, page_size or dtype)";
+    case ASPD_ERR_CUDA: return "CUDA runtime or launch error";
+    case ASPD_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case ASPD_ERR_NOMEM: return "out of memory";
+    case ASPD_ERR_TOO_LARGE: return "size exceeds a stated maximum";
+    default: return "unknown status";
+  }
+}
+
+size_t aspd_pool_bytes(const aspd_shape_t* shape, int64_t n_pages) {
+  if (check_shape(shape) != ASPD_OK || n_pages < 0) return 0;
+  return (size_t)n_pages * shape->n_kv_heads * tile_bytes(shape->page_size, shape->head_dim, esize_of(shape->dtype));
+}
+
+int aspd_count_new_tokens(const aspd_request_t* req, const aspd_branch_t* br, int n_req, int mode) {
+  int rc = check_counts(req, br, n_req, mode);
+  if (rc != ASPD_OK) return rc;
+  long n = 0;
+  for (int r = 0; r < n_req; ++r) {
+    if (mode == ASPD_MODE_SERIAL) { ++n; continue; }
+    for (int b = 0; b < req[r].n_branches; ++b) n += br[req[r].branch_begin + b].q_len;
+  }
+  if (n > (1 << 24)) return ASPD_ERR_TOO_LARGE;
+  return (int)n;
+}
+
+int aspd_positions(const aspd_request_t* req, const aspd_branch_t* br, int n_req, int mode, int32_t* pos_out,
+                   int32_t* slot_out, int32_t* req_out) {
+  int n = aspd_count_new_tokens(req, br, n_req, mode);
+  if (n < 0) return n;
+  if (n > 0 && (!pos_out || !slot_out)) return ASPD_ERR_INVALID_ARG;
+  int t = 0;
+  for (int r = 0; r < n_req; ++r) {
+    const aspd_request_t& q = req[r];
+    if (mode == ASPD_MODE_BRANCH) {
+      for (int b = 0; b < q.n_branches; ++b) {
+        const aspd_branch_t& x = br[q.branch_begin + b];
+        for (int i = 0; i < x.q_len; ++i, ++t) {
+          int k = x.kv_len - x.q_len + i;        // index of the token inside its branch
+          pos_out[t] = x.pos_start + k;          // Eq. 4: stage_start + delta
+          slot_out[t] = x.kv_off + k;
+          if (req_out) req_out[t] = r;
+        }
+      }
+    } else {
+      long total = q.prefix_len;                  // Eq. 4, main branch: every cached token counts
+      for (int b = 0; b < q.n_branches; ++b) total += br[q.branch_begin + b].kv_len;
+      pos_out[t] = (int32_t)(total + q.tail_len - 1);
+      slot_out[t] = q.tail_off + q.tail_len - 1;
+      if (req_out) req_out[t] = r;
+      ++t;
+    }
+  }
+  return ASPD_OK;
+}
+
+int aspd_visible_slots(const aspd_request_t* req, const aspd_branch_t* br, int n_req, int mode, int n_slots,
+                       uint8_t* vis_out) {
+  int n = aspd_count_new_tokens(req, br, n_req, mode);
+  if (n < 0) return n;
+  if (!vis_out || n_slots < 0) return ASPD_ERR_INVALID_ARG;
+  memset(vis_out, 0, (size_t)n * n_slots);
+  int t = 0;
+  auto mark = [&](int tok, int lo, int hi) -> int {
+    if (hi > n_slots) return ASPD_ERR_INVALID_ARG;
+    for (int s = lo; s < hi; ++s) vis_out[(size_t)tok * n_slots + s] = 1;
+    return ASPD_OK;
+  };
+  for (int r = 0; r < n_req; ++r) {
+    const aspd_request_t& q = req[r];
+    if (mode == ASPD_MODE_BRANCH) {
+      for (int b = 0; b < q.n_branches; ++b) {
+        const aspd_branch_t& x = br[q.branch_begin + b];
+        for (int i = 0; i < x.q_len; ++i, ++t) {
+          if (mark(t, 0, q.prefix_len)) return ASPD_ERR_INVALID_ARG;
+          if (mark(t, x.kv_off, x.kv_off + x.kv_len - x.q_len + i + 1)) return ASPD_ERR_INVALID_ARG;
+        }
+      }
+    } else {
+      if (mark(t, 0, q.prefix_len)) return ASPD_ERR_INVALID_ARG;
+      for (int b = 0; b < q.n_branches; ++b) {
+        const aspd_branch_t& x = br[q.branch_begin + b];
+        if (mark(t, x.kv_off, x.kv_off + x.kv_len)) return ASPD_ERR_INVALID_ARG;
+      }
+      if (mark(t, q.tail_off, q.tail_off + q.tail_len)) return ASPD_ERR_INVALID_ARG;
+      ++t;
+    }
+  }
+  return ASPD_OK;
+}
+
+int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const aspd_branch_t* br,
+                     const int32_t* page_ids, int n_req, int64_t n_pool_pages, int mode, const int32_t* q_pos,
+                     const aspd_tuning_t* tuning, void* stream, aspd_plan_t** plan_out) {
+  if (!plan_out) return ASPD_ERR_INVALID_ARG;
+  *plan_out = nullptr;
+  int rc = check_shape(shape);
+  if (rc) return rc;
+  rc = check_counts(req, br, n_req, mode);
+  if (rc) return rc;
+  rc = check_layout(shape, req, br, page_ids, n_req, n_pool_pages, mode);
+  if (rc) return rc;
+  const int n_new = aspd_count_new_tokens(req, br, n_req, mode);
+  if (n_new < 0) return n_new;
+
+  aspd_tuning_t tune = {ASPD_KERNEL_AUTO, 0, 0, 0};
+  if (tuning) tune = *tuning;
+  const int ps = shape->page_size, d = shape->head_dim, Hq = shape->n_q_heads, Hkv = shape->n_kv_heads;
+  const int G = Hq / Hkv, es = esize_of(shape->dtype);
+  if (tune.chunk_tokens < 0 || tune.chunk_tokens % ps || tune.n_ctas < 0) return ASPD_ERR_INVALID_ARG;
+  const bool mma_ok = shape->dtype == ASPD_DTYPE_BF16 && d == 128 && ps == 16;
+  int kernel = tune.kernel;
+  if (kernel == ASPD_KERNEL_AUTO) kernel = mma_ok ? ASPD_KERNEL_MMA : ASPD_KERNEL_GENERIC;
+  if (kernel == ASPD_KERNEL_MMA && !mma_ok) return ASPD_ERR_UNSUPPORTED;
+  if (kernel != ASPD_KERNEL_MMA && kernel != ASPD_KERNEL_GENERIC) return ASPD_ERR_INVALID_ARG;
+
+  aspd_plan* p = new (std::nothrow) aspd_plan();
+  if (!p) return ASPD_ERR_NOMEM;
+  p->shape = *shape; p->mode = mode; p->n_req = n_req; p->n_new = n_new; p->kernel = kernel;
+  p->host_only = tune.host_only; p->n_pool_pages = n_pool_pages; p->device_base = nullptr; p->device_bytes = 0;
+  memset(&p->dev, 0, sizeof(p->dev));
+  p->sm_count = 148;
+  if (!tune.host_only) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+      delete p; return ASPD_ERR_CUDA;
+    }
+    p->sm_count = sms;
+  }
+
+  // ---- new-token table --------------------------------------------------------------
+  std::vector<int32_t> pos(n_new), slot(n_new), treq(n_new), tok_page(n_new), tok_row(n_new);
+  rc = aspd_positions(req, br, n_req, mode, pos.data(), slot.data(), treq.data());
+  if (rc) { delete p; return rc; }
+  for (int t = 0; t < n_new; ++t) {
+    tok_page[t] = page_ids[req[treq[t]].page_begin + slot[t] / ps];
+    tok_row[t] = slot[t] % ps;
+    if (q_pos) { if (q_pos[t] < 0) { delete p; return ASPD_ERR_INVALID_ARG; } pos[t] = q_pos[t]; }
+  }
+
+  // ---- segments: (key range, rows that see it, causal rule) ---------------------------
+  const int max_tok = std::max(1, kMaxRowsPerItem / G);
+  std::vector<std::vector<Segment>> segs(n_req);
+  std::vector<int> req_tok0(n_req + 1, 0);
+  long total_cost = 0;
+  int64_t kv_tokens = 0;
+  {
+    int t = 0;
+    for (int r = 0; r < n_req; ++r) {
+      const aspd_request_t& q = req[r];
+      req_tok0[r] = t;
+      if (mode == ASPD_MODE_BRANCH) {
+        int nq = 0;
+        for (int b = 0; b < q.n_branches; ++b) nq += br[q.branch_begin + b].q_len;
+        if (nq > 0 && q.prefix_len > 0) segs[r].push_back({0, q.prefix_len, kCausalAll, t, nq, 0});
+        if (nq > 0) kv_tokens += q.prefix_len;
+        for (int b = 0; b < q.n_branches; ++b) {
+          const aspd_branch_t& x = br[q.branch_begin + b];
+          if (x.q_len > 0) {
+            segs[r].push_back({x.kv_off, x.kv_len, x.kv_len - x.q_len, t, x.q_len, 0});
+            kv_tokens += x.kv_len;
+          }
+          t += x.q_len;
+        }
+      } else {
+        if (q.prefix_len > 0) segs[r].push_back({0, q.prefix_len, kCausalAll, t, 1, 0});
+        kv_tokens += q.prefix_len;
+        for (int b = 0; b < q.n_branches; ++b) {
+          const aspd_branch_t& x = br[q.branch_begin + b];
+          if (x.kv_len > 0) segs[r].push_back({x.kv_off, x.kv_len, kCausalAll, t, 1, 0});
+          kv_tokens += x.kv_len;
+        }
+        segs[r].push_back({q.tail_off, q.tail_len, kCausalAll, t, 1, 0});
+        kv_tokens += q.tail_len;
+        t += 1;
+      }
+      for (const Segment& s : segs[r]) total_cost += (long)ceil_div(s.n_keys, ps) * ceil_div(s.n_tok, max_tok) * Hkv;
+    }
+    req_tok0[n_req] = t;
+  }
+
+  // ---- chunk size: about four items per CTA of the persistent grid --------------------
+  int n_ctas = tune.n_ctas > 0 ? tune.n_ctas : p->sm_count;
+  int chunk = tune.chunk_tokens;
+  if (chunk == 0) {
+    long target_items = (long)n_ctas * 4;
+    long pages = std::max(1L, (total_cost + target_items - 1) / target_items);
+    pages = std::min(std::max(pages, 8L), 256L);
+    chunk = (int)pages * ps;
+  }
+  p->chunk_tokens = chunk; p->n_ctas = n_ctas;
+
+  // ---- items and partial slots --------------------------------------------------------
+  std::vector<int32_t> n_parts(n_new, 0), part_base(n_new + 1, 0);
+  for (int r = 0; r < n_req; ++r) {
+    for (Segment& s : segs[r]) {
+      // equal-sized chunks (whole pages) instead of full chunks plus a sliver
+      const int per = ceil_div(ceil_div(s.n_keys, ceil_div(s.n_keys, chunk)), ps) * ps;
+      const int n_chunks = ceil_div(s.n_keys, per);
+      // every token of the segment gets n_chunks consecutive partial slots
+      int slot0 = n_parts[s.tok0];
+      for (int i = 0; i < s.n_tok; ++i) n_parts[s.tok0 + i] += n_chunks;
+      s.slot0 = slot0;
+      for (int c = 0; c < n_chunks; ++c) {
+        const int k0 = c * per, nk = std::min(per, s.n_keys - k0);
+        for (int i0 = 0; i0 < s.n_tok; i0 += max_tok) {
+          const int nt = std::min(max_tok, s.n_tok - i0);
+          for (int h = 0; h < Hkv; ++h) {
+            DeviceItem it;
+            it.q_tok0 = s.tok0 + i0; it.n_q_tok = nt; it.kv_head = h;
+            it.page0 = req[r].page_begin + (s.key0 + k0) / ps;
+            it.n_keys = nk;
+            it.causal0 = s.causal0 == kCausalAll ? kCausalAll : s.causal0 - k0 + i0;
+            it.part_slot = slot0 + c; it.request = r;
+            p->items.push_back(it);
+          }
+        }
+      }
+    }
+  }
+  // In branch mode the prefix segment comes first for every token of a request, so its
+  // slots [0, n_chunks) coincide for all of them; branch segments follow per branch.
+  for (int t = 0; t < n_new; ++t) part_base[t + 1] = part_base[t] + n_parts[t];
+  std::stable_sort(p->items.begin(), p->items.end(), [](const DeviceItem& a, const DeviceItem& b) {
+    return (long)a.n_keys * (a.n_q_tok > 2 ? 2 : 1) > (long)b.n_keys * (b.n_q_tok > 2 ? 2 : 1);
+  });
+  p->n_items = (int)p->items.size();
+  p->n_partials = part_base[n_new];
+  p->kv_tokens_read = kv_tokens;
+  p->algorithmic_bytes = 2LL * Hkv * d * es * kv_tokens + 2LL * es * Hq * d * n_new + 2LL * Hkv * d * es * n_new;
+  if (tune.host_only) { *plan_out = p; return ASPD_OK; }
+
+  // ---- one device allocation, one staging blob ------------------------------------------
+  int total_pages = 0;
+  for (int r = 0; r < n_req; ++r) total_pages = std::max(total_pages, req[r].page_begin + req[r].n_pages);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t o_items = take(sizeof(DeviceItem) * std::max(1, p->n_items));
+  const size_t o_pages = take(sizeof(int32_t) * std::max(1, total_pages));
+  const size_t o_tpage = take(sizeof(int32_t) * std::max(1, n_new));
+  const size_t o_trow = take(sizeof(int32_t) * std::max(1, n_new));
+  const size_t o_qcs = take(sizeof(float2) * std::max(1, n_new) * (d / 2));
+  const size_t o_pbase = take(sizeof(int32_t) * (n_new + 1));
+  const size_t o_freq = take(sizeof(double) * (d / 2));
+  const size_t o_status = take(sizeof(int32_t) * 2);
+  const size_t upload_bytes = off;
+  const size_t o_wso = take(sizeof(float) * (size_t)std::max(1, p->n_partials) * Hq * d);
+  const size_t o_wsml = take(sizeof(float2) * (size_t)std::max(1, p->n_partials) * Hq);
+  const size_t o_stq = take((size_t)es * std::max(1, n_new) * Hq * d);
+  const size_t o_stk = take((size_t)es * std::max(1, n_new) * Hkv * d);
+  const size_t o_stv = take((size_t)es * std::max(1, n_new) * Hkv * d);
+  const size_t o_sto = take((size_t)es * std::max(1, n_new) * Hq * d);
+  const size_t o_stp = take(sizeof(int32_t) * std::max(1, n_new));
+  p->device_bytes = off;
+
+  std::vector<uint8_t> blob(upload_bytes, 0);
+  if (p->n_items) memcpy(blob.data() + o_items, p->items.data(), sizeof(DeviceItem) * p->n_items);
+  if (total_pages) memcpy(blob.data() + o_pages, page_ids, sizeof(int32_t) * total_pages);
+  if (n_new) {
+    memcpy(blob.data() + o_tpage, tok_page.data(), sizeof(int32_t) * n_new);
+    memcpy(blob.data() + o_trow, tok_row.data(), sizeof(int32_t) * n_new);
+  }
+  memcpy(blob.data() + o_pbase, part_base.data(), sizeof(int32_t) * (n_new + 1));
+  double* freq = reinterpret_cast<double*>(blob.data() + o_freq);
+  for (int i = 0; i < d / 2; ++i) freq[i] = pow((double)shape->rope_theta, -2.0 * i / d);
+  float2* qcs = reinterpret_cast<float2*>(blob.data() + o_qcs);
+  for (int t = 0; t < n_new; ++t)
+    for (int i = 0; i < d / 2; ++i) {
+      double a = (double)pos[t] * freq[i];
+      qcs[(size_t)t * (d / 2) + i] = make_float2((float)cos(a), (float)sin(a));
+    }
+
+  cudaStream_t s = (cudaStream_t)stream;
+  void* base = nullptr;
+  if (cudaMalloc(&base, p->device_bytes) != cudaSuccess) { delete p; return ASPD_ERR_NOMEM; }
+  if (cudaMemcpyAsync(base, blob.data(), upload_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+    cudaFree(base); delete p; return ASPD_ERR_CUDA;
+  }
+  // the blob is pageable: the copy above has been staged by the time the call returns
+  uint8_t* b8 = (uint8_t*)base;
+  p->device_base = base;
+  p->dev.items = (const DeviceItem*)(b8 + o_items);
+  p->dev.page_ids = (const int32_t*)(b8 + o_pages);
+  p->dev.tok_page = (const int32_t*)(b8 + o_tpage);
+  p->dev.tok_row = (const int32_t*)(b8 + o_trow);
+  p->dev.q_cs = (const float2*)(b8 + o_qcs);
+  p->dev.part_base = (const int32_t*)(b8 + o_pbase);
+  p->dev.inv_freq = (const double*)(b8 + o_freq);
+  p->dev.status = (int32_t*)(b8 + o_status);
+  p->dev.work_counter = p->dev.status + 1;
+  p->dev.ws_o = (float*)(b8 + o_wso);
+  p->dev.ws_ml = (float2*)(b8 + o_wsml);
+  p->dev.st_q = b8 + o_stq; p->dev.st_k = b8 + o_stk; p->dev.st_v = b8 + o_stv; p->dev.st_out = b8 + o_sto;
+  p->dev.st_pos = (int32_t*)(b8 + o_stp);
+  *plan_out = p;
+  return ASPD_OK;
+}
+
+int aspd_plan_destroy(aspd_plan_t* plan) {
+  if (!plan) return ASPD_OK;
+  int rc = ASPD_OK;
+  if (plan->device_base && cudaFree(plan->device_base) != cudaSuccess) rc = ASPD_ERR_CUDA;
+  delete plan;
+  return rc;
+}
+
+int aspd_plan_info(const aspd_plan_t* p, aspd_plan_info_t* info) {
+  if (!p || !info) return ASPD_ERR_INVALID_ARG;
+  info->n_new = p->n_new; info->n_items = p->n_items; info->n_partials = p->n_partials; info->kernel = p->kernel;
+  info->chunk_tokens = p->chunk_tokens; info->n_ctas = p->n_ctas; info->workspace_bytes = (int64_t)p->device_bytes;
+  info->kv_tokens_read = p->kv_tokens_read; info->algorithmic_bytes = p->algorithmic_bytes;
+  return ASPD_OK;
+}
+
+int aspd_plan_items(const aspd_plan_t* p, aspd_item_t* items, int max_items) {
+  if (!p || (max_items > 0 && !items) || max_items < 0) return ASPD_ERR_INVALID_ARG;
+  int n = std::min(max_items, p->n_items);
+  static_assert(sizeof(aspd_item_t) == sizeof(DeviceItem), "item layouts must match");
+  if (n) memcpy(items, p->items.data(), sizeof(DeviceItem) * n);
+  return p->n_items;
+}
+
+int aspd_plan_status(aspd_plan_t* p, void* stream) {
+  if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
+  int32_t st = 0;
+  if (cudaMemcpyAsync(&st, p->dev.status, sizeof(st), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess)
+    return ASPD_ERR_CUDA;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return ASPD_ERR_CUDA;
+  return st;
+}
+
+int aspd_kv_append(aspd_plan_t* p, const void* k_new, const void* v_new, const int32_t* pos, void* k_pool,
+                   void* v_pool, void* stream) {
+  if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
+  if (p->n_new == 0) return ASPD_OK;
+  if (!k_new || !v_new || !pos || !k_pool || !v_pool) return ASPD_ERR_INVALID_ARG;
+  return launch_append(p, k_new, v_new, pos, k_pool, v_pool, (cudaStream_t)stream);
+}
+
+int aspd_attn_partials(aspd_plan_t* p, const void* q, const void* k_pool, const void* v_pool, void* stream) {
+  if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
+  if (p->n_new == 0) return ASPD_OK;
+  if (!q || !k_pool || !v_pool) return ASPD_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  return p->kernel == ASPD_KERNEL_MMA ? launch_attn_mma(p, q, k_pool, v_pool, s)
+                                      : launch_attn_generic(p, q, k_pool, v_pool, s);
+}
+
+int aspd_attn_combine(aspd_plan_t* p, void* out, void* stream) {
+  if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
+  if (p->n_new == 0) return ASPD_OK;
+  if (!out) return ASPD_ERR_INVALID_ARG;
+  return launch_combine(p, out, (cudaStream_t)stream);
+}
+
+static int run_attn(aspd_plan_t* p, int mode, const void* q, const void* k_pool, const void* v_pool, void* out,
+                    void* stream) {
+  if (!p || p->host_only || p->mode != mode) return ASPD_ERR_INVALID_ARG;
+  if (p->n_new == 0) return ASPD_OK;
+  if (!q || !k_pool || !v_pool || !out) return ASPD_ERR_INVALID_ARG;
+  int rc = aspd_attn_partials(p, q, k_pool, v_pool, stream);
+  if (rc) return rc;
+  return aspd_attn_combine(p, out, stream);
+}
+
+int aspd_branch_attn(aspd_plan_t* p, const void* q, const void* k_pool, const void* v_pool, void* out, void* stream) {
+  return run_attn(p, ASPD_MODE_BRANCH, q, k_pool, v_pool, out, stream);
+}
+
+int aspd_serial_attn(aspd_plan_t* p, const void* q, const void* k_pool, const void* v_pool, void* out, void* stream) {
+  return run_attn(p, ASPD_MODE_SERIAL, q, k_pool, v_pool, out, stream);
+}
+
+int aspd_step_host(aspd_plan_t* p, const void* q, const void* k_new, const void* v_new, const int32_t* pos,
+                   void* k_pool, void* v_pool, void* out, void* stream) {
+  if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
+  if (p->n_new == 0) return ASPD_OK;
+  if (!q || !k_new || !v_new || !pos || !k_pool || !v_pool || !out) return ASPD_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  const aspd_shape_t& sh = p->shape;
+  const size_t es = esize_of(sh.dtype);
+  const size_t qb = es * p->n_new * sh.n_q_heads * sh.head_dim, kb = es * p->n_new * sh.n_kv_heads * sh.head_dim;
+  if (cudaMemcpyAsync(p->dev.st_q, q, qb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(p->dev.st_k, k_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(p->dev.st_v, v_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(p->dev.st_pos, pos, sizeof(int32_t) * p->n_new, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return ASPD_ERR_CUDA;
+  int rc = launch_append(p, p->dev.st_k, p->dev.st_v, p->dev.st_pos, k_pool, v_pool, s);
+  if (rc) return rc;
+  rc = run_attn(p, p->mode, p->dev.st_q, k_pool, v_pool, p->dev.st_out, stream);
+  if (rc) return rc;
+  if (cudaMemcpyAsync(out, p->dev.st_out, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return ASPD_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return ASPD_ERR_CUDA;
+  return ASPD_OK;
+}
+
+int aspd_debug_read_token(const aspd_shape_t* shape, const void* pool, int64_t page, int row, int kv_head, float* out,
+                          void* stream) {
+  int rc = check_shape(shape);
+  if (rc) return rc;
+  if (!pool || !out || page < 0 || row < 0 || row >= shape->page_size || kv_head < 0 || kv_head >= shape->n_kv_heads)
+    return ASPD_ERR_INVALID_ARG;
+  float* tmp = nullptr;
+  if (cudaMalloc(&tmp, sizeof(float) * shape->head_dim) != cudaSuccess) return ASPD_ERR_NOMEM;
+  cudaStream_t s = (cudaStream_t)stream;
+  rc = launch_read_token(shape, pool, page, row, kv_head, tmp, s);
+  if (rc == ASPD_OK && (cudaMemcpyAsync(out, tmp, sizeof(float) * shape->head_dim, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+                        cudaStreamSynchronize(s) != cudaSuccess))
+    rc = ASPD_ERR_CUDA;
+  cudaFree(tmp);
+  return rc;
+}
+
+}  // extern "C"

@@ -1,0 +1,93 @@
+"""Glue that drives workload phases through the C ABI on one GPU (marshalling only).
+
+Used by the GPU tests, the smoke check and the benchmark.  torch provides device memory and
+streams; every computation happens inside the CUDA library.
+"""
+from __future__ import annotations
+
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import workloads as W
+
+
+def to_device(x32: np.ndarray, dtype: str, device="cuda") -> torch.Tensor:
+    """float32 numpy values (already storage-rounded) -> device tensor of the storage dtype."""
+    if dtype == "bf16":
+        bits = W.bf16_bits(x32).view(np.int16)
+        return torch.from_numpy(bits).to(device).view(torch.bfloat16)
+    return torch.from_numpy(np.ascontiguousarray(x32, dtype=np.float32)).to(device)
+
+
+def to_host_f32(t: torch.Tensor) -> np.ndarray:
+    return t.detach().float().cpu().numpy()
+
+
+def torch_dtype(dtype: str):
+    return torch.bfloat16 if dtype == "bf16" else torch.float32
+
+
+class LayerCache:
+    """K and V pools of one attention layer (opaque tile format, see ``aspd.h``)."""
+
+    def __init__(self, shape: B.Shape, n_pool_pages: int, device="cuda"):
+        nbytes = B.pool_bytes(shape, n_pool_pages)
+        if nbytes == 0 and n_pool_pages > 0:
+            raise B.AspdError(-3, "aspd_pool_bytes")
+        self.k = torch.zeros(max(nbytes, 16), dtype=torch.uint8, device=device)
+        self.v = torch.zeros(max(nbytes, 16), dtype=torch.uint8, device=device)
+
+
+class WorkloadRun:
+    """Runs the phases of a workload through kv_append + attention, keeping compared outputs."""
+
+    def __init__(self, wl: W.Workload, kernel: int = B.KERNEL_AUTO, chunk_tokens: int = 0, n_ctas: int = 0,
+                 device="cuda"):
+        self.wl, self.kernel, self.chunk_tokens, self.n_ctas, self.device = wl, kernel, chunk_tokens, n_ctas, device
+        self.shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
+        self.cache = LayerCache(self.shape, wl.n_pool_pages, device)
+        self.outputs: List[np.ndarray] = []
+        self.positions = []
+        self.plans = []
+
+    def step(self, ph: W.Phase, attend: bool = True, keep_plan: bool = False) -> Optional[np.ndarray]:
+        wl = self.wl
+        plan = B.Plan(self.shape, ph.desc, wl.n_pool_pages, ph.mode, kernel=self.kernel,
+                      chunk_tokens=self.chunk_tokens, n_ctas=self.n_ctas)
+        pos, slot, req = B.positions(ph.desc, ph.mode)
+        self.positions.append((pos, slot, req))
+        out = None
+        if plan.n_new > 0:
+            pos_d = torch.from_numpy(pos.copy()).to(self.device)
+            k_d, v_d = to_device(ph.k_new, wl.dtype, self.device), to_device(ph.v_new, wl.dtype, self.device)
+            B.kv_append(plan, k_d, v_d, pos_d, self.cache.k, self.cache.v)
+            if attend and ph.q is not None:
+                q_d = to_device(ph.q, wl.dtype, self.device)
+                out_d = torch.empty_like(q_d)
+                (B.branch_attn if ph.mode == W.MODE_BRANCH else B.serial_attn)(plan, q_d, self.cache.k, self.cache.v, out_d)
+                torch.cuda.synchronize()
+                st = plan.status()
+                if st != 0:
+                    raise B.AspdError(st, "device status")
+                out = to_host_f32(out_d)
+                if ph.compare:
+                    self.outputs.append(out)
+        if keep_plan:
+            self.plans.append(plan)
+        else:
+            torch.cuda.synchronize()
+            plan.destroy()
+        return out
+
+    def read_token(self, pool: str, page: int, row: int, head: int) -> np.ndarray:
+        return B.debug_read_token(self.shape, self.cache.k if pool == "k" else self.cache.v, page, row, head)
+
+
+def run_workload(wl: W.Workload, **kw) -> WorkloadRun:
+    run = WorkloadRun(wl, **kw)
+    for ph in wl.phases:
+        run.step(ph)
+    return run

