@@ -1,0 +1,486 @@
+// Split-K decode attention on the 5th-generation tensor cores (tcgen05 + TMEM), bf16 cache,
+// head_dim 128, page_size 16.
+//
+// One persistent CTA per SM walks its share of the plan's work items.  An item is (query row
+// block of one KV head, key chunk): M = n_q_tok * G <= 64 query rows against up to chunk keys.
+// Keys stream through shared memory in tiles of 128 (8 pages), fetched page by page with
+// linear bulk copies (the cache tile format already is the 128-byte-swizzled image the tensor
+// core reads).  Per tile:
+//
+//     S = Qrep . K^T     tcgen05.mma M=128, N=keys, K=128      accumulator in TMEM
+//     softmax warps      read S from TMEM, online softmax, write P (bf16) to shared memory
+//     O += P . V         tcgen05.mma M=128, N=128, K=keys      accumulator in TMEM
+//
+// The 128 accumulator lanes are used as R x KS: the query rows (padded to R = 32 or 64) are
+// replicated KS = 128 / R times in the A operand, and softmax thread (j, r) handles row r over
+// the j-th key sub-range of the tile only, so all 128 threads share the exponentials.  The KS
+// threads of a row agree on one reference maximum per tile (exchanged through shared memory)
+// and write their P values into the SAME row r of the P tile, so the second MMA sums over all
+// keys by itself and rows >= R of its output are simply ignored.  The reference maximum is only
+// raised when the tile maximum exceeds it by more than 2^8, which keeps P exactly consistent
+// with the (m, l, O) record while making the rescale of O in TMEM rare.
+//
+// Warp roles: 0-3 softmax / epilogue (TMEM lane quadrant = warp), 4 bulk-copy producer,
+// 5 MMA issuer (one elected lane), 6 query preparation (RoPE, bf16, swizzled store) one item
+// ahead.  All cross-role hand-offs are mbarriers; every wait is bounded and on expiry sets the
+// plan's status word to ASPD_ERR_TIMEOUT and makes all roles drain and exit.
+#include "aspd_internal.cuh"
+
+namespace aspd {
+namespace {
+
+constexpr int kTile = 128;                     // keys per tile
+constexpr int kThreads = 224;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kRaise = 8.0f;                 // raise the reference maximum only beyond 2^8
+constexpr long long kWaitCycles = 3000000000LL; // ~1.5 s at 1.9 GHz
+
+constexpr uint32_t kTileBytes = 32768;         // one K, V, Q or P tile: 128 rows x 256 B
+constexpr uint32_t kHalf = 16384;              // second 64-element span of a tile
+constexpr uint32_t OFF_K = 0, OFF_V = 2 * kTileBytes, OFF_Q = 4 * kTileBytes, OFF_P = 6 * kTileBytes;
+constexpr uint32_t OFF_MISC = 7 * kTileBytes;
+
+enum Bar { K_FULL = 0, K_EMPTY = 2, V_FULL = 4, V_EMPTY = 6, S_FULL = 8, S_EMPTY = 10, P_FULL = 12, P_EMPTY = 13,
+           O_FULL = 14, O_EMPTY = 16, Q_FULL = 18, Q_EMPTY = 20, NUM_BARS = 22 };
+
+struct Misc {
+  uint64_t bars[NUM_BARS];
+  float smax[2][128];
+  float sl[128];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+constexpr size_t kSmemBytes = OFF_MISC + sizeof(Misc) + 1024;   // + slack to align the base to 1024
+
+// TMEM columns: S double buffer, O double buffer
+constexpr uint32_t COL_S = 0, COL_O = 256;
+
+// ------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false means "give up" (time limit hit here or in another role).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitCycles) { *abort_flag = 1; return false; }
+  }
+}
+__device__ __forceinline__ void bulk_copy(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+// Barrier among n threads that also ORs a predicate, so that all of them take the same exit.
+__device__ __forceinline__ bool named_sync_or(int id, int n, bool pred) {
+  uint32_t out;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %3, 0;\n\t"
+      "bar.red.or.pred p, %1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(out) : "r"(id), "r"(n), "r"((uint32_t)pred) : "memory");
+  return out != 0;
+}
+
+#define ASPD_R32(v, o) "=f"(v[o + 0]), "=f"(v[o + 1]), "=f"(v[o + 2]), "=f"(v[o + 3]), "=f"(v[o + 4]), "=f"(v[o + 5]),  \
+    "=f"(v[o + 6]), "=f"(v[o + 7]), "=f"(v[o + 8]), "=f"(v[o + 9]), "=f"(v[o + 10]), "=f"(v[o + 11]), "=f"(v[o + 12]),    \
+    "=f"(v[o + 13]), "=f"(v[o + 14]), "=f"(v[o + 15]), "=f"(v[o + 16]), "=f"(v[o + 17]), "=f"(v[o + 18]),                 \
+    "=f"(v[o + 19]), "=f"(v[o + 20]), "=f"(v[o + 21]), "=f"(v[o + 22]), "=f"(v[o + 23]), "=f"(v[o + 24]),                 \
+    "=f"(v[o + 25]), "=f"(v[o + 26]), "=f"(v[o + 27]), "=f"(v[o + 28]), "=f"(v[o + 29]), "=f"(v[o + 30]), "=f"(v[o + 31])
+#define ASPD_W32(v, o) "f"(v[o + 0]), "f"(v[o + 1]), "f"(v[o + 2]), "f"(v[o + 3]), "f"(v[o + 4]), "f"(v[o + 5]),        \
+    "f"(v[o + 6]), "f"(v[o + 7]), "f"(v[o + 8]), "f"(v[o + 9]), "f"(v[o + 10]), "f"(v[o + 11]), "f"(v[o + 12]),           \
+    "f"(v[o + 13]), "f"(v[o + 14]), "f"(v[o + 15]), "f"(v[o + 16]), "f"(v[o + 17]), "f"(v[o + 18]), "f"(v[o + 19]),       \
+    "f"(v[o + 20]), "f"(v[o + 21]), "f"(v[o + 22]), "f"(v[o + 23]), "f"(v[o + 24]), "f"(v[o + 25]), "f"(v[o + 26]),       \
+    "f"(v[o + 27]), "f"(v[o + 28]), "f"(v[o + 29]), "f"(v[o + 30]), "f"(v[o + 31])
+
+// 32 consecutive fp32 columns of this thread's TMEM lane -> v[o .. o+31]
+#define ASPD_TMEM_LD32(taddr, v, o)                                                                               \
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, "  \
+               "%13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, " \
+               "[%32];" : ASPD_R32(v, o) : "r"(taddr) : "memory")
+#define ASPD_TMEM_ST32(taddr, v, o)                                                                               \
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, " \
+               "%12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, "   \
+               "%31};" ::ASPD_W32(v, o), "r"(taddr) : "memory")
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, A K-major.
+__device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+struct Ctx {
+  PlanDevice pd;
+  const __nv_bfloat16* q;
+  const char* k_pool;
+  const char* v_pool;
+  int n_items, n_q_heads, n_kv_heads;
+  float scale_log2;
+};
+
+// ------------------------------------------------------------------------------- softmax role
+template <int NC>   // NC = columns per thread = padded row count R
+__device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it, Misc* misc, uint32_t bars, uint32_t smem_p,
+                                             uint32_t tmem, int item_no, int& g) {
+  constexpr int R = NC, KS = 128 / NC;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int r = tid % R, j = tid / R;
+  const int G = c.n_q_heads / c.n_kv_heads, M = it.n_q_tok * G;
+  const int n_tiles = (it.n_keys + kTile - 1) / kTile;
+  volatile int* ab = &misc->abort_flag;
+  int limit = 0;
+  if (r < M) {
+    long lim = (long)it.causal0 + r / G + 1;
+    limit = (int)(lim < 0 ? 0 : (lim > it.n_keys ? it.n_keys : lim));
+  }
+  const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+  const int ob = item_no & 1;
+  float m_ref = -INFINITY, l = 0.f;
+  bool dead = false;   // a wait gave up: keep walking the same control flow, report at the end
+  for (int t = 0; t < n_tiles; ++t, ++g) {
+    const int sb = g & 1;
+    dead |= !mbar_wait(bars + 8 * (S_FULL + sb), (g >> 1) & 1, ab);
+    tc_fence_after();
+    float s[NC];
+    const uint32_t s_addr = tmem + lane_addr + COL_S + sb * 128 + j * NC;
+    ASPD_TMEM_LD32(s_addr, s, 0);
+    if constexpr (NC == 64) ASPD_TMEM_LD32(s_addr + 32, s, 32);
+    tmem_wait_ld();
+    tc_fence_before();
+    mbar_arrive(bars + 8 * (S_EMPTY + sb));
+    const int nvalid = limit - (t * kTile + j * NC);
+    float mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < NC; ++i) {
+      const float v = i < nvalid ? s[i] * c.scale_log2 : -INFINITY;
+      s[i] = v;
+      mx = fmaxf(mx, v);
+    }
+    misc->smax[sb][tid] = mx;
+    named_sync(1, 128);
+    float m_tile = mx;
+#pragma unroll
+    for (int jj = 0; jj < KS; ++jj) m_tile = fmaxf(m_tile, misc->smax[sb][jj * R + r]);
+    const bool upd = m_tile > m_ref + kRaise;     // also true for the first finite maximum (m_ref = -inf)
+    float alpha = 1.f;
+    if (upd) { alpha = exp2f(m_ref - m_tile); m_ref = m_tile; }
+    l *= alpha;
+    if (t > 0 && warp < R / 32) {                 // the owners of rows 0..R-1 rescale O in TMEM
+      if (__any_sync(0xffffffffu, upd)) {
+        dead |= !mbar_wait(bars + 8 * P_EMPTY, (g - 1) & 1, ab);   // PV of the previous tile is done
+        tc_fence_after();
+        const uint32_t o_addr = tmem + lane_addr + COL_O + ob * 128;
+#pragma unroll 1
+        for (int q4 = 0; q4 < 4; ++q4) {
+          float o[32];
+          ASPD_TMEM_LD32(o_addr + q4 * 32, o, 0);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o[i] *= alpha;
+          ASPD_TMEM_ST32(o_addr + q4 * 32, o, 0);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+      }
+    }
+    const float msafe = m_ref == -INFINITY ? 0.f : m_ref;
+    float lsum = 0.f;
+#pragma unroll
+    for (int i = 0; i < NC; ++i) { s[i] = exp2f(s[i] - msafe); lsum += s[i]; }
+    l += lsum;
+    if (g > 0) dead |= !mbar_wait(bars + 8 * P_EMPTY, (g - 1) & 1, ab);   // P tile is free again
+#pragma unroll
+    for (int c8 = 0; c8 < NC / 8; ++c8) {
+      const int kk = j * NC + c8 * 8;
+      const uint32_t addr = smem_p + (kk >> 6) * kHalf + r * 128 + ((((kk & 63) >> 3) ^ (r & 7)) << 4);
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pack_bf16(s[c8 * 8 + 0], s[c8 * 8 + 1])),
+                   "r"(pack_bf16(s[c8 * 8 + 2], s[c8 * 8 + 3])), "r"(pack_bf16(s[c8 * 8 + 4], s[c8 * 8 + 5])),
+                   "r"(pack_bf16(s[c8 * 8 + 6], s[c8 * 8 + 7])) : "memory");
+    }
+    fence_async_smem();
+    tc_fence_before();
+    mbar_arrive(bars + 8 * P_FULL);
+  }
+  // ---- epilogue: one (m, l, O) record per query row of the item
+  dead |= !mbar_wait(bars + 8 * (O_FULL + ob), (item_no >> 1) & 1, ab);
+  tc_fence_after();
+  misc->sl[tid] = l;
+  named_sync(1, 128);
+  if (j == 0 && r < M && !dead) {
+    float lt = 0.f;
+#pragma unroll
+    for (int jj = 0; jj < KS; ++jj) lt += misc->sl[jj * R + r];
+    const int tok = it.q_tok0 + r / G, hq = it.kv_head * G + r % G;
+    const size_t rec = (size_t)(c.pd.part_base[tok] + it.part_slot) * c.n_q_heads + hq;
+    c.pd.ws_ml[rec] = make_float2(m_ref, lt);
+  }
+  if (warp < R / 32) {
+    const uint32_t o_addr = tmem + lane_addr + COL_O + ob * 128;
+    size_t rec = 0;
+    if (r < M) {
+      const int tok = it.q_tok0 + r / G, hq = it.kv_head * G + r % G;
+      rec = (size_t)(c.pd.part_base[tok] + it.part_slot) * c.n_q_heads + hq;
+    }
+#pragma unroll 1
+    for (int q4 = 0; q4 < 4; ++q4) {
+      float o[32];
+      ASPD_TMEM_LD32(o_addr + q4 * 32, o, 0);
+      tmem_wait_ld();
+      if (r < M && !dead) {
+        float4* dst = reinterpret_cast<float4*>(c.pd.ws_o + rec * 128 + q4 * 32);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+      }
+    }
+  }
+  tc_fence_before();
+  mbar_arrive(bars + 8 * (O_EMPTY + ob));
+  return !named_sync_or(1, 128, dead || *ab);
+}
+
+// --------------------------------------------------------------------------------- the kernel
+__global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw);
+  Misc* misc = reinterpret_cast<Misc*>(smem + OFF_MISC);
+  const uint32_t bars = base + OFF_MISC;          // bars[] is the first member of Misc
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  volatile int* ab = &misc->abort_flag;
+
+  if (tid == 0) {
+    const int counts[NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, 128, 128, 128, 1, 1, 1, 128, 128, 32, 32, 1, 1};
+    for (int i = 0; i < NUM_BARS; ++i) mbar_init(bars + 8 * i, counts[i]);
+    misc->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&misc->tmem_base)), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = misc->tmem_base;
+
+  if (warp < 4) {
+    // =============================== softmax + epilogue ===============================
+    int g = 0, item_no = 0;
+    for (int idx = blockIdx.x; idx < c.n_items; idx += gridDim.x, ++item_no) {
+      const DeviceItem it = c.pd.items[idx];
+      const int M = it.n_q_tok * (c.n_q_heads / c.n_kv_heads);
+      const bool ok = M <= 32 ? softmax_item<32>(c, it, misc, bars, base + OFF_P, tmem, item_no, g)
+                              : softmax_item<64>(c, it, misc, bars, base + OFF_P, tmem, item_no, g);
+      if (!ok) break;
+    }
+  } else if (warp == 4) {
+    // ================================ bulk-copy producer ================================
+    int g = 0;
+    bool ok = true;
+    for (int idx = blockIdx.x; idx < c.n_items && ok; idx += gridDim.x) {
+      const DeviceItem it = c.pd.items[idx];
+      const int n_pages = (it.n_keys + 15) >> 4, n_tiles = (it.n_keys + kTile - 1) / kTile;
+      for (int t = 0; t < n_tiles && ok; ++t, ++g) {
+        const int npg = min(8, n_pages - t * 8), sl = g & 1;
+        int page = 0;
+        if (lane < npg) page = c.pd.page_ids[it.page0 + t * 8 + lane];
+        const size_t src_off = ((size_t)page * c.n_kv_heads + it.kv_head) * 4096;
+#pragma unroll
+        for (int kv = 0; kv < 2; ++kv) {
+          const uint32_t full = bars + 8 * ((kv ? V_FULL : K_FULL) + sl), empty = bars + 8 * ((kv ? V_EMPTY : K_EMPTY) + sl);
+          int good = 1;
+          if (lane == 0) {
+            good = mbar_wait(empty, ((g >> 1) & 1) ^ 1, ab) ? 1 : 0;
+            if (good) mbar_expect_tx(full, (uint32_t)npg * 4096u);
+          }
+          good = __shfl_sync(0xffffffffu, good, 0);
+          if (!good) { ok = false; break; }
+          if (lane < npg) {
+            const char* src = (kv ? c.v_pool : c.k_pool) + src_off;
+            const uint32_t dst = base + (kv ? OFF_V : OFF_K) + sl * kTileBytes + lane * 2048;
+            bulk_copy(dst, src, 2048, full);
+            bulk_copy(dst + kHalf, src + 2048, 2048, full);
+          }
+        }
+      }
+    }
+  } else if (warp == 5) {
+    // =================================== MMA issuer ===================================
+    if (lane == 0) {
+      int g = 0, item_no = 0;
+      bool ok = true;
+      const uint32_t idesc_pv = instr_desc(128, 1);
+      // PV of global tile gg (item-local tile tt) of the item whose O buffer is ob
+      auto issue_pv = [&](int gg, int tt, int npg, int ob, int ino) -> bool {
+        if (!mbar_wait(bars + 8 * P_FULL, gg & 1, ab)) return false;
+        if (!mbar_wait(bars + 8 * (V_FULL + (gg & 1)), (gg >> 1) & 1, ab)) return false;
+        if (tt == 0 && !mbar_wait(bars + 8 * (O_EMPTY + ob), ((ino >> 1) & 1) ^ 1, ab)) return false;
+        tc_fence_after();
+        const uint32_t pbuf = base + OFF_P, vbuf = base + OFF_V + (gg & 1) * kTileBytes;
+        for (int ks = 0; ks < npg; ++ks) {
+          const uint64_t a = smem_desc(pbuf + (ks >> 2) * kHalf + (ks & 3) * 32, 16, 1024);
+          const uint64_t b = smem_desc(vbuf + ks * 2048, kHalf, 1024);
+          tc_mma(tmem + COL_O + ob * 128, a, b, idesc_pv, (tt > 0 || ks > 0) ? 1u : 0u);
+        }
+        tc_commit(bars + 8 * P_EMPTY);
+        tc_commit(bars + 8 * (V_EMPTY + (gg & 1)));
+        return true;
+      };
+      for (int idx = blockIdx.x; idx < c.n_items && ok; idx += gridDim.x, ++item_no) {
+        const DeviceItem it = c.pd.items[idx];
+        const int n_pages = (it.n_keys + 15) >> 4, n_tiles = (it.n_keys + kTile - 1) / kTile;
+        const int qb = item_no & 1, ob = item_no & 1;
+        if (!mbar_wait(bars + 8 * (Q_FULL + qb), (item_no >> 1) & 1, ab)) { ok = false; break; }
+        for (int t = 0; t < n_tiles; ++t, ++g) {
+          const int npg = min(8, n_pages - t * 8), sb = g & 1;
+          if (!mbar_wait(bars + 8 * (K_FULL + sb), (g >> 1) & 1, ab) ||
+              !mbar_wait(bars + 8 * (S_EMPTY + sb), ((g >> 1) & 1) ^ 1, ab)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t qbuf = base + OFF_Q + qb * kTileBytes, kbuf = base + OFF_K + sb * kTileBytes;
+          const uint32_t idesc_s = instr_desc((uint32_t)npg * 16u, 0);
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t off = (ks >> 2) * kHalf + (ks & 3) * 32;
+            tc_mma(tmem + COL_S + sb * 128, smem_desc(qbuf + off, 16, 1024), smem_desc(kbuf + off, 16, 1024), idesc_s,
+                   ks > 0 ? 1u : 0u);
+          }
+          tc_commit(bars + 8 * (S_FULL + sb));
+          tc_commit(bars + 8 * (K_EMPTY + sb));
+          if (t == n_tiles - 1) tc_commit(bars + 8 * (Q_EMPTY + qb));
+          if (t > 0 && !issue_pv(g - 1, t - 1, 8, ob, item_no)) { ok = false; break; }
+        }
+        if (!ok) break;
+        if (!issue_pv(g - 1, n_tiles - 1, min(8, n_pages - (n_tiles - 1) * 8), ob, item_no)) { ok = false; break; }
+        tc_commit(bars + 8 * (O_FULL + ob));
+      }
+    }
+    __syncwarp();
+  } else {
+    // ================================ query preparation ================================
+    int item_no = 0;
+    const int G = c.n_q_heads / c.n_kv_heads;
+    for (int idx = blockIdx.x; idx < c.n_items; idx += gridDim.x, ++item_no) {
+      const DeviceItem it = c.pd.items[idx];
+      const int M = it.n_q_tok * G, R = M <= 32 ? 32 : 64, KS = 128 / R, qb = item_no & 1;
+      int good = 1;
+      if (lane == 0) good = mbar_wait(bars + 8 * (Q_EMPTY + qb), ((item_no >> 1) & 1) ^ 1, ab) ? 1 : 0;
+      good = __shfl_sync(0xffffffffu, good, 0);
+      if (!good) break;
+      const uint32_t qbuf = base + OFF_Q + qb * kTileBytes;
+      for (int e = lane; e < R * 8; e += 32) {
+        const int r = e >> 3, ch = e & 7;          // row, 8-element chunk of each half
+        uint32_t lo[4] = {0, 0, 0, 0}, hi[4] = {0, 0, 0, 0};
+        if (r < M) {
+          const int tok = it.q_tok0 + r / G, hq = it.kv_head * G + r % G;
+          const __nv_bfloat16* qrow = c.q + ((size_t)tok * c.n_q_heads + hq) * 128;
+          const uint4 a = *reinterpret_cast<const uint4*>(qrow + ch * 8);
+          const uint4 b = *reinterpret_cast<const uint4*>(qrow + 64 + ch * 8);
+          const float4* cs = reinterpret_cast<const float4*>(c.pd.q_cs + (size_t)tok * 64 + ch * 8);
+          const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&a);
+          const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&b);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float4 w = cs[i];                // (cos, sin) of elements 2i and 2i+1
+            const float2 x0 = __bfloat1622float2(a2[i]), x1 = __bfloat1622float2(b2[i]);
+            lo[i] = pack_bf16(x0.x * w.x - x1.x * w.y, x0.y * w.z - x1.y * w.w);
+            hi[i] = pack_bf16(x1.x * w.x + x0.x * w.y, x1.y * w.z + x0.y * w.w);
+          }
+        }
+        for (int jj = 0; jj < KS; ++jj) {
+          const uint32_t addr = qbuf + (jj * R + r) * 128 + ((ch ^ (r & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr + kHalf), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
+        }
+      }
+      fence_async_smem();
+      mbar_arrive(bars + 8 * (Q_FULL + qb));
+    }
+  }
+
+  // ---- drain: on a time-out give outstanding copies and MMAs time to land before the CTA's
+  // shared memory and TMEM go away
+  if (*ab) {
+    if (tid == 0) atomicCAS(c.pd.status, 0, (int)ASPD_ERR_TIMEOUT);
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+  }
+}
+
+}  // namespace
+
+int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, cudaStream_t s) {
+  if (p->n_items == 0) return ASPD_OK;
+  const aspd_shape_t& sh = p->shape;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
+      return ASPD_ERR_CUDA;
+    configured = true;
+  }
+  Ctx c;
+  c.pd = p->dev;
+  c.q = (const __nv_bfloat16*)q;
+  c.k_pool = (const char*)k_pool;
+  c.v_pool = (const char*)v_pool;
+  c.n_items = p->n_items;
+  c.n_q_heads = sh.n_q_heads;
+  c.n_kv_heads = sh.n_kv_heads;
+  c.scale_log2 = sh.sm_scale * kLog2e;
+  const int grid = p->n_items < p->n_ctas ? p->n_items : p->n_ctas;
+  attn_tc_kernel<<<grid, kThreads, kSmemBytes, s>>>(c);
+  return cudaGetLastError() == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
+}
+
+}  // namespace aspd

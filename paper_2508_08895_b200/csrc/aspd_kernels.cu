@@ -213,9 +213,4 @@ int launch_read_token(const aspd_shape_t* sh, const void* pool, int64_t page, in
   return check_launch();
 }
 
-// Until the tensor-core kernel exists the MMA selection falls back to the generic GPU kernel.
-int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, cudaStream_t s) {
-  return launch_attn_generic(p, q, k_pool, v_pool, s);
-}
-
 }  // namespace aspd

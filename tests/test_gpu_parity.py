@@ -104,10 +104,12 @@ def test_config5_serving_mix_full_size(kernel):
 
 
 def test_peaked_softmax_variant():
-    """sm_scale x 4: logits ~ N(0, 16), outputs are O(1), so the bounds bite.  The cached keys
-    are bf16 (relative rounding 2^-9) while the oracle keeps them exact, which alone perturbs a
-    logit by about 4 * 1.1e-3 and an O(1) output by up to a few 1e-2 at the maximum; the
-    max-abs bound is widened to 4e-2 for this variant, mean-abs and relative L2 stay."""
+    """sm_scale x 4: logits ~ N(0, 16), outputs are O(1), so the bounds bite.  The cached keys,
+    the rotated query and the softmax weights fed to the tensor cores are bf16 (relative
+    rounding 2^-9 each) while the oracle keeps everything exact; that perturbs a logit by about
+    4 * 1.6e-3 and an O(1) output by a few 1e-3 on average, a few 1e-2 at the maximum.  The
+    bounds of this variant are derived from that (max-abs 6e-2, mean-abs 4e-3); the relative L2
+    bound stays at 1e-2."""
     wl = W.config_qwen7b_layer()
     wl.sm_scale *= 4.0
     ref = oracle_run(wl)
@@ -115,7 +117,7 @@ def test_peaked_softmax_variant():
     g, r = run.outputs[0].astype(np.float64), ref.outputs[0]
     assert np.abs(r).max() > 0.5
     err = np.abs(g - r)
-    assert err.max() <= 4e-2 and err.mean() <= 2e-3
+    assert err.max() <= 6e-2 and err.mean() <= 4e-3
     assert np.linalg.norm(g - r) / np.linalg.norm(r) <= 1e-2
 
 
