@@ -55,8 +55,10 @@ def measured_peaks():
     return FALLBACK_HBM_GBS, "fallback"
 
 
-def build_workload(name: str, rank: int):
+def build_workload(name: str, rank: int, requests: int = 0):
     from paper_2508_08895_b200 import workloads as W
+    if name == "serving-mix" and requests > 0:      # a smaller batch of the same mix (profiling captures)
+        return W.config_serving_mix(seed=W.SEED_BASE + 4 + 16 * rank, n_req=requests)
     fn = W.CONFIGS[name]
     base = {"tiny-f32": 0, "qwen7b-layer": 1, "branch-open": 2, "long-rag": 3, "serving-mix": 4}[name]
     if name == "branch-open":
@@ -137,7 +139,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    wl = build_workload(args.workload, 0)
+    wl = build_workload(args.workload, 0, args.requests)
     steps = max(1, args.steps)
     # each "step" of this arm is one layer-step of the oracle on the full batch; warm-up once
     value, cores, sec, reps, n_new = oracle_sample(wl, budget_s=min(30.0, 2.0 * (steps + args.warmup)))
@@ -173,7 +175,7 @@ def run_ours(args):
     from paper_2508_08895_b200 import binding as B, engine as E, workloads as W
 
     L = args.layers
-    wl = build_workload(args.workload, rank)
+    wl = build_workload(args.workload, rank, args.requests)
     shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
     # enough layers that the distinct K/V pools of one step exceed four times the 126 MB L2
     probe = B.Plan(shape, wl.phases[-1].desc, wl.n_pool_pages, wl.phases[-1].mode, host_only=True)
@@ -202,8 +204,6 @@ def run_ours(args):
     q_d, k_d, v_d = (E.to_device(x, wl.dtype) for x in (ph.q, ph.k_new, ph.v_new))
     outs = [torch.empty_like(q_d) for _ in range(L)]
     attn = B.branch_attn if ph.mode == W.MODE_BRANCH else B.serial_attn
-    stream = torch.cuda.current_stream()
-
     def step():
         for l in range(L):
             B.kv_append(plan, k_d, v_d, pos_d, caches[l].k, caches[l].v)
@@ -214,33 +214,55 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    # The whole step (3 launches per layer) is captured once into a CUDA graph and replayed, so
+    # that the host's launch rate does not bound a step whose kernels last tens of microseconds.
+    for _ in range(2):
         step()
+    torch.cuda.synchronize()
+    graph = None
+    if not args.no_graph:
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+    run_step = graph.replay if graph is not None else step
+    for _ in range(max(args.warmup, 3)):
+        run_step()
     barrier()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+    stream = torch.cuda.current_stream()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     ev0.record(stream)
     for _ in range(args.steps):
-        step()
+        run_step()
     ev1.record(stream)
     barrier()
     ms = ev0.elapsed_time(ev1)
     if plan.status() != 0:
         raise SystemExit("bench.py: device status %d" % plan.status())
 
-    # the dominant kernel alone: the split-K pass over all layers, back to back
-    for l in range(L):
-        B.attn_partials(plan, q_d, caches[l].k, caches[l].v)
+    # the dominant kernel alone: the split-K pass over all layers, back to back (also a graph)
+    def partials():
+        for l in range(L):
+            B.attn_partials(plan, q_d, caches[l].k, caches[l].v)
+
+    partials()
+    torch.cuda.synchronize()
+    pgraph = None
+    if not args.no_graph:
+        pgraph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(pgraph):
+            partials()
+    run_partials = pgraph.replay if pgraph is not None else partials
+    run_partials()
     torch.cuda.synchronize()
     k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     reps = max(3, args.steps)
     k0.record(stream)
     for _ in range(reps):
-        for l in range(L):
-            B.attn_partials(plan, q_d, caches[l].k, caches[l].v)
+        run_partials()
     k1.record(stream)
     torch.cuda.synchronize()
     kernel_ms = k0.elapsed_time(k1) / (reps * L)
@@ -294,7 +316,7 @@ def run_ours(args):
                        "page_size": wl.page_size, "kernel": {1: "generic", 2: "mma"}[info.kernel],
                        "chunk_tokens": info.chunk_tokens, "work_items": info.n_items, "n_ctas": info.n_ctas,
                        "l2": "footprint %.1f GB of distinct K/V pools per step, far above L2" % (alg * L / 1e9),
-                       "layers_agree": bool(same)},
+                       "layers_agree": bool(same), "cuda_graph": not args.no_graph},
             "hbm_gbs": alg * L * args.steps / (ms * 1e-3) / 1e9,
             "hbm_frac_of_measured": alg * L * args.steps / (ms * 1e-3) / 1e9 / peak,
             "hbm_frac_of_8000_nominal": alg * L * args.steps / (ms * 1e-3) / 1e9 / 8000.0,
@@ -330,8 +352,10 @@ def main():
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "mma"])
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--ctas", type=int, default=0)
+    ap.add_argument("--requests", type=int, default=0, help="serving-mix only: number of requests (default 32)")
     ap.add_argument("--cpu-budget", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

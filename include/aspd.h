@@ -85,31 +85,38 @@ typedef struct {
 /* Optional knobs of plan creation (NULL = all automatic). */
 typedef struct {
   int32_t kernel;       /* ASPD_KERNEL_* */
-  int32_t chunk_tokens; /* keys per split-K work item (multiple of page_size); 0 = auto   */
+  int32_t chunk_tokens; /* cut work items at least every this many keys (multiple of
+                           page_size); 0 = only at the CTA boundaries                      */
   int32_t n_ctas;       /* size of the persistent grid; 0 = auto                           */
   int32_t host_only;    /* 1: build the work list on the host only (no CUDA call at all);
                            such a plan serves aspd_plan_info / aspd_plan_items only        */
 } aspd_tuning_t;
 
-/* One split-K work item of a plan, as aspd_plan_items reports it. */
+/* One split-K work item of a plan, as aspd_plan_items reports it.  The pages a request's
+ * step must read form one key stream (prefix, then the branches that have queries, or every
+ * branch and the tail in serial mode); an item is a run of pages of that stream for one KV
+ * head and one block of query tokens.  Key k of the stream is row k % page_size of stream page
+ * k / page_size. */
 typedef struct {
   int32_t q_tok0;     /* first new token (step order) of the item's row block               */
-  int32_t n_q_tok;    /* tokens in the block; rows = n_q_tok * (n_q_heads / n_kv_heads)     */
+  int32_t n_q_tok;    /* tokens in the block; rows = n_q_tok * (n_q_heads / n_kv_heads) <= 64 */
   int32_t kv_head;
-  int32_t page0;      /* index into page_ids[] of the chunk's first page                    */
-  int32_t n_keys;     /* keys of the chunk, starting at row 0 of page0                      */
-  int32_t causal0;    /* token i of the block sees chunk key j iff j <= causal0 + i         */
-  int32_t part_slot;  /* which of the token's partial results this item writes              */
+  int32_t page0;      /* index of the item's first page in the plan's stream-page list       */
+  int32_t n_pages;    /* pages of the item                                                   */
+  int32_t key0;       /* stream key index of the item's first key                            */
+  int32_t part_slot;  /* which partial record of (token, KV head) this item writes           */
   int32_t request;
 } aspd_item_t;
 
 typedef struct {
   int32_t n_new;            /* new tokens (= query tokens) of the step                      */
   int32_t n_items;          /* split-K work items                                           */
-  int32_t n_partials;       /* partial (m, l, O) records per query head, summed over tokens */
+  int32_t n_partials;       /* partial (m, l, O) records, summed over (token, KV head)      */
+  int32_t n_stream_pages;   /* entries of the stream-page list                             */
   int32_t kernel;           /* ASPD_KERNEL_* actually chosen                                */
-  int32_t chunk_tokens;
-  int32_t n_ctas;
+  int32_t chunk_tokens;     /* forced maximum keys per item (0: none)                       */
+  int32_t n_ctas;           /* CTAs of the persistent grid = shares the streams are cut into */
+  int32_t reserved;
   int64_t workspace_bytes;  /* device memory the plan holds                                 */
   int64_t kv_tokens_read;   /* cached tokens the step must read (each once)                 */
   int64_t algorithmic_bytes;/* K+V of those tokens + q in + out + appended K/V              */
@@ -165,6 +172,12 @@ int aspd_plan_destroy(aspd_plan_t* plan);
 int aspd_plan_info(const aspd_plan_t* plan, aspd_plan_info_t* info /*host*/);
 /* Copy up to max_items work items to `items` (host); returns the number of items. */
 int aspd_plan_items(const aspd_plan_t* plan, aspd_item_t* items, int max_items);
+/* The plan's stream-page list: physical page and number of valid rows of every page the step
+ * reads (host arrays of n_stream_pages entries each). */
+int aspd_plan_stream_pages(const aspd_plan_t* plan, int32_t* page_ids /*host*/, int32_t* n_valid /*host*/,
+                           int max_pages);
+/* Per new token, the stream keys it may attend: [0, pe) and [lo, hi) (host arrays of n_new). */
+int aspd_plan_token_ranges(const aspd_plan_t* plan, int32_t* pe, int32_t* lo, int32_t* hi, int max_tokens);
 /* Device status word of the plan (synchronises `stream`): ASPD_OK, or the first error a
  * kernel recorded (ASPD_ERR_TIMEOUT from a bounded wait, ASPD_ERR_BAD_DESCRIPTOR from a
  * bounds check). */

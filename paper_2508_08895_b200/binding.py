@@ -24,7 +24,7 @@ REQUEST_DTYPE = np.dtype([(n, np.int32) for n in
                           ("prefix_len", "n_branches", "branch_begin", "page_begin", "n_pages", "tail_off", "tail_len")])
 BRANCH_DTYPE = np.dtype([(n, np.int32) for n in ("kv_off", "kv_len", "pos_start", "q_len")])
 ITEM_DTYPE = np.dtype([(n, np.int32) for n in
-                       ("q_tok0", "n_q_tok", "kv_head", "page0", "n_keys", "causal0", "part_slot", "request")])
+                       ("q_tok0", "n_q_tok", "kv_head", "page0", "n_pages", "key0", "part_slot", "request")])
 
 
 class Shape(ctypes.Structure):
@@ -40,7 +40,8 @@ class Tuning(ctypes.Structure):
 
 class PlanInfo(ctypes.Structure):
     _fields_ = [("n_new", ctypes.c_int32), ("n_items", ctypes.c_int32), ("n_partials", ctypes.c_int32),
-                ("kernel", ctypes.c_int32), ("chunk_tokens", ctypes.c_int32), ("n_ctas", ctypes.c_int32),
+                ("n_stream_pages", ctypes.c_int32), ("kernel", ctypes.c_int32), ("chunk_tokens", ctypes.c_int32),
+                ("n_ctas", ctypes.c_int32), ("reserved", ctypes.c_int32),
                 ("workspace_bytes", ctypes.c_int64), ("kv_tokens_read", ctypes.c_int64),
                 ("algorithmic_bytes", ctypes.c_int64)]
 
@@ -52,7 +53,8 @@ class AspdError(RuntimeError):
 
 
 EXPORTS = ("aspd_strerror", "aspd_pool_bytes", "aspd_count_new_tokens", "aspd_positions", "aspd_visible_slots",
-           "aspd_plan_create", "aspd_plan_destroy", "aspd_plan_info", "aspd_plan_items", "aspd_plan_status",
+           "aspd_plan_create", "aspd_plan_destroy", "aspd_plan_info", "aspd_plan_items", "aspd_plan_stream_pages",
+           "aspd_plan_token_ranges", "aspd_plan_status",
            "aspd_kv_append", "aspd_branch_attn", "aspd_serial_attn", "aspd_attn_partials", "aspd_attn_combine",
            "aspd_step_host", "aspd_debug_read_token")
 
@@ -67,7 +69,8 @@ def lib() -> ctypes.CDLL:
     """Load the CUDA library (building it first if the sources are newer).  Fails loudly."""
     global _lib
     if _lib is None:
-        path = _build.build()
+        # ASPD_LIBRARY selects another build of the same sources (e.g. one with profiling hooks)
+        path = os.environ.get("ASPD_LIBRARY") or _build.build()
         L = ctypes.CDLL(path)
         L.aspd_strerror.restype = ctypes.c_char_p
         L.aspd_strerror.argtypes = [ctypes.c_int]
@@ -81,6 +84,8 @@ def lib() -> ctypes.CDLL:
         L.aspd_plan_destroy.argtypes = [vp]
         L.aspd_plan_info.argtypes = [vp, vp]
         L.aspd_plan_items.argtypes = [vp, vp, ci]
+        L.aspd_plan_stream_pages.argtypes = [vp, vp, vp, ci]
+        L.aspd_plan_token_ranges.argtypes = [vp, vp, vp, vp, ci]
         L.aspd_plan_status.argtypes = [vp, vp]
         L.aspd_kv_append.argtypes = [vp] * 7
         L.aspd_branch_attn.argtypes = [vp] * 6
@@ -198,6 +203,20 @@ class Plan:
         items = np.zeros(max(self.info.n_items, 1), dtype=ITEM_DTYPE)
         _check(lib().aspd_plan_items(self._h, _ptr(items), self.info.n_items), "aspd_plan_items")
         return items[: self.info.n_items]
+
+    def stream_pages(self):
+        """(physical page, valid rows) of every page the step reads, as two int32 arrays."""
+        n = self.info.n_stream_pages
+        ids, nv = np.zeros(max(n, 1), np.int32), np.zeros(max(n, 1), np.int32)
+        _check(lib().aspd_plan_stream_pages(self._h, _ptr(ids), _ptr(nv), n), "aspd_plan_stream_pages")
+        return ids[:n], nv[:n]
+
+    def token_ranges(self):
+        """(pe, lo, hi) per new token: it may attend stream keys [0, pe) and [lo, hi)."""
+        n = self.n_new
+        pe, lo, hi = (np.zeros(max(n, 1), np.int32) for _ in range(3))
+        _check(lib().aspd_plan_token_ranges(self._h, _ptr(pe), _ptr(lo), _ptr(hi), n), "aspd_plan_token_ranges")
+        return pe[:n], lo[:n], hi[:n]
 
     def status(self, stream=None) -> int:
         return lib().aspd_plan_status(self._h, _stream(stream))

@@ -20,17 +20,19 @@
 // raised when the tile maximum exceeds it by more than 2^8, which keeps P exactly consistent
 // with the (m, l, O) record while making the rescale of O in TMEM rare.
 //
-// Warp roles: 0-3 softmax / epilogue (TMEM lane quadrant = warp), 4 bulk-copy producer,
-// 5 MMA issuer (one elected lane), 6 query preparation (RoPE, bf16, swizzled store) one item
-// ahead.  All cross-role hand-offs are mbarriers; every wait is bounded and on expiry sets the
+// Warp roles: 0-3 softmax / epilogue (TMEM lane quadrant = warp), 4 and 7 bulk-copy producers
+// (K and V), 5 MMA issuer (one elected lane), 6 query preparation (RoPE, bf16, swizzled
+// store) one item ahead.  All cross-role hand-offs are mbarriers; every wait is bounded and on expiry sets the
 // plan's status word to ASPD_ERR_TIMEOUT and makes all roles drain and exit.
+#include <stdlib.h>
+
 #include "aspd_internal.cuh"
 
 namespace aspd {
 namespace {
 
 constexpr int kTile = 128;                     // keys per tile
-constexpr int kThreads = 224;
+constexpr int kThreads = 256;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRaise = 8.0f;                 // raise the reference maximum only beyond 2^8
 constexpr long long kWaitCycles = 3000000000LL; // ~1.5 s at 1.9 GHz
@@ -47,6 +49,7 @@ struct Misc {
   uint64_t bars[NUM_BARS];
   float smax[2][128];
   float sl[128];
+  int nval[4][8];              // valid rows of the 8 pages of a tile (ring over 4 tiles)
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -149,13 +152,27 @@ __device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t b_mn_major) 
   return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
+#ifdef ASPD_TC_PROFILE
+// Development aid: CTA 0 stamps clock64() at pipeline events of its first 64 tiles into the
+// buffer whose address is given by the environment (see launch_attn_mma).
+#define ASPD_STAMP(c, g, ev) do { if ((c).prof && blockIdx.x == 0 && (g) < 64) (c).prof[(g) * 16 + (ev)] = clock64(); } while (0)
+#else
+#define ASPD_STAMP(c, g, ev) do { } while (0)
+#endif
+
 struct Ctx {
   PlanDevice pd;
+  long long* prof;
   const __nv_bfloat16* q;
   const char* k_pool;
   const char* v_pool;
@@ -164,6 +181,12 @@ struct Ctx {
 };
 
 // ------------------------------------------------------------------------------- softmax role
+// 16-bit mask with bits [lo, hi) set (arguments are clamped to 0..16).
+__device__ __forceinline__ uint32_t bits_between(int lo, int hi) {
+  lo = max(lo, 0); hi = min(hi, 16);
+  return hi > lo ? ((0xFFFFu >> (16 - hi)) & ~((1u << lo) - 1u)) : 0u;
+}
+
 template <int NC>   // NC = columns per thread = padded row count R
 __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it, Misc* misc, uint32_t bars, uint32_t smem_p,
                                              uint32_t tmem, int item_no, int& g) {
@@ -171,13 +194,10 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
   const int tid = threadIdx.x, warp = tid >> 5;
   const int r = tid % R, j = tid / R;
   const int G = c.n_q_heads / c.n_kv_heads, M = it.n_q_tok * G;
-  const int n_tiles = (it.n_keys + kTile - 1) / kTile;
+  const int n_tiles = (it.n_pages + 7) >> 3;
   volatile int* ab = &misc->abort_flag;
-  int limit = 0;
-  if (r < M) {
-    long lim = (long)it.causal0 + r / G + 1;
-    limit = (int)(lim < 0 ? 0 : (lim > it.n_keys ? it.n_keys : lim));
-  }
+  int4 vis = make_int4(0, 0, 0, 0);             // padding rows see nothing
+  if (r < M) vis = c.pd.tok_vis[it.q_tok0 + r / G];
   const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
   const int ob = item_no & 1;
   float m_ref = -INFINITY, l = 0.f;
@@ -186,6 +206,7 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
     const int sb = g & 1;
     dead |= !mbar_wait(bars + 8 * (S_FULL + sb), (g >> 1) & 1, ab);
     tc_fence_after();
+    if (tid == 0) ASPD_STAMP(c, g, 0);
     float s[NC];
     const uint32_t s_addr = tmem + lane_addr + COL_S + sb * 128 + j * NC;
     ASPD_TMEM_LD32(s_addr, s, 0);
@@ -193,22 +214,36 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
     tmem_wait_ld();
     tc_fence_before();
     mbar_arrive(bars + 8 * (S_EMPTY + sb));
-    const int nvalid = limit - (t * kTile + j * NC);
+    if (tid == 0) ASPD_STAMP(c, g, 1);
+    // visibility of my NC keys: valid rows of each page, and the token's ranges [0, pe), [lo, hi)
     float mx = -INFINITY;
 #pragma unroll
-    for (int i = 0; i < NC; ++i) {
-      const float v = i < nvalid ? s[i] * c.scale_log2 : -INFINITY;
-      s[i] = v;
-      mx = fmaxf(mx, v);
+    for (int pg = 0; pg < NC / 16; ++pg) {
+      const int nv = misc->nval[g & 3][j * (NC / 16) + pg];
+      const int kb = it.key0 + t * kTile + j * NC + pg * 16;     // stream key of the page's first row
+      const uint32_t mask = bits_between(0, min(nv, vis.x - kb)) | bits_between(vis.y - kb, min(nv, vis.z - kb));
+      if (mask == 0xFFFFu) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) mx = fmaxf(mx, s[pg * 16 + i]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const float v = (mask >> i) & 1u ? s[pg * 16 + i] : -INFINITY;
+          s[pg * 16 + i] = v;
+          mx = fmaxf(mx, v);
+        }
+      }
     }
+    mx *= c.scale_log2;                           // the scale is positive: max commutes with it
     misc->smax[sb][tid] = mx;
     named_sync(1, 128);
+    if (tid == 0) ASPD_STAMP(c, g, 2);
     float m_tile = mx;
 #pragma unroll
     for (int jj = 0; jj < KS; ++jj) m_tile = fmaxf(m_tile, misc->smax[sb][jj * R + r]);
     const bool upd = m_tile > m_ref + kRaise;     // also true for the first finite maximum (m_ref = -inf)
     float alpha = 1.f;
-    if (upd) { alpha = exp2f(m_ref - m_tile); m_ref = m_tile; }
+    if (upd) { alpha = ex2(m_ref - m_tile); m_ref = m_tile; }
     l *= alpha;
     if (t > 0 && warp < R / 32) {                 // the owners of rows 0..R-1 rescale O in TMEM
       if (__any_sync(0xffffffffu, upd)) {
@@ -228,12 +263,19 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
         tc_fence_before();
       }
     }
-    const float msafe = m_ref == -INFINITY ? 0.f : m_ref;
-    float lsum = 0.f;
+    const float nmsafe = m_ref == -INFINITY ? 0.f : -m_ref;
+    float lsum0 = 0.f, lsum1 = 0.f;
 #pragma unroll
-    for (int i = 0; i < NC; ++i) { s[i] = exp2f(s[i] - msafe); lsum += s[i]; }
-    l += lsum;
+    for (int i = 0; i < NC; i += 2) {             // p = 2^(s * scale - m): one FFMA, one MUFU
+      s[i] = ex2(fmaf(s[i], c.scale_log2, nmsafe));
+      s[i + 1] = ex2(fmaf(s[i + 1], c.scale_log2, nmsafe));
+      lsum0 += s[i];
+      lsum1 += s[i + 1];
+    }
+    l += lsum0 + lsum1;
+    if (tid == 0) ASPD_STAMP(c, g, 3);
     if (g > 0) dead |= !mbar_wait(bars + 8 * P_EMPTY, (g - 1) & 1, ab);   // P tile is free again
+    if (tid == 0) ASPD_STAMP(c, g, 4);
 #pragma unroll
     for (int c8 = 0; c8 < NC / 8; ++c8) {
       const int kk = j * NC + c8 * 8;
@@ -245,6 +287,7 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
     fence_async_smem();
     tc_fence_before();
     mbar_arrive(bars + 8 * P_FULL);
+    if (tid == 0) ASPD_STAMP(c, g, 5);
   }
   // ---- epilogue: one (m, l, O) record per query row of the item
   dead |= !mbar_wait(bars + 8 * (O_FULL + ob), (item_no >> 1) & 1, ab);
@@ -255,16 +298,16 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
     float lt = 0.f;
 #pragma unroll
     for (int jj = 0; jj < KS; ++jj) lt += misc->sl[jj * R + r];
-    const int tok = it.q_tok0 + r / G, hq = it.kv_head * G + r % G;
-    const size_t rec = (size_t)(c.pd.part_base[tok] + it.part_slot) * c.n_q_heads + hq;
+    const int tok = it.q_tok0 + r / G;
+    const size_t rec = (size_t)(c.pd.part_base[tok * c.n_kv_heads + it.kv_head] + it.part_slot) * G + r % G;
     c.pd.ws_ml[rec] = make_float2(m_ref, lt);
   }
   if (warp < R / 32) {
     const uint32_t o_addr = tmem + lane_addr + COL_O + ob * 128;
     size_t rec = 0;
     if (r < M) {
-      const int tok = it.q_tok0 + r / G, hq = it.kv_head * G + r % G;
-      rec = (size_t)(c.pd.part_base[tok] + it.part_slot) * c.n_q_heads + hq;
+      const int tok = it.q_tok0 + r / G;
+      rec = (size_t)(c.pd.part_base[tok * c.n_kv_heads + it.kv_head] + it.part_slot) * G + r % G;
     }
 #pragma unroll 1
     for (int q4 = 0; q4 < 4; ++q4) {
@@ -283,6 +326,41 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
   return !named_sync_or(1, 128, dead || *ab);
 }
 
+// Rotate the item's query rows (RoPE at the token's position, table from the plan), round to
+// bf16 and store them, replicated KS times, as the 128-byte-swizzled A operand.  Called by
+// `nthr` threads with ranks `rank`.
+__device__ __forceinline__ void prep_q(const Ctx& c, const DeviceItem& it, uint32_t qbuf, int rank, int nthr) {
+  const int G = c.n_q_heads / c.n_kv_heads;
+  const int M = it.n_q_tok * G, R = M <= 32 ? 32 : 64, KS = 128 / R;
+#pragma unroll 2
+  for (int e = rank; e < R * 8; e += nthr) {
+    const int r = e >> 3, ch = e & 7;            // row, 8-element chunk of each half
+    uint32_t lo[4] = {0, 0, 0, 0}, hi[4] = {0, 0, 0, 0};
+    if (r < M) {
+      const int tok = it.q_tok0 + r / G, hq = it.kv_head * G + r % G;
+      const __nv_bfloat16* qrow = c.q + ((size_t)tok * c.n_q_heads + hq) * 128;
+      const uint4 a = *reinterpret_cast<const uint4*>(qrow + ch * 8);
+      const uint4 b = *reinterpret_cast<const uint4*>(qrow + 64 + ch * 8);
+      const float4* cs = reinterpret_cast<const float4*>(c.pd.q_cs + (size_t)tok * 64 + ch * 8);
+      const float4 w0 = cs[0], w1 = cs[1], w2 = cs[2], w3 = cs[3];
+      const float4 w[4] = {w0, w1, w2, w3};      // (cos, sin) of elements 2i and 2i+1 of the chunk
+      const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&a);
+      const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&b);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 x0 = __bfloat1622float2(a2[i]), x1 = __bfloat1622float2(b2[i]);
+        lo[i] = pack_bf16(x0.x * w[i].x - x1.x * w[i].y, x0.y * w[i].z - x1.y * w[i].w);
+        hi[i] = pack_bf16(x1.x * w[i].x + x0.x * w[i].y, x1.y * w[i].z + x0.y * w[i].w);
+      }
+    }
+    for (int jj = 0; jj < KS; ++jj) {
+      const uint32_t addr = qbuf + (jj * R + r) * 128 + ((ch ^ (r & 7)) << 4);
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr + kHalf), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
+    }
+  }
+}
+
 // --------------------------------------------------------------------------------- the kernel
 __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   extern __shared__ uint8_t smem_raw[];
@@ -293,6 +371,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   const uint32_t bars = base + OFF_MISC;          // bars[] is the first member of Misc
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* ab = &misc->abort_flag;
+  const int item_begin = c.pd.cta_item0[blockIdx.x], item_end = c.pd.cta_item0[blockIdx.x + 1];
 
   if (tid == 0) {
     const int counts[NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, 128, 128, 128, 1, 1, 1, 128, 128, 32, 32, 1, 1};
@@ -312,43 +391,64 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
 
   if (warp < 4) {
     // =============================== softmax + epilogue ===============================
+    // the first item's query tile is prepared here by all four warps (they have nothing else
+    // to do yet); later items are prepared one item ahead by the query warp
+    if (item_begin < item_end) {
+      prep_q(c, c.pd.items[item_begin], base + OFF_Q, tid, 128);
+      fence_async_smem();
+      named_sync(1, 128);
+      if (warp == 0) mbar_arrive(bars + 8 * Q_FULL);
+    }
     int g = 0, item_no = 0;
-    for (int idx = blockIdx.x; idx < c.n_items; idx += gridDim.x, ++item_no) {
+    for (int idx = item_begin; idx < item_end; ++idx, ++item_no) {
       const DeviceItem it = c.pd.items[idx];
       const int M = it.n_q_tok * (c.n_q_heads / c.n_kv_heads);
       const bool ok = M <= 32 ? softmax_item<32>(c, it, misc, bars, base + OFF_P, tmem, item_no, g)
                               : softmax_item<64>(c, it, misc, bars, base + OFF_P, tmem, item_no, g);
       if (!ok) break;
     }
-  } else if (warp == 4) {
-    // ================================ bulk-copy producer ================================
+  } else if (warp == 4 || warp == 7) {
+    // ================================ bulk-copy producers ================================
+    // Warp 4 streams the K tiles and warp 7 the V tiles, each on its own ring, so that a K load
+    // never queues behind a V slot that is still being read (and vice versa).
+    // Lane l keeps stream-page entry (batch * 32 + l) of the item in a register; the next batch
+    // of 32 entries (4 tiles) is requested before the current one is consumed, so the page list
+    // never sits on the critical path.
+    const int kv = warp == 4 ? 0 : 1;
+    const char* pool = kv ? c.v_pool : c.k_pool;
     int g = 0;
     bool ok = true;
-    for (int idx = blockIdx.x; idx < c.n_items && ok; idx += gridDim.x) {
+    for (int idx = item_begin; idx < item_end && ok; ++idx) {
       const DeviceItem it = c.pd.items[idx];
-      const int n_pages = (it.n_keys + 15) >> 4, n_tiles = (it.n_keys + kTile - 1) / kTile;
+      const int n_tiles = (it.n_pages + 7) >> 3;
+      int2 cur = make_int2(0, 0), nxt = make_int2(0, 0);
+      if (lane < it.n_pages) cur = c.pd.visit[it.page0 + lane];
       for (int t = 0; t < n_tiles && ok; ++t, ++g) {
-        const int npg = min(8, n_pages - t * 8), sl = g & 1;
-        int page = 0;
-        if (lane < npg) page = c.pd.page_ids[it.page0 + t * 8 + lane];
-        const size_t src_off = ((size_t)page * c.n_kv_heads + it.kv_head) * 4096;
-#pragma unroll
-        for (int kv = 0; kv < 2; ++kv) {
-          const uint32_t full = bars + 8 * ((kv ? V_FULL : K_FULL) + sl), empty = bars + 8 * ((kv ? V_EMPTY : K_EMPTY) + sl);
-          int good = 1;
-          if (lane == 0) {
-            good = mbar_wait(empty, ((g >> 1) & 1) ^ 1, ab) ? 1 : 0;
-            if (good) mbar_expect_tx(full, (uint32_t)npg * 4096u);
-          }
-          good = __shfl_sync(0xffffffffu, good, 0);
-          if (!good) { ok = false; break; }
-          if (lane < npg) {
-            const char* src = (kv ? c.v_pool : c.k_pool) + src_off;
-            const uint32_t dst = base + (kv ? OFF_V : OFF_K) + sl * kTileBytes + lane * 2048;
-            bulk_copy(dst, src, 2048, full);
-            bulk_copy(dst + kHalf, src + 2048, 2048, full);
-          }
+        if ((t & 3) == 0) {
+          if (t > 0) cur = nxt;
+          const int ahead = (t + 4) * 8 + lane;
+          nxt = make_int2(0, 0);
+          if (ahead < it.n_pages) nxt = c.pd.visit[it.page0 + ahead];
         }
+        const int npg = min(8, it.n_pages - t * 8), sl = g & 1;
+        int2 pg;
+        pg.x = __shfl_sync(0xffffffffu, cur.x, (t & 3) * 8 + (lane & 7));
+        pg.y = __shfl_sync(0xffffffffu, cur.y, (t & 3) * 8 + (lane & 7));
+        if (lane >= npg) pg = make_int2(0, 0);
+        const uint32_t full = bars + 8 * ((kv ? V_FULL : K_FULL) + sl), empty = bars + 8 * ((kv ? V_EMPTY : K_EMPTY) + sl);
+        int good = 1;
+        if (lane == 0) good = mbar_wait(empty, ((g >> 1) & 1) ^ 1, ab) ? 1 : 0;
+        good = __shfl_sync(0xffffffffu, good, 0);
+        if (!good) { ok = false; break; }
+        if (lane == 0) ASPD_STAMP(c, g, 6 + kv);
+        if (kv == 0 && lane < 8) misc->nval[g & 3][lane] = pg.y;      // read by the softmax warps of tile g
+        __syncwarp();
+        if (lane == 0) mbar_expect_tx(full, (uint32_t)npg * 4096u);
+        __syncwarp();
+        if (lane < npg)
+          bulk_copy(base + (kv ? OFF_V : OFF_K) + sl * kTileBytes + lane * 4096,
+                    pool + ((size_t)pg.x * c.n_kv_heads + it.kv_head) * 4096, 4096, full);
+        if (lane == 0) ASPD_STAMP(c, g, 13 + kv);
       }
     }
   } else if (warp == 5) {
@@ -359,86 +459,66 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
       const uint32_t idesc_pv = instr_desc(128, 1);
       // PV of global tile gg (item-local tile tt) of the item whose O buffer is ob
       auto issue_pv = [&](int gg, int tt, int npg, int ob, int ino) -> bool {
+        ASPD_STAMP(c, gg, 10);
         if (!mbar_wait(bars + 8 * P_FULL, gg & 1, ab)) return false;
+        ASPD_STAMP(c, gg, 11);
         if (!mbar_wait(bars + 8 * (V_FULL + (gg & 1)), (gg >> 1) & 1, ab)) return false;
         if (tt == 0 && !mbar_wait(bars + 8 * (O_EMPTY + ob), ((ino >> 1) & 1) ^ 1, ab)) return false;
         tc_fence_after();
         const uint32_t pbuf = base + OFF_P, vbuf = base + OFF_V + (gg & 1) * kTileBytes;
         for (int ks = 0; ks < npg; ++ks) {
           const uint64_t a = smem_desc(pbuf + (ks >> 2) * kHalf + (ks & 3) * 32, 16, 1024);
-          const uint64_t b = smem_desc(vbuf + ks * 2048, kHalf, 1024);
+          const uint64_t b = smem_desc(vbuf + ks * 4096, 1024, 2048);   // 16 keys = one page per k-step
           tc_mma(tmem + COL_O + ob * 128, a, b, idesc_pv, (tt > 0 || ks > 0) ? 1u : 0u);
         }
+        ASPD_STAMP(c, gg, 12);
         tc_commit(bars + 8 * P_EMPTY);
         tc_commit(bars + 8 * (V_EMPTY + (gg & 1)));
         return true;
       };
-      for (int idx = blockIdx.x; idx < c.n_items && ok; idx += gridDim.x, ++item_no) {
+      for (int idx = item_begin; idx < item_end && ok; ++idx, ++item_no) {
         const DeviceItem it = c.pd.items[idx];
-        const int n_pages = (it.n_keys + 15) >> 4, n_tiles = (it.n_keys + kTile - 1) / kTile;
+        const int n_tiles = (it.n_pages + 7) >> 3;
         const int qb = item_no & 1, ob = item_no & 1;
         if (!mbar_wait(bars + 8 * (Q_FULL + qb), (item_no >> 1) & 1, ab)) { ok = false; break; }
         for (int t = 0; t < n_tiles; ++t, ++g) {
-          const int npg = min(8, n_pages - t * 8), sb = g & 1;
+          const int npg = min(8, it.n_pages - t * 8), sb = g & 1;
           if (!mbar_wait(bars + 8 * (K_FULL + sb), (g >> 1) & 1, ab) ||
               !mbar_wait(bars + 8 * (S_EMPTY + sb), ((g >> 1) & 1) ^ 1, ab)) { ok = false; break; }
           tc_fence_after();
+          ASPD_STAMP(c, g, 8);
           const uint32_t qbuf = base + OFF_Q + qb * kTileBytes, kbuf = base + OFF_K + sb * kTileBytes;
           const uint32_t idesc_s = instr_desc((uint32_t)npg * 16u, 0);
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
-            const uint32_t off = (ks >> 2) * kHalf + (ks & 3) * 32;
-            tc_mma(tmem + COL_S + sb * 128, smem_desc(qbuf + off, 16, 1024), smem_desc(kbuf + off, 16, 1024), idesc_s,
-                   ks > 0 ? 1u : 0u);
+            // k-step ks covers head_dim elements [16 ks, 16 ks + 16): span ks / 4, 32 bytes per step
+            const uint64_t a = smem_desc(qbuf + (ks >> 2) * kHalf + (ks & 3) * 32, 16, 1024);
+            const uint64_t b = smem_desc(kbuf + (ks >> 2) * 1024 + (ks & 3) * 32, 16, 2048);
+            tc_mma(tmem + COL_S + sb * 128, a, b, idesc_s, ks > 0 ? 1u : 0u);
           }
+          ASPD_STAMP(c, g, 9);
           tc_commit(bars + 8 * (S_FULL + sb));
           tc_commit(bars + 8 * (K_EMPTY + sb));
           if (t == n_tiles - 1) tc_commit(bars + 8 * (Q_EMPTY + qb));
           if (t > 0 && !issue_pv(g - 1, t - 1, 8, ob, item_no)) { ok = false; break; }
         }
         if (!ok) break;
-        if (!issue_pv(g - 1, n_tiles - 1, min(8, n_pages - (n_tiles - 1) * 8), ob, item_no)) { ok = false; break; }
+        if (!issue_pv(g - 1, n_tiles - 1, min(8, it.n_pages - (n_tiles - 1) * 8), ob, item_no)) { ok = false; break; }
         tc_commit(bars + 8 * (O_FULL + ob));
       }
     }
     __syncwarp();
   } else {
     // ================================ query preparation ================================
-    int item_no = 0;
-    const int G = c.n_q_heads / c.n_kv_heads;
-    for (int idx = blockIdx.x; idx < c.n_items; idx += gridDim.x, ++item_no) {
+    int item_no = 1;
+    for (int idx = item_begin + 1; idx < item_end; ++idx, ++item_no) {
       const DeviceItem it = c.pd.items[idx];
-      const int M = it.n_q_tok * G, R = M <= 32 ? 32 : 64, KS = 128 / R, qb = item_no & 1;
+      const int qb = item_no & 1;
       int good = 1;
       if (lane == 0) good = mbar_wait(bars + 8 * (Q_EMPTY + qb), ((item_no >> 1) & 1) ^ 1, ab) ? 1 : 0;
       good = __shfl_sync(0xffffffffu, good, 0);
       if (!good) break;
-      const uint32_t qbuf = base + OFF_Q + qb * kTileBytes;
-      for (int e = lane; e < R * 8; e += 32) {
-        const int r = e >> 3, ch = e & 7;          // row, 8-element chunk of each half
-        uint32_t lo[4] = {0, 0, 0, 0}, hi[4] = {0, 0, 0, 0};
-        if (r < M) {
-          const int tok = it.q_tok0 + r / G, hq = it.kv_head * G + r % G;
-          const __nv_bfloat16* qrow = c.q + ((size_t)tok * c.n_q_heads + hq) * 128;
-          const uint4 a = *reinterpret_cast<const uint4*>(qrow + ch * 8);
-          const uint4 b = *reinterpret_cast<const uint4*>(qrow + 64 + ch * 8);
-          const float4* cs = reinterpret_cast<const float4*>(c.pd.q_cs + (size_t)tok * 64 + ch * 8);
-          const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&a);
-          const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&b);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float4 w = cs[i];                // (cos, sin) of elements 2i and 2i+1
-            const float2 x0 = __bfloat1622float2(a2[i]), x1 = __bfloat1622float2(b2[i]);
-            lo[i] = pack_bf16(x0.x * w.x - x1.x * w.y, x0.y * w.z - x1.y * w.w);
-            hi[i] = pack_bf16(x1.x * w.x + x0.x * w.y, x1.y * w.z + x0.y * w.w);
-          }
-        }
-        for (int jj = 0; jj < KS; ++jj) {
-          const uint32_t addr = qbuf + (jj * R + r) * 128 + ((ch ^ (r & 7)) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr + kHalf), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
-        }
-      }
+      prep_q(c, it, base + OFF_Q + qb * kTileBytes, lane, 32);
       fence_async_smem();
       mbar_arrive(bars + 8 * (Q_FULL + qb));
     }
@@ -471,6 +551,10 @@ int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const
   }
   Ctx c;
   c.pd = p->dev;
+  c.prof = nullptr;
+#ifdef ASPD_TC_PROFILE
+  if (const char* e = getenv("ASPD_TC_PROFILE_BUF")) c.prof = (long long*)strtoull(e, nullptr, 0);
+#endif
   c.q = (const __nv_bfloat16*)q;
   c.k_pool = (const char*)k_pool;
   c.v_pool = (const char*)v_pool;
@@ -478,8 +562,7 @@ int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const
   c.n_q_heads = sh.n_q_heads;
   c.n_kv_heads = sh.n_kv_heads;
   c.scale_log2 = sh.sm_scale * kLog2e;
-  const int grid = p->n_items < p->n_ctas ? p->n_items : p->n_ctas;
-  attn_tc_kernel<<<grid, kThreads, kSmemBytes, s>>>(c);
+  attn_tc_kernel<<<p->n_ctas, kThreads, kSmemBytes, s>>>(c);
   return cudaGetLastError() == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
 }
 

@@ -12,38 +12,44 @@
 namespace aspd {
 
 constexpr int kMaxRowsPerItem = 64;   // query rows (tokens x group heads) one work item carries
-constexpr int kCausalAll = 1 << 29;   // causal0 value of a fully visible chunk
+constexpr int kCausalAll = 1 << 29;   // prefix end of a token that sees its whole key stream
 
 // ---------------------------------------------------------------------------------------
-// Cache tile format.  One (page, KV head) tile holds page_size tokens x head_dim elements.
-// A token row is cut into 128-byte spans; span s of all tokens is stored together as
-// [page_size][128 B], and inside it the 16-byte chunk index is XOR-ed with (token & 7).
-// That is the 128-byte-swizzled, K-major shared-memory image the tensor-core and ldmatrix
-// paths want, so a tile lands in shared memory with linear bulk copies and no re-layout.
+// Cache tile format.  One (page, KV head) tile holds page_size tokens x head_dim elements,
+// row_bytes = head_dim * element size per token.  Tokens are taken in groups of 8 and a token
+// row is cut into 128-byte spans; the tile is stored as [token group][span][8 tokens][128 B],
+// and inside each 1 KiB block the 16-byte chunk index is XOR-ed with (token & 7).  Every 1 KiB
+// block is a 128-byte-swizzle atom of the tensor core's shared-memory operands, and the blocks
+// of one span lie a constant 8 * row_bytes apart even across consecutive tiles, so whole tiles
+// copied back to back into shared memory (one linear bulk copy each) form a valid K-major
+// operand (keys x head_dim, for Q.K^T) and MN-major operand (head_dim x keys, for P.V) as is.
 // ---------------------------------------------------------------------------------------
 __host__ __device__ inline size_t tile_bytes(int page_size, int head_dim, int esize) {
   return (size_t)page_size * head_dim * esize;
 }
 // Byte offset, inside a tile, of byte `b` (multiple of the element size) of token `t`'s row.
-__host__ __device__ inline uint32_t tile_offset(int t, uint32_t b, int page_size) {
-  uint32_t span = b >> 7, in = b & 127u;
-  return span * (uint32_t)page_size * 128u + (uint32_t)t * 128u + ((((in >> 4) ^ (uint32_t)(t & 7)) << 4) | (in & 15u));
+__host__ __device__ inline uint32_t tile_offset(int t, uint32_t b, uint32_t row_bytes) {
+  const uint32_t span = b >> 7, in = b & 127u;
+  return (uint32_t)(t >> 3) * (8u * row_bytes) + span * 1024u + (uint32_t)(t & 7) * 128u +
+         ((((in >> 4) ^ (uint32_t)(t & 7)) << 4) | (in & 15u));
 }
 
 struct DeviceItem {       // mirrors aspd_item_t, 32 bytes
-  int32_t q_tok0, n_q_tok, kv_head, page0, n_keys, causal0, part_slot, request;
+  int32_t q_tok0, n_q_tok, kv_head, page0, n_pages, key0, part_slot, request;
 };
 
 struct PlanDevice {       // pointers into the plan's single device allocation
   const DeviceItem* items;
-  const int32_t* page_ids;     // concatenated page tables (physical page per logical page)
+  const int32_t* cta_item0;    // [n_ctas + 1] items of CTA c are [cta_item0[c], cta_item0[c + 1])
+  const int2* visit;           // key streams: (physical page, valid rows) per page to read
+  const int4* tok_vis;         // [n_new] (pe, lo, hi, -): visible stream keys are [0, pe) and [lo, hi)
   const int32_t* tok_page;     // [n_new] physical page the new token's K/V goes to
   const int32_t* tok_row;      // [n_new] row inside that page
   const float2* q_cs;          // [n_new][head_dim/2] (cos, sin) of the query's RoPE angle
-  const int32_t* part_base;    // [n_new + 1] first partial record of each new token
+  const int32_t* part_base;    // [n_new * n_kv_heads + 1] first partial record of (new token, KV head)
   const double* inv_freq;      // [head_dim/2]
-  float* ws_o;                 // [n_partials][n_q_heads][head_dim] un-normalised partial outputs
-  float2* ws_ml;               // [n_partials][n_q_heads] (running max in log2 units, sum)
+  float* ws_o;                 // [n_partials][G][head_dim] un-normalised partial outputs
+  float2* ws_ml;               // [n_partials][G] (reference max in log2 units, sum)
   int32_t* status;             // first error recorded by a kernel
   int32_t* work_counter;       // dynamic work-list cursor (reset by its last reader)
   // staging for aspd_step_host
@@ -71,6 +77,8 @@ struct aspd_plan {
   void* device_base;
   aspd::PlanDevice dev;
   std::vector<aspd::DeviceItem> items;
+  std::vector<int2> visit;
+  std::vector<int4> tok_vis;
 };
 
 namespace aspd {

@@ -35,7 +35,8 @@ __global__ void append_kernel(const T* __restrict__ k_new, const T* __restrict__
   const float y0 = x0 * cs - x1 * sn, y1 = x1 * cs + x0 * sn;
   const size_t tile = ((size_t)tok_page[t] * n_kv_heads + h) * tile_bytes(page_size, head_dim, sizeof(T));
   const int row = tok_row[t];
-  const uint32_t o0 = tile_offset(row, i * sizeof(T), page_size), o1 = tile_offset(row, (i + half) * sizeof(T), page_size);
+  const uint32_t rb = head_dim * sizeof(T);
+  const uint32_t o0 = tile_offset(row, i * sizeof(T), rb), o1 = tile_offset(row, (i + half) * sizeof(T), rb);
   char* kp = reinterpret_cast<char*>(k_pool) + tile;
   char* vp = reinterpret_cast<char*>(v_pool) + tile;
   *reinterpret_cast<T*>(kp + o0) = from_f32<T>(y0);
@@ -57,7 +58,7 @@ __global__ void __launch_bounds__(128) attn_generic_kernel(PlanDevice pd, const 
   __shared__ float q_s[4][D];
   const DeviceItem it = pd.items[blockIdx.x];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int G = n_q_heads / n_kv_heads, n_rows = it.n_q_tok * G;
+  const int G = n_q_heads / n_kv_heads, n_rows = it.n_q_tok * G, n_keys = it.n_pages * page_size;
   const size_t tb = tile_bytes(page_size, D, sizeof(T));
   for (int r = warp; r < n_rows; r += 4) {
     const int tl = r / G, g = r % G, tok = it.q_tok0 + tl, hq = it.kv_head * G + g;
@@ -70,54 +71,60 @@ __global__ void __launch_bounds__(128) attn_generic_kernel(PlanDevice pd, const 
       q_s[warp][i + D / 2] = (x1 * cs.x + x0 * cs.y) * scale_log2;
     }
     __syncwarp();
-    long lim = (long)it.causal0 + tl + 1;
-    const int limit = (int)(lim < 0 ? 0 : (lim > it.n_keys ? it.n_keys : lim));
+    const int4 vis = pd.tok_vis[tok];           // stream keys [0, pe) and [lo, hi) are visible
     float m = -INFINITY, l = 0.f, acc[EPL];
 #pragma unroll
     for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-    for (int base = 0; base < limit; base += 32) {
+    for (int base = 0; base < n_keys; base += 32) {
       const int j = base + lane;
+      bool seen = false;
       float s = -INFINITY;
-      if (j < limit) {
-        const int page = pd.page_ids[it.page0 + j / page_size], row = j % page_size;
-        const char* tile = reinterpret_cast<const char*>(k_pool) + ((size_t)page * n_kv_heads + it.kv_head) * tb;
-        float dot = 0.f;
+      if (j < n_keys) {
+        const int2 pg = pd.visit[it.page0 + j / page_size];
+        const int row = j % page_size, kg = it.key0 + j;
+        seen = row < pg.y && (kg < vis.x || (kg >= vis.y && kg < vis.z));
+        if (seen) {
+          const char* tile = reinterpret_cast<const char*>(k_pool) + ((size_t)pg.x * n_kv_heads + it.kv_head) * tb;
+          float dot = 0.f;
 #pragma unroll 4
-        for (int c = 0; c < D / EPC; ++c) {
-          const uint4 raw = *reinterpret_cast<const uint4*>(tile + tile_offset(row, c * 16, page_size));
-          const T* e8 = reinterpret_cast<const T*>(&raw);
+          for (int c = 0; c < D / EPC; ++c) {
+            const uint4 raw = *reinterpret_cast<const uint4*>(tile + tile_offset(row, c * 16, D * sizeof(T)));
+            const T* e8 = reinterpret_cast<const T*>(&raw);
 #pragma unroll
-          for (int e = 0; e < EPC; ++e) dot = fmaf(q_s[warp][c * EPC + e], to_f32(e8[e]), dot);
+            for (int e = 0; e < EPC; ++e) dot = fmaf(q_s[warp][c * EPC + e], to_f32(e8[e]), dot);
+          }
+          s = dot;
         }
-        s = dot;
       }
+      if (!__any_sync(0xffffffffu, seen)) continue;
       float mx = s;
 #pragma unroll
       for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-      const float m_new = fmaxf(m, mx);
-      const float p = j < limit ? exp2f(s - m_new) : 0.f;
-      const float alpha = exp2f(m - m_new);           // m = -inf on the first group: alpha = 0
+      const float m_new = fmaxf(m, mx);           // finite: at least one key of the group is seen
+      const float p = seen ? exp2f(s - m_new) : 0.f;
+      const float alpha = exp2f(m - m_new);       // m = -inf before the first seen key: alpha = 0
       float ps = p;
 #pragma unroll
       for (int o = 16; o; o >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
       l = l * alpha + ps;
 #pragma unroll
       for (int e = 0; e < EPL; ++e) acc[e] *= alpha;
-      const int cnt = min(32, limit - base);
+      const int cnt = min(32, n_keys - base);
       for (int jj = 0; jj < cnt; ++jj) {
         const float pj = __shfl_sync(0xffffffffu, p, jj);
+        if (pj == 0.f) continue;                  // masked (or negligible) key: its V row is not touched
         const int key = base + jj;
-        const int page = pd.page_ids[it.page0 + key / page_size], row = key % page_size;
-        const char* tile = reinterpret_cast<const char*>(v_pool) + ((size_t)page * n_kv_heads + it.kv_head) * tb;
+        const int2 pg = pd.visit[it.page0 + key / page_size];
+        const char* tile = reinterpret_cast<const char*>(v_pool) + ((size_t)pg.x * n_kv_heads + it.kv_head) * tb;
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {
-          const T v = *reinterpret_cast<const T*>(tile + tile_offset(row, (lane * EPL + e) * sizeof(T), page_size));
+          const T v = *reinterpret_cast<const T*>(tile + tile_offset(key % page_size, (lane * EPL + e) * sizeof(T), D * sizeof(T)));
           acc[e] = fmaf(pj, to_f32(v), acc[e]);
         }
       }
       m = m_new;
     }
-    const size_t rec = (size_t)(pd.part_base[tok] + it.part_slot) * n_q_heads + hq;
+    const size_t rec = (size_t)(pd.part_base[tok * n_kv_heads + it.kv_head] + it.part_slot) * G + g;
     if (lane == 0) pd.ws_ml[rec] = make_float2(m, l);
 #pragma unroll
     for (int e = 0; e < EPL; ++e) pd.ws_o[rec * D + lane * EPL + e] = acc[e];
@@ -126,33 +133,60 @@ __global__ void __launch_bounds__(128) attn_generic_kernel(PlanDevice pd, const 
 }
 
 // ------------------------------------------------------------------------------ combine
-// One warp per (new token, query head): merge the token's partial records.
-template <typename T>
-__global__ void combine_kernel(PlanDevice pd, T* __restrict__ out, int n_new, int n_q_heads, int head_dim) {
+// One warp per (new token, query head): merge the partial records of (token, KV head) by
+// log-sum-exp.  The (max, sum) pairs are read lane-parallel; the O rows are then streamed with
+// several independent loads in flight.
+template <typename T, int D>
+__global__ void combine_kernel(PlanDevice pd, T* __restrict__ out, int n_new, int n_q_heads, int n_kv_heads) {
+  constexpr int EPL = D / 32;
   const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (w >= n_new * n_q_heads) return;
-  const int tok = w / n_q_heads, hq = w % n_q_heads;
-  const int p0 = pd.part_base[tok], p1 = pd.part_base[tok + 1];
+  const int tok = w / n_q_heads, hq = w % n_q_heads, G = n_q_heads / n_kv_heads, h = hq / G, g = hq % G;
+  const int p0 = pd.part_base[tok * n_kv_heads + h], n = pd.part_base[tok * n_kv_heads + h + 1] - p0;
   float M = -INFINITY;
-  for (int p = p0; p < p1; ++p) M = fmaxf(M, pd.ws_ml[(size_t)p * n_q_heads + hq].x);
-  float L = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
-  const int epl = head_dim / 32;
-  for (int p = p0; p < p1; ++p) {
-    const size_t rec = (size_t)p * n_q_heads + hq;
-    const float2 ml = pd.ws_ml[rec];
-    if (ml.y == 0.f) continue;                        // a chunk with no visible key
-    const float w8 = exp2f(ml.x - M);
-    L += ml.y * w8;
-    for (int e = 0; e < epl; ++e) acc[e] = fmaf(pd.ws_o[rec * head_dim + lane * epl + e], w8, acc[e]);
+  for (int i = lane; i < n; i += 32) {
+    const float2 ml = pd.ws_ml[(size_t)(p0 + i) * G + g];
+    if (ml.y > 0.f) M = fmaxf(M, ml.x);
   }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  float L = 0.f, acc[EPL];
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+  for (int base = 0; base < n; base += 32) {
+    float wt = 0.f;
+    if (base + lane < n) {
+      const float2 ml = pd.ws_ml[(size_t)(p0 + base + lane) * G + g];
+      if (ml.y > 0.f) { wt = exp2f(ml.x - M); L += ml.y * wt; }     // records of chunks with no visible key have sum 0
+    }
+    const int cnt = min(32, n - base);
+#pragma unroll 4
+    for (int i = 0; i < cnt; ++i) {
+      const float wi = __shfl_sync(0xffffffffu, wt, i);
+      const float* row = pd.ws_o + ((size_t)(p0 + base + i) * G + g) * D + lane * EPL;
+      if (wi != 0.f) {
+        if constexpr (EPL == 4) {
+          const float4 v = *reinterpret_cast<const float4*>(row);
+          acc[0] = fmaf(v.x, wi, acc[0]); acc[1] = fmaf(v.y, wi, acc[1]); acc[2] = fmaf(v.z, wi, acc[2]); acc[3] = fmaf(v.w, wi, acc[3]);
+        } else {
+          const float2 v = *reinterpret_cast<const float2*>(row);
+          acc[0] = fmaf(v.x, wi, acc[0]); acc[1] = fmaf(v.y, wi, acc[1]);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
   const float inv = 1.f / L;
-  for (int e = 0; e < epl; ++e) out[((size_t)tok * n_q_heads + hq) * head_dim + lane * epl + e] = from_f32<T>(acc[e] * inv);
+  T* dst = out + ((size_t)tok * n_q_heads + hq) * D + lane * EPL;
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) dst[e] = from_f32<T>(acc[e] * inv);
 }
 
 template <typename T>
-__global__ void read_token_kernel(const T* pool, size_t tile, int row, int page_size, float* out) {
+__global__ void read_token_kernel(const T* pool, size_t tile, int row, int head_dim, float* out) {
   const int e = threadIdx.x;
-  out[e] = to_f32(*reinterpret_cast<const T*>(reinterpret_cast<const char*>(pool) + tile + tile_offset(row, e * sizeof(T), page_size)));
+  out[e] = to_f32(*reinterpret_cast<const T*>(reinterpret_cast<const char*>(pool) + tile + tile_offset(row, e * sizeof(T), head_dim * sizeof(T))));
 }
 
 inline int check_launch() { return cudaGetLastError() == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA; }
@@ -195,10 +229,12 @@ int launch_combine(const aspd_plan* p, void* out, cudaStream_t s) {
   const aspd_shape_t& sh = p->shape;
   const int warps = p->n_new * sh.n_q_heads;
   const dim3 block(128), grid((warps + 3) / 4);
-  if (sh.dtype == ASPD_DTYPE_BF16)
-    combine_kernel<__nv_bfloat16><<<grid, block, 0, s>>>(p->dev, (__nv_bfloat16*)out, p->n_new, sh.n_q_heads, sh.head_dim);
-  else
-    combine_kernel<float><<<grid, block, 0, s>>>(p->dev, (float*)out, p->n_new, sh.n_q_heads, sh.head_dim);
+#define ASPD_CMB(T, D) combine_kernel<T, D><<<grid, block, 0, s>>>(p->dev, (T*)out, p->n_new, sh.n_q_heads, sh.n_kv_heads)
+  if (sh.dtype == ASPD_DTYPE_BF16 && sh.head_dim == 128) ASPD_CMB(__nv_bfloat16, 128);
+  else if (sh.dtype == ASPD_DTYPE_BF16) ASPD_CMB(__nv_bfloat16, 64);
+  else if (sh.head_dim == 128) ASPD_CMB(float, 128);
+  else ASPD_CMB(float, 64);
+#undef ASPD_CMB
   return check_launch();
 }
 
@@ -207,9 +243,9 @@ int launch_read_token(const aspd_shape_t* sh, const void* pool, int64_t page, in
   const int es = esize_of(sh->dtype);
   const size_t tile = ((size_t)page * sh->n_kv_heads + kv_head) * tile_bytes(sh->page_size, sh->head_dim, es);
   if (sh->dtype == ASPD_DTYPE_BF16)
-    read_token_kernel<__nv_bfloat16><<<1, sh->head_dim, 0, s>>>((const __nv_bfloat16*)pool, tile, row, sh->page_size, out_dev);
+    read_token_kernel<__nv_bfloat16><<<1, sh->head_dim, 0, s>>>((const __nv_bfloat16*)pool, tile, row, sh->head_dim, out_dev);
   else
-    read_token_kernel<float><<<1, sh->head_dim, 0, s>>>((const float*)pool, tile, row, sh->page_size, out_dev);
+    read_token_kernel<float><<<1, sh->head_dim, 0, s>>>((const float*)pool, tile, row, sh->head_dim, out_dev);
   return check_launch();
 }
 

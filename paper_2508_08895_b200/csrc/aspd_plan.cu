@@ -89,8 +89,6 @@ int check_layout(const aspd_shape_t* s, const aspd_request_t* req, const aspd_br
   return ASPD_OK;
 }
 
-struct Segment { int key0, n_keys, causal0, tok0, n_tok, slot0; };
-
 }  // namespace
 
 extern "C" {
@@ -241,114 +239,123 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
     if (q_pos) { if (q_pos[t] < 0) { delete p; return ASPD_ERR_INVALID_ARG; } pos[t] = q_pos[t]; }
   }
 
-  // ---- segments: (key range, rows that see it, causal rule) ---------------------------
+  // ---- key streams -------------------------------------------------------------------
+  // Per request, the pages the step must read, in one sequence: the prefix, then every branch
+  // that has queries (branch mode) or every branch and the tail (serial mode).  Each entry is
+  // (physical page, valid rows); the padding rows of partly filled pages are masked by the
+  // kernels.  A new token sees stream keys [0, pe) (the prefix) and [lo, hi) (its own branch up
+  // to itself); a serial token sees the whole stream.
   const int max_tok = std::max(1, kMaxRowsPerItem / G);
-  std::vector<std::vector<Segment>> segs(n_req);
-  std::vector<int> req_tok0(n_req + 1, 0);
-  long total_cost = 0;
+  std::vector<int2> visit;
+  std::vector<int> visit0(n_req + 1, 0), req_tok0(n_req + 1, 0);
+  std::vector<int4> tok_vis(n_new);
   int64_t kv_tokens = 0;
   {
     int t = 0;
+    auto push_region = [&](const aspd_request_t& q, int slot0, int len) {
+      for (int s0 = 0; s0 < len; s0 += ps)
+        visit.push_back(make_int2(page_ids[q.page_begin + (slot0 + s0) / ps], std::min(ps, len - s0)));
+      kv_tokens += len;
+    };
     for (int r = 0; r < n_req; ++r) {
       const aspd_request_t& q = req[r];
       req_tok0[r] = t;
+      visit0[r] = (int)visit.size();
       if (mode == ASPD_MODE_BRANCH) {
         int nq = 0;
         for (int b = 0; b < q.n_branches; ++b) nq += br[q.branch_begin + b].q_len;
-        if (nq > 0 && q.prefix_len > 0) segs[r].push_back({0, q.prefix_len, kCausalAll, t, nq, 0});
-        if (nq > 0) kv_tokens += q.prefix_len;
-        for (int b = 0; b < q.n_branches; ++b) {
-          const aspd_branch_t& x = br[q.branch_begin + b];
-          if (x.q_len > 0) {
-            segs[r].push_back({x.kv_off, x.kv_len, x.kv_len - x.q_len, t, x.q_len, 0});
-            kv_tokens += x.kv_len;
+        if (nq > 0) {
+          push_region(q, 0, q.prefix_len);
+          const int pe = ((int)visit.size() - visit0[r]) * ps;
+          for (int b = 0; b < q.n_branches; ++b) {
+            const aspd_branch_t& x = br[q.branch_begin + b];
+            if (x.q_len == 0) continue;
+            const int lo = ((int)visit.size() - visit0[r]) * ps;
+            push_region(q, x.kv_off, x.kv_len);
+            for (int i = 0; i < x.q_len; ++i) tok_vis[t++] = make_int4(pe, lo, lo + x.kv_len - x.q_len + i + 1, 0);
           }
-          t += x.q_len;
         }
       } else {
-        if (q.prefix_len > 0) segs[r].push_back({0, q.prefix_len, kCausalAll, t, 1, 0});
-        kv_tokens += q.prefix_len;
+        push_region(q, 0, q.prefix_len);
         for (int b = 0; b < q.n_branches; ++b) {
           const aspd_branch_t& x = br[q.branch_begin + b];
-          if (x.kv_len > 0) segs[r].push_back({x.kv_off, x.kv_len, kCausalAll, t, 1, 0});
-          kv_tokens += x.kv_len;
+          push_region(q, x.kv_off, x.kv_len);
         }
-        segs[r].push_back({q.tail_off, q.tail_len, kCausalAll, t, 1, 0});
-        kv_tokens += q.tail_len;
-        t += 1;
+        push_region(q, q.tail_off, q.tail_len);
+        tok_vis[t++] = make_int4(kCausalAll, 0, 0, 0);
       }
-      for (const Segment& s : segs[r]) total_cost += (long)ceil_div(s.n_keys, ps) * ceil_div(s.n_tok, max_tok) * Hkv;
     }
     req_tok0[n_req] = t;
+    visit0[n_req] = (int)visit.size();
   }
 
-  // ---- chunk size: about four items per CTA of the persistent grid --------------------
-  int n_ctas = tune.n_ctas > 0 ? tune.n_ctas : p->sm_count;
-  int chunk = tune.chunk_tokens;
-  if (chunk == 0) {
-    long target_items = (long)n_ctas * 4;
-    long pages = std::max(1L, (total_cost + target_items - 1) / target_items);
-    pages = std::min(std::max(pages, 8L), 256L);
-    chunk = (int)pages * ps;
-  }
-  p->chunk_tokens = chunk; p->n_ctas = n_ctas;
-
-  // ---- items and partial slots --------------------------------------------------------
-  std::vector<int32_t> n_parts(n_new, 0), part_base(n_new + 1, 0);
+  // ---- work items: a contiguous, equal share of all pages for every CTA -----------------
+  // Streams are walked in the order (request, row block, KV head); the concatenation of all
+  // streams is cut at the CTA boundaries (and, if asked for, every chunk_tokens keys).
+  struct Stream { int request, tok0, n_tok, head, page0, n_pages; };
+  std::vector<Stream> streams;
+  long total_pages = 0;
   for (int r = 0; r < n_req; ++r) {
-    for (Segment& s : segs[r]) {
-      // equal-sized chunks (whole pages) instead of full chunks plus a sliver
-      const int per = ceil_div(ceil_div(s.n_keys, ceil_div(s.n_keys, chunk)), ps) * ps;
-      const int n_chunks = ceil_div(s.n_keys, per);
-      // every token of the segment gets n_chunks consecutive partial slots
-      int slot0 = n_parts[s.tok0];
-      for (int i = 0; i < s.n_tok; ++i) n_parts[s.tok0 + i] += n_chunks;
-      s.slot0 = slot0;
-      for (int c = 0; c < n_chunks; ++c) {
-        const int k0 = c * per, nk = std::min(per, s.n_keys - k0);
-        for (int i0 = 0; i0 < s.n_tok; i0 += max_tok) {
-          const int nt = std::min(max_tok, s.n_tok - i0);
-          for (int h = 0; h < Hkv; ++h) {
-            DeviceItem it;
-            it.q_tok0 = s.tok0 + i0; it.n_q_tok = nt; it.kv_head = h;
-            it.page0 = req[r].page_begin + (s.key0 + k0) / ps;
-            it.n_keys = nk;
-            it.causal0 = s.causal0 == kCausalAll ? kCausalAll : s.causal0 - k0 + i0;
-            it.part_slot = slot0 + c; it.request = r;
-            p->items.push_back(it);
-          }
-        }
+    const int nt = req_tok0[r + 1] - req_tok0[r], np = visit0[r + 1] - visit0[r];
+    if (nt == 0 || np == 0) continue;
+    for (int i0 = 0; i0 < nt; i0 += max_tok)
+      for (int h = 0; h < Hkv; ++h) {
+        streams.push_back({r, req_tok0[r] + i0, std::min(max_tok, nt - i0), h, visit0[r], np});
+        total_pages += np;
       }
-    }
   }
-  // In branch mode the prefix segment comes first for every token of a request, so its
-  // slots [0, n_chunks) coincide for all of them; branch segments follow per branch.
-  for (int t = 0; t < n_new; ++t) part_base[t + 1] = part_base[t] + n_parts[t];
-  std::stable_sort(p->items.begin(), p->items.end(), [](const DeviceItem& a, const DeviceItem& b) {
-    return (long)a.n_keys * (a.n_q_tok > 2 ? 2 : 1) > (long)b.n_keys * (b.n_q_tok > 2 ? 2 : 1);
-  });
+  const int min_pages = 4;                       // do not cut finer than 64 keys per CTA
+  int n_ctas = tune.n_ctas > 0 ? tune.n_ctas : p->sm_count;
+  n_ctas = (int)std::max(1L, std::min((long)n_ctas, (total_pages + min_pages - 1) / min_pages));
+  const int chunk_pages = tune.chunk_tokens > 0 ? tune.chunk_tokens / ps : (1 << 28);
+  p->chunk_tokens = tune.chunk_tokens; p->n_ctas = n_ctas;
+  std::vector<int32_t> n_parts((size_t)n_new * Hkv, 0), part_base((size_t)n_new * Hkv + 1, 0), cta_item0(n_ctas + 1, 0);
+  {
+    long g0 = 0;                                 // global page offset of the current stream
+    int cta = 0;
+    auto boundary = [&](int c) { return (long)c * total_pages / n_ctas; };
+    for (const Stream& st : streams) {
+      int at = 0, slot = 0;
+      while (at < st.n_pages) {
+        while (cta + 1 < n_ctas && boundary(cta + 1) <= g0 + at) cta_item0[++cta] = (int)p->items.size();
+        long stop = std::min<long>(st.n_pages, at + chunk_pages);
+        if (cta + 1 <= n_ctas) stop = std::min<long>(stop, std::max<long>(boundary(cta + 1) - g0, at + 1));
+        DeviceItem it;
+        it.q_tok0 = st.tok0; it.n_q_tok = st.n_tok; it.kv_head = st.head; it.page0 = st.page0 + at;
+        it.n_pages = (int)stop - at; it.key0 = at * ps; it.part_slot = slot++; it.request = st.request;
+        p->items.push_back(it);
+        at = (int)stop;
+      }
+      for (int i = 0; i < st.n_tok; ++i) n_parts[(size_t)(st.tok0 + i) * Hkv + st.head] = slot;
+      g0 += st.n_pages;
+    }
+    while (cta < n_ctas) cta_item0[++cta] = (int)p->items.size();
+  }
+  for (size_t i = 0; i < n_parts.size(); ++i) part_base[i + 1] = part_base[i] + n_parts[i];
   p->n_items = (int)p->items.size();
-  p->n_partials = part_base[n_new];
+  p->n_partials = part_base[n_parts.size()];
   p->kv_tokens_read = kv_tokens;
   p->algorithmic_bytes = 2LL * Hkv * d * es * kv_tokens + 2LL * es * Hq * d * n_new + 2LL * Hkv * d * es * n_new;
+  p->visit = visit;
+  p->tok_vis = tok_vis;
   if (tune.host_only) { *plan_out = p; return ASPD_OK; }
 
   // ---- one device allocation, one staging blob ------------------------------------------
-  int total_pages = 0;
-  for (int r = 0; r < n_req; ++r) total_pages = std::max(total_pages, req[r].page_begin + req[r].n_pages);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   const size_t o_items = take(sizeof(DeviceItem) * std::max(1, p->n_items));
-  const size_t o_pages = take(sizeof(int32_t) * std::max(1, total_pages));
+  const size_t o_cta = take(sizeof(int32_t) * (n_ctas + 1));
+  const size_t o_visit = take(sizeof(int2) * std::max<size_t>(1, visit.size()));
   const size_t o_tpage = take(sizeof(int32_t) * std::max(1, n_new));
   const size_t o_trow = take(sizeof(int32_t) * std::max(1, n_new));
+  const size_t o_tvis = take(sizeof(int4) * std::max(1, n_new));
   const size_t o_qcs = take(sizeof(float2) * std::max(1, n_new) * (d / 2));
-  const size_t o_pbase = take(sizeof(int32_t) * (n_new + 1));
+  const size_t o_pbase = take(sizeof(int32_t) * part_base.size());
   const size_t o_freq = take(sizeof(double) * (d / 2));
   const size_t o_status = take(sizeof(int32_t) * 2);
   const size_t upload_bytes = off;
-  const size_t o_wso = take(sizeof(float) * (size_t)std::max(1, p->n_partials) * Hq * d);
-  const size_t o_wsml = take(sizeof(float2) * (size_t)std::max(1, p->n_partials) * Hq);
+  const size_t o_wso = take(sizeof(float) * (size_t)std::max(1, p->n_partials) * G * d);
+  const size_t o_wsml = take(sizeof(float2) * (size_t)std::max(1, p->n_partials) * G);
   const size_t o_stq = take((size_t)es * std::max(1, n_new) * Hq * d);
   const size_t o_stk = take((size_t)es * std::max(1, n_new) * Hkv * d);
   const size_t o_stv = take((size_t)es * std::max(1, n_new) * Hkv * d);
@@ -358,12 +365,14 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
 
   std::vector<uint8_t> blob(upload_bytes, 0);
   if (p->n_items) memcpy(blob.data() + o_items, p->items.data(), sizeof(DeviceItem) * p->n_items);
-  if (total_pages) memcpy(blob.data() + o_pages, page_ids, sizeof(int32_t) * total_pages);
+  memcpy(blob.data() + o_cta, cta_item0.data(), sizeof(int32_t) * (n_ctas + 1));
+  if (!visit.empty()) memcpy(blob.data() + o_visit, visit.data(), sizeof(int2) * visit.size());
   if (n_new) {
     memcpy(blob.data() + o_tpage, tok_page.data(), sizeof(int32_t) * n_new);
     memcpy(blob.data() + o_trow, tok_row.data(), sizeof(int32_t) * n_new);
+    memcpy(blob.data() + o_tvis, tok_vis.data(), sizeof(int4) * n_new);
   }
-  memcpy(blob.data() + o_pbase, part_base.data(), sizeof(int32_t) * (n_new + 1));
+  memcpy(blob.data() + o_pbase, part_base.data(), sizeof(int32_t) * part_base.size());
   double* freq = reinterpret_cast<double*>(blob.data() + o_freq);
   for (int i = 0; i < d / 2; ++i) freq[i] = pow((double)shape->rope_theta, -2.0 * i / d);
   float2* qcs = reinterpret_cast<float2*>(blob.data() + o_qcs);
@@ -383,7 +392,9 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   uint8_t* b8 = (uint8_t*)base;
   p->device_base = base;
   p->dev.items = (const DeviceItem*)(b8 + o_items);
-  p->dev.page_ids = (const int32_t*)(b8 + o_pages);
+  p->dev.cta_item0 = (const int32_t*)(b8 + o_cta);
+  p->dev.visit = (const int2*)(b8 + o_visit);
+  p->dev.tok_vis = (const int4*)(b8 + o_tvis);
   p->dev.tok_page = (const int32_t*)(b8 + o_tpage);
   p->dev.tok_row = (const int32_t*)(b8 + o_trow);
   p->dev.q_cs = (const float2*)(b8 + o_qcs);
@@ -409,8 +420,9 @@ int aspd_plan_destroy(aspd_plan_t* plan) {
 
 int aspd_plan_info(const aspd_plan_t* p, aspd_plan_info_t* info) {
   if (!p || !info) return ASPD_ERR_INVALID_ARG;
-  info->n_new = p->n_new; info->n_items = p->n_items; info->n_partials = p->n_partials; info->kernel = p->kernel;
-  info->chunk_tokens = p->chunk_tokens; info->n_ctas = p->n_ctas; info->workspace_bytes = (int64_t)p->device_bytes;
+  info->n_new = p->n_new; info->n_items = p->n_items; info->n_partials = p->n_partials;
+  info->n_stream_pages = (int32_t)p->visit.size(); info->kernel = p->kernel;
+  info->chunk_tokens = p->chunk_tokens; info->n_ctas = p->n_ctas; info->reserved = 0; info->workspace_bytes = (int64_t)p->device_bytes;
   info->kv_tokens_read = p->kv_tokens_read; info->algorithmic_bytes = p->algorithmic_bytes;
   return ASPD_OK;
 }
@@ -421,6 +433,20 @@ int aspd_plan_items(const aspd_plan_t* p, aspd_item_t* items, int max_items) {
   static_assert(sizeof(aspd_item_t) == sizeof(DeviceItem), "item layouts must match");
   if (n) memcpy(items, p->items.data(), sizeof(DeviceItem) * n);
   return p->n_items;
+}
+
+int aspd_plan_stream_pages(const aspd_plan_t* p, int32_t* page_ids, int32_t* n_valid, int max_pages) {
+  if (!p || max_pages < 0 || (max_pages > 0 && (!page_ids || !n_valid))) return ASPD_ERR_INVALID_ARG;
+  const int n = std::min<int>(max_pages, (int)p->visit.size());
+  for (int i = 0; i < n; ++i) { page_ids[i] = p->visit[i].x; n_valid[i] = p->visit[i].y; }
+  return (int)p->visit.size();
+}
+
+int aspd_plan_token_ranges(const aspd_plan_t* p, int32_t* pe, int32_t* lo, int32_t* hi, int max_tokens) {
+  if (!p || max_tokens < 0 || (max_tokens > 0 && (!pe || !lo || !hi))) return ASPD_ERR_INVALID_ARG;
+  const int n = std::min<int>(max_tokens, (int)p->tok_vis.size());
+  for (int i = 0; i < n; ++i) { pe[i] = p->tok_vis[i].x; lo[i] = p->tok_vis[i].y; hi[i] = p->tok_vis[i].z; }
+  return (int)p->tok_vis.size();
 }
 
 int aspd_plan_status(aspd_plan_t* p, void* stream) {

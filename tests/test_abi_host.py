@@ -80,39 +80,70 @@ def _shape(wl):
     return B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
 
 
-@pytest.mark.parametrize("chunk", [0, 16, 48, 4096])
-def test_work_list_covers_every_visible_key_exactly_once(chunk):
-    """Integers only: the split-K items of a plan, expanded to (token, KV head, slot) triples
-    under their causal rule, are exactly the visible sets, each key once."""
+@pytest.mark.parametrize("chunk,n_ctas", [(0, 0), (16, 0), (48, 5), (4096, 1), (0, 1000)])
+def test_work_list_covers_every_visible_key_exactly_once(chunk, n_ctas):
+    """Integers only: the work items of a plan, expanded through its stream-page list and the
+    per-token visible ranges to (token, KV head, logical slot) triples, are exactly the oracle's
+    visible sets, each key once."""
     for wl in small_workloads():
         for ph in wl.phases:
-            plan = B.Plan(_shape(wl), ph.desc, wl.n_pool_pages, ph.mode, chunk_tokens=chunk, host_only=True)
+            plan = B.Plan(_shape(wl), ph.desc, wl.n_pool_pages, ph.mode, chunk_tokens=chunk, n_ctas=n_ctas, host_only=True)
             n_slots = int(ph.desc["n_pages"].max()) * wl.page_size
             vis = oracle.visible_slots(ph.desc, ph.mode, n_slots)
             _, _, treq = oracle.new_tokens(ph.desc, ph.mode)
+            page_ids, n_valid = plan.stream_pages()
+            pe, lo, hi = plan.token_ranges()
+            # physical page -> (request, logical page)
+            where = {}
+            for r in range(len(ph.desc["prefix_len"])):
+                pb = int(ph.desc["page_begin"][r])
+                for lp in range(int(ph.desc["n_pages"][r])):
+                    where[int(ph.desc["page_ids"][pb + lp])] = (r, lp)
             count = np.zeros((plan.n_new, wl.Hkv, n_slots), dtype=np.int32)
             slots_seen = {}
+            ps = wl.page_size
             for it in plan.items():
-                r = int(it["request"])
-                lp0 = int(it["page0"]) - int(ph.desc["page_begin"][r])
-                assert 0 <= lp0 < int(ph.desc["n_pages"][r])
-                assert it["n_q_tok"] * wl.G <= 64 and it["n_keys"] >= 1
+                assert it["n_q_tok"] * wl.G <= 64 and it["n_pages"] >= 1 and it["key0"] % ps == 0
+                if chunk:
+                    assert it["n_pages"] * ps <= chunk
                 for i in range(int(it["n_q_tok"])):
                     tok = int(it["q_tok0"]) + i
-                    assert treq[tok] == r
-                    lim = min(int(it["n_keys"]), int(it["causal0"]) + i + 1)
-                    if lim > 0:
-                        count[tok, int(it["kv_head"]), lp0 * wl.page_size: lp0 * wl.page_size + lim] += 1
-                    key = (tok, int(it["kv_head"]))
-                    slots_seen.setdefault(key, []).append(int(it["part_slot"]))
+                    assert treq[tok] == it["request"]
+                    for pg in range(int(it["n_pages"])):
+                        e = int(it["page0"]) + pg
+                        r, lp = where[int(page_ids[e])]
+                        assert r == it["request"]
+                        for row in range(int(n_valid[e])):
+                            kg = int(it["key0"]) + pg * ps + row
+                            if kg < pe[tok] or lo[tok] <= kg < hi[tok]:
+                                count[tok, int(it["kv_head"]), lp * ps + row] += 1
+                    slots_seen.setdefault((tok, int(it["kv_head"])), []).append(int(it["part_slot"]))
             for h in range(wl.Hkv):
                 np.testing.assert_array_equal(count[:, h, :], vis.astype(np.int32))
             # partial slots of a (token, head) are 0 .. n-1, each used once
             for key, sl in slots_seen.items():
                 assert sorted(sl) == list(range(len(sl)))
-            assert plan.info.n_partials == sum(len(v) for k, v in slots_seen.items() if k[1] == 0)
-            assert plan.info.kv_tokens_read * 1 >= 0
+            assert plan.info.n_partials == sum(len(v) for v in slots_seen.values())
+            # pages read = pages of the streams, every one with 1..page_size valid rows
+            assert ((n_valid >= 1) & (n_valid <= ps)).all()
+            assert plan.info.kv_tokens_read == int(n_valid.sum())
             plan.destroy()
+
+
+def test_streams_are_cut_into_equal_shares():
+    wl = W.build_segment_workload("cut", 12, 28, 4, 128, "bf16", 1e6, [1000, 300, 2000], [[100, 30], [10], [5, 5, 5]],
+                                  [[1, 1], [1], [1, 1, 1]])
+    ph = wl.phases[-1]
+    for n_ctas in (1, 7, 32):
+        plan = B.Plan(_shape(wl), ph.desc, wl.n_pool_pages, ph.mode, n_ctas=n_ctas, host_only=True)
+        items = plan.items()
+        total = int(items["n_pages"].sum())
+        assert total == plan.info.n_stream_pages * wl.Hkv
+        assert plan.info.n_ctas == n_ctas
+        # the items, in order, tile the concatenated streams; cutting it into n_ctas contiguous
+        # shares of (almost) equal size never needs more than one extra item per share
+        assert len(items) <= 3 * wl.Hkv + n_ctas
+        plan.destroy()
 
 
 def test_algorithmic_bytes_formula():
