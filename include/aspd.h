@@ -106,6 +106,8 @@ typedef struct {
   int32_t key0;       /* stream key index of the item's first key                            */
   int32_t part_slot;  /* which partial record of (token, KV head) this item writes           */
   int32_t request;
+  int32_t row_block;  /* index of the item's block of query tokens among all blocks of the step */
+  int32_t reserved;
 } aspd_item_t;
 
 typedef struct {

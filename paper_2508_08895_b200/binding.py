@@ -24,7 +24,8 @@ REQUEST_DTYPE = np.dtype([(n, np.int32) for n in
                           ("prefix_len", "n_branches", "branch_begin", "page_begin", "n_pages", "tail_off", "tail_len")])
 BRANCH_DTYPE = np.dtype([(n, np.int32) for n in ("kv_off", "kv_len", "pos_start", "q_len")])
 ITEM_DTYPE = np.dtype([(n, np.int32) for n in
-                       ("q_tok0", "n_q_tok", "kv_head", "page0", "n_pages", "key0", "part_slot", "request")])
+                       ("q_tok0", "n_q_tok", "kv_head", "page0", "n_pages", "key0", "part_slot", "request", "row_block",
+                        "reserved")])
 
 
 class Shape(ctypes.Structure):

@@ -32,7 +32,7 @@ namespace aspd {
 namespace {
 
 constexpr int kTile = 128;                     // keys per tile
-constexpr int kThreads = 256;
+constexpr int kThreads = 384;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRaise = 8.0f;                 // raise the reference maximum only beyond 2^8
 constexpr long long kWaitCycles = 3000000000LL; // ~1.5 s at 1.9 GHz
@@ -40,20 +40,24 @@ constexpr long long kWaitCycles = 3000000000LL; // ~1.5 s at 1.9 GHz
 constexpr uint32_t kTileBytes = 32768;         // one K, V, Q or P tile: 128 rows x 256 B
 constexpr uint32_t kHalf = 16384;              // second 64-element span of a tile
 constexpr uint32_t OFF_K = 0, OFF_V = 2 * kTileBytes, OFF_Q = 4 * kTileBytes, OFF_P = 6 * kTileBytes;
-constexpr uint32_t OFF_MISC = 7 * kTileBytes;
+// Rows 64..127 of the P tile are never written (R <= 64) and the rows of O they produce are
+// never read, so the barriers and small exchange arrays live in that hole of the first span.
+constexpr uint32_t OFF_MISC = OFF_P + 8192;
 
 enum Bar { K_FULL = 0, K_EMPTY = 2, V_FULL = 4, V_EMPTY = 6, S_FULL = 8, S_EMPTY = 10, P_FULL = 12, P_EMPTY = 13,
-           O_FULL = 14, O_EMPTY = 16, Q_FULL = 18, Q_EMPTY = 20, NUM_BARS = 22 };
+           O_FULL = 14, O_EMPTY = 16, Q_FULL = 18, Q_EMPTY = 20, E_FULL = 22, NUM_BARS = 24 };
 
 struct Misc {
   uint64_t bars[NUM_BARS];
   float smax[2][128];
-  float sl[128];
+  float fin_m[2][128];         // per item parity: reference maximum and sum of every softmax thread
+  float fin_l[2][128];
   int nval[4][8];              // valid rows of the 8 pages of a tile (ring over 4 tiles)
   uint32_t tmem_base;
   int abort_flag;
 };
-constexpr size_t kSmemBytes = OFF_MISC + sizeof(Misc) + 1024;   // + slack to align the base to 1024
+static_assert(sizeof(Misc) <= 8192, "Misc must fit into the unused rows of the P tile");
+constexpr size_t kSmemBytes = 7 * kTileBytes + 1024;   // + slack to align the base to 1024
 
 // TMEM columns: S double buffer, O double buffer
 constexpr uint32_t COL_S = 0, COL_O = 256;
@@ -166,8 +170,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 // Development aid: CTA 0 stamps clock64() at pipeline events of its first 64 tiles into the
 // buffer whose address is given by the environment (see launch_attn_mma).
 #define ASPD_STAMP(c, g, ev) do { if ((c).prof && blockIdx.x == 0 && (g) < 64) (c).prof[(g) * 16 + (ev)] = clock64(); } while (0)
+// every CTA: globaltimer (ns) at entry / after set-up / after its last epilogue / at exit
+__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define ASPD_CTA_STAMP(c, ev) do { if ((c).prof) (c).prof[1024 + blockIdx.x * 4 + (ev)] = gtime(); } while (0)
 #else
 #define ASPD_STAMP(c, g, ev) do { } while (0)
+#define ASPD_CTA_STAMP(c, ev) do { } while (0)
 #endif
 
 struct Ctx {
@@ -289,75 +297,49 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
     mbar_arrive(bars + 8 * P_FULL);
     if (tid == 0) ASPD_STAMP(c, g, 5);
   }
-  // ---- epilogue: one (m, l, O) record per query row of the item
-  dead |= !mbar_wait(bars + 8 * (O_FULL + ob), (item_no >> 1) & 1, ab);
-  tc_fence_after();
-  misc->sl[tid] = l;
-  named_sync(1, 128);
-  if (j == 0 && r < M && !dead) {
-    float lt = 0.f;
-#pragma unroll
-    for (int jj = 0; jj < KS; ++jj) lt += misc->sl[jj * R + r];
-    const int tok = it.q_tok0 + r / G;
-    const size_t rec = (size_t)(c.pd.part_base[tok * c.n_kv_heads + it.kv_head] + it.part_slot) * G + r % G;
-    c.pd.ws_ml[rec] = make_float2(m_ref, lt);
-  }
-  if (warp < R / 32) {
-    const uint32_t o_addr = tmem + lane_addr + COL_O + ob * 128;
-    size_t rec = 0;
-    if (r < M) {
-      const int tok = it.q_tok0 + r / G;
-      rec = (size_t)(c.pd.part_base[tok * c.n_kv_heads + it.kv_head] + it.part_slot) * G + r % G;
-    }
-#pragma unroll 1
-    for (int q4 = 0; q4 < 4; ++q4) {
-      float o[32];
-      ASPD_TMEM_LD32(o_addr + q4 * 32, o, 0);
-      tmem_wait_ld();
-      if (r < M && !dead) {
-        float4* dst = reinterpret_cast<float4*>(c.pd.ws_o + rec * 128 + q4 * 32);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
-      }
-    }
-  }
-  tc_fence_before();
-  mbar_arrive(bars + 8 * (O_EMPTY + ob));
+  // ---- hand the item's statistics to the epilogue warps and move on to the next item
+  dead |= !mbar_wait(bars + 8 * (O_EMPTY + ob), ((item_no >> 1) & 1) ^ 1, ab);   // epilogue of item_no - 2 is done
+  misc->fin_m[ob][tid] = m_ref;
+  misc->fin_l[ob][tid] = l;
+  mbar_arrive(bars + 8 * (E_FULL + ob));
   return !named_sync_or(1, 128, dead || *ab);
 }
 
-// Rotate the item's query rows (RoPE at the token's position, table from the plan), round to
-// bf16 and store them, replicated KS times, as the 128-byte-swizzled A operand.  Called by
-// `nthr` threads with ranks `rank`.
-__device__ __forceinline__ void prep_q(const Ctx& c, const DeviceItem& it, uint32_t qbuf, int rank, int nthr) {
-  const int G = c.n_q_heads / c.n_kv_heads;
-  const int M = it.n_q_tok * G, R = M <= 32 ? 32 : 64, KS = 128 / R;
-#pragma unroll 2
-  for (int e = rank; e < R * 8; e += nthr) {
-    const int r = e >> 3, ch = e & 7;            // row, 8-element chunk of each half
-    uint32_t lo[4] = {0, 0, 0, 0}, hi[4] = {0, 0, 0, 0};
+// Pre-pass: rotate the query rows of every (row block, KV head) (RoPE at the token's position,
+// table from the plan), round to bf16 and store them as the image of the A operand:
+// [2 spans][R rows][128 B], 16-byte chunks XOR-ed with (row & 7), R = 32 or 64, rows >= M zero.
+// The main kernel then brings a query tile in with a few linear bulk copies.
+__global__ void __launch_bounds__(128) q_rotate_kernel(PlanDevice pd, const __nv_bfloat16* __restrict__ q, int n_q_heads,
+                                                       int n_kv_heads) {
+  const int rb = blockIdx.x / n_kv_heads, head = blockIdx.x % n_kv_heads;
+  const int2 blk = pd.row_blocks[rb];
+  const int G = n_q_heads / n_kv_heads, M = blk.y * G, R = M <= 32 ? 32 : 64;
+  char* img = pd.q_img + (size_t)blockIdx.x * kQImageBytes;
+  for (int e = threadIdx.x; e < R * 8; e += 128) {
+    const int r = e >> 3, ch = e & 7;            // row, 8-element chunk of each span
+    uint4 lo = make_uint4(0, 0, 0, 0), hi = make_uint4(0, 0, 0, 0);
     if (r < M) {
-      const int tok = it.q_tok0 + r / G, hq = it.kv_head * G + r % G;
-      const __nv_bfloat16* qrow = c.q + ((size_t)tok * c.n_q_heads + hq) * 128;
+      const int tok = blk.x + r / G, hq = head * G + r % G;
+      const __nv_bfloat16* qrow = q + ((size_t)tok * n_q_heads + hq) * 128;
       const uint4 a = *reinterpret_cast<const uint4*>(qrow + ch * 8);
       const uint4 b = *reinterpret_cast<const uint4*>(qrow + 64 + ch * 8);
-      const float4* cs = reinterpret_cast<const float4*>(c.pd.q_cs + (size_t)tok * 64 + ch * 8);
-      const float4 w0 = cs[0], w1 = cs[1], w2 = cs[2], w3 = cs[3];
-      const float4 w[4] = {w0, w1, w2, w3};      // (cos, sin) of elements 2i and 2i+1 of the chunk
+      const float4* cs = reinterpret_cast<const float4*>(pd.q_cs + (size_t)tok * 64 + ch * 8);
+      const float4 w[4] = {cs[0], cs[1], cs[2], cs[3]};   // (cos, sin) of elements 2i and 2i+1 of the chunk
       const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&a);
       const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&b);
+      uint32_t l4[4], h4[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const float2 x0 = __bfloat1622float2(a2[i]), x1 = __bfloat1622float2(b2[i]);
-        lo[i] = pack_bf16(x0.x * w[i].x - x1.x * w[i].y, x0.y * w[i].z - x1.y * w[i].w);
-        hi[i] = pack_bf16(x1.x * w[i].x + x0.x * w[i].y, x1.y * w[i].z + x0.y * w[i].w);
+        l4[i] = pack_bf16(x0.x * w[i].x - x1.x * w[i].y, x0.y * w[i].z - x1.y * w[i].w);
+        h4[i] = pack_bf16(x1.x * w[i].x + x0.x * w[i].y, x1.y * w[i].z + x0.y * w[i].w);
       }
+      lo = make_uint4(l4[0], l4[1], l4[2], l4[3]);
+      hi = make_uint4(h4[0], h4[1], h4[2], h4[3]);
     }
-    for (int jj = 0; jj < KS; ++jj) {
-      const uint32_t addr = qbuf + (jj * R + r) * 128 + ((ch ^ (r & 7)) << 4);
-      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
-      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr + kHalf), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
-    }
+    const uint32_t off = r * 128 + ((ch ^ (r & 7)) << 4);
+    *reinterpret_cast<uint4*>(img + off) = lo;
+    *reinterpret_cast<uint4*>(img + R * 128 + off) = hi;
   }
 }
 
@@ -371,10 +353,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   const uint32_t bars = base + OFF_MISC;          // bars[] is the first member of Misc
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* ab = &misc->abort_flag;
+  if (tid == 0) ASPD_CTA_STAMP(c, 0);
   const int item_begin = c.pd.cta_item0[blockIdx.x], item_end = c.pd.cta_item0[blockIdx.x + 1];
 
   if (tid == 0) {
-    const int counts[NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, 128, 128, 128, 1, 1, 1, 128, 128, 32, 32, 1, 1};
+    const int counts[NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, 128, 128, 128, 1, 1, 1, 128, 128, 1, 1, 1, 1, 128, 128};
     for (int i = 0; i < NUM_BARS; ++i) mbar_init(bars + 8 * i, counts[i]);
     misc->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -388,17 +371,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = misc->tmem_base;
+  if (tid == 0) ASPD_CTA_STAMP(c, 1);
 
   if (warp < 4) {
     // =============================== softmax + epilogue ===============================
-    // the first item's query tile is prepared here by all four warps (they have nothing else
-    // to do yet); later items are prepared one item ahead by the query warp
-    if (item_begin < item_end) {
-      prep_q(c, c.pd.items[item_begin], base + OFF_Q, tid, 128);
-      fence_async_smem();
-      named_sync(1, 128);
-      if (warp == 0) mbar_arrive(bars + 8 * Q_FULL);
-    }
     int g = 0, item_no = 0;
     for (int idx = item_begin; idx < item_end; ++idx, ++item_no) {
       const DeviceItem it = c.pd.items[idx];
@@ -453,74 +429,132 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     }
   } else if (warp == 5) {
     // =================================== MMA issuer ===================================
+    // The tiles of all items form one pipeline: S of tile g is issued before P.V of tile g - 1,
+    // also across an item boundary, so the tensor pipe and the softmax warps never drain
+    // between items.
     if (lane == 0) {
-      int g = 0, item_no = 0;
-      bool ok = true;
+      struct TileRef { int npg, first, last, qb, ob, item_no; };
       const uint32_t idesc_pv = instr_desc(128, 1);
-      // PV of global tile gg (item-local tile tt) of the item whose O buffer is ob
-      auto issue_pv = [&](int gg, int tt, int npg, int ob, int ino) -> bool {
-        ASPD_STAMP(c, gg, 10);
-        if (!mbar_wait(bars + 8 * P_FULL, gg & 1, ab)) return false;
-        ASPD_STAMP(c, gg, 11);
-        if (!mbar_wait(bars + 8 * (V_FULL + (gg & 1)), (gg >> 1) & 1, ab)) return false;
-        if (tt == 0 && !mbar_wait(bars + 8 * (O_EMPTY + ob), ((ino >> 1) & 1) ^ 1, ab)) return false;
+      auto issue_s = [&](const TileRef& tr, int g) -> bool {
+        const int sb = g & 1;
+        if (tr.first && !mbar_wait(bars + 8 * (Q_FULL + tr.qb), (tr.item_no >> 1) & 1, ab)) return false;
+        if (!mbar_wait(bars + 8 * (K_FULL + sb), (g >> 1) & 1, ab)) return false;
+        if (!mbar_wait(bars + 8 * (S_EMPTY + sb), ((g >> 1) & 1) ^ 1, ab)) return false;
         tc_fence_after();
-        const uint32_t pbuf = base + OFF_P, vbuf = base + OFF_V + (gg & 1) * kTileBytes;
-        for (int ks = 0; ks < npg; ++ks) {
-          const uint64_t a = smem_desc(pbuf + (ks >> 2) * kHalf + (ks & 3) * 32, 16, 1024);
-          const uint64_t b = smem_desc(vbuf + ks * 4096, 1024, 2048);   // 16 keys = one page per k-step
-          tc_mma(tmem + COL_O + ob * 128, a, b, idesc_pv, (tt > 0 || ks > 0) ? 1u : 0u);
+        ASPD_STAMP(c, g, 8);
+        const uint32_t qbuf = base + OFF_Q + tr.qb * kTileBytes, kbuf = base + OFF_K + sb * kTileBytes;
+        const uint32_t idesc_s = instr_desc((uint32_t)tr.npg * 16u, 0);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          // k-step ks covers head_dim elements [16 ks, 16 ks + 16): span ks / 4, 32 bytes per step
+          const uint64_t a = smem_desc(qbuf + (ks >> 2) * kHalf + (ks & 3) * 32, 16, 1024);
+          const uint64_t b = smem_desc(kbuf + (ks >> 2) * 1024 + (ks & 3) * 32, 16, 2048);
+          tc_mma(tmem + COL_S + sb * 128, a, b, idesc_s, ks > 0 ? 1u : 0u);
         }
-        ASPD_STAMP(c, gg, 12);
-        tc_commit(bars + 8 * P_EMPTY);
-        tc_commit(bars + 8 * (V_EMPTY + (gg & 1)));
+        ASPD_STAMP(c, g, 9);
+        tc_commit(bars + 8 * (S_FULL + sb));
+        tc_commit(bars + 8 * (K_EMPTY + sb));
+        if (tr.last) tc_commit(bars + 8 * (Q_EMPTY + tr.qb));
         return true;
       };
-      for (int idx = item_begin; idx < item_end && ok; ++idx, ++item_no) {
-        const DeviceItem it = c.pd.items[idx];
-        const int n_tiles = (it.n_pages + 7) >> 3;
-        const int qb = item_no & 1, ob = item_no & 1;
-        if (!mbar_wait(bars + 8 * (Q_FULL + qb), (item_no >> 1) & 1, ab)) { ok = false; break; }
-        for (int t = 0; t < n_tiles; ++t, ++g) {
-          const int npg = min(8, it.n_pages - t * 8), sb = g & 1;
-          if (!mbar_wait(bars + 8 * (K_FULL + sb), (g >> 1) & 1, ab) ||
-              !mbar_wait(bars + 8 * (S_EMPTY + sb), ((g >> 1) & 1) ^ 1, ab)) { ok = false; break; }
-          tc_fence_after();
-          ASPD_STAMP(c, g, 8);
-          const uint32_t qbuf = base + OFF_Q + qb * kTileBytes, kbuf = base + OFF_K + sb * kTileBytes;
-          const uint32_t idesc_s = instr_desc((uint32_t)npg * 16u, 0);
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            // k-step ks covers head_dim elements [16 ks, 16 ks + 16): span ks / 4, 32 bytes per step
-            const uint64_t a = smem_desc(qbuf + (ks >> 2) * kHalf + (ks & 3) * 32, 16, 1024);
-            const uint64_t b = smem_desc(kbuf + (ks >> 2) * 1024 + (ks & 3) * 32, 16, 2048);
-            tc_mma(tmem + COL_S + sb * 128, a, b, idesc_s, ks > 0 ? 1u : 0u);
-          }
-          ASPD_STAMP(c, g, 9);
-          tc_commit(bars + 8 * (S_FULL + sb));
-          tc_commit(bars + 8 * (K_EMPTY + sb));
-          if (t == n_tiles - 1) tc_commit(bars + 8 * (Q_EMPTY + qb));
-          if (t > 0 && !issue_pv(g - 1, t - 1, 8, ob, item_no)) { ok = false; break; }
+      auto issue_pv = [&](const TileRef& tr, int g) -> bool {
+        ASPD_STAMP(c, g, 10);
+        if (!mbar_wait(bars + 8 * P_FULL, g & 1, ab)) return false;
+        ASPD_STAMP(c, g, 11);
+        if (!mbar_wait(bars + 8 * (V_FULL + (g & 1)), (g >> 1) & 1, ab)) return false;
+        if (tr.first && !mbar_wait(bars + 8 * (O_EMPTY + tr.ob), ((tr.item_no >> 1) & 1) ^ 1, ab)) return false;
+        tc_fence_after();
+        const uint32_t pbuf = base + OFF_P, vbuf = base + OFF_V + (g & 1) * kTileBytes;
+        for (int ks = 0; ks < tr.npg; ++ks) {
+          const uint64_t a = smem_desc(pbuf + (ks >> 2) * kHalf + (ks & 3) * 32, 16, 1024);
+          const uint64_t b = smem_desc(vbuf + ks * 4096, 1024, 2048);   // 16 keys = one page per k-step
+          tc_mma(tmem + COL_O + tr.ob * 128, a, b, idesc_pv, (!tr.first || ks > 0) ? 1u : 0u);
         }
-        if (!ok) break;
-        if (!issue_pv(g - 1, n_tiles - 1, min(8, it.n_pages - (n_tiles - 1) * 8), ob, item_no)) { ok = false; break; }
-        tc_commit(bars + 8 * (O_FULL + ob));
+        ASPD_STAMP(c, g, 12);
+        tc_commit(bars + 8 * P_EMPTY);
+        tc_commit(bars + 8 * (V_EMPTY + (g & 1)));
+        if (tr.last) tc_commit(bars + 8 * (O_FULL + tr.ob));
+        return true;
+      };
+      int g = 0, item_no = 0;
+      bool ok = true, have_prev = false;
+      TileRef prev = {0, 0, 0, 0, 0, 0};
+      for (int idx = item_begin; idx < item_end && ok; ++idx, ++item_no) {
+        const int n_pages = c.pd.items[idx].n_pages, n_tiles = (n_pages + 7) >> 3;
+        for (int t = 0; t < n_tiles && ok; ++t, ++g) {
+          const TileRef cur = {min(8, n_pages - t * 8), t == 0, t == n_tiles - 1, item_no & 1, item_no & 1, item_no};
+          ok = issue_s(cur, g);
+          if (ok && have_prev) ok = issue_pv(prev, g - 1);
+          prev = cur;
+          have_prev = true;
+        }
       }
+      if (ok && have_prev) issue_pv(prev, g - 1);
     }
     __syncwarp();
-  } else {
-    // ================================ query preparation ================================
-    int item_no = 1;
-    for (int idx = item_begin + 1; idx < item_end; ++idx, ++item_no) {
+  } else if (warp >= 8) {
+    // ===================================== epilogue =====================================
+    // One (m, l, O) record per query row of every item, written while the other warps are
+    // already working on the next item (O and the statistics are double-buffered by item).
+    const int et = tid - 256, ew = warp - 8;       // TMEM lane quadrant = warp % 4 = ew
+    const int G = c.n_q_heads / c.n_kv_heads;
+    int item_no = 0;
+    bool dead = false;
+    for (int idx = item_begin; idx < item_end; ++idx, ++item_no) {
       const DeviceItem it = c.pd.items[idx];
-      const int qb = item_no & 1;
+      const int ob = item_no & 1, M = it.n_q_tok * G, R = M <= 32 ? 32 : 64, KS = 128 / R;
+      dead |= !mbar_wait(bars + 8 * (E_FULL + ob), (item_no >> 1) & 1, ab);
+      dead |= !mbar_wait(bars + 8 * (O_FULL + ob), (item_no >> 1) & 1, ab);
+      tc_fence_after();
+      if (ew < R / 32) {
+        const int r = et;                          // row of O held by this thread's TMEM lane
+        size_t rec = 0;
+        if (r < M) {
+          const int tok = it.q_tok0 + r / G;
+          rec = (size_t)(c.pd.part_base[tok * c.n_kv_heads + it.kv_head] + it.part_slot) * G + r % G;
+          float lt = 0.f;
+          for (int jj = 0; jj < KS; ++jj) lt += misc->fin_l[ob][jj * R + r];
+          if (!dead) c.pd.ws_ml[rec] = make_float2(misc->fin_m[ob][r], lt);
+        }
+        const uint32_t o_addr = tmem + ((uint32_t)(ew * 32) << 16) + COL_O + ob * 128;
+#pragma unroll 1
+        for (int q4 = 0; q4 < 4; ++q4) {
+          float o[32];
+          ASPD_TMEM_LD32(o_addr + q4 * 32, o, 0);
+          tmem_wait_ld();
+          if (r < M && !dead) {
+            float4* dst = reinterpret_cast<float4*>(c.pd.ws_o + rec * 128 + q4 * 32);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(bars + 8 * (O_EMPTY + ob));
+      if (named_sync_or(2, 128, dead || *ab)) break;
+    }
+    if (et == 0) ASPD_CTA_STAMP(c, 2);
+  } else {
+    // =================================== query loader ===================================
+    // The rotated rows of the item's (row block, KV head) come from the pre-pass image; they
+    // are replicated KS = 128 / R times down the 128 rows of the A operand.
+    int item_no = 0;
+    const int G = c.n_q_heads / c.n_kv_heads;
+    for (int idx = item_begin; idx < item_end; ++idx, ++item_no) {
+      const DeviceItem it = c.pd.items[idx];
+      const int qb = item_no & 1, R = it.n_q_tok * G <= 32 ? 32 : 64, KS = 128 / R;
       int good = 1;
       if (lane == 0) good = mbar_wait(bars + 8 * (Q_EMPTY + qb), ((item_no >> 1) & 1) ^ 1, ab) ? 1 : 0;
       good = __shfl_sync(0xffffffffu, good, 0);
       if (!good) break;
-      prep_q(c, it, base + OFF_Q + qb * kTileBytes, lane, 32);
-      fence_async_smem();
-      mbar_arrive(bars + 8 * (Q_FULL + qb));
+      const uint32_t full = bars + 8 * (Q_FULL + qb);
+      if (lane == 0) mbar_expect_tx(full, kTileBytes);
+      __syncwarp();
+      if (lane < 2 * KS) {
+        const int span = lane & 1, rep = lane >> 1;
+        const char* img = c.pd.q_img + ((size_t)it.row_block * c.n_kv_heads + it.kv_head) * kQImageBytes;
+        bulk_copy(base + OFF_Q + qb * kTileBytes + span * kHalf + rep * R * 128, img + span * R * 128, R * 128, full);
+      }
     }
   }
 
@@ -532,6 +566,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   }
   tc_fence_before();
   __syncthreads();
+  if (tid == 0) ASPD_CTA_STAMP(c, 3);
   if (warp == 0) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
@@ -539,6 +574,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
 }
 
 }  // namespace
+
+int launch_q_rotate(const aspd_plan* p, const void* q, cudaStream_t s) {
+  if (p->n_row_blocks == 0) return ASPD_OK;
+  q_rotate_kernel<<<p->n_row_blocks * p->shape.n_kv_heads, 128, 0, s>>>(p->dev, (const __nv_bfloat16*)q, p->shape.n_q_heads,
+                                                                        p->shape.n_kv_heads);
+  return cudaGetLastError() == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
+}
 
 int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, cudaStream_t s) {
   if (p->n_items == 0) return ASPD_OK;

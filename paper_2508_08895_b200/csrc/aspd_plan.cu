@@ -292,17 +292,20 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   // ---- work items: a contiguous, equal share of all pages for every CTA -----------------
   // Streams are walked in the order (request, row block, KV head); the concatenation of all
   // streams is cut at the CTA boundaries (and, if asked for, every chunk_tokens keys).
-  struct Stream { int request, tok0, n_tok, head, page0, n_pages; };
+  struct Stream { int request, tok0, n_tok, head, page0, n_pages, row_block; };
+  std::vector<int2> row_blocks;
   std::vector<Stream> streams;
   long total_pages = 0;
   for (int r = 0; r < n_req; ++r) {
     const int nt = req_tok0[r + 1] - req_tok0[r], np = visit0[r + 1] - visit0[r];
     if (nt == 0 || np == 0) continue;
-    for (int i0 = 0; i0 < nt; i0 += max_tok)
+    for (int i0 = 0; i0 < nt; i0 += max_tok) {
+      row_blocks.push_back(make_int2(req_tok0[r] + i0, std::min(max_tok, nt - i0)));
       for (int h = 0; h < Hkv; ++h) {
-        streams.push_back({r, req_tok0[r] + i0, std::min(max_tok, nt - i0), h, visit0[r], np});
+        streams.push_back({r, req_tok0[r] + i0, std::min(max_tok, nt - i0), h, visit0[r], np, (int)row_blocks.size() - 1});
         total_pages += np;
       }
+    }
   }
   const int min_pages = 4;                       // do not cut finer than 64 keys per CTA
   int n_ctas = tune.n_ctas > 0 ? tune.n_ctas : p->sm_count;
@@ -323,6 +326,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
         DeviceItem it;
         it.q_tok0 = st.tok0; it.n_q_tok = st.n_tok; it.kv_head = st.head; it.page0 = st.page0 + at;
         it.n_pages = (int)stop - at; it.key0 = at * ps; it.part_slot = slot++; it.request = st.request;
+        it.row_block = st.row_block; it.reserved = 0;
         p->items.push_back(it);
         at = (int)stop;
       }
@@ -337,6 +341,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   p->kv_tokens_read = kv_tokens;
   p->algorithmic_bytes = 2LL * Hkv * d * es * kv_tokens + 2LL * es * Hq * d * n_new + 2LL * Hkv * d * es * n_new;
   p->visit = visit;
+  p->n_row_blocks = (int)row_blocks.size();
   p->tok_vis = tok_vis;
   if (tune.host_only) { *plan_out = p; return ASPD_OK; }
 
@@ -349,12 +354,14 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   const size_t o_tpage = take(sizeof(int32_t) * std::max(1, n_new));
   const size_t o_trow = take(sizeof(int32_t) * std::max(1, n_new));
   const size_t o_tvis = take(sizeof(int4) * std::max(1, n_new));
+  const size_t o_rb = take(sizeof(int2) * std::max<size_t>(1, row_blocks.size()));
   const size_t o_qcs = take(sizeof(float2) * std::max(1, n_new) * (d / 2));
   const size_t o_pbase = take(sizeof(int32_t) * part_base.size());
   const size_t o_freq = take(sizeof(double) * (d / 2));
   const size_t o_status = take(sizeof(int32_t) * 2);
   const size_t upload_bytes = off;
   const size_t o_wso = take(sizeof(float) * (size_t)std::max(1, p->n_partials) * G * d);
+  const size_t o_qimg = take((size_t)kQImageBytes * std::max<size_t>(1, row_blocks.size()) * Hkv);
   const size_t o_wsml = take(sizeof(float2) * (size_t)std::max(1, p->n_partials) * G);
   const size_t o_stq = take((size_t)es * std::max(1, n_new) * Hq * d);
   const size_t o_stk = take((size_t)es * std::max(1, n_new) * Hkv * d);
@@ -372,6 +379,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
     memcpy(blob.data() + o_trow, tok_row.data(), sizeof(int32_t) * n_new);
     memcpy(blob.data() + o_tvis, tok_vis.data(), sizeof(int4) * n_new);
   }
+  if (!row_blocks.empty()) memcpy(blob.data() + o_rb, row_blocks.data(), sizeof(int2) * row_blocks.size());
   memcpy(blob.data() + o_pbase, part_base.data(), sizeof(int32_t) * part_base.size());
   double* freq = reinterpret_cast<double*>(blob.data() + o_freq);
   for (int i = 0; i < d / 2; ++i) freq[i] = pow((double)shape->rope_theta, -2.0 * i / d);
@@ -395,6 +403,8 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   p->dev.cta_item0 = (const int32_t*)(b8 + o_cta);
   p->dev.visit = (const int2*)(b8 + o_visit);
   p->dev.tok_vis = (const int4*)(b8 + o_tvis);
+  p->dev.row_blocks = (const int2*)(b8 + o_rb);
+  p->dev.q_img = (char*)(b8 + o_qimg);
   p->dev.tok_page = (const int32_t*)(b8 + o_tpage);
   p->dev.tok_row = (const int32_t*)(b8 + o_trow);
   p->dev.q_cs = (const float2*)(b8 + o_qcs);
@@ -430,7 +440,7 @@ int aspd_plan_info(const aspd_plan_t* p, aspd_plan_info_t* info) {
 int aspd_plan_items(const aspd_plan_t* p, aspd_item_t* items, int max_items) {
   if (!p || (max_items > 0 && !items) || max_items < 0) return ASPD_ERR_INVALID_ARG;
   int n = std::min(max_items, p->n_items);
-  static_assert(sizeof(aspd_item_t) == sizeof(DeviceItem), "item layouts must match");
+  static_assert(sizeof(aspd_item_t) == sizeof(DeviceItem) && sizeof(DeviceItem) == 40, "item layouts must match");
   if (n) memcpy(items, p->items.data(), sizeof(DeviceItem) * n);
   return p->n_items;
 }
@@ -471,8 +481,10 @@ int aspd_attn_partials(aspd_plan_t* p, const void* q, const void* k_pool, const 
   if (p->n_new == 0) return ASPD_OK;
   if (!q || !k_pool || !v_pool) return ASPD_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
-  return p->kernel == ASPD_KERNEL_MMA ? launch_attn_mma(p, q, k_pool, v_pool, s)
-                                      : launch_attn_generic(p, q, k_pool, v_pool, s);
+  if (p->kernel != ASPD_KERNEL_MMA) return launch_attn_generic(p, q, k_pool, v_pool, s);
+  int rc = launch_q_rotate(p, q, s);
+  if (rc) return rc;
+  return launch_attn_mma(p, q, k_pool, v_pool, s);
 }
 
 int aspd_attn_combine(aspd_plan_t* p, void* out, void* stream) {

@@ -29,7 +29,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_struct_sizes_and_strerror():
-    assert B.REQUEST_DTYPE.itemsize == 28 and B.BRANCH_DTYPE.itemsize == 16 and B.ITEM_DTYPE.itemsize == 32
+    assert B.REQUEST_DTYPE.itemsize == 28 and B.BRANCH_DTYPE.itemsize == 16 and B.ITEM_DTYPE.itemsize == 40
     assert ctypes.sizeof(B.Shape) == 28
     assert B.strerror(0) == "ok"
     for code in range(-7, 0):
