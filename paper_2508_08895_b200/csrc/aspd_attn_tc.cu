@@ -305,41 +305,49 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
   return !named_sync_or(1, 128, dead || *ab);
 }
 
-// Pre-pass: rotate the query rows of every (row block, KV head) (RoPE at the token's position,
-// table from the plan), round to bf16 and store them as the image of the A operand:
-// [2 spans][R rows][128 B], 16-byte chunks XOR-ed with (row & 7), R = 32 or 64, rows >= M zero.
-// The main kernel then brings a query tile in with a few linear bulk copies.
-__global__ void __launch_bounds__(128) q_rotate_kernel(PlanDevice pd, const __nv_bfloat16* __restrict__ q, int n_q_heads,
-                                                       int n_kv_heads) {
-  const int rb = blockIdx.x / n_kv_heads, head = blockIdx.x % n_kv_heads;
-  const int2 blk = pd.row_blocks[rb];
-  const int G = n_q_heads / n_kv_heads, M = blk.y * G, R = M <= 32 ? 32 : 64;
-  char* img = pd.q_img + (size_t)blockIdx.x * kQImageBytes;
-  for (int e = threadIdx.x; e < R * 8; e += 128) {
-    const int r = e >> 3, ch = e & 7;            // row, 8-element chunk of each span
-    uint4 lo = make_uint4(0, 0, 0, 0), hi = make_uint4(0, 0, 0, 0);
-    if (r < M) {
-      const int tok = blk.x + r / G, hq = head * G + r % G;
-      const __nv_bfloat16* qrow = q + ((size_t)tok * n_q_heads + hq) * 128;
-      const uint4 a = *reinterpret_cast<const uint4*>(qrow + ch * 8);
-      const uint4 b = *reinterpret_cast<const uint4*>(qrow + 64 + ch * 8);
-      const float4* cs = reinterpret_cast<const float4*>(pd.q_cs + (size_t)tok * 64 + ch * 8);
-      const float4 w[4] = {cs[0], cs[1], cs[2], cs[3]};   // (cos, sin) of elements 2i and 2i+1 of the chunk
-      const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&a);
-      const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&b);
-      uint32_t l4[4], h4[4];
+// Rotate the item's query rows (RoPE at the token's position, cos/sin table from the plan),
+// round to bf16 and store them, replicated KS = 128 / R times, as the 128-byte-swizzled K-major
+// A operand.  Called by the 128 epilogue threads (rank 0..127); all loads of a thread's rows
+// are issued before the first use.
+__device__ __forceinline__ void prep_q(const Ctx& c, const DeviceItem& it, uint32_t qbuf, int rank) {
+  const int G = c.n_q_heads / c.n_kv_heads;
+  const int M = it.n_q_tok * G, R = M <= 32 ? 32 : 64, KS = 128 / R;
+  uint4 a[4], b[4];
+  float4 w[4][4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float2 x0 = __bfloat1622float2(a2[i]), x1 = __bfloat1622float2(b2[i]);
-        l4[i] = pack_bf16(x0.x * w[i].x - x1.x * w[i].y, x0.y * w[i].z - x1.y * w[i].w);
-        h4[i] = pack_bf16(x1.x * w[i].x + x0.x * w[i].y, x1.y * w[i].z + x0.y * w[i].w);
-      }
-      lo = make_uint4(l4[0], l4[1], l4[2], l4[3]);
-      hi = make_uint4(h4[0], h4[1], h4[2], h4[3]);
+  for (int u = 0; u < 4; ++u) {
+    const int e = rank + u * 128, r = e >> 3, ch = e & 7;     // row, 8-element chunk of each span
+    a[u] = make_uint4(0, 0, 0, 0); b[u] = make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) w[u][i] = make_float4(1.f, 0.f, 1.f, 0.f);
+    if (e < R * 8 && r < M) {
+      const int tok = it.q_tok0 + r / G, hq = it.kv_head * G + r % G;
+      const __nv_bfloat16* qrow = c.q + ((size_t)tok * c.n_q_heads + hq) * 128;
+      a[u] = *reinterpret_cast<const uint4*>(qrow + ch * 8);
+      b[u] = *reinterpret_cast<const uint4*>(qrow + 64 + ch * 8);
+      const float4* cs = reinterpret_cast<const float4*>(c.pd.q_cs + (size_t)tok * 64 + ch * 8);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) w[u][i] = cs[i];              // (cos, sin) of elements 2i and 2i+1 of the chunk
     }
-    const uint32_t off = r * 128 + ((ch ^ (r & 7)) << 4);
-    *reinterpret_cast<uint4*>(img + off) = lo;
-    *reinterpret_cast<uint4*>(img + R * 128 + off) = hi;
+  }
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const int e = rank + u * 128, r = e >> 3, ch = e & 7;
+    if (e >= R * 8) break;
+    const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&a[u]);
+    const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&b[u]);
+    uint32_t lo[4], hi[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 x0 = __bfloat1622float2(a2[i]), x1 = __bfloat1622float2(b2[i]);
+      lo[i] = pack_bf16(x0.x * w[u][i].x - x1.x * w[u][i].y, x0.y * w[u][i].z - x1.y * w[u][i].w);
+      hi[i] = pack_bf16(x1.x * w[u][i].x + x0.x * w[u][i].y, x1.y * w[u][i].z + x0.y * w[u][i].w);
+    }
+    for (int jj = 0; jj < KS; ++jj) {
+      const uint32_t addr = qbuf + (jj * R + r) * 128 + ((ch ^ (r & 7)) << 4);
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr + kHalf), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
+    }
   }
 }
 
@@ -357,7 +365,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   const int item_begin = c.pd.cta_item0[blockIdx.x], item_end = c.pd.cta_item0[blockIdx.x + 1];
 
   if (tid == 0) {
-    const int counts[NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, 128, 128, 128, 1, 1, 1, 128, 128, 1, 1, 1, 1, 128, 128};
+    const int counts[NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, 128, 128, 128, 1, 1, 1, 128, 128, 128, 128, 1, 1, 128, 128};
     for (int i = 0; i < NUM_BARS; ++i) mbar_init(bars + 8 * i, counts[i]);
     misc->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -500,9 +508,21 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     const int G = c.n_q_heads / c.n_kv_heads;
     int item_no = 0;
     bool dead = false;
+    if (item_begin < item_end) {                   // the first query tile, while the first K/V tiles are in flight
+      prep_q(c, c.pd.items[item_begin], base + OFF_Q, et);
+      fence_async_smem();
+      mbar_arrive(bars + 8 * Q_FULL);
+    }
     for (int idx = item_begin; idx < item_end; ++idx, ++item_no) {
       const DeviceItem it = c.pd.items[idx];
       const int ob = item_no & 1, M = it.n_q_tok * G, R = M <= 32 ? 32 : 64, KS = 128 / R;
+      if (idx + 1 < item_end) {                    // the next item's query tile, into the other buffer
+        const int qn = (item_no + 1) & 1;
+        dead |= !mbar_wait(bars + 8 * (Q_EMPTY + qn), (((item_no + 1) >> 1) & 1) ^ 1, ab);
+        prep_q(c, c.pd.items[idx + 1], base + OFF_Q + qn * kTileBytes, et);
+        fence_async_smem();
+        mbar_arrive(bars + 8 * (Q_FULL + qn));
+      }
       dead |= !mbar_wait(bars + 8 * (E_FULL + ob), (item_no >> 1) & 1, ab);
       dead |= !mbar_wait(bars + 8 * (O_FULL + ob), (item_no >> 1) & 1, ab);
       tc_fence_after();
@@ -534,28 +554,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
       if (named_sync_or(2, 128, dead || *ab)) break;
     }
     if (et == 0) ASPD_CTA_STAMP(c, 2);
-  } else {
-    // =================================== query loader ===================================
-    // The rotated rows of the item's (row block, KV head) come from the pre-pass image; they
-    // are replicated KS = 128 / R times down the 128 rows of the A operand.
-    int item_no = 0;
-    const int G = c.n_q_heads / c.n_kv_heads;
-    for (int idx = item_begin; idx < item_end; ++idx, ++item_no) {
-      const DeviceItem it = c.pd.items[idx];
-      const int qb = item_no & 1, R = it.n_q_tok * G <= 32 ? 32 : 64, KS = 128 / R;
-      int good = 1;
-      if (lane == 0) good = mbar_wait(bars + 8 * (Q_EMPTY + qb), ((item_no >> 1) & 1) ^ 1, ab) ? 1 : 0;
-      good = __shfl_sync(0xffffffffu, good, 0);
-      if (!good) break;
-      const uint32_t full = bars + 8 * (Q_FULL + qb);
-      if (lane == 0) mbar_expect_tx(full, kTileBytes);
-      __syncwarp();
-      if (lane < 2 * KS) {
-        const int span = lane & 1, rep = lane >> 1;
-        const char* img = c.pd.q_img + ((size_t)it.row_block * c.n_kv_heads + it.kv_head) * kQImageBytes;
-        bulk_copy(base + OFF_Q + qb * kTileBytes + span * kHalf + rep * R * 128, img + span * R * 128, R * 128, full);
-      }
-    }
   }
 
   // ---- drain: on a time-out give outstanding copies and MMAs time to land before the CTA's
@@ -574,13 +572,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
 }
 
 }  // namespace
-
-int launch_q_rotate(const aspd_plan* p, const void* q, cudaStream_t s) {
-  if (p->n_row_blocks == 0) return ASPD_OK;
-  q_rotate_kernel<<<p->n_row_blocks * p->shape.n_kv_heads, 128, 0, s>>>(p->dev, (const __nv_bfloat16*)q, p->shape.n_q_heads,
-                                                                        p->shape.n_kv_heads);
-  return cudaGetLastError() == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
-}
 
 int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, cudaStream_t s) {
   if (p->n_items == 0) return ASPD_OK;

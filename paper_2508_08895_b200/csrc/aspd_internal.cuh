@@ -37,7 +37,6 @@ __host__ __device__ inline uint32_t tile_offset(int t, uint32_t b, uint32_t row_
 struct DeviceItem {       // mirrors aspd_item_t, 40 bytes
   int32_t q_tok0, n_q_tok, kv_head, page0, n_pages, key0, part_slot, request, row_block, reserved;
 };
-constexpr int kQImageBytes = 16384;   // rotated query rows of one (row block, KV head): [2 spans][<= 64 rows][128 B]
 
 struct PlanDevice {       // pointers into the plan's single device allocation
   const DeviceItem* items;
@@ -45,7 +44,6 @@ struct PlanDevice {       // pointers into the plan's single device allocation
   const int2* visit;           // key streams: (physical page, valid rows) per page to read
   const int4* tok_vis;         // [n_new] (pe, lo, hi, -): visible stream keys are [0, pe) and [lo, hi)
   const int2* row_blocks;      // [n_row_blocks] (first new token, number of tokens)
-  char* q_img;                 // [n_row_blocks][n_kv_heads][kQImageBytes] rotated bf16 queries, operand layout
   const int32_t* tok_page;     // [n_new] physical page the new token's K/V goes to
   const int32_t* tok_row;      // [n_new] row inside that page
   const float2* q_cs;          // [n_new][head_dim/2] (cos, sin) of the query's RoPE angle
@@ -94,7 +92,6 @@ int launch_attn_generic(const aspd_plan* p, const void* q, const void* k_pool, c
 int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool,
                     cudaStream_t s);
 int launch_combine(const aspd_plan* p, void* out, cudaStream_t s);
-int launch_q_rotate(const aspd_plan* p, const void* q, cudaStream_t s);
 int launch_read_token(const aspd_shape_t* shape, const void* pool, int64_t page, int row, int kv_head,
                       float* out_dev, cudaStream_t s);
 inline int esize_of(int dtype) { return dtype == ASPD_DTYPE_BF16 ? 2 : 4; }

@@ -160,18 +160,26 @@ __global__ void combine_kernel(PlanDevice pd, T* __restrict__ out, int n_new, in
       if (ml.y > 0.f) { wt = exp2f(ml.x - M); L += ml.y * wt; }     // records of chunks with no visible key have sum 0
     }
     const int cnt = min(32, n - base);
-#pragma unroll 4
-    for (int i = 0; i < cnt; ++i) {
-      const float wi = __shfl_sync(0xffffffffu, wt, i);
-      const float* row = pd.ws_o + ((size_t)(p0 + base + i) * G + g) * D + lane * EPL;
-      if (wi != 0.f) {
+    for (int i0 = 0; i0 < cnt; i0 += 8) {        // eight independent row loads in flight per lane
+      float v[8][EPL];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int i = min(i0 + u, cnt - 1);
+        const float* row = pd.ws_o + ((size_t)(p0 + base + i) * G + g) * D + lane * EPL;
         if constexpr (EPL == 4) {
-          const float4 v = *reinterpret_cast<const float4*>(row);
-          acc[0] = fmaf(v.x, wi, acc[0]); acc[1] = fmaf(v.y, wi, acc[1]); acc[2] = fmaf(v.z, wi, acc[2]); acc[3] = fmaf(v.w, wi, acc[3]);
+          const float4 x = *reinterpret_cast<const float4*>(row);
+          v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
         } else {
-          const float2 v = *reinterpret_cast<const float2*>(row);
-          acc[0] = fmaf(v.x, wi, acc[0]); acc[1] = fmaf(v.y, wi, acc[1]);
+          const float2 x = *reinterpret_cast<const float2*>(row);
+          v[u][0] = x.x; v[u][1] = x.y;
         }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        float wi = __shfl_sync(0xffffffffu, wt, min(i0 + u, cnt - 1));
+        if (i0 + u >= cnt) wi = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc[e] += wi != 0.f ? v[u][e] * wi : 0.f;   // a skipped record may hold anything
       }
     }
   }

@@ -361,7 +361,6 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   const size_t o_status = take(sizeof(int32_t) * 2);
   const size_t upload_bytes = off;
   const size_t o_wso = take(sizeof(float) * (size_t)std::max(1, p->n_partials) * G * d);
-  const size_t o_qimg = take((size_t)kQImageBytes * std::max<size_t>(1, row_blocks.size()) * Hkv);
   const size_t o_wsml = take(sizeof(float2) * (size_t)std::max(1, p->n_partials) * G);
   const size_t o_stq = take((size_t)es * std::max(1, n_new) * Hq * d);
   const size_t o_stk = take((size_t)es * std::max(1, n_new) * Hkv * d);
@@ -404,7 +403,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   p->dev.visit = (const int2*)(b8 + o_visit);
   p->dev.tok_vis = (const int4*)(b8 + o_tvis);
   p->dev.row_blocks = (const int2*)(b8 + o_rb);
-  p->dev.q_img = (char*)(b8 + o_qimg);
+
   p->dev.tok_page = (const int32_t*)(b8 + o_tpage);
   p->dev.tok_row = (const int32_t*)(b8 + o_trow);
   p->dev.q_cs = (const float2*)(b8 + o_qcs);
@@ -481,10 +480,8 @@ int aspd_attn_partials(aspd_plan_t* p, const void* q, const void* k_pool, const 
   if (p->n_new == 0) return ASPD_OK;
   if (!q || !k_pool || !v_pool) return ASPD_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
-  if (p->kernel != ASPD_KERNEL_MMA) return launch_attn_generic(p, q, k_pool, v_pool, s);
-  int rc = launch_q_rotate(p, q, s);
-  if (rc) return rc;
-  return launch_attn_mma(p, q, k_pool, v_pool, s);
+  return p->kernel == ASPD_KERNEL_MMA ? launch_attn_mma(p, q, k_pool, v_pool, s)
+                                      : launch_attn_generic(p, q, k_pool, v_pool, s);
 }
 
 int aspd_attn_combine(aspd_plan_t* p, void* out, void* stream) {
