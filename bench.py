@@ -79,7 +79,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -156,6 +156,19 @@ def run_reference(args):
     }
     print(json.dumps(line))
     return 0
+
+
+def reduce_over_ranks(times_ms, units, device, world):
+    """Whole-job figures from per-rank ones: every time becomes its maximum over the ranks, the
+    units (query tokens a rank processed) their sum.  A no-op for one rank."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(x) for x in times_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([float(units)], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return [float(x) for x in t.tolist()], float(u.item())
 
 
 # ------------------------------------------------------------------------------ our arm
@@ -259,7 +272,7 @@ def run_ours(args):
     run_partials()
     torch.cuda.synchronize()
     k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    reps = max(3, args.steps)
+    reps = max(3, min(args.steps, 50))
     k0.record(stream)
     for _ in range(reps):
         run_partials()
@@ -281,7 +294,7 @@ def run_ours(args):
     for _ in range(2):
         step_e2e()
     barrier()
-    e_steps = max(1, min(args.steps, 5))
+    e_steps = max(1, min(args.steps, 10))
     t0 = time.perf_counter()
     for _ in range(e_steps):
         step_e2e()
@@ -289,13 +302,7 @@ def run_ours(args):
     e2e_ms = (time.perf_counter() - t0) * 1e3
 
     # max over ranks, on the device-side times
-    times = torch.tensor([ms, e2e_ms, kernel_ms], dtype=torch.float64, device="cuda")
-    toks = torch.tensor([float(n_new)], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-        dist.all_reduce(toks, op=dist.ReduceOp.SUM)
-    ms, e2e_ms, kernel_ms = (float(x) for x in times.tolist())
-    total_new = float(toks.item())
+    (ms, e2e_ms, kernel_ms), total_new = reduce_over_ranks([ms, e2e_ms, kernel_ms], n_new, "cuda", world)
 
     # parity of layer 0 against the oracle is the tests' business; here only a sanity check that
     # the layers agree with each other (same inputs, distinct pools)
@@ -344,7 +351,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="serving-mix", choices=["qwen7b-layer", "branch-open", "long-rag", "serving-mix"])
