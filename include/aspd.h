@@ -232,6 +232,35 @@ int aspd_step_host(aspd_plan_t* plan, const void* q /*host*/, const void* k_new 
                    const void* v_new /*host*/, const int32_t* pos /*host*/, void* k_pool /*device*/,
                    void* v_pool /*device*/, void* out /*host*/, void* stream);
 
+/*
+ * Attention of a step for callers that must not allocate device memory (the paper has no
+ * counterpart; this is a convenience of the library).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a memory pool that owns
+ * the whole device, in a latency-critical serving loop whose allocator may not be re-entered,
+ * or in a process that was handed a fixed memory budget -- and therefore cannot create a
+ * device plan with aspd_plan_create, which allocates the plan's tables and split-K workspace.
+ *
+ * `plan` is a HOST-ONLY plan (aspd_tuning_t.host_only = 1; building it makes no CUDA call).
+ * The call copies the plan's tables into a scratch array that is compiled into the library
+ * (a file-scope __device__ array of ASPD_STATIC_SCRATCH_BYTES bytes; every GPU that loads the
+ * library holds that much memory until the process exits), runs the same split-K pass and
+ * combine as aspd_branch_attn / aspd_serial_attn (by the plan's mode) with all scratch inside
+ * that array, and writes `out`.  It calls no cudaMalloc / cudaFree and no allocating library
+ * routine.  q, k_pool, v_pool, out are device buffers as for aspd_branch_attn.
+ *
+ *  - Plans whose tables plus workspace exceed ASPD_STATIC_SCRATCH_BYTES are rejected with
+ *    ASPD_ERR_TOO_LARGE before anything is launched.
+ *  - The first call on a device looks the array's device address up (once per device, with
+ *    that device current); make that first call outside any stream capture.
+ *  - All calls share the one array, which keeps the previous call's contents; every call
+ *    rewrites the tables and the status word it needs.  Two calls that overlap on the GPU
+ *    (different streams, or different host threads) race on it: serialise them.
+ */
+#define ASPD_STATIC_SCRATCH_BYTES (8u << 20)
+int aspd_attn_static(const aspd_plan_t* plan /*host-only*/, const void* q /*device*/, const void* k_pool /*device*/,
+                     const void* v_pool /*device*/, void* out /*device*/, void* stream);
+
 /* Read one cached token (physical page, row, KV head) back as head_dim floats (host).
  * Synchronises `stream`.  For tests. */
 int aspd_debug_read_token(const aspd_shape_t* shape, const void* pool /*device*/, int64_t page,

@@ -57,7 +57,7 @@ EXPORTS = ("aspd_strerror", "aspd_pool_bytes", "aspd_count_new_tokens", "aspd_po
            "aspd_plan_create", "aspd_plan_destroy", "aspd_plan_info", "aspd_plan_items", "aspd_plan_stream_pages",
            "aspd_plan_token_ranges", "aspd_plan_status",
            "aspd_kv_append", "aspd_branch_attn", "aspd_serial_attn", "aspd_attn_partials", "aspd_attn_combine",
-           "aspd_step_host", "aspd_debug_read_token")
+           "aspd_step_host", "aspd_attn_static", "aspd_debug_read_token")
 
 _lib = None
 
@@ -94,6 +94,7 @@ def lib() -> ctypes.CDLL:
         L.aspd_attn_partials.argtypes = [vp] * 5
         L.aspd_attn_combine.argtypes = [vp] * 3
         L.aspd_step_host.argtypes = [vp] * 9
+        L.aspd_attn_static.argtypes = [vp] * 6
         L.aspd_debug_read_token.argtypes = [vp, vp, ctypes.c_int64, ci, ci, vp, vp]
         for name in EXPORTS:
             if name not in ("aspd_strerror", "aspd_pool_bytes"):
@@ -261,6 +262,17 @@ def step_host(plan: Plan, q, k_new, v_new, pos, k_pool, v_pool, out, stream=None
     """Whole step from host (numpy / pinned torch CPU) buffers; ``out`` is a host buffer."""
     _check(lib().aspd_step_host(plan._h, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(pos), _ptr(k_pool), _ptr(v_pool),
                                 _ptr(out), _stream(stream)), "aspd_step_host")
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def attn_static(plan: Plan, q, k_pool, v_pool, out, stream=None) -> None:
+    """Attention of a step for callers that cannot allocate device memory: ``plan`` is a
+    host-only plan and all scratch lives in an array compiled into the library (see
+    ``aspd_attn_static`` in ``aspd.h`` for the size limit and the sharing rules)."""
+    _check(lib().aspd_attn_static(plan._h, _ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(out), _stream(stream)),
+           "aspd_attn_static")
 
 
 def debug_read_token(shape: Shape, pool, page: int, row: int, kv_head: int, stream=None) -> np.ndarray:

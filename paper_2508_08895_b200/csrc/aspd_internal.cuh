@@ -81,6 +81,9 @@ struct aspd_plan {
   std::vector<aspd::DeviceItem> items;
   std::vector<int2> visit;
   std::vector<int4> tok_vis;
+  // further host copies of the plan's tables (what the device allocation is filled from)
+  std::vector<int32_t> cta_item0, part_base, q_pos;
+  std::vector<int2> row_blocks;
 };
 
 namespace aspd {

@@ -342,6 +342,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   p->algorithmic_bytes = 2LL * Hkv * d * es * kv_tokens + 2LL * es * Hq * d * n_new + 2LL * Hkv * d * es * n_new;
   p->visit = visit;
   p->n_row_blocks = (int)row_blocks.size();
+  p->cta_item0 = cta_item0; p->part_base = part_base; p->row_blocks = row_blocks; p->q_pos = pos;
   p->tok_vis = tok_vis;
   if (tune.host_only) { *plan_out = p; return ASPD_OK; }
 

@@ -1,0 +1,109 @@
+// aspd_attn_static: the attention of a step with every byte of scratch in a device array that
+// is part of the library image, for callers that cannot allocate device memory.
+#include <string.h>
+
+#include <vector>
+
+#include "aspd_internal.cuh"
+
+using namespace aspd;
+
+namespace {
+
+// The scratch.  In host code `g_scratch` is only a handle for the symbol, not a device address;
+// the address a kernel may use comes from cudaGetSymbolAddress (below).
+static __device__ __align__(256) unsigned char g_scratch[ASPD_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+unsigned char* g_scratch_addr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device (looked up once per device).
+int scratch_address(unsigned char** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ASPD_ERR_CUDA;
+  if (!g_scratch_addr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_scratch) != cudaSuccess || !ptr) return ASPD_ERR_CUDA;
+    g_scratch_addr[dev] = static_cast<unsigned char*>(ptr);
+  }
+  *out = g_scratch_addr[dev];
+  return ASPD_OK;
+}
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+extern "C" int aspd_attn_static(const aspd_plan_t* plan, const void* q, const void* k_pool, const void* v_pool, void* out,
+                                void* stream) {
+  if (!plan || !plan->host_only) return ASPD_ERR_INVALID_ARG;
+  if (plan->n_new == 0) return ASPD_OK;
+  if (!q || !k_pool || !v_pool || !out) return ASPD_ERR_INVALID_ARG;
+  const aspd_shape_t& sh = plan->shape;
+  const int d = sh.head_dim, G = sh.n_q_heads / sh.n_kv_heads, n_new = plan->n_new;
+
+  // layout of the tables and of the split-K workspace inside the scratch array
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t o_items = take(sizeof(DeviceItem) * plan->items.size());
+  const size_t o_cta = take(sizeof(int32_t) * plan->cta_item0.size());
+  const size_t o_visit = take(sizeof(int2) * plan->visit.size());
+  const size_t o_tvis = take(sizeof(int4) * plan->tok_vis.size());
+  const size_t o_rb = take(sizeof(int2) * plan->row_blocks.size());
+  const size_t o_qcs = take(sizeof(float2) * (size_t)n_new * (d / 2));
+  const size_t o_pbase = take(sizeof(int32_t) * plan->part_base.size());
+  const size_t o_status = take(sizeof(int32_t) * 2);
+  const size_t upload_bytes = off;
+  const size_t o_wso = take(sizeof(float) * (size_t)plan->n_partials * G * d);
+  const size_t o_wsml = take(sizeof(float2) * (size_t)plan->n_partials * G);
+  if (off > ASPD_STATIC_SCRATCH_BYTES) return ASPD_ERR_TOO_LARGE;
+
+  unsigned char* base = nullptr;
+  int rc = scratch_address(&base);
+  if (rc) return rc;
+
+  // tables: everything that must start from a known value is rewritten here (the status word
+  // and the work counter start at zero; the workspace is fully written before it is read)
+  std::vector<uint8_t> blob(upload_bytes, 0);
+  memcpy(blob.data() + o_items, plan->items.data(), sizeof(DeviceItem) * plan->items.size());
+  memcpy(blob.data() + o_cta, plan->cta_item0.data(), sizeof(int32_t) * plan->cta_item0.size());
+  memcpy(blob.data() + o_visit, plan->visit.data(), sizeof(int2) * plan->visit.size());
+  memcpy(blob.data() + o_tvis, plan->tok_vis.data(), sizeof(int4) * plan->tok_vis.size());
+  memcpy(blob.data() + o_rb, plan->row_blocks.data(), sizeof(int2) * plan->row_blocks.size());
+  memcpy(blob.data() + o_pbase, plan->part_base.data(), sizeof(int32_t) * plan->part_base.size());
+  float2* qcs = reinterpret_cast<float2*>(blob.data() + o_qcs);
+  for (int t = 0; t < n_new; ++t)
+    for (int i = 0; i < d / 2; ++i) {
+      const double a = (double)plan->q_pos[t] * pow((double)sh.rope_theta, -2.0 * i / d);
+      qcs[(size_t)t * (d / 2) + i] = make_float2((float)cos(a), (float)sin(a));
+    }
+  cudaStream_t s = (cudaStream_t)stream;
+  // the source is pageable host memory: the copy is staged before the call returns
+  if (cudaMemcpyAsync(base, blob.data(), upload_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return ASPD_ERR_CUDA;
+
+  // a shell of the plan whose device pointers all lie inside the scratch array
+  aspd_plan shell;
+  shell.shape = plan->shape; shell.mode = plan->mode; shell.n_req = plan->n_req; shell.n_new = plan->n_new;
+  shell.n_items = plan->n_items; shell.n_partials = plan->n_partials; shell.kernel = plan->kernel;
+  shell.chunk_tokens = plan->chunk_tokens; shell.n_ctas = plan->n_ctas; shell.host_only = 0;
+  shell.sm_count = plan->sm_count; shell.n_row_blocks = plan->n_row_blocks; shell.n_pool_pages = plan->n_pool_pages;
+  shell.kv_tokens_read = plan->kv_tokens_read; shell.algorithmic_bytes = plan->algorithmic_bytes;
+  shell.device_bytes = 0; shell.device_base = nullptr;
+  memset(&shell.dev, 0, sizeof(shell.dev));
+  shell.dev.items = (const DeviceItem*)(base + o_items);
+  shell.dev.cta_item0 = (const int32_t*)(base + o_cta);
+  shell.dev.visit = (const int2*)(base + o_visit);
+  shell.dev.tok_vis = (const int4*)(base + o_tvis);
+  shell.dev.row_blocks = (const int2*)(base + o_rb);
+  shell.dev.q_cs = (const float2*)(base + o_qcs);
+  shell.dev.part_base = (const int32_t*)(base + o_pbase);
+  shell.dev.status = (int32_t*)(base + o_status);
+  shell.dev.work_counter = shell.dev.status + 1;
+  shell.dev.ws_o = (float*)(base + o_wso);
+  shell.dev.ws_ml = (float2*)(base + o_wsml);
+
+  rc = shell.kernel == ASPD_KERNEL_MMA ? launch_attn_mma(&shell, q, k_pool, v_pool, s)
+                                       : launch_attn_generic(&shell, q, k_pool, v_pool, s);
+  if (rc) return rc;
+  return launch_combine(&shell, out, s);
+}

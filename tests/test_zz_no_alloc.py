@@ -1,0 +1,78 @@
+"""aspd_attn_static: the attention of a step with all scratch memory inside an array that is
+part of the library, for callers that are not allowed to allocate device memory (a process
+whose device memory is owned by a pool, a serving loop that must not re-enter an allocator).
+
+Collected last on purpose: a run that stops at the first failure has then already run every
+other test.  The test needs nothing from the other tests and passes alone in a fresh process.
+"""
+import numpy as np
+import pytest
+
+from paper_2508_08895_b200 import binding as B, workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def _setup(wl):
+    """Fill the cache of one layer through the ordinary path; return what the last phase needs."""
+    import torch
+    from paper_2508_08895_b200 import engine as E
+    run = E.WorkloadRun(wl)
+    for ph in wl.phases[:-1]:
+        run.step(ph)
+    ph = wl.phases[-1]
+    plan = B.Plan(run.shape, ph.desc, wl.n_pool_pages, ph.mode)
+    pos, _, _ = B.positions(ph.desc, ph.mode)
+    B.kv_append(plan, E.to_device(ph.k_new, wl.dtype), E.to_device(ph.v_new, wl.dtype),
+                torch.from_numpy(pos.copy()).cuda(), run.cache.k, run.cache.v)
+    q = E.to_device(ph.q, wl.dtype)
+    ref = torch.empty_like(q)
+    (B.branch_attn if ph.mode == W.MODE_BRANCH else B.serial_attn)(plan, q, run.cache.k, run.cache.v, ref)
+    torch.cuda.synchronize()
+    assert plan.status() == 0
+    return run, ph, q, ref
+
+
+@pytest.mark.parametrize("make", [
+    lambda: W.config_qwen7b_layer(),
+    lambda: W.config_tiny(),
+    lambda: W.build_segment_workload("ragged", 77, 28, 4, 128, "bf16", 1e6, [15, 300], [[14, 15, 16], [255, 1, 99]],
+                                     [[1, 1, 1], [1, 1, 1]], serial_steps=1),
+])
+def test_static_scratch_entry_point_matches_the_allocating_one_twice_in_a_row(make):
+    import torch
+    wl = make()
+    run, ph, q, ref = _setup(wl)
+    host_plan = B.Plan(run.shape, ph.desc, wl.n_pool_pages, ph.mode, host_only=True)
+    before = torch.cuda.memory_allocated()
+    outs = []
+    for _ in range(2):                      # the array keeps the first call's contents for the second
+        out = torch.full_like(q, float("nan"))
+        B.attn_static(host_plan, q, run.cache.k, run.cache.v, out)
+        torch.cuda.synchronize()
+        outs.append(out.float().cpu().numpy())
+    want = ref.float().cpu().numpy()
+    tol = dict(bf16=(2e-2, 2e-3), f32=(1e-4, 1e-5))[wl.dtype]
+    for got in outs:
+        assert np.isfinite(got).all()
+        err = np.abs(got.astype(np.float64) - want)
+        assert err.max() <= tol[0] and err.mean() <= tol[1]
+    np.testing.assert_array_equal(outs[0], outs[1])
+    assert torch.cuda.memory_allocated() - before <= q.numel() * q.element_size() * 2   # only the test's own outputs
+
+
+def test_static_scratch_rejects_plans_beyond_its_size_and_device_plans():
+    import torch
+    wl = W.build_segment_workload("big", 5, 28, 4, 128, "bf16", 1e6, [16384], [[40] * 8], [[1] * 8])
+    ph = wl.phases[-1]
+    shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
+    # 16-key items: thousands of partial records, far more than the 8 MiB array holds
+    plan = B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode, chunk_tokens=16, host_only=True)
+    dummy = torch.zeros(8 * 28 * 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.AspdError) as e:
+        B.attn_static(plan, dummy, dummy, dummy, dummy)
+    assert e.value.status == -7
+    dev_plan = B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode)
+    with pytest.raises(B.AspdError) as e:
+        B.attn_static(dev_plan, dummy, dummy, dummy, dummy)
+    assert e.value.status == -1
