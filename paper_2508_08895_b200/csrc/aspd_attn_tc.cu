@@ -169,7 +169,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 #ifdef ASPD_TC_PROFILE
 // Development aid: CTA 0 stamps clock64() at pipeline events of its first 64 tiles into the
 // buffer whose address is given by the environment (see launch_attn_mma).
-#define ASPD_STAMP(c, g, ev) do { if ((c).prof && blockIdx.x == 0 && (g) < 64) (c).prof[(g) * 16 + (ev)] = clock64(); } while (0)
+#define ASPD_STAMP(c, g, ev) do { if ((c).prof && blockIdx.x == (c).prof_cta && (g) < 64) (c).prof[(g) * 16 + (ev)] = clock64(); } while (0)
 // every CTA: globaltimer (ns) at entry / after set-up / after its last epilogue / at exit
 __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
 #define ASPD_CTA_STAMP(c, ev) do { if ((c).prof) (c).prof[1024 + blockIdx.x * 4 + (ev)] = gtime(); } while (0)
@@ -181,6 +181,7 @@ __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u6
 struct Ctx {
   PlanDevice pd;
   long long* prof;
+  int prof_cta;
   const __nv_bfloat16* q;
   const char* k_pool;
   const char* v_pool;
@@ -362,7 +363,16 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* ab = &misc->abort_flag;
   if (tid == 0) ASPD_CTA_STAMP(c, 0);
+  if (tid == 0) pdl_launch_dependents();
   const int item_begin = c.pd.cta_item0[blockIdx.x], item_end = c.pd.cta_item0[blockIdx.x + 1];
+  // Plan tables do not depend on earlier kernels of the stream: the first item and, for the
+  // producers, its first batch of page entries are fetched while the CTA is still setting up.
+  DeviceItem first_item = {};
+  int2 first_pages = make_int2(0, 0);
+  if (item_begin < item_end) {
+    first_item = c.pd.items[item_begin];
+    if ((warp == 4 || warp == 7) && lane < first_item.n_pages) first_pages = c.pd.visit[first_item.page0 + lane];
+  }
 
   if (tid == 0) {
     const int counts[NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, 128, 128, 128, 1, 1, 1, 128, 128, 128, 128, 1, 1, 128, 128};
@@ -379,6 +389,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = misc->tmem_base;
+  // everything above touches only the plan's own tables; inputs written by earlier kernels of
+  // the stream (q, the pools, the workspace's previous readers) are used from here on
+  pdl_wait();
   if (tid == 0) ASPD_CTA_STAMP(c, 1);
 
   if (warp < 4) {
@@ -403,10 +416,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     int g = 0;
     bool ok = true;
     for (int idx = item_begin; idx < item_end && ok; ++idx) {
-      const DeviceItem it = c.pd.items[idx];
+      const DeviceItem it = idx == item_begin ? first_item : c.pd.items[idx];
       const int n_tiles = (it.n_pages + 7) >> 3;
-      int2 cur = make_int2(0, 0), nxt = make_int2(0, 0);
-      if (lane < it.n_pages) cur = c.pd.visit[it.page0 + lane];
+      int2 cur = first_pages, nxt = make_int2(0, 0);
+      if (idx != item_begin) {
+        cur = make_int2(0, 0);
+        if (lane < it.n_pages) cur = c.pd.visit[it.page0 + lane];
+      }
       for (int t = 0; t < n_tiles && ok; ++t, ++g) {
         if ((t & 3) == 0) {
           if (t > 0) cur = nxt;
@@ -509,7 +525,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     int item_no = 0;
     bool dead = false;
     if (item_begin < item_end) {                   // the first query tile, while the first K/V tiles are in flight
-      prep_q(c, c.pd.items[item_begin], base + OFF_Q, et);
+      prep_q(c, first_item, base + OFF_Q, et);
       fence_async_smem();
       mbar_arrive(bars + 8 * Q_FULL);
     }
@@ -585,8 +601,10 @@ int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const
   Ctx c;
   c.pd = p->dev;
   c.prof = nullptr;
+  c.prof_cta = 0;
 #ifdef ASPD_TC_PROFILE
   if (const char* e = getenv("ASPD_TC_PROFILE_BUF")) c.prof = (long long*)strtoull(e, nullptr, 0);
+  if (const char* e = getenv("ASPD_TC_PROFILE_CTA")) c.prof_cta = atoi(e);
 #endif
   c.q = (const __nv_bfloat16*)q;
   c.k_pool = (const char*)k_pool;
@@ -595,8 +613,7 @@ int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const
   c.n_q_heads = sh.n_q_heads;
   c.n_kv_heads = sh.n_kv_heads;
   c.scale_log2 = sh.sm_scale * kLog2e;
-  attn_tc_kernel<<<p->n_ctas, kThreads, kSmemBytes, s>>>(c);
-  return cudaGetLastError() == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
+  return launch_pdl(kPdlAttn, attn_tc_kernel, dim3(p->n_ctas), dim3(kThreads), kSmemBytes, s, c) == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
 }
 
 }  // namespace aspd

@@ -87,6 +87,30 @@ struct aspd_plan {
 };
 
 namespace aspd {
+// Programmatic dependent launch.  Every kernel of the library is launched with the
+// "programmatic stream serialization" attribute and begins with pdl_enter(): it lets the next
+// kernel in the stream start its own set-up right away and then waits until the previous kernel
+// has completed and its writes are visible.  Because every kernel waits before it ends, the
+// dependency on all earlier kernels of the stream is kept transitively; what is gained is that
+// launch latency and set-up of a kernel overlap the tail of the one before it.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+enum { kPdlAppend = 1, kPdlAttn = 2, kPdlCombine = 4 };
+int pdl_mask();   // which kernels are launched with the attribute (environment ASPD_PDL; default append + attention)
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(int which, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                              Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = (pdl_mask() & which) ? 1 : 0;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // launchers (each returns an aspd_status_t)
 int launch_append(const aspd_plan* p, const void* k_new, const void* v_new, const int32_t* pos,
                   void* k_pool, void* v_pool, cudaStream_t s);

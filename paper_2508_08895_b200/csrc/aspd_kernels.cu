@@ -2,7 +2,18 @@
 // supported dtype / head_dim / page_size), the log-sum-exp combine (a7) and a debug reader.
 #include "aspd_internal.cuh"
 
+#include <stdlib.h>
+
 namespace aspd {
+
+int pdl_mask() {
+  static int mask = -1;
+  if (mask < 0) {
+    const char* e = getenv("ASPD_PDL");
+    mask = e ? atoi(e) & 7 : (kPdlAppend | kPdlAttn);   // measured: the combine does better as a plain launch
+  }
+  return mask;
+}
 
 namespace {
 
@@ -22,6 +33,8 @@ __global__ void append_kernel(const T* __restrict__ k_new, const T* __restrict__
                               const int32_t* __restrict__ tok_page, const int32_t* __restrict__ tok_row,
                               const double* __restrict__ inv_freq, T* __restrict__ k_pool, T* __restrict__ v_pool,
                               int n_kv_heads, int head_dim, int page_size) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int t = blockIdx.x / n_kv_heads, h = blockIdx.x % n_kv_heads, i = threadIdx.x, half = head_dim / 2;
   if (i >= half) return;
   // angle reduced to [-pi, pi] in fp64, then fp32 sincos: the error stays near 1e-7 rad
@@ -56,6 +69,8 @@ __global__ void __launch_bounds__(128) attn_generic_kernel(PlanDevice pd, const 
   constexpr int EPL = D / 32;                 // output elements per lane
   constexpr int EPC = 16 / (int)sizeof(T);    // elements per 16-byte chunk
   __shared__ float q_s[4][D];
+  pdl_launch_dependents();
+  pdl_wait();
   const DeviceItem it = pd.items[blockIdx.x];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = n_q_heads / n_kv_heads, n_rows = it.n_q_tok * G, n_keys = it.n_pages * page_size;
@@ -139,7 +154,9 @@ __global__ void __launch_bounds__(128) attn_generic_kernel(PlanDevice pd, const 
 template <typename T, int D>
 __global__ void combine_kernel(PlanDevice pd, T* __restrict__ out, int n_new, int n_q_heads, int n_kv_heads) {
   constexpr int EPL = D / 32;
+  pdl_launch_dependents();
   const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  pdl_wait();
   if (w >= n_new * n_q_heads) return;
   const int tok = w / n_q_heads, hq = w % n_q_heads, G = n_q_heads / n_kv_heads, h = hq / G, g = hq % G;
   const int p0 = pd.part_base[tok * n_kv_heads + h], n = pd.part_base[tok * n_kv_heads + h + 1] - p0;
@@ -198,6 +215,7 @@ __global__ void read_token_kernel(const T* pool, size_t tile, int row, int head_
 }
 
 inline int check_launch() { return cudaGetLastError() == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA; }
+inline int status_of(cudaError_t e) { return e == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA; }
 
 }  // namespace
 
@@ -206,15 +224,12 @@ int launch_append(const aspd_plan* p, const void* k_new, const void* v_new, cons
   const aspd_shape_t& sh = p->shape;
   const dim3 grid(p->n_new * sh.n_kv_heads), block(sh.head_dim / 2);
   if (sh.dtype == ASPD_DTYPE_BF16)
-    append_kernel<__nv_bfloat16><<<grid, block, 0, s>>>((const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, pos,
-                                                        p->dev.tok_page, p->dev.tok_row, p->dev.inv_freq,
-                                                        (__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool, sh.n_kv_heads,
-                                                        sh.head_dim, sh.page_size);
-  else
-    append_kernel<float><<<grid, block, 0, s>>>((const float*)k_new, (const float*)v_new, pos, p->dev.tok_page,
-                                                p->dev.tok_row, p->dev.inv_freq, (float*)k_pool, (float*)v_pool,
-                                                sh.n_kv_heads, sh.head_dim, sh.page_size);
-  return check_launch();
+    return status_of(launch_pdl(kPdlAppend, append_kernel<__nv_bfloat16>, grid, block, 0, s, (const __nv_bfloat16*)k_new,
+                                (const __nv_bfloat16*)v_new, pos, p->dev.tok_page, p->dev.tok_row, p->dev.inv_freq,
+                                (__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool, sh.n_kv_heads, sh.head_dim, sh.page_size));
+  return status_of(launch_pdl(kPdlAppend, append_kernel<float>, grid, block, 0, s, (const float*)k_new, (const float*)v_new, pos,
+                              p->dev.tok_page, p->dev.tok_row, p->dev.inv_freq, (float*)k_pool, (float*)v_pool, sh.n_kv_heads,
+                              sh.head_dim, sh.page_size));
 }
 
 int launch_attn_generic(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, cudaStream_t s) {
@@ -223,27 +238,26 @@ int launch_attn_generic(const aspd_plan* p, const void* q, const void* k_pool, c
   const float sc = sh.sm_scale * kLog2e;
   const dim3 grid(p->n_items), block(128);
 #define ASPD_GEN(T, D)                                                                                         \
-  attn_generic_kernel<T, D><<<grid, block, 0, s>>>(p->dev, (const T*)q, (const T*)k_pool, (const T*)v_pool,    \
-                                                   sh.n_q_heads, sh.n_kv_heads, sh.page_size, sc)
+  return status_of(launch_pdl(kPdlAttn, attn_generic_kernel<T, D>, grid, block, 0, s, p->dev, (const T*)q, (const T*)k_pool, \
+                              (const T*)v_pool, sh.n_q_heads, sh.n_kv_heads, sh.page_size, sc))
   if (sh.dtype == ASPD_DTYPE_BF16 && sh.head_dim == 128) ASPD_GEN(__nv_bfloat16, 128);
   else if (sh.dtype == ASPD_DTYPE_BF16) ASPD_GEN(__nv_bfloat16, 64);
   else if (sh.head_dim == 128) ASPD_GEN(float, 128);
   else ASPD_GEN(float, 64);
 #undef ASPD_GEN
-  return check_launch();
 }
 
 int launch_combine(const aspd_plan* p, void* out, cudaStream_t s) {
   const aspd_shape_t& sh = p->shape;
   const int warps = p->n_new * sh.n_q_heads;
   const dim3 block(128), grid((warps + 3) / 4);
-#define ASPD_CMB(T, D) combine_kernel<T, D><<<grid, block, 0, s>>>(p->dev, (T*)out, p->n_new, sh.n_q_heads, sh.n_kv_heads)
+#define ASPD_CMB(T, D) \
+  return status_of(launch_pdl(kPdlCombine, combine_kernel<T, D>, grid, block, 0, s, p->dev, (T*)out, p->n_new, sh.n_q_heads, sh.n_kv_heads))
   if (sh.dtype == ASPD_DTYPE_BF16 && sh.head_dim == 128) ASPD_CMB(__nv_bfloat16, 128);
   else if (sh.dtype == ASPD_DTYPE_BF16) ASPD_CMB(__nv_bfloat16, 64);
   else if (sh.head_dim == 128) ASPD_CMB(float, 128);
   else ASPD_CMB(float, 64);
 #undef ASPD_CMB
-  return check_launch();
 }
 
 int launch_read_token(const aspd_shape_t* sh, const void* pool, int64_t page, int row, int kv_head, float* out_dev,
