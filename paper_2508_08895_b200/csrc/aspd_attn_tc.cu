@@ -47,12 +47,17 @@ constexpr uint32_t OFF_MISC = OFF_P + 8192;
 enum Bar { K_FULL = 0, K_EMPTY = 2, V_FULL = 4, V_EMPTY = 6, S_FULL = 8, S_EMPTY = 10, P_FULL = 12, P_EMPTY = 13,
            O_FULL = 14, O_EMPTY = 16, Q_FULL = 18, Q_EMPTY = 20, E_FULL = 22, NUM_BARS = 24 };
 
+constexpr int kItemCache = 12;      // items of a CTA kept in shared memory (more are read from global)
+constexpr int kMaxTokPerItem = 16;  // tokens of a row block whose ranges are cached (n_q_tok is at most 64 / G)
+
 struct Misc {
   uint64_t bars[NUM_BARS];
   float smax[2][128];
   float fin_m[2][128];         // per item parity: reference maximum and sum of every softmax thread
   float fin_l[2][128];
   int nval[4][8];              // valid rows of the 8 pages of a tile (ring over 4 tiles)
+  DeviceItem items[kItemCache];        // this CTA's first items and, per item, the visible ranges of
+  int4 vis[kItemCache][kMaxTokPerItem]; // its query tokens: no global-load chain at an item boundary
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -189,6 +194,12 @@ struct Ctx {
   float scale_log2;
 };
 
+// Item idx of this CTA (rel = idx - item_begin): from the shared-memory cache when it is there.
+__device__ __forceinline__ DeviceItem get_item(const Ctx& c, const Misc* misc, int idx, int item_begin) {
+  const int rel = idx - item_begin;
+  return rel < kItemCache ? misc->items[rel] : c.pd.items[idx];
+}
+
 // ------------------------------------------------------------------------------- softmax role
 // 16-bit mask with bits [lo, hi) set (arguments are clamped to 0..16).
 __device__ __forceinline__ uint32_t bits_between(int lo, int hi) {
@@ -198,7 +209,7 @@ __device__ __forceinline__ uint32_t bits_between(int lo, int hi) {
 
 template <int NC>   // NC = columns per thread = padded row count R
 __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it, Misc* misc, uint32_t bars, uint32_t smem_p,
-                                             uint32_t tmem, int item_no, int& g) {
+                                             uint32_t tmem, int item_no, int& g) {   // item_no = index among this CTA's items
   constexpr int R = NC, KS = 128 / NC;
   const int tid = threadIdx.x, warp = tid >> 5;
   const int r = tid % R, j = tid / R;
@@ -206,7 +217,7 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
   const int n_tiles = (it.n_pages + 7) >> 3;
   volatile int* ab = &misc->abort_flag;
   int4 vis = make_int4(0, 0, 0, 0);             // padding rows see nothing
-  if (r < M) vis = c.pd.tok_vis[it.q_tok0 + r / G];
+  if (r < M) vis = (item_no < kItemCache && r / G < kMaxTokPerItem) ? misc->vis[item_no][r / G] : c.pd.tok_vis[it.q_tok0 + r / G];
   const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
   const int ob = item_no & 1;
   float m_ref = -INFINITY, l = 0.f;
@@ -367,11 +378,15 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   const int item_begin = c.pd.cta_item0[blockIdx.x], item_end = c.pd.cta_item0[blockIdx.x + 1];
   // Plan tables do not depend on earlier kernels of the stream: the first item and, for the
   // producers, its first batch of page entries are fetched while the CTA is still setting up.
-  DeviceItem first_item = {};
-  int2 first_pages = make_int2(0, 0);
-  if (item_begin < item_end) {
-    first_item = c.pd.items[item_begin];
-    if ((warp == 4 || warp == 7) && lane < first_item.n_pages) first_pages = c.pd.visit[first_item.page0 + lane];
+  {
+    const int n_cached = min(item_end - item_begin, kItemCache);
+    for (int e = tid; e < n_cached * (int)(sizeof(DeviceItem) / 4); e += kThreads)
+      reinterpret_cast<int*>(misc->items)[e] = reinterpret_cast<const int*>(c.pd.items + item_begin)[e];
+    for (int e = tid; e < n_cached * kMaxTokPerItem; e += kThreads) {
+      const DeviceItem& ci = c.pd.items[item_begin + e / kMaxTokPerItem];
+      const int tl = e % kMaxTokPerItem;
+      if (tl < ci.n_q_tok) misc->vis[e / kMaxTokPerItem][tl] = c.pd.tok_vis[ci.q_tok0 + tl];
+    }
   }
 
   if (tid == 0) {
@@ -398,7 +413,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     // =============================== softmax + epilogue ===============================
     int g = 0, item_no = 0;
     for (int idx = item_begin; idx < item_end; ++idx, ++item_no) {
-      const DeviceItem it = c.pd.items[idx];
+      const DeviceItem it = get_item(c, misc, idx, item_begin);
       const int M = it.n_q_tok * (c.n_q_heads / c.n_kv_heads);
       const bool ok = M <= 32 ? softmax_item<32>(c, it, misc, bars, base + OFF_P, tmem, item_no, g)
                               : softmax_item<64>(c, it, misc, bars, base + OFF_P, tmem, item_no, g);
@@ -415,20 +430,28 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     const char* pool = kv ? c.v_pool : c.k_pool;
     int g = 0;
     bool ok = true;
+    // (item, batch of 32 pages) pairs are walked as one sequence: `cur` holds the batch being
+    // consumed, `nxt` the one after it, which may already belong to the next item.
+    int2 nxt = make_int2(0, 0);
+    if (item_begin < item_end) {
+      const DeviceItem f = get_item(c, misc, item_begin, item_begin);
+      if (lane < f.n_pages) nxt = c.pd.visit[f.page0 + lane];
+    }
     for (int idx = item_begin; idx < item_end && ok; ++idx) {
-      const DeviceItem it = idx == item_begin ? first_item : c.pd.items[idx];
+      const DeviceItem it = get_item(c, misc, idx, item_begin);
       const int n_tiles = (it.n_pages + 7) >> 3;
-      int2 cur = first_pages, nxt = make_int2(0, 0);
-      if (idx != item_begin) {
-        cur = make_int2(0, 0);
-        if (lane < it.n_pages) cur = c.pd.visit[it.page0 + lane];
-      }
+      int2 cur = make_int2(0, 0);
       for (int t = 0; t < n_tiles && ok; ++t, ++g) {
         if ((t & 3) == 0) {
-          if (t > 0) cur = nxt;
-          const int ahead = (t + 4) * 8 + lane;
+          cur = nxt;
           nxt = make_int2(0, 0);
-          if (ahead < it.n_pages) nxt = c.pd.visit[it.page0 + ahead];
+          const int ahead = (t + 4) * 8 + lane;
+          if ((t + 4) * 8 < it.n_pages) {
+            if (ahead < it.n_pages) nxt = c.pd.visit[it.page0 + ahead];
+          } else if (idx + 1 < item_end) {          // first batch of the next item
+            const DeviceItem nx = get_item(c, misc, idx + 1, item_begin);
+            if (lane < nx.n_pages) nxt = c.pd.visit[nx.page0 + lane];
+          }
         }
         const int npg = min(8, it.n_pages - t * 8), sl = g & 1;
         int2 pg;
@@ -504,7 +527,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
       bool ok = true, have_prev = false;
       TileRef prev = {0, 0, 0, 0, 0, 0};
       for (int idx = item_begin; idx < item_end && ok; ++idx, ++item_no) {
-        const int n_pages = c.pd.items[idx].n_pages, n_tiles = (n_pages + 7) >> 3;
+        const int n_pages = get_item(c, misc, idx, item_begin).n_pages, n_tiles = (n_pages + 7) >> 3;
         for (int t = 0; t < n_tiles && ok; ++t, ++g) {
           const TileRef cur = {min(8, n_pages - t * 8), t == 0, t == n_tiles - 1, item_no & 1, item_no & 1, item_no};
           ok = issue_s(cur, g);
@@ -525,17 +548,17 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     int item_no = 0;
     bool dead = false;
     if (item_begin < item_end) {                   // the first query tile, while the first K/V tiles are in flight
-      prep_q(c, first_item, base + OFF_Q, et);
+      prep_q(c, get_item(c, misc, item_begin, item_begin), base + OFF_Q, et);
       fence_async_smem();
       mbar_arrive(bars + 8 * Q_FULL);
     }
     for (int idx = item_begin; idx < item_end; ++idx, ++item_no) {
-      const DeviceItem it = c.pd.items[idx];
+      const DeviceItem it = get_item(c, misc, idx, item_begin);
       const int ob = item_no & 1, M = it.n_q_tok * G, R = M <= 32 ? 32 : 64, KS = 128 / R;
       if (idx + 1 < item_end) {                    // the next item's query tile, into the other buffer
         const int qn = (item_no + 1) & 1;
         dead |= !mbar_wait(bars + 8 * (Q_EMPTY + qn), (((item_no + 1) >> 1) & 1) ^ 1, ab);
-        prep_q(c, c.pd.items[idx + 1], base + OFF_Q + qn * kTileBytes, et);
+        prep_q(c, get_item(c, misc, idx + 1, item_begin), base + OFF_Q + qn * kTileBytes, et);
         fence_async_smem();
         mbar_arrive(bars + 8 * (Q_FULL + qn));
       }
