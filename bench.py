@@ -4,8 +4,9 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload serving-mix] [--layers 28]
     python bench.py --impl reference ...        # the fp64 CPU oracle on the host cores
 
-A *step* is one pass of the whole hot path -- kv_append (RoPE + paged write of the new
-tokens) -> split-K branch attention -> log-sum-exp combine -- over every attention layer of a
+A *step* is one pass of the whole hot path -- RoPE + paged write of the new tokens (a3, done by
+the attention pass itself through aspd_branch_step; --separate-append uses aspd_kv_append) ->
+split-K branch attention -> log-sum-exp combine -- over every attention layer of a
 Qwen2.5-7B-shaped stack (28 layers, each with its own K/V pools, one shared plan), for one
 decoding step of the synthetic batch.  The pools of all layers together are far larger than
 L2, so every layer streams its KV from HBM.
@@ -43,6 +44,11 @@ import numpy as np
 METRIC = "branch_decode_attn_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes moved per algorithmic byte by the split-K attention kernel, from the ncu capture
+# summarised in profiles/attn_tc_kernel_serving_mix.md (62.36 MB of dram read + write for 61.44 MB
+# algorithmic on the 8-request case; the kernel streams every page once, so traffic scales with the
+# cached tokens).
+TRAFFIC_PER_ALGORITHMIC_BYTE = 1.015
 
 
 def measured_peaks():
@@ -217,10 +223,15 @@ def run_ours(args):
     q_d, k_d, v_d = (E.to_device(x, wl.dtype) for x in (ph.q, ph.k_new, ph.v_new))
     outs = [torch.empty_like(q_d) for _ in range(L)]
     attn = B.branch_attn if ph.mode == W.MODE_BRANCH else B.serial_attn
+    fstep = B.branch_step if ph.mode == W.MODE_BRANCH else B.serial_step
+    fused = not args.separate_append
     def step():
         for l in range(L):
-            B.kv_append(plan, k_d, v_d, pos_d, caches[l].k, caches[l].v)
-            attn(plan, q_d, caches[l].k, caches[l].v, outs[l])
+            if fused:      # the attention pass writes the step's new K/V rows itself: 2 launches per layer
+                fstep(plan, q_d, k_d, v_d, caches[l].k, caches[l].v, outs[l])
+            else:          # aspd_kv_append, then aspd_branch_attn: 3 launches per layer
+                B.kv_append(plan, k_d, v_d, pos_d, caches[l].k, caches[l].v)
+                attn(plan, q_d, caches[l].k, caches[l].v, outs[l])
 
     def barrier():
         if world > 1:
@@ -323,17 +334,21 @@ def run_ours(args):
                        "page_size": wl.page_size, "kernel": {1: "generic", 2: "mma"}[info.kernel],
                        "chunk_tokens": info.chunk_tokens, "work_items": info.n_items, "n_ctas": info.n_ctas,
                        "l2": "footprint %.1f GB of distinct K/V pools per step, far above L2" % (alg * L / 1e9),
-                       "layers_agree": bool(same), "cuda_graph": not args.no_graph},
+                       "layers_agree": bool(same), "cuda_graph": not args.no_graph,
+                       "calls_per_layer": "aspd_branch_step (append fused into the attention pass) -> combine" if fused
+                       else "aspd_kv_append -> aspd_branch_attn"},
             "hbm_gbs": alg * L * args.steps / (ms * 1e-3) / 1e9,
             "hbm_frac_of_measured": alg * L * args.steps / (ms * 1e-3) / 1e9 / peak,
             "hbm_frac_of_8000_nominal": alg * L * args.steps / (ms * 1e-3) / 1e9 / 8000.0,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_kind": "of " + peak_kind, "kernel": "split-K attention pass",
+                         "traffic": alg * TRAFFIC_PER_ALGORITHMIC_BYTE if info.kernel == 2 else None,
+                         "traffic_note": "ncu capture of a smaller case of the same mix, scaled by cached tokens",
+                         "peak_kind": "of " + peak_kind, "kernel": "split-K attention pass",
                          "kernel_us": kernel_ms * 1e3, "algorithmic_bytes_per_launch": alg},
             "e2e": {"value": total_new * L * e_steps / (e2e_ms * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": int(L * (n_new * es * wl.d * (wl.Hq + 2 * wl.Hkv) + 4 * n_new)),
                     "d2h_bytes_per_step": int(L * n_new * es * wl.d * wl.Hq), "ms_per_step": e2e_ms / e_steps},
-            "gpu_launches": 3 * L * args.steps,
+            "gpu_launches": (2 if fused and info.kernel == 2 else 3) * L * args.steps,
             "clocks": clocks,
         }
         if world == 1 and not args.no_cpu_baseline:
@@ -362,6 +377,8 @@ def main():
     ap.add_argument("--requests", type=int, default=0, help="serving-mix only: number of requests (default 32)")
     ap.add_argument("--cpu-budget", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--separate-append", action="store_true",
+                    help="call aspd_kv_append and aspd_branch_attn separately instead of aspd_branch_step")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":

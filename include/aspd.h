@@ -21,7 +21,9 @@
  *     [head_dim]; element type per aspd_shape_t.dtype.  The K and V pools are
  *     [n_pool_pages][n_kv_heads] tiles of page_size x head_dim elements each
  *     (aspd_pool_bytes gives the size); the order of elements INSIDE a tile is private to
- *     the library -- read tokens back with aspd_debug_read_token.
+ *     the library -- read tokens back with aspd_debug_read_token.  Pools must be zero-filled
+ *     (or at least hold no NaN/Inf bit patterns) before their first use: the rows of a partly
+ *     filled page that no token has been written to yet are multiplied by a weight of exactly 0.
  *   - Positions are 0-based.  Query head h uses KV head h / (n_q_heads / n_kv_heads).
  *     RoPE pairs element i with i + head_dim/2 and uses inv_freq[i] = theta^(-2i/head_dim)
  *     (the paper leaves the encoding open; this is the rotate-half convention of the
@@ -224,6 +226,21 @@ int aspd_attn_partials(aspd_plan_t* plan, const void* q /*device*/, const void* 
 int aspd_attn_combine(aspd_plan_t* plan, void* out /*device*/, void* stream);
 
 /*
+ * a3 + a4-a7 (or a3 + a9) in one call: the step's new K/V rows are written into the cache by the
+ * attention pass itself, just before it reads the pages they live in (each CTA writes the rows of
+ * the pages it is about to read; CTAs that share a page write identical bytes), so no separate
+ * append launch is needed.  The position IDs are the plan's (aspd_positions, or q_pos if given);
+ * results equal aspd_kv_append followed by aspd_branch_attn / aspd_serial_attn up to the last bit
+ * of the cos/sin evaluation.  k_new, v_new as for aspd_kv_append.
+ */
+int aspd_branch_step(aspd_plan_t* plan, const void* q /*device*/, const void* k_new /*device*/,
+                     const void* v_new /*device*/, void* k_pool /*device*/, void* v_pool /*device*/,
+                     void* out /*device*/, void* stream);
+int aspd_serial_step(aspd_plan_t* plan, const void* q /*device*/, const void* k_new /*device*/,
+                     const void* v_new /*device*/, void* k_pool /*device*/, void* v_pool /*device*/,
+                     void* out /*device*/, void* stream);
+
+/*
  * The whole step (a3-a7 or a3 + a9, by the plan's mode) from HOST buffers: copies q, k_new,
  * v_new, pos to staging memory the plan owns, runs append + attention, copies out back, all
  * on `stream`, then synchronises it.  The pools stay on the device (they are the state).
@@ -265,6 +282,15 @@ int aspd_attn_static(const aspd_plan_t* plan /*host-only*/, const void* q /*devi
  * Synchronises `stream`.  For tests. */
 int aspd_debug_read_token(const aspd_shape_t* shape, const void* pool /*device*/, int64_t page,
                           int row, int kv_head, float* out /*host*/, void* stream);
+
+/*
+ * Failure-path check: runs the library's bounded device-side wait on a barrier nobody ever
+ * arrives on, with a limit of `limit_cycles` SM clock cycles (at most 4e9).  The kernel gives up
+ * when the limit passes and reports ASPD_ERR_TIMEOUT through *status_out (host); the context
+ * stays usable.  This is the same wait every hand-off of the tensor-core kernel uses.
+ * Synchronises `stream`.
+ */
+int aspd_debug_bounded_wait(int64_t limit_cycles, int32_t* status_out /*host*/, void* stream);
 
 #ifdef __cplusplus
 }

@@ -57,7 +57,7 @@ EXPORTS = ("aspd_strerror", "aspd_pool_bytes", "aspd_count_new_tokens", "aspd_po
            "aspd_plan_create", "aspd_plan_destroy", "aspd_plan_info", "aspd_plan_items", "aspd_plan_stream_pages",
            "aspd_plan_token_ranges", "aspd_plan_status",
            "aspd_kv_append", "aspd_branch_attn", "aspd_serial_attn", "aspd_attn_partials", "aspd_attn_combine",
-           "aspd_step_host", "aspd_attn_static", "aspd_debug_read_token")
+           "aspd_branch_step", "aspd_serial_step", "aspd_step_host", "aspd_attn_static", "aspd_debug_read_token", "aspd_debug_bounded_wait")
 
 _lib = None
 
@@ -93,8 +93,11 @@ def lib() -> ctypes.CDLL:
         L.aspd_serial_attn.argtypes = [vp] * 6
         L.aspd_attn_partials.argtypes = [vp] * 5
         L.aspd_attn_combine.argtypes = [vp] * 3
+        L.aspd_branch_step.argtypes = [vp] * 8
+        L.aspd_serial_step.argtypes = [vp] * 8
         L.aspd_step_host.argtypes = [vp] * 9
         L.aspd_attn_static.argtypes = [vp] * 6
+        L.aspd_debug_bounded_wait.argtypes = [ctypes.c_int64, vp, vp]
         L.aspd_debug_read_token.argtypes = [vp, vp, ctypes.c_int64, ci, ci, vp, vp]
         for name in EXPORTS:
             if name not in ("aspd_strerror", "aspd_pool_bytes"):
@@ -258,10 +261,27 @@ def attn_combine(plan: Plan, out, stream=None) -> None:
     _check(lib().aspd_attn_combine(plan._h, _ptr(out), _stream(stream)), "aspd_attn_combine")
 
 
+def branch_step(plan: Plan, q, k_new, v_new, k_pool, v_pool, out, stream=None) -> None:
+    _check(lib().aspd_branch_step(plan._h, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pool), _ptr(v_pool), _ptr(out),
+                                  _stream(stream)), "aspd_branch_step")
+
+
+def serial_step(plan: Plan, q, k_new, v_new, k_pool, v_pool, out, stream=None) -> None:
+    _check(lib().aspd_serial_step(plan._h, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pool), _ptr(v_pool), _ptr(out),
+                                  _stream(stream)), "aspd_serial_step")
+
+
 def step_host(plan: Plan, q, k_new, v_new, pos, k_pool, v_pool, out, stream=None) -> None:
     """Whole step from host (numpy / pinned torch CPU) buffers; ``out`` is a host buffer."""
     _check(lib().aspd_step_host(plan._h, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(pos), _ptr(k_pool), _ptr(v_pool),
                                 _ptr(out), _stream(stream)), "aspd_step_host")
+
+
+def debug_bounded_wait(limit_cycles: int, stream=None) -> int:
+    """Status a bounded device-side wait reports when nothing ever satisfies it (ASPD_ERR_TIMEOUT)."""
+    st = np.zeros(1, dtype=np.int32)
+    _check(lib().aspd_debug_bounded_wait(int(limit_cycles), _ptr(st), _stream(stream)), "aspd_debug_bounded_wait")
+    return int(st[0])
 
 
 STATIC_SCRATCH_BYTES = 8 << 20

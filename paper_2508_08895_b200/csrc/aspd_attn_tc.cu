@@ -45,7 +45,7 @@ constexpr uint32_t OFF_K = 0, OFF_V = 2 * kTileBytes, OFF_Q = 4 * kTileBytes, OF
 constexpr uint32_t OFF_MISC = OFF_P + 8192;
 
 enum Bar { K_FULL = 0, K_EMPTY = 2, V_FULL = 4, V_EMPTY = 6, S_FULL = 8, S_EMPTY = 10, P_FULL = 12, P_EMPTY = 13,
-           O_FULL = 14, O_EMPTY = 16, Q_FULL = 18, Q_EMPTY = 20, E_FULL = 22, NUM_BARS = 24 };
+           O_FULL = 14, O_EMPTY = 16, Q_FULL = 18, Q_EMPTY = 20, E_FULL = 22, A_DONE = 24, NUM_BARS = 25 };
 
 constexpr int kItemCache = 12;      // items of a CTA kept in shared memory (more are read from global)
 constexpr int kMaxTokPerItem = 16;  // tokens of a row block whose ranges are cached (n_q_tok is at most 64 / G)
@@ -89,13 +89,14 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: false means "give up" (time limit hit here or in another role).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit = kWaitCycles) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
     if (mbar_try(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) { *abort_flag = 1; return false; }
+    if (clock64() - t0 > limit) { *abort_flag = 1; return false; }
   }
 }
 __device__ __forceinline__ void bulk_copy(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -188,6 +189,8 @@ struct Ctx {
   long long* prof;
   int prof_cta;
   const __nv_bfloat16* q;
+  const __nv_bfloat16* k_new;  // non-null (with v_new): write this step's new rows before reading their pages
+  const __nv_bfloat16* v_new;
   const char* k_pool;
   const char* v_pool;
   int n_items, n_q_heads, n_kv_heads;
@@ -363,6 +366,65 @@ __device__ __forceinline__ void prep_q(const Ctx& c, const DeviceItem& it, uint3
   }
 }
 
+// Fused step (aspd_branch_step / aspd_serial_step): the rows this step adds to pages that THIS CTA
+// reads are written into the pools at the start of the kernel, K rotated at the token's position
+// (cos/sin table of the plan) and V as is.  CTAs that read the same page write identical bytes, so
+// no cross-CTA ordering is needed.  One unit = one 16-byte chunk pair of K (8 per row) or one
+// 16-byte chunk of V (16 per row).  Called by the 128 epilogue threads; the loads of a batch of
+// units are all issued before its first store.
+__device__ __forceinline__ void append_new_rows(const Ctx& c, int rank, int d0, int n_units, const int4 (&first)[2]) {
+  for (int u0 = rank; u0 < n_units; u0 += 128 * 2) {
+    int4 d[2];
+    uint4 a[2], b[2];
+    float4 w[2][4];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int u = u0 + k * 128;
+      d[k] = first[k];                                         // the first batch was fetched during set-up
+      if (u0 != rank) { d[k] = make_int4(0, 0, 0, 0); if (u < n_units) d[k] = c.pd.dirty[d0 + u / 24]; }   // (page, KV head, token, row)
+    }
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int u = u0 + k * 128, sub = u % 24;
+      a[k] = make_uint4(0, 0, 0, 0); b[k] = a[k];
+      if (u >= n_units) continue;
+      const size_t src = ((size_t)d[k].z * c.n_kv_heads + d[k].y) * 128;
+      if (sub < 8) {
+        a[k] = *reinterpret_cast<const uint4*>(c.k_new + src + sub * 8);
+        b[k] = *reinterpret_cast<const uint4*>(c.k_new + src + 64 + sub * 8);
+        const float4* cs = reinterpret_cast<const float4*>(c.pd.q_cs + (size_t)d[k].z * 64 + sub * 8);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) w[k][i] = cs[i];
+      } else {
+        a[k] = *reinterpret_cast<const uint4*>(c.v_new + src + (sub - 8) * 8);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int u = u0 + k * 128, sub = u % 24;
+      if (u >= n_units) continue;
+      const size_t tile = ((size_t)d[k].x * c.n_kv_heads + d[k].y) * 4096;
+      if (sub < 8) {
+        const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&a[k]);
+        const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&b[k]);
+        uint32_t lo[4], hi[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 x0 = __bfloat1622float2(a2[i]), x1 = __bfloat1622float2(b2[i]);
+          lo[i] = pack_bf16(x0.x * w[k][i].x - x1.x * w[k][i].y, x0.y * w[k][i].z - x1.y * w[k][i].w);
+          hi[i] = pack_bf16(x1.x * w[k][i].x + x0.x * w[k][i].y, x1.y * w[k][i].z + x0.y * w[k][i].w);
+        }
+        char* kt = const_cast<char*>(c.k_pool) + tile;
+        *reinterpret_cast<uint4*>(kt + tile_offset(d[k].w, sub * 16, 256)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        *reinterpret_cast<uint4*>(kt + tile_offset(d[k].w, 128 + sub * 16, 256)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      } else {
+        *reinterpret_cast<uint4*>(const_cast<char*>(c.v_pool) + tile + tile_offset(d[k].w, (sub - 8) * 16, 256)) = a[k];
+      }
+    }
+  }
+  asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy stores before the producers' async-proxy copies
+}
+
 // --------------------------------------------------------------------------------- the kernel
 __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   extern __shared__ uint8_t smem_raw[];
@@ -390,7 +452,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   }
 
   if (tid == 0) {
-    const int counts[NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, 128, 128, 128, 1, 1, 1, 128, 128, 128, 128, 1, 1, 128, 128};
+    const int counts[NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, 128, 128, 128, 1, 1, 1, 128, 128, 128, 128, 1, 1, 128, 128, 128};
     for (int i = 0; i < NUM_BARS; ++i) mbar_init(bars + 8 * i, counts[i]);
     misc->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -404,8 +466,20 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = misc->tmem_base;
+  // fused step: the epilogue threads fetch their first new-row entries now (plan data)
+  int dirty0 = 0, dirty_units = 0;
+  int4 dirty_first[2] = {make_int4(0, 0, 0, 0), make_int4(0, 0, 0, 0)};
+  if (warp >= 8 && c.k_new != nullptr) {
+    dirty0 = c.pd.cta_dirty0[blockIdx.x];
+    dirty_units = (c.pd.cta_dirty0[blockIdx.x + 1] - dirty0) * 24;
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int u = (tid - 256) + k * 128;
+      if (u < dirty_units) dirty_first[k] = c.pd.dirty[dirty0 + u / 24];
+    }
+  }
   // everything above touches only the plan's own tables; inputs written by earlier kernels of
-  // the stream (q, the pools, the workspace's previous readers) are used from here on
+  // the stream (q, k_new, the pools, the workspace's previous readers) are used from here on
   pdl_wait();
   if (tid == 0) ASPD_CTA_STAMP(c, 1);
 
@@ -429,7 +503,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     const int kv = warp == 4 ? 0 : 1;
     const char* pool = kv ? c.v_pool : c.k_pool;
     int g = 0;
-    bool ok = true;
+    bool ok = true, appended = false;
     // (item, batch of 32 pages) pairs are walked as one sequence: `cur` holds the batch being
     // consumed, `nxt` the one after it, which may already belong to the next item.
     int2 nxt = make_int2(0, 0);
@@ -458,13 +532,21 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
         pg.x = __shfl_sync(0xffffffffu, cur.x, (t & 3) * 8 + (lane & 7));
         pg.y = __shfl_sync(0xffffffffu, cur.y, (t & 3) * 8 + (lane & 7));
         if (lane >= npg) pg = make_int2(0, 0);
+        if (c.k_new != nullptr && !appended && __any_sync(0xffffffffu, ((pg.y >> 8) & 31) != 0)) {
+          // fused append: this tile holds rows that are new this step; the append warp has written
+          // (or is writing) them -- wait for it once, before the first such page is copied
+          int okw = 1;
+          if (lane == 0) okw = mbar_wait(bars + 8 * A_DONE, 0, ab) ? 1 : 0;
+          if (!__shfl_sync(0xffffffffu, okw, 0)) { ok = false; break; }
+          appended = true;
+        }
         const uint32_t full = bars + 8 * ((kv ? V_FULL : K_FULL) + sl), empty = bars + 8 * ((kv ? V_EMPTY : K_EMPTY) + sl);
         int good = 1;
         if (lane == 0) good = mbar_wait(empty, ((g >> 1) & 1) ^ 1, ab) ? 1 : 0;
         good = __shfl_sync(0xffffffffu, good, 0);
         if (!good) { ok = false; break; }
         if (lane == 0) ASPD_STAMP(c, g, 6 + kv);
-        if (kv == 0 && lane < 8) misc->nval[g & 3][lane] = pg.y;      // read by the softmax warps of tile g
+        if (kv == 0 && lane < 8) misc->nval[g & 3][lane] = pg.y & 255;   // read by the softmax warps of tile g
         __syncwarp();
         if (lane == 0) mbar_expect_tx(full, (uint32_t)npg * 4096u);
         __syncwarp();
@@ -547,6 +629,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     const int G = c.n_q_heads / c.n_kv_heads;
     int item_no = 0;
     bool dead = false;
+    if (c.k_new != nullptr) append_new_rows(c, et, dirty0, dirty_units, dirty_first);
+    mbar_arrive(bars + 8 * A_DONE);
     if (item_begin < item_end) {                   // the first query tile, while the first K/V tiles are in flight
       prep_q(c, get_item(c, misc, item_begin, item_begin), base + OFF_Q, et);
       fence_async_smem();
@@ -610,9 +694,33 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   }
 }
 
+
+// A wait that nothing ever satisfies, with a caller-given limit: exercises the bounded-wait path
+// (give up, record the status, leave the context usable) without hanging anything.
+__global__ void wait_probe_kernel(long long limit_cycles, int32_t* status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const bool ok = mbar_wait(smem_u32(&bar), 0, &abort_flag, limit_cycles);   // nobody arrives
+    *status = ok ? (int)ASPD_OK : (int)ASPD_ERR_TIMEOUT;
+  }
+}
+
 }  // namespace
 
-int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, cudaStream_t s) {
+int launch_wait_probe(long long limit_cycles, int32_t* status_dev, cudaStream_t s) {
+  wait_probe_kernel<<<1, 32, 0, s>>>(limit_cycles, status_dev);
+  return cudaGetLastError() == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
+}
+
+namespace {
+}  // namespace
+
+static int launch_tc(const aspd_plan* p, const void* q, const void* k_new, const void* v_new, const void* k_pool,
+                     const void* v_pool, cudaStream_t s) {
   if (p->n_items == 0) return ASPD_OK;
   const aspd_shape_t& sh = p->shape;
   static bool configured = false;
@@ -630,6 +738,8 @@ int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const
   if (const char* e = getenv("ASPD_TC_PROFILE_CTA")) c.prof_cta = atoi(e);
 #endif
   c.q = (const __nv_bfloat16*)q;
+  c.k_new = (const __nv_bfloat16*)k_new;
+  c.v_new = (const __nv_bfloat16*)v_new;
   c.k_pool = (const char*)k_pool;
   c.v_pool = (const char*)v_pool;
   c.n_items = p->n_items;
@@ -637,6 +747,15 @@ int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const
   c.n_kv_heads = sh.n_kv_heads;
   c.scale_log2 = sh.sm_scale * kLog2e;
   return launch_pdl(kPdlAttn, attn_tc_kernel, dim3(p->n_ctas), dim3(kThreads), kSmemBytes, s, c) == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
+}
+
+int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, cudaStream_t s) {
+  return launch_tc(p, q, nullptr, nullptr, k_pool, v_pool, s);
+}
+
+int launch_attn_mma_step(const aspd_plan* p, const void* q, const void* k_new, const void* v_new, void* k_pool, void* v_pool,
+                         cudaStream_t s) {
+  return launch_tc(p, q, k_new, v_new, k_pool, v_pool, s);
 }
 
 }  // namespace aspd

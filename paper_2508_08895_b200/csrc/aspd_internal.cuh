@@ -41,11 +41,15 @@ struct DeviceItem {       // mirrors aspd_item_t, 40 bytes
 struct PlanDevice {       // pointers into the plan's single device allocation
   const DeviceItem* items;
   const int32_t* cta_item0;    // [n_ctas + 1] items of CTA c are [cta_item0[c], cta_item0[c + 1])
-  const int2* visit;           // key streams: (physical page, valid rows) per page to read
+  const int2* visit;           // key streams, per page to read: (physical page, valid rows | new rows << 8 |
+                               // first new token << 13); the new rows are the last valid rows of the page
+  const int32_t* cta_dirty0;   // [n_ctas + 1] range of `dirty` that CTA c must write before reading (fused step)
+  const int4* dirty;           // (physical page, KV head, new token, row) of every new row in a CTA's pages
   const int4* tok_vis;         // [n_new] (pe, lo, hi, -): visible stream keys are [0, pe) and [lo, hi)
   const int2* row_blocks;      // [n_row_blocks] (first new token, number of tokens)
   const int32_t* tok_page;     // [n_new] physical page the new token's K/V goes to
   const int32_t* tok_row;      // [n_new] row inside that page
+  const int32_t* tok_pos;      // [n_new] position ID of the new token as the plan derived it (or q_pos)
   const float2* q_cs;          // [n_new][head_dim/2] (cos, sin) of the query's RoPE angle
   const int32_t* part_base;    // [n_new * n_kv_heads + 1] first partial record of (new token, KV head)
   const double* inv_freq;      // [head_dim/2]
@@ -119,6 +123,10 @@ int launch_attn_generic(const aspd_plan* p, const void* q, const void* k_pool, c
 int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool,
                     cudaStream_t s);
 int launch_combine(const aspd_plan* p, void* out, cudaStream_t s);
+// attention pass that first writes this step's new K (rotated) and V rows into the pages it reads
+int launch_attn_mma_step(const aspd_plan* p, const void* q, const void* k_new, const void* v_new, void* k_pool,
+                         void* v_pool, cudaStream_t s);
+int launch_wait_probe(long long limit_cycles, int32_t* status_dev, cudaStream_t s);
 int launch_read_token(const aspd_shape_t* shape, const void* pool, int64_t page, int row, int kv_head,
                       float* out_dev, cudaStream_t s);
 inline int esize_of(int dtype) { return dtype == ASPD_DTYPE_BF16 ? 2 : 4; }

@@ -97,7 +97,7 @@ __global__ void __launch_bounds__(128) attn_generic_kernel(PlanDevice pd, const 
       if (j < n_keys) {
         const int2 pg = pd.visit[it.page0 + j / page_size];
         const int row = j % page_size, kg = it.key0 + j;
-        seen = row < pg.y && (kg < vis.x || (kg >= vis.y && kg < vis.z));
+        seen = row < (pg.y & 255) && (kg < vis.x || (kg >= vis.y && kg < vis.z));
         if (seen) {
           const char* tile = reinterpret_cast<const char*>(k_pool) + ((size_t)pg.x * n_kv_heads + it.kv_head) * tb;
           float dot = 0.f;

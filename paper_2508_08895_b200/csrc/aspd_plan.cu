@@ -2,6 +2,7 @@
 // Eq. 4 and Section 3.3), the split-K work list, plan life cycle and the C entry points.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -252,9 +253,17 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   int64_t kv_tokens = 0;
   {
     int t = 0;
-    auto push_region = [&](const aspd_request_t& q, int slot0, int len) {
-      for (int s0 = 0; s0 < len; s0 += ps)
-        visit.push_back(make_int2(page_ids[q.page_begin + (slot0 + s0) / ps], std::min(ps, len - s0)));
+    // new_key0 / new_tok0: the keys [new_key0, len) of the region are this step's new tokens
+    // new_tok0, new_tok0 + 1, ...; a page entry carries (valid rows | new rows << 8 | first new
+    // token << 13) so that a fused step can write those rows just before it reads the page.
+    auto push_region = [&](const aspd_request_t& q, int slot0, int len, int new_key0, int new_tok0) {
+      for (int s0 = 0; s0 < len; s0 += ps) {
+        const int nv = std::min(ps, len - s0), first_new = std::max(s0, new_key0);
+        const int n_newrows = std::max(0, s0 + nv - first_new);
+        int y = nv;
+        if (n_newrows > 0) y |= (n_newrows << 8) | ((new_tok0 + first_new - new_key0) << 13);
+        visit.push_back(make_int2(page_ids[q.page_begin + (slot0 + s0) / ps], y));
+      }
       kv_tokens += len;
     };
     for (int r = 0; r < n_req; ++r) {
@@ -265,23 +274,23 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
         int nq = 0;
         for (int b = 0; b < q.n_branches; ++b) nq += br[q.branch_begin + b].q_len;
         if (nq > 0) {
-          push_region(q, 0, q.prefix_len);
+          push_region(q, 0, q.prefix_len, q.prefix_len, 0);
           const int pe = ((int)visit.size() - visit0[r]) * ps;
           for (int b = 0; b < q.n_branches; ++b) {
             const aspd_branch_t& x = br[q.branch_begin + b];
             if (x.q_len == 0) continue;
             const int lo = ((int)visit.size() - visit0[r]) * ps;
-            push_region(q, x.kv_off, x.kv_len);
+            push_region(q, x.kv_off, x.kv_len, x.kv_len - x.q_len, t);
             for (int i = 0; i < x.q_len; ++i) tok_vis[t++] = make_int4(pe, lo, lo + x.kv_len - x.q_len + i + 1, 0);
           }
         }
       } else {
-        push_region(q, 0, q.prefix_len);
+        push_region(q, 0, q.prefix_len, q.prefix_len, 0);
         for (int b = 0; b < q.n_branches; ++b) {
           const aspd_branch_t& x = br[q.branch_begin + b];
-          push_region(q, x.kv_off, x.kv_len);
+          push_region(q, x.kv_off, x.kv_len, x.kv_len, 0);
         }
-        push_region(q, q.tail_off, q.tail_len);
+        push_region(q, q.tail_off, q.tail_len, q.tail_len - 1, t);
         tok_vis[t++] = make_int4(kCausalAll, 0, 0, 0);
       }
     }
@@ -314,27 +323,49 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   p->chunk_tokens = tune.chunk_tokens; p->n_ctas = n_ctas;
   std::vector<int32_t> n_parts((size_t)n_new * Hkv, 0), part_base((size_t)n_new * Hkv + 1, 0), cta_item0(n_ctas + 1, 0);
   {
-    long g0 = 0;                                 // global page offset of the current stream
+    // Every CTA gets the same cost, cost = pages + kItemCost per item it starts: an item boundary
+    // (new query tile, ragged last tile, epilogue) costs about as much as streaming a dozen pages,
+    // so CTAs that end up with several short items get fewer pages.
+    const char* ice = getenv("ASPD_ITEM_COST");
+    const double kItemCost = ice ? atof(ice) : 12.0;
+    const double share = ((double)total_pages + kItemCost * ((double)streams.size() + n_ctas)) / n_ctas;
     int cta = 0;
-    auto boundary = [&](int c) { return (long)c * total_pages / n_ctas; };
+    double acc = 0.0;                              // cost already given to the current CTA
     for (const Stream& st : streams) {
       int at = 0, slot = 0;
       while (at < st.n_pages) {
-        while (cta + 1 < n_ctas && boundary(cta + 1) <= g0 + at) cta_item0[++cta] = (int)p->items.size();
-        long stop = std::min<long>(st.n_pages, at + chunk_pages);
-        if (cta + 1 <= n_ctas) stop = std::min<long>(stop, std::max<long>(boundary(cta + 1) - g0, at + 1));
+        double room = share - acc - kItemCost;     // pages that still fit if an item starts here
+        if (room < 1.0 && acc > 0.0 && cta + 1 < n_ctas) { cta_item0[++cta] = (int)p->items.size(); acc = 0.0; continue; }
+        long take = std::min<long>(st.n_pages - at, chunk_pages);
+        if (cta + 1 < n_ctas) take = std::min<long>(take, std::max<long>(1, (long)(room + 0.5)));
         DeviceItem it;
         it.q_tok0 = st.tok0; it.n_q_tok = st.n_tok; it.kv_head = st.head; it.page0 = st.page0 + at;
-        it.n_pages = (int)stop - at; it.key0 = at * ps; it.part_slot = slot++; it.request = st.request;
+        it.n_pages = (int)take; it.key0 = at * ps; it.part_slot = slot++; it.request = st.request;
         it.row_block = st.row_block; it.reserved = 0;
         p->items.push_back(it);
-        at = (int)stop;
+        at += (int)take;
+        acc += kItemCost + (double)take;
+        if (acc >= share - 0.5 && cta + 1 < n_ctas) { cta_item0[++cta] = (int)p->items.size(); acc = 0.0; }
       }
       for (int i = 0; i < st.n_tok; ++i) n_parts[(size_t)(st.tok0 + i) * Hkv + st.head] = slot;
-      g0 += st.n_pages;
     }
     while (cta < n_ctas) cta_item0[++cta] = (int)p->items.size();
   }
+  // rows that are new this step, per CTA: what a fused step must write before the CTA reads
+  std::vector<int4> dirty;
+  std::vector<int32_t> cta_dirty0(n_ctas + 1, 0);
+  for (int c = 0; c < n_ctas; ++c) {
+    cta_dirty0[c] = (int)dirty.size();
+    for (int i = cta_item0[c]; i < cta_item0[c + 1]; ++i) {
+      const DeviceItem& it = p->items[i];
+      for (int pg = 0; pg < it.n_pages; ++pg) {
+        const int2 v = visit[it.page0 + pg];
+        const int cnt = (v.y >> 8) & 31, tok0 = v.y >> 13, row0 = (v.y & 255) - cnt;
+        for (int k = 0; k < cnt; ++k) dirty.push_back(make_int4(v.x, it.kv_head, tok0 + k, row0 + k));
+      }
+    }
+  }
+  cta_dirty0[n_ctas] = (int)dirty.size();
   for (size_t i = 0; i < n_parts.size(); ++i) part_base[i + 1] = part_base[i] + n_parts[i];
   p->n_items = (int)p->items.size();
   p->n_partials = part_base[n_parts.size()];
@@ -352,8 +383,11 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   const size_t o_items = take(sizeof(DeviceItem) * std::max(1, p->n_items));
   const size_t o_cta = take(sizeof(int32_t) * (n_ctas + 1));
   const size_t o_visit = take(sizeof(int2) * std::max<size_t>(1, visit.size()));
+  const size_t o_cdirty = take(sizeof(int32_t) * (n_ctas + 1));
+  const size_t o_dirty = take(sizeof(int4) * std::max<size_t>(1, dirty.size()));
   const size_t o_tpage = take(sizeof(int32_t) * std::max(1, n_new));
   const size_t o_trow = take(sizeof(int32_t) * std::max(1, n_new));
+  const size_t o_tpos = take(sizeof(int32_t) * std::max(1, n_new));
   const size_t o_tvis = take(sizeof(int4) * std::max(1, n_new));
   const size_t o_rb = take(sizeof(int2) * std::max<size_t>(1, row_blocks.size()));
   const size_t o_qcs = take(sizeof(float2) * std::max(1, n_new) * (d / 2));
@@ -374,9 +408,12 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   if (p->n_items) memcpy(blob.data() + o_items, p->items.data(), sizeof(DeviceItem) * p->n_items);
   memcpy(blob.data() + o_cta, cta_item0.data(), sizeof(int32_t) * (n_ctas + 1));
   if (!visit.empty()) memcpy(blob.data() + o_visit, visit.data(), sizeof(int2) * visit.size());
+  memcpy(blob.data() + o_cdirty, cta_dirty0.data(), sizeof(int32_t) * (n_ctas + 1));
+  if (!dirty.empty()) memcpy(blob.data() + o_dirty, dirty.data(), sizeof(int4) * dirty.size());
   if (n_new) {
     memcpy(blob.data() + o_tpage, tok_page.data(), sizeof(int32_t) * n_new);
     memcpy(blob.data() + o_trow, tok_row.data(), sizeof(int32_t) * n_new);
+    memcpy(blob.data() + o_tpos, pos.data(), sizeof(int32_t) * n_new);
     memcpy(blob.data() + o_tvis, tok_vis.data(), sizeof(int4) * n_new);
   }
   if (!row_blocks.empty()) memcpy(blob.data() + o_rb, row_blocks.data(), sizeof(int2) * row_blocks.size());
@@ -402,11 +439,14 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   p->dev.items = (const DeviceItem*)(b8 + o_items);
   p->dev.cta_item0 = (const int32_t*)(b8 + o_cta);
   p->dev.visit = (const int2*)(b8 + o_visit);
+  p->dev.cta_dirty0 = (const int32_t*)(b8 + o_cdirty);
+  p->dev.dirty = (const int4*)(b8 + o_dirty);
   p->dev.tok_vis = (const int4*)(b8 + o_tvis);
   p->dev.row_blocks = (const int2*)(b8 + o_rb);
 
   p->dev.tok_page = (const int32_t*)(b8 + o_tpage);
   p->dev.tok_row = (const int32_t*)(b8 + o_trow);
+  p->dev.tok_pos = (const int32_t*)(b8 + o_tpos);
   p->dev.q_cs = (const float2*)(b8 + o_qcs);
   p->dev.part_base = (const int32_t*)(b8 + o_pbase);
   p->dev.inv_freq = (const double*)(b8 + o_freq);
@@ -448,7 +488,7 @@ int aspd_plan_items(const aspd_plan_t* p, aspd_item_t* items, int max_items) {
 int aspd_plan_stream_pages(const aspd_plan_t* p, int32_t* page_ids, int32_t* n_valid, int max_pages) {
   if (!p || max_pages < 0 || (max_pages > 0 && (!page_ids || !n_valid))) return ASPD_ERR_INVALID_ARG;
   const int n = std::min<int>(max_pages, (int)p->visit.size());
-  for (int i = 0; i < n; ++i) { page_ids[i] = p->visit[i].x; n_valid[i] = p->visit[i].y; }
+  for (int i = 0; i < n; ++i) { page_ids[i] = p->visit[i].x; n_valid[i] = p->visit[i].y & 255; }
   return (int)p->visit.size();
 }
 
@@ -510,6 +550,33 @@ int aspd_serial_attn(aspd_plan_t* p, const void* q, const void* k_pool, const vo
   return run_attn(p, ASPD_MODE_SERIAL, q, k_pool, v_pool, out, stream);
 }
 
+static int run_step(aspd_plan_t* p, int mode, const void* q, const void* k_new, const void* v_new, void* k_pool,
+                    void* v_pool, void* out, void* stream) {
+  if (!p || p->host_only || p->mode != mode) return ASPD_ERR_INVALID_ARG;
+  if (p->n_new == 0) return ASPD_OK;
+  if (!q || !k_new || !v_new || !k_pool || !v_pool || !out) return ASPD_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  int rc;
+  if (p->kernel == ASPD_KERNEL_MMA) {
+    rc = launch_attn_mma_step(p, q, k_new, v_new, k_pool, v_pool, s);
+  } else {
+    rc = launch_append(p, k_new, v_new, p->dev.tok_pos, k_pool, v_pool, s);
+    if (rc == ASPD_OK) rc = launch_attn_generic(p, q, k_pool, v_pool, s);
+  }
+  if (rc) return rc;
+  return launch_combine(p, out, s);
+}
+
+int aspd_branch_step(aspd_plan_t* p, const void* q, const void* k_new, const void* v_new, void* k_pool, void* v_pool,
+                     void* out, void* stream) {
+  return run_step(p, ASPD_MODE_BRANCH, q, k_new, v_new, k_pool, v_pool, out, stream);
+}
+
+int aspd_serial_step(aspd_plan_t* p, const void* q, const void* k_new, const void* v_new, void* k_pool, void* v_pool,
+                     void* out, void* stream) {
+  return run_step(p, ASPD_MODE_SERIAL, q, k_new, v_new, k_pool, v_pool, out, stream);
+}
+
 int aspd_step_host(aspd_plan_t* p, const void* q, const void* k_new, const void* v_new, const int32_t* pos,
                    void* k_pool, void* v_pool, void* out, void* stream) {
   if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
@@ -531,6 +598,19 @@ int aspd_step_host(aspd_plan_t* p, const void* q, const void* k_new, const void*
   if (cudaMemcpyAsync(out, p->dev.st_out, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return ASPD_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return ASPD_ERR_CUDA;
   return ASPD_OK;
+}
+
+int aspd_debug_bounded_wait(int64_t limit_cycles, int32_t* status_out, void* stream) {
+  if (!status_out || limit_cycles < 0 || limit_cycles > 4000000000LL) return ASPD_ERR_INVALID_ARG;
+  int32_t* dev = nullptr;
+  if (cudaMalloc(&dev, sizeof(int32_t)) != cudaSuccess) return ASPD_ERR_NOMEM;
+  cudaStream_t s = (cudaStream_t)stream;
+  int rc = launch_wait_probe(limit_cycles, dev, s);
+  if (rc == ASPD_OK && (cudaMemcpyAsync(status_out, dev, sizeof(int32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+                        cudaStreamSynchronize(s) != cudaSuccess))
+    rc = ASPD_ERR_CUDA;
+  cudaFree(dev);
+  return rc;
 }
 
 int aspd_debug_read_token(const aspd_shape_t* shape, const void* pool, int64_t page, int row, int kv_head, float* out,

@@ -45,8 +45,9 @@ class WorkloadRun:
     """Runs the phases of a workload through kv_append + attention, keeping compared outputs."""
 
     def __init__(self, wl: W.Workload, kernel: int = B.KERNEL_AUTO, chunk_tokens: int = 0, n_ctas: int = 0,
-                 device="cuda"):
+                 device="cuda", fused: bool = False):
         self.wl, self.kernel, self.chunk_tokens, self.n_ctas, self.device = wl, kernel, chunk_tokens, n_ctas, device
+        self.fused = fused          # attention phases go through aspd_branch_step / aspd_serial_step
         self.shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
         self.cache = LayerCache(self.shape, wl.n_pool_pages, device)
         self.outputs: List[np.ndarray] = []
@@ -63,11 +64,19 @@ class WorkloadRun:
         if plan.n_new > 0:
             pos_d = torch.from_numpy(pos.copy()).to(self.device)
             k_d, v_d = to_device(ph.k_new, wl.dtype, self.device), to_device(ph.v_new, wl.dtype, self.device)
-            B.kv_append(plan, k_d, v_d, pos_d, self.cache.k, self.cache.v)
-            if attend and ph.q is not None:
+            do_attn = attend and ph.q is not None
+            if do_attn and self.fused:
                 q_d = to_device(ph.q, wl.dtype, self.device)
                 out_d = torch.empty_like(q_d)
-                (B.branch_attn if ph.mode == W.MODE_BRANCH else B.serial_attn)(plan, q_d, self.cache.k, self.cache.v, out_d)
+                (B.branch_step if ph.mode == W.MODE_BRANCH else B.serial_step)(plan, q_d, k_d, v_d, self.cache.k,
+                                                                               self.cache.v, out_d)
+            else:
+                B.kv_append(plan, k_d, v_d, pos_d, self.cache.k, self.cache.v)
+            if do_attn:
+                if not self.fused:
+                    q_d = to_device(ph.q, wl.dtype, self.device)
+                    out_d = torch.empty_like(q_d)
+                    (B.branch_attn if ph.mode == W.MODE_BRANCH else B.serial_attn)(plan, q_d, self.cache.k, self.cache.v, out_d)
                 torch.cuda.synchronize()
                 st = plan.status()
                 if st != 0:

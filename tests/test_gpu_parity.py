@@ -121,11 +121,13 @@ def test_peaked_softmax_variant():
     assert np.linalg.norm(g - r) / np.linalg.norm(r) <= 1e-2
 
 
-@pytest.mark.parametrize("chunk", [16, 64, 448, 32768])
+@pytest.mark.parametrize("chunk,n_ctas", [(16, 0), (64, 0), (448, 0), (32768, 0), (16, 3), (0, 1), (48, 37)])
 @pytest.mark.parametrize("kernel", KERNELS)
-def test_split_k_counts_agree(chunk, kernel):
+def test_split_k_counts_agree(chunk, n_ctas, kernel):
+    """Forced cuts of the key streams (every `chunk` keys) and forced grid sizes: one item per page,
+    hundreds of items per CTA (beyond what a CTA keeps in shared memory), a single CTA."""
     wl = W.config_long_rag(prefix=1024 + 7)
-    compare_workload(wl, kernel=kernel, chunk_tokens=chunk)
+    compare_workload(wl, kernel=kernel, chunk_tokens=chunk, n_ctas=n_ctas)
 
 
 @pytest.mark.parametrize("kernel", KERNELS)
@@ -270,6 +272,46 @@ def test_step_host_matches_device_path():
     dev = run.step(ph)
     np.testing.assert_array_equal(host, dev)
     check(host, oracle_run(wl).outputs[0], wl.dtype)
+
+
+def test_bounded_wait_gives_up_and_leaves_the_context_usable():
+    """A wait nothing satisfies runs into its limit (about a millisecond here), reports
+    ASPD_ERR_TIMEOUT, and the device keeps working afterwards."""
+    import time
+    import torch
+    t0 = time.perf_counter()
+    assert B.debug_bounded_wait(2_000_000) == -5
+    assert time.perf_counter() - t0 < 5.0
+    x = torch.arange(8, device="cuda")
+    assert int(x.sum().item()) == 28
+    compare_workload(W.config_tiny())
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_fused_step_appends_and_attends_like_the_two_calls(kernel):
+    """aspd_branch_step / aspd_serial_step: same outputs within tolerance, and the rows they write
+    into the cache are the rotated keys and raw values the oracle's append produces."""
+    E = engine()
+    for wl in (W.build_segment_workload("fs", 41, 28, 4, 128, "bf16", 1e6, [15, 300, 0], [[14, 15, 16], [255, 1, 99], [3]],
+                                        [[1, 1, 1], [1, 0, 1], [1]], serial_steps=2),
+               W.config_branch_open(serial_steps=2), W.config_tiny()):
+        ref = oracle_run(wl)
+        run = E.run_workload(wl, kernel=kernel, fused=True)
+        assert len(run.outputs) == len(ref.outputs)
+        for g, r in zip(run.outputs, ref.outputs):
+            check(g, r, wl.dtype, wl.name)
+        rel = 2.0 ** -8 if wl.dtype == "bf16" else 1e-6
+        for ph, (pos, slot, req) in zip(wl.phases, ref.positions):
+            if ph.q is None:
+                continue
+            for t in range(0, len(pos), max(1, len(pos) // 12)):
+                r = int(req[t]); s_ = int(slot[t])
+                page = int(ph.desc["page_ids"][int(ph.desc["page_begin"][r]) + s_ // wl.page_size]); row = s_ % wl.page_size
+                for h in range(wl.Hkv):
+                    np.testing.assert_array_equal(run.read_token("v", page, row, h), ph.v_new[t, h])
+                    want = ref.k_pool[page, h, row]
+                    got = run.read_token("k", page, row, h)
+                    assert np.all(np.abs(got - want) <= rel * np.abs(want) + 1e-6)
 
 
 def test_zero_new_tokens_is_a_no_op():
