@@ -2,7 +2,7 @@
 // head_dim 128, page_size 16.
 //
 // One persistent CTA per SM walks its share of the plan's work items.  An item is (query row
-// block of one KV head, key chunk): M = n_q_tok * G <= 64 query rows against up to chunk keys.
+// block of one KV head, run of pages of the request's key stream): M = n_q_tok * G <= 64 query rows.
 // Keys stream through shared memory in tiles of 128 (8 pages), fetched page by page with
 // linear bulk copies (the cache tile format already is the 128-byte-swizzled image the tensor
 // core reads).  Per tile:
@@ -20,10 +20,12 @@
 // raised when the tile maximum exceeds it by more than 2^8, which keeps P exactly consistent
 // with the (m, l, O) record while making the rescale of O in TMEM rare.
 //
-// Warp roles: 0-3 softmax / epilogue (TMEM lane quadrant = warp), 4 and 7 bulk-copy producers
-// (K and V), 5 MMA issuer (one elected lane), 6 query preparation (RoPE, bf16, swizzled
-// store) one item ahead.  All cross-role hand-offs are mbarriers; every wait is bounded and on expiry sets the
-// plan's status word to ASPD_ERR_TIMEOUT and makes all roles drain and exit.
+// Warp roles: 0-3 softmax (TMEM lane quadrant = warp), 4 and 7 bulk-copy producers (K and V),
+// 5 MMA issuer (one elected lane), 8-11 fused append of the step's new rows (aspd_branch_step /
+// aspd_serial_step), query preparation (RoPE, bf16, swizzled store, one item ahead) and epilogue
+// (TMEM lane quadrant = warp - 8); warp 6 is idle.  All cross-role hand-offs are mbarriers; every
+// wait is bounded and on expiry sets the plan's status word to ASPD_ERR_TIMEOUT and makes all
+// roles drain and exit.
 #include <stdlib.h>
 
 #include "aspd_internal.cuh"
