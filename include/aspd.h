@@ -176,6 +176,9 @@ int aspd_plan_destroy(aspd_plan_t* plan);
 int aspd_plan_info(const aspd_plan_t* plan, aspd_plan_info_t* info /*host*/);
 /* Copy up to max_items work items to `items` (host); returns the number of items. */
 int aspd_plan_items(const aspd_plan_t* plan, aspd_item_t* items, int max_items);
+/* First work item of every CTA of the persistent grid: CTA c owns items [first[c], first[c + 1])
+ * of aspd_plan_items (host array of n_ctas + 1 entries). Returns n_ctas. */
+int aspd_plan_cta_ranges(const aspd_plan_t* plan, int32_t* first /*host*/, int max_entries);
 /* The plan's stream-page list: physical page and number of valid rows of every page the step
  * reads (host arrays of n_stream_pages entries each). */
 int aspd_plan_stream_pages(const aspd_plan_t* plan, int32_t* page_ids /*host*/, int32_t* n_valid /*host*/,

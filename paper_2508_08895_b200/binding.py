@@ -54,7 +54,7 @@ class AspdError(RuntimeError):
 
 
 EXPORTS = ("aspd_strerror", "aspd_pool_bytes", "aspd_count_new_tokens", "aspd_positions", "aspd_visible_slots",
-           "aspd_plan_create", "aspd_plan_destroy", "aspd_plan_info", "aspd_plan_items", "aspd_plan_stream_pages",
+           "aspd_plan_create", "aspd_plan_destroy", "aspd_plan_info", "aspd_plan_items", "aspd_plan_cta_ranges", "aspd_plan_stream_pages",
            "aspd_plan_token_ranges", "aspd_plan_status",
            "aspd_kv_append", "aspd_branch_attn", "aspd_serial_attn", "aspd_attn_partials", "aspd_attn_combine",
            "aspd_branch_step", "aspd_serial_step", "aspd_step_host", "aspd_attn_static", "aspd_debug_read_token", "aspd_debug_bounded_wait")
@@ -85,6 +85,7 @@ def lib() -> ctypes.CDLL:
         L.aspd_plan_destroy.argtypes = [vp]
         L.aspd_plan_info.argtypes = [vp, vp]
         L.aspd_plan_items.argtypes = [vp, vp, ci]
+        L.aspd_plan_cta_ranges.argtypes = [vp, vp, ci]
         L.aspd_plan_stream_pages.argtypes = [vp, vp, vp, ci]
         L.aspd_plan_token_ranges.argtypes = [vp, vp, vp, vp, ci]
         L.aspd_plan_status.argtypes = [vp, vp]
@@ -208,6 +209,12 @@ class Plan:
         items = np.zeros(max(self.info.n_items, 1), dtype=ITEM_DTYPE)
         _check(lib().aspd_plan_items(self._h, _ptr(items), self.info.n_items), "aspd_plan_items")
         return items[: self.info.n_items]
+
+    def cta_ranges(self) -> np.ndarray:
+        """first[c] .. first[c + 1]: the items CTA c of the persistent grid owns."""
+        first = np.zeros(self.info.n_ctas + 1, np.int32)
+        _check(lib().aspd_plan_cta_ranges(self._h, _ptr(first), len(first)), "aspd_plan_cta_ranges")
+        return first
 
     def stream_pages(self):
         """(physical page, valid rows) of every page the step reads, as two int32 arrays."""

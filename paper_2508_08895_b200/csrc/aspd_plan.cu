@@ -328,14 +328,21 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
     // so CTAs that end up with several short items get fewer pages.
     const char* ice = getenv("ASPD_ITEM_COST");
     const double kItemCost = ice ? atof(ice) : 12.0;
-    const double share = ((double)total_pages + kItemCost * ((double)streams.size() + n_ctas)) / n_ctas;
+    // the share is re-derived from what is left whenever a CTA is closed, so rounding does not pile up
+    long pages_left = total_pages, streams_left = (long)streams.size();
+    auto share_now = [&](int ctas_left) {
+      return ((double)pages_left + kItemCost * ((double)streams_left + ctas_left)) / std::max(1, ctas_left);
+    };
+    double share = share_now(n_ctas);
     int cta = 0;
     double acc = 0.0;                              // cost already given to the current CTA
+    auto next_cta = [&]() { cta_item0[++cta] = (int)p->items.size(); acc = 0.0; share = share_now(n_ctas - cta); };
     for (const Stream& st : streams) {
       int at = 0, slot = 0;
+      --streams_left;
       while (at < st.n_pages) {
         double room = share - acc - kItemCost;     // pages that still fit if an item starts here
-        if (room < 1.0 && acc > 0.0 && cta + 1 < n_ctas) { cta_item0[++cta] = (int)p->items.size(); acc = 0.0; continue; }
+        if (room < 1.0 && acc > 0.0 && cta + 1 < n_ctas) { next_cta(); continue; }
         long take = std::min<long>(st.n_pages - at, chunk_pages);
         if (cta + 1 < n_ctas) take = std::min<long>(take, std::max<long>(1, (long)(room + 0.5)));
         DeviceItem it;
@@ -344,8 +351,9 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
         it.row_block = st.row_block; it.reserved = 0;
         p->items.push_back(it);
         at += (int)take;
+        pages_left -= take;
         acc += kItemCost + (double)take;
-        if (acc >= share - 0.5 && cta + 1 < n_ctas) { cta_item0[++cta] = (int)p->items.size(); acc = 0.0; }
+        if (acc >= share - 0.5 && cta + 1 < n_ctas) next_cta();
       }
       for (int i = 0; i < st.n_tok; ++i) n_parts[(size_t)(st.tok0 + i) * Hkv + st.head] = slot;
     }
@@ -483,6 +491,13 @@ int aspd_plan_items(const aspd_plan_t* p, aspd_item_t* items, int max_items) {
   static_assert(sizeof(aspd_item_t) == sizeof(DeviceItem) && sizeof(DeviceItem) == 40, "item layouts must match");
   if (n) memcpy(items, p->items.data(), sizeof(DeviceItem) * n);
   return p->n_items;
+}
+
+int aspd_plan_cta_ranges(const aspd_plan_t* p, int32_t* first, int max_entries) {
+  if (!p || max_entries < 0 || (max_entries > 0 && !first)) return ASPD_ERR_INVALID_ARG;
+  const int n = std::min<int>(max_entries, (int)p->cta_item0.size());
+  for (int i = 0; i < n; ++i) first[i] = p->cta_item0[i];
+  return p->n_ctas;
 }
 
 int aspd_plan_stream_pages(const aspd_plan_t* p, int32_t* page_ids, int32_t* n_valid, int max_pages) {

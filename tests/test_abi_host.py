@@ -140,6 +140,11 @@ def test_streams_are_cut_into_equal_shares():
         total = int(items["n_pages"].sum())
         assert total == plan.info.n_stream_pages * wl.Hkv
         assert plan.info.n_ctas == n_ctas
+        first = plan.cta_ranges()
+        assert first[0] == 0 and first[-1] == len(items) and (np.diff(first) >= 0).all()
+        pages = np.array([int(items['n_pages'][first[c]:first[c + 1]].sum()) for c in range(n_ctas)])
+        if n_ctas > 1:
+            assert pages.max() - pages.min() <= 0.35 * pages.mean() + 16     # cost-balanced, not page-balanced
         # the items, in order, tile the concatenated streams; cutting it into n_ctas contiguous
         # shares of (almost) equal size never needs more than one extra item per share
         assert len(items) <= 3 * wl.Hkv + n_ctas
