@@ -216,7 +216,10 @@ def run_ours(args):
         del k_d, v_d
 
     ph = wl.phases[-1]
-    plan = B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode, kernel=kernel, chunk_tokens=args.chunk, n_ctas=args.ctas)
+    # decode loop: a layer's pools are written only by that layer's own step, so the plan may carry
+    # the stable-cache promise (the kernel starts fetching before the previous layer's combine ends)
+    plan = B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode, kernel=kernel, chunk_tokens=args.chunk, n_ctas=args.ctas,
+                  stable_cache=not args.no_stable_cache)
     pos, _, _ = B.positions(ph.desc, ph.mode)
     n_new = plan.n_new
     pos_d = torch.from_numpy(pos.copy()).cuda()
@@ -334,7 +337,7 @@ def run_ours(args):
                        "page_size": wl.page_size, "kernel": {1: "generic", 2: "mma"}[info.kernel],
                        "chunk_tokens": info.chunk_tokens, "work_items": info.n_items, "n_ctas": info.n_ctas,
                        "l2": "footprint %.1f GB of distinct K/V pools per step, far above L2" % (alg * L / 1e9),
-                       "layers_agree": bool(same), "cuda_graph": not args.no_graph,
+                       "layers_agree": bool(same), "cuda_graph": not args.no_graph, "stable_cache": not args.no_stable_cache,
                        "calls_per_layer": "aspd_branch_step (append fused into the attention pass) -> combine" if fused
                        else "aspd_kv_append -> aspd_branch_attn"},
             "hbm_gbs": alg * L * args.steps / (ms * 1e-3) / 1e9,
@@ -379,6 +382,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--separate-append", action="store_true",
                     help="call aspd_kv_append and aspd_branch_attn separately instead of aspd_branch_step")
+    ap.add_argument("--no-stable-cache", action="store_true", help="create the plan without the stable-cache promise")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":

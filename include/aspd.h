@@ -92,6 +92,13 @@ typedef struct {
   int32_t n_ctas;       /* size of the persistent grid; 0 = auto                           */
   int32_t host_only;    /* 1: build the work list on the host only (no CUDA call at all);
                            such a plan serves aspd_plan_info / aspd_plan_items only        */
+  int32_t stable_cache; /* 1: the caller promises that, when an attention call of this plan is
+                           made, nothing still in flight on the stream writes K/V pages the plan
+                           reads, except this step's own new rows (written by aspd_kv_append with
+                           this plan, or by the fused step).  True for a decode loop, where a
+                           layer's pools are only touched by that layer's own step.  The kernel
+                           may then start fetching such pages before the previous kernel on the
+                           stream has finished.  0 (default): full stream ordering for the pools */
 } aspd_tuning_t;
 
 /* One split-K work item of a plan, as aspd_plan_items reports it.  The pages a request's

@@ -36,7 +36,7 @@ class Shape(ctypes.Structure):
 
 class Tuning(ctypes.Structure):
     _fields_ = [("kernel", ctypes.c_int32), ("chunk_tokens", ctypes.c_int32), ("n_ctas", ctypes.c_int32),
-                ("host_only", ctypes.c_int32)]
+                ("host_only", ctypes.c_int32), ("stable_cache", ctypes.c_int32)]
 
 
 class PlanInfo(ctypes.Structure):
@@ -190,10 +190,10 @@ class Plan:
     """Owner of an ``aspd_plan_t`` (see ``aspd_plan_create``)."""
 
     def __init__(self, shape: Shape, desc, n_pool_pages: int, mode: int, q_pos=None, kernel: int = KERNEL_AUTO,
-                 chunk_tokens: int = 0, n_ctas: int = 0, host_only: bool = False, stream=None):
+                 chunk_tokens: int = 0, n_ctas: int = 0, host_only: bool = False, stable_cache: bool = False, stream=None):
         self.shape, self.mode = shape, mode
         req, br, pages = pack_descriptors(desc)
-        tune = Tuning(kernel, chunk_tokens, n_ctas, 1 if host_only else 0)
+        tune = Tuning(kernel, chunk_tokens, n_ctas, 1 if host_only else 0, 1 if stable_cache else 0)
         qp = None if q_pos is None else np.ascontiguousarray(q_pos, dtype=np.int32)
         handle = ctypes.c_void_p()
         self._h = None

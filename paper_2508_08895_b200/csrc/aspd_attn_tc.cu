@@ -197,6 +197,7 @@ struct Ctx {
   const char* v_pool;
   int n_items, n_q_heads, n_kv_heads;
   float scale_log2;
+  int early_fetch;             // plan promise: pages without new rows are not written by in-flight work
 };
 
 // Item idx of this CTA (rel = idx - item_begin): from the shared-memory cache when it is there.
@@ -481,8 +482,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     }
   }
   // everything above touches only the plan's own tables; inputs written by earlier kernels of
-  // the stream (q, k_new, the pools, the workspace's previous readers) are used from here on
-  pdl_wait();
+  // the stream (q, k_new, the pools, the workspace's previous readers) are used from here on.
+  // With the plan's stable-cache promise the two producer warps go ahead and fetch pages that
+  // hold no new rows; they wait themselves before the first page that does.
+  const bool producer_runs_ahead = c.early_fetch && (warp == 4 || warp == 7);
+  if (!producer_runs_ahead) pdl_wait();
   if (tid == 0) ASPD_CTA_STAMP(c, 1);
 
   if (warp < 4) {
@@ -505,7 +509,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     const int kv = warp == 4 ? 0 : 1;
     const char* pool = kv ? c.v_pool : c.k_pool;
     int g = 0;
-    bool ok = true, appended = false;
+    bool ok = true, appended = false, waited = false;
     // (item, batch of 32 pages) pairs are walked as one sequence: `cur` holds the batch being
     // consumed, `nxt` the one after it, which may already belong to the next item.
     int2 nxt = make_int2(0, 0);
@@ -534,6 +538,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
         pg.x = __shfl_sync(0xffffffffu, cur.x, (t & 3) * 8 + (lane & 7));
         pg.y = __shfl_sync(0xffffffffu, cur.y, (t & 3) * 8 + (lane & 7));
         if (lane >= npg) pg = make_int2(0, 0);
+        if (producer_runs_ahead && !waited && __any_sync(0xffffffffu, ((pg.y >> 8) & 31) != 0)) {
+          pdl_wait();                                  // new rows come from the previous kernel (or from this one)
+          waited = true;
+        }
         if (c.k_new != nullptr && !appended && __any_sync(0xffffffffu, ((pg.y >> 8) & 31) != 0)) {
           // fused append: this tile holds rows that are new this step; the append warp has written
           // (or is writing) them -- wait for it once, before the first such page is copied
@@ -748,6 +756,7 @@ static int launch_tc(const aspd_plan* p, const void* q, const void* k_new, const
   c.n_q_heads = sh.n_q_heads;
   c.n_kv_heads = sh.n_kv_heads;
   c.scale_log2 = sh.sm_scale * kLog2e;
+  c.early_fetch = p->stable_cache;
   return launch_pdl(kPdlAttn, attn_tc_kernel, dim3(p->n_ctas), dim3(kThreads), kSmemBytes, s, c) == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
 }
 

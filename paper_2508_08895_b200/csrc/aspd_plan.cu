@@ -204,7 +204,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   const int n_new = aspd_count_new_tokens(req, br, n_req, mode);
   if (n_new < 0) return n_new;
 
-  aspd_tuning_t tune = {ASPD_KERNEL_AUTO, 0, 0, 0};
+  aspd_tuning_t tune = {ASPD_KERNEL_AUTO, 0, 0, 0, 0};
   if (tuning) tune = *tuning;
   const int ps = shape->page_size, d = shape->head_dim, Hq = shape->n_q_heads, Hkv = shape->n_kv_heads;
   const int G = Hq / Hkv, es = esize_of(shape->dtype);
@@ -218,6 +218,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   aspd_plan* p = new (std::nothrow) aspd_plan();
   if (!p) return ASPD_ERR_NOMEM;
   p->shape = *shape; p->mode = mode; p->n_req = n_req; p->n_new = n_new; p->kernel = kernel;
+  p->stable_cache = tune.stable_cache ? 1 : 0;
   p->host_only = tune.host_only; p->n_pool_pages = n_pool_pages; p->device_base = nullptr; p->device_bytes = 0;
   memset(&p->dev, 0, sizeof(p->dev));
   p->sm_count = 148;

@@ -45,8 +45,9 @@ class WorkloadRun:
     """Runs the phases of a workload through kv_append + attention, keeping compared outputs."""
 
     def __init__(self, wl: W.Workload, kernel: int = B.KERNEL_AUTO, chunk_tokens: int = 0, n_ctas: int = 0,
-                 device="cuda", fused: bool = False):
+                 device="cuda", fused: bool = False, stable_cache: bool = False):
         self.wl, self.kernel, self.chunk_tokens, self.n_ctas, self.device = wl, kernel, chunk_tokens, n_ctas, device
+        self.stable_cache = stable_cache
         self.fused = fused          # attention phases go through aspd_branch_step / aspd_serial_step
         self.shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
         self.cache = LayerCache(self.shape, wl.n_pool_pages, device)
@@ -57,7 +58,7 @@ class WorkloadRun:
     def step(self, ph: W.Phase, attend: bool = True, keep_plan: bool = False) -> Optional[np.ndarray]:
         wl = self.wl
         plan = B.Plan(self.shape, ph.desc, wl.n_pool_pages, ph.mode, kernel=self.kernel,
-                      chunk_tokens=self.chunk_tokens, n_ctas=self.n_ctas)
+                      chunk_tokens=self.chunk_tokens, n_ctas=self.n_ctas, stable_cache=self.stable_cache)
         pos, slot, req = B.positions(ph.desc, ph.mode)
         self.positions.append((pos, slot, req))
         out = None

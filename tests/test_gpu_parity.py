@@ -314,6 +314,17 @@ def test_fused_step_appends_and_attends_like_the_two_calls(kernel):
                     assert np.all(np.abs(got - want) <= rel * np.abs(want) + 1e-6)
 
 
+@pytest.mark.parametrize("fused", [False, True])
+def test_stable_cache_promise_changes_nothing_but_timing(fused):
+    """With aspd_tuning_t.stable_cache the producers fetch pages that hold no new rows before the
+    previous kernel on the stream has finished; results are the same."""
+    for wl in (W.config_serving_mix(n_req=6), W.config_branch_open(serial_steps=3)):
+        run, ref = compare_workload(wl, fused=fused, stable_cache=True)
+        base = engine().run_workload(wl, fused=fused)
+        for a, b in zip(run.outputs, base.outputs):
+            np.testing.assert_array_equal(a, b)
+
+
 def test_zero_new_tokens_is_a_no_op():
     E = engine()
     wl = W.build_segment_workload("e", 8, 28, 4, 128, "bf16", 1e6, [20], [[5, 9]], [[1, 1]])
