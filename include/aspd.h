@@ -52,6 +52,9 @@ typedef enum {
 
 enum { ASPD_MODE_BRANCH = 0, ASPD_MODE_SERIAL = 1 };
 enum { ASPD_DTYPE_F32 = 0, ASPD_DTYPE_BF16 = 1 };
+/* aspd_branch_t.q_len of a region that belongs to an EARLIER stage (a merged branch, or the serial
+ * tokens written between two parallel stages): every token of the step sees all of it. */
+enum { ASPD_Q_SHARED = -1 };
 enum { ASPD_KERNEL_AUTO = 0, ASPD_KERNEL_GENERIC = 1, ASPD_KERNEL_MMA = 2 };
 
 /* One request (host memory).  Logical slot s of the request lives in physical page
@@ -71,8 +74,11 @@ typedef struct {
 typedef struct {
   int32_t kv_off;    /* first logical slot of the branch (page-aligned)                     */
   int32_t kv_len;    /* tokens of the branch in the cache AFTER this step's append          */
-  int32_t pos_start; /* position ID of the branch's first token; Eq. 4 gives prefix_len     */
-  int32_t q_len;     /* query tokens this step = the LAST q_len tokens (0: finished branch) */
+  int32_t pos_start; /* position ID of the branch's first token; Eq. 4 gives the number of tokens
+                        before the stage: prefix_len plus the lengths of all ASPD_Q_SHARED regions */
+  int32_t q_len;     /* query tokens this step = the LAST q_len tokens (0: finished branch of the
+                        current stage, invisible to the other branches; ASPD_Q_SHARED: region of an
+                        earlier stage, visible to every branch -- Eq. 3, different stages)       */
 } aspd_branch_t;
 
 typedef struct {

@@ -121,7 +121,7 @@ def n_new_tokens(desc, mode: int) -> int:
     n = 0
     for r in range(len(d["prefix_len"])):
         b0 = int(d["branch_begin"][r])
-        n += int(d["br_q_len"][b0:b0 + int(d["n_branches"][r])].sum())
+        n += int(np.clip(d["br_q_len"][b0:b0 + int(d["n_branches"][r])], 0, None).sum())
     return n
 
 

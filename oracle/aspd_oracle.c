@@ -211,7 +211,12 @@ int aspd_oracle_dense_attn(int L, int Hq, int Hkv, int d, double theta,
  * and a branch b by
  *   br_kv_off[b]     first logical slot of the branch
  *   br_kv_len[b]     tokens of the branch in the cache AFTER this step's append
- *   br_q_len[b]      query tokens of the branch this step = its LAST q_len tokens
+ *   br_q_len[b]      query tokens of the branch this step = its LAST q_len tokens;
+ *                    0: a branch of the current stage that has finished (invisible to the others);
+ *                    -1: a region of an EARLIER stage (a merged branch, or serial tokens written
+ *                    between two parallel stages): Eq. 3's third case makes it visible to every
+ *                    token of the current stage (the engine switches between serial and parallel
+ *                    stages repeatedly, Section 3.3)
  *
  * mode 0 (parallel step): the new tokens are, request-major then branch-major,
  * the last q_len tokens of every branch.  mode 1 (serial step): one new token
@@ -235,12 +240,15 @@ int aspd_oracle_new_tokens(int n_req, int mode, const int* prefix_len,
   for (int r = 0; r < n_req; ++r) {
     int P = prefix_len[r];
     if (mode == MODE_BRANCH) {
+      int stage_start = P;                        /* tokens before the stage: prefix + earlier stages */
+      for (int b = 0; b < n_branches[r]; ++b)
+        if (br_q_len[branch_begin[r] + b] == -1) stage_start += br_kv_len[branch_begin[r] + b];
       for (int b = 0; b < n_branches[r]; ++b) {
         int B = branch_begin[r] + b;
         for (int i = 0; i < br_q_len[B]; ++i) {
           int k = br_kv_len[B] - br_q_len[B] + i; /* index inside the branch */
           if (k < 0) return ORACLE_BAD;
-          pos_out[n] = P + k;                     /* stage_start + delta     */
+          pos_out[n] = stage_start + k;           /* stage_start + delta     */
           slot_out[n] = br_kv_off[B] + k;
           req_out[n] = r;
           ++n;
@@ -315,11 +323,12 @@ int aspd_oracle_attn(int n_req, int mode, int Hq, int Hkv, int d,
   int cap = 0;
   for (int r = 0; r < n_req; ++r) {
     if (mode == MODE_SERIAL) cap += 1;
-    else for (int b = 0; b < n_branches[r]; ++b) cap += br_q_len[branch_begin[r] + b];
+    else for (int b = 0; b < n_branches[r]; ++b) cap += br_q_len[branch_begin[r] + b] > 0 ? br_q_len[branch_begin[r] + b] : 0;
   }
   int* t_req = (int*)malloc(sizeof(int) * (cap + 1));
   int* t_br = (int*)malloc(sizeof(int) * (cap + 1));
   int* t_k = (int*)malloc(sizeof(int) * (cap + 1));
+  int* t_pos0 = (int*)malloc(sizeof(int) * (cap + 1));   /* stage_start of the token's stage */
   int n = 0;
   long max_keys = 0;
   for (int r = 0; r < n_req; ++r) {
@@ -328,12 +337,15 @@ int aspd_oracle_attn(int n_req, int mode, int Hq, int Hkv, int d,
     total += tail_len ? tail_len[r] : 0;
     if (total > max_keys) max_keys = total;
     if (mode == MODE_SERIAL) {
-      t_req[n] = r; t_br[n] = -1; t_k[n] = 0; ++n;
+      t_req[n] = r; t_br[n] = -1; t_k[n] = 0; t_pos0[n] = 0; ++n;
     } else {
       for (int b = 0; b < n_branches[r]; ++b) {
         int B = branch_begin[r] + b;
         for (int i = 0; i < br_q_len[B]; ++i) {
-          t_req[n] = r; t_br[n] = B; t_k[n] = br_kv_len[B] - br_q_len[B] + i; ++n;
+          int stage_start = prefix_len[r];        /* tokens before the stage: prefix + earlier stages */
+          for (int c = 0; c < n_branches[r]; ++c)
+            if (br_q_len[branch_begin[r] + c] == -1) stage_start += br_kv_len[branch_begin[r] + c];
+          t_req[n] = r; t_br[n] = B; t_k[n] = br_kv_len[B] - br_q_len[B] + i; t_pos0[n] = stage_start; ++n;
         }
       }
     }
@@ -358,13 +370,23 @@ int aspd_oracle_attn(int n_req, int mode, int Hq, int Hkv, int d,
         }
         if (mode == MODE_BRANCH) {
           int B = t_br[t];
+          for (int b = 0; b < n_branches[r]; ++b) {        /* regions of earlier stages */
+            int S = branch_begin[r] + b;
+            if (br_q_len[S] != -1) continue;
+            for (int j = 0; j < br_kv_len[S]; ++j) {
+              int s = br_kv_off[S] + j;
+              keys[m] = cached(k_pool, page_ids, pb, s, h, Hkv, page_size, d);
+              vals[m] = cached(v_pool, page_ids, pb, s, h, Hkv, page_size, d);
+              ++m;
+            }
+          }
           for (int j = 0; j <= t_k[t]; ++j) {
             int s = br_kv_off[B] + j;
             keys[m] = cached(k_pool, page_ids, pb, s, h, Hkv, page_size, d);
             vals[m] = cached(v_pool, page_ids, pb, s, h, Hkv, page_size, d);
             ++m;
           }
-          qpos = P + t_k[t];
+          qpos = t_pos0[t] + t_k[t];
         } else {
           int total = P;
           for (int b = 0; b < n_branches[r]; ++b) {
@@ -392,7 +414,7 @@ int aspd_oracle_attn(int n_req, int mode, int Hq, int Hkv, int d,
       }
     free(keys); free(vals); free(logits); free(qhat);
   }
-  free(t_req); free(t_br); free(t_k);
+  free(t_req); free(t_br); free(t_k); free(t_pos0);
   return fail ? ORACLE_BAD : ORACLE_OK;
 }
 
@@ -417,6 +439,10 @@ int aspd_oracle_visible_slots(int n_req, int mode, int n_slots,
           uint8_t* row = vis_out + (size_t)n * n_slots;
           memset(row, 0, n_slots);
           for (int s = 0; s < P; ++s) row[s] = 1;
+          for (int c = 0; c < n_branches[r]; ++c) {
+            int S = branch_begin[r] + c;
+            if (br_q_len[S] == -1) for (int j = 0; j < br_kv_len[S]; ++j) row[br_kv_off[S] + j] = 1;
+          }
           for (int j = 0; j <= br_kv_len[B] - br_q_len[B] + i; ++j) row[br_kv_off[B] + j] = 1;
           ++n;
         }

@@ -19,6 +19,7 @@ from . import build as _build
 MODE_BRANCH, MODE_SERIAL = 0, 1
 DTYPE_F32, DTYPE_BF16 = 0, 1
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_MMA = 0, 1, 2
+Q_SHARED = -1
 
 REQUEST_DTYPE = np.dtype([(n, np.int32) for n in
                           ("prefix_len", "n_branches", "branch_begin", "page_begin", "n_pages", "tail_off", "tail_len")])
@@ -141,7 +142,7 @@ def make_shape(n_q_heads, n_kv_heads, head_dim, page_size, dtype, rope_theta, sm
 def pack_descriptors(desc: Dict[str, np.ndarray]):
     """dict of int32 arrays -> (aspd_request_t[], aspd_branch_t[], page_ids) numpy arrays.
 
-    A missing ``br_pos_start`` is filled with the request's prefix length, the paper's
+    A missing ``br_pos_start`` is filled with the number of tokens before the stage, the paper's
     shared position-ID rule (Eq. 4: stage_start)."""
     n_req = len(desc["prefix_len"])
     req = np.zeros(n_req, dtype=REQUEST_DTYPE)
@@ -153,9 +154,11 @@ def pack_descriptors(desc: Dict[str, np.ndarray]):
     if "br_pos_start" in desc:
         br["pos_start"] = desc["br_pos_start"]
     else:
+        # Eq. 4, stage_start: tokens before the stage = prefix + every region of an earlier stage
         for r in range(n_req):
-            b0 = int(req["branch_begin"][r])
-            br["pos_start"][b0:b0 + int(req["n_branches"][r])] = req["prefix_len"][r]
+            b0, nb = int(req["branch_begin"][r]), int(req["n_branches"][r])
+            shared = br["q_len"][b0:b0 + nb] == Q_SHARED
+            br["pos_start"][b0:b0 + nb] = req["prefix_len"][r] + int(br["kv_len"][b0:b0 + nb][shared].sum())
     pages = np.ascontiguousarray(desc["page_ids"], dtype=np.int32)
     return req, br, pages
 

@@ -40,7 +40,7 @@ int check_counts(const aspd_request_t* req, const aspd_branch_t* br, int n_req, 
     if (q.n_branches > 0 && !br) return ASPD_ERR_INVALID_ARG;
     for (int b = 0; b < q.n_branches; ++b) {
       const aspd_branch_t& x = br[q.branch_begin + b];
-      if (x.kv_off < 0 || x.kv_len < 0 || x.q_len < 0 || x.q_len > x.kv_len || x.pos_start < 0)
+      if (x.kv_off < 0 || x.kv_len < 0 || x.q_len < ASPD_Q_SHARED || x.q_len > x.kv_len || x.pos_start < 0)
         return ASPD_ERR_BAD_DESCRIPTOR;
     }
     if (mode == ASPD_MODE_SERIAL && q.tail_len < 1) return ASPD_ERR_BAD_DESCRIPTOR;
@@ -119,7 +119,7 @@ int aspd_count_new_tokens(const aspd_request_t* req, const aspd_branch_t* br, in
   long n = 0;
   for (int r = 0; r < n_req; ++r) {
     if (mode == ASPD_MODE_SERIAL) { ++n; continue; }
-    for (int b = 0; b < req[r].n_branches; ++b) n += br[req[r].branch_begin + b].q_len;
+    for (int b = 0; b < req[r].n_branches; ++b) n += std::max(0, br[req[r].branch_begin + b].q_len);
   }
   if (n > (1 << 24)) return ASPD_ERR_TOO_LARGE;
   return (int)n;
@@ -174,6 +174,10 @@ int aspd_visible_slots(const aspd_request_t* req, const aspd_branch_t* br, int n
         const aspd_branch_t& x = br[q.branch_begin + b];
         for (int i = 0; i < x.q_len; ++i, ++t) {
           if (mark(t, 0, q.prefix_len)) return ASPD_ERR_INVALID_ARG;
+          for (int s2 = 0; s2 < q.n_branches; ++s2) {          // regions of earlier stages (Eq. 3, third case)
+            const aspd_branch_t& y = br[q.branch_begin + s2];
+            if (y.q_len == ASPD_Q_SHARED && mark(t, y.kv_off, y.kv_off + y.kv_len)) return ASPD_ERR_INVALID_ARG;
+          }
           if (mark(t, x.kv_off, x.kv_off + x.kv_len - x.q_len + i + 1)) return ASPD_ERR_INVALID_ARG;
         }
       }
@@ -273,13 +277,17 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
       visit0[r] = (int)visit.size();
       if (mode == ASPD_MODE_BRANCH) {
         int nq = 0;
-        for (int b = 0; b < q.n_branches; ++b) nq += br[q.branch_begin + b].q_len;
+        for (int b = 0; b < q.n_branches; ++b) nq += std::max(0, br[q.branch_begin + b].q_len);
         if (nq > 0) {
           push_region(q, 0, q.prefix_len, q.prefix_len, 0);
+          for (int b = 0; b < q.n_branches; ++b) {             // regions of earlier stages: seen by every branch
+            const aspd_branch_t& x = br[q.branch_begin + b];
+            if (x.q_len == ASPD_Q_SHARED) push_region(q, x.kv_off, x.kv_len, x.kv_len, 0);
+          }
           const int pe = ((int)visit.size() - visit0[r]) * ps;
           for (int b = 0; b < q.n_branches; ++b) {
             const aspd_branch_t& x = br[q.branch_begin + b];
-            if (x.q_len == 0) continue;
+            if (x.q_len <= 0) continue;
             const int lo = ((int)visit.size() - visit0[r]) * ps;
             push_region(q, x.kv_off, x.kv_len, x.kv_len - x.q_len, t);
             for (int i = 0; i < x.q_len; ++i) tok_vis[t++] = make_int4(pe, lo, lo + x.kv_len - x.q_len + i + 1, 0);

@@ -290,6 +290,65 @@ def build_segment_workload(name: str, seed: int, Hq: int, Hkv: int, d: int, dtyp
     return wl
 
 
+def build_two_stage_workload(name: str, seed: int, Hq: int, Hkv: int, d: int, dtype: str, theta: float, prefix: int,
+                             stage1: List[int], tail1: int, prior2: List[int], q2: List[int], serial_steps: int = 1,
+                             page_size: int = 16) -> Workload:
+    """One request that has already been through a parallel stage and opens a second one (the
+    engine switches between serial and parallel decoding repeatedly).
+
+    Cache before the measured step: ``prefix`` tokens, the merged branches of the first stage
+    (``stage1`` lengths), ``tail1`` serial tokens decoded after it, and ``prior2`` tokens in each
+    branch of the second stage.  The measured step adds ``q2`` tokens per second-stage branch;
+    then ``serial_steps`` serial steps follow.  Regions of the earlier stage are marked with
+    ``br_q_len = -1`` (visible to every branch of the current stage).
+    """
+    n1, n2 = len(stage1), len(prior2)
+    caps = list(stage1) + [tail1] + [prior2[b] + q2[b] for b in range(n2)]
+    rq = _Request(prefix, caps, serial_steps, page_size)
+    n_pool_pages = rq.n_pages + 3
+    table = permutation(seed, 7, n_pool_pages)[: rq.n_pages]
+    vals = _Values(seed, Hq, Hkv, d, dtype, rq.n_slots + 1)
+    wl = Workload(name=name, Hq=Hq, Hkv=Hkv, d=d, page_size=page_size, dtype=dtype, theta=float(theta),
+                  sm_scale=float(1.0 / np.sqrt(d)), n_pool_pages=n_pool_pages, seed=seed)
+
+    def desc(P, regions, tail_off, tail_len):
+        """regions: list of (slot offset, kv_len, q_len)."""
+        out = {"prefix_len": [P], "n_branches": [len(regions)], "branch_begin": [0], "page_begin": [0],
+               "n_pages": [rq.n_pages], "tail_off": [tail_off], "tail_len": [tail_len],
+               "br_kv_off": [r[0] for r in regions], "br_kv_len": [r[1] for r in regions], "br_q_len": [r[2] for r in regions]}
+        out = {k: np.asarray(v, dtype=np.int32) for k, v in out.items()}
+        out["page_ids"] = np.asarray(table, dtype=np.int32)
+        return out
+
+    def span(off, lo, hi):
+        return np.arange(off + lo, off + hi, dtype=np.int64)
+
+    off1, off_t1, off2 = rq.br_off[:n1], rq.br_off[n1], rq.br_off[n1 + 1:]
+    # prefix (an empty prefix plus one "branch" that is the prefix itself), then the first stage
+    wl.phases.append(_phase(vals, MODE_BRANCH, desc(0, [(0, prefix, prefix)], rq.tail_off, 0), [span(0, 0, prefix)],
+                            False, False, "fill-prefix"))
+    wl.phases.append(_phase(vals, MODE_BRANCH, desc(prefix, [(off1[b], stage1[b], stage1[b]) for b in range(n1)], rq.tail_off, 0),
+                            [np.concatenate([span(off1[b], 0, stage1[b]) for b in range(n1)])], False, False, "fill-stage1"))
+    # serial tokens between the stages, one step each
+    merged1 = [(off1[b], stage1[b], 0) for b in range(n1)]
+    for s_ in range(tail1):
+        wl.phases.append(_phase(vals, MODE_SERIAL, desc(prefix, merged1, off_t1, s_ + 1), [span(off_t1, s_, s_ + 1)],
+                                False, False, f"fill-tail1-{s_}"))
+    shared = [(off1[b], stage1[b], -1) for b in range(n1)] + ([(off_t1, tail1, -1)] if tail1 > 0 else [])
+    if sum(prior2) > 0:
+        wl.phases.append(_phase(vals, MODE_BRANCH, desc(prefix, shared + [(off2[b], prior2[b], prior2[b]) for b in range(n2)],
+                                                        rq.tail_off, 0),
+                                [np.concatenate([span(off2[b], 0, prior2[b]) for b in range(n2)])], False, False, "fill-stage2"))
+    final2 = [prior2[b] + q2[b] for b in range(n2)]
+    wl.phases.append(_phase(vals, MODE_BRANCH, desc(prefix, shared + [(off2[b], final2[b], q2[b]) for b in range(n2)], rq.tail_off, 0),
+                            [np.concatenate([span(off2[b], prior2[b], final2[b]) for b in range(n2)])], True, True, "parallel-step"))
+    for s_ in range(serial_steps):
+        wl.phases.append(_phase(vals, MODE_SERIAL, desc(prefix, shared + [(off2[b], final2[b], 0) for b in range(n2)],
+                                                        rq.tail_off, s_ + 1),
+                                [span(rq.tail_off, s_, s_ + 1)], True, True, f"serial-{s_}"))
+    return wl
+
+
 # ------------------------------------------------------------------- the five configurations
 def config_tiny(seed: int = SEED_BASE + 0) -> Workload:
     """4 q heads, 1 KV head, d 64, fp32; prefix 256; branches hold 16/9/23 + 1 new; theta 1e4."""

@@ -41,6 +41,7 @@ def small_workloads():
     yield W.build_segment_workload("b", 4, 28, 4, 128, "bf16", 1e6, [15, 16, 17, 0], [[16, 1], [17], [0, 0, 33], [4]],
                                    [[1, 1], [1], [12, 5, 1], [1]], serial_steps=1)
     yield W.config_tiny()
+    yield W.build_two_stage_workload("ts", 5, 28, 4, 128, "bf16", 1e6, 37, [30, 1, 17], 3, [5, 0, 40], [1, 2, 1], serial_steps=2)
     yield W.config_branch_open(serial_steps=3)
 
 

@@ -325,6 +325,21 @@ def test_stable_cache_promise_changes_nothing_but_timing(fused):
             np.testing.assert_array_equal(a, b)
 
 
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("fused", [False, True])
+def test_second_parallel_stage(kernel, fused):
+    """Iterative serial/parallel switching: branches of a second stage see the prefix, the merged
+    branches of the first stage and the serial tokens between the stages (regions with
+    q_len = ASPD_Q_SHARED), plus their own branch; positions continue from the complete sequence."""
+    for wl in (W.build_two_stage_workload("ts", 5, 28, 4, 128, "bf16", 1e6, 700, [130, 1, 47], 5, [33, 0, 140, 16],
+                                          [1, 1, 1, 1], serial_steps=2),
+               W.build_two_stage_workload("ts-open", 6, 28, 4, 128, "bf16", 1e6, 90, [20, 31], 0, [0, 0, 0], [12, 12, 12],
+                                          serial_steps=1),
+               W.build_two_stage_workload("ts-f32", 7, 4, 1, 64, "f32", 1e4, 33, [9, 16], 2, [3, 7], [1, 1], serial_steps=1)):
+        run, ref = compare_workload(wl, kernel=kernel, fused=fused)
+        assert len(run.outputs) == 1 + sum(p.label.startswith("serial") for p in wl.phases)
+
+
 def test_zero_new_tokens_is_a_no_op():
     E = engine()
     wl = W.build_segment_workload("e", 8, 28, 4, 128, "bf16", 1e6, [20], [[5, 9]], [[1, 1]])

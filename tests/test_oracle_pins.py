@@ -336,6 +336,43 @@ def test_dense_and_descriptor_forms_agree():
         np.testing.assert_allclose(dense[P:], np.array(outs), atol=1e-12)
 
 
+def test_second_parallel_stage_descriptor_form_equals_dense_form():
+    """A request that opens a second parallel stage (regions of the first stage and the serial
+    tokens between the stages marked as shared): the descriptor form gives the positions and
+    visible sets of the hand-derived table, and the same outputs as Eq. 1-4 taken literally."""
+    rows = load_example()
+    Hq, Hkv, d, theta = 4, 2, 16, 1e4
+    wl = W.build_two_stage_workload("ts", 5, Hq, Hkv, d, "f32", theta, 5, [3, 1, 2], 2, [1, 0], [1, 1], serial_steps=1)
+    run = run_workload(wl)
+    # raw values by logical slot
+    n_slots = int(wl.phases[0].desc["n_pages"][0]) * wl.page_size
+    kk = np.zeros((n_slots, Hkv, d)); vv = np.zeros((n_slots, Hkv, d)); qq = np.zeros((n_slots, Hq, d))
+    for ph, (pos, slot, req) in zip(wl.phases, run.positions):
+        kk[slot] = ph.k_new; vv[slot] = ph.v_new
+        if ph.q is not None:
+            qq[slot] = ph.q
+    last = wl.phases[-1].desc
+    off = last["br_kv_off"]          # stage-1 branches 0..2, serial tokens between the stages, stage-2 branches 0..1
+    flat_slot = ([0, 1, 2, 3, 4] + [off[0], off[1], off[2], off[0] + 1, off[2] + 1, off[0] + 2] + [off[3], off[3] + 1]
+                 + [off[4], off[5], off[4] + 1] + [int(last["tail_off"][0])])
+    assert len(flat_slot) == len(rows)
+    branch = [r[1] for r in rows]; stage = [r[2] for r in rows]
+    dense = oracle.dense_attn(qq[flat_slot], kk[flat_slot], vv[flat_slot], branch, stage, theta, wl.sm_scale)
+    par, ser = run.outputs
+    np.testing.assert_allclose(par[0], dense[15], atol=1e-12)       # second token of stage-2 branch 0
+    np.testing.assert_allclose(par[1], dense[14], atol=1e-12)       # first token of stage-2 branch 1
+    np.testing.assert_allclose(ser[0], dense[16], atol=1e-12)
+    # positions and visible sets against the hand-derived table
+    ph = [p for p in wl.phases if p.label == "parallel-step"][0]
+    pos, slot, _ = oracle.new_tokens(ph.desc, oracle.MODE_BRANCH)
+    assert pos.tolist() == [rows[15][3], rows[14][3]]
+    vis = oracle.visible_slots(ph.desc, oracle.MODE_BRANCH, n_slots)
+    for t, flat in enumerate((15, 14)):
+        assert sorted(np.flatnonzero(vis[t]).tolist()) == sorted(int(flat_slot[j]) for j in rows[flat][4])
+    pos, _, _ = oracle.new_tokens(wl.phases[-1].desc, oracle.MODE_SERIAL)
+    assert pos.tolist() == [rows[16][3]]
+
+
 # ------------------------------------------------------------------ softmax closed forms
 def test_softmax_closed_forms():
     wl = W.build_segment_workload("c", 21, 4, 2, 16, "f32", 10000.0, [19], [[4, 9]], [[1, 1]], serial_steps=1)
