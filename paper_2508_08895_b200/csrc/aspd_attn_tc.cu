@@ -20,10 +20,11 @@
 // raised when the tile maximum exceeds it by more than 2^8, which keeps P exactly consistent
 // with the (m, l, O) record while making the rescale of O in TMEM rare.
 //
-// Warp roles: 0-3 softmax (TMEM lane quadrant = warp), 4 and 7 bulk-copy producers (K and V),
-// 5 MMA issuer (one elected lane), 8-11 fused append of the step's new rows (aspd_branch_step /
+// Warp roles: 0-7 softmax (TMEM lane quadrant = warp % 4; warps w and w + 4 share the rows of a
+// quadrant and take half of the columns each), 8 and 11 bulk-copy producers (K and V), 9 MMA
+// issuer (one elected lane), 12-15 fused append of the step's new rows (aspd_branch_step /
 // aspd_serial_step), query preparation (RoPE, bf16, swizzled store, one item ahead) and epilogue
-// (TMEM lane quadrant = warp - 8); warp 6 is idle.  All cross-role hand-offs are mbarriers; every
+// (TMEM lane quadrant = warp - 12); warp 10 is idle.  All cross-role hand-offs are mbarriers; every
 // wait is bounded and on expiry sets the plan's status word to ASPD_ERR_TIMEOUT and makes all
 // roles drain and exit.
 #include <stdlib.h>
@@ -34,7 +35,9 @@ namespace aspd {
 namespace {
 
 constexpr int kTile = 128;                     // keys per tile
-constexpr int kThreads = 384;
+constexpr int kThreads = 512;
+constexpr int kSoftmaxThreads = 256;           // two warps per TMEM lane quadrant, each taking half of the columns
+constexpr int W_KPROD = 8, W_MMA = 9, W_VPROD = 11, W_EPI = 12;   // warp roles (0-7 softmax, 10 idle, 12-15 epilogue)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRaise = 8.0f;                 // raise the reference maximum only beyond 2^8
 constexpr long long kWaitCycles = 3000000000LL; // ~1.5 s at 1.9 GHz
@@ -49,14 +52,14 @@ constexpr uint32_t OFF_MISC = OFF_P + 8192;
 enum Bar { K_FULL = 0, K_EMPTY = 2, V_FULL = 4, V_EMPTY = 6, S_FULL = 8, S_EMPTY = 10, P_FULL = 12, P_EMPTY = 13,
            O_FULL = 14, O_EMPTY = 16, Q_FULL = 18, Q_EMPTY = 20, E_FULL = 22, A_DONE = 24, NUM_BARS = 25 };
 
-constexpr int kItemCache = 12;      // items of a CTA kept in shared memory (more are read from global)
+constexpr int kItemCache = 10;      // items of a CTA kept in shared memory (more are read from global)
 constexpr int kMaxTokPerItem = 16;  // tokens of a row block whose ranges are cached (n_q_tok is at most 64 / G)
 
 struct Misc {
   uint64_t bars[NUM_BARS];
-  float smax[2][128];
-  float fin_m[2][128];         // per item parity: reference maximum and sum of every softmax thread
-  float fin_l[2][128];
+  float smax[2][256];          // per S buffer: tile maximum of every softmax thread
+  float fin_m[2][64];          // per item parity: reference maximum of every query row ...
+  float fin_l[2][256];         // ... and the sum of every softmax thread
   int nval[4][8];              // valid rows of the 8 pages of a tile (ring over 4 tiles)
   DeviceItem items[kItemCache];        // this CTA's first items and, per item, the visible ranges of
   int4 vis[kItemCache][kMaxTokPerItem]; // its query tokens: no global-load chain at an item boundary
@@ -151,6 +154,13 @@ __device__ __forceinline__ bool named_sync_or(int id, int n, bool pred) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, " \
                "%12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, "   \
                "%31};" ::ASPD_W32(v, o), "r"(taddr) : "memory")
+#define ASPD_TMEM_LD16(taddr, v, o)                                                                               \
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, "  \
+               "%13, %14, %15}, [%16];"                                                                          \
+               : "=f"(v[o + 0]), "=f"(v[o + 1]), "=f"(v[o + 2]), "=f"(v[o + 3]), "=f"(v[o + 4]), "=f"(v[o + 5]),  \
+                 "=f"(v[o + 6]), "=f"(v[o + 7]), "=f"(v[o + 8]), "=f"(v[o + 9]), "=f"(v[o + 10]), "=f"(v[o + 11]), \
+                 "=f"(v[o + 12]), "=f"(v[o + 13]), "=f"(v[o + 14]), "=f"(v[o + 15])                               \
+               : "r"(taddr) : "memory")
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -213,18 +223,21 @@ __device__ __forceinline__ uint32_t bits_between(int lo, int hi) {
   return hi > lo ? ((0xFFFFu >> (16 - hi)) & ~((1u << lo) - 1u)) : 0u;
 }
 
-template <int NC>   // NC = columns per thread = padded row count R
+template <int NC>   // NC = padded row count R = columns of a row replica; a thread takes half of them
 __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it, Misc* misc, uint32_t bars, uint32_t smem_p,
                                              uint32_t tmem, int item_no, int& g) {   // item_no = index among this CTA's items
-  constexpr int R = NC, KS = 128 / NC;
+  constexpr int R = NC, KS = 128 / NC, HC = NC / 2;
   const int tid = threadIdx.x, warp = tid >> 5;
-  const int r = tid % R, j = tid / R;
+  const int tl = tid & 127, half = tid >> 7;     // TMEM lane of the thread; which half of the replica's columns
+  const int r = tl % R, j = tl / R;
+  const int col0 = j * NC + half * HC;           // first tile column (key) of this thread
   const int G = c.n_q_heads / c.n_kv_heads, M = it.n_q_tok * G;
   const int n_tiles = (it.n_pages + 7) >> 3;
   volatile int* ab = &misc->abort_flag;
   int4 vis = make_int4(0, 0, 0, 0);             // padding rows see nothing
   if (r < M) vis = (item_no < kItemCache && r / G < kMaxTokPerItem) ? misc->vis[item_no][r / G] : c.pd.tok_vis[it.q_tok0 + r / G];
-  const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+  const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+  const bool o_owner = half == 0 && (warp & 3) < R / 32;   // threads whose TMEM lane holds a row of O
   const int ob = item_no & 1;
   float m_ref = -INFINITY, l = 0.f;
   bool dead = false;   // a wait gave up: keep walking the same control flow, report at the end
@@ -233,20 +246,20 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
     dead |= !mbar_wait(bars + 8 * (S_FULL + sb), (g >> 1) & 1, ab);
     tc_fence_after();
     if (tid == 0) ASPD_STAMP(c, g, 0);
-    float s[NC];
-    const uint32_t s_addr = tmem + lane_addr + COL_S + sb * 128 + j * NC;
-    ASPD_TMEM_LD32(s_addr, s, 0);
-    if constexpr (NC == 64) ASPD_TMEM_LD32(s_addr + 32, s, 32);
+    float s[HC];
+    const uint32_t s_addr = tmem + lane_addr + COL_S + sb * 128 + col0;
+    if constexpr (HC == 32) ASPD_TMEM_LD32(s_addr, s, 0);
+    else ASPD_TMEM_LD16(s_addr, s, 0);
     tmem_wait_ld();
     tc_fence_before();
     mbar_arrive(bars + 8 * (S_EMPTY + sb));
     if (tid == 0) ASPD_STAMP(c, g, 1);
-    // visibility of my NC keys: valid rows of each page, and the token's ranges [0, pe), [lo, hi)
+    // visibility of my HC keys: valid rows of each page, and the token's ranges [0, pe), [lo, hi)
     float mx = -INFINITY;
 #pragma unroll
-    for (int pg = 0; pg < NC / 16; ++pg) {
-      const int nv = misc->nval[g & 3][j * (NC / 16) + pg];
-      const int kb = it.key0 + t * kTile + j * NC + pg * 16;     // stream key of the page's first row
+    for (int pg = 0; pg < HC / 16; ++pg) {
+      const int nv = misc->nval[g & 3][col0 / 16 + pg];
+      const int kb = it.key0 + t * kTile + col0 + pg * 16;       // stream key of the page's first row
       const uint32_t mask = bits_between(0, min(nv, vis.x - kb)) | bits_between(vis.y - kb, min(nv, vis.z - kb));
       if (mask == 0xFFFFu) {
 #pragma unroll
@@ -262,16 +275,17 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
     }
     mx *= c.scale_log2;                           // the scale is positive: max commutes with it
     misc->smax[sb][tid] = mx;
-    named_sync(1, 128);
+    named_sync(1, kSoftmaxThreads);
     if (tid == 0) ASPD_STAMP(c, g, 2);
     float m_tile = mx;
 #pragma unroll
-    for (int jj = 0; jj < KS; ++jj) m_tile = fmaxf(m_tile, misc->smax[sb][jj * R + r]);
+    for (int jj = 0; jj < KS; ++jj)
+      m_tile = fmaxf(m_tile, fmaxf(misc->smax[sb][jj * R + r], misc->smax[sb][128 + jj * R + r]));
     const bool upd = m_tile > m_ref + kRaise;     // also true for the first finite maximum (m_ref = -inf)
     float alpha = 1.f;
     if (upd) { alpha = ex2(m_ref - m_tile); m_ref = m_tile; }
     l *= alpha;
-    if (t > 0 && warp < R / 32) {                 // the owners of rows 0..R-1 rescale O in TMEM
+    if (t > 0 && o_owner) {                       // the owners of rows 0..R-1 rescale O in TMEM
       if (__any_sync(0xffffffffu, upd)) {
         dead |= !mbar_wait(bars + 8 * P_EMPTY, (g - 1) & 1, ab);   // PV of the previous tile is done
         tc_fence_after();
@@ -292,7 +306,7 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
     const float nmsafe = m_ref == -INFINITY ? 0.f : -m_ref;
     float lsum0 = 0.f, lsum1 = 0.f;
 #pragma unroll
-    for (int i = 0; i < NC; i += 2) {             // p = 2^(s * scale - m): one FFMA, one MUFU
+    for (int i = 0; i < HC; i += 2) {             // p = 2^(s * scale - m): one FFMA, one MUFU
       s[i] = ex2(fmaf(s[i], c.scale_log2, nmsafe));
       s[i + 1] = ex2(fmaf(s[i + 1], c.scale_log2, nmsafe));
       lsum0 += s[i];
@@ -303,8 +317,8 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
     if (g > 0) dead |= !mbar_wait(bars + 8 * P_EMPTY, (g - 1) & 1, ab);   // P tile is free again
     if (tid == 0) ASPD_STAMP(c, g, 4);
 #pragma unroll
-    for (int c8 = 0; c8 < NC / 8; ++c8) {
-      const int kk = j * NC + c8 * 8;
+    for (int c8 = 0; c8 < HC / 8; ++c8) {
+      const int kk = col0 + c8 * 8;
       const uint32_t addr = smem_p + (kk >> 6) * kHalf + r * 128 + ((((kk & 63) >> 3) ^ (r & 7)) << 4);
       asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pack_bf16(s[c8 * 8 + 0], s[c8 * 8 + 1])),
                    "r"(pack_bf16(s[c8 * 8 + 2], s[c8 * 8 + 3])), "r"(pack_bf16(s[c8 * 8 + 4], s[c8 * 8 + 5])),
@@ -317,10 +331,10 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
   }
   // ---- hand the item's statistics to the epilogue warps and move on to the next item
   dead |= !mbar_wait(bars + 8 * (O_EMPTY + ob), ((item_no >> 1) & 1) ^ 1, ab);   // epilogue of item_no - 2 is done
-  misc->fin_m[ob][tid] = m_ref;
+  if (j == 0 && half == 0) misc->fin_m[ob][r] = m_ref;
   misc->fin_l[ob][tid] = l;
   mbar_arrive(bars + 8 * (E_FULL + ob));
-  return !named_sync_or(1, 128, dead || *ab);
+  return !named_sync_or(1, kSoftmaxThreads, dead || *ab);
 }
 
 // Rotate the item's query rows (RoPE at the token's position, cos/sin table from the plan),
@@ -455,7 +469,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   }
 
   if (tid == 0) {
-    const int counts[NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, 128, 128, 128, 1, 1, 1, 128, 128, 128, 128, 1, 1, 128, 128, 128};
+    const int counts[NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, 256, 256, 256, 1, 1, 1, 128, 128, 128, 128, 1, 1, 256, 256, 128};
     for (int i = 0; i < NUM_BARS; ++i) mbar_init(bars + 8 * i, counts[i]);
     misc->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -472,12 +486,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   // fused step: the epilogue threads fetch their first new-row entries now (plan data)
   int dirty0 = 0, dirty_units = 0;
   int4 dirty_first[2] = {make_int4(0, 0, 0, 0), make_int4(0, 0, 0, 0)};
-  if (warp >= 8 && c.k_new != nullptr) {
+  if (warp >= W_EPI && c.k_new != nullptr) {
     dirty0 = c.pd.cta_dirty0[blockIdx.x];
     dirty_units = (c.pd.cta_dirty0[blockIdx.x + 1] - dirty0) * 24;
 #pragma unroll
     for (int k = 0; k < 2; ++k) {
-      const int u = (tid - 256) + k * 128;
+      const int u = (tid - W_EPI * 32) + k * 128;
       if (u < dirty_units) dirty_first[k] = c.pd.dirty[dirty0 + u / 24];
     }
   }
@@ -485,12 +499,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   // the stream (q, k_new, the pools, the workspace's previous readers) are used from here on.
   // With the plan's stable-cache promise the two producer warps go ahead and fetch pages that
   // hold no new rows; they wait themselves before the first page that does.
-  const bool producer_runs_ahead = c.early_fetch && (warp == 4 || warp == 7);
+  const bool producer_runs_ahead = c.early_fetch && (warp == W_KPROD || warp == W_VPROD);
   if (!producer_runs_ahead) pdl_wait();
   if (tid == 0) ASPD_CTA_STAMP(c, 1);
 
-  if (warp < 4) {
-    // =============================== softmax + epilogue ===============================
+  if (warp < 8) {
+    // =============================== softmax ===============================
     int g = 0, item_no = 0;
     for (int idx = item_begin; idx < item_end; ++idx, ++item_no) {
       const DeviceItem it = get_item(c, misc, idx, item_begin);
@@ -499,14 +513,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
                               : softmax_item<64>(c, it, misc, bars, base + OFF_P, tmem, item_no, g);
       if (!ok) break;
     }
-  } else if (warp == 4 || warp == 7) {
+  } else if (warp == W_KPROD || warp == W_VPROD) {
     // ================================ bulk-copy producers ================================
     // Warp 4 streams the K tiles and warp 7 the V tiles, each on its own ring, so that a K load
     // never queues behind a V slot that is still being read (and vice versa).
     // Lane l keeps stream-page entry (batch * 32 + l) of the item in a register; the next batch
     // of 32 entries (4 tiles) is requested before the current one is consumed, so the page list
     // never sits on the critical path.
-    const int kv = warp == 4 ? 0 : 1;
+    const int kv = warp == W_KPROD ? 0 : 1;
     const char* pool = kv ? c.v_pool : c.k_pool;
     int g = 0;
     bool ok = true, appended = false, waited = false;
@@ -566,7 +580,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
         if (lane == 0) ASPD_STAMP(c, g, 13 + kv);
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == W_MMA) {
     // =================================== MMA issuer ===================================
     // The tiles of all items form one pipeline: S of tile g is issued before P.V of tile g - 1,
     // also across an item boundary, so the tensor pipe and the softmax warps never drain
@@ -631,11 +645,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
       if (ok && have_prev) issue_pv(prev, g - 1);
     }
     __syncwarp();
-  } else if (warp >= 8) {
+  } else if (warp >= W_EPI) {
     // ===================================== epilogue =====================================
     // One (m, l, O) record per query row of every item, written while the other warps are
     // already working on the next item (O and the statistics are double-buffered by item).
-    const int et = tid - 256, ew = warp - 8;       // TMEM lane quadrant = warp % 4 = ew
+    const int et = tid - W_EPI * 32, ew = warp - W_EPI;   // TMEM lane quadrant = warp % 4 = ew
     const int G = c.n_q_heads / c.n_kv_heads;
     int item_no = 0;
     bool dead = false;
@@ -666,7 +680,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
           const int tok = it.q_tok0 + r / G;
           rec = (size_t)(c.pd.part_base[tok * c.n_kv_heads + it.kv_head] + it.part_slot) * G + r % G;
           float lt = 0.f;
-          for (int jj = 0; jj < KS; ++jj) lt += misc->fin_l[ob][jj * R + r];
+          for (int jj = 0; jj < KS; ++jj) lt += misc->fin_l[ob][jj * R + r] + misc->fin_l[ob][128 + jj * R + r];
           if (!dead) c.pd.ws_ml[rec] = make_float2(misc->fin_m[ob][r], lt);
         }
         const uint32_t o_addr = tmem + ((uint32_t)(ew * 32) << 16) + COL_O + ob * 128;
