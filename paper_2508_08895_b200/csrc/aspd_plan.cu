@@ -337,10 +337,17 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
     // so CTAs that end up with several short items get fewer pages.
     const char* ice = getenv("ASPD_ITEM_COST");
     const double kItemCost = ice ? atof(ice) : 12.0;
+    // a page costs a little more the more query rows are scored against it (best measured balance:
+    // 0.35 % per row), so streams of requests with many branches weigh more
+    const char* rce = getenv("ASPD_ROW_COST");
+    const double kRowCost = rce ? atof(rce) : 0.0035;
+    auto page_cost = [&](const Stream& st) { return 1.0 + kRowCost * st.n_tok * G; };
     // the share is re-derived from what is left whenever a CTA is closed, so rounding does not pile up
-    long pages_left = total_pages, streams_left = (long)streams.size();
+    double cost_left = 0.0;
+    for (const Stream& st : streams) cost_left += page_cost(st) * st.n_pages;
+    long streams_left = (long)streams.size();
     auto share_now = [&](int ctas_left) {
-      return ((double)pages_left + kItemCost * ((double)streams_left + ctas_left)) / std::max(1, ctas_left);
+      return (cost_left + kItemCost * ((double)streams_left + ctas_left)) / std::max(1, ctas_left);
     };
     double share = share_now(n_ctas);
     int cta = 0;
@@ -348,9 +355,10 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
     auto next_cta = [&]() { cta_item0[++cta] = (int)p->items.size(); acc = 0.0; share = share_now(n_ctas - cta); };
     for (const Stream& st : streams) {
       int at = 0, slot = 0;
+      const double pc = page_cost(st);
       --streams_left;
       while (at < st.n_pages) {
-        double room = share - acc - kItemCost;     // pages that still fit if an item starts here
+        double room = (share - acc - kItemCost) / pc;   // pages that still fit if an item starts here
         if (room < 1.0 && acc > 0.0 && cta + 1 < n_ctas) { next_cta(); continue; }
         long take = std::min<long>(st.n_pages - at, chunk_pages);
         if (cta + 1 < n_ctas) take = std::min<long>(take, std::max<long>(1, (long)(room + 0.5)));
@@ -360,8 +368,8 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
         it.row_block = st.row_block; it.reserved = 0;
         p->items.push_back(it);
         at += (int)take;
-        pages_left -= take;
-        acc += kItemCost + (double)take;
+        cost_left -= pc * take;
+        acc += kItemCost + pc * (double)take;
         if (acc >= share - 0.5 && cta + 1 < n_ctas) next_cta();
       }
       for (int i = 0; i < st.n_tok; ++i) n_parts[(size_t)(st.tok0 + i) * Hkv + st.head] = slot;
