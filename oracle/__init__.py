@@ -43,7 +43,7 @@ def lib() -> ctypes.CDLL:
         _lib = ctypes.CDLL(build())
         _lib.aspd_oracle_rope.restype = None
         for name in ("aspd_oracle_dense_positions", "aspd_oracle_dense_visible", "aspd_oracle_dense_attn",
-                     "aspd_oracle_new_tokens", "aspd_oracle_kv_append", "aspd_oracle_attn",
+                     "aspd_oracle_new_tokens", "aspd_oracle_kv_append", "aspd_oracle_attn", "aspd_oracle_attn_at",
                      "aspd_oracle_visible_slots", "aspd_oracle_threads"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
@@ -159,14 +159,25 @@ def kv_append(desc, k_new, v_new, pos, req, slot, k_pool, v_pool, theta: float) 
     assert rc == 0
 
 
-def attn(desc, mode: int, q, k_pool, v_pool, theta: float, sm_scale: float) -> np.ndarray:
-    """a4-a7 (mode 0) / a9 (mode 1): out [n_new][Hq][d] for raw queries q [n_new][Hq][d]."""
+def attn(desc, mode: int, q, k_pool, v_pool, theta: float, sm_scale: float, q_pos=None) -> np.ndarray:
+    """a4-a7 (mode 0) / a9 (mode 1): out [n_new][Hq][d] for raw queries q [n_new][Hq][d].
+    ``q_pos``: query positions of a position-ID variant (default: Eq. 4)."""
     d = _desc(desc)
     q = _f64(q)
     n_new, Hq, hd = q.shape
     assert n_new == n_new_tokens(d, mode)
     Hkv, page_size = k_pool.shape[1], k_pool.shape[2]
     out = np.empty_like(q)
+    if q_pos is not None:
+        qp = _i32(q_pos)
+        assert len(qp) == n_new
+        rc = lib().aspd_oracle_attn_at(len(d["prefix_len"]), mode, Hq, Hkv, hd, page_size, ctypes.c_double(theta),
+                                       ctypes.c_double(sm_scale), _p(d["prefix_len"]), _p(d["n_branches"]),
+                                       _p(d["branch_begin"]), _p(d["page_begin"]), _p(d["tail_off"]), _p(d["tail_len"]),
+                                       _p(d["br_kv_off"]), _p(d["br_kv_len"]), _p(d["br_q_len"]), _p(d["page_ids"]),
+                                       _p(q), _p(qp), _p(k_pool), _p(v_pool), _p(out))
+        assert rc == 0, rc
+        return out
     rc = lib().aspd_oracle_attn(len(d["prefix_len"]), mode, Hq, Hkv, hd, page_size, ctypes.c_double(theta),
                                 ctypes.c_double(sm_scale), _p(d["prefix_len"]), _p(d["n_branches"]),
                                 _p(d["branch_begin"]), _p(d["page_begin"]), _p(d["tail_off"]), _p(d["tail_len"]),

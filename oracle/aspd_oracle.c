@@ -309,13 +309,14 @@ static const double* cached(const double* pool, const int* page_ids, int pbeg,
  * Visible set of the serial token: prefix, every token of every branch, and
  * the tail up to and including itself.
  */
-int aspd_oracle_attn(int n_req, int mode, int Hq, int Hkv, int d,
+static int attn_impl(int n_req, int mode, int Hq, int Hkv, int d,
                      int page_size, double theta, double sm_scale,
                      const int* prefix_len, const int* n_branches,
                      const int* branch_begin, const int* page_begin,
                      const int* tail_off, const int* tail_len,
                      const int* br_kv_off, const int* br_kv_len,
                      const int* br_q_len, const int* page_ids, const double* q,
+                     const int* q_pos_given,
                      const double* k_pool, const double* v_pool, double* out) {
   if (Hq % Hkv || d % 2) return ORACLE_BAD;
   int G = Hq / Hkv;
@@ -408,6 +409,7 @@ int aspd_oracle_attn(int n_req, int mode, int Hq, int Hkv, int d,
           }
           qpos = total + tail_len[r] - 1;
         }
+        if (q_pos_given) qpos = q_pos_given[t];   /* a position-ID variant: the caller's rule, not Eq. 4 */
         aspd_oracle_rope(q + ((size_t)t * Hq + hq) * d, d, (double)qpos, theta, qhat);
         attend_one(qhat, d, sm_scale, keys, vals, m, logits,
                    out + ((size_t)t * Hq + hq) * d);
@@ -416,6 +418,38 @@ int aspd_oracle_attn(int n_req, int mode, int Hq, int Hkv, int d,
   }
   free(t_req); free(t_br); free(t_k); free(t_pos0);
   return fail ? ORACLE_BAD : ORACLE_OK;
+}
+
+int aspd_oracle_attn(int n_req, int mode, int Hq, int Hkv, int d,
+                     int page_size, double theta, double sm_scale,
+                     const int* prefix_len, const int* n_branches,
+                     const int* branch_begin, const int* page_begin,
+                     const int* tail_off, const int* tail_len,
+                     const int* br_kv_off, const int* br_kv_len,
+                     const int* br_q_len, const int* page_ids, const double* q,
+                     const double* k_pool, const double* v_pool, double* out) {
+  return attn_impl(n_req, mode, Hq, Hkv, d, page_size, theta, sm_scale, prefix_len, n_branches, branch_begin,
+                   page_begin, tail_off, tail_len, br_kv_off, br_kv_len, br_q_len, page_ids, q, 0, k_pool, v_pool, out);
+}
+
+/*
+ * The same attention with the query positions given by the caller instead of Eq. 4: the
+ * position-ID variants of the paper's ablation (pre-allocated fixed-length intervals per branch;
+ * "Same-Max": the serial token resumes at the largest branch position).  Masking is unchanged;
+ * the keys carry whatever positions they were appended with.
+ */
+int aspd_oracle_attn_at(int n_req, int mode, int Hq, int Hkv, int d,
+                        int page_size, double theta, double sm_scale,
+                        const int* prefix_len, const int* n_branches,
+                        const int* branch_begin, const int* page_begin,
+                        const int* tail_off, const int* tail_len,
+                        const int* br_kv_off, const int* br_kv_len,
+                        const int* br_q_len, const int* page_ids, const double* q,
+                        const int* q_pos,
+                        const double* k_pool, const double* v_pool, double* out) {
+  if (!q_pos) return ORACLE_BAD;
+  return attn_impl(n_req, mode, Hq, Hkv, d, page_size, theta, sm_scale, prefix_len, n_branches, branch_begin,
+                   page_begin, tail_off, tail_len, br_kv_off, br_kv_len, br_q_len, page_ids, q, q_pos, k_pool, v_pool, out);
 }
 
 /*

@@ -18,13 +18,18 @@ class OracleRun:
         self.outputs = []      # one [n_new][Hq][d] array per compared phase
         self.positions = []    # per phase: (pos, slot, req) int32 arrays
 
-    def step(self, ph, attend=True):
+    def step(self, ph, attend=True, pos_override=None):
+        """pos_override: position IDs of a position-ID variant for this phase's new tokens (keys
+        and queries); default: the paper's rule (Eq. 4)."""
         wl = self.wl
         pos, slot, req = oracle.new_tokens(ph.desc, ph.mode)
+        if pos_override is not None:
+            pos = np.ascontiguousarray(pos_override, dtype=np.int32)
         self.positions.append((pos, slot, req))
         oracle.kv_append(ph.desc, ph.k_new, ph.v_new, pos, req, slot, self.k_pool, self.v_pool, wl.theta)
         if attend and ph.q is not None:
-            out = oracle.attn(ph.desc, ph.mode, ph.q, self.k_pool, self.v_pool, wl.theta, wl.sm_scale)
+            out = oracle.attn(ph.desc, ph.mode, ph.q, self.k_pool, self.v_pool, wl.theta, wl.sm_scale,
+                              q_pos=pos if pos_override is not None else None)
             if ph.compare:
                 self.outputs.append(out)
             return out

@@ -55,11 +55,15 @@ class WorkloadRun:
         self.positions = []
         self.plans = []
 
-    def step(self, ph: W.Phase, attend: bool = True, keep_plan: bool = False) -> Optional[np.ndarray]:
+    def step(self, ph: W.Phase, attend: bool = True, keep_plan: bool = False, pos_override=None) -> Optional[np.ndarray]:
+        """pos_override: caller-given position IDs of the phase's new tokens (a position-ID variant):
+        passed to aspd_kv_append and, as q_pos, to the plan."""
         wl = self.wl
-        plan = B.Plan(self.shape, ph.desc, wl.n_pool_pages, ph.mode, kernel=self.kernel,
+        plan = B.Plan(self.shape, ph.desc, wl.n_pool_pages, ph.mode, q_pos=pos_override, kernel=self.kernel,
                       chunk_tokens=self.chunk_tokens, n_ctas=self.n_ctas, stable_cache=self.stable_cache)
         pos, slot, req = B.positions(ph.desc, ph.mode)
+        if pos_override is not None:
+            pos = np.ascontiguousarray(pos_override, dtype=np.int32)
         self.positions.append((pos, slot, req))
         out = None
         if plan.n_new > 0:

@@ -373,6 +373,55 @@ def test_second_parallel_stage_descriptor_form_equals_dense_form():
     assert pos.tolist() == [rows[16][3]]
 
 
+def _variant_positions(wl, rule, k=32):
+    """Position IDs of every phase under a position-ID variant of the paper's ablation (written
+    here, in the test, from the variant's definition): "fix-k" gives branch b the pre-allocated
+    interval starting at P + b*k; "same-max" keeps the shared IDs but lets the serial token resume
+    right after the largest branch position."""
+    out = []
+    for ph in wl.phases:
+        d = ph.desc
+        P = int(d["prefix_len"][0])
+        if ph.mode == W.MODE_BRANCH:
+            pos = []
+            for b in range(int(d["n_branches"][0])):
+                kv, ql = int(d["br_kv_len"][b]), int(d["br_q_len"][b])
+                start = P + (b * k if rule == "fix-k" and P > 0 else 0)
+                pos += [start + kv - ql + i for i in range(max(ql, 0))]
+            out.append(np.array(pos, dtype=np.int32))
+        else:
+            lens = [int(x) for x in d["br_kv_len"]]
+            base = P + (max(lens) if rule == "same-max" else len(lens) * k)
+            out.append(np.array([base + int(d["tail_len"][0]) - 1], dtype=np.int32))
+    return out
+
+
+def test_position_id_variants_through_caller_given_positions():
+    """aspd_oracle_attn_at: with Eq. 4's own positions it is aspd_oracle_attn; with the ablation's
+    variants each branch still equals a standalone causal sequence at the variant's positions
+    (library SDPA), i.e. only the position IDs changed, not the mask."""
+    wl = W.build_segment_workload("var", 17, 4, 2, 16, "f32", 1e4, [23], [[5, 2, 9]], [[1, 1, 1]], serial_steps=1)
+    base = run_workload(wl)
+    same = oracle.run.OracleRun(wl)
+    for ph, (pos, _, _) in zip(wl.phases, base.positions):
+        same.step(ph, pos_override=pos)
+    for a, b in zip(base.outputs, same.outputs):
+        np.testing.assert_array_equal(a, b)
+    P, kpre, vpre, kb, vb, _ = _branch_tokens(wl)
+    par = [p for p in wl.phases if p.label == "parallel-step"][0]
+    for rule in ("fix-k", "same-max"):
+        run = oracle.run.OracleRun(wl)
+        for ph, pos in zip(wl.phases, _variant_positions(wl, rule)):
+            run.step(ph, pos_override=pos)
+        for b in range(3):
+            start = P + (32 * b if rule == "fix-k" else 0)
+            positions = np.concatenate([np.arange(P), start + np.arange(len(kb[b]))])
+            ref = _sdpa_causal_last(par.q[b], np.concatenate([kpre, kb[b]]), np.concatenate([vpre, vb[b]]), positions,
+                                    wl.theta, wl.sm_scale, wl.G)
+            np.testing.assert_allclose(run.outputs[0][b], ref, atol=1e-10)
+        assert not np.allclose(run.outputs[1], base.outputs[1])      # the serial token sits elsewhere
+
+
 # ------------------------------------------------------------------ softmax closed forms
 def test_softmax_closed_forms():
     wl = W.build_segment_workload("c", 21, 4, 2, 16, "f32", 10000.0, [19], [[4, 9]], [[1, 1]], serial_steps=1)
