@@ -133,7 +133,8 @@ typedef struct {
   int32_t kernel;           /* ASPD_KERNEL_* actually chosen                                */
   int32_t chunk_tokens;     /* forced maximum keys per item (0: none)                       */
   int32_t n_ctas;           /* CTAs of the persistent grid = shares the streams are cut into */
-  int32_t reserved;
+  int32_t fused_append;     /* 1: aspd_branch_step / aspd_serial_step write the new rows inside the
+                               attention pass; 0: they run the append kernel first               */
   int64_t workspace_bytes;  /* device memory the plan holds                                 */
   int64_t kv_tokens_read;   /* cached tokens the step must read (each once)                 */
   int64_t algorithmic_bytes;/* K+V of those tokens + q in + out + appended K/V              */

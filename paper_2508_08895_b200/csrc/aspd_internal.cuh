@@ -76,6 +76,7 @@ struct aspd_plan {
   int host_only;
   int sm_count;
   int n_row_blocks;
+  int fuse_append;             // few enough new rows per CTA for the attention pass to write them itself
   int stable_cache;            // producers may fetch pages without new rows before the dependency wait
   int64_t n_pool_pages;
   int64_t kv_tokens_read;

@@ -391,6 +391,13 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
     }
   }
   cta_dirty0[n_ctas] = (int)dirty.size();
+  {
+    // the fused step writes a CTA's new rows in batches at the start of the kernel; with many new
+    // rows per CTA (a branch-open step) the separate append kernel is the faster way
+    int most = 0;
+    for (int c = 0; c < n_ctas; ++c) most = std::max(most, cta_dirty0[c + 1] - cta_dirty0[c]);
+    p->fuse_append = most <= 20 ? 1 : 0;
+  }
   for (size_t i = 0; i < n_parts.size(); ++i) part_base[i + 1] = part_base[i] + n_parts[i];
   p->n_items = (int)p->items.size();
   p->n_partials = part_base[n_parts.size()];
@@ -497,7 +504,7 @@ int aspd_plan_info(const aspd_plan_t* p, aspd_plan_info_t* info) {
   if (!p || !info) return ASPD_ERR_INVALID_ARG;
   info->n_new = p->n_new; info->n_items = p->n_items; info->n_partials = p->n_partials;
   info->n_stream_pages = (int32_t)p->visit.size(); info->kernel = p->kernel;
-  info->chunk_tokens = p->chunk_tokens; info->n_ctas = p->n_ctas; info->reserved = 0; info->workspace_bytes = (int64_t)p->device_bytes;
+  info->chunk_tokens = p->chunk_tokens; info->n_ctas = p->n_ctas; info->fused_append = (p->kernel == ASPD_KERNEL_MMA && p->fuse_append) ? 1 : 0; info->workspace_bytes = (int64_t)p->device_bytes;
   info->kv_tokens_read = p->kv_tokens_read; info->algorithmic_bytes = p->algorithmic_bytes;
   return ASPD_OK;
 }
@@ -589,8 +596,11 @@ static int run_step(aspd_plan_t* p, int mode, const void* q, const void* k_new, 
   if (!q || !k_new || !v_new || !k_pool || !v_pool || !out) return ASPD_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   int rc;
-  if (p->kernel == ASPD_KERNEL_MMA) {
+  if (p->kernel == ASPD_KERNEL_MMA && p->fuse_append) {
     rc = launch_attn_mma_step(p, q, k_new, v_new, k_pool, v_pool, s);
+  } else if (p->kernel == ASPD_KERNEL_MMA) {
+    rc = launch_append(p, k_new, v_new, p->dev.tok_pos, k_pool, v_pool, s);
+    if (rc == ASPD_OK) rc = launch_attn_mma(p, q, k_pool, v_pool, s);
   } else {
     rc = launch_append(p, k_new, v_new, p->dev.tok_pos, k_pool, v_pool, s);
     if (rc == ASPD_OK) rc = launch_attn_generic(p, q, k_pool, v_pool, s);

@@ -86,7 +86,7 @@ extern "C" int aspd_attn_static(const aspd_plan_t* plan, const void* q, const vo
   shell.shape = plan->shape; shell.mode = plan->mode; shell.n_req = plan->n_req; shell.n_new = plan->n_new;
   shell.n_items = plan->n_items; shell.n_partials = plan->n_partials; shell.kernel = plan->kernel;
   shell.chunk_tokens = plan->chunk_tokens; shell.n_ctas = plan->n_ctas; shell.host_only = 0;
-  shell.sm_count = plan->sm_count; shell.n_row_blocks = plan->n_row_blocks; shell.stable_cache = 0; shell.n_pool_pages = plan->n_pool_pages;
+  shell.sm_count = plan->sm_count; shell.n_row_blocks = plan->n_row_blocks; shell.stable_cache = 0; shell.fuse_append = 0; shell.n_pool_pages = plan->n_pool_pages;
   shell.kv_tokens_read = plan->kv_tokens_read; shell.algorithmic_bytes = plan->algorithmic_bytes;
   shell.device_bytes = 0; shell.device_base = nullptr;
   memset(&shell.dev, 0, sizeof(shell.dev));
