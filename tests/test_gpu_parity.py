@@ -386,6 +386,16 @@ def test_deterministic_across_repeated_launches():
     assert plan.status() == 0
 
 
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_masked_prefill_of_a_parallel_segment(kernel):
+    """Many query tokens per branch in one step (block-diagonal across branches, causal inside a
+    branch, over a shared prefix): 240 query tokens = 27 row blocks that each stream the keys."""
+    wl = W.build_segment_workload("prefill", 29, 28, 4, 128, "bf16", 1e6, [300, 40], [[0, 17, 5], [0]],
+                                  [[100, 60, 31], [49]], serial_steps=1)
+    run, ref = compare_workload(wl, kernel=kernel)
+    assert run.outputs[0].shape[0] == 240
+
+
 def test_zero_new_tokens_is_a_no_op():
     E = engine()
     wl = W.build_segment_workload("e", 8, 28, 4, 128, "bf16", 1e6, [20], [[5, 9]], [[1, 1]])

@@ -336,6 +336,30 @@ def test_dense_and_descriptor_forms_agree():
         np.testing.assert_allclose(dense[P:], np.array(outs), atol=1e-12)
 
 
+def test_whole_branches_at_once_equal_dense_form():
+    """Teacher-forcing layout: every branch gets all its tokens in one step (block-diagonal mask
+    across branches, causal inside a branch).  The descriptor form equals Eq. 1-4 taken literally
+    for every one of those tokens, whatever order the branches are laid out in."""
+    Hq, Hkv, d, theta = 4, 2, 16, 1e4
+    P, lens = 6, [4, 1, 7]
+    wl = W.build_segment_workload("tf", 23, Hq, Hkv, d, "f32", theta, [P], [[0, 0, 0]], [lens], serial_steps=1)
+    run = run_workload(wl)
+    fill = wl.phases[0]
+    par = [p for p in wl.phases if p.label == "parallel-step"][0]
+    ser = wl.phases[-1]
+    # flat list in training order: prefix, then the branches one after the other, then the serial token
+    branch = [-1] * P + [b for b, n in enumerate(lens) for _ in range(n)] + [-1]
+    stage = [0] * P + [1] * sum(lens) + [2]
+    q = np.concatenate([np.zeros((P, Hq, d)), par.q, ser.q])
+    k = np.concatenate([fill.k_new, par.k_new, ser.k_new])
+    v = np.concatenate([fill.v_new, par.v_new, ser.v_new])
+    dense = oracle.dense_attn(q, k, v, branch, stage, theta, wl.sm_scale)
+    np.testing.assert_allclose(run.outputs[0], dense[P:P + sum(lens)], atol=1e-12)
+    np.testing.assert_allclose(run.outputs[1][0], dense[-1], atol=1e-12)
+    pos, _, _ = oracle.new_tokens(par.desc, oracle.MODE_BRANCH)
+    assert pos.tolist() == [P + i for n in lens for i in range(n)]
+
+
 def test_second_parallel_stage_descriptor_form_equals_dense_form():
     """A request that opens a second parallel stage (regions of the first stage and the serial
     tokens between the stages marked as shared): the descriptor form gives the positions and
