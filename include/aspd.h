@@ -301,6 +301,18 @@ int aspd_debug_read_token(const aspd_shape_t* shape, const void* pool /*device*/
                           int row, int kv_head, float* out /*host*/, void* stream);
 
 /*
+ * Move cached keys to new position IDs in place: K'(pos + delta) = RoPE(K'(pos), delta).  The
+ * paper's "Same-Re" variant renumbers the positions of a finished parallel segment sequentially
+ * and pays for it with a re-prefill of the KV cache (its position-ID ablation); because rotations
+ * compose, re-rotating the cached keys does the same with one read and one write per key and no
+ * model pass.  Token t is row rows[t] of physical page pages[t] (all KV heads); delta[t] may be
+ * negative.  pages, rows, delta: device int32[n].  V is untouched.  Each call rounds the keys to
+ * the storage dtype once more.
+ */
+int aspd_k_rerotate(const aspd_shape_t* shape, void* k_pool /*device*/, const int32_t* pages /*device*/,
+                    const int32_t* rows /*device*/, const int32_t* delta /*device*/, int n, void* stream);
+
+/*
  * Failure-path check: runs the library's bounded device-side wait on a barrier nobody ever
  * arrives on, with a limit of `limit_cycles` SM clock cycles (at most 4e9).  The kernel gives up
  * when the limit passes and reports ASPD_ERR_TIMEOUT through *status_out (host); the context

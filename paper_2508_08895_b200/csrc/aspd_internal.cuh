@@ -128,6 +128,8 @@ int launch_combine(const aspd_plan* p, void* out, cudaStream_t s);
 // attention pass that first writes this step's new K (rotated) and V rows into the pages it reads
 int launch_attn_mma_step(const aspd_plan* p, const void* q, const void* k_new, const void* v_new, void* k_pool,
                          void* v_pool, cudaStream_t s);
+int launch_rerotate(const aspd_shape_t* shape, void* k_pool, const int32_t* pages, const int32_t* rows, const int32_t* delta,
+                    int n, cudaStream_t s);
 int launch_wait_probe(long long limit_cycles, int32_t* status_dev, cudaStream_t s);
 int launch_read_token(const aspd_shape_t* shape, const void* pool, int64_t page, int row, int kv_head,
                       float* out_dev, cudaStream_t s);

@@ -58,6 +58,30 @@ __global__ void append_kernel(const T* __restrict__ k_new, const T* __restrict__
   *reinterpret_cast<T*>(vp + o1) = v_new[src + i + half];
 }
 
+// --------------------------------------------------------------------------- re-rotation
+// K'(pos + delta) = RoPE(K'(pos), delta): rotations compose, so cached keys can be moved to new
+// position IDs in place, reading and writing each key once, instead of being re-encoded from
+// the raw keys.  One block per (token, KV head); thread i rotates the pair (i, i + d/2).
+template <typename T>
+__global__ void rerotate_kernel(T* __restrict__ k_pool, const int32_t* __restrict__ pages, const int32_t* __restrict__ rows,
+                                const int32_t* __restrict__ delta, double theta, int n_kv_heads, int head_dim, int page_size) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int t = blockIdx.x / n_kv_heads, h = blockIdx.x % n_kv_heads, i = threadIdx.x, half = head_dim / 2;
+  if (i >= half) return;
+  double a = (double)delta[t] * pow(theta, -2.0 * (double)i / (double)head_dim);
+  a -= rint(a * 0.15915494309189535) * 6.283185307179586;
+  float sn, cs;
+  sincosf((float)a, &sn, &cs);
+  const uint32_t rb = head_dim * sizeof(T);
+  char* tile = reinterpret_cast<char*>(k_pool) + ((size_t)pages[t] * n_kv_heads + h) * tile_bytes(page_size, head_dim, sizeof(T));
+  T* p0 = reinterpret_cast<T*>(tile + tile_offset(rows[t], i * sizeof(T), rb));
+  T* p1 = reinterpret_cast<T*>(tile + tile_offset(rows[t], (i + half) * sizeof(T), rb));
+  const float x0 = to_f32(*p0), x1 = to_f32(*p1);
+  *p0 = from_f32<T>(x0 * cs - x1 * sn);
+  *p1 = from_f32<T>(x1 * cs + x0 * sn);
+}
+
 // ------------------------------------------------------------------- generic attention
 // One block per work item, one warp per query row at a time.  Lane j scores key j of each
 // group of 32 keys (a full dot product against the rotated, pre-scaled query held in shared
@@ -260,6 +284,16 @@ int launch_combine(const aspd_plan* p, void* out, cudaStream_t s) {
   else if (sh.head_dim == 128) ASPD_CMB(float, 128);
   else ASPD_CMB(float, 64);
 #undef ASPD_CMB
+}
+
+int launch_rerotate(const aspd_shape_t* sh, void* k_pool, const int32_t* pages, const int32_t* rows, const int32_t* delta,
+                    int n, cudaStream_t s) {
+  const dim3 grid(n * sh->n_kv_heads), block(sh->head_dim / 2);
+  if (sh->dtype == ASPD_DTYPE_BF16)
+    return status_of(launch_pdl(kPdlAppend, rerotate_kernel<__nv_bfloat16>, grid, block, 0, s, (__nv_bfloat16*)k_pool, pages, rows,
+                                delta, (double)sh->rope_theta, sh->n_kv_heads, sh->head_dim, sh->page_size));
+  return status_of(launch_pdl(kPdlAppend, rerotate_kernel<float>, grid, block, 0, s, (float*)k_pool, pages, rows, delta,
+                              (double)sh->rope_theta, sh->n_kv_heads, sh->head_dim, sh->page_size));
 }
 
 int launch_read_token(const aspd_shape_t* sh, const void* pool, int64_t page, int row, int kv_head, float* out_dev,

@@ -642,6 +642,16 @@ int aspd_step_host(aspd_plan_t* p, const void* q, const void* k_new, const void*
   return ASPD_OK;
 }
 
+int aspd_k_rerotate(const aspd_shape_t* shape, void* k_pool, const int32_t* pages, const int32_t* rows,
+                    const int32_t* delta, int n, void* stream) {
+  int rc = check_shape(shape);
+  if (rc) return rc;
+  if (n < 0) return ASPD_ERR_INVALID_ARG;
+  if (n == 0) return ASPD_OK;
+  if (!k_pool || !pages || !rows || !delta) return ASPD_ERR_INVALID_ARG;
+  return launch_rerotate(shape, k_pool, pages, rows, delta, n, (cudaStream_t)stream);
+}
+
 int aspd_debug_bounded_wait(int64_t limit_cycles, int32_t* status_out, void* stream) {
   if (!status_out || limit_cycles < 0 || limit_cycles > 4000000000LL) return ASPD_ERR_INVALID_ARG;
   int32_t* dev = nullptr;

@@ -396,6 +396,77 @@ def test_masked_prefill_of_a_parallel_segment(kernel):
     assert run.outputs[0].shape[0] == 240
 
 
+def test_rerotation_moves_cached_keys_to_new_positions():
+    """Same-Re without a re-prefill: after a segment, the branch tokens are renumbered
+    sequentially by rotating their cached keys by (new - old) positions in place."""
+    import torch
+    E = engine()
+    for wl in (W.build_segment_workload("re", 19, 28, 4, 128, "bf16", 1e6, [40], [[17, 3, 30]], [[1, 1, 1]]), W.config_tiny()):
+        run = E.run_workload(wl)
+        ref = oracle_run(wl)
+        d = wl.phases[-1].desc
+        P = int(d["prefix_len"][0])
+        pages, rows, delta, want = [], [], [], []
+        at = P                                         # sequential renumbering: branch after branch
+        for b in range(int(d["n_branches"][0])):
+            for k in range(int(d["br_kv_len"][b])):
+                s_ = int(d["br_kv_off"][b]) + k
+                pages.append(int(d["page_ids"][s_ // wl.page_size])); rows.append(s_ % wl.page_size)
+                delta.append(at - (P + k)); at += 1
+        t = lambda x: torch.tensor(x, dtype=torch.int32, device="cuda")
+        before = [run.read_token("k", pg, r, 0) for pg, r in zip(pages, rows)]
+        vbefore = run.cache.v.clone()
+        B.k_rerotate(run.shape, run.cache.k, t(pages), t(rows), t(delta))
+        torch.cuda.synchronize()
+        assert torch.equal(run.cache.v, vbefore)
+        # Two roundings to the storage dtype: the stored key is off by half an ulp of each element,
+        # the rotation mixes the pair (i, i + d/2), and the result is rounded again.
+        ulp_half = 2.0 ** -8 if wl.dtype == "bf16" else 4e-6    # bf16: 8 significand bits
+        moved = 0
+        for (pg, r, dl, old) in zip(pages, rows, delta, before):
+            for h in range(wl.Hkv):
+                got = run.read_token("k", pg, r, h)
+                want = oracle.rope(ref.k_pool[pg, h, r], float(dl), wl.theta)     # = RoPE(k, new position)
+                pair = np.hypot(want[:wl.d // 2], want[wl.d // 2:])
+                bound = 1.05 * ulp_half * (np.sqrt(2.0) * np.tile(pair, 2) + np.abs(want)) + 1e-7
+                assert np.all(np.abs(got - want) <= bound), (pg, r, h, float(np.max(np.abs(got - want) / bound)))
+            moved += int(dl != 0 and not np.array_equal(run.read_token("k", pg, r, 0), old))
+        assert moved > 0
+
+
+def test_same_re_serial_decoding_after_rerotation():
+    """The paper's Same-Re variant end to end: after the segment the branch tokens get sequential
+    position IDs (keys re-rotated in place), then serial decoding continues over the merged cache.
+    The oracle rotates its own fp64 keys by the same offsets (RoPE composition, pinned on the CPU)."""
+    import torch
+    E = engine()
+    wl = W.build_segment_workload("same-re", 23, 28, 4, 128, "bf16", 1e6, [70, 33], [[20, 9, 31], [5, 40]],
+                                  [[1, 1, 1], [1, 1]], serial_steps=2)
+    run, ref = E.WorkloadRun(wl), OracleRun(wl)
+    serial = [i for i, ph in enumerate(wl.phases) if ph.mode == W.MODE_SERIAL]
+    for ph in wl.phases[:serial[0]]:
+        run.step(ph); ref.step(ph)
+    d = wl.phases[serial[0] - 1].desc
+    pages, rows, delta = [], [], []
+    for r in range(len(d["prefix_len"])):
+        P, at = int(d["prefix_len"][r]), int(d["prefix_len"][r])
+        pg0 = int(d["page_begin"][r])
+        for b in range(int(d["branch_begin"][r]), int(d["branch_begin"][r]) + int(d["n_branches"][r])):
+            for k in range(int(d["br_kv_len"][b])):
+                s_ = int(d["br_kv_off"][b]) + k
+                pages.append(int(d["page_ids"][pg0 + s_ // wl.page_size])); rows.append(s_ % wl.page_size)
+                delta.append(at - (P + k)); at += 1
+    t = lambda x: torch.tensor(x, dtype=torch.int32, device="cuda")
+    B.k_rerotate(run.shape, run.cache.k, t(pages), t(rows), t(delta))
+    for pg, r, dl in zip(pages, rows, delta):
+        for h in range(wl.Hkv):
+            ref.k_pool[pg, h, r] = oracle.rope(ref.k_pool[pg, h, r], float(dl), wl.theta)
+    assert max(delta) > 0
+    for i in serial:                        # the serial position P + sum(len) is already sequential
+        got, want = run.step(wl.phases[i]), ref.step(wl.phases[i])
+        check(got, want, wl.dtype, "same-re serial step")
+
+
 def test_zero_new_tokens_is_a_no_op():
     E = engine()
     wl = W.build_segment_workload("e", 8, 28, 4, 128, "bf16", 1e6, [20], [[5, 9]], [[1, 1]])

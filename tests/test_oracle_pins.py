@@ -135,6 +135,14 @@ def test_rope_closed_forms():
             np.testing.assert_allclose(y, np.concatenate([z.real, z.imag]), atol=1e-10)
 
 
+def test_rope_rotations_compose():
+    """RoPE(RoPE(x, p), delta) = RoPE(x, p + delta): what re-rotating cached keys relies on."""
+    rng = np.random.default_rng(4)
+    x = rng.standard_normal(128)
+    for p, dlt in [(5.0, 11.0), (1040.0, -17.0), (16384.0, 300.0)]:
+        np.testing.assert_allclose(oracle.rope(oracle.rope(x, p, 1e6), dlt, 1e6), oracle.rope(x, p + dlt, 1e6), atol=1e-9)
+
+
 def _library_rotary(x, positions, theta):
     """cos/sin tables from the definition of the frequencies, applied by the rotate-half
     routine of the `transformers` Llama implementation (a library routine)."""
