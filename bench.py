@@ -178,6 +178,85 @@ def reduce_over_ranks(times_ms, units, device, world):
 
 
 # ------------------------------------------------------------------------------ our arm
+def fill_caches(wl, shape, caches):
+    """Fill every layer's pools through the library's own append (same values, distinct memory)."""
+    import torch
+    from paper_2508_08895_b200 import binding as B, engine as E
+    for ph in wl.phases[:-1]:
+        plan = B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode)
+        pos, _, _ = B.positions(ph.desc, ph.mode)
+        pos_d = torch.from_numpy(pos.copy()).cuda()
+        k_d, v_d = E.to_device(ph.k_new, wl.dtype), E.to_device(ph.v_new, wl.dtype)
+        for c in caches:
+            B.kv_append(plan, k_d, v_d, pos_d, c.k, c.v)
+        torch.cuda.synchronize()
+        plan.destroy()
+        del k_d, v_d
+
+
+def run_rerotate(args):
+    """--op rerotate: the Same-Re renumbering of a finished segment, aspd_k_rerotate over every
+    branch token of the workload, one launch per layer.  One GPU; prints its own JSON line."""
+    import torch
+    from paper_2508_08895_b200 import binding as B, engine as E
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback")
+    wl = build_workload(args.workload, 0, args.requests)
+    shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
+    d = wl.phases[-1].desc
+    pages, rows, delta = [], [], []
+    for r in range(len(d["prefix_len"])):
+        P = at = int(d["prefix_len"][r])
+        for b in range(int(d["branch_begin"][r]), int(d["branch_begin"][r]) + int(d["n_branches"][r])):
+            k = np.arange(int(d["br_kv_len"][b]))
+            s_ = int(d["br_kv_off"][b]) + k
+            pages.append(d["page_ids"][int(d["page_begin"][r]) + s_ // wl.page_size]); rows.append(s_ % wl.page_size)
+            delta.append(at - P + 0 * k); at += len(k)        # sequential renumbering: (at + k) - (P + k)
+    pages, rows, delta = (torch.from_numpy(np.concatenate(x).astype(np.int32)).cuda() for x in (pages, rows, delta))
+    n = int(pages.numel())
+    es = 2 if wl.dtype == "bf16" else 4
+    alg = n * (2 * wl.Hkv * wl.d * es + 12)
+    L = max(args.layers, int(np.ceil(4 * 126e6 / alg)))
+    caches = [E.LayerCache(shape, wl.n_pool_pages) for _ in range(L)]
+    fill_caches(wl, shape, caches)
+
+    def step():
+        for c in caches:
+            B.k_rerotate(shape, c.k, pages, rows, delta)
+    for _ in range(2):
+        step()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for _ in range(max(args.warmup, 3)):
+        graph.replay()
+    sampler = ClockSampler(0)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    for _ in range(args.steps):
+        graph.replay()
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop()
+    peak, peak_kind = measured_peaks()
+    achieved = alg * L * args.steps / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "op": "rerotate", "metric": "rerotated_key_tokens_per_second", "value": n * L * args.steps / (ms * 1e-3),
+        "unit": "tokens/s", "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
+        "higher_is_better": True, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "layers": L, "tokens_per_layer": n, "heads": wl.Hkv, "head_dim": wl.d,
+                   "l2": "%.1f GB of distinct keys per step" % (alg * L / 1e9)},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "peak_kind": "of " + peak_kind, "kernel": "rerotate_kernel",
+                     "kernel_us": ms / args.steps / L * 1e3, "algorithmic_bytes_per_launch": alg},
+        "gpu_launches": L * args.steps, "clocks": clocks}))
+    return 0
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -203,17 +282,7 @@ def run_ours(args):
     caches = [E.LayerCache(shape, wl.n_pool_pages) for _ in range(L)]
     kernel = {"auto": B.KERNEL_AUTO, "generic": B.KERNEL_GENERIC, "mma": B.KERNEL_MMA}[args.kernel]
 
-    # fill every layer's pools through the library's own append (same values, distinct memory)
-    for ph in wl.phases[:-1]:
-        plan = B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode)
-        pos, _, _ = B.positions(ph.desc, ph.mode)
-        pos_d = torch.from_numpy(pos.copy()).cuda()
-        k_d, v_d = E.to_device(ph.k_new, wl.dtype), E.to_device(ph.v_new, wl.dtype)
-        for c in caches:
-            B.kv_append(plan, k_d, v_d, pos_d, c.k, c.v)
-        torch.cuda.synchronize()
-        plan.destroy()
-        del k_d, v_d
+    fill_caches(wl, shape, caches)
 
     ph = wl.phases[-1]
     # decode loop: a layer's pools are written only by that layer's own step, so the plan may carry
@@ -374,6 +443,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="serving-mix", choices=["qwen7b-layer", "branch-open", "long-rag", "serving-mix"])
+    ap.add_argument("--op", default="step", choices=["step", "rerotate"],
+                    help="step: the attention step (the benchmark); rerotate: the Same-Re key re-rotation kernel alone")
     ap.add_argument("--layers", type=int, default=28)
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "mma"])
     ap.add_argument("--chunk", type=int, default=0)
@@ -388,6 +459,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.op == "rerotate":
+        return run_rerotate(args)
     return run_ours(args)
 
 

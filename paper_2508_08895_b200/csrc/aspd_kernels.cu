@@ -61,25 +61,56 @@ __global__ void append_kernel(const T* __restrict__ k_new, const T* __restrict__
 // --------------------------------------------------------------------------- re-rotation
 // K'(pos + delta) = RoPE(K'(pos), delta): rotations compose, so cached keys can be moved to new
 // position IDs in place, reading and writing each key once, instead of being re-encoded from
-// the raw keys.  One block per (token, KV head); thread i rotates the pair (i, i + d/2).
+// the raw keys.  A thread owns one 16-byte chunk of the first half of a token's row and its
+// partner chunk in the second half (the pairs (i, i + d/2)), computes the chunk's sines and
+// cosines once and applies them to every KV head of the token.
+constexpr int kRerotateThreads = 256;
+struct InvFreq {          // theta^(-2i/d), computed by the host in double; by value in the launch
+  double f[64];
+};
 template <typename T>
-__global__ void rerotate_kernel(T* __restrict__ k_pool, const int32_t* __restrict__ pages, const int32_t* __restrict__ rows,
-                                const int32_t* __restrict__ delta, double theta, int n_kv_heads, int head_dim, int page_size) {
+__global__ void __launch_bounds__(kRerotateThreads)
+rerotate_kernel(T* __restrict__ k_pool, const int32_t* __restrict__ pages, const int32_t* __restrict__ rows,
+                const int32_t* __restrict__ delta, const InvFreq table, int n, int n_kv_heads, int head_dim, int page_size) {
+  constexpr int VEC = 16 / sizeof(T);
+  __shared__ double inv_freq[64];
   pdl_launch_dependents();
+  const int half = head_dim / 2, chunks = half / VEC;
+  if (threadIdx.x < half) inv_freq[threadIdx.x] = table.f[threadIdx.x];
+  __syncthreads();
   pdl_wait();
-  const int t = blockIdx.x / n_kv_heads, h = blockIdx.x % n_kv_heads, i = threadIdx.x, half = head_dim / 2;
-  if (i >= half) return;
-  double a = (double)delta[t] * pow(theta, -2.0 * (double)i / (double)head_dim);
-  a -= rint(a * 0.15915494309189535) * 6.283185307179586;
-  float sn, cs;
-  sincosf((float)a, &sn, &cs);
+  const long gid = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long t = gid / chunks;
+  const int c = (int)(gid % chunks);
+  if (t >= n) return;
+  float sn[VEC], cs[VEC];
+  const double dl = (double)delta[t];
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) {
+    double a = dl * inv_freq[c * VEC + j];
+    a -= rint(a * 0.15915494309189535) * 6.283185307179586;
+    sincosf((float)a, &sn[j], &cs[j]);
+  }
   const uint32_t rb = head_dim * sizeof(T);
-  char* tile = reinterpret_cast<char*>(k_pool) + ((size_t)pages[t] * n_kv_heads + h) * tile_bytes(page_size, head_dim, sizeof(T));
-  T* p0 = reinterpret_cast<T*>(tile + tile_offset(rows[t], i * sizeof(T), rb));
-  T* p1 = reinterpret_cast<T*>(tile + tile_offset(rows[t], (i + half) * sizeof(T), rb));
-  const float x0 = to_f32(*p0), x1 = to_f32(*p1);
-  *p0 = from_f32<T>(x0 * cs - x1 * sn);
-  *p1 = from_f32<T>(x1 * cs + x0 * sn);
+  const size_t tb = tile_bytes(page_size, head_dim, sizeof(T));
+  char* tile = reinterpret_cast<char*>(k_pool) + (size_t)pages[t] * n_kv_heads * tb;
+  const uint32_t o0 = tile_offset(rows[t], c * 16, rb), o1 = tile_offset(rows[t], half * sizeof(T) + c * 16, rb);
+#pragma unroll 4
+  for (int h = 0; h < n_kv_heads; ++h) {
+    uint4* p0 = reinterpret_cast<uint4*>(tile + h * tb + o0);
+    uint4* p1 = reinterpret_cast<uint4*>(tile + h * tb + o1);
+    uint4 u0 = *p0, u1 = *p1;
+    T* x0 = reinterpret_cast<T*>(&u0);
+    T* x1 = reinterpret_cast<T*>(&u1);
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+      const float a = to_f32(x0[j]), b = to_f32(x1[j]);
+      x0[j] = from_f32<T>(a * cs[j] - b * sn[j]);
+      x1[j] = from_f32<T>(b * cs[j] + a * sn[j]);
+    }
+    *p0 = u0;
+    *p1 = u1;
+  }
 }
 
 // ------------------------------------------------------------------- generic attention
@@ -288,12 +319,15 @@ int launch_combine(const aspd_plan* p, void* out, cudaStream_t s) {
 
 int launch_rerotate(const aspd_shape_t* sh, void* k_pool, const int32_t* pages, const int32_t* rows, const int32_t* delta,
                     int n, cudaStream_t s) {
-  const dim3 grid(n * sh->n_kv_heads), block(sh->head_dim / 2);
+  const int chunks = sh->head_dim / 2 / (16 / esize_of(sh->dtype));
+  const dim3 grid((unsigned)(((long)n * chunks + kRerotateThreads - 1) / kRerotateThreads)), block(kRerotateThreads);
+  InvFreq table;
+  for (int i = 0; i < sh->head_dim / 2; ++i) table.f[i] = pow((double)sh->rope_theta, -2.0 * i / (double)sh->head_dim);
   if (sh->dtype == ASPD_DTYPE_BF16)
     return status_of(launch_pdl(kPdlAppend, rerotate_kernel<__nv_bfloat16>, grid, block, 0, s, (__nv_bfloat16*)k_pool, pages, rows,
-                                delta, (double)sh->rope_theta, sh->n_kv_heads, sh->head_dim, sh->page_size));
+                                delta, table, n, sh->n_kv_heads, sh->head_dim, sh->page_size));
   return status_of(launch_pdl(kPdlAppend, rerotate_kernel<float>, grid, block, 0, s, (float*)k_pool, pages, rows, delta,
-                              (double)sh->rope_theta, sh->n_kv_heads, sh->head_dim, sh->page_size));
+                              table, n, sh->n_kv_heads, sh->head_dim, sh->page_size));
 }
 
 int launch_read_token(const aspd_shape_t* sh, const void* pool, int64_t page, int row, int kv_head, float* out_dev,
