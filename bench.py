@@ -51,6 +51,30 @@ FALLBACK_HBM_GBS = 6650.0
 TRAFFIC_PER_ALGORITHMIC_BYTE = 1.015
 
 
+def measured_tensor_peak():
+    """Dense bf16 TFLOP/s of a library GEMM inside a long step (the sustained figure)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["bf16_tflops_sustained"]), "measured (sustained)"
+        except Exception:
+            pass
+    return 1400.0, "fallback (sustained)"
+
+
+def attention_flops(desc, Hq: int, d: int) -> float:
+    """2 contractions x 2 flops x d per (query row, visible key) of a parallel-mode step."""
+    pairs = 0
+    for r in range(len(desc["prefix_len"])):
+        b0, nb = int(desc["branch_begin"][r]), int(desc["n_branches"][r])
+        ql, kl = desc["br_q_len"][b0:b0 + nb].astype(np.int64), desc["br_kv_len"][b0:b0 + nb].astype(np.int64)
+        shared = int(desc["prefix_len"][r]) + int(kl[ql < 0].sum())
+        for q, k in zip(ql, kl):
+            if q > 0:
+                pairs += q * (shared + k - q) + q * (q + 1) // 2
+    return 4.0 * d * Hq * float(pairs)
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -65,6 +89,8 @@ def build_workload(name: str, rank: int, requests: int = 0):
     from paper_2508_08895_b200 import workloads as W
     if name == "serving-mix" and requests > 0:      # a smaller batch of the same mix (profiling captures)
         return W.config_serving_mix(seed=W.SEED_BASE + 4 + 16 * rank, n_req=requests)
+    if name == "masked-prefill":
+        return W.config_masked_prefill(seed=W.SEED_BASE + 5 + 16 * rank, n_req=requests or 32)
     fn = W.CONFIGS[name]
     base = {"tiny-f32": 0, "qwen7b-layer": 1, "branch-open": 2, "long-rag": 3, "serving-mix": 4}[name]
     if name == "branch-open":
@@ -397,6 +423,13 @@ def run_ours(args):
         alg = float(info.algorithmic_bytes)
         value = total_new * L * args.steps / (ms * 1e-3)
         achieved = alg / (kernel_ms * 1e-3) / 1e9
+        tensor = None
+        if args.workload == "masked-prefill":      # many query rows per key: the contraction bounds it, not HBM
+            tpeak, tkind = measured_tensor_peak()
+            fl = attention_flops(ph.desc, wl.Hq, wl.d)
+            tensor = {"bound": "tensor", "achieved": fl / (kernel_ms * 1e-3) / 1e12, "peak": tpeak, "unit": "TFLOP/s",
+                      "frac": fl / (kernel_ms * 1e-3) / 1e12 / tpeak, "traffic": None, "peak_kind": "of " + tkind,
+                      "kernel": "split-K attention pass", "kernel_us": kernel_ms * 1e3, "flops_per_launch": fl}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -424,6 +457,8 @@ def run_ours(args):
             "gpu_launches": (2 if fused and info.fused_append else 3) * L * args.steps,
             "clocks": clocks,
         }
+        if tensor is not None:
+            line["roofline_hbm"], line["roofline"] = line["roofline"], tensor
         if world == 1 and not args.no_cpu_baseline:
             v, cores, sec, reps_o, n_o = oracle_sample(wl, budget_s=args.cpu_budget)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
@@ -442,7 +477,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="serving-mix", choices=["qwen7b-layer", "branch-open", "long-rag", "serving-mix"])
+    ap.add_argument("--workload", default="serving-mix", choices=["qwen7b-layer", "branch-open", "long-rag", "serving-mix", "masked-prefill"])
     ap.add_argument("--op", default="step", choices=["step", "rerotate"],
                     help="step: the attention step (the benchmark); rerotate: the Same-Re key re-rotation kernel alone")
     ap.add_argument("--layers", type=int, default=28)

@@ -55,6 +55,11 @@ enum Bar { K_FULL = 0, K_EMPTY = 2, V_FULL = 4, V_EMPTY = 6, S_FULL = 8, S_EMPTY
 constexpr int kItemCache = 10;      // items of a CTA kept in shared memory (more are read from global)
 constexpr int kMaxTokPerItem = 16;  // tokens of a row block whose ranges are cached (n_q_tok is at most 64 / G)
 
+// The wide variant of the kernel (row blocks of up to 128 query rows, no replication) fills all
+// rows of the P tile; it keeps a single query tile and puts Misc, followed by the reference maxima
+// of 2 x 128 rows, where the second query tile would be.
+constexpr uint32_t OFF_MISC_WIDE = OFF_Q + kTileBytes;
+
 struct Misc {
   uint64_t bars[NUM_BARS];
   float smax[2][256];          // per S buffer: tile maximum of every softmax thread
@@ -119,6 +124,24 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+// The same two, executed by a whole warp with warp-uniform operands; lane 0 alone issues.  With
+// uniform control flow around them the descriptors stay in the uniform datapath.
+__device__ __forceinline__ void tc_commit_lane0(uint32_t bar) {
+  asm volatile(
+      "{\n\t.reg .pred e;\n\t.reg .u32 l;\n\t"
+      "mov.u32 l, %%laneid;\n\t"
+      "setp.eq.u32 e, l, 0;\n\t"
+      "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_lane0(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p, e;\n\t.reg .u32 l;\n\t"
+      "mov.u32 l, %%laneid;\n\t"
+      "setp.eq.u32 e, l, 0;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
 }
 __device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
@@ -337,18 +360,137 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
   return !named_sync_or(1, kSoftmaxThreads, dead || *ab);
 }
 
+// Row blocks of 65..128 query rows: every TMEM lane is a row of its own (no replication), thread
+// (half, r) takes columns [64 half, 64 half + 64) of row r in two chunks of 32.  One pass per
+// tile: the exponentials are taken against the current reference maximum while the largest
+// exponent is tracked; only when a row's largest exponent exceeds 2^8 (always on the row's first
+// visible key) the reference is raised and the warp repeats the pass from TMEM.
+__device__ __forceinline__ bool softmax_item_wide(const Ctx& c, const DeviceItem& it, Misc* misc, uint32_t bars, uint32_t smem_p,
+                                                  uint32_t tmem, int item_no, int& g) {
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int r = tid & 127, half = tid >> 7;
+  const int col0 = half * 64;
+  const int G = c.n_q_heads / c.n_kv_heads, M = it.n_q_tok * G;
+  const int n_tiles = (it.n_pages + 7) >> 3;
+  volatile int* ab = &misc->abort_flag;
+  float* fin_m_wide = reinterpret_cast<float*>(misc + 1);
+  int4 vis = make_int4(0, 0, 0, 0);
+  if (r < M) vis = (item_no < kItemCache && r / G < kMaxTokPerItem) ? misc->vis[item_no][r / G] : c.pd.tok_vis[it.q_tok0 + r / G];
+  const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+  const bool o_owner = half == 0;
+  const int ob = item_no & 1;
+  float m_ref = -INFINITY, l = 0.f;
+  bool dead = false;
+  for (int t = 0; t < n_tiles; ++t, ++g) {
+    const int sb = g & 1;
+    dead |= !mbar_wait(bars + 8 * (S_FULL + sb), (g >> 1) & 1, ab);
+    tc_fence_after();
+    if (tid == 0) ASPD_STAMP(c, g, 0);
+    const uint32_t s_addr = tmem + lane_addr + COL_S + sb * 128 + col0;
+    uint32_t pk[32];                                // the row's 64 probabilities of this tile, bf16 pairs
+    float tile_sum, tmax;
+    // p = 2^(s * scale - base) for the thread's 64 columns; tmax = largest exponent
+    auto pass = [&](float base) {
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+      float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+      const float nb = -base;
+#pragma unroll
+      for (int ch = 0; ch < 2; ++ch) {
+        float s[32];
+        ASPD_TMEM_LD32(s_addr + ch * 32, s, 0);
+        tmem_wait_ld();
+#pragma unroll
+        for (int pg = 0; pg < 2; ++pg) {
+          const int nv = misc->nval[g & 3][col0 / 16 + ch * 2 + pg];
+          const int kb = it.key0 + t * kTile + col0 + ch * 32 + pg * 16;
+          const uint32_t mask = bits_between(0, min(nv, vis.x - kb)) | bits_between(vis.y - kb, min(nv, vis.z - kb));
+#pragma unroll
+          for (int i = 0; i < 16; i += 4) {
+            float e0 = fmaf(s[pg * 16 + i], c.scale_log2, nb), e1 = fmaf(s[pg * 16 + i + 1], c.scale_log2, nb);
+            float e2 = fmaf(s[pg * 16 + i + 2], c.scale_log2, nb), e3 = fmaf(s[pg * 16 + i + 3], c.scale_log2, nb);
+            if (mask != 0xFFFFu) {
+              e0 = (mask >> i) & 1u ? e0 : -INFINITY;
+              e1 = (mask >> (i + 1)) & 1u ? e1 : -INFINITY;
+              e2 = (mask >> (i + 2)) & 1u ? e2 : -INFINITY;
+              e3 = (mask >> (i + 3)) & 1u ? e3 : -INFINITY;
+            }
+            mx0 = fmaxf(mx0, e0); mx1 = fmaxf(mx1, e1); mx2 = fmaxf(mx2, e2); mx3 = fmaxf(mx3, e3);
+            e0 = ex2(e0); e1 = ex2(e1); e2 = ex2(e2); e3 = ex2(e3);
+            sum0 += e0; sum1 += e1; sum2 += e2; sum3 += e3;
+            pk[ch * 16 + pg * 8 + (i >> 1)] = pack_bf16(e0, e1);
+            pk[ch * 16 + pg * 8 + (i >> 1) + 1] = pack_bf16(e2, e3);
+          }
+        }
+      }
+      tile_sum = (sum0 + sum1) + (sum2 + sum3);
+      tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+    };
+    const float base = m_ref == -INFINITY ? 0.f : m_ref;
+    pass(base);
+    if (tid == 0) ASPD_STAMP(c, g, 1);
+    misc->smax[sb][tid] = tmax;
+    named_sync(1, kSoftmaxThreads);
+    if (tid == 0) ASPD_STAMP(c, g, 2);
+    const float row_tmax = fmaxf(misc->smax[sb][r], misc->smax[sb][128 + r]);
+    // raise the reference: on the row's first visible key, or when an exponent passed 2^8
+    const bool upd = m_ref == -INFINITY ? row_tmax > -INFINITY : row_tmax > kRaise;
+    float alpha = 1.f;
+    if (upd) { alpha = m_ref == -INFINITY ? 0.f : ex2(-row_tmax); m_ref = base + row_tmax; }
+    l *= alpha;
+    const bool any_upd = __any_sync(0xffffffffu, upd);
+    if (t > 0 && o_owner && any_upd) {              // the owners of the rows rescale O in TMEM
+      dead |= !mbar_wait(bars + 8 * P_EMPTY, (g - 1) & 1, ab);   // PV of the previous tile is done
+      tc_fence_after();
+      const uint32_t o_addr = tmem + lane_addr + COL_O + ob * 128;
+#pragma unroll 1
+      for (int q4 = 0; q4 < 4; ++q4) {
+        float o[32];
+        ASPD_TMEM_LD32(o_addr + q4 * 32, o, 0);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] *= alpha;
+        ASPD_TMEM_ST32(o_addr + q4 * 32, o, 0);
+      }
+      tmem_wait_st();
+    }
+    if (any_upd) pass(m_ref == -INFINITY ? 0.f : m_ref);   // the whole warp again (TMEM loads are warp-wide)
+    l += tile_sum;
+    tc_fence_before();
+    mbar_arrive(bars + 8 * (S_EMPTY + sb));
+    if (tid == 0) ASPD_STAMP(c, g, 3);
+    if (g > 0) dead |= !mbar_wait(bars + 8 * P_EMPTY, (g - 1) & 1, ab);
+    if (tid == 0) ASPD_STAMP(c, g, 4);
+#pragma unroll
+    for (int c8 = 0; c8 < 8; ++c8) {
+      const int kk = col0 + c8 * 8;
+      const uint32_t addr = smem_p + (kk >> 6) * kHalf + r * 128 + ((((kk & 63) >> 3) ^ (r & 7)) << 4);
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[c8 * 4 + 0]), "r"(pk[c8 * 4 + 1]),
+                   "r"(pk[c8 * 4 + 2]), "r"(pk[c8 * 4 + 3]) : "memory");
+    }
+    fence_async_smem();
+    tc_fence_before();
+    mbar_arrive(bars + 8 * P_FULL);
+    if (tid == 0) ASPD_STAMP(c, g, 5);
+  }
+  dead |= !mbar_wait(bars + 8 * (O_EMPTY + ob), ((item_no >> 1) & 1) ^ 1, ab);
+  if (half == 0) fin_m_wide[ob * 128 + r] = m_ref;
+  misc->fin_l[ob][tid] = l;
+  mbar_arrive(bars + 8 * (E_FULL + ob));
+  return !named_sync_or(1, kSoftmaxThreads, dead || *ab);
+}
+
 // Rotate the item's query rows (RoPE at the token's position, cos/sin table from the plan),
 // round to bf16 and store them, replicated KS = 128 / R times, as the 128-byte-swizzled K-major
 // A operand.  Called by the 128 epilogue threads (rank 0..127); all loads of a thread's rows
 // are issued before the first use.
-__device__ __forceinline__ void prep_q(const Ctx& c, const DeviceItem& it, uint32_t qbuf, int rank) {
+__device__ __forceinline__ void prep_q(const Ctx& c, const DeviceItem& it, uint32_t qbuf, int rank, int e0 = 0) {
   const int G = c.n_q_heads / c.n_kv_heads;
-  const int M = it.n_q_tok * G, R = M <= 32 ? 32 : 64, KS = 128 / R;
+  const int M = it.n_q_tok * G, R = M <= 32 ? 32 : (M <= 64 ? 64 : 128), KS = 128 / R;   // R = 128: second call with e0 = 512
   uint4 a[4], b[4];
   float4 w[4][4];
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
-    const int e = rank + u * 128, r = e >> 3, ch = e & 7;     // row, 8-element chunk of each span
+    const int e = e0 + rank + u * 128, r = e >> 3, ch = e & 7;     // row, 8-element chunk of each span
     a[u] = make_uint4(0, 0, 0, 0); b[u] = make_uint4(0, 0, 0, 0);
 #pragma unroll
     for (int i = 0; i < 4; ++i) w[u][i] = make_float4(1.f, 0.f, 1.f, 0.f);
@@ -364,7 +506,7 @@ __device__ __forceinline__ void prep_q(const Ctx& c, const DeviceItem& it, uint3
   }
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
-    const int e = rank + u * 128, r = e >> 3, ch = e & 7;
+    const int e = e0 + rank + u * 128, r = e >> 3, ch = e & 7;
     if (e >= R * 8) break;
     const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&a[u]);
     const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&b[u]);
@@ -443,13 +585,17 @@ __device__ __forceinline__ void append_new_rows(const Ctx& c, int rank, int d0, 
 }
 
 // --------------------------------------------------------------------------------- the kernel
+// WIDE: row blocks of up to 128 query rows (plans that deal whole streams to the CTAs); one
+// query tile instead of two, Misc in the place of the second.
+template <bool WIDE>
 __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
-  Misc* misc = reinterpret_cast<Misc*>(smem + OFF_MISC);
-  const uint32_t bars = base + OFF_MISC;          // bars[] is the first member of Misc
+  constexpr uint32_t off_misc = WIDE ? OFF_MISC_WIDE : OFF_MISC;
+  Misc* misc = reinterpret_cast<Misc*>(smem + off_misc);
+  const uint32_t bars = base + off_misc;          // bars[] is the first member of Misc
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* ab = &misc->abort_flag;
   if (tid == 0) ASPD_CTA_STAMP(c, 0);
@@ -509,8 +655,15 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     for (int idx = item_begin; idx < item_end; ++idx, ++item_no) {
       const DeviceItem it = get_item(c, misc, idx, item_begin);
       const int M = it.n_q_tok * (c.n_q_heads / c.n_kv_heads);
-      const bool ok = M <= 32 ? softmax_item<32>(c, it, misc, bars, base + OFF_P, tmem, item_no, g)
-                              : softmax_item<64>(c, it, misc, bars, base + OFF_P, tmem, item_no, g);
+      bool ok;
+      if constexpr (WIDE) {
+        ok = M <= 32 ? softmax_item<32>(c, it, misc, bars, base + OFF_P, tmem, item_no, g)
+           : M <= 64 ? softmax_item<64>(c, it, misc, bars, base + OFF_P, tmem, item_no, g)
+                     : softmax_item_wide(c, it, misc, bars, base + OFF_P, tmem, item_no, g);
+      } else {
+        ok = M <= 32 ? softmax_item<32>(c, it, misc, bars, base + OFF_P, tmem, item_no, g)
+                     : softmax_item<64>(c, it, misc, bars, base + OFF_P, tmem, item_no, g);
+      }
       if (!ok) break;
     }
   } else if (warp == W_KPROD || warp == W_VPROD) {
@@ -584,58 +737,69 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     // =================================== MMA issuer ===================================
     // The tiles of all items form one pipeline: S of tile g is issued before P.V of tile g - 1,
     // also across an item boundary, so the tensor pipe and the softmax warps never drain
-    // between items.
-    if (lane == 0) {
-      struct TileRef { int npg, first, last, qb, ob, item_no; };
+    // between items.  The whole warp walks the loops with warp-uniform values (what comes from
+    // shared memory is broadcast from lane 0), lane 0 issues the MMAs and commits.
+    {
+      const uint32_t full_mask = 0xffffffffu;
+      const uint32_t tmem_u = __shfl_sync(full_mask, tmem, 0);
+      const uint32_t base_u = __shfl_sync(full_mask, base, 0), bars_u = base_u + off_misc;
+      struct TileRef { int npg, first, last, qb, ob, item_no; };   // qb: query tile (always 0 in the wide kernel)
+      auto q_fill = [](int item_no) { return WIDE ? item_no : item_no >> 1; };   // how often the item's query tile was filled before
+      auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(full_mask, mbar_wait(bar, parity, ab)) != 0; };
       const uint32_t idesc_pv = instr_desc(128, 1);
       auto issue_s = [&](const TileRef& tr, int g) -> bool {
         const int sb = g & 1;
-        if (tr.first && !mbar_wait(bars + 8 * (Q_FULL + tr.qb), (tr.item_no >> 1) & 1, ab)) return false;
-        if (!mbar_wait(bars + 8 * (K_FULL + sb), (g >> 1) & 1, ab)) return false;
-        if (!mbar_wait(bars + 8 * (S_EMPTY + sb), ((g >> 1) & 1) ^ 1, ab)) return false;
+        if (tr.first && !wait_all(bars_u + 8 * (Q_FULL + tr.qb), q_fill(tr.item_no) & 1)) return false;
+        if (!wait_all(bars_u + 8 * (K_FULL + sb), (g >> 1) & 1)) return false;
+        if (lane == 0) ASPD_STAMP(c, g, 15);
+        if (!wait_all(bars_u + 8 * (S_EMPTY + sb), ((g >> 1) & 1) ^ 1)) return false;
         tc_fence_after();
-        ASPD_STAMP(c, g, 8);
-        const uint32_t qbuf = base + OFF_Q + tr.qb * kTileBytes, kbuf = base + OFF_K + sb * kTileBytes;
+        if (lane == 0) ASPD_STAMP(c, g, 8);
+        const uint32_t qbuf = base_u + OFF_Q + tr.qb * kTileBytes, kbuf = base_u + OFF_K + sb * kTileBytes;
         const uint32_t idesc_s = instr_desc((uint32_t)tr.npg * 16u, 0);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
           // k-step ks covers head_dim elements [16 ks, 16 ks + 16): span ks / 4, 32 bytes per step
           const uint64_t a = smem_desc(qbuf + (ks >> 2) * kHalf + (ks & 3) * 32, 16, 1024);
           const uint64_t b = smem_desc(kbuf + (ks >> 2) * 1024 + (ks & 3) * 32, 16, 2048);
-          tc_mma(tmem + COL_S + sb * 128, a, b, idesc_s, ks > 0 ? 1u : 0u);
+          tc_mma_lane0(tmem_u + COL_S + sb * 128, a, b, idesc_s, ks > 0 ? 1u : 0u);
         }
-        ASPD_STAMP(c, g, 9);
-        tc_commit(bars + 8 * (S_FULL + sb));
-        tc_commit(bars + 8 * (K_EMPTY + sb));
-        if (tr.last) tc_commit(bars + 8 * (Q_EMPTY + tr.qb));
+        if (lane == 0) ASPD_STAMP(c, g, 9);
+        tc_commit_lane0(bars_u + 8 * (S_FULL + sb));
+        tc_commit_lane0(bars_u + 8 * (K_EMPTY + sb));
+        if (tr.last) tc_commit_lane0(bars_u + 8 * (Q_EMPTY + tr.qb));
         return true;
       };
       auto issue_pv = [&](const TileRef& tr, int g) -> bool {
-        ASPD_STAMP(c, g, 10);
-        if (!mbar_wait(bars + 8 * P_FULL, g & 1, ab)) return false;
-        ASPD_STAMP(c, g, 11);
-        if (!mbar_wait(bars + 8 * (V_FULL + (g & 1)), (g >> 1) & 1, ab)) return false;
-        if (tr.first && !mbar_wait(bars + 8 * (O_EMPTY + tr.ob), ((tr.item_no >> 1) & 1) ^ 1, ab)) return false;
+        if (lane == 0) ASPD_STAMP(c, g, 10);
+        if (!wait_all(bars_u + 8 * P_FULL, g & 1)) return false;
+        if (lane == 0) ASPD_STAMP(c, g, 11);
+        if (!wait_all(bars_u + 8 * (V_FULL + (g & 1)), (g >> 1) & 1)) return false;
+        if (tr.first && !wait_all(bars_u + 8 * (O_EMPTY + tr.ob), ((tr.item_no >> 1) & 1) ^ 1)) return false;
         tc_fence_after();
-        const uint32_t pbuf = base + OFF_P, vbuf = base + OFF_V + (g & 1) * kTileBytes;
-        for (int ks = 0; ks < tr.npg; ++ks) {
-          const uint64_t a = smem_desc(pbuf + (ks >> 2) * kHalf + (ks & 3) * 32, 16, 1024);
-          const uint64_t b = smem_desc(vbuf + ks * 4096, 1024, 2048);   // 16 keys = one page per k-step
-          tc_mma(tmem + COL_O + tr.ob * 128, a, b, idesc_pv, (!tr.first || ks > 0) ? 1u : 0u);
+        const uint32_t pbuf = base_u + OFF_P, vbuf = base_u + OFF_V + (g & 1) * kTileBytes;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          if (ks < tr.npg) {
+            const uint64_t a = smem_desc(pbuf + (ks >> 2) * kHalf + (ks & 3) * 32, 16, 1024);
+            const uint64_t b = smem_desc(vbuf + ks * 4096, 1024, 2048);   // 16 keys = one page per k-step
+            tc_mma_lane0(tmem_u + COL_O + tr.ob * 128, a, b, idesc_pv, (!tr.first || ks > 0) ? 1u : 0u);
+          }
         }
-        ASPD_STAMP(c, g, 12);
-        tc_commit(bars + 8 * P_EMPTY);
-        tc_commit(bars + 8 * (V_EMPTY + (g & 1)));
-        if (tr.last) tc_commit(bars + 8 * (O_FULL + tr.ob));
+        if (lane == 0) ASPD_STAMP(c, g, 12);
+        tc_commit_lane0(bars_u + 8 * P_EMPTY);
+        tc_commit_lane0(bars_u + 8 * (V_EMPTY + (g & 1)));
+        if (tr.last) tc_commit_lane0(bars_u + 8 * (O_FULL + tr.ob));
         return true;
       };
       int g = 0, item_no = 0;
       bool ok = true, have_prev = false;
       TileRef prev = {0, 0, 0, 0, 0, 0};
-      for (int idx = item_begin; idx < item_end && ok; ++idx, ++item_no) {
-        const int n_pages = get_item(c, misc, idx, item_begin).n_pages, n_tiles = (n_pages + 7) >> 3;
+      const int ib = __shfl_sync(full_mask, item_begin, 0), ie = __shfl_sync(full_mask, item_end, 0);
+      for (int idx = ib; idx < ie && ok; ++idx, ++item_no) {
+        const int n_pages = __shfl_sync(full_mask, get_item(c, misc, idx, ib).n_pages, 0), n_tiles = (n_pages + 7) >> 3;
         for (int t = 0; t < n_tiles && ok; ++t, ++g) {
-          const TileRef cur = {min(8, n_pages - t * 8), t == 0, t == n_tiles - 1, item_no & 1, item_no & 1, item_no};
+          const TileRef cur = {min(8, n_pages - t * 8), t == 0, t == n_tiles - 1, WIDE ? 0 : item_no & 1, item_no & 1, item_no};
           ok = issue_s(cur, g);
           if (ok && have_prev) ok = issue_pv(prev, g - 1);
           prev = cur;
@@ -657,16 +821,19 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     mbar_arrive(bars + 8 * A_DONE);
     if (item_begin < item_end) {                   // the first query tile, while the first K/V tiles are in flight
       prep_q(c, get_item(c, misc, item_begin, item_begin), base + OFF_Q, et);
+      if constexpr (WIDE) prep_q(c, get_item(c, misc, item_begin, item_begin), base + OFF_Q, et, 512);
       fence_async_smem();
       mbar_arrive(bars + 8 * Q_FULL);
     }
     for (int idx = item_begin; idx < item_end; ++idx, ++item_no) {
       const DeviceItem it = get_item(c, misc, idx, item_begin);
-      const int ob = item_no & 1, M = it.n_q_tok * G, R = M <= 32 ? 32 : 64, KS = 128 / R;
-      if (idx + 1 < item_end) {                    // the next item's query tile, into the other buffer
-        const int qn = (item_no + 1) & 1;
-        dead |= !mbar_wait(bars + 8 * (Q_EMPTY + qn), (((item_no + 1) >> 1) & 1) ^ 1, ab);
+      const int ob = item_no & 1, M = it.n_q_tok * G, R = M <= 32 ? 32 : (M <= 64 ? 64 : 128), KS = 128 / R;
+      if (idx + 1 < item_end) {                    // the next item's query tile: into the other buffer, or (wide
+        const int qn = WIDE ? 0 : (item_no + 1) & 1;   // kernel) into the only one once this item's last S is issued
+        const int fills = WIDE ? item_no + 1 : (item_no + 1) >> 1;
+        dead |= !mbar_wait(bars + 8 * (Q_EMPTY + qn), (fills & 1) ^ 1, ab);
         prep_q(c, get_item(c, misc, idx + 1, item_begin), base + OFF_Q + qn * kTileBytes, et);
+        if constexpr (WIDE) prep_q(c, get_item(c, misc, idx + 1, item_begin), base + OFF_Q + qn * kTileBytes, et, 512);
         fence_async_smem();
         mbar_arrive(bars + 8 * (Q_FULL + qn));
       }
@@ -681,7 +848,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
           rec = (size_t)(c.pd.part_base[tok * c.n_kv_heads + it.kv_head] + it.part_slot) * G + r % G;
           float lt = 0.f;
           for (int jj = 0; jj < KS; ++jj) lt += misc->fin_l[ob][jj * R + r] + misc->fin_l[ob][128 + jj * R + r];
-          if (!dead) c.pd.ws_ml[rec] = make_float2(misc->fin_m[ob][r], lt);
+          const float mr = R == 128 ? reinterpret_cast<const float*>(misc + 1)[ob * 128 + r] : misc->fin_m[ob][r];
+          if (!dead) c.pd.ws_ml[rec] = make_float2(mr, lt);
         }
         const uint32_t o_addr = tmem + ((uint32_t)(ew * 32) << 16) + COL_O + ob * 128;
 #pragma unroll 1
@@ -749,7 +917,8 @@ static int launch_tc(const aspd_plan* p, const void* q, const void* k_new, const
   const aspd_shape_t& sh = p->shape;
   static bool configured = false;
   if (!configured) {
-    if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
+    if (cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
       return ASPD_ERR_CUDA;
     configured = true;
   }
@@ -771,7 +940,9 @@ static int launch_tc(const aspd_plan* p, const void* q, const void* k_new, const
   c.n_kv_heads = sh.n_kv_heads;
   c.scale_log2 = sh.sm_scale * kLog2e;
   c.early_fetch = p->stable_cache;
-  return launch_pdl(kPdlAttn, attn_tc_kernel, dim3(p->n_ctas), dim3(kThreads), kSmemBytes, s, c) == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
+  const cudaError_t e = p->wide ? launch_pdl(kPdlAttn, attn_tc_kernel<true>, dim3(p->n_ctas), dim3(kThreads), kSmemBytes, s, c)
+                                : launch_pdl(kPdlAttn, attn_tc_kernel<false>, dim3(p->n_ctas), dim3(kThreads), kSmemBytes, s, c);
+  return e == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
 }
 
 int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, cudaStream_t s) {

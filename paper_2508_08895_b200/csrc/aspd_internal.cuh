@@ -12,6 +12,7 @@
 namespace aspd {
 
 constexpr int kMaxRowsPerItem = 64;   // query rows (tokens x group heads) one work item carries
+constexpr int kMaxRowsWide = 128;     // ... in a plan that deals whole streams to the tensor-core kernel's CTAs
 constexpr int kCausalAll = 1 << 29;   // prefix end of a token that sees its whole key stream
 
 // ---------------------------------------------------------------------------------------
@@ -78,6 +79,8 @@ struct aspd_plan {
   int n_row_blocks;
   int fuse_append;             // few enough new rows per CTA for the attention pass to write them itself
   int stable_cache;            // producers may fetch pages without new rows before the dependency wait
+  int dealt;                   // whole streams dealt to the CTAs in turn (many more streams than CTAs)
+  int wide;                    // dealt plan of the tensor-core kernel: row blocks of up to kMaxRowsWide rows
   int64_t n_pool_pages;
   int64_t kv_tokens_read;
   int64_t algorithmic_bytes;

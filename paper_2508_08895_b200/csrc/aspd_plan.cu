@@ -251,12 +251,18 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   // (physical page, valid rows); the padding rows of partly filled pages are masked by the
   // kernels.  A new token sees stream keys [0, pe) (the prefix) and [lo, hi) (its own branch up
   // to itself); a serial token sees the whole stream.
+  // With block_tok > 0 (plans that deal whole streams) every run of block_tok query tokens of a
+  // request gets a sequence of its own: the prefix and, of the branches, only the pages that one
+  // of the run's tokens can see.
   const int max_tok = std::max(1, kMaxRowsPerItem / G);
+  struct Block { int request, tok0, n_tok, visit0, n_pages; };
   std::vector<int2> visit;
-  std::vector<int> visit0(n_req + 1, 0), req_tok0(n_req + 1, 0);
+  std::vector<Block> blocks;
   std::vector<int4> tok_vis(n_new);
   int64_t kv_tokens = 0;
-  {
+  auto build_visit = [&](int block_tok) {
+    visit.clear(); blocks.clear();
+    int64_t kv_count = 0;
     int t = 0;
     // new_key0 / new_tok0: the keys [new_key0, len) of the region are this step's new tokens
     // new_tok0, new_tok0 + 1, ...; a page entry carries (valid rows | new rows << 8 | first new
@@ -269,43 +275,75 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
         if (n_newrows > 0) y |= (n_newrows << 8) | ((new_tok0 + first_new - new_key0) << 13);
         visit.push_back(make_int2(page_ids[q.page_begin + (slot0 + s0) / ps], y));
       }
-      kv_tokens += len;
+    };
+    auto push_shared = [&](const aspd_request_t& q) {            // prefix and regions of earlier stages: seen by every branch
+      push_region(q, 0, q.prefix_len, q.prefix_len, 0);
+      for (int b = 0; b < q.n_branches; ++b) {
+        const aspd_branch_t& x = br[q.branch_begin + b];
+        if (x.q_len == ASPD_Q_SHARED) push_region(q, x.kv_off, x.kv_len, x.kv_len, 0);
+      }
     };
     for (int r = 0; r < n_req; ++r) {
       const aspd_request_t& q = req[r];
-      req_tok0[r] = t;
-      visit0[r] = (int)visit.size();
+      const int t_req = t, v0 = (int)visit.size();
       if (mode == ASPD_MODE_BRANCH) {
         int nq = 0;
-        for (int b = 0; b < q.n_branches; ++b) nq += std::max(0, br[q.branch_begin + b].q_len);
-        if (nq > 0) {
-          push_region(q, 0, q.prefix_len, q.prefix_len, 0);
-          for (int b = 0; b < q.n_branches; ++b) {             // regions of earlier stages: seen by every branch
-            const aspd_branch_t& x = br[q.branch_begin + b];
-            if (x.q_len == ASPD_Q_SHARED) push_region(q, x.kv_off, x.kv_len, x.kv_len, 0);
-          }
-          const int pe = ((int)visit.size() - visit0[r]) * ps;
+        int64_t kv_req = q.prefix_len;                         // keys of this request that the step reads
+        for (int b = 0; b < q.n_branches; ++b) {
+          const aspd_branch_t& x = br[q.branch_begin + b];
+          nq += std::max(0, x.q_len);
+          if (x.q_len != 0) kv_req += x.kv_len;
+        }
+        if (nq == 0) continue;
+        kv_count += kv_req;
+        if (block_tok == 0) {
+          push_shared(q);
+          const int pe = ((int)visit.size() - v0) * ps;
           for (int b = 0; b < q.n_branches; ++b) {
             const aspd_branch_t& x = br[q.branch_begin + b];
             if (x.q_len <= 0) continue;
-            const int lo = ((int)visit.size() - visit0[r]) * ps;
+            const int lo = ((int)visit.size() - v0) * ps;
             push_region(q, x.kv_off, x.kv_len, x.kv_len - x.q_len, t);
             for (int i = 0; i < x.q_len; ++i) tok_vis[t++] = make_int4(pe, lo, lo + x.kv_len - x.q_len + i + 1, 0);
           }
+          blocks.push_back({r, t_req, nq, v0, (int)visit.size() - v0});
+        } else {
+          for (int blk0 = 0; blk0 < nq; blk0 += block_tok) {
+            const int blk1 = std::min(nq, blk0 + block_tok), bv0 = (int)visit.size();
+            push_shared(q);
+            const int pe = ((int)visit.size() - bv0) * ps;
+            int off = 0;                                       // index, among the request's new tokens, of the branch's first
+            for (int b = 0; b < q.n_branches; ++b) {
+              const aspd_branch_t& x = br[q.branch_begin + b];
+              if (x.q_len <= 0) continue;
+              const int a = std::max(blk0, off), e = std::min(blk1, off + x.q_len);
+              if (a < e) {
+                const int lo = ((int)visit.size() - bv0) * ps, prior = x.kv_len - x.q_len;
+                push_region(q, x.kv_off, prior + (e - off), prior, t_req + off);   // up to the run's last token of this branch
+                for (int i = a - off; i < e - off; ++i) tok_vis[t_req + off + i] = make_int4(pe, lo, lo + prior + i + 1, 0);
+              }
+              off += x.q_len;
+            }
+            blocks.push_back({r, t_req + blk0, blk1 - blk0, bv0, (int)visit.size() - bv0});
+          }
+          t += nq;
         }
       } else {
         push_region(q, 0, q.prefix_len, q.prefix_len, 0);
+        kv_count += q.prefix_len + q.tail_len;
         for (int b = 0; b < q.n_branches; ++b) {
           const aspd_branch_t& x = br[q.branch_begin + b];
           push_region(q, x.kv_off, x.kv_len, x.kv_len, 0);
+          kv_count += x.kv_len;
         }
         push_region(q, q.tail_off, q.tail_len, q.tail_len - 1, t);
         tok_vis[t++] = make_int4(kCausalAll, 0, 0, 0);
+        blocks.push_back({r, t_req, 1, v0, (int)visit.size() - v0});
       }
     }
-    req_tok0[n_req] = t;
-    visit0[n_req] = (int)visit.size();
-  }
+    kv_tokens = kv_count;
+  };
+  build_visit(0);
 
   // ---- work items: a contiguous, equal share of all pages for every CTA -----------------
   // Streams are walked in the order (request, row block, KV head); the concatenation of all
@@ -314,24 +352,66 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   std::vector<int2> row_blocks;
   std::vector<Stream> streams;
   long total_pages = 0;
-  for (int r = 0; r < n_req; ++r) {
-    const int nt = req_tok0[r + 1] - req_tok0[r], np = visit0[r + 1] - visit0[r];
-    if (nt == 0 || np == 0) continue;
-    for (int i0 = 0; i0 < nt; i0 += max_tok) {
-      row_blocks.push_back(make_int2(req_tok0[r] + i0, std::min(max_tok, nt - i0)));
-      for (int h = 0; h < Hkv; ++h) {
-        streams.push_back({r, req_tok0[r] + i0, std::min(max_tok, nt - i0), h, visit0[r], np, (int)row_blocks.size() - 1});
-        total_pages += np;
+  auto build_streams = [&](int tok_per_block) {
+    row_blocks.clear(); streams.clear(); total_pages = 0;
+    for (const Block& bk : blocks) {
+      if (bk.n_tok == 0 || bk.n_pages == 0) continue;
+      for (int i0 = 0; i0 < bk.n_tok; i0 += tok_per_block) {
+        row_blocks.push_back(make_int2(bk.tok0 + i0, std::min(tok_per_block, bk.n_tok - i0)));
+        for (int h = 0; h < Hkv; ++h) {
+          streams.push_back({bk.request, bk.tok0 + i0, std::min(tok_per_block, bk.n_tok - i0), h, bk.visit0, bk.n_pages,
+                             (int)row_blocks.size() - 1});
+          total_pages += bk.n_pages;
+        }
       }
     }
+  };
+  build_streams(max_tok);
+  auto ctas_for = [&](long pages) {
+    const int want = tune.n_ctas > 0 ? tune.n_ctas : p->sm_count;
+    return (int)std::max(1L, std::min((long)want, (pages + 3) / 4));     // do not cut finer than 64 keys per CTA
+  };
+  // With many more streams than CTAs (a step with many query tokens per branch: masked prefill,
+  // teacher forcing) nothing is cut: every stream is one item, and the streams are dealt to the
+  // CTAs in turn, longest requests first, so that at any moment all CTAs read the K/V pages of the
+  // same one or two requests (which then stay in L2) and every CTA gets one stream of each round.
+  // Every row block then gets a page sequence of its own, without the branch pages none of its
+  // tokens sees, and the tensor-core kernel takes row blocks of up to 128 rows (its wide variant).
+  bool deal_streams = mode == ASPD_MODE_BRANCH && tune.chunk_tokens == 0 && (long)streams.size() >= 4L * ctas_for(total_pages);
+  p->wide = 0;
+  if (deal_streams) {
+    p->wide = (kernel == ASPD_KERNEL_MMA && kMaxRowsWide / G > max_tok) ? 1 : 0;
+    const int tok_per_block = p->wide ? kMaxRowsWide / G : max_tok;
+    build_visit(tok_per_block);
+    build_streams(tok_per_block);
   }
-  const int min_pages = 4;                       // do not cut finer than 64 keys per CTA
-  int n_ctas = tune.n_ctas > 0 ? tune.n_ctas : p->sm_count;
-  n_ctas = (int)std::max(1L, std::min((long)n_ctas, (total_pages + min_pages - 1) / min_pages));
+  const int n_ctas = ctas_for(total_pages);
   const int chunk_pages = tune.chunk_tokens > 0 ? tune.chunk_tokens / ps : (1 << 28);
   p->chunk_tokens = tune.chunk_tokens; p->n_ctas = n_ctas;
   std::vector<int32_t> n_parts((size_t)n_new * Hkv, 0), part_base((size_t)n_new * Hkv + 1, 0), cta_item0(n_ctas + 1, 0);
-  {
+  p->dealt = deal_streams ? 1 : 0;
+  if (deal_streams) {
+    std::vector<int> order(streams.size());
+    for (size_t i = 0; i < order.size(); ++i) order[i] = (int)i;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return streams[a].n_pages > streams[b].n_pages; });
+    std::vector<std::vector<int>> mine(n_ctas);
+    for (size_t i = 0; i < order.size(); ++i) {
+      const int round = (int)(i / n_ctas), k = (int)(i % n_ctas);
+      mine[(round & 1) ? n_ctas - 1 - k : k].push_back(order[i]);       // back and forth: evens out the rounds
+    }
+    for (int c = 0; c < n_ctas; ++c) {
+      cta_item0[c] = (int)p->items.size();
+      for (int si : mine[c]) {
+        const Stream& st = streams[si];
+        DeviceItem it;
+        it.q_tok0 = st.tok0; it.n_q_tok = st.n_tok; it.kv_head = st.head; it.page0 = st.page0; it.n_pages = st.n_pages;
+        it.key0 = 0; it.part_slot = 0; it.request = st.request; it.row_block = st.row_block; it.reserved = 0;
+        p->items.push_back(it);
+        for (int i = 0; i < st.n_tok; ++i) n_parts[(size_t)(st.tok0 + i) * Hkv + st.head] = 1;
+      }
+    }
+    cta_item0[n_ctas] = (int)p->items.size();
+  } else {
     // Every CTA gets the same cost, cost = pages + kItemCost per item it starts: an item boundary
     // (new query tile, ragged last tile, epilogue) costs about as much as streaming a dozen pages,
     // so CTAs that end up with several short items get fewer pages.

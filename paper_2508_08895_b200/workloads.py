@@ -390,10 +390,19 @@ def config_serving_mix(seed: int = SEED_BASE + 4, theta: float = 1.0e6, n_req: i
                                   [[1] * len(p) for p in prior])
 
 
+def config_masked_prefill(seed: int = SEED_BASE + 5, theta: float = 1.0e6, n_req: int = 32) -> Workload:
+    """The serving mix's requests in the teacher-forcing layout: every branch's tokens (its 1-256
+    earlier ones and the new one) are query tokens of ONE step over the request's cached prefix."""
+    prefix, prior = serving_mix_lengths(seed, n_req)
+    return build_segment_workload("masked-prefill", seed, 28, 4, 128, "bf16", theta, prefix, [[0] * len(p) for p in prior],
+                                  [[x + 1 for x in p] for p in prior])
+
+
 CONFIGS = {
     "tiny-f32": config_tiny,
     "qwen7b-layer": config_qwen7b_layer,
     "branch-open": config_branch_open,
     "long-rag": config_long_rag,
     "serving-mix": config_serving_mix,
+    "masked-prefill": config_masked_prefill,
 }

@@ -81,54 +81,101 @@ def _shape(wl):
     return B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
 
 
+def _check_cover(wl, ph, plan, chunk=0, dealt=False):
+    """The plan's work items, expanded through its stream-page list and the per-token visible
+    ranges to (token, KV head, logical slot) triples, are exactly the oracle's visible sets."""
+    n_slots = int(ph.desc["n_pages"].max()) * wl.page_size
+    vis = oracle.visible_slots(ph.desc, ph.mode, n_slots)
+    _, _, treq = oracle.new_tokens(ph.desc, ph.mode)
+    page_ids, n_valid = plan.stream_pages()
+    pe, lo, hi = plan.token_ranges()
+    # physical page -> (request, logical page)
+    where = {}
+    for r in range(len(ph.desc["prefix_len"])):
+        pb = int(ph.desc["page_begin"][r])
+        for lp in range(int(ph.desc["n_pages"][r])):
+            where[int(ph.desc["page_ids"][pb + lp])] = (r, lp)
+    count = np.zeros((plan.n_new, wl.Hkv, n_slots), dtype=np.int32)
+    slots_seen = {}
+    ps = wl.page_size
+    for it in plan.items():
+        assert it["n_q_tok"] * wl.G <= (128 if dealt else 64) and it["n_pages"] >= 1 and it["key0"] % ps == 0
+        if chunk:
+            assert it["n_pages"] * ps <= chunk
+        for i in range(int(it["n_q_tok"])):
+            tok = int(it["q_tok0"]) + i
+            assert treq[tok] == it["request"]
+            for pg in range(int(it["n_pages"])):
+                e = int(it["page0"]) + pg
+                r, lp = where[int(page_ids[e])]
+                assert r == it["request"]
+                for row in range(int(n_valid[e])):
+                    kg = int(it["key0"]) + pg * ps + row
+                    if kg < pe[tok] or lo[tok] <= kg < hi[tok]:
+                        count[tok, int(it["kv_head"]), lp * ps + row] += 1
+            slots_seen.setdefault((tok, int(it["kv_head"])), []).append(int(it["part_slot"]))
+    for h in range(wl.Hkv):
+        np.testing.assert_array_equal(count[:, h, :], vis.astype(np.int32))
+    # partial slots of a (token, head) are 0 .. n-1, each used once
+    for key, sl in slots_seen.items():
+        assert sorted(sl) == list(range(len(sl)))
+    assert plan.info.n_partials == sum(len(v) for v in slots_seen.values())
+    # every listed page has 1..page_size valid rows
+    assert ((n_valid >= 1) & (n_valid <= ps)).all()
+    if not dealt:       # pages read = pages of the streams
+        assert plan.info.kv_tokens_read == int(n_valid.sum())
+    return slots_seen
+
+
 @pytest.mark.parametrize("chunk,n_ctas", [(0, 0), (16, 0), (48, 5), (4096, 1), (0, 1000)])
 def test_work_list_covers_every_visible_key_exactly_once(chunk, n_ctas):
-    """Integers only: the work items of a plan, expanded through its stream-page list and the
-    per-token visible ranges to (token, KV head, logical slot) triples, are exactly the oracle's
-    visible sets, each key once."""
+    """Integers only, each visible key once, for every phase of the small workloads."""
     for wl in small_workloads():
         for ph in wl.phases:
             plan = B.Plan(_shape(wl), ph.desc, wl.n_pool_pages, ph.mode, chunk_tokens=chunk, n_ctas=n_ctas, host_only=True)
-            n_slots = int(ph.desc["n_pages"].max()) * wl.page_size
-            vis = oracle.visible_slots(ph.desc, ph.mode, n_slots)
-            _, _, treq = oracle.new_tokens(ph.desc, ph.mode)
-            page_ids, n_valid = plan.stream_pages()
-            pe, lo, hi = plan.token_ranges()
-            # physical page -> (request, logical page)
-            where = {}
-            for r in range(len(ph.desc["prefix_len"])):
-                pb = int(ph.desc["page_begin"][r])
-                for lp in range(int(ph.desc["n_pages"][r])):
-                    where[int(ph.desc["page_ids"][pb + lp])] = (r, lp)
-            count = np.zeros((plan.n_new, wl.Hkv, n_slots), dtype=np.int32)
-            slots_seen = {}
-            ps = wl.page_size
-            for it in plan.items():
-                assert it["n_q_tok"] * wl.G <= 64 and it["n_pages"] >= 1 and it["key0"] % ps == 0
-                if chunk:
-                    assert it["n_pages"] * ps <= chunk
-                for i in range(int(it["n_q_tok"])):
-                    tok = int(it["q_tok0"]) + i
-                    assert treq[tok] == it["request"]
-                    for pg in range(int(it["n_pages"])):
-                        e = int(it["page0"]) + pg
-                        r, lp = where[int(page_ids[e])]
-                        assert r == it["request"]
-                        for row in range(int(n_valid[e])):
-                            kg = int(it["key0"]) + pg * ps + row
-                            if kg < pe[tok] or lo[tok] <= kg < hi[tok]:
-                                count[tok, int(it["kv_head"]), lp * ps + row] += 1
-                    slots_seen.setdefault((tok, int(it["kv_head"])), []).append(int(it["part_slot"]))
-            for h in range(wl.Hkv):
-                np.testing.assert_array_equal(count[:, h, :], vis.astype(np.int32))
-            # partial slots of a (token, head) are 0 .. n-1, each used once
-            for key, sl in slots_seen.items():
-                assert sorted(sl) == list(range(len(sl)))
-            assert plan.info.n_partials == sum(len(v) for v in slots_seen.values())
-            # pages read = pages of the streams, every one with 1..page_size valid rows
-            assert ((n_valid >= 1) & (n_valid <= ps)).all()
-            assert plan.info.kv_tokens_read == int(n_valid.sum())
+            _check_cover(wl, ph, plan, chunk=chunk)
             plan.destroy()
+
+
+@pytest.mark.parametrize("kernel", [B.KERNEL_MMA, B.KERNEL_GENERIC])
+def test_dealt_plan_of_a_step_with_many_query_tokens(kernel):
+    """Many more streams than CTAs: whole streams are dealt out, one record per (token, head);
+    each row block lists the prefix and only the branch pages its tokens see (up to 128 rows
+    for the tensor-core kernel), and the visible sets are still exactly the oracle's."""
+    wl = W.build_segment_workload("deal", 31, 28, 4, 128, "bf16", 1e6, [70, 9, 33], [[0, 17, 5, 2], [3], [0, 0]],
+                                  [[40, 25, 31, 1], [21], [2, 50]], serial_steps=0)
+    ph = wl.phases[-1]
+    plan = B.Plan(_shape(wl), ph.desc, wl.n_pool_pages, ph.mode, kernel=kernel, n_ctas=6, host_only=True)
+    items = plan.items()
+    assert int(items["n_q_tok"].max()) == (18 if kernel == B.KERNEL_MMA else 9)
+    assert (items["part_slot"] == 0).all() and (items["key0"] == 0).all()
+    seen = _check_cover(wl, ph, plan, dealt=True)
+    assert all(len(v) == 1 for v in seen.values())
+    first = plan.cta_ranges()
+    per_cta = np.diff(first)
+    assert per_cta.max() - per_cta.min() <= 1 and per_cta.sum() == len(items)
+    # no row block lists a page of a branch that none of its tokens belongs to
+    page_ids, n_valid = plan.stream_pages()
+    pe, _, _ = plan.token_ranges()
+    _, slot, treq = oracle.new_tokens(ph.desc, ph.mode)
+    d = ph.desc
+    def branch_of(r, s_):
+        for b in range(int(d["branch_begin"][r]), int(d["branch_begin"][r]) + int(d["n_branches"][r])):
+            if int(d["br_kv_off"][b]) <= s_ < int(d["br_kv_off"][b]) + int(d["br_kv_len"][b]):
+                return b
+        return -1
+    logical = {}
+    for r in range(len(d["prefix_len"])):
+        for lp in range(int(d["n_pages"][r])):
+            logical[int(d["page_ids"][int(d["page_begin"][r]) + lp])] = lp
+    for it in items:
+        toks = range(int(it["q_tok0"]), int(it["q_tok0"]) + int(it["n_q_tok"]))
+        own = {branch_of(int(it["request"]), int(slot[t])) for t in toks}
+        for pg in range(int(it["n_pages"])):
+            if pg * wl.page_size >= pe[toks[0]]:
+                e = int(it["page0"]) + pg
+                assert branch_of(int(it["request"]), logical[int(page_ids[e])] * wl.page_size) in own
+    plan.destroy()
 
 
 def test_streams_are_cut_into_equal_shares():

@@ -394,6 +394,35 @@ def test_masked_prefill_of_a_parallel_segment(kernel):
                                   [[100, 60, 31], [49]], serial_steps=1)
     run, ref = compare_workload(wl, kernel=kernel)
     assert run.outputs[0].shape[0] == 240
+    # with few CTAs the plan has many more streams than CTAs and deals whole streams instead of
+    # cutting; the tensor-core kernel then runs its wide variant (row blocks of up to 18 tokens)
+    compare_workload(wl, kernel=kernel, n_ctas=8)
+
+
+def test_wide_row_blocks_mixed_sizes_and_raised_maxima():
+    """The wide variant of the tensor-core kernel on a dealt plan whose row blocks have 1 to 18
+    tokens (7 to 126 rows: all three softmax layouts in one launch, tiles with padding rows,
+    requests whose only visible keys are their own), at the default scale and with logits x 4
+    (the reference maximum of a row is raised many times along its key stream; bounds derived as
+    for the peaked decode variant)."""
+    E = engine()
+    wl = W.build_segment_workload("wide", 37, 28, 4, 128, "bf16", 1e6, [700, 33, 0, 129], [[0, 40, 3], [5], [0, 0], [200]],
+                                  [[130, 9, 4], [1], [20, 3], [57]], serial_steps=1)
+    shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
+    ph = [x for x in wl.phases if x.mode == W.MODE_BRANCH and x.q is not None][-1]
+    plan = B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode, n_ctas=5, host_only=True)
+    ntok = plan.items()["n_q_tok"]
+    assert ntok.max() == 18 and ntok.min() <= 4 and ((ntok > 4) & (ntok <= 9)).any()
+    plan.destroy()
+    compare_workload(wl, n_ctas=5)
+    compare_workload(wl, n_ctas=5, fused=True)
+    wl.sm_scale *= 4.0
+    ref = oracle_run(wl)
+    run = E.run_workload(wl, n_ctas=5)
+    g, r = run.outputs[0].astype(np.float64), ref.outputs[0]
+    err = np.abs(g - r)
+    assert err.max() <= 6e-2 and err.mean() <= 4e-3
+    assert np.linalg.norm(g - r) / np.linalg.norm(r) <= 1e-2
 
 
 def test_rerotation_moves_cached_keys_to_new_positions():
