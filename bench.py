@@ -441,6 +441,7 @@ def run_ours(args):
                        "l2": "footprint %.1f GB of distinct K/V pools per step, far above L2" % (alg * L / 1e9),
                        "layers_agree": bool(same), "cuda_graph": not args.no_graph, "stable_cache": not args.no_stable_cache,
                        "calls_per_layer": ("aspd_branch_step (append fused into the attention pass) -> combine" if info.fused_append
+                                           else "aspd_branch_step (append kernel -> attention pass writing the output)" if info.direct_output
                                            else "aspd_branch_step (append kernel -> attention pass -> combine)") if fused
                        else "aspd_kv_append -> aspd_branch_attn"},
             "hbm_gbs": alg * L * args.steps / (ms * 1e-3) / 1e9,
@@ -454,7 +455,7 @@ def run_ours(args):
             "e2e": {"value": total_new * L * e_steps / (e2e_ms * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": int(L * (n_new * es * wl.d * (wl.Hq + 2 * wl.Hkv) + 4 * n_new)),
                     "d2h_bytes_per_step": int(L * n_new * es * wl.d * wl.Hq), "ms_per_step": e2e_ms / e_steps},
-            "gpu_launches": (2 if fused and info.fused_append else 3) * L * args.steps,
+            "gpu_launches": (2 if (fused and info.fused_append) or info.direct_output else 3) * L * args.steps,
             "clocks": clocks,
         }
         if tensor is not None:

@@ -135,6 +135,9 @@ typedef struct {
   int32_t n_ctas;           /* CTAs of the persistent grid = shares the streams are cut into */
   int32_t fused_append;     /* 1: aspd_branch_step / aspd_serial_step write the new rows inside the
                                attention pass; 0: they run the append kernel first               */
+  int32_t direct_output;    /* 1: one item per (token, KV head) and the attention kernel writes the
+                               output itself (no records, no combine launch)                     */
+  int32_t max_rows_per_item;/* query rows (tokens x group heads) an item may carry: 64 or 128       */
   int64_t workspace_bytes;  /* device memory the plan holds                                 */
   int64_t kv_tokens_read;   /* cached tokens the step must read (each once)                 */
   int64_t algorithmic_bytes;/* K+V of those tokens + q in + out + appended K/V              */

@@ -231,6 +231,7 @@ struct Ctx {
   int n_items, n_q_heads, n_kv_heads;
   float scale_log2;
   int early_fetch;             // plan promise: pages without new rows are not written by in-flight work
+  __nv_bfloat16* out;          // non-null (plans with one item per (token, KV head)): the epilogue writes O / l here
 };
 
 // Item idx of this CTA (rel = idx - item_begin): from the shared-memory cache when it is there.
@@ -843,7 +844,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
       if (ew < R / 32) {
         const int r = et;                          // row of O held by this thread's TMEM lane
         size_t rec = 0;
-        if (r < M) {
+        if (r < M && c.out == nullptr) {
           const int tok = it.q_tok0 + r / G;
           rec = (size_t)(c.pd.part_base[tok * c.n_kv_heads + it.kv_head] + it.part_slot) * G + r % G;
           float lt = 0.f;
@@ -852,12 +853,28 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
           if (!dead) c.pd.ws_ml[rec] = make_float2(mr, lt);
         }
         const uint32_t o_addr = tmem + ((uint32_t)(ew * 32) << 16) + COL_O + ob * 128;
+        float inv_l = 0.f;                         // direct output: the item is the row's whole key stream
+        __nv_bfloat16* orow = nullptr;
+        if (c.out != nullptr && r < M) {
+          float lt = 0.f;
+          for (int jj = 0; jj < KS; ++jj) lt += misc->fin_l[ob][jj * R + r] + misc->fin_l[ob][128 + jj * R + r];
+          inv_l = lt > 0.f ? 1.f / lt : 0.f;
+          orow = c.out + ((size_t)(it.q_tok0 + r / G) * c.n_q_heads + it.kv_head * G + r % G) * 128;
+        }
 #pragma unroll 1
         for (int q4 = 0; q4 < 4; ++q4) {
           float o[32];
           ASPD_TMEM_LD32(o_addr + q4 * 32, o, 0);
           tmem_wait_ld();
-          if (r < M && !dead) {
+          if (c.out != nullptr) {
+            if (r < M && !dead) {
+              uint4* dst = reinterpret_cast<uint4*>(orow + q4 * 32);
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                dst[i] = make_uint4(pack_bf16(o[8 * i] * inv_l, o[8 * i + 1] * inv_l), pack_bf16(o[8 * i + 2] * inv_l, o[8 * i + 3] * inv_l),
+                                    pack_bf16(o[8 * i + 4] * inv_l, o[8 * i + 5] * inv_l), pack_bf16(o[8 * i + 6] * inv_l, o[8 * i + 7] * inv_l));
+            }
+          } else if (r < M && !dead) {
             float4* dst = reinterpret_cast<float4*>(c.pd.ws_o + rec * 128 + q4 * 32);
 #pragma unroll
             for (int i = 0; i < 8; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
@@ -912,7 +929,7 @@ namespace {
 }  // namespace
 
 static int launch_tc(const aspd_plan* p, const void* q, const void* k_new, const void* v_new, const void* k_pool,
-                     const void* v_pool, cudaStream_t s) {
+                     const void* v_pool, void* out, cudaStream_t s) {
   if (p->n_items == 0) return ASPD_OK;
   const aspd_shape_t& sh = p->shape;
   static bool configured = false;
@@ -940,18 +957,19 @@ static int launch_tc(const aspd_plan* p, const void* q, const void* k_new, const
   c.n_kv_heads = sh.n_kv_heads;
   c.scale_log2 = sh.sm_scale * kLog2e;
   c.early_fetch = p->stable_cache;
+  c.out = p->dealt ? (__nv_bfloat16*)out : nullptr;   // only when every (token, KV head) has a single item
   const cudaError_t e = p->wide ? launch_pdl(kPdlAttn, attn_tc_kernel<true>, dim3(p->n_ctas), dim3(kThreads), kSmemBytes, s, c)
                                 : launch_pdl(kPdlAttn, attn_tc_kernel<false>, dim3(p->n_ctas), dim3(kThreads), kSmemBytes, s, c);
   return e == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
 }
 
-int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, cudaStream_t s) {
-  return launch_tc(p, q, nullptr, nullptr, k_pool, v_pool, s);
+int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, void* out, cudaStream_t s) {
+  return launch_tc(p, q, nullptr, nullptr, k_pool, v_pool, out, s);
 }
 
 int launch_attn_mma_step(const aspd_plan* p, const void* q, const void* k_new, const void* v_new, void* k_pool, void* v_pool,
-                         cudaStream_t s) {
-  return launch_tc(p, q, k_new, v_new, k_pool, v_pool, s);
+                         void* out, cudaStream_t s) {
+  return launch_tc(p, q, k_new, v_new, k_pool, v_pool, out, s);
 }
 
 }  // namespace aspd

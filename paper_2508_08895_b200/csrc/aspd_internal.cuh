@@ -125,12 +125,15 @@ int launch_append(const aspd_plan* p, const void* k_new, const void* v_new, cons
                   void* k_pool, void* v_pool, cudaStream_t s);
 int launch_attn_generic(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool,
                         cudaStream_t s);
-int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool,
+// out: null = (m, l, O) records for the combine kernel; non-null = final output, written by the
+// kernel itself when the plan has one item per (token, KV head) (ignored otherwise)
+int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, void* out,
                     cudaStream_t s);
+inline bool attn_mma_writes_output(const aspd_plan* p) { return p->kernel == ASPD_KERNEL_MMA && p->dealt; }
 int launch_combine(const aspd_plan* p, void* out, cudaStream_t s);
 // attention pass that first writes this step's new K (rotated) and V rows into the pages it reads
 int launch_attn_mma_step(const aspd_plan* p, const void* q, const void* k_new, const void* v_new, void* k_pool,
-                         void* v_pool, cudaStream_t s);
+                         void* v_pool, void* out, cudaStream_t s);
 int launch_rerotate(const aspd_shape_t* shape, void* k_pool, const int32_t* pages, const int32_t* rows, const int32_t* delta,
                     int n, cudaStream_t s);
 int launch_wait_probe(long long limit_cycles, int32_t* status_dev, cudaStream_t s);

@@ -584,7 +584,9 @@ int aspd_plan_info(const aspd_plan_t* p, aspd_plan_info_t* info) {
   if (!p || !info) return ASPD_ERR_INVALID_ARG;
   info->n_new = p->n_new; info->n_items = p->n_items; info->n_partials = p->n_partials;
   info->n_stream_pages = (int32_t)p->visit.size(); info->kernel = p->kernel;
-  info->chunk_tokens = p->chunk_tokens; info->n_ctas = p->n_ctas; info->fused_append = (p->kernel == ASPD_KERNEL_MMA && p->fuse_append) ? 1 : 0; info->workspace_bytes = (int64_t)p->device_bytes;
+  info->chunk_tokens = p->chunk_tokens; info->n_ctas = p->n_ctas; info->fused_append = (p->kernel == ASPD_KERNEL_MMA && p->fuse_append) ? 1 : 0;
+  info->direct_output = attn_mma_writes_output(p) ? 1 : 0; info->max_rows_per_item = p->wide ? kMaxRowsWide : kMaxRowsPerItem;
+  info->workspace_bytes = (int64_t)p->device_bytes;
   info->kv_tokens_read = p->kv_tokens_read; info->algorithmic_bytes = p->algorithmic_bytes;
   return ASPD_OK;
 }
@@ -640,7 +642,7 @@ int aspd_attn_partials(aspd_plan_t* p, const void* q, const void* k_pool, const 
   if (p->n_new == 0) return ASPD_OK;
   if (!q || !k_pool || !v_pool) return ASPD_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
-  return p->kernel == ASPD_KERNEL_MMA ? launch_attn_mma(p, q, k_pool, v_pool, s)
+  return p->kernel == ASPD_KERNEL_MMA ? launch_attn_mma(p, q, k_pool, v_pool, nullptr, s)
                                       : launch_attn_generic(p, q, k_pool, v_pool, s);
 }
 
@@ -656,6 +658,8 @@ static int run_attn(aspd_plan_t* p, int mode, const void* q, const void* k_pool,
   if (!p || p->host_only || p->mode != mode) return ASPD_ERR_INVALID_ARG;
   if (p->n_new == 0) return ASPD_OK;
   if (!q || !k_pool || !v_pool || !out) return ASPD_ERR_INVALID_ARG;
+  // a plan with one item per (token, KV head) needs no records: the kernel normalises and writes the output
+  if (attn_mma_writes_output(p)) return launch_attn_mma(p, q, k_pool, v_pool, out, (cudaStream_t)stream);
   int rc = aspd_attn_partials(p, q, k_pool, v_pool, stream);
   if (rc) return rc;
   return aspd_attn_combine(p, out, stream);
@@ -677,15 +681,15 @@ static int run_step(aspd_plan_t* p, int mode, const void* q, const void* k_new, 
   cudaStream_t s = (cudaStream_t)stream;
   int rc;
   if (p->kernel == ASPD_KERNEL_MMA && p->fuse_append) {
-    rc = launch_attn_mma_step(p, q, k_new, v_new, k_pool, v_pool, s);
+    rc = launch_attn_mma_step(p, q, k_new, v_new, k_pool, v_pool, out, s);
   } else if (p->kernel == ASPD_KERNEL_MMA) {
     rc = launch_append(p, k_new, v_new, p->dev.tok_pos, k_pool, v_pool, s);
-    if (rc == ASPD_OK) rc = launch_attn_mma(p, q, k_pool, v_pool, s);
+    if (rc == ASPD_OK) rc = launch_attn_mma(p, q, k_pool, v_pool, out, s);
   } else {
     rc = launch_append(p, k_new, v_new, p->dev.tok_pos, k_pool, v_pool, s);
     if (rc == ASPD_OK) rc = launch_attn_generic(p, q, k_pool, v_pool, s);
   }
-  if (rc) return rc;
+  if (rc || attn_mma_writes_output(p)) return rc;
   return launch_combine(p, out, s);
 }
 
