@@ -40,6 +40,7 @@ constexpr int kSoftmaxThreads = 256;           // two warps per TMEM lane quadra
 constexpr int W_KPROD = 8, W_MMA = 9, W_VPROD = 11, W_EPI = 12;   // warp roles (0-7 softmax, 10 idle, 12-15 epilogue)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRaise = 8.0f;                 // raise the reference maximum only beyond 2^8
+constexpr float kLower = 32.0f;                // wide variant: lower the initial reference (0) when a row's first keys are below 2^-32
 constexpr long long kWaitCycles = 3000000000LL; // ~1.5 s at 1.9 GHz
 
 constexpr uint32_t kTileBytes = 32768;         // one K, V, Q or P tile: 128 rows x 256 B
@@ -380,7 +381,10 @@ __device__ __forceinline__ bool softmax_item_wide(const Ctx& c, const DeviceItem
   const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
   const bool o_owner = half == 0;
   const int ob = item_no & 1;
-  float m_ref = -INFINITY, l = 0.f;
+  // The reference starts at 0 (exponents of typical logits are within +-2^8 of it, so the first
+  // tile needs no second pass); until the row has seen a key it may also be lowered.
+  float m_ref = 0.f, l = 0.f;
+  bool seen = false;
   bool dead = false;
   for (int t = 0; t < n_tiles; ++t, ++g) {
     const int sb = g & 1;
@@ -426,17 +430,20 @@ __device__ __forceinline__ bool softmax_item_wide(const Ctx& c, const DeviceItem
       tile_sum = (sum0 + sum1) + (sum2 + sum3);
       tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
     };
-    const float base = m_ref == -INFINITY ? 0.f : m_ref;
-    pass(base);
+    pass(m_ref);
     if (tid == 0) ASPD_STAMP(c, g, 1);
     misc->smax[sb][tid] = tmax;
     named_sync(1, kSoftmaxThreads);
     if (tid == 0) ASPD_STAMP(c, g, 2);
     const float row_tmax = fmaxf(misc->smax[sb][r], misc->smax[sb][128 + r]);
-    // raise the reference: on the row's first visible key, or when an exponent passed 2^8
-    const bool upd = m_ref == -INFINITY ? row_tmax > -INFINITY : row_tmax > kRaise;
+    // move the reference: up when an exponent passed 2^8; down only while the row has not seen a
+    // key yet (l and its row of O are still exactly 0, so nothing is rescaled then)
+    const bool raise = row_tmax > kRaise, lower = !seen && row_tmax < -kLower && row_tmax > -INFINITY;
+    const bool upd = raise || lower;
+    seen |= row_tmax > -INFINITY;
     float alpha = 1.f;
-    if (upd) { alpha = m_ref == -INFINITY ? 0.f : ex2(-row_tmax); m_ref = base + row_tmax; }
+    if (raise) alpha = ex2(-row_tmax);
+    if (upd) m_ref += row_tmax;
     l *= alpha;
     const bool any_upd = __any_sync(0xffffffffu, upd);
     if (t > 0 && o_owner && any_upd) {              // the owners of the rows rescale O in TMEM
@@ -454,7 +461,7 @@ __device__ __forceinline__ bool softmax_item_wide(const Ctx& c, const DeviceItem
       }
       tmem_wait_st();
     }
-    if (any_upd) pass(m_ref == -INFINITY ? 0.f : m_ref);   // the whole warp again (TMEM loads are warp-wide)
+    if (any_upd) pass(m_ref);   // the whole warp again (TMEM loads are warp-wide)
     l += tile_sum;
     tc_fence_before();
     mbar_arrive(bars + 8 * (S_EMPTY + sb));
@@ -483,15 +490,19 @@ __device__ __forceinline__ bool softmax_item_wide(const Ctx& c, const DeviceItem
 // Rotate the item's query rows (RoPE at the token's position, cos/sin table from the plan),
 // round to bf16 and store them, replicated KS = 128 / R times, as the 128-byte-swizzled K-major
 // A operand.  Called by the 128 epilogue threads (rank 0..127); all loads of a thread's rows
-// are issued before the first use.
-__device__ __forceinline__ void prep_q(const Ctx& c, const DeviceItem& it, uint32_t qbuf, int rank, int e0 = 0) {
+// are issued before the first use.  Unit e = (row e / 8, 16-byte chunk e % 8 of each span); a
+// call covers units e0 + rank + 128 u, u < 4 (row blocks of 128 rows need two calls).
+struct QUnits {
+  uint32_t lo[4][4], hi[4][4];   // per unit: the rotated chunk of the first and of the second span, bf16 pairs
+};
+__device__ __forceinline__ void prep_q_compute(const Ctx& c, const DeviceItem& it, int rank, int e0, QUnits& qu) {
   const int G = c.n_q_heads / c.n_kv_heads;
-  const int M = it.n_q_tok * G, R = M <= 32 ? 32 : (M <= 64 ? 64 : 128), KS = 128 / R;   // R = 128: second call with e0 = 512
+  const int M = it.n_q_tok * G, R = M <= 32 ? 32 : (M <= 64 ? 64 : 128);
   uint4 a[4], b[4];
   float4 w[4][4];
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
-    const int e = e0 + rank + u * 128, r = e >> 3, ch = e & 7;     // row, 8-element chunk of each span
+    const int e = e0 + rank + u * 128, r = e >> 3, ch = e & 7;
     a[u] = make_uint4(0, 0, 0, 0); b[u] = make_uint4(0, 0, 0, 0);
 #pragma unroll
     for (int i = 0; i < 4; ++i) w[u][i] = make_float4(1.f, 0.f, 1.f, 0.f);
@@ -507,23 +518,36 @@ __device__ __forceinline__ void prep_q(const Ctx& c, const DeviceItem& it, uint3
   }
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
-    const int e = e0 + rank + u * 128, r = e >> 3, ch = e & 7;
-    if (e >= R * 8) break;
     const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&a[u]);
     const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&b[u]);
-    uint32_t lo[4], hi[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const float2 x0 = __bfloat1622float2(a2[i]), x1 = __bfloat1622float2(b2[i]);
-      lo[i] = pack_bf16(x0.x * w[u][i].x - x1.x * w[u][i].y, x0.y * w[u][i].z - x1.y * w[u][i].w);
-      hi[i] = pack_bf16(x1.x * w[u][i].x + x0.x * w[u][i].y, x1.y * w[u][i].z + x0.y * w[u][i].w);
-    }
-    for (int jj = 0; jj < KS; ++jj) {
-      const uint32_t addr = qbuf + (jj * R + r) * 128 + ((ch ^ (r & 7)) << 4);
-      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
-      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr + kHalf), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
+      qu.lo[u][i] = pack_bf16(x0.x * w[u][i].x - x1.x * w[u][i].y, x0.y * w[u][i].z - x1.y * w[u][i].w);
+      qu.hi[u][i] = pack_bf16(x1.x * w[u][i].x + x0.x * w[u][i].y, x1.y * w[u][i].z + x0.y * w[u][i].w);
     }
   }
+}
+__device__ __forceinline__ void prep_q_store(const Ctx& c, const DeviceItem& it, uint32_t qbuf, int rank, int e0, const QUnits& qu) {
+  const int G = c.n_q_heads / c.n_kv_heads;
+  const int M = it.n_q_tok * G, R = M <= 32 ? 32 : (M <= 64 ? 64 : 128), KS = 128 / R;
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const int e = e0 + rank + u * 128, r = e >> 3, ch = e & 7;
+    if (e >= R * 8) break;
+    for (int jj = 0; jj < KS; ++jj) {
+      const uint32_t addr = qbuf + (jj * R + r) * 128 + ((ch ^ (r & 7)) << 4);
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(qu.lo[u][0]), "r"(qu.lo[u][1]), "r"(qu.lo[u][2]),
+                   "r"(qu.lo[u][3]) : "memory");
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr + kHalf), "r"(qu.hi[u][0]), "r"(qu.hi[u][1]), "r"(qu.hi[u][2]),
+                   "r"(qu.hi[u][3]) : "memory");
+    }
+  }
+}
+__device__ __forceinline__ void prep_q(const Ctx& c, const DeviceItem& it, uint32_t qbuf, int rank, int e0 = 0) {
+  QUnits qu;
+  prep_q_compute(c, it, rank, e0, qu);
+  prep_q_store(c, it, qbuf, rank, e0, qu);
 }
 
 // Fused step (aspd_branch_step / aspd_serial_step): the rows this step adds to pages that THIS CTA
@@ -832,9 +856,20 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
       if (idx + 1 < item_end) {                    // the next item's query tile: into the other buffer, or (wide
         const int qn = WIDE ? 0 : (item_no + 1) & 1;   // kernel) into the only one once this item's last S is issued
         const int fills = WIDE ? item_no + 1 : (item_no + 1) >> 1;
-        dead |= !mbar_wait(bars + 8 * (Q_EMPTY + qn), (fills & 1) ^ 1, ab);
-        prep_q(c, get_item(c, misc, idx + 1, item_begin), base + OFF_Q + qn * kTileBytes, et);
-        if constexpr (WIDE) prep_q(c, get_item(c, misc, idx + 1, item_begin), base + OFF_Q + qn * kTileBytes, et, 512);
+        if constexpr (WIDE) {
+          // the only query tile is free once this item's last S has been issued: rotate the next
+          // item's rows into registers first, so that only the stores are left for after the wait
+          const DeviceItem nx = get_item(c, misc, idx + 1, item_begin);
+          QUnits q0, q1;
+          prep_q_compute(c, nx, et, 0, q0);
+          prep_q_compute(c, nx, et, 512, q1);
+          dead |= !mbar_wait(bars + 8 * (Q_EMPTY + qn), (fills & 1) ^ 1, ab);
+          prep_q_store(c, nx, base + OFF_Q, et, 0, q0);
+          prep_q_store(c, nx, base + OFF_Q, et, 512, q1);
+        } else {
+          dead |= !mbar_wait(bars + 8 * (Q_EMPTY + qn), (fills & 1) ^ 1, ab);
+          prep_q(c, get_item(c, misc, idx + 1, item_begin), base + OFF_Q + qn * kTileBytes, et);
+        }
         fence_async_smem();
         mbar_arrive(bars + 8 * (Q_FULL + qn));
       }
@@ -849,7 +884,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
           rec = (size_t)(c.pd.part_base[tok * c.n_kv_heads + it.kv_head] + it.part_slot) * G + r % G;
           float lt = 0.f;
           for (int jj = 0; jj < KS; ++jj) lt += misc->fin_l[ob][jj * R + r] + misc->fin_l[ob][128 + jj * R + r];
-          const float mr = R == 128 ? reinterpret_cast<const float*>(misc + 1)[ob * 128 + r] : misc->fin_m[ob][r];
+          float mr = R == 128 ? reinterpret_cast<const float*>(misc + 1)[ob * 128 + r] : misc->fin_m[ob][r];
+          if (lt == 0.f) mr = -INFINITY;           // no visible key in this item (the wide variant's reference starts at 0)
           if (!dead) c.pd.ws_ml[rec] = make_float2(mr, lt);
         }
         const uint32_t o_addr = tmem + ((uint32_t)(ew * 32) << 16) + COL_O + ob * 128;

@@ -425,6 +425,22 @@ def test_wide_row_blocks_mixed_sizes_and_raised_maxima():
     assert np.linalg.norm(g - r) / np.linalg.norm(r) <= 1e-2
 
 
+def test_wide_row_blocks_with_very_negative_logits():
+    """All logits near -130 in log2 units (keys and queries opposite along the slowest rotary pair,
+    so the rotation hardly changes them): against the wide variant's initial reference of 0 every
+    weight would underflow to 0; the reference has to come down to the row's first keys.  The
+    softmax is then close to uniform and the output the mean of the visible V rows."""
+    wl = W.build_segment_workload("neg", 41, 28, 4, 128, "bf16", 1e6, [130, 20], [[0, 7], [0]], [[40, 22], [30]])
+    for ph in wl.phases:
+        ph.k_new[:] = 0.0
+        ph.k_new[:, :, 63] = 32.0
+        if ph.q is not None:
+            ph.q[:] = 0.0
+            ph.q[:, :, 63] = -32.0
+    run, ref = compare_workload(wl, n_ctas=3)
+    assert np.abs(ref.outputs[0]).max() < 1.0 and run.outputs[0].shape[0] == 92
+
+
 def test_rerotation_moves_cached_keys_to_new_positions():
     """Same-Re without a re-prefill: after a segment, the branch tokens are renumbered
     sequentially by rotating their cached keys by (new - old) positions in place."""
