@@ -25,6 +25,8 @@ _LIB = os.path.join(_HERE, "libaspd_oracle.so")
 
 MODE_BRANCH = 0
 MODE_SERIAL = 1
+MASK_BRANCH_INVISIBLE = 0   # Eq. 2-3
+MASK_SHARED = 1             # the visible mask of the attention-mask ablation
 
 _lib = None
 
@@ -44,7 +46,8 @@ def lib() -> ctypes.CDLL:
         _lib.aspd_oracle_rope.restype = None
         for name in ("aspd_oracle_dense_positions", "aspd_oracle_dense_visible", "aspd_oracle_dense_attn",
                      "aspd_oracle_new_tokens", "aspd_oracle_kv_append", "aspd_oracle_attn", "aspd_oracle_attn_at",
-                     "aspd_oracle_visible_slots", "aspd_oracle_threads"):
+                     "aspd_oracle_visible_slots", "aspd_oracle_threads", "aspd_oracle_dense_visible_shared",
+                     "aspd_oracle_dense_attn_shared", "aspd_oracle_attn_masked", "aspd_oracle_visible_slots_masked"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
 
@@ -91,15 +94,26 @@ def dense_visible(branch, stage, pos=None) -> np.ndarray:
     return vis
 
 
-def dense_attn(q, k, v, branch, stage, theta: float, sm_scale: float) -> np.ndarray:
+def dense_visible_shared(pos) -> np.ndarray:
+    """Visible ("Shared") mask of the ablation: i sees j iff pos[j] < pos[i], or j == i."""
+    pos = _i32(pos)
+    L = len(pos)
+    vis = np.zeros((L, L), dtype=np.uint8)
+    rc = lib().aspd_oracle_dense_visible_shared(L, _p(pos), _p(vis))
+    assert rc == 0
+    return vis
+
+
+def dense_attn(q, k, v, branch, stage, theta: float, sm_scale: float, mask: int = MASK_BRANCH_INVISIBLE) -> np.ndarray:
     """q [L][Hq][d], k/v [L][Hkv][d] raw (un-rotated); returns out [L][Hq][d]."""
     q, k, v = _f64(q), _f64(k), _f64(v)
     branch, stage = _i32(branch), _i32(stage)
     L, Hq, d = q.shape
     Hkv = k.shape[1]
     out = np.empty_like(q)
-    rc = lib().aspd_oracle_dense_attn(L, Hq, Hkv, d, ctypes.c_double(theta), ctypes.c_double(sm_scale),
-                                      _p(q), _p(k), _p(v), _p(branch), _p(stage), _p(out))
+    fn = lib().aspd_oracle_dense_attn_shared if mask == MASK_SHARED else lib().aspd_oracle_dense_attn
+    rc = fn(L, Hq, Hkv, d, ctypes.c_double(theta), ctypes.c_double(sm_scale),
+            _p(q), _p(k), _p(v), _p(branch), _p(stage), _p(out))
     assert rc == 0, rc
     return out
 
@@ -159,15 +173,26 @@ def kv_append(desc, k_new, v_new, pos, req, slot, k_pool, v_pool, theta: float) 
     assert rc == 0
 
 
-def attn(desc, mode: int, q, k_pool, v_pool, theta: float, sm_scale: float, q_pos=None) -> np.ndarray:
+def attn(desc, mode: int, q, k_pool, v_pool, theta: float, sm_scale: float, q_pos=None,
+         mask: int = MASK_BRANCH_INVISIBLE) -> np.ndarray:
     """a4-a7 (mode 0) / a9 (mode 1): out [n_new][Hq][d] for raw queries q [n_new][Hq][d].
-    ``q_pos``: query positions of a position-ID variant (default: Eq. 4)."""
+    ``q_pos``: query positions of a position-ID variant (default: Eq. 4); ``mask``: the
+    branch-invisible mask of Eq. 2-3 or the ablation's visible one."""
     d = _desc(desc)
     q = _f64(q)
     n_new, Hq, hd = q.shape
     assert n_new == n_new_tokens(d, mode)
     Hkv, page_size = k_pool.shape[1], k_pool.shape[2]
     out = np.empty_like(q)
+    if mask != MASK_BRANCH_INVISIBLE:
+        qp = None if q_pos is None else _i32(q_pos)
+        rc = lib().aspd_oracle_attn_masked(len(d["prefix_len"]), mode, Hq, Hkv, hd, page_size, ctypes.c_double(theta),
+                                           ctypes.c_double(sm_scale), _p(d["prefix_len"]), _p(d["n_branches"]),
+                                           _p(d["branch_begin"]), _p(d["page_begin"]), _p(d["tail_off"]), _p(d["tail_len"]),
+                                           _p(d["br_kv_off"]), _p(d["br_kv_len"]), _p(d["br_q_len"]), _p(d["page_ids"]),
+                                           _p(q), None if qp is None else _p(qp), ctypes.c_int(mask), _p(k_pool), _p(v_pool), _p(out))
+        assert rc == 0, rc
+        return out
     if q_pos is not None:
         qp = _i32(q_pos)
         assert len(qp) == n_new
@@ -187,14 +212,14 @@ def attn(desc, mode: int, q, k_pool, v_pool, theta: float, sm_scale: float, q_po
     return out
 
 
-def visible_slots(desc, mode: int, n_slots: int) -> np.ndarray:
+def visible_slots(desc, mode: int, n_slots: int, mask: int = MASK_BRANCH_INVISIBLE) -> np.ndarray:
     """[n_new][n_slots] 0/1: logical slots of its own request that each new token may see."""
     d = _desc(desc)
     n = n_new_tokens(d, mode)
     vis = np.zeros((n, n_slots), dtype=np.uint8)
-    rc = lib().aspd_oracle_visible_slots(len(d["prefix_len"]), mode, n_slots, _p(d["prefix_len"]),
-                                         _p(d["n_branches"]), _p(d["branch_begin"]), _p(d["tail_off"]),
-                                         _p(d["tail_len"]), _p(d["br_kv_off"]), _p(d["br_kv_len"]),
-                                         _p(d["br_q_len"]), _p(vis))
+    rc = lib().aspd_oracle_visible_slots_masked(len(d["prefix_len"]), mode, n_slots, _p(d["prefix_len"]),
+                                                _p(d["n_branches"]), _p(d["branch_begin"]), _p(d["tail_off"]),
+                                                _p(d["tail_len"]), _p(d["br_kv_off"]), _p(d["br_kv_len"]),
+                                                _p(d["br_q_len"]), ctypes.c_int(mask), _p(vis))
     assert rc == n
     return vis

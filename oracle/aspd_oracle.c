@@ -157,18 +157,31 @@ int aspd_oracle_dense_visible(int L, const int* branch, const int* stage,
   return ORACLE_OK;
 }
 
+/* The visible ("Shared") mask of the paper's attention-mask ablation: the visibility function is
+ * 1 for every pair, so all that is left of Eq. 2 is the order of the position IDs -- token i
+ * sees token j iff j's position precedes i's (and itself).  With the shared position IDs a
+ * branch token at offset delta therefore sees the first delta tokens of EVERY branch of its stage:
+ * exactly the tokens that exist when the branches decode in lockstep. */
+int aspd_oracle_dense_visible_shared(int L, const int* pos, uint8_t* vis) {
+  for (int i = 0; i < L; ++i)
+    for (int j = 0; j < L; ++j)
+      vis[(size_t)i * L + j] = (uint8_t)((pos[i] > pos[j] || i == j) ? 1 : 0);
+  return ORACLE_OK;
+}
+
 /* Eq. 1 for every token of the flat list, every query head. */
-int aspd_oracle_dense_attn(int L, int Hq, int Hkv, int d, double theta,
+static int dense_attn_impl(int L, int Hq, int Hkv, int d, double theta,
                            double sm_scale, const double* q, const double* k,
                            const double* v, const int* branch,
-                           const int* stage, double* out) {
+                           const int* stage, int shared_mask, double* out) {
   if (L <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv || d <= 0 || d % 2) return ORACLE_BAD;
   int G = Hq / Hkv;
   int* pos = (int*)malloc(sizeof(int) * L);
   uint8_t* vis = (uint8_t*)malloc((size_t)L * L);
   double* khat = (double*)malloc(sizeof(double) * (size_t)L * Hkv * d);
   aspd_oracle_dense_positions(L, branch, stage, pos);
-  aspd_oracle_dense_visible(L, branch, stage, pos, vis);
+  if (shared_mask) aspd_oracle_dense_visible_shared(L, pos, vis);
+  else aspd_oracle_dense_visible(L, branch, stage, pos, vis);
   for (int j = 0; j < L; ++j)
     for (int h = 0; h < Hkv; ++h)
       aspd_oracle_rope(k + ((size_t)j * Hkv + h) * d, d, (double)pos[j], theta,
@@ -193,6 +206,21 @@ int aspd_oracle_dense_attn(int L, int Hq, int Hkv, int d, double theta,
     }
   free(pos); free(vis); free(khat); free(keys); free(vals); free(logits); free(qhat);
   return ORACLE_OK;
+}
+
+int aspd_oracle_dense_attn(int L, int Hq, int Hkv, int d, double theta,
+                           double sm_scale, const double* q, const double* k,
+                           const double* v, const int* branch,
+                           const int* stage, double* out) {
+  return dense_attn_impl(L, Hq, Hkv, d, theta, sm_scale, q, k, v, branch, stage, 0, out);
+}
+
+/* Eq. 1 under the visible ("Shared") mask of the ablation. */
+int aspd_oracle_dense_attn_shared(int L, int Hq, int Hkv, int d, double theta,
+                                  double sm_scale, const double* q, const double* k,
+                                  const double* v, const int* branch,
+                                  const int* stage, double* out) {
+  return dense_attn_impl(L, Hq, Hkv, d, theta, sm_scale, q, k, v, branch, stage, 1, out);
 }
 
 /* ======================================================================== */
@@ -224,6 +252,8 @@ int aspd_oracle_dense_attn(int L, int Hq, int Hkv, int d, double theta,
  */
 #define MODE_BRANCH 0
 #define MODE_SERIAL 1
+#define MASK_BRANCH_INVISIBLE 0   /* Eq. 2-3 */
+#define MASK_SHARED 1             /* the ablation's visible mask */
 
 /*
  * a1 + a2: position ID (Eq. 4) and logical slot of every new token.
@@ -316,7 +346,7 @@ static int attn_impl(int n_req, int mode, int Hq, int Hkv, int d,
                      const int* tail_off, const int* tail_len,
                      const int* br_kv_off, const int* br_kv_len,
                      const int* br_q_len, const int* page_ids, const double* q,
-                     const int* q_pos_given,
+                     const int* q_pos_given, int mask_mode,
                      const double* k_pool, const double* v_pool, double* out) {
   if (Hq % Hkv || d % 2) return ORACLE_BAD;
   int G = Hq / Hkv;
@@ -387,6 +417,18 @@ static int attn_impl(int n_req, int mode, int Hq, int Hkv, int d,
             vals[m] = cached(v_pool, page_ids, pb, s, h, Hkv, page_size, d);
             ++m;
           }
+          if (mask_mode == MASK_SHARED) {                  /* the other branches of the stage, at smaller offsets */
+            for (int b = 0; b < n_branches[r]; ++b) {
+              int C = branch_begin[r] + b;
+              if (C == B || br_q_len[C] == -1) continue;
+              for (int j = 0; j < br_kv_len[C] && j < t_k[t]; ++j) {
+                int s = br_kv_off[C] + j;
+                keys[m] = cached(k_pool, page_ids, pb, s, h, Hkv, page_size, d);
+                vals[m] = cached(v_pool, page_ids, pb, s, h, Hkv, page_size, d);
+                ++m;
+              }
+            }
+          }
           qpos = t_pos0[t] + t_k[t];
         } else {
           int total = P;
@@ -429,7 +471,7 @@ int aspd_oracle_attn(int n_req, int mode, int Hq, int Hkv, int d,
                      const int* br_q_len, const int* page_ids, const double* q,
                      const double* k_pool, const double* v_pool, double* out) {
   return attn_impl(n_req, mode, Hq, Hkv, d, page_size, theta, sm_scale, prefix_len, n_branches, branch_begin,
-                   page_begin, tail_off, tail_len, br_kv_off, br_kv_len, br_q_len, page_ids, q, 0, k_pool, v_pool, out);
+                   page_begin, tail_off, tail_len, br_kv_off, br_kv_len, br_q_len, page_ids, q, 0, MASK_BRANCH_INVISIBLE, k_pool, v_pool, out);
 }
 
 /*
@@ -449,7 +491,22 @@ int aspd_oracle_attn_at(int n_req, int mode, int Hq, int Hkv, int d,
                         const double* k_pool, const double* v_pool, double* out) {
   if (!q_pos) return ORACLE_BAD;
   return attn_impl(n_req, mode, Hq, Hkv, d, page_size, theta, sm_scale, prefix_len, n_branches, branch_begin,
-                   page_begin, tail_off, tail_len, br_kv_off, br_kv_len, br_q_len, page_ids, q, q_pos, k_pool, v_pool, out);
+                   page_begin, tail_off, tail_len, br_kv_off, br_kv_len, br_q_len, page_ids, q, q_pos, MASK_BRANCH_INVISIBLE, k_pool, v_pool, out);
+}
+
+/* The same with the mask of the attention-mask ablation chosen by mask_mode (q_pos may be null). */
+int aspd_oracle_attn_masked(int n_req, int mode, int Hq, int Hkv, int d,
+                            int page_size, double theta, double sm_scale,
+                            const int* prefix_len, const int* n_branches,
+                            const int* branch_begin, const int* page_begin,
+                            const int* tail_off, const int* tail_len,
+                            const int* br_kv_off, const int* br_kv_len,
+                            const int* br_q_len, const int* page_ids, const double* q,
+                            const int* q_pos, int mask_mode,
+                            const double* k_pool, const double* v_pool, double* out) {
+  if (mask_mode != MASK_BRANCH_INVISIBLE && mask_mode != MASK_SHARED) return ORACLE_BAD;
+  return attn_impl(n_req, mode, Hq, Hkv, d, page_size, theta, sm_scale, prefix_len, n_branches, branch_begin,
+                   page_begin, tail_off, tail_len, br_kv_off, br_kv_len, br_q_len, page_ids, q, q_pos, mask_mode, k_pool, v_pool, out);
 }
 
 /*
@@ -457,12 +514,12 @@ int aspd_oracle_attn_at(int n_req, int mode, int Hq, int Hkv, int d,
  * defines it (integers only; used to compare mask membership bit for bit).
  * vis_out [n_new][n_slots] (0/1); n_slots = slots per request row given.
  */
-int aspd_oracle_visible_slots(int n_req, int mode, int n_slots,
+static int visible_slots_impl(int n_req, int mode, int n_slots,
                               const int* prefix_len, const int* n_branches,
                               const int* branch_begin, const int* tail_off,
                               const int* tail_len, const int* br_kv_off,
                               const int* br_kv_len, const int* br_q_len,
-                              uint8_t* vis_out) {
+                              int mask_mode, uint8_t* vis_out) {
   int n = 0;
   for (int r = 0; r < n_req; ++r) {
     int P = prefix_len[r];
@@ -478,6 +535,12 @@ int aspd_oracle_visible_slots(int n_req, int mode, int n_slots,
             if (br_q_len[S] == -1) for (int j = 0; j < br_kv_len[S]; ++j) row[br_kv_off[S] + j] = 1;
           }
           for (int j = 0; j <= br_kv_len[B] - br_q_len[B] + i; ++j) row[br_kv_off[B] + j] = 1;
+          if (mask_mode == MASK_SHARED)                     /* other branches of the stage: offsets below the token's own */
+            for (int c = 0; c < n_branches[r]; ++c) {
+              int C = branch_begin[r] + c;
+              if (C == B || br_q_len[C] == -1) continue;
+              for (int j = 0; j < br_kv_len[C] && j < br_kv_len[B] - br_q_len[B] + i; ++j) row[br_kv_off[C] + j] = 1;
+            }
           ++n;
         }
       }
@@ -494,4 +557,25 @@ int aspd_oracle_visible_slots(int n_req, int mode, int n_slots,
     }
   }
   return n;
+}
+
+int aspd_oracle_visible_slots(int n_req, int mode, int n_slots,
+                              const int* prefix_len, const int* n_branches,
+                              const int* branch_begin, const int* tail_off,
+                              const int* tail_len, const int* br_kv_off,
+                              const int* br_kv_len, const int* br_q_len,
+                              uint8_t* vis_out) {
+  return visible_slots_impl(n_req, mode, n_slots, prefix_len, n_branches, branch_begin, tail_off, tail_len, br_kv_off,
+                            br_kv_len, br_q_len, MASK_BRANCH_INVISIBLE, vis_out);
+}
+
+int aspd_oracle_visible_slots_masked(int n_req, int mode, int n_slots,
+                                     const int* prefix_len, const int* n_branches,
+                                     const int* branch_begin, const int* tail_off,
+                                     const int* tail_len, const int* br_kv_off,
+                                     const int* br_kv_len, const int* br_q_len,
+                                     int mask_mode, uint8_t* vis_out) {
+  if (mask_mode != MASK_BRANCH_INVISIBLE && mask_mode != MASK_SHARED) return ORACLE_BAD;
+  return visible_slots_impl(n_req, mode, n_slots, prefix_len, n_branches, branch_begin, tail_off, tail_len, br_kv_off,
+                            br_kv_len, br_q_len, mask_mode, vis_out);
 }

@@ -12,8 +12,9 @@ import oracle
 
 
 class OracleRun:
-    def __init__(self, wl):
+    def __init__(self, wl, mask=oracle.MASK_BRANCH_INVISIBLE):
         self.wl = wl
+        self.mask = mask       # attention mask of the parallel steps (the ablation's visible mask: MASK_SHARED)
         self.k_pool, self.v_pool = oracle.make_pools(wl.n_pool_pages, wl.Hkv, wl.page_size, wl.d)
         self.outputs = []      # one [n_new][Hq][d] array per compared phase
         self.positions = []    # per phase: (pos, slot, req) int32 arrays
@@ -29,15 +30,15 @@ class OracleRun:
         oracle.kv_append(ph.desc, ph.k_new, ph.v_new, pos, req, slot, self.k_pool, self.v_pool, wl.theta)
         if attend and ph.q is not None:
             out = oracle.attn(ph.desc, ph.mode, ph.q, self.k_pool, self.v_pool, wl.theta, wl.sm_scale,
-                              q_pos=pos if pos_override is not None else None)
+                              q_pos=pos if pos_override is not None else None, mask=self.mask)
             if ph.compare:
                 self.outputs.append(out)
             return out
         return None
 
 
-def run_workload(wl) -> OracleRun:
-    run = OracleRun(wl)
+def run_workload(wl, mask=oracle.MASK_BRANCH_INVISIBLE) -> OracleRun:
+    run = OracleRun(wl, mask)
     for ph in wl.phases:
         run.step(ph)
     return run

@@ -297,9 +297,11 @@ def test_branch_permutation_permutes_outputs():
     np.testing.assert_array_equal(outp, base[perm])
 
 
-def test_dense_and_descriptor_forms_agree():
+@pytest.mark.parametrize("mask", [oracle.MASK_BRANCH_INVISIBLE, oracle.MASK_SHARED])
+def test_dense_and_descriptor_forms_agree(mask):
     """oracle-S (engine prose) computes exactly what oracle-D (Eq. 1-4) does, whatever the
-    arrangement of tokens in memory: branch-contiguous slots vs interleaved decoding order."""
+    arrangement of tokens in memory: branch-contiguous slots vs interleaved decoding order.
+    Also under the ablation's visible mask."""
     rng = np.random.default_rng(11)
     for trial in range(12):
         P = int(rng.integers(1, 9)); nb = int(rng.integers(1, 5))
@@ -317,7 +319,7 @@ def test_dense_and_descriptor_forms_agree():
         # reference layout: final lengths known, decode step by step
         final = W.build_segment_workload("g", 100 + trial, Hq, Hkv, d, "f32", theta, [P], [[0] * nb], [lens],
                                          serial_steps=n_serial)
-        run = oracle.run.OracleRun(final)
+        run = oracle.run.OracleRun(final, mask)
         run.step(final.phases[0])                               # prefix
         par = [p for p in final.phases if p.label == "parallel-step"][0]
         # split the one-shot parallel phase (q_len = len) into per-token steps
@@ -340,18 +342,19 @@ def test_dense_and_descriptor_forms_agree():
             flat_branch.append(-1); flat_stage.append(2)
             flat_k.append(ph.k_new[0]); flat_v.append(ph.v_new[0]); flat_q.append(ph.q[0]); outs.append(o[0])
         dense = oracle.dense_attn(np.array(flat_q), np.array(flat_k), np.array(flat_v), flat_branch, flat_stage,
-                                  theta, final.sm_scale)
+                                  theta, final.sm_scale, mask=mask)
         np.testing.assert_allclose(dense[P:], np.array(outs), atol=1e-12)
 
 
-def test_whole_branches_at_once_equal_dense_form():
+@pytest.mark.parametrize("mask", [oracle.MASK_BRANCH_INVISIBLE, oracle.MASK_SHARED])
+def test_whole_branches_at_once_equal_dense_form(mask):
     """Teacher-forcing layout: every branch gets all its tokens in one step (block-diagonal mask
     across branches, causal inside a branch).  The descriptor form equals Eq. 1-4 taken literally
     for every one of those tokens, whatever order the branches are laid out in."""
     Hq, Hkv, d, theta = 4, 2, 16, 1e4
     P, lens = 6, [4, 1, 7]
     wl = W.build_segment_workload("tf", 23, Hq, Hkv, d, "f32", theta, [P], [[0, 0, 0]], [lens], serial_steps=1)
-    run = run_workload(wl)
+    run = run_workload(wl, mask)
     fill = wl.phases[0]
     par = [p for p in wl.phases if p.label == "parallel-step"][0]
     ser = wl.phases[-1]
@@ -361,7 +364,7 @@ def test_whole_branches_at_once_equal_dense_form():
     q = np.concatenate([np.zeros((P, Hq, d)), par.q, ser.q])
     k = np.concatenate([fill.k_new, par.k_new, ser.k_new])
     v = np.concatenate([fill.v_new, par.v_new, ser.v_new])
-    dense = oracle.dense_attn(q, k, v, branch, stage, theta, wl.sm_scale)
+    dense = oracle.dense_attn(q, k, v, branch, stage, theta, wl.sm_scale, mask=mask)
     np.testing.assert_allclose(run.outputs[0], dense[P:P + sum(lens)], atol=1e-12)
     np.testing.assert_allclose(run.outputs[1][0], dense[-1], atol=1e-12)
     pos, _, _ = oracle.new_tokens(par.desc, oracle.MODE_BRANCH)
@@ -455,6 +458,102 @@ def test_position_id_variants_through_caller_given_positions():
 
 
 # ------------------------------------------------------------------ softmax closed forms
+# ------------------------------------------------- the ablation's visible ("Shared") mask
+GOLDEN_SHARED = os.path.join(os.path.dirname(__file__), "golden", "worked_example_shared_mask.txt")
+
+
+def test_shared_mask_worked_example():
+    """Hand-derived visible sets of the worked example when the visibility function is 1
+    everywhere and only the order of the position IDs remains."""
+    rows = load_example()
+    pos = oracle.dense_positions([r[1] for r in rows], [r[2] for r in rows])
+    vis = oracle.dense_visible_shared(pos)
+    n = 0
+    for line in open(GOLDEN_SHARED):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        idx, p_, want = line.split()
+        assert int(p_) == pos[int(idx)]
+        assert np.flatnonzero(vis[int(idx)]).tolist() == [int(x) for x in want.split(",")], idx
+        n += 1
+    assert n == len(rows)
+    # a superset of the branch-invisible mask, equal to it on the main branch
+    iso = oracle.dense_visible([r[1] for r in rows], [r[2] for r in rows])
+    assert (vis >= iso).all() and (vis != iso).any()
+    for i, r in enumerate(rows):
+        if r[1] < 0:
+            assert (vis[i] == iso[i]).all()
+
+
+def test_shared_mask_is_what_exists_under_lockstep_decoding():
+    """Another description of the same mask, by time instead of by position: a serial step decodes
+    one token, a parallel step one token of every live branch; a token sees what earlier STEPS
+    produced, and itself.  Random multi-stage requests; also the attention itself against library
+    SDPA with that boolean mask."""
+    rng = np.random.default_rng(19)
+    for trial in range(30):
+        branch, stage, born = [], [], []
+        st, step = 0, 0
+        for _seg in range(int(rng.integers(1, 4))):
+            for _ in range(int(rng.integers(1, 5))):
+                branch.append(-1); stage.append(st); born.append(step); step += 1
+            st += 1
+            lens = rng.integers(1, 5, size=int(rng.integers(1, 4)))
+            for k in range(int(lens.max())):
+                for b in range(len(lens)):
+                    if k < lens[b]:
+                        branch.append(b); stage.append(st); born.append(step)
+                step += 1
+            st += 1
+        branch.append(-1); stage.append(st); born.append(step)
+        L = len(branch)
+        want = np.array([[1 if (born[j] < born[i] or i == j) else 0 for j in range(L)] for i in range(L)], dtype=np.uint8)
+        pos = oracle.dense_positions(branch, stage)
+        np.testing.assert_array_equal(oracle.dense_visible_shared(pos), want)
+        if trial < 4:
+            Hq, Hkv, d, theta, scale = 4, 2, 8, 77.0, 0.3
+            q = rng.standard_normal((L, Hq, d)); k = rng.standard_normal((L, Hkv, d)); v = rng.standard_normal((L, Hkv, d))
+            out = oracle.dense_attn(q, k, v, branch, stage, theta, scale, mask=oracle.MASK_SHARED)
+            qh = torch.tensor(_library_rotary(q, pos, theta)).permute(1, 0, 2)
+            kh = torch.tensor(_library_rotary(k, pos, theta)).permute(1, 0, 2).repeat_interleave(Hq // Hkv, dim=0)
+            vv = torch.tensor(v).permute(1, 0, 2).repeat_interleave(Hq // Hkv, dim=0)
+            ref = torch.nn.functional.scaled_dot_product_attention(qh[None], kh[None], vv[None],
+                                                                   attn_mask=torch.tensor(want.astype(bool)), scale=scale)
+            np.testing.assert_allclose(out, ref[0].permute(1, 0, 2).numpy(), atol=1e-12)
+
+
+def test_shared_mask_descriptor_visible_sets():
+    """Descriptor form, integers: a new token at offset k of its branch sees the prefix, earlier
+    stages, its own branch up to itself and the first k tokens of every other branch of its
+    stage -- also of branches that decode nothing in this step."""
+    wl = W.build_two_stage_workload("ts", 5, 4, 2, 8, "f32", 1e4, 7, [3, 1, 2], 2, [4, 0, 6], [1, 2, 1])
+    ph = [p for p in wl.phases if p.mode == W.MODE_BRANCH and p.q is not None][-1]
+    d = ph.desc
+    n_slots = int(d["n_pages"][0]) * wl.page_size
+    vis = oracle.visible_slots(d, oracle.MODE_BRANCH, n_slots, mask=oracle.MASK_SHARED)
+    iso = oracle.visible_slots(d, oracle.MODE_BRANCH, n_slots)
+    t = 0
+    for b in range(int(d["n_branches"][0])):
+        for i in range(max(0, int(d["br_q_len"][b]))):
+            k = int(d["br_kv_len"][b]) - int(d["br_q_len"][b]) + i
+            extra = set()
+            for c in range(int(d["n_branches"][0])):
+                if c != b and int(d["br_q_len"][c]) >= 0:
+                    extra |= {int(d["br_kv_off"][c]) + j for j in range(min(k, int(d["br_kv_len"][c])))}
+            assert set(np.flatnonzero(vis[t])) == set(np.flatnonzero(iso[t])) | extra, (b, i)
+            t += 1
+    assert t == len(vis) and (vis != iso).any()
+
+
+def test_shared_mask_single_branch_is_plain_causal():
+    """With one branch there is nobody else to see: both masks give the same attention."""
+    wl = W.build_segment_workload("one", 9, 4, 2, 16, "f32", 1e4, [11], [[5]], [[3]], serial_steps=1)
+    a, b = run_workload(wl), run_workload(wl, oracle.MASK_SHARED)
+    for x, y in zip(a.outputs, b.outputs):
+        np.testing.assert_array_equal(x, y)
+
+
 def test_softmax_closed_forms():
     wl = W.build_segment_workload("c", 21, 4, 2, 16, "f32", 10000.0, [19], [[4, 9]], [[1, 1]], serial_steps=1)
     ph = {p.label: p for p in wl.phases}
