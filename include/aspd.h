@@ -105,7 +105,17 @@ typedef struct {
                            layer's pools are only touched by that layer's own step.  The kernel
                            may then start fetching such pages before the previous kernel on the
                            stream has finished.  0 (default): full stream ordering for the pools */
+  int32_t mask;         /* ASPD_MASK_*: attention mask of a parallel step (default: branch-invisible) */
 } aspd_tuning_t;
+
+/* Attention mask of a parallel step.  BRANCH_INVISIBLE is the paper's mask (its Eq. 2-3).  SHARED
+ * is the visible mask of its attention-mask ablation, read as "only the order of the position IDs
+ * remains": a new token at offset k of its branch also sees the first k tokens of every other
+ * branch of its stage (branches with q_len = 0 included) -- what exists when the branches decode
+ * in lockstep.  Serial steps are the same under both.  SHARED plans never fuse the append into the
+ * attention pass and never deal whole streams. */
+#define ASPD_MASK_BRANCH_INVISIBLE 0
+#define ASPD_MASK_SHARED 1
 
 /* One split-K work item of a plan, as aspd_plan_items reports it.  The pages a request's
  * step must read form one key stream (prefix, then the branches that have queries, or every
@@ -185,6 +195,9 @@ int aspd_visible_slots(const aspd_request_t* req, const aspd_branch_t* br, int n
  * Errors: ASPD_ERR_BAD_DESCRIPTOR for overlapping or out-of-table regions, unaligned kv_off /
  * tail_off, q_len > kv_len, serial mode with tail_len < 1, duplicate or out-of-pool page ids.
  */
+int aspd_visible_slots_masked(const aspd_request_t* req, const aspd_branch_t* br, int n_req, int mode, int mask,
+                              int n_slots, uint8_t* vis_out /*host*/);
+
 int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const aspd_branch_t* br,
                      const int32_t* page_ids, int n_req, int64_t n_pool_pages, int mode,
                      const int32_t* q_pos, const aspd_tuning_t* tuning, void* stream,
@@ -202,6 +215,10 @@ int aspd_plan_stream_pages(const aspd_plan_t* plan, int32_t* page_ids /*host*/, 
                            int max_pages);
 /* Per new token, the stream keys it may attend: [0, pe) and [lo, hi) (host arrays of n_new). */
 int aspd_plan_token_ranges(const aspd_plan_t* plan, int32_t* pe, int32_t* lo, int32_t* hi, int max_tokens);
+/* Plans with ASPD_MASK_SHARED: per new token its offset k in its branch (it also attends keys of
+ * other branches at offsets below k), and per stream page the page's index inside its branch
+ * (host arrays of n_new and n_stream_pages entries).  ASPD_ERR_INVALID_ARG for other plans. */
+int aspd_plan_shared_mask_tables(const aspd_plan_t* plan, int32_t* below /*host*/, int32_t* page_in_branch /*host*/);
 /* Device status word of the plan (synchronises `stream`): ASPD_OK, or the first error a
  * kernel recorded (ASPD_ERR_TIMEOUT from a bounded wait, ASPD_ERR_BAD_DESCRIPTOR from a
  * bounds check). */

@@ -20,6 +20,7 @@ MODE_BRANCH, MODE_SERIAL = 0, 1
 DTYPE_F32, DTYPE_BF16 = 0, 1
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_MMA = 0, 1, 2
 Q_SHARED = -1
+MASK_BRANCH_INVISIBLE, MASK_SHARED = 0, 1
 
 REQUEST_DTYPE = np.dtype([(n, np.int32) for n in
                           ("prefix_len", "n_branches", "branch_begin", "page_begin", "n_pages", "tail_off", "tail_len")])
@@ -37,7 +38,7 @@ class Shape(ctypes.Structure):
 
 class Tuning(ctypes.Structure):
     _fields_ = [("kernel", ctypes.c_int32), ("chunk_tokens", ctypes.c_int32), ("n_ctas", ctypes.c_int32),
-                ("host_only", ctypes.c_int32), ("stable_cache", ctypes.c_int32)]
+                ("host_only", ctypes.c_int32), ("stable_cache", ctypes.c_int32), ("mask", ctypes.c_int32)]
 
 
 class PlanInfo(ctypes.Structure):
@@ -56,8 +57,8 @@ class AspdError(RuntimeError):
 
 
 EXPORTS = ("aspd_strerror", "aspd_pool_bytes", "aspd_count_new_tokens", "aspd_positions", "aspd_visible_slots",
-           "aspd_plan_create", "aspd_plan_destroy", "aspd_plan_info", "aspd_plan_items", "aspd_plan_cta_ranges", "aspd_plan_stream_pages",
-           "aspd_plan_token_ranges", "aspd_plan_status",
+           "aspd_visible_slots_masked", "aspd_plan_create", "aspd_plan_destroy", "aspd_plan_info", "aspd_plan_items", "aspd_plan_cta_ranges", "aspd_plan_stream_pages",
+           "aspd_plan_token_ranges", "aspd_plan_shared_mask_tables", "aspd_plan_status",
            "aspd_kv_append", "aspd_branch_attn", "aspd_serial_attn", "aspd_attn_partials", "aspd_attn_combine",
            "aspd_branch_step", "aspd_serial_step", "aspd_step_host", "aspd_attn_static", "aspd_k_rerotate", "aspd_debug_read_token", "aspd_debug_bounded_wait")
 
@@ -83,6 +84,7 @@ def lib() -> ctypes.CDLL:
         L.aspd_count_new_tokens.argtypes = [vp, vp, ci, ci]
         L.aspd_positions.argtypes = [vp, vp, ci, ci, vp, vp, vp]
         L.aspd_visible_slots.argtypes = [vp, vp, ci, ci, ci, vp]
+        L.aspd_visible_slots_masked.argtypes = [vp, vp, ci, ci, ci, ci, vp]
         L.aspd_plan_create.argtypes = [vp, vp, vp, vp, ci, ctypes.c_int64, ci, vp, vp, vp, vp]
         L.aspd_plan_destroy.argtypes = [vp]
         L.aspd_plan_info.argtypes = [vp, vp]
@@ -90,6 +92,7 @@ def lib() -> ctypes.CDLL:
         L.aspd_plan_cta_ranges.argtypes = [vp, vp, ci]
         L.aspd_plan_stream_pages.argtypes = [vp, vp, vp, ci]
         L.aspd_plan_token_ranges.argtypes = [vp, vp, vp, vp, ci]
+        L.aspd_plan_shared_mask_tables.argtypes = [vp, vp, vp]
         L.aspd_plan_status.argtypes = [vp, vp]
         L.aspd_kv_append.argtypes = [vp] * 7
         L.aspd_branch_attn.argtypes = [vp] * 6
@@ -183,11 +186,15 @@ def positions(desc, mode: int):
     return pos[:n], slot[:n], rq[:n]
 
 
-def visible_slots(desc, mode: int, n_slots: int) -> np.ndarray:
+def visible_slots(desc, mode: int, n_slots: int, mask: int = 0) -> np.ndarray:
     req, br, _ = pack_descriptors(desc)
     n = _check(lib().aspd_count_new_tokens(_ptr(req), _ptr(br), len(req), mode), "aspd_count_new_tokens")
     vis = np.zeros((max(n, 1), n_slots), dtype=np.uint8)
-    _check(lib().aspd_visible_slots(_ptr(req), _ptr(br), len(req), mode, n_slots, _ptr(vis)), "aspd_visible_slots")
+    if mask == MASK_BRANCH_INVISIBLE:
+        _check(lib().aspd_visible_slots(_ptr(req), _ptr(br), len(req), mode, n_slots, _ptr(vis)), "aspd_visible_slots")
+    else:
+        _check(lib().aspd_visible_slots_masked(_ptr(req), _ptr(br), len(req), mode, mask, n_slots, _ptr(vis)),
+               "aspd_visible_slots_masked")
     return vis[:n]
 
 
@@ -195,10 +202,11 @@ class Plan:
     """Owner of an ``aspd_plan_t`` (see ``aspd_plan_create``)."""
 
     def __init__(self, shape: Shape, desc, n_pool_pages: int, mode: int, q_pos=None, kernel: int = KERNEL_AUTO,
-                 chunk_tokens: int = 0, n_ctas: int = 0, host_only: bool = False, stable_cache: bool = False, stream=None):
+                 chunk_tokens: int = 0, n_ctas: int = 0, host_only: bool = False, stable_cache: bool = False, stream=None,
+                 mask: int = 0):
         self.shape, self.mode = shape, mode
         req, br, pages = pack_descriptors(desc)
-        tune = Tuning(kernel, chunk_tokens, n_ctas, 1 if host_only else 0, 1 if stable_cache else 0)
+        tune = Tuning(kernel, chunk_tokens, n_ctas, 1 if host_only else 0, 1 if stable_cache else 0, mask)
         qp = None if q_pos is None else np.ascontiguousarray(q_pos, dtype=np.int32)
         handle = ctypes.c_void_p()
         self._h = None
@@ -234,6 +242,13 @@ class Plan:
         pe, lo, hi = (np.zeros(max(n, 1), np.int32) for _ in range(3))
         _check(lib().aspd_plan_token_ranges(self._h, _ptr(pe), _ptr(lo), _ptr(hi), n), "aspd_plan_token_ranges")
         return pe[:n], lo[:n], hi[:n]
+
+    def shared_mask_tables(self):
+        """(below per new token, page index in its branch per stream page) of a MASK_SHARED plan."""
+        below = np.zeros(max(self.n_new, 1), np.int32)
+        pib = np.zeros(max(self.info.n_stream_pages, 1), np.int32)
+        _check(lib().aspd_plan_shared_mask_tables(self._h, _ptr(below), _ptr(pib)), "aspd_plan_shared_mask_tables")
+        return below[: self.n_new], pib[: self.info.n_stream_pages]
 
     def status(self, stream=None) -> int:
         return lib().aspd_plan_status(self._h, _stream(stream))

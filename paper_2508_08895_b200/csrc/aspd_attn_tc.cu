@@ -66,7 +66,7 @@ struct Misc {
   float smax[2][256];          // per S buffer: tile maximum of every softmax thread
   float fin_m[2][64];          // per item parity: reference maximum of every query row ...
   float fin_l[2][256];         // ... and the sum of every softmax thread
-  int nval[4][8];              // valid rows of the 8 pages of a tile (ring over 4 tiles)
+  int nval[4][8];              // page entries (valid rows | ... | upper bits) of the 8 pages of a tile (ring over 4 tiles)
   DeviceItem items[kItemCache];        // this CTA's first items and, per item, the visible ranges of
   int4 vis[kItemCache][kMaxTokPerItem]; // its query tokens: no global-load chain at an item boundary
   uint32_t tmem_base;
@@ -283,9 +283,11 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
     float mx = -INFINITY;
 #pragma unroll
     for (int pg = 0; pg < HC / 16; ++pg) {
-      const int nv = misc->nval[g & 3][col0 / 16 + pg];
+      const int ye = misc->nval[g & 3][col0 / 16 + pg], nv = ye & 255;
       const int kb = it.key0 + t * kTile + col0 + pg * 16;       // stream key of the page's first row
-      const uint32_t mask = bits_between(0, min(nv, vis.x - kb)) | bits_between(vis.y - kb, min(nv, vis.z - kb));
+      // [0, pe), [lo, hi) and, under the shared mask (vis.w > 0), offsets below vis.w in other branches
+      const uint32_t mask = bits_between(0, min(nv, vis.x - kb)) | bits_between(vis.y - kb, min(nv, vis.z - kb)) |
+                            bits_between(0, min(nv, vis.w - (ye >> 13) * 16));
       if (mask == 0xFFFFu) {
 #pragma unroll
         for (int i = 0; i < 16; ++i) mx = fmaxf(mx, s[pg * 16 + i]);
@@ -406,9 +408,10 @@ __device__ __forceinline__ bool softmax_item_wide(const Ctx& c, const DeviceItem
         tmem_wait_ld();
 #pragma unroll
         for (int pg = 0; pg < 2; ++pg) {
-          const int nv = misc->nval[g & 3][col0 / 16 + ch * 2 + pg];
+          const int ye = misc->nval[g & 3][col0 / 16 + ch * 2 + pg], nv = ye & 255;
           const int kb = it.key0 + t * kTile + col0 + ch * 32 + pg * 16;
-          const uint32_t mask = bits_between(0, min(nv, vis.x - kb)) | bits_between(vis.y - kb, min(nv, vis.z - kb));
+          const uint32_t mask = bits_between(0, min(nv, vis.x - kb)) | bits_between(vis.y - kb, min(nv, vis.z - kb)) |
+                                bits_between(0, min(nv, vis.w - (ye >> 13) * 16));
 #pragma unroll
           for (int i = 0; i < 16; i += 4) {
             float e0 = fmaf(s[pg * 16 + i], c.scale_log2, nb), e1 = fmaf(s[pg * 16 + i + 1], c.scale_log2, nb);
@@ -748,7 +751,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
         good = __shfl_sync(0xffffffffu, good, 0);
         if (!good) { ok = false; break; }
         if (lane == 0) ASPD_STAMP(c, g, 6 + kv);
-        if (kv == 0 && lane < 8) misc->nval[g & 3][lane] = pg.y & 255;   // read by the softmax warps of tile g
+        if (kv == 0 && lane < 8) misc->nval[g & 3][lane] = pg.y;   // read by the softmax warps of tile g
         __syncwarp();
         if (lane == 0) mbar_expect_tx(full, (uint32_t)npg * 4096u);
         __syncwarp();

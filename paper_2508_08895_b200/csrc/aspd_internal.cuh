@@ -80,6 +80,7 @@ struct aspd_plan {
   int fuse_append;             // few enough new rows per CTA for the attention pass to write them itself
   int stable_cache;            // producers may fetch pages without new rows before the dependency wait
   int dealt;                   // whole streams dealt to the CTAs in turn (many more streams than CTAs)
+  int shared_mask;             // parallel step under the ablation's visible mask
   int wide;                    // dealt plan of the tensor-core kernel: row blocks of up to kMaxRowsWide rows
   int64_t n_pool_pages;
   int64_t kv_tokens_read;

@@ -141,7 +141,9 @@ __global__ void __launch_bounds__(128) attn_generic_kernel(PlanDevice pd, const 
       q_s[warp][i + D / 2] = (x1 * cs.x + x0 * cs.y) * scale_log2;
     }
     __syncwarp();
-    const int4 vis = pd.tok_vis[tok];           // stream keys [0, pe) and [lo, hi) are visible
+    // stream keys [0, pe) and [lo, hi) are visible; under the shared mask (w > 0) also keys of other
+    // branches whose offset in their branch (page index in the upper bits of the page entry) is below w
+    const int4 vis = pd.tok_vis[tok];
     float m = -INFINITY, l = 0.f, acc[EPL];
 #pragma unroll
     for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
@@ -152,7 +154,7 @@ __global__ void __launch_bounds__(128) attn_generic_kernel(PlanDevice pd, const 
       if (j < n_keys) {
         const int2 pg = pd.visit[it.page0 + j / page_size];
         const int row = j % page_size, kg = it.key0 + j;
-        seen = row < (pg.y & 255) && (kg < vis.x || (kg >= vis.y && kg < vis.z));
+        seen = row < (pg.y & 255) && (kg < vis.x || (kg >= vis.y && kg < vis.z) || (pg.y >> 13) * page_size + row < vis.w);
         if (seen) {
           const char* tile = reinterpret_cast<const char*>(k_pool) + ((size_t)pg.x * n_kv_heads + it.kv_head) * tb;
           float dot = 0.f;

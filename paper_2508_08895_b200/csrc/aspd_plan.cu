@@ -157,9 +157,14 @@ int aspd_positions(const aspd_request_t* req, const aspd_branch_t* br, int n_req
 
 int aspd_visible_slots(const aspd_request_t* req, const aspd_branch_t* br, int n_req, int mode, int n_slots,
                        uint8_t* vis_out) {
+  return aspd_visible_slots_masked(req, br, n_req, mode, ASPD_MASK_BRANCH_INVISIBLE, n_slots, vis_out);
+}
+
+int aspd_visible_slots_masked(const aspd_request_t* req, const aspd_branch_t* br, int n_req, int mode, int mask, int n_slots,
+                              uint8_t* vis_out) {
   int n = aspd_count_new_tokens(req, br, n_req, mode);
   if (n < 0) return n;
-  if (!vis_out || n_slots < 0) return ASPD_ERR_INVALID_ARG;
+  if (!vis_out || n_slots < 0 || (mask != ASPD_MASK_BRANCH_INVISIBLE && mask != ASPD_MASK_SHARED)) return ASPD_ERR_INVALID_ARG;
   memset(vis_out, 0, (size_t)n * n_slots);
   int t = 0;
   auto mark = [&](int tok, int lo, int hi) -> int {
@@ -178,7 +183,13 @@ int aspd_visible_slots(const aspd_request_t* req, const aspd_branch_t* br, int n
             const aspd_branch_t& y = br[q.branch_begin + s2];
             if (y.q_len == ASPD_Q_SHARED && mark(t, y.kv_off, y.kv_off + y.kv_len)) return ASPD_ERR_INVALID_ARG;
           }
-          if (mark(t, x.kv_off, x.kv_off + x.kv_len - x.q_len + i + 1)) return ASPD_ERR_INVALID_ARG;
+          const int k = x.kv_len - x.q_len + i;                // the token's offset in its branch
+          if (mark(t, x.kv_off, x.kv_off + k + 1)) return ASPD_ERR_INVALID_ARG;
+          if (mask == ASPD_MASK_SHARED)                         // smaller offsets of the stage's other branches
+            for (int s2 = 0; s2 < q.n_branches; ++s2) {
+              const aspd_branch_t& y = br[q.branch_begin + s2];
+              if (s2 != b && y.q_len != ASPD_Q_SHARED && mark(t, y.kv_off, y.kv_off + std::min(k, y.kv_len))) return ASPD_ERR_INVALID_ARG;
+            }
         }
       }
     } else {
@@ -208,11 +219,13 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   const int n_new = aspd_count_new_tokens(req, br, n_req, mode);
   if (n_new < 0) return n_new;
 
-  aspd_tuning_t tune = {ASPD_KERNEL_AUTO, 0, 0, 0, 0};
+  aspd_tuning_t tune = {ASPD_KERNEL_AUTO, 0, 0, 0, 0, ASPD_MASK_BRANCH_INVISIBLE};
   if (tuning) tune = *tuning;
   const int ps = shape->page_size, d = shape->head_dim, Hq = shape->n_q_heads, Hkv = shape->n_kv_heads;
   const int G = Hq / Hkv, es = esize_of(shape->dtype);
   if (tune.chunk_tokens < 0 || tune.chunk_tokens % ps || tune.n_ctas < 0) return ASPD_ERR_INVALID_ARG;
+  if (tune.mask != ASPD_MASK_BRANCH_INVISIBLE && tune.mask != ASPD_MASK_SHARED) return ASPD_ERR_INVALID_ARG;
+  const bool shared_mask = tune.mask == ASPD_MASK_SHARED && mode == ASPD_MODE_BRANCH;
   const bool mma_ok = shape->dtype == ASPD_DTYPE_BF16 && d == 128 && ps == 16;
   int kernel = tune.kernel;
   if (kernel == ASPD_KERNEL_AUTO) kernel = mma_ok ? ASPD_KERNEL_MMA : ASPD_KERNEL_GENERIC;
@@ -223,6 +236,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   if (!p) return ASPD_ERR_NOMEM;
   p->shape = *shape; p->mode = mode; p->n_req = n_req; p->n_new = n_new; p->kernel = kernel;
   p->stable_cache = tune.stable_cache ? 1 : 0;
+  p->shared_mask = (tune.mask == ASPD_MASK_SHARED && mode == ASPD_MODE_BRANCH) ? 1 : 0;
   p->host_only = tune.host_only; p->n_pool_pages = n_pool_pages; p->device_base = nullptr; p->device_bytes = 0;
   memset(&p->dev, 0, sizeof(p->dev));
   p->sm_count = 148;
@@ -267,12 +281,17 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
     // new_key0 / new_tok0: the keys [new_key0, len) of the region are this step's new tokens
     // new_tok0, new_tok0 + 1, ...; a page entry carries (valid rows | new rows << 8 | first new
     // token << 13) so that a fused step can write those rows just before it reads the page.
-    auto push_region = [&](const aspd_request_t& q, int slot0, int len, int new_key0, int new_tok0) {
+    // Under the shared mask the upper bits carry the page's index inside its branch instead (its
+    // first key's offset / page_size; such plans never fuse the append): a token at offset k
+    // also sees the keys of other branches whose offset is below k.
+    auto push_region = [&](const aspd_request_t& q, int slot0, int len, int new_key0, int new_tok0, bool branch_pages = false) {
       for (int s0 = 0; s0 < len; s0 += ps) {
         const int nv = std::min(ps, len - s0), first_new = std::max(s0, new_key0);
         const int n_newrows = std::max(0, s0 + nv - first_new);
         int y = nv;
-        if (n_newrows > 0) y |= (n_newrows << 8) | ((new_tok0 + first_new - new_key0) << 13);
+        if (n_newrows > 0) y |= (n_newrows << 8);
+        if (shared_mask) y |= branch_pages ? (s0 / ps) << 13 : 0;
+        else if (n_newrows > 0) y |= (new_tok0 + first_new - new_key0) << 13;
         visit.push_back(make_int2(page_ids[q.page_begin + (slot0 + s0) / ps], y));
       }
     };
@@ -292,7 +311,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
         for (int b = 0; b < q.n_branches; ++b) {
           const aspd_branch_t& x = br[q.branch_begin + b];
           nq += std::max(0, x.q_len);
-          if (x.q_len != 0) kv_req += x.kv_len;
+          if (x.q_len != 0 || shared_mask) kv_req += x.kv_len;
         }
         if (nq == 0) continue;
         kv_count += kv_req;
@@ -301,10 +320,10 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
           const int pe = ((int)visit.size() - v0) * ps;
           for (int b = 0; b < q.n_branches; ++b) {
             const aspd_branch_t& x = br[q.branch_begin + b];
-            if (x.q_len <= 0) continue;
-            const int lo = ((int)visit.size() - v0) * ps;
-            push_region(q, x.kv_off, x.kv_len, x.kv_len - x.q_len, t);
-            for (int i = 0; i < x.q_len; ++i) tok_vis[t++] = make_int4(pe, lo, lo + x.kv_len - x.q_len + i + 1, 0);
+            if (x.q_len < 0 || (x.q_len == 0 && !shared_mask)) continue;     // shared mask: also branches without queries
+            const int lo = ((int)visit.size() - v0) * ps, prior = x.kv_len - x.q_len;
+            push_region(q, x.kv_off, x.kv_len, prior, t, true);
+            for (int i = 0; i < x.q_len; ++i) tok_vis[t++] = make_int4(pe, lo, lo + prior + i + 1, shared_mask ? prior + i : 0);
           }
           blocks.push_back({r, t_req, nq, v0, (int)visit.size() - v0});
         } else {
@@ -377,7 +396,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   // same one or two requests (which then stay in L2) and every CTA gets one stream of each round.
   // Every row block then gets a page sequence of its own, without the branch pages none of its
   // tokens sees, and the tensor-core kernel takes row blocks of up to 128 rows (its wide variant).
-  bool deal_streams = mode == ASPD_MODE_BRANCH && tune.chunk_tokens == 0 && (long)streams.size() >= 4L * ctas_for(total_pages);
+  bool deal_streams = mode == ASPD_MODE_BRANCH && !shared_mask && tune.chunk_tokens == 0 && (long)streams.size() >= 4L * ctas_for(total_pages);
   p->wide = 0;
   if (deal_streams) {
     p->wide = (kernel == ASPD_KERNEL_MMA && kMaxRowsWide / G > max_tok) ? 1 : 0;
@@ -461,7 +480,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   std::vector<int32_t> cta_dirty0(n_ctas + 1, 0);
   for (int c = 0; c < n_ctas; ++c) {
     cta_dirty0[c] = (int)dirty.size();
-    for (int i = cta_item0[c]; i < cta_item0[c + 1]; ++i) {
+    for (int i = cta_item0[c]; i < cta_item0[c + 1] && !shared_mask; ++i) {
       const DeviceItem& it = p->items[i];
       for (int pg = 0; pg < it.n_pages; ++pg) {
         const int2 v = visit[it.page0 + pg];
@@ -476,7 +495,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
     // rows per CTA (a branch-open step) the separate append kernel is the faster way
     int most = 0;
     for (int c = 0; c < n_ctas; ++c) most = std::max(most, cta_dirty0[c + 1] - cta_dirty0[c]);
-    p->fuse_append = most <= 20 ? 1 : 0;
+    p->fuse_append = (most <= 20 && !shared_mask) ? 1 : 0;
   }
   for (size_t i = 0; i < n_parts.size(); ++i) part_base[i + 1] = part_base[i] + n_parts[i];
   p->n_items = (int)p->items.size();
@@ -618,6 +637,13 @@ int aspd_plan_token_ranges(const aspd_plan_t* p, int32_t* pe, int32_t* lo, int32
   const int n = std::min<int>(max_tokens, (int)p->tok_vis.size());
   for (int i = 0; i < n; ++i) { pe[i] = p->tok_vis[i].x; lo[i] = p->tok_vis[i].y; hi[i] = p->tok_vis[i].z; }
   return (int)p->tok_vis.size();
+}
+
+int aspd_plan_shared_mask_tables(const aspd_plan_t* p, int32_t* below, int32_t* page_in_branch) {
+  if (!p || !p->shared_mask || !below || !page_in_branch) return ASPD_ERR_INVALID_ARG;
+  for (size_t i = 0; i < p->tok_vis.size(); ++i) below[i] = p->tok_vis[i].w;
+  for (size_t i = 0; i < p->visit.size(); ++i) page_in_branch[i] = p->visit[i].y >> 13;
+  return ASPD_OK;
 }
 
 int aspd_plan_status(aspd_plan_t* p, void* stream) {

@@ -45,8 +45,9 @@ class WorkloadRun:
     """Runs the phases of a workload through kv_append + attention, keeping compared outputs."""
 
     def __init__(self, wl: W.Workload, kernel: int = B.KERNEL_AUTO, chunk_tokens: int = 0, n_ctas: int = 0,
-                 device="cuda", fused: bool = False, stable_cache: bool = False):
+                 device="cuda", fused: bool = False, stable_cache: bool = False, mask: int = B.MASK_BRANCH_INVISIBLE):
         self.wl, self.kernel, self.chunk_tokens, self.n_ctas, self.device = wl, kernel, chunk_tokens, n_ctas, device
+        self.mask = mask            # attention mask of the parallel steps (ASPD_MASK_*)
         self.stable_cache = stable_cache
         self.fused = fused          # attention phases go through aspd_branch_step / aspd_serial_step
         self.shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
@@ -60,7 +61,7 @@ class WorkloadRun:
         passed to aspd_kv_append and, as q_pos, to the plan."""
         wl = self.wl
         plan = B.Plan(self.shape, ph.desc, wl.n_pool_pages, ph.mode, q_pos=pos_override, kernel=self.kernel,
-                      chunk_tokens=self.chunk_tokens, n_ctas=self.n_ctas, stable_cache=self.stable_cache)
+                      chunk_tokens=self.chunk_tokens, n_ctas=self.n_ctas, stable_cache=self.stable_cache, mask=self.mask)
         pos, slot, req = B.positions(ph.desc, ph.mode)
         if pos_override is not None:
             pos = np.ascontiguousarray(pos_override, dtype=np.int32)

@@ -81,14 +81,16 @@ def _shape(wl):
     return B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
 
 
-def _check_cover(wl, ph, plan, chunk=0, dealt=False):
+def _check_cover(wl, ph, plan, chunk=0, dealt=False, mask=0):
     """The plan's work items, expanded through its stream-page list and the per-token visible
     ranges to (token, KV head, logical slot) triples, are exactly the oracle's visible sets."""
     n_slots = int(ph.desc["n_pages"].max()) * wl.page_size
-    vis = oracle.visible_slots(ph.desc, ph.mode, n_slots)
+    vis = oracle.visible_slots(ph.desc, ph.mode, n_slots, mask=mask)
     _, _, treq = oracle.new_tokens(ph.desc, ph.mode)
     page_ids, n_valid = plan.stream_pages()
     pe, lo, hi = plan.token_ranges()
+    shared = bool(mask) and ph.mode == B.MODE_BRANCH
+    below, page_in_branch = plan.shared_mask_tables() if shared else (np.zeros(plan.n_new, np.int32), None)
     # physical page -> (request, logical page)
     where = {}
     for r in range(len(ph.desc["prefix_len"])):
@@ -111,7 +113,8 @@ def _check_cover(wl, ph, plan, chunk=0, dealt=False):
                 assert r == it["request"]
                 for row in range(int(n_valid[e])):
                     kg = int(it["key0"]) + pg * ps + row
-                    if kg < pe[tok] or lo[tok] <= kg < hi[tok]:
+                    other = shared and page_in_branch[e] * ps + row < below[tok]     # shared mask: smaller offset, any branch
+                    if kg < pe[tok] or lo[tok] <= kg < hi[tok] or other:
                         count[tok, int(it["kv_head"]), lp * ps + row] += 1
             slots_seen.setdefault((tok, int(it["kv_head"])), []).append(int(it["part_slot"]))
     for h in range(wl.Hkv):
@@ -135,6 +138,24 @@ def test_work_list_covers_every_visible_key_exactly_once(chunk, n_ctas):
             plan = B.Plan(_shape(wl), ph.desc, wl.n_pool_pages, ph.mode, chunk_tokens=chunk, n_ctas=n_ctas, host_only=True)
             _check_cover(wl, ph, plan, chunk=chunk)
             plan.destroy()
+
+
+def test_shared_mask_plans_cover_the_oracles_visible_sets():
+    """The visible mask of the ablation: the library's visible sets and the plans' work lists equal
+    the oracle's, bit for bit; such plans neither fuse the append nor deal whole streams."""
+    for wl in small_workloads():
+        for ph in wl.phases:
+            n_slots = int(ph.desc["n_pages"].max()) * wl.page_size
+            np.testing.assert_array_equal(B.visible_slots(ph.desc, ph.mode, n_slots, mask=B.MASK_SHARED),
+                                          oracle.visible_slots(ph.desc, ph.mode, n_slots, mask=oracle.MASK_SHARED))
+            for chunk, n_ctas in ((0, 0), (32, 3), (0, 2)):
+                plan = B.Plan(_shape(wl), ph.desc, wl.n_pool_pages, ph.mode, chunk_tokens=chunk, n_ctas=n_ctas, host_only=True,
+                              mask=B.MASK_SHARED)
+                if ph.mode == B.MODE_BRANCH:
+                    assert not plan.info.fused_append and not plan.info.direct_output
+                _check_cover(wl, ph, plan, chunk=chunk, mask=oracle.MASK_SHARED)
+                plan.destroy()
+    assert _plan_rc(W.config_tiny(), W.config_tiny().phases[-1].desc, W.config_tiny().phases[-1].mode, mask=7) == -1     # ASPD_ERR_INVALID_ARG
 
 
 @pytest.mark.parametrize("kernel", [B.KERNEL_MMA, B.KERNEL_GENERIC])

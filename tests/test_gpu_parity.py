@@ -36,7 +36,7 @@ def check(gpu, ref, dtype, what=""):
 
 
 def compare_workload(wl, **kw):
-    ref = oracle_run(wl)
+    ref = oracle_run(wl, kw.get("mask", 0))            # ASPD_MASK_* and the oracle's MASK_* are the same numbers
     run = engine().run_workload(wl, **kw)
     assert len(run.outputs) == len(ref.outputs) and len(ref.outputs) > 0
     for n, (g, r) in enumerate(zip(run.outputs, ref.outputs)):
@@ -199,8 +199,9 @@ def _probe(wl, r_digit, n_digits):
     return wl
 
 
+@pytest.mark.parametrize("mask", [B.MASK_BRANCH_INVISIBLE, B.MASK_SHARED])
 @pytest.mark.parametrize("kernel", KERNELS)
-def test_mask_membership_through_the_kernels_is_exact(kernel):
+def test_mask_membership_through_the_kernels_is_exact(kernel, mask):
     """With all keys zero every visible key weighs exactly 1/n; with one-hot V rows the output
     column c is (number of visible keys whose slot digit is c) / n.  The counts recovered from
     the kernels' output equal the oracle's visible sets as integers (fp32), and the zero
@@ -211,14 +212,14 @@ def test_mask_membership_through_the_kernels_is_exact(kernel):
             wl = W.build_segment_workload("probe", 55, Hq, Hkv, d, dtype, 1e4, [70, 9], [[14, 15, 16], [200]],
                                           [[2, 1, 3], [1]], serial_steps=1)
             wl = _probe(wl, r_digit, d)
-            run = E.run_workload(wl, kernel=kernel)
+            run = E.run_workload(wl, kernel=kernel, mask=mask)
             outs = iter(run.outputs)
             for ph in wl.phases:
                 if not ph.compare:
                     continue
                 out = next(outs)
                 n_slots = int(ph.desc["n_pages"].max()) * wl.page_size
-                vis = oracle.visible_slots(ph.desc, ph.mode, n_slots)
+                vis = oracle.visible_slots(ph.desc, ph.mode, n_slots, mask=mask)
                 for t in range(vis.shape[0]):
                     slots = np.flatnonzero(vis[t])
                     digit = (slots >> (r_digit * int(np.log2(d)))) & (d - 1)
@@ -510,6 +511,27 @@ def test_same_re_serial_decoding_after_rerotation():
     for i in serial:                        # the serial position P + sum(len) is already sequential
         got, want = run.step(wl.phases[i]), ref.step(wl.phases[i])
         check(got, want, wl.dtype, "same-re serial step")
+
+
+@pytest.mark.parametrize("fused", [False, True])
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_shared_mask_variant(kernel, fused):
+    """The visible mask of the paper's attention-mask ablation (a token at offset k also sees the
+    first k tokens of the other branches of its stage): decode steps over branches of different
+    lengths, one of which decodes nothing; a second parallel stage; whole branches in one step;
+    split-K cuts inside other branches' regions.  The result differs from the paper's mask."""
+    assert oracle.MASK_SHARED == B.MASK_SHARED
+    decode = W.build_segment_workload("sh", 43, 28, 4, 128, "bf16", 1e6, [300, 40], [[20, 9, 131, 4], [5, 40]],
+                                      [[1, 1, 1, 0], [1, 1]], serial_steps=1)
+    two = W.build_two_stage_workload("sh2", 44, 28, 4, 128, "bf16", 1e6, 90, [30, 1, 17], 3, [5, 0, 40], [1, 2, 1], serial_steps=1)
+    whole = W.build_segment_workload("sh3", 45, 28, 4, 128, "bf16", 1e6, [100], [[0, 17, 5]], [[40, 25, 31]])
+    for wl in (decode, two, whole):
+        run, ref = compare_workload(wl, kernel=kernel, fused=fused, mask=B.MASK_SHARED)
+        iso = oracle_run(wl)
+        assert max(np.abs(a - b).max() for a, b in zip(ref.outputs, iso.outputs)) > 1e-2
+    compare_workload(decode, kernel=kernel, fused=fused, mask=B.MASK_SHARED, chunk_tokens=32, n_ctas=5)
+    small = W.config_tiny()
+    compare_workload(small, kernel=B.KERNEL_GENERIC, fused=fused, mask=B.MASK_SHARED)
 
 
 def test_zero_new_tokens_is_a_no_op():
