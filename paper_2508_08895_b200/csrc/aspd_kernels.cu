@@ -27,35 +27,64 @@ template <> __device__ inline float from_f32<float>(float x) { return x; }
 template <> __device__ inline __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
 
 // ------------------------------------------------------------------------------- append
-// One block per (new token, KV head); thread i rotates the pair (i, i + d/2).
+// A thread owns one 16-byte chunk of the first half of a new token's rows and its partner chunk
+// in the second half (the pairs (i, i + d/2)): it computes the chunk's sines and cosines once and
+// rotates that chunk pair of K, and copies that chunk pair of V, for every KV head of the token.
+constexpr int kAppendThreads = 128;
 template <typename T>
-__global__ void append_kernel(const T* __restrict__ k_new, const T* __restrict__ v_new, const int32_t* __restrict__ pos,
-                              const int32_t* __restrict__ tok_page, const int32_t* __restrict__ tok_row,
-                              const double* __restrict__ inv_freq, T* __restrict__ k_pool, T* __restrict__ v_pool,
-                              int n_kv_heads, int head_dim, int page_size) {
+__global__ void __launch_bounds__(kAppendThreads)
+append_kernel(const T* __restrict__ k_new, const T* __restrict__ v_new, const int32_t* __restrict__ pos,
+              const int32_t* __restrict__ tok_page, const int32_t* __restrict__ tok_row,
+              const double* __restrict__ inv_freq, T* __restrict__ k_pool, T* __restrict__ v_pool,
+              int n_new, int n_kv_heads, int head_dim, int page_size) {
+  constexpr int VEC = 16 / sizeof(T);
   pdl_launch_dependents();
+  const int half = head_dim / 2, chunks = half / VEC;
+  const long gid = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long t = gid / chunks;
+  const int c = (int)(gid % chunks);
+  double f[VEC];                                   // plan data: may be read before the dependency wait
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) f[j] = inv_freq[c * VEC + j];
   pdl_wait();
-  const int t = blockIdx.x / n_kv_heads, h = blockIdx.x % n_kv_heads, i = threadIdx.x, half = head_dim / 2;
-  if (i >= half) return;
+  if (t >= n_new) return;
   // angle reduced to [-pi, pi] in fp64, then fp32 sincos: the error stays near 1e-7 rad
   // however large the position is
-  double a = (double)pos[t] * inv_freq[i];
-  a -= rint(a * 0.15915494309189535) * 6.283185307179586;
-  float sn, cs;
-  sincosf((float)a, &sn, &cs);
-  const size_t src = ((size_t)t * n_kv_heads + h) * head_dim;
-  const float x0 = to_f32(k_new[src + i]), x1 = to_f32(k_new[src + i + half]);
-  const float y0 = x0 * cs - x1 * sn, y1 = x1 * cs + x0 * sn;
-  const size_t tile = ((size_t)tok_page[t] * n_kv_heads + h) * tile_bytes(page_size, head_dim, sizeof(T));
-  const int row = tok_row[t];
+  float sn[VEC], cs[VEC];
+  const double p = (double)pos[t];
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) {
+    double a = p * f[j];
+    a -= rint(a * 0.15915494309189535) * 6.283185307179586;
+    sincosf((float)a, &sn[j], &cs[j]);
+  }
   const uint32_t rb = head_dim * sizeof(T);
-  const uint32_t o0 = tile_offset(row, i * sizeof(T), rb), o1 = tile_offset(row, (i + half) * sizeof(T), rb);
-  char* kp = reinterpret_cast<char*>(k_pool) + tile;
-  char* vp = reinterpret_cast<char*>(v_pool) + tile;
-  *reinterpret_cast<T*>(kp + o0) = from_f32<T>(y0);
-  *reinterpret_cast<T*>(kp + o1) = from_f32<T>(y1);
-  *reinterpret_cast<T*>(vp + o0) = v_new[src + i];
-  *reinterpret_cast<T*>(vp + o1) = v_new[src + i + half];
+  const size_t tb = tile_bytes(page_size, head_dim, sizeof(T));
+  const size_t tile0 = (size_t)tok_page[t] * n_kv_heads * tb;
+  const int row = tok_row[t];
+  const uint32_t o0 = tile_offset(row, c * 16, rb), o1 = tile_offset(row, half * sizeof(T) + c * 16, rb);
+#pragma unroll 4
+  for (int h = 0; h < n_kv_heads; ++h) {
+    const size_t src = ((size_t)t * n_kv_heads + h) * head_dim;
+    uint4 u0 = *reinterpret_cast<const uint4*>(k_new + src + c * VEC);
+    uint4 u1 = *reinterpret_cast<const uint4*>(k_new + src + half + c * VEC);
+    const uint4 w0 = *reinterpret_cast<const uint4*>(v_new + src + c * VEC);
+    const uint4 w1 = *reinterpret_cast<const uint4*>(v_new + src + half + c * VEC);
+    T* x0 = reinterpret_cast<T*>(&u0);
+    T* x1 = reinterpret_cast<T*>(&u1);
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+      const float a = to_f32(x0[j]), b = to_f32(x1[j]);
+      x0[j] = from_f32<T>(a * cs[j] - b * sn[j]);
+      x1[j] = from_f32<T>(b * cs[j] + a * sn[j]);
+    }
+    char* kp = reinterpret_cast<char*>(k_pool) + tile0 + h * tb;
+    char* vp = reinterpret_cast<char*>(v_pool) + tile0 + h * tb;
+    *reinterpret_cast<uint4*>(kp + o0) = u0;
+    *reinterpret_cast<uint4*>(kp + o1) = u1;
+    *reinterpret_cast<uint4*>(vp + o0) = w0;
+    *reinterpret_cast<uint4*>(vp + o1) = w1;
+  }
 }
 
 // --------------------------------------------------------------------------- re-rotation
@@ -281,14 +310,15 @@ inline int status_of(cudaError_t e) { return e == cudaSuccess ? ASPD_OK : ASPD_E
 int launch_append(const aspd_plan* p, const void* k_new, const void* v_new, const int32_t* pos, void* k_pool,
                   void* v_pool, cudaStream_t s) {
   const aspd_shape_t& sh = p->shape;
-  const dim3 grid(p->n_new * sh.n_kv_heads), block(sh.head_dim / 2);
+  const int chunks = sh.head_dim / 2 / (16 / esize_of(sh.dtype));
+  const dim3 grid((unsigned)(((long)p->n_new * chunks + kAppendThreads - 1) / kAppendThreads)), block(kAppendThreads);
   if (sh.dtype == ASPD_DTYPE_BF16)
     return status_of(launch_pdl(kPdlAppend, append_kernel<__nv_bfloat16>, grid, block, 0, s, (const __nv_bfloat16*)k_new,
                                 (const __nv_bfloat16*)v_new, pos, p->dev.tok_page, p->dev.tok_row, p->dev.inv_freq,
-                                (__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool, sh.n_kv_heads, sh.head_dim, sh.page_size));
+                                (__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool, p->n_new, sh.n_kv_heads, sh.head_dim, sh.page_size));
   return status_of(launch_pdl(kPdlAppend, append_kernel<float>, grid, block, 0, s, (const float*)k_new, (const float*)v_new, pos,
-                              p->dev.tok_page, p->dev.tok_row, p->dev.inv_freq, (float*)k_pool, (float*)v_pool, sh.n_kv_heads,
-                              sh.head_dim, sh.page_size));
+                              p->dev.tok_page, p->dev.tok_row, p->dev.inv_freq, (float*)k_pool, (float*)v_pool, p->n_new,
+                              sh.n_kv_heads, sh.head_dim, sh.page_size));
 }
 
 int launch_attn_generic(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, cudaStream_t s) {

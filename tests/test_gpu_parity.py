@@ -103,6 +103,20 @@ def test_config5_serving_mix_full_size(kernel):
     assert singles
 
 
+def test_masked_prefill_full_size():
+    """The masked-prefill workload of the benchmark (the serving mix in teacher-forcing layout,
+    17 069 query tokens) at full size, in the launch configuration the benchmark times: dealt
+    streams, wide row blocks, output written by the attention kernel (fused step call)."""
+    wl = W.config_masked_prefill()
+    ph = wl.phases[-1]
+    shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
+    plan = B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode, host_only=True)
+    assert plan.info.direct_output and plan.info.max_rows_per_item == 128 and plan.info.n_ctas == 148
+    plan.destroy()
+    run, ref = compare_workload(wl, fused=True, stable_cache=True)
+    assert run.outputs[0].shape[0] == 17069
+
+
 def test_peaked_softmax_variant():
     """sm_scale x 4: logits ~ N(0, 16), outputs are O(1), so the bounds bite.  The cached keys,
     the rotated query and the softmax weights fed to the tensor cores are bf16 (relative
