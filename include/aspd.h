@@ -24,8 +24,9 @@
  *     the library -- read tokens back with aspd_debug_read_token.  Pools must be zero-filled
  *     (or at least hold no NaN/Inf bit patterns) before their first use: the rows of a partly
  *     filled page that no token has been written to yet are multiplied by a weight of exactly 0.
- *     Device buffers (q, out, k_new, v_new, the pools) must start on a 16-byte boundary; the
- *     kernels move them in 16-byte pieces.
+ *     Device buffers (q, out, k_new, v_new, the pools) must start on a 16-byte boundary (the
+ *     kernels move them in 16-byte pieces); a call given one that does not returns
+ *     ASPD_ERR_INVALID_ARG and launches nothing.
  *   - Positions are 0-based.  Query head h uses KV head h / (n_q_heads / n_kv_heads).
  *     RoPE pairs element i with i + head_dim/2 and uses inv_freq[i] = theta^(-2i/head_dim)
  *     (the paper leaves the encoding open; this is the rotate-half convention of the

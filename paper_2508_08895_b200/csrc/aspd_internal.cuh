@@ -141,4 +141,10 @@ int launch_wait_probe(long long limit_cycles, int32_t* status_dev, cudaStream_t 
 int launch_read_token(const aspd_shape_t* shape, const void* pool, int64_t page, int row, int kv_head,
                       float* out_dev, cudaStream_t s);
 inline int esize_of(int dtype) { return dtype == ASPD_DTYPE_BF16 ? 2 : 4; }
+// device buffers are moved in 16-byte pieces: a pointer off that boundary is refused, not dereferenced
+inline bool misaligned16(const void* a, const void* b = nullptr, const void* c = nullptr, const void* d = nullptr,
+                         const void* e = nullptr, const void* f = nullptr) {
+  return ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b) | reinterpret_cast<uintptr_t>(c) |
+           reinterpret_cast<uintptr_t>(d) | reinterpret_cast<uintptr_t>(e) | reinterpret_cast<uintptr_t>(f)) & 15u) != 0;
+}
 }  // namespace aspd

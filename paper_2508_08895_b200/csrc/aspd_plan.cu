@@ -659,14 +659,14 @@ int aspd_kv_append(aspd_plan_t* p, const void* k_new, const void* v_new, const i
                    void* v_pool, void* stream) {
   if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
   if (p->n_new == 0) return ASPD_OK;
-  if (!k_new || !v_new || !pos || !k_pool || !v_pool) return ASPD_ERR_INVALID_ARG;
+  if (!k_new || !v_new || !pos || !k_pool || !v_pool || misaligned16(k_new, v_new, k_pool, v_pool)) return ASPD_ERR_INVALID_ARG;
   return launch_append(p, k_new, v_new, pos, k_pool, v_pool, (cudaStream_t)stream);
 }
 
 int aspd_attn_partials(aspd_plan_t* p, const void* q, const void* k_pool, const void* v_pool, void* stream) {
   if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
   if (p->n_new == 0) return ASPD_OK;
-  if (!q || !k_pool || !v_pool) return ASPD_ERR_INVALID_ARG;
+  if (!q || !k_pool || !v_pool || misaligned16(q, k_pool, v_pool)) return ASPD_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   return p->kernel == ASPD_KERNEL_MMA ? launch_attn_mma(p, q, k_pool, v_pool, nullptr, s)
                                       : launch_attn_generic(p, q, k_pool, v_pool, s);
@@ -675,7 +675,7 @@ int aspd_attn_partials(aspd_plan_t* p, const void* q, const void* k_pool, const 
 int aspd_attn_combine(aspd_plan_t* p, void* out, void* stream) {
   if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
   if (p->n_new == 0) return ASPD_OK;
-  if (!out) return ASPD_ERR_INVALID_ARG;
+  if (!out || misaligned16(out)) return ASPD_ERR_INVALID_ARG;
   return launch_combine(p, out, (cudaStream_t)stream);
 }
 
@@ -683,7 +683,7 @@ static int run_attn(aspd_plan_t* p, int mode, const void* q, const void* k_pool,
                     void* stream) {
   if (!p || p->host_only || p->mode != mode) return ASPD_ERR_INVALID_ARG;
   if (p->n_new == 0) return ASPD_OK;
-  if (!q || !k_pool || !v_pool || !out) return ASPD_ERR_INVALID_ARG;
+  if (!q || !k_pool || !v_pool || !out || misaligned16(q, k_pool, v_pool, out)) return ASPD_ERR_INVALID_ARG;
   // a plan with one item per (token, KV head) needs no records: the kernel normalises and writes the output
   if (attn_mma_writes_output(p)) return launch_attn_mma(p, q, k_pool, v_pool, out, (cudaStream_t)stream);
   int rc = aspd_attn_partials(p, q, k_pool, v_pool, stream);
@@ -703,7 +703,7 @@ static int run_step(aspd_plan_t* p, int mode, const void* q, const void* k_new, 
                     void* v_pool, void* out, void* stream) {
   if (!p || p->host_only || p->mode != mode) return ASPD_ERR_INVALID_ARG;
   if (p->n_new == 0) return ASPD_OK;
-  if (!q || !k_new || !v_new || !k_pool || !v_pool || !out) return ASPD_ERR_INVALID_ARG;
+  if (!q || !k_new || !v_new || !k_pool || !v_pool || !out || misaligned16(q, k_new, v_new, k_pool, v_pool, out)) return ASPD_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   int rc;
   if (p->kernel == ASPD_KERNEL_MMA && p->fuse_append) {
@@ -733,7 +733,7 @@ int aspd_step_host(aspd_plan_t* p, const void* q, const void* k_new, const void*
                    void* k_pool, void* v_pool, void* out, void* stream) {
   if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
   if (p->n_new == 0) return ASPD_OK;
-  if (!q || !k_new || !v_new || !pos || !k_pool || !v_pool || !out) return ASPD_ERR_INVALID_ARG;
+  if (!q || !k_new || !v_new || !pos || !k_pool || !v_pool || !out || misaligned16(k_pool, v_pool)) return ASPD_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   const aspd_shape_t& sh = p->shape;
   const size_t es = esize_of(sh.dtype);
@@ -758,7 +758,7 @@ int aspd_k_rerotate(const aspd_shape_t* shape, void* k_pool, const int32_t* page
   if (rc) return rc;
   if (n < 0) return ASPD_ERR_INVALID_ARG;
   if (n == 0) return ASPD_OK;
-  if (!k_pool || !pages || !rows || !delta) return ASPD_ERR_INVALID_ARG;
+  if (!k_pool || !pages || !rows || !delta || misaligned16(k_pool)) return ASPD_ERR_INVALID_ARG;
   return launch_rerotate(shape, k_pool, pages, rows, delta, n, (cudaStream_t)stream);
 }
 

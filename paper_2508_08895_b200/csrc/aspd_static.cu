@@ -38,7 +38,7 @@ extern "C" int aspd_attn_static(const aspd_plan_t* plan, const void* q, const vo
                                 void* stream) {
   if (!plan || !plan->host_only) return ASPD_ERR_INVALID_ARG;
   if (plan->n_new == 0) return ASPD_OK;
-  if (!q || !k_pool || !v_pool || !out) return ASPD_ERR_INVALID_ARG;
+  if (!q || !k_pool || !v_pool || !out || aspd::misaligned16(q, k_pool, v_pool, out)) return ASPD_ERR_INVALID_ARG;
   const aspd_shape_t& sh = plan->shape;
   const int d = sh.head_dim, G = sh.n_q_heads / sh.n_kv_heads, n_new = plan->n_new;
 

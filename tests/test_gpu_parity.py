@@ -548,6 +548,41 @@ def test_shared_mask_variant(kernel, fused):
     compare_workload(small, kernel=B.KERNEL_GENERIC, fused=fused, mask=B.MASK_SHARED)
 
 
+def test_misaligned_device_buffers_are_refused_before_any_launch():
+    """Buffers are moved in 16-byte pieces; a pointer off that boundary gets ASPD_ERR_INVALID_ARG
+    (no kernel runs, the context stays usable and the next call is correct)."""
+    import torch
+    E = engine()
+    wl = W.build_segment_workload("al", 47, 28, 4, 128, "bf16", 1e6, [40], [[17, 3]], [[1, 1]])
+    run = E.WorkloadRun(wl)
+    for ph in wl.phases[:-1]:
+        run.step(ph)
+    ph = wl.phases[-1]
+    plan = B.Plan(run.shape, ph.desc, wl.n_pool_pages, ph.mode)
+    q, k, v = (E.to_device(x, wl.dtype) for x in (ph.q, ph.k_new, ph.v_new))
+    out = torch.empty_like(q)
+    def off(t):                                   # same values, storage shifted by one element (2 bytes)
+        buf = torch.empty(t.numel() + 8, dtype=t.dtype, device=t.device)
+        view = buf[1:1 + t.numel()].view(t.shape)
+        view.copy_(t)
+        return view
+    calls = [lambda: B.branch_step(plan, off(q), k, v, run.cache.k, run.cache.v, out),
+             lambda: B.branch_step(plan, q, off(k), v, run.cache.k, run.cache.v, out),
+             lambda: B.branch_step(plan, q, k, v, run.cache.k, run.cache.v, off(out)),
+             lambda: B.branch_attn(plan, off(q), run.cache.k, run.cache.v, out),
+             lambda: B.attn_partials(plan, off(q), run.cache.k, run.cache.v)]
+    for call in calls:
+        with pytest.raises(B.AspdError) as e:
+            call()
+        assert e.value.status == -1
+    B.branch_step(plan, q, k, v, run.cache.k, run.cache.v, out)
+    torch.cuda.synchronize()
+    assert plan.status() == 0
+    ref = oracle_run(wl)
+    check(E.to_host_f32(out), ref.outputs[0], wl.dtype, "after refused calls")
+    plan.destroy()
+
+
 def test_zero_new_tokens_is_a_no_op():
     E = engine()
     wl = W.build_segment_workload("e", 8, 28, 4, 128, "bf16", 1e6, [20], [[5, 9]], [[1, 1]])
