@@ -106,8 +106,9 @@ namespace aspd {
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-enum { kPdlAppend = 1, kPdlAttn = 2, kPdlCombine = 4 };
-int pdl_mask();   // which kernels are launched with the attribute (environment ASPD_PDL; default append + attention)
+enum { kPdlAppend = 1, kPdlAttn = 2, kPdlCombine = 4, kPdlCombineLarge = 8 };
+int pdl_mask();   // which kernels are launched with the attribute (environment ASPD_PDL: bits 1 append, 2 attention,
+                  // 4 combine; default: append, attention, and the combine of large steps)
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(int which, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,

@@ -10,7 +10,7 @@ int pdl_mask() {
   static int mask = -1;
   if (mask < 0) {
     const char* e = getenv("ASPD_PDL");
-    mask = e ? atoi(e) & 7 : (kPdlAppend | kPdlAttn);   // measured: the combine does better as a plain launch
+    mask = e ? atoi(e) & 7 : (kPdlAppend | kPdlAttn | kPdlCombineLarge);   // the combine only on large steps (see launch_combine)
   }
   return mask;
 }
@@ -27,9 +27,9 @@ template <> __device__ inline float from_f32<float>(float x) { return x; }
 template <> __device__ inline __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
 
 // ------------------------------------------------------------------------------- append
-// A thread owns one 16-byte chunk of the first half of a new token's rows and its partner chunk
-// in the second half (the pairs (i, i + d/2)): it computes the chunk's sines and cosines once and
-// rotates that chunk pair of K, and copies that chunk pair of V, for every KV head of the token.
+// A thread owns one 16-byte chunk of the first half of a (new token, KV head) row and its partner
+// chunk in the second half (the pairs (i, i + d/2)): it rotates that chunk pair of K and copies
+// that chunk pair of V.
 constexpr int kAppendThreads = 128;
 template <typename T>
 __global__ void __launch_bounds__(kAppendThreads)
@@ -41,8 +41,8 @@ append_kernel(const T* __restrict__ k_new, const T* __restrict__ v_new, const in
   pdl_launch_dependents();
   const int half = head_dim / 2, chunks = half / VEC;
   const long gid = (long)blockIdx.x * blockDim.x + threadIdx.x;
-  const long t = gid / chunks;
-  const int c = (int)(gid % chunks);
+  const long t = gid / (chunks * n_kv_heads);
+  const int h = (int)(gid / chunks % n_kv_heads), c = (int)(gid % chunks);
   double f[VEC];                                   // plan data: may be read before the dependency wait
 #pragma unroll
   for (int j = 0; j < VEC; ++j) f[j] = inv_freq[c * VEC + j];
@@ -63,8 +63,7 @@ append_kernel(const T* __restrict__ k_new, const T* __restrict__ v_new, const in
   const size_t tile0 = (size_t)tok_page[t] * n_kv_heads * tb;
   const int row = tok_row[t];
   const uint32_t o0 = tile_offset(row, c * 16, rb), o1 = tile_offset(row, half * sizeof(T) + c * 16, rb);
-#pragma unroll 4
-  for (int h = 0; h < n_kv_heads; ++h) {
+  {
     const size_t src = ((size_t)t * n_kv_heads + h) * head_dim;
     uint4 u0 = *reinterpret_cast<const uint4*>(k_new + src + c * VEC);
     uint4 u1 = *reinterpret_cast<const uint4*>(k_new + src + half + c * VEC);
@@ -311,7 +310,7 @@ int launch_append(const aspd_plan* p, const void* k_new, const void* v_new, cons
                   void* v_pool, cudaStream_t s) {
   const aspd_shape_t& sh = p->shape;
   const int chunks = sh.head_dim / 2 / (16 / esize_of(sh.dtype));
-  const dim3 grid((unsigned)(((long)p->n_new * chunks + kAppendThreads - 1) / kAppendThreads)), block(kAppendThreads);
+  const dim3 grid((unsigned)(((long)p->n_new * sh.n_kv_heads * chunks + kAppendThreads - 1) / kAppendThreads)), block(kAppendThreads);
   if (sh.dtype == ASPD_DTYPE_BF16)
     return status_of(launch_pdl(kPdlAppend, append_kernel<__nv_bfloat16>, grid, block, 0, s, (const __nv_bfloat16*)k_new,
                                 (const __nv_bfloat16*)v_new, pos, p->dev.tok_page, p->dev.tok_row, p->dev.inv_freq,
@@ -340,8 +339,13 @@ int launch_combine(const aspd_plan* p, void* out, cudaStream_t s) {
   const aspd_shape_t& sh = p->shape;
   const int warps = p->n_new * sh.n_q_heads;
   const dim3 block(128), grid((warps + 3) / 4);
+  // Measured: with the attribute the combine's blocks wait on the SMs while the attention pass
+  // ends, which wins a little on a large step (serving mix: 48.6 against 49.2 us per layer) and
+  // loses a lot on small ones (long context, one request: 24.9 against 17.6), so it follows the
+  // step's size unless the environment decides.
+  const int which = p->algorithmic_bytes >= (128LL << 20) ? (kPdlCombine | kPdlCombineLarge) : kPdlCombine;
 #define ASPD_CMB(T, D) \
-  return status_of(launch_pdl(kPdlCombine, combine_kernel<T, D>, grid, block, 0, s, p->dev, (T*)out, p->n_new, sh.n_q_heads, sh.n_kv_heads))
+  return status_of(launch_pdl(which, combine_kernel<T, D>, grid, block, 0, s, p->dev, (T*)out, p->n_new, sh.n_q_heads, sh.n_kv_heads))
   if (sh.dtype == ASPD_DTYPE_BF16 && sh.head_dim == 128) ASPD_CMB(__nv_bfloat16, 128);
   else if (sh.dtype == ASPD_DTYPE_BF16) ASPD_CMB(__nv_bfloat16, 64);
   else if (sh.head_dim == 128) ASPD_CMB(float, 128);
