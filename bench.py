@@ -396,9 +396,19 @@ def run_ours(args):
     pos_h = torch.from_numpy(pos.copy()).pin_memory()
     out_h = [torch.empty_like(q_h).pin_memory() for _ in range(L)]
 
+    # The layers rotate over a few plans (each owns its staging memory), each on a stream of its
+    # own, so that the host copies of one layer overlap the kernels of others; one
+    # synchronisation per step, after which every layer's output is in host memory.
+    n_e = max(1, args.e2e_streams)
+    e_plans = [plan] + [B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode, kernel=kernel, chunk_tokens=args.chunk, n_ctas=args.ctas)
+                        for _ in range(n_e - 1)]
+    e_streams = [torch.cuda.Stream() for _ in range(n_e)]
+
     def step_e2e():
         for l in range(L):
-            B.step_host(plan, q_h, k_h, v_h, pos_h, caches[l].k, caches[l].v, out_h[l])
+            B.step_host_async(e_plans[l % n_e], q_h, k_h, v_h, pos_h, caches[l].k, caches[l].v, out_h[l], stream=e_streams[l % n_e])
+        for st in e_streams:
+            st.synchronize()
 
     for _ in range(2):
         step_e2e()
@@ -454,7 +464,9 @@ def run_ours(args):
                          "kernel_us": kernel_ms * 1e3, "algorithmic_bytes_per_launch": alg},
             "e2e": {"value": total_new * L * e_steps / (e2e_ms * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": int(L * (n_new * es * wl.d * (wl.Hq + 2 * wl.Hkv) + 4 * n_new)),
-                    "d2h_bytes_per_step": int(L * n_new * es * wl.d * wl.Hq), "ms_per_step": e2e_ms / e_steps},
+                    "d2h_bytes_per_step": int(L * n_new * es * wl.d * wl.Hq), "ms_per_step": e2e_ms / e_steps,
+                    "calls": "aspd_step_host_async per layer, layers rotating over %d plans on %d streams, "
+                             "one synchronisation per step" % (n_e, n_e)},
             "gpu_launches": (2 if (fused and info.fused_append) or info.direct_output else 3) * L * args.steps,
             "clocks": clocks,
         }
@@ -466,7 +478,8 @@ def run_ours(args):
                                     "sample": f"{reps_o} repetitions of one layer-step of the same batch "
                                               f"({n_o} query tokens), {sec:.3f} s each"}
         print(json.dumps(line))
-    plan.destroy()
+    for pl in e_plans:
+        pl.destroy()
     if world > 1:
         dist.destroy_process_group()
     return 0
@@ -491,6 +504,7 @@ def main():
     ap.add_argument("--separate-append", action="store_true",
                     help="call aspd_kv_append and aspd_branch_attn separately instead of aspd_branch_step")
     ap.add_argument("--no-stable-cache", action="store_true", help="create the plan without the stable-cache promise")
+    ap.add_argument("--e2e-streams", type=int, default=4, help="plans/streams the layers rotate over in the end-to-end leg")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -290,6 +290,18 @@ int aspd_step_host(aspd_plan_t* plan, const void* q /*host*/, const void* k_new 
                    void* v_pool /*device*/, void* out /*host*/, void* stream);
 
 /*
+ * The same without the final synchronisation: everything is enqueued on `stream` and the call
+ * returns.  The host buffers must be page-locked and stay valid (out: unread) until the stream
+ * has passed the call.  The staging memory belongs to the plan, so calls with the same plan are
+ * ordered by using one stream for them; to overlap the copies of one call with the kernels of
+ * another, give the calls different plans and different streams (e.g. the layers of a model
+ * alternating between two plans of the same step).
+ */
+int aspd_step_host_async(aspd_plan_t* plan, const void* q /*host*/, const void* k_new /*host*/,
+                   const void* v_new /*host*/, const int32_t* pos /*host*/, void* k_pool /*device*/,
+                   void* v_pool /*device*/, void* out /*host*/, void* stream);
+
+/*
  * Attention of a step for callers that must not allocate device memory (the paper has no
  * counterpart; this is a convenience of the library).
  *

@@ -60,7 +60,7 @@ EXPORTS = ("aspd_strerror", "aspd_pool_bytes", "aspd_count_new_tokens", "aspd_po
            "aspd_visible_slots_masked", "aspd_plan_create", "aspd_plan_destroy", "aspd_plan_info", "aspd_plan_items", "aspd_plan_cta_ranges", "aspd_plan_stream_pages",
            "aspd_plan_token_ranges", "aspd_plan_shared_mask_tables", "aspd_plan_status",
            "aspd_kv_append", "aspd_branch_attn", "aspd_serial_attn", "aspd_attn_partials", "aspd_attn_combine",
-           "aspd_branch_step", "aspd_serial_step", "aspd_step_host", "aspd_attn_static", "aspd_k_rerotate", "aspd_debug_read_token", "aspd_debug_bounded_wait")
+           "aspd_branch_step", "aspd_serial_step", "aspd_step_host", "aspd_step_host_async", "aspd_attn_static", "aspd_k_rerotate", "aspd_debug_read_token", "aspd_debug_bounded_wait")
 
 _lib = None
 
@@ -102,6 +102,7 @@ def lib() -> ctypes.CDLL:
         L.aspd_branch_step.argtypes = [vp] * 8
         L.aspd_serial_step.argtypes = [vp] * 8
         L.aspd_step_host.argtypes = [vp] * 9
+        L.aspd_step_host_async.argtypes = [vp] * 9
         L.aspd_attn_static.argtypes = [vp] * 6
         L.aspd_k_rerotate.argtypes = [vp, vp, vp, vp, vp, ci, vp]
         L.aspd_debug_bounded_wait.argtypes = [ctypes.c_int64, vp, vp]
@@ -302,6 +303,12 @@ def step_host(plan: Plan, q, k_new, v_new, pos, k_pool, v_pool, out, stream=None
     """Whole step from host (numpy / pinned torch CPU) buffers; ``out`` is a host buffer."""
     _check(lib().aspd_step_host(plan._h, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(pos), _ptr(k_pool), _ptr(v_pool),
                                 _ptr(out), _stream(stream)), "aspd_step_host")
+
+
+def step_host_async(plan: Plan, q, k_new, v_new, pos, k_pool, v_pool, out, stream=None) -> None:
+    """``step_host`` without the final synchronisation (pinned host buffers; see ``aspd_step_host_async``)."""
+    _check(lib().aspd_step_host_async(plan._h, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(pos), _ptr(k_pool), _ptr(v_pool),
+                                      _ptr(out), _stream(stream)), "aspd_step_host_async")
 
 
 def k_rerotate(shape: Shape, k_pool, pages, rows, delta, stream=None) -> None:

@@ -729,8 +729,8 @@ int aspd_serial_step(aspd_plan_t* p, const void* q, const void* k_new, const voi
   return run_step(p, ASPD_MODE_SERIAL, q, k_new, v_new, k_pool, v_pool, out, stream);
 }
 
-int aspd_step_host(aspd_plan_t* p, const void* q, const void* k_new, const void* v_new, const int32_t* pos,
-                   void* k_pool, void* v_pool, void* out, void* stream) {
+int aspd_step_host_async(aspd_plan_t* p, const void* q, const void* k_new, const void* v_new, const int32_t* pos,
+                         void* k_pool, void* v_pool, void* out, void* stream) {
   if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
   if (p->n_new == 0) return ASPD_OK;
   if (!q || !k_new || !v_new || !pos || !k_pool || !v_pool || !out || misaligned16(k_pool, v_pool)) return ASPD_ERR_INVALID_ARG;
@@ -748,7 +748,14 @@ int aspd_step_host(aspd_plan_t* p, const void* q, const void* k_new, const void*
   rc = run_attn(p, p->mode, p->dev.st_q, k_pool, v_pool, p->dev.st_out, stream);
   if (rc) return rc;
   if (cudaMemcpyAsync(out, p->dev.st_out, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return ASPD_ERR_CUDA;
-  if (cudaStreamSynchronize(s) != cudaSuccess) return ASPD_ERR_CUDA;
+  return ASPD_OK;
+}
+
+int aspd_step_host(aspd_plan_t* p, const void* q, const void* k_new, const void* v_new, const int32_t* pos,
+                   void* k_pool, void* v_pool, void* out, void* stream) {
+  const int rc = aspd_step_host_async(p, q, k_new, v_new, pos, k_pool, v_pool, out, stream);
+  if (rc) return rc;
+  if (p->n_new > 0 && cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return ASPD_ERR_CUDA;
   return ASPD_OK;
 }
 

@@ -287,6 +287,20 @@ def test_step_host_matches_device_path():
     dev = run.step(ph)
     np.testing.assert_array_equal(host, dev)
     check(host, oracle_run(wl).outputs[0], wl.dtype)
+    # the asynchronous form: two plans on two streams (as two layers of a model would), one wait at the end
+    plan_b = B.Plan(run.shape, ph.desc, wl.n_pool_pages, ph.mode)
+    outs = [torch.zeros_like(q).pin_memory() for _ in range(4)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    pos_h = torch.from_numpy(np.ascontiguousarray(pos)).pin_memory()
+    torch.cuda.synchronize()
+    for i, o in enumerate(outs):
+        B.step_host_async((plan, plan_b)[i & 1], q, k, v, pos_h, run.cache.k, run.cache.v, o, stream=streams[i & 1])
+    for st in streams:
+        st.synchronize()
+    for o in outs:
+        np.testing.assert_array_equal(o.float().numpy(), dev)
+    assert plan.status() == 0 and plan_b.status() == 0
+    plan.destroy(); plan_b.destroy()
 
 
 def test_bounded_wait_gives_up_and_leaves_the_context_usable():
