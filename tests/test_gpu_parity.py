@@ -454,6 +454,24 @@ def test_wide_row_blocks_mixed_sizes_and_raised_maxima():
     assert np.linalg.norm(g - r) / np.linalg.norm(r) <= 1e-2
 
 
+def test_large_decode_batch_takes_the_dealt_plan():
+    """A decode step with many more (request, KV head) streams than CTAs: whole streams are dealt
+    out, the append is still fused into the attention launch (few new rows per CTA), the kernel
+    writes the output itself, and every item has at most 3 x 7 rows (the narrow softmax layouts
+    inside the wide kernel)."""
+    rng = np.random.default_rng(3)
+    prefix = [int(x) for x in rng.integers(20, 400, size=10)]
+    prior = [[int(x) for x in rng.integers(1, 60, size=int(rng.integers(1, 4)))] for _ in prefix]
+    wl = W.build_segment_workload("big", 53, 28, 4, 128, "bf16", 1e6, prefix, prior, [[1] * len(p) for p in prior], serial_steps=1)
+    ph = [x for x in wl.phases if x.mode == W.MODE_BRANCH and x.q is not None][-1]
+    shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
+    plan = B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode, n_ctas=8, host_only=True)
+    assert plan.info.direct_output and plan.info.fused_append and plan.info.n_items == 40
+    plan.destroy()
+    for fused in (True, False):
+        compare_workload(wl, n_ctas=8, fused=fused, stable_cache=fused)
+
+
 def test_wide_row_blocks_with_very_negative_logits():
     """All logits near -130 in log2 units (keys and queries opposite along the slowest rotary pair,
     so the rotation hardly changes them): against the wide variant's initial reference of 0 every
