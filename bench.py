@@ -91,6 +91,8 @@ def build_workload(name: str, rank: int, requests: int = 0):
         return W.config_serving_mix(seed=W.SEED_BASE + 4 + 16 * rank, n_req=requests)
     if name == "masked-prefill":
         return W.config_masked_prefill(seed=W.SEED_BASE + 5 + 16 * rank, n_req=requests or 32)
+    if name == "serving-mix-serial":
+        return W.config_serving_mix_serial(seed=W.SEED_BASE + 4 + 16 * rank, n_req=requests or 32)
     fn = W.CONFIGS[name]
     base = {"tiny-f32": 0, "qwen7b-layer": 1, "branch-open": 2, "long-rag": 3, "serving-mix": 4}[name]
     if name == "branch-open":
@@ -323,6 +325,8 @@ def run_ours(args):
     attn = B.branch_attn if ph.mode == W.MODE_BRANCH else B.serial_attn
     fstep = B.branch_step if ph.mode == W.MODE_BRANCH else B.serial_step
     fused = not args.separate_append
+    step_name, attn_name = ("aspd_branch_step", "aspd_branch_attn") if ph.mode == W.MODE_BRANCH else ("aspd_serial_step", "aspd_serial_attn")
+
     def step():
         for l in range(L):
             if fused:      # the attention pass writes the step's new K/V rows itself: 2 launches per layer
@@ -450,10 +454,10 @@ def run_ours(args):
                        "chunk_tokens": info.chunk_tokens, "work_items": info.n_items, "n_ctas": info.n_ctas,
                        "l2": "footprint %.1f GB of distinct K/V pools per step, far above L2" % (alg * L / 1e9),
                        "layers_agree": bool(same), "cuda_graph": not args.no_graph, "stable_cache": not args.no_stable_cache,
-                       "calls_per_layer": ("aspd_branch_step (append fused into the attention pass) -> combine" if info.fused_append
-                                           else "aspd_branch_step (append kernel -> attention pass writing the output)" if info.direct_output
-                                           else "aspd_branch_step (append kernel -> attention pass -> combine)") if fused
-                       else "aspd_kv_append -> aspd_branch_attn"},
+                       "calls_per_layer": (step_name + (" (append fused into the attention pass) -> combine" if info.fused_append
+                                                       else " (append kernel -> attention pass writing the output)" if info.direct_output
+                                                       else " (append kernel -> attention pass -> combine)")) if fused
+                       else "aspd_kv_append -> " + attn_name},
             "hbm_gbs": alg * L * args.steps / (ms * 1e-3) / 1e9,
             "hbm_frac_of_measured": alg * L * args.steps / (ms * 1e-3) / 1e9 / peak,
             "hbm_frac_of_8000_nominal": alg * L * args.steps / (ms * 1e-3) / 1e9 / 8000.0,
@@ -491,7 +495,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="serving-mix", choices=["qwen7b-layer", "branch-open", "long-rag", "serving-mix", "masked-prefill"])
+    ap.add_argument("--workload", default="serving-mix", choices=["qwen7b-layer", "branch-open", "long-rag", "serving-mix", "masked-prefill", "serving-mix-serial"])
     ap.add_argument("--op", default="step", choices=["step", "rerotate"],
                     help="step: the attention step (the benchmark); rerotate: the Same-Re key re-rotation kernel alone")
     ap.add_argument("--layers", type=int, default=28)

@@ -398,6 +398,14 @@ def config_masked_prefill(seed: int = SEED_BASE + 5, theta: float = 1.0e6, n_req
                                   [[x + 1 for x in p] for p in prior])
 
 
+def config_serving_mix_serial(seed: int = SEED_BASE + 4, theta: float = 1.0e6, n_req: int = 32) -> Workload:
+    """The serving mix one step later: the segment has ended, every request decodes one serial
+    token over its merged cache (prefix, all branches, tail) -- nothing was moved or recomputed."""
+    prefix, prior = serving_mix_lengths(seed, n_req)
+    return build_segment_workload("serving-mix-serial", seed, 28, 4, 128, "bf16", theta, prefix, prior,
+                                  [[1] * len(p) for p in prior], serial_steps=1)
+
+
 CONFIGS = {
     "tiny-f32": config_tiny,
     "qwen7b-layer": config_qwen7b_layer,
@@ -405,4 +413,5 @@ CONFIGS = {
     "long-rag": config_long_rag,
     "serving-mix": config_serving_mix,
     "masked-prefill": config_masked_prefill,
+    "serving-mix-serial": config_serving_mix_serial,
 }
