@@ -285,6 +285,80 @@ def run_rerotate(args):
     return 0
 
 
+def run_serial_chain(args):
+    """--op serial-chain: a segment of 6 branches opens (12-token headers) over a 1024-token
+    prefix, merges, and 64 serial tokens are decoded one after the other (aspd_serial_step, one
+    plan per step, every step through all layers); the whole chain is one CUDA graph.  Tiny data
+    per call (2.3 MB): a latency measurement.  One GPU; prints its own JSON line."""
+    import torch
+    from paper_2508_08895_b200 import binding as B, engine as E, workloads as W
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback")
+    n_serial = 64
+    wl = W.config_branch_open(serial_steps=n_serial)
+    shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
+    L = args.layers
+    caches = [E.LayerCache(shape, wl.n_pool_pages) for _ in range(L)]
+    serial = [ph for ph in wl.phases if ph.mode == W.MODE_SERIAL]
+    assert len(serial) == n_serial and all(ph.mode != W.MODE_SERIAL for ph in wl.phases[:-n_serial])
+    for ph in wl.phases[:-n_serial]:                  # prefix and the opening step: cache fill
+        plan = B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode)
+        pos, _, _ = B.positions(ph.desc, ph.mode)
+        pos_d = torch.from_numpy(pos.copy()).cuda()
+        k_d, v_d = E.to_device(ph.k_new, wl.dtype), E.to_device(ph.v_new, wl.dtype)
+        for c in caches:
+            B.kv_append(plan, k_d, v_d, pos_d, c.k, c.v)
+        torch.cuda.synchronize()
+        plan.destroy()
+    plans = [B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode, stable_cache=True) for ph in serial]
+    qkv = [tuple(E.to_device(x, wl.dtype) for x in (ph.q, ph.k_new, ph.v_new)) for ph in serial]
+    outs = [torch.empty_like(q) for q, _, _ in qkv]
+    alg = float(sum(pl.info.algorithmic_bytes for pl in plans))
+
+    def chain():
+        for s_, pl in enumerate(plans):
+            q, k, v = qkv[s_]
+            for c in caches:
+                B.serial_step(pl, q, k, v, c.k, c.v, outs[s_])
+    chain()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        chain()
+    reps = max(1, min(args.steps, 50))
+    for _ in range(max(args.warmup, 3)):
+        graph.replay()
+    sampler = ClockSampler(0)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    for _ in range(reps):
+        graph.replay()
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop()
+    if any(pl.status() != 0 for pl in plans):
+        raise SystemExit("bench.py: device status")
+    peak, peak_kind = measured_peaks()
+    gbs = alg * L * reps / (ms * 1e-3) / 1e9
+    launches = sum(2 if pl.info.fused_append else 3 for pl in plans) * L * reps
+    print(json.dumps({
+        "op": "serial-chain", "metric": "serial_decode_steps_per_second", "value": n_serial * reps / (ms * 1e-3), "unit": "steps/s",
+        "n_gpus": 1, "steps": reps, "warmup": max(args.warmup, 3), "ms_per_step": ms / reps, "higher_is_better": True,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "branch-open, then 64 serial steps over the merged cache (1097 + s keys at step s)", "layers": L,
+                   "serial_steps": n_serial, "heads": f"{wl.Hq}/{wl.Hkv}", "head_dim": wl.d, "cuda_graph": True,
+                   "calls": "aspd_serial_step per (step, layer), one plan per step"},
+        "layer_step_us": ms / reps / (n_serial * L) * 1e3,
+        "hbm_gbs": gbs, "hbm_frac_of_measured": gbs / peak, "peak_kind": "of " + peak_kind,
+        "algorithmic_bytes_per_chain_per_layer": alg, "gpu_launches": launches, "clocks": clocks}))
+    for pl in plans:
+        pl.destroy()
+    return 0
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -368,6 +442,22 @@ def run_ours(args):
     ms = ev0.elapsed_time(ev1)
     if plan.status() != 0:
         raise SystemExit("bench.py: device status %d" % plan.status())
+
+    # latency of a single layer call launched from the host (no graph), cold pools: median of 50
+    lat = []
+    la, lb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(50):
+        l = i % L
+        torch.cuda.synchronize()
+        la.record(stream)
+        if fused:
+            fstep(plan, q_d, k_d, v_d, caches[l].k, caches[l].v, outs[l])
+        else:
+            B.kv_append(plan, k_d, v_d, pos_d, caches[l].k, caches[l].v)
+            attn(plan, q_d, caches[l].k, caches[l].v, outs[l])
+        lb.record(stream)
+        torch.cuda.synchronize()
+        lat.append(la.elapsed_time(lb) * 1e3)
 
     # the dominant kernel alone: the split-K pass over all layers, back to back (also a graph)
     def partials():
@@ -471,6 +561,8 @@ def run_ours(args):
                     "d2h_bytes_per_step": int(L * n_new * es * wl.d * wl.Hq), "ms_per_step": e2e_ms / e_steps,
                     "calls": "aspd_step_host_async per layer, layers rotating over %d plans on %d streams, "
                              "one synchronisation per step" % (n_e, n_e)},
+            "single_call_us": {"median": float(np.median(lat)), "best": float(np.min(lat)), "calls": len(lat),
+                               "what": "one layer's step call launched from the host, CUDA events around it"},
             "gpu_launches": (2 if (fused and info.fused_append) or info.direct_output else 3) * L * args.steps,
             "clocks": clocks,
         }
@@ -496,8 +588,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="serving-mix", choices=["qwen7b-layer", "branch-open", "long-rag", "serving-mix", "masked-prefill", "serving-mix-serial"])
-    ap.add_argument("--op", default="step", choices=["step", "rerotate"],
-                    help="step: the attention step (the benchmark); rerotate: the Same-Re key re-rotation kernel alone")
+    ap.add_argument("--op", default="step", choices=["step", "rerotate", "serial-chain"],
+                    help="step: the attention step (the benchmark); rerotate: the Same-Re key re-rotation kernel alone; "
+                         "serial-chain: 64 serial steps after a merged segment, one graph")
     ap.add_argument("--layers", type=int, default=28)
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "mma"])
     ap.add_argument("--chunk", type=int, default=0)
@@ -515,6 +608,8 @@ def main():
         return run_reference(args)
     if args.op == "rerotate":
         return run_rerotate(args)
+    if args.op == "serial-chain":
+        return run_serial_chain(args)
     return run_ours(args)
 
 
