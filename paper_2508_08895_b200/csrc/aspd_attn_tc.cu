@@ -971,12 +971,15 @@ static int launch_tc(const aspd_plan* p, const void* q, const void* k_new, const
                      const void* v_pool, void* out, cudaStream_t s) {
   if (p->n_items == 0) return ASPD_OK;
   const aspd_shape_t& sh = p->shape;
-  static bool configured = false;
-  if (!configured) {
+  // the attribute belongs to the (function, device) pair: set it once on every device that launches
+  static bool configured[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return ASPD_ERR_CUDA;
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
     if (cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
       return ASPD_ERR_CUDA;
-    configured = true;
+    if (dev >= 0 && dev < 64) configured[dev] = true;
   }
   Ctx c;
   c.pd = p->dev;
