@@ -76,3 +76,29 @@ def test_static_scratch_rejects_plans_beyond_its_size_and_device_plans():
     with pytest.raises(B.AspdError) as e:
         B.attn_static(dev_plan, dummy, dummy, dummy, dummy)
     assert e.value.status == -1
+
+
+def test_static_scratch_runs_the_plans_other_regimes():
+    """Host-only plans made for the wide kernel variant (whole streams dealt, 128-row blocks) and
+    for the visible mask of the ablation run through the scratch array like any other."""
+    import torch
+    wl = W.build_segment_workload("prefill", 29, 28, 4, 128, "bf16", 1e6, [300, 40], [[0, 17, 5], [0]], [[100, 60, 31], [49]])
+    run, ph, q, ref = _setup(wl)
+    want = ref.float().cpu().numpy()
+    wide = B.Plan(run.shape, ph.desc, wl.n_pool_pages, ph.mode, n_ctas=8, host_only=True)
+    assert wide.info.max_rows_per_item == 128
+    out = torch.full_like(q, float("nan"))
+    B.attn_static(wide, q, run.cache.k, run.cache.v, out)
+    torch.cuda.synchronize()
+    err = np.abs(out.float().cpu().numpy().astype(np.float64) - want)
+    assert err.max() <= 2e-2 and err.mean() <= 2e-3
+    shared_dev = B.Plan(run.shape, ph.desc, wl.n_pool_pages, ph.mode, mask=B.MASK_SHARED)
+    ref2 = torch.empty_like(q)
+    B.branch_attn(shared_dev, q, run.cache.k, run.cache.v, ref2)
+    shared_host = B.Plan(run.shape, ph.desc, wl.n_pool_pages, ph.mode, mask=B.MASK_SHARED, host_only=True)
+    out2 = torch.full_like(q, float("nan"))
+    B.attn_static(shared_host, q, run.cache.k, run.cache.v, out2)
+    torch.cuda.synchronize()
+    a, b = out2.float().cpu().numpy().astype(np.float64), ref2.float().cpu().numpy().astype(np.float64)
+    assert np.abs(a - b).max() <= 2e-2 and np.abs(a - b).mean() <= 2e-3
+    assert np.abs(b - want).max() > 1e-2          # the other mask really is another result
