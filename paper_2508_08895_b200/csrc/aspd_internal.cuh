@@ -65,29 +65,29 @@ struct PlanDevice {       // pointers into the plan's single device allocation
 }  // namespace aspd
 
 struct aspd_plan {
-  aspd_shape_t shape;
-  int mode;
-  int n_req;
-  int n_new;
-  int n_items;
-  int n_partials;
-  int kernel;
-  int chunk_tokens;
-  int n_ctas;
-  int host_only;
-  int sm_count;
-  int n_row_blocks;
-  int fuse_append;             // few enough new rows per CTA for the attention pass to write them itself
-  int stable_cache;            // producers may fetch pages without new rows before the dependency wait
-  int dealt;                   // whole streams dealt to the CTAs in turn (many more streams than CTAs)
-  int shared_mask;             // parallel step under the ablation's visible mask
-  int wide;                    // dealt plan of the tensor-core kernel: row blocks of up to kMaxRowsWide rows
-  int64_t n_pool_pages;
-  int64_t kv_tokens_read;
-  int64_t algorithmic_bytes;
-  size_t device_bytes;
-  void* device_base;
-  aspd::PlanDevice dev;
+  aspd_shape_t shape = {};
+  int mode = 0;
+  int n_req = 0;
+  int n_new = 0;
+  int n_items = 0;
+  int n_partials = 0;
+  int kernel = 0;
+  int chunk_tokens = 0;
+  int n_ctas = 0;
+  int host_only = 0;
+  int sm_count = 0;
+  int n_row_blocks = 0;
+  int fuse_append = 0;             // few enough new rows per CTA for the attention pass to write them itself
+  int stable_cache = 0;            // producers may fetch pages without new rows before the dependency wait
+  int dealt = 0;                   // whole streams dealt to the CTAs in turn (many more streams than CTAs)
+  int shared_mask = 0;             // parallel step under the ablation's visible mask
+  int wide = 0;                    // dealt plan of the tensor-core kernel: row blocks of up to kMaxRowsWide rows
+  int64_t n_pool_pages = 0;
+  int64_t kv_tokens_read = 0;
+  int64_t algorithmic_bytes = 0;
+  size_t device_bytes = 0;
+  void* device_base = nullptr;
+  aspd::PlanDevice dev = {};
   std::vector<aspd::DeviceItem> items;
   std::vector<int2> visit;
   std::vector<int4> tok_vis;
