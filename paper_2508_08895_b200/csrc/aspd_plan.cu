@@ -289,7 +289,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
         const int nv = std::min(ps, len - s0), first_new = std::max(s0, new_key0);
         const int n_newrows = std::max(0, s0 + nv - first_new);
         int y = nv;
-        if (n_newrows > 0) y |= (n_newrows << 8);
+        if (n_newrows > 0) y |= (std::min(n_newrows, 31) << 8);   // 5 bits; a count is only needed where pages have 16 rows
         if (shared_mask) y |= branch_pages ? (s0 / ps) << 13 : 0;
         else if (n_newrows > 0) y |= (new_tok0 + first_new - new_key0) << 13;
         visit.push_back(make_int2(page_ids[q.page_begin + (slot0 + s0) / ps], y));

@@ -155,6 +155,13 @@ def test_shared_mask_plans_cover_the_oracles_visible_sets():
                     assert not plan.info.fused_append and not plan.info.direct_output
                 _check_cover(wl, ph, plan, chunk=chunk, mask=oracle.MASK_SHARED)
                 plan.destroy()
+    # pages of 32 rows that are new in full (the page entry's bit fields must not run into each other)
+    wl = W.build_segment_workload("p32", 8, 4, 2, 64, "f32", 1e4, [33], [[0, 31, 2]], [[70, 40, 1]], page_size=32)
+    ph = wl.phases[-1]
+    for mask in (B.MASK_BRANCH_INVISIBLE, B.MASK_SHARED):
+        plan = B.Plan(_shape(wl), ph.desc, wl.n_pool_pages, ph.mode, host_only=True, mask=mask)
+        _check_cover(wl, ph, plan, mask=mask, dealt=bool(plan.info.direct_output) or plan.info.n_partials == plan.n_new * wl.Hkv)
+        plan.destroy()
     assert _plan_rc(W.config_tiny(), W.config_tiny().phases[-1].desc, W.config_tiny().phases[-1].mode, mask=7) == -1     # ASPD_ERR_INVALID_ARG
 
 
