@@ -274,6 +274,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   std::vector<Block> blocks;
   std::vector<int4> tok_vis(n_new);
   int64_t kv_tokens = 0;
+  const bool tok_field_fits = n_new < (1 << 18);      // the 18 bits above bit 13 of a page entry hold a token index
   auto build_visit = [&](int block_tok) {
     visit.clear(); blocks.clear();
     int64_t kv_count = 0;
@@ -291,7 +292,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
         int y = nv;
         if (n_newrows > 0) y |= (std::min(n_newrows, 31) << 8);   // 5 bits; a count is only needed where pages have 16 rows
         if (shared_mask) y |= branch_pages ? (s0 / ps) << 13 : 0;
-        else if (n_newrows > 0) y |= (new_tok0 + first_new - new_key0) << 13;
+        else if (n_newrows > 0 && tok_field_fits) y |= (new_tok0 + first_new - new_key0) << 13;
         visit.push_back(make_int2(page_ids[q.page_begin + (slot0 + s0) / ps], y));
       }
     };
@@ -495,7 +496,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
     // rows per CTA (a branch-open step) the separate append kernel is the faster way
     int most = 0;
     for (int c = 0; c < n_ctas; ++c) most = std::max(most, cta_dirty0[c + 1] - cta_dirty0[c]);
-    p->fuse_append = (most <= 20 && !shared_mask) ? 1 : 0;
+    p->fuse_append = (most <= 20 && !shared_mask && tok_field_fits) ? 1 : 0;
   }
   for (size_t i = 0; i < n_parts.size(); ++i) part_base[i + 1] = part_base[i] + n_parts[i];
   p->n_items = (int)p->items.size();
