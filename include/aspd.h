@@ -205,7 +205,17 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
                      const int32_t* page_ids, int n_req, int64_t n_pool_pages, int mode,
                      const int32_t* q_pos, const aspd_tuning_t* tuning, void* stream,
                      aspd_plan_t** plan_out);
+/*
+ * Destroys the plan.  Work of the plan that is still in flight need not be waited for: the plan's
+ * device block is parked with an event recorded on every stream the plan was used on, and a later
+ * aspd_plan_create reuses a parked block of fitting size after making its own stream wait for
+ * those events (so a decode loop that makes a plan per step neither allocates nor synchronises in
+ * steady state).  Up to 8 blocks and 2 GiB in total are kept per process; what does not fit is
+ * freed at once (cudaFree, which waits for the device).
+ */
 int aspd_plan_destroy(aspd_plan_t* plan);
+/* Frees the parked device blocks (e.g. before handing the GPU's memory to someone else). */
+int aspd_release_cached_memory(void);
 int aspd_plan_info(const aspd_plan_t* plan, aspd_plan_info_t* info /*host*/);
 /* Copy up to max_items work items to `items` (host); returns the number of items. */
 int aspd_plan_items(const aspd_plan_t* plan, aspd_item_t* items, int max_items);

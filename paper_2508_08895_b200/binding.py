@@ -57,7 +57,7 @@ class AspdError(RuntimeError):
 
 
 EXPORTS = ("aspd_strerror", "aspd_pool_bytes", "aspd_count_new_tokens", "aspd_positions", "aspd_visible_slots",
-           "aspd_visible_slots_masked", "aspd_plan_create", "aspd_plan_destroy", "aspd_plan_info", "aspd_plan_items", "aspd_plan_cta_ranges", "aspd_plan_stream_pages",
+           "aspd_visible_slots_masked", "aspd_plan_create", "aspd_plan_destroy", "aspd_release_cached_memory", "aspd_plan_info", "aspd_plan_items", "aspd_plan_cta_ranges", "aspd_plan_stream_pages",
            "aspd_plan_token_ranges", "aspd_plan_shared_mask_tables", "aspd_plan_status",
            "aspd_kv_append", "aspd_branch_attn", "aspd_serial_attn", "aspd_attn_partials", "aspd_attn_combine",
            "aspd_branch_step", "aspd_serial_step", "aspd_step_host", "aspd_step_host_async", "aspd_attn_static", "aspd_k_rerotate", "aspd_debug_read_token", "aspd_debug_bounded_wait")
@@ -87,6 +87,7 @@ def lib() -> ctypes.CDLL:
         L.aspd_visible_slots_masked.argtypes = [vp, vp, ci, ci, ci, ci, vp]
         L.aspd_plan_create.argtypes = [vp, vp, vp, vp, ci, ctypes.c_int64, ci, vp, vp, vp, vp]
         L.aspd_plan_destroy.argtypes = [vp]
+        L.aspd_release_cached_memory.argtypes = []
         L.aspd_plan_info.argtypes = [vp, vp]
         L.aspd_plan_items.argtypes = [vp, vp, ci]
         L.aspd_plan_cta_ranges.argtypes = [vp, vp, ci]
@@ -303,6 +304,11 @@ def step_host(plan: Plan, q, k_new, v_new, pos, k_pool, v_pool, out, stream=None
     """Whole step from host (numpy / pinned torch CPU) buffers; ``out`` is a host buffer."""
     _check(lib().aspd_step_host(plan._h, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(pos), _ptr(k_pool), _ptr(v_pool),
                                 _ptr(out), _stream(stream)), "aspd_step_host")
+
+
+def release_cached_memory() -> None:
+    """Free the device blocks of destroyed plans that the library keeps for reuse."""
+    _check(lib().aspd_release_cached_memory(), "aspd_release_cached_memory")
 
 
 def step_host_async(plan: Plan, q, k_new, v_new, pos, k_pool, v_pool, out, stream=None) -> None:

@@ -86,6 +86,8 @@ struct aspd_plan {
   int64_t kv_tokens_read = 0;
   int64_t algorithmic_bytes = 0;
   size_t device_bytes = 0;
+  size_t block_bytes = 0;          // size of the device block the plan holds (a reused block may be larger than needed)
+  std::vector<cudaStream_t> streams;   // streams the plan's work was enqueued on
   void* device_base = nullptr;
   aspd::PlanDevice dev = {};
   std::vector<aspd::DeviceItem> items;
@@ -133,6 +135,8 @@ int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const
                     cudaStream_t s);
 inline bool attn_mma_writes_output(const aspd_plan* p) { return p->kernel == ASPD_KERNEL_MMA && p->dealt; }
 int launch_combine(const aspd_plan* p, void* out, cudaStream_t s);
+// fills the plan's cos/sin table from its position and frequency tables (plan creation, after the upload)
+int launch_qcs(const aspd_plan* p, cudaStream_t s);
 // attention pass that first writes this step's new K (rotated) and V rows into the pages it reads
 int launch_attn_mma_step(const aspd_plan* p, const void* q, const void* k_new, const void* v_new, void* k_pool,
                          void* v_pool, void* out, cudaStream_t s);

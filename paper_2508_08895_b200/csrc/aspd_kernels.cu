@@ -86,6 +86,21 @@ append_kernel(const T* __restrict__ k_new, const T* __restrict__ v_new, const in
   }
 }
 
+// ------------------------------------------------------------------- cos/sin table of a plan
+// q_cs[t][i] = (cos, sin)(pos[t] * inv_freq[i]): the rotation of new token t's query (and, in the
+// fused step, of its key).  Same arithmetic as the append kernel: angle reduced in fp64, fp32 sincos.
+__global__ void qcs_kernel(const int32_t* __restrict__ pos, const double* __restrict__ inv_freq, float2* __restrict__ q_cs,
+                           int n_new, int half) {
+  const long gid = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= (long)n_new * half) return;
+  const int t = (int)(gid / half), i = (int)(gid % half);
+  double a = (double)pos[t] * inv_freq[i];
+  a -= rint(a * 0.15915494309189535) * 6.283185307179586;
+  float sn, cs;
+  sincosf((float)a, &sn, &cs);
+  q_cs[gid] = make_float2(cs, sn);
+}
+
 // --------------------------------------------------------------------------- re-rotation
 // K'(pos + delta) = RoPE(K'(pos), delta): rotations compose, so cached keys can be moved to new
 // position IDs in place, reading and writing each key once, instead of being re-encoded from
@@ -333,6 +348,13 @@ int launch_attn_generic(const aspd_plan* p, const void* q, const void* k_pool, c
   else if (sh.head_dim == 128) ASPD_GEN(float, 128);
   else ASPD_GEN(float, 64);
 #undef ASPD_GEN
+}
+
+int launch_qcs(const aspd_plan* p, cudaStream_t s) {
+  const int half = p->shape.head_dim / 2;
+  const long n = (long)p->n_new * half;
+  qcs_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(p->dev.tok_pos, p->dev.inv_freq, const_cast<float2*>(p->dev.q_cs), p->n_new, half);
+  return check_launch();
 }
 
 int launch_combine(const aspd_plan* p, void* out, cudaStream_t s) {

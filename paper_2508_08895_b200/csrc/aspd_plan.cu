@@ -6,6 +6,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -17,6 +18,90 @@ namespace {
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---- device blocks of destroyed plans are kept for the next plan --------------------------------
+// A decode loop makes a new plan every step; cudaMalloc and cudaFree (which waits for the whole
+// device) would cost more than the step's host work.  aspd_plan_destroy therefore parks the plan's
+// block together with an event recorded on every stream the plan was used on, and
+// aspd_plan_create takes a parked block of fitting size and makes its stream wait for those events
+// before the new tables are uploaded -- no host synchronisation on either side.
+struct ParkedBlock { void* ptr; size_t bytes; int device; std::vector<cudaEvent_t> events; };
+std::mutex g_blocks_mu;
+std::vector<ParkedBlock> g_blocks;
+constexpr size_t kParkedMax = 8;                       // blocks kept per process
+constexpr size_t kParkedMaxBytes = 2048ull << 20;     // all parked blocks together; what does not fit is freed right away
+
+int block_acquire(size_t bytes, cudaStream_t s, void** out, size_t* got) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return ASPD_ERR_CUDA;
+  {
+    std::lock_guard<std::mutex> lock(g_blocks_mu);
+    int best = -1;
+    for (int i = 0; i < (int)g_blocks.size(); ++i)
+      if (g_blocks[i].device == dev && g_blocks[i].bytes >= bytes && g_blocks[i].bytes <= 4 * bytes + (1u << 20) &&
+          (best < 0 || g_blocks[i].bytes < g_blocks[best].bytes))
+        best = i;
+    if (best >= 0) {
+      ParkedBlock b = g_blocks[best];
+      g_blocks.erase(g_blocks.begin() + best);
+      int rc = ASPD_OK;
+      for (cudaEvent_t e : b.events) {
+        if (cudaStreamWaitEvent(s, e, 0) != cudaSuccess) rc = ASPD_ERR_CUDA;
+        cudaEventDestroy(e);
+      }
+      if (rc) { cudaFree(b.ptr); return rc; }
+      *out = b.ptr; *got = b.bytes;
+      return ASPD_OK;
+    }
+  }
+  if (cudaMalloc(out, bytes) != cudaSuccess) return ASPD_ERR_NOMEM;
+  *got = bytes;
+  return ASPD_OK;
+}
+
+int block_release(void* ptr, size_t bytes, const std::vector<cudaStream_t>& streams) {
+  int dev = 0;
+  bool park = cudaGetDevice(&dev) == cudaSuccess;
+  cudaPointerAttributes attr;
+  if (park && (cudaPointerGetAttributes(&attr, ptr) != cudaSuccess || attr.device != dev)) park = false;   // freed from another device's context
+  std::vector<cudaEvent_t> events;
+  for (size_t i = 0; park && i < streams.size(); ++i) {
+    cudaEvent_t e;
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess || cudaEventRecord(e, streams[i]) != cudaSuccess) park = false;
+    else events.push_back(e);
+  }
+  if (park) {
+    std::lock_guard<std::mutex> lock(g_blocks_mu);
+    size_t parked = 0;
+    for (const ParkedBlock& b : g_blocks) parked += b.bytes;
+    if (g_blocks.size() < kParkedMax && parked + bytes <= kParkedMaxBytes) {
+      g_blocks.push_back({ptr, bytes, dev, events});
+      return ASPD_OK;
+    }
+  }
+  for (cudaEvent_t e : events) cudaEventDestroy(e);
+  return cudaFree(ptr) == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
+}
+
+int block_cache_clear() {
+  std::vector<ParkedBlock> all;
+  {
+    std::lock_guard<std::mutex> lock(g_blocks_mu);
+    all.swap(g_blocks);
+  }
+  int rc = ASPD_OK;
+  for (ParkedBlock& b : all) {
+    for (cudaEvent_t e : b.events) cudaEventDestroy(e);
+    if (cudaFree(b.ptr) != cudaSuccess) rc = ASPD_ERR_CUDA;
+  }
+  return rc;
+}
+
+// every stream a plan's work was enqueued on (a handful at most): what its block must wait for when reused
+inline void note_stream(aspd_plan* p, void* stream) {
+  cudaStream_t s = (cudaStream_t)stream;
+  if (std::find(p->streams.begin(), p->streams.end(), s) == p->streams.end()) p->streams.push_back(s);
+}
 
 int check_shape(const aspd_shape_t* s) {
   if (!s) return ASPD_ERR_INVALID_ARG;
@@ -522,11 +607,11 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   const size_t o_tpos = take(sizeof(int32_t) * std::max(1, n_new));
   const size_t o_tvis = take(sizeof(int4) * std::max(1, n_new));
   const size_t o_rb = take(sizeof(int2) * std::max<size_t>(1, row_blocks.size()));
-  const size_t o_qcs = take(sizeof(float2) * std::max(1, n_new) * (d / 2));
   const size_t o_pbase = take(sizeof(int32_t) * part_base.size());
   const size_t o_freq = take(sizeof(double) * (d / 2));
   const size_t o_status = take(sizeof(int32_t) * 2);
   const size_t upload_bytes = off;
+  const size_t o_qcs = take(sizeof(float2) * std::max(1, n_new) * (d / 2));   // filled on the device from tok_pos and inv_freq
   const size_t o_wso = take(sizeof(float) * (size_t)std::max(1, p->n_partials) * G * d);
   const size_t o_wsml = take(sizeof(float2) * (size_t)std::max(1, p->n_partials) * G);
   const size_t o_stq = take((size_t)es * std::max(1, n_new) * Hq * d);
@@ -552,19 +637,15 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   memcpy(blob.data() + o_pbase, part_base.data(), sizeof(int32_t) * part_base.size());
   double* freq = reinterpret_cast<double*>(blob.data() + o_freq);
   for (int i = 0; i < d / 2; ++i) freq[i] = pow((double)shape->rope_theta, -2.0 * i / d);
-  float2* qcs = reinterpret_cast<float2*>(blob.data() + o_qcs);
-  for (int t = 0; t < n_new; ++t)
-    for (int i = 0; i < d / 2; ++i) {
-      double a = (double)pos[t] * freq[i];
-      qcs[(size_t)t * (d / 2) + i] = make_float2((float)cos(a), (float)sin(a));
-    }
 
   cudaStream_t s = (cudaStream_t)stream;
   void* base = nullptr;
-  if (cudaMalloc(&base, p->device_bytes) != cudaSuccess) { delete p; return ASPD_ERR_NOMEM; }
+  rc = block_acquire(p->device_bytes, s, &base, &p->block_bytes);
+  if (rc) { delete p; return rc; }
   if (cudaMemcpyAsync(base, blob.data(), upload_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
     cudaFree(base); delete p; return ASPD_ERR_CUDA;
   }
+  p->streams.push_back(s);
   // the blob is pageable: the copy above has been staged by the time the call returns
   uint8_t* b8 = (uint8_t*)base;
   p->device_base = base;
@@ -588,6 +669,8 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   p->dev.ws_ml = (float2*)(b8 + o_wsml);
   p->dev.st_q = b8 + o_stq; p->dev.st_k = b8 + o_stk; p->dev.st_v = b8 + o_stv; p->dev.st_out = b8 + o_sto;
   p->dev.st_pos = (int32_t*)(b8 + o_stp);
+  // cos/sin of every new token's position (query rotation, fused append): on the device, after the upload
+  if (n_new > 0 && (rc = launch_qcs(p, s)) != ASPD_OK) { cudaFree(base); delete p; return rc; }
   *plan_out = p;
   return ASPD_OK;
 }
@@ -595,10 +678,12 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
 int aspd_plan_destroy(aspd_plan_t* plan) {
   if (!plan) return ASPD_OK;
   int rc = ASPD_OK;
-  if (plan->device_base && cudaFree(plan->device_base) != cudaSuccess) rc = ASPD_ERR_CUDA;
+  if (plan->device_base) rc = block_release(plan->device_base, plan->block_bytes, plan->streams);
   delete plan;
   return rc;
 }
+
+int aspd_release_cached_memory(void) { return block_cache_clear(); }
 
 int aspd_plan_info(const aspd_plan_t* p, aspd_plan_info_t* info) {
   if (!p || !info) return ASPD_ERR_INVALID_ARG;
@@ -661,6 +746,7 @@ int aspd_kv_append(aspd_plan_t* p, const void* k_new, const void* v_new, const i
   if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
   if (p->n_new == 0) return ASPD_OK;
   if (!k_new || !v_new || !pos || !k_pool || !v_pool || misaligned16(k_new, v_new, k_pool, v_pool)) return ASPD_ERR_INVALID_ARG;
+  note_stream(p, stream);
   return launch_append(p, k_new, v_new, pos, k_pool, v_pool, (cudaStream_t)stream);
 }
 
@@ -669,6 +755,7 @@ int aspd_attn_partials(aspd_plan_t* p, const void* q, const void* k_pool, const 
   if (p->n_new == 0) return ASPD_OK;
   if (!q || !k_pool || !v_pool || misaligned16(q, k_pool, v_pool)) return ASPD_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
+  note_stream(p, stream);
   return p->kernel == ASPD_KERNEL_MMA ? launch_attn_mma(p, q, k_pool, v_pool, nullptr, s)
                                       : launch_attn_generic(p, q, k_pool, v_pool, s);
 }
@@ -677,6 +764,7 @@ int aspd_attn_combine(aspd_plan_t* p, void* out, void* stream) {
   if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
   if (p->n_new == 0) return ASPD_OK;
   if (!out || misaligned16(out)) return ASPD_ERR_INVALID_ARG;
+  note_stream(p, stream);
   return launch_combine(p, out, (cudaStream_t)stream);
 }
 
@@ -685,6 +773,7 @@ static int run_attn(aspd_plan_t* p, int mode, const void* q, const void* k_pool,
   if (!p || p->host_only || p->mode != mode) return ASPD_ERR_INVALID_ARG;
   if (p->n_new == 0) return ASPD_OK;
   if (!q || !k_pool || !v_pool || !out || misaligned16(q, k_pool, v_pool, out)) return ASPD_ERR_INVALID_ARG;
+  note_stream(p, stream);
   // a plan with one item per (token, KV head) needs no records: the kernel normalises and writes the output
   if (attn_mma_writes_output(p)) return launch_attn_mma(p, q, k_pool, v_pool, out, (cudaStream_t)stream);
   int rc = aspd_attn_partials(p, q, k_pool, v_pool, stream);
@@ -706,6 +795,7 @@ static int run_step(aspd_plan_t* p, int mode, const void* q, const void* k_new, 
   if (p->n_new == 0) return ASPD_OK;
   if (!q || !k_new || !v_new || !k_pool || !v_pool || !out || misaligned16(q, k_new, v_new, k_pool, v_pool, out)) return ASPD_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
+  note_stream(p, stream);
   int rc;
   if (p->kernel == ASPD_KERNEL_MMA && p->fuse_append) {
     rc = launch_attn_mma_step(p, q, k_new, v_new, k_pool, v_pool, out, s);
@@ -736,6 +826,7 @@ int aspd_step_host_async(aspd_plan_t* p, const void* q, const void* k_new, const
   if (p->n_new == 0) return ASPD_OK;
   if (!q || !k_new || !v_new || !pos || !k_pool || !v_pool || !out || misaligned16(k_pool, v_pool)) return ASPD_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
+  note_stream(p, stream);
   const aspd_shape_t& sh = p->shape;
   const size_t es = esize_of(sh.dtype);
   const size_t qb = es * p->n_new * sh.n_q_heads * sh.head_dim, kb = es * p->n_new * sh.n_kv_heads * sh.head_dim;

@@ -615,6 +615,47 @@ def test_misaligned_device_buffers_are_refused_before_any_launch():
     plan.destroy()
 
 
+def test_plan_per_step_reuses_device_blocks_without_synchronising():
+    """A plan per step, destroyed while its work may still be in flight and on alternating streams:
+    the block of a destroyed plan is reused only after the streams it was used on have passed its
+    work (events, no host synchronisation), free device memory stays flat, every result is right."""
+    import torch
+    E = engine()
+    wl = W.config_serving_mix(n_req=8)
+    run = E.WorkloadRun(wl)
+    for ph in wl.phases[:-1]:
+        run.step(ph)
+    ph = wl.phases[-1]
+    q, k, v = (E.to_device(x, wl.dtype) for x in (ph.q, ph.k_new, ph.v_new))
+    ref_plan = B.Plan(run.shape, ph.desc, wl.n_pool_pages, ph.mode)
+    ref = torch.empty_like(q)
+    B.branch_step(ref_plan, q, k, v, run.cache.k, run.cache.v, ref)
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = [torch.zeros_like(q) for _ in range(30)]
+    B.release_cached_memory()
+    free0 = None
+    for i, o in enumerate(outs):
+        st = streams[i % 3]
+        plan = B.Plan(run.shape, ph.desc, wl.n_pool_pages, ph.mode, stream=st, n_ctas=[0, 37, 148][i % 3])
+        B.branch_step(plan, q, k, v, run.cache.k, run.cache.v, o, stream=st)
+        plan.destroy()                             # not waited for
+        if i == 8:
+            free0 = torch.cuda.mem_get_info()[0]
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] >= free0 - (1 << 20)      # no growth once the first blocks are parked
+    want = ref.float().cpu().numpy()
+    for i, o in enumerate(outs):
+        got = o.float().cpu().numpy()
+        if i % 3 == 0:
+            np.testing.assert_array_equal(got, want)              # same plan options: same bits
+        else:
+            assert np.abs(got - want).max() <= 2e-2
+    check(outs[-1].float().cpu().numpy(), oracle_run(wl).outputs[0], wl.dtype)
+    ref_plan.destroy()
+    B.release_cached_memory()
+
+
 def test_zero_new_tokens_is_a_no_op():
     E = engine()
     wl = W.build_segment_workload("e", 8, 28, 4, 128, "bf16", 1e6, [20], [[5, 9]], [[1, 1]])
