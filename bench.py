@@ -359,6 +359,96 @@ def run_serial_chain(args):
     return 0
 
 
+def run_decode_loop(args):
+    """--op decode-loop: 64 consecutive parallel decoding steps of the serving mix as an engine would
+    run them: every step the branches are one token longer, so every step gets its own plan
+    (created on the host, uploaded, destroyed after its 28 layer calls were enqueued; no graph,
+    no synchronisation inside the loop).  Measures what is left of the kernel rate once planning
+    and host launches are part of the loop.  One GPU; prints its own JSON line."""
+    import torch
+    from paper_2508_08895_b200 import binding as B, engine as E, workloads as W
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback")
+    n_steps = 64
+    prefix, prior = W.serving_mix_lengths(W.SEED_BASE + 4, args.requests or 32)
+    # regions sized for the last step; step t reads prior + t + 1 tokens of every branch
+    wl = W.build_segment_workload("serving-mix-loop", W.SEED_BASE + 4, 28, 4, 128, "bf16", 1.0e6, prefix,
+                                  [[x + n_steps - 1 for x in p] for p in prior], [[1] * len(p) for p in prior])
+    shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
+    L = args.layers
+    caches = [E.LayerCache(shape, wl.n_pool_pages) for _ in range(L)]
+    fill_caches(wl, shape, caches)
+    ph = wl.phases[-1]
+    q_d, k_d, v_d = (E.to_device(x, wl.dtype) for x in (ph.q, ph.k_new, ph.v_new))
+    outs = [torch.empty_like(q_d) for _ in range(L)]
+    n_new = int(q_d.shape[0])
+    descs = []
+    for t in range(n_steps):
+        d = {k: v.copy() for k, v in ph.desc.items()}
+        d["br_kv_len"] = (ph.desc["br_kv_len"] - (n_steps - 1 - t)).astype(np.int32)
+        descs.append(d)
+
+    # The C ABI called as a native engine would: descriptors packed ahead of the loop (an engine
+    # keeps them up to date incrementally), pointers resolved once, one foreign call per library call.
+    import ctypes
+    lib = B.lib()
+    packed = [B.pack_descriptors(d) for d in descs]
+    tune = B.Tuning(B.KERNEL_AUTO, 0, 0, 0, 1, 0)
+    stream = torch.cuda.current_stream().cuda_stream
+    qp, kp, vp = q_d.data_ptr(), k_d.data_ptr(), v_d.data_ptr()
+    layer_ptrs = [(c.k.data_ptr(), c.v.data_ptr(), o.data_ptr()) for c, o in zip(caches, outs)]
+    shape_p, tune_p = ctypes.addressof(shape), ctypes.addressof(tune)
+    handle = ctypes.c_void_p()
+    handle_p = ctypes.addressof(handle)
+
+    def loop():
+        plan_s = 0.0
+        for req, br, pages in packed:
+            t0 = time.perf_counter()
+            rc = lib.aspd_plan_create(shape_p, req.ctypes.data, br.ctypes.data, pages.ctypes.data, len(req), wl.n_pool_pages,
+                                      ph.mode, None, tune_p, stream, handle_p)
+            plan_s += time.perf_counter() - t0
+            if rc:
+                raise SystemExit("bench.py: aspd_plan_create returned %d" % rc)
+            for kc, vc, oc in layer_ptrs:
+                rc |= lib.aspd_branch_step(handle, qp, kp, vp, kc, vc, oc, stream)
+            rc |= lib.aspd_plan_destroy(handle)
+            if rc:
+                raise SystemExit("bench.py: a step call returned %d" % rc)
+        return plan_s
+    loop()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    reps = max(1, min(args.steps, 10))
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    ev0.record()
+    plan_s = sum(loop() for _ in range(reps))
+    host_s = time.perf_counter() - t0
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop()
+    total_steps = n_steps * reps
+    probe = B.Plan(shape, descs[n_steps // 2], wl.n_pool_pages, ph.mode, host_only=True)
+    alg = float(probe.info.algorithmic_bytes)
+    probe.destroy()
+    peak, peak_kind = measured_peaks()
+    gbs = alg * L * total_steps / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "op": "decode-loop", "metric": METRIC, "value": n_new * L * total_steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+        "steps": total_steps, "warmup": n_steps, "ms_per_step": ms / total_steps, "higher_is_better": True, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": "serving-mix, 64 consecutive decoding steps, a new plan every step", "layers": L,
+                   "query_tokens_per_step": n_new, "cuda_graph": False,
+                   "calls_per_step": "aspd_plan_create, %d x aspd_branch_step, aspd_plan_destroy" % L},
+        "host_ms_per_step": host_s / total_steps * 1e3, "plan_create_ms_per_step": plan_s / total_steps * 1e3,
+        "hbm_gbs": gbs, "hbm_frac_of_measured": gbs / peak, "peak_kind": "of " + peak_kind,
+        "gpu_launches": 2 * L * total_steps + total_steps, "clocks": clocks}))
+    return 0
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -588,9 +678,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="serving-mix", choices=["qwen7b-layer", "branch-open", "long-rag", "serving-mix", "masked-prefill", "serving-mix-serial"])
-    ap.add_argument("--op", default="step", choices=["step", "rerotate", "serial-chain"],
+    ap.add_argument("--op", default="step", choices=["step", "rerotate", "serial-chain", "decode-loop"],
                     help="step: the attention step (the benchmark); rerotate: the Same-Re key re-rotation kernel alone; "
-                         "serial-chain: 64 serial steps after a merged segment, one graph")
+                         "serial-chain: 64 serial steps after a merged segment, one graph; "
+                         "decode-loop: 64 decoding steps with a new plan each, launched from the host")
     ap.add_argument("--layers", type=int, default=28)
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "mma"])
     ap.add_argument("--chunk", type=int, default=0)
@@ -610,6 +701,8 @@ def main():
         return run_rerotate(args)
     if args.op == "serial-chain":
         return run_serial_chain(args)
+    if args.op == "decode-loop":
+        return run_decode_loop(args)
     return run_ours(args)
 
 

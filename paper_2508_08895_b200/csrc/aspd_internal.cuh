@@ -86,6 +86,9 @@ struct aspd_plan {
   int64_t kv_tokens_read = 0;
   int64_t algorithmic_bytes = 0;
   size_t device_bytes = 0;
+  void* host_block = nullptr;      // page-locked host buffer the tables were assembled in (travels with the device block)
+  size_t host_block_bytes = 0;
+  cudaEvent_t upload_done = nullptr;   // recorded after the table copy: the host buffer may be rewritten once it has completed
   size_t block_bytes = 0;          // size of the device block the plan holds (a reused block may be larger than needed)
   std::vector<cudaStream_t> streams;   // streams the plan's work was enqueued on
   void* device_base = nullptr;

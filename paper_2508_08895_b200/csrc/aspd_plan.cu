@@ -24,14 +24,19 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // device) would cost more than the step's host work.  aspd_plan_destroy therefore parks the plan's
 // block together with an event recorded on every stream the plan was used on, and
 // aspd_plan_create takes a parked block of fitting size and makes its stream wait for those events
-// before the new tables are uploaded -- no host synchronisation on either side.
-struct ParkedBlock { void* ptr; size_t bytes; int device; std::vector<cudaEvent_t> events; };
+// before the new tables are uploaded -- no host synchronisation on either side.  With the block goes
+// the page-locked host buffer the tables are assembled in (a copy from pageable memory would make
+// the host wait for everything queued before it on the stream).
+// upload_done: recorded right after the plan's table copy; the host may write the buffer again only
+// once it has completed, so a block whose copy is still queued is passed over (a fresh one is
+// allocated instead and the pool settles at the depth the loop needs).
+struct ParkedBlock { void* ptr; size_t bytes; void* host; size_t host_bytes; int device; cudaEvent_t upload_done; std::vector<cudaEvent_t> events; };
 std::mutex g_blocks_mu;
 std::vector<ParkedBlock> g_blocks;
 constexpr size_t kParkedMax = 8;                       // blocks kept per process
 constexpr size_t kParkedMaxBytes = 2048ull << 20;     // all parked blocks together; what does not fit is freed right away
 
-int block_acquire(size_t bytes, cudaStream_t s, void** out, size_t* got) {
+int block_acquire(size_t bytes, size_t host_need, cudaStream_t s, void** out, size_t* got, void** host, size_t* host_got) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return ASPD_ERR_CUDA;
   {
@@ -39,27 +44,37 @@ int block_acquire(size_t bytes, cudaStream_t s, void** out, size_t* got) {
     int best = -1;
     for (int i = 0; i < (int)g_blocks.size(); ++i)
       if (g_blocks[i].device == dev && g_blocks[i].bytes >= bytes && g_blocks[i].bytes <= 4 * bytes + (1u << 20) &&
-          (best < 0 || g_blocks[i].bytes < g_blocks[best].bytes))
+          (best < 0 || g_blocks[i].bytes < g_blocks[best].bytes) &&
+          (g_blocks[i].upload_done == nullptr || cudaEventQuery(g_blocks[i].upload_done) == cudaSuccess))
         best = i;
     if (best >= 0) {
       ParkedBlock b = g_blocks[best];
       g_blocks.erase(g_blocks.begin() + best);
       int rc = ASPD_OK;
+      if (b.upload_done) cudaEventDestroy(b.upload_done);
       for (cudaEvent_t e : b.events) {
         if (cudaStreamWaitEvent(s, e, 0) != cudaSuccess) rc = ASPD_ERR_CUDA;
         cudaEventDestroy(e);
       }
-      if (rc) { cudaFree(b.ptr); return rc; }
-      *out = b.ptr; *got = b.bytes;
+      if (rc == ASPD_OK && b.host_bytes < host_need) {           // too small for the new tables (its last copy has completed)
+        cudaFreeHost(b.host);
+        b.host = nullptr; b.host_bytes = 0;
+        if (rc == ASPD_OK && cudaMallocHost(&b.host, host_need) != cudaSuccess) rc = ASPD_ERR_NOMEM;
+        if (rc == ASPD_OK) b.host_bytes = host_need;
+      }
+      if (rc) { cudaFree(b.ptr); if (b.host) cudaFreeHost(b.host); return rc; }
+      *out = b.ptr; *got = b.bytes; *host = b.host; *host_got = b.host_bytes;
       return ASPD_OK;
     }
   }
   if (cudaMalloc(out, bytes) != cudaSuccess) return ASPD_ERR_NOMEM;
-  *got = bytes;
+  if (cudaMallocHost(host, host_need) != cudaSuccess) { cudaFree(*out); return ASPD_ERR_NOMEM; }
+  *got = bytes; *host_got = host_need;
   return ASPD_OK;
 }
 
-int block_release(void* ptr, size_t bytes, const std::vector<cudaStream_t>& streams) {
+int block_release(void* ptr, size_t bytes, void* host, size_t host_bytes, cudaEvent_t upload_done,
+                  const std::vector<cudaStream_t>& streams) {
   int dev = 0;
   bool park = cudaGetDevice(&dev) == cudaSuccess;
   cudaPointerAttributes attr;
@@ -75,12 +90,15 @@ int block_release(void* ptr, size_t bytes, const std::vector<cudaStream_t>& stre
     size_t parked = 0;
     for (const ParkedBlock& b : g_blocks) parked += b.bytes;
     if (g_blocks.size() < kParkedMax && parked + bytes <= kParkedMaxBytes) {
-      g_blocks.push_back({ptr, bytes, dev, events});
+      g_blocks.push_back({ptr, bytes, host, host_bytes, dev, upload_done, events});
       return ASPD_OK;
     }
   }
   for (cudaEvent_t e : events) cudaEventDestroy(e);
-  return cudaFree(ptr) == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
+  if (upload_done) cudaEventDestroy(upload_done);
+  const bool ok = cudaFree(ptr) == cudaSuccess;      // waits for the device: the buffer's last copy is done after it
+  if (host) cudaFreeHost(host);
+  return ok ? ASPD_OK : ASPD_ERR_CUDA;
 }
 
 int block_cache_clear() {
@@ -92,7 +110,9 @@ int block_cache_clear() {
   int rc = ASPD_OK;
   for (ParkedBlock& b : all) {
     for (cudaEvent_t e : b.events) cudaEventDestroy(e);
+    if (b.upload_done) cudaEventDestroy(b.upload_done);
     if (cudaFree(b.ptr) != cudaSuccess) rc = ASPD_ERR_CUDA;
+    if (b.host) cudaFreeHost(b.host);
   }
   return rc;
 }
@@ -621,7 +641,12 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   const size_t o_stp = take(sizeof(int32_t) * std::max(1, n_new));
   p->device_bytes = off;
 
-  std::vector<uint8_t> blob(upload_bytes, 0);
+  cudaStream_t s = (cudaStream_t)stream;
+  void* base = nullptr;
+  rc = block_acquire(p->device_bytes, upload_bytes, s, &base, &p->block_bytes, &p->host_block, &p->host_block_bytes);
+  if (rc) { delete p; return rc; }
+  struct { uint8_t* d; uint8_t* data() const { return d; } } blob = {static_cast<uint8_t*>(p->host_block)};
+  memset(blob.data(), 0, upload_bytes);
   if (p->n_items) memcpy(blob.data() + o_items, p->items.data(), sizeof(DeviceItem) * p->n_items);
   memcpy(blob.data() + o_cta, cta_item0.data(), sizeof(int32_t) * (n_ctas + 1));
   if (!visit.empty()) memcpy(blob.data() + o_visit, visit.data(), sizeof(int2) * visit.size());
@@ -638,15 +663,17 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   double* freq = reinterpret_cast<double*>(blob.data() + o_freq);
   for (int i = 0; i < d / 2; ++i) freq[i] = pow((double)shape->rope_theta, -2.0 * i / d);
 
-  cudaStream_t s = (cudaStream_t)stream;
-  void* base = nullptr;
-  rc = block_acquire(p->device_bytes, s, &base, &p->block_bytes);
-  if (rc) { delete p; return rc; }
   if (cudaMemcpyAsync(base, blob.data(), upload_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
-    cudaFree(base); delete p; return ASPD_ERR_CUDA;
+    cudaFree(base); cudaFreeHost(p->host_block); delete p; return ASPD_ERR_CUDA;
+  }
+  if (cudaEventCreateWithFlags(&p->upload_done, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventRecord(p->upload_done, s) != cudaSuccess) {
+    if (p->upload_done) cudaEventDestroy(p->upload_done);
+    p->upload_done = nullptr;
+    cudaStreamSynchronize(s);                      // no event to tell when the buffer is free again: be done with it now
   }
   p->streams.push_back(s);
-  // the blob is pageable: the copy above has been staged by the time the call returns
+  // the tables were assembled in the plan's page-locked buffer, which lives as long as the device block
   uint8_t* b8 = (uint8_t*)base;
   p->device_base = base;
   p->dev.items = (const DeviceItem*)(b8 + o_items);
@@ -670,7 +697,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   p->dev.st_q = b8 + o_stq; p->dev.st_k = b8 + o_stk; p->dev.st_v = b8 + o_stv; p->dev.st_out = b8 + o_sto;
   p->dev.st_pos = (int32_t*)(b8 + o_stp);
   // cos/sin of every new token's position (query rotation, fused append): on the device, after the upload
-  if (n_new > 0 && (rc = launch_qcs(p, s)) != ASPD_OK) { cudaFree(base); delete p; return rc; }
+  if (n_new > 0 && (rc = launch_qcs(p, s)) != ASPD_OK) { cudaFree(base); cudaFreeHost(p->host_block); delete p; return rc; }
   *plan_out = p;
   return ASPD_OK;
 }
@@ -678,7 +705,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
 int aspd_plan_destroy(aspd_plan_t* plan) {
   if (!plan) return ASPD_OK;
   int rc = ASPD_OK;
-  if (plan->device_base) rc = block_release(plan->device_base, plan->block_bytes, plan->streams);
+  if (plan->device_base) rc = block_release(plan->device_base, plan->block_bytes, plan->host_block, plan->host_block_bytes, plan->upload_done, plan->streams);
   delete plan;
   return rc;
 }
