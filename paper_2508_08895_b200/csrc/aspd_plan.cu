@@ -41,12 +41,18 @@ int block_acquire(size_t bytes, size_t host_need, cudaStream_t s, void** out, si
   if (cudaGetDevice(&dev) != cudaSuccess) return ASPD_ERR_CUDA;
   {
     std::lock_guard<std::mutex> lock(g_blocks_mu);
-    int best = -1;
-    for (int i = 0; i < (int)g_blocks.size(); ++i)
-      if (g_blocks[i].device == dev && g_blocks[i].bytes >= bytes && g_blocks[i].bytes <= 4 * bytes + (1u << 20) &&
-          (best < 0 || g_blocks[i].bytes < g_blocks[best].bytes) &&
+    int best = -1, oldest = -1, fitting = 0;
+    for (int i = 0; i < (int)g_blocks.size(); ++i) {
+      if (g_blocks[i].device != dev || g_blocks[i].bytes < bytes || g_blocks[i].bytes > 4 * bytes + (1u << 20)) continue;
+      ++fitting;
+      if (oldest < 0) oldest = i;
+      if ((best < 0 || g_blocks[i].bytes < g_blocks[best].bytes) &&
           (g_blocks[i].upload_done == nullptr || cudaEventQuery(g_blocks[i].upload_done) == cudaSuccess))
         best = i;
+    }
+    // every fitting block still has its copy queued: with a couple of them parked the host is simply
+    // ahead of the GPU and waits for the oldest one instead of allocating more
+    if (best < 0 && fitting >= 2 && cudaEventSynchronize(g_blocks[oldest].upload_done) == cudaSuccess) best = oldest;
     if (best >= 0) {
       ParkedBlock b = g_blocks[best];
       g_blocks.erase(g_blocks.begin() + best);
