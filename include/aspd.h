@@ -151,6 +151,9 @@ typedef struct {
   int32_t direct_output;    /* 1: one item per (token, KV head) and the attention kernel writes the
                                output itself (no records, no combine launch)                     */
   int32_t max_rows_per_item;/* query rows (tokens x group heads) an item may carry: 64 or 128       */
+  int32_t dealt;            /* 1: whole streams dealt to the CTAs (every row block has a page list of its
+                               own, so n_stream_pages counts shared pages once per row block); 0: stream-K cuts */
+  int32_t reserved;
   int64_t workspace_bytes;  /* device memory the plan holds                                 */
   int64_t kv_tokens_read;   /* cached tokens the step must read (each once)                 */
   int64_t algorithmic_bytes;/* K+V of those tokens + q in + out + appended K/V              */

@@ -46,6 +46,7 @@ class PlanInfo(ctypes.Structure):
                 ("n_stream_pages", ctypes.c_int32), ("kernel", ctypes.c_int32), ("chunk_tokens", ctypes.c_int32),
                 ("n_ctas", ctypes.c_int32), ("fused_append", ctypes.c_int32),
                 ("direct_output", ctypes.c_int32), ("max_rows_per_item", ctypes.c_int32),
+                ("dealt", ctypes.c_int32), ("reserved", ctypes.c_int32),
                 ("workspace_bytes", ctypes.c_int64), ("kv_tokens_read", ctypes.c_int64),
                 ("algorithmic_bytes", ctypes.c_int64)]
 

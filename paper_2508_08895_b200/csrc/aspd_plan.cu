@@ -500,7 +500,9 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   build_streams(max_tok);
   auto ctas_for = [&](long pages) {
     const int want = tune.n_ctas > 0 ? tune.n_ctas : p->sm_count;
-    return (int)std::max(1L, std::min((long)want, (pages + 3) / 4));     // do not cut finer than 64 keys per CTA
+    // do not cut finer than one 128-key tile per CTA (measured on a 2.5 k-token step: 80 CTAs with a
+    // full tile each take 10.6 us per layer, 148 CTAs with half a tile 11.9: fewer records to combine)
+    return (int)std::max(1L, std::min((long)want, (pages + 7) / 8));
   };
   // With many more streams than CTAs (a step with many query tokens per branch: masked prefill,
   // teacher forcing) nothing is cut: every stream is one item, and the streams are dealt to the
@@ -508,7 +510,9 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   // same one or two requests (which then stay in L2) and every CTA gets one stream of each round.
   // Every row block then gets a page sequence of its own, without the branch pages none of its
   // tokens sees, and the tensor-core kernel takes row blocks of up to 128 rows (its wide variant).
-  bool deal_streams = mode == ASPD_MODE_BRANCH && !shared_mask && tune.chunk_tokens == 0 && (long)streams.size() >= 4L * ctas_for(total_pages);
+  // (only where the step fills the grid, or the caller chose the grid: a step of a few pages has few CTAs and many streams by default)
+  bool deal_streams = mode == ASPD_MODE_BRANCH && !shared_mask && tune.chunk_tokens == 0 &&
+                      (long)streams.size() >= 4L * ctas_for(total_pages) && (tune.n_ctas > 0 || ctas_for(total_pages) >= p->sm_count);
   p->wide = 0;
   if (deal_streams) {
     p->wide = (kernel == ASPD_KERNEL_MMA && kMaxRowsWide / G > max_tok) ? 1 : 0;
@@ -724,6 +728,7 @@ int aspd_plan_info(const aspd_plan_t* p, aspd_plan_info_t* info) {
   info->n_stream_pages = (int32_t)p->visit.size(); info->kernel = p->kernel;
   info->chunk_tokens = p->chunk_tokens; info->n_ctas = p->n_ctas; info->fused_append = (p->kernel == ASPD_KERNEL_MMA && p->fuse_append) ? 1 : 0;
   info->direct_output = attn_mma_writes_output(p) ? 1 : 0; info->max_rows_per_item = p->wide ? kMaxRowsWide : kMaxRowsPerItem;
+  info->dealt = p->dealt; info->reserved = 0;
   info->workspace_bytes = (int64_t)p->device_bytes;
   info->kv_tokens_read = p->kv_tokens_read; info->algorithmic_bytes = p->algorithmic_bytes;
   return ASPD_OK;

@@ -84,6 +84,7 @@ def _shape(wl):
 def _check_cover(wl, ph, plan, chunk=0, dealt=False, mask=0):
     """The plan's work items, expanded through its stream-page list and the per-token visible
     ranges to (token, KV head, logical slot) triples, are exactly the oracle's visible sets."""
+    dealt = dealt or bool(plan.info.dealt)
     n_slots = int(ph.desc["n_pages"].max()) * wl.page_size
     vis = oracle.visible_slots(ph.desc, ph.mode, n_slots, mask=mask)
     _, _, treq = oracle.new_tokens(ph.desc, ph.mode)
