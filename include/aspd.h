@@ -109,6 +109,7 @@ typedef struct {
                            may then start fetching such pages before the previous kernel on the
                            stream has finished.  0 (default): full stream ordering for the pools */
   int32_t mask;         /* ASPD_MASK_*: attention mask of a parallel step (default: branch-invisible) */
+  int32_t updatable;    /* 1: leave room in the plan's tables (25 %) for aspd_plan_update                */
 } aspd_tuning_t;
 
 /* Attention mask of a parallel step.  BRANCH_INVISIBLE is the paper's mask (its Eq. 2-3).  SHARED
@@ -217,6 +218,20 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
  * freed at once (cudaFree, which waits for the device).
  */
 int aspd_plan_destroy(aspd_plan_t* plan);
+/*
+ * Re-plans an existing device plan for the NEXT step of the same batch, in place: same requests and
+ * branches decoding (the number of new tokens, the grid and the kernel variant must come out the
+ * same), lengths as given by the new descriptors.  The tables are rebuilt on the host and uploaded
+ * on `stream` to the addresses they already have, so kernel launches recorded in a CUDA graph with
+ * this plan stay valid: a decode loop captures one step once and per step calls aspd_plan_update
+ * and replays the graph, on one stream.  Create the plan with tuning->updatable = 1 so that the
+ * length-dependent tables have room to grow.
+ * Returns ASPD_ERR_UNSUPPORTED when the new step needs another launch sequence (other number of
+ * new tokens, grid, kernel variant, fused or separate append) and ASPD_ERR_TOO_LARGE when a table
+ * has outgrown its room; the plan is unchanged then and the caller makes a new one (and a new graph).
+ */
+int aspd_plan_update(aspd_plan_t* plan, const aspd_request_t* req, const aspd_branch_t* br, const int32_t* page_ids,
+                     int n_req, const int32_t* q_pos /*host, optional*/, void* stream);
 /* Frees the parked device blocks (e.g. before handing the GPU's memory to someone else). */
 int aspd_release_cached_memory(void);
 int aspd_plan_info(const aspd_plan_t* plan, aspd_plan_info_t* info /*host*/);

@@ -38,7 +38,8 @@ class Shape(ctypes.Structure):
 
 class Tuning(ctypes.Structure):
     _fields_ = [("kernel", ctypes.c_int32), ("chunk_tokens", ctypes.c_int32), ("n_ctas", ctypes.c_int32),
-                ("host_only", ctypes.c_int32), ("stable_cache", ctypes.c_int32), ("mask", ctypes.c_int32)]
+                ("host_only", ctypes.c_int32), ("stable_cache", ctypes.c_int32), ("mask", ctypes.c_int32),
+                ("updatable", ctypes.c_int32)]
 
 
 class PlanInfo(ctypes.Structure):
@@ -58,7 +59,7 @@ class AspdError(RuntimeError):
 
 
 EXPORTS = ("aspd_strerror", "aspd_pool_bytes", "aspd_count_new_tokens", "aspd_positions", "aspd_visible_slots",
-           "aspd_visible_slots_masked", "aspd_plan_create", "aspd_plan_destroy", "aspd_release_cached_memory", "aspd_plan_info", "aspd_plan_items", "aspd_plan_cta_ranges", "aspd_plan_stream_pages",
+           "aspd_visible_slots_masked", "aspd_plan_create", "aspd_plan_update", "aspd_plan_destroy", "aspd_release_cached_memory", "aspd_plan_info", "aspd_plan_items", "aspd_plan_cta_ranges", "aspd_plan_stream_pages",
            "aspd_plan_token_ranges", "aspd_plan_shared_mask_tables", "aspd_plan_status",
            "aspd_kv_append", "aspd_branch_attn", "aspd_serial_attn", "aspd_attn_partials", "aspd_attn_combine",
            "aspd_branch_step", "aspd_serial_step", "aspd_step_host", "aspd_step_host_async", "aspd_attn_static", "aspd_k_rerotate", "aspd_debug_read_token", "aspd_debug_bounded_wait")
@@ -88,6 +89,7 @@ def lib() -> ctypes.CDLL:
         L.aspd_visible_slots_masked.argtypes = [vp, vp, ci, ci, ci, ci, vp]
         L.aspd_plan_create.argtypes = [vp, vp, vp, vp, ci, ctypes.c_int64, ci, vp, vp, vp, vp]
         L.aspd_plan_destroy.argtypes = [vp]
+        L.aspd_plan_update.argtypes = [vp, vp, vp, vp, ci, vp, vp]
         L.aspd_release_cached_memory.argtypes = []
         L.aspd_plan_info.argtypes = [vp, vp]
         L.aspd_plan_items.argtypes = [vp, vp, ci]
@@ -206,10 +208,10 @@ class Plan:
 
     def __init__(self, shape: Shape, desc, n_pool_pages: int, mode: int, q_pos=None, kernel: int = KERNEL_AUTO,
                  chunk_tokens: int = 0, n_ctas: int = 0, host_only: bool = False, stable_cache: bool = False, stream=None,
-                 mask: int = 0):
+                 mask: int = 0, updatable: bool = False):
         self.shape, self.mode = shape, mode
         req, br, pages = pack_descriptors(desc)
-        tune = Tuning(kernel, chunk_tokens, n_ctas, 1 if host_only else 0, 1 if stable_cache else 0, mask)
+        tune = Tuning(kernel, chunk_tokens, n_ctas, 1 if host_only else 0, 1 if stable_cache else 0, mask, 1 if updatable else 0)
         qp = None if q_pos is None else np.ascontiguousarray(q_pos, dtype=np.int32)
         handle = ctypes.c_void_p()
         self._h = None
@@ -220,6 +222,14 @@ class Plan:
         self.info = PlanInfo()
         _check(lib().aspd_plan_info(self._h, ctypes.addressof(self.info)), "aspd_plan_info")
         self.n_new = self.info.n_new
+
+    def update(self, desc, q_pos=None, stream=None) -> None:
+        """Re-plan in place for the next step of the same batch (see ``aspd_plan_update``)."""
+        req, br, pages = pack_descriptors(desc)
+        qp = None if q_pos is None else np.ascontiguousarray(q_pos, dtype=np.int32)
+        _check(lib().aspd_plan_update(self._h, _ptr(req), _ptr(br), _ptr(pages), len(req), _ptr(qp), _stream(stream)),
+               "aspd_plan_update")
+        _check(lib().aspd_plan_info(self._h, ctypes.addressof(self.info)), "aspd_plan_info")
 
     def items(self) -> np.ndarray:
         items = np.zeros(max(self.info.n_items, 1), dtype=ITEM_DTYPE)

@@ -64,6 +64,17 @@ struct PlanDevice {       // pointers into the plan's single device allocation
 
 }  // namespace aspd
 
+namespace aspd {
+// Byte offsets of the plan's tables inside its device block, and how many entries the
+// length-dependent ones have room for.
+struct PlanLayout {
+  size_t o_items = 0, o_cta = 0, o_visit = 0, o_cdirty = 0, o_dirty = 0, o_tpage = 0, o_trow = 0, o_tpos = 0, o_tvis = 0,
+         o_rb = 0, o_pbase = 0, o_freq = 0, o_status = 0, upload_bytes = 0, o_qcs = 0, o_wso = 0, o_wsml = 0, o_stq = 0,
+         o_stk = 0, o_stv = 0, o_sto = 0, o_stp = 0, device_bytes = 0;
+  size_t cap_items = 0, cap_visit = 0, cap_dirty = 0, cap_partials = 0, n_row_blocks = 0, n_part_base = 0;
+};
+}  // namespace aspd
+
 struct aspd_plan {
   aspd_shape_t shape = {};
   int mode = 0;
@@ -99,6 +110,10 @@ struct aspd_plan {
   // further host copies of the plan's tables (what the device allocation is filled from)
   std::vector<int32_t> cta_item0, part_base, q_pos;
   std::vector<int2> row_blocks;
+  std::vector<int32_t> tok_page, tok_row, cta_dirty0;
+  std::vector<int4> dirty;
+  aspd_tuning_t tune = {};
+  aspd::PlanLayout layout;
 };
 
 namespace aspd {

@@ -316,9 +316,13 @@ int aspd_visible_slots_masked(const aspd_request_t* req, const aspd_branch_t* br
   return ASPD_OK;
 }
 
-int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const aspd_branch_t* br,
-                     const int32_t* page_ids, int n_req, int64_t n_pool_pages, int mode, const int32_t* q_pos,
-                     const aspd_tuning_t* tuning, void* stream, aspd_plan_t** plan_out) {
+static int plan_to_device(aspd_plan* p, cudaStream_t s);
+
+// sm_count_override > 0: plan for a grid of that many SMs without asking the device (aspd_plan_update
+// re-plans on the host for the device the plan already lives on)
+static int plan_create_impl(const aspd_shape_t* shape, const aspd_request_t* req, const aspd_branch_t* br,
+                            const int32_t* page_ids, int n_req, int64_t n_pool_pages, int mode, const int32_t* q_pos,
+                            const aspd_tuning_t* tuning, void* stream, int sm_count_override, aspd_plan_t** plan_out) {
   if (!plan_out) return ASPD_ERR_INVALID_ARG;
   *plan_out = nullptr;
   int rc = check_shape(shape);
@@ -330,7 +334,7 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   const int n_new = aspd_count_new_tokens(req, br, n_req, mode);
   if (n_new < 0) return n_new;
 
-  aspd_tuning_t tune = {ASPD_KERNEL_AUTO, 0, 0, 0, 0, ASPD_MASK_BRANCH_INVISIBLE};
+  aspd_tuning_t tune = {ASPD_KERNEL_AUTO, 0, 0, 0, 0, ASPD_MASK_BRANCH_INVISIBLE, 0};
   if (tuning) tune = *tuning;
   const int ps = shape->page_size, d = shape->head_dim, Hq = shape->n_q_heads, Hkv = shape->n_kv_heads;
   const int G = Hq / Hkv, es = esize_of(shape->dtype);
@@ -350,8 +354,9 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   p->shared_mask = (tune.mask == ASPD_MASK_SHARED && mode == ASPD_MODE_BRANCH) ? 1 : 0;
   p->host_only = tune.host_only; p->n_pool_pages = n_pool_pages; p->device_base = nullptr; p->device_bytes = 0;
   memset(&p->dev, 0, sizeof(p->dev));
-  p->sm_count = 148;
-  if (!tune.host_only) {
+  p->tune = tune;
+  p->sm_count = sm_count_override > 0 ? sm_count_override : 148;
+  if (!tune.host_only && sm_count_override <= 0) {
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
@@ -622,94 +627,159 @@ int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const
   p->n_row_blocks = (int)row_blocks.size();
   p->cta_item0 = cta_item0; p->part_base = part_base; p->row_blocks = row_blocks; p->q_pos = pos;
   p->tok_vis = tok_vis;
+  p->tok_page = tok_page; p->tok_row = tok_row; p->dirty = dirty; p->cta_dirty0 = cta_dirty0;
   if (tune.host_only) { *plan_out = p; return ASPD_OK; }
+  rc = plan_to_device(p, (cudaStream_t)stream);
+  if (rc) { delete p; return rc; }
+  *plan_out = p;
+  return ASPD_OK;
+}
 
-  // ---- one device allocation, one staging blob ------------------------------------------
+int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const aspd_branch_t* br,
+                     const int32_t* page_ids, int n_req, int64_t n_pool_pages, int mode, const int32_t* q_pos,
+                     const aspd_tuning_t* tuning, void* stream, aspd_plan_t** plan_out) {
+  return plan_create_impl(shape, req, br, page_ids, n_req, n_pool_pages, mode, q_pos, tuning, stream, 0, plan_out);
+}
+
+// ---- one device allocation, one staging blob ----------------------------------------------
+// Offsets of the plan's tables inside its device block.  The tables whose size depends on the
+// lengths of the step (items, page list, new-row list, partial records) get `slack` times the room
+// they need now, so that aspd_plan_update can re-plan into the same addresses.
+static void plan_layout(const aspd_plan* p, double slack, aspd::PlanLayout* L) {
+  const aspd_shape_t& sh = p->shape;
+  const int d = sh.head_dim, Hq = sh.n_q_heads, Hkv = sh.n_kv_heads, G = Hq / Hkv, es = esize_of(sh.dtype), n_new = p->n_new;
+  auto cap = [&](size_t n) { return std::max<size_t>(1, (size_t)((double)n * slack) + (slack > 1.0 ? 64 : 0)); };
+  L->cap_items = cap(p->items.size()); L->cap_visit = cap(p->visit.size()); L->cap_dirty = cap(p->dirty.size());
+  L->cap_partials = cap((size_t)p->n_partials);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-  const size_t o_items = take(sizeof(DeviceItem) * std::max(1, p->n_items));
-  const size_t o_cta = take(sizeof(int32_t) * (n_ctas + 1));
-  const size_t o_visit = take(sizeof(int2) * std::max<size_t>(1, visit.size()));
-  const size_t o_cdirty = take(sizeof(int32_t) * (n_ctas + 1));
-  const size_t o_dirty = take(sizeof(int4) * std::max<size_t>(1, dirty.size()));
-  const size_t o_tpage = take(sizeof(int32_t) * std::max(1, n_new));
-  const size_t o_trow = take(sizeof(int32_t) * std::max(1, n_new));
-  const size_t o_tpos = take(sizeof(int32_t) * std::max(1, n_new));
-  const size_t o_tvis = take(sizeof(int4) * std::max(1, n_new));
-  const size_t o_rb = take(sizeof(int2) * std::max<size_t>(1, row_blocks.size()));
-  const size_t o_pbase = take(sizeof(int32_t) * part_base.size());
-  const size_t o_freq = take(sizeof(double) * (d / 2));
-  const size_t o_status = take(sizeof(int32_t) * 2);
-  const size_t upload_bytes = off;
-  const size_t o_qcs = take(sizeof(float2) * std::max(1, n_new) * (d / 2));   // filled on the device from tok_pos and inv_freq
-  const size_t o_wso = take(sizeof(float) * (size_t)std::max(1, p->n_partials) * G * d);
-  const size_t o_wsml = take(sizeof(float2) * (size_t)std::max(1, p->n_partials) * G);
-  const size_t o_stq = take((size_t)es * std::max(1, n_new) * Hq * d);
-  const size_t o_stk = take((size_t)es * std::max(1, n_new) * Hkv * d);
-  const size_t o_stv = take((size_t)es * std::max(1, n_new) * Hkv * d);
-  const size_t o_sto = take((size_t)es * std::max(1, n_new) * Hq * d);
-  const size_t o_stp = take(sizeof(int32_t) * std::max(1, n_new));
-  p->device_bytes = off;
+  L->o_items = take(sizeof(DeviceItem) * L->cap_items);
+  L->o_cta = take(sizeof(int32_t) * (p->n_ctas + 1));
+  L->o_visit = take(sizeof(int2) * L->cap_visit);
+  L->o_cdirty = take(sizeof(int32_t) * (p->n_ctas + 1));
+  L->o_dirty = take(sizeof(int4) * L->cap_dirty);
+  L->o_tpage = take(sizeof(int32_t) * std::max(1, n_new));
+  L->o_trow = take(sizeof(int32_t) * std::max(1, n_new));
+  L->o_tpos = take(sizeof(int32_t) * std::max(1, n_new));
+  L->o_tvis = take(sizeof(int4) * std::max(1, n_new));
+  L->o_rb = take(sizeof(int2) * std::max<size_t>(1, p->row_blocks.size()));
+  L->o_pbase = take(sizeof(int32_t) * p->part_base.size());
+  L->o_freq = take(sizeof(double) * (d / 2));
+  L->o_status = take(sizeof(int32_t) * 2);
+  L->upload_bytes = off;
+  L->o_qcs = take(sizeof(float2) * std::max(1, n_new) * (d / 2));   // filled on the device from tok_pos and inv_freq
+  L->o_wso = take(sizeof(float) * L->cap_partials * G * d);
+  L->o_wsml = take(sizeof(float2) * L->cap_partials * G);
+  L->o_stq = take((size_t)es * std::max(1, n_new) * Hq * d);
+  L->o_stk = take((size_t)es * std::max(1, n_new) * Hkv * d);
+  L->o_stv = take((size_t)es * std::max(1, n_new) * Hkv * d);
+  L->o_sto = take((size_t)es * std::max(1, n_new) * Hq * d);
+  L->o_stp = take(sizeof(int32_t) * std::max(1, n_new));
+  L->device_bytes = off;
+  L->n_row_blocks = p->row_blocks.size(); L->n_part_base = p->part_base.size();
+}
 
-  cudaStream_t s = (cudaStream_t)stream;
-  void* base = nullptr;
-  rc = block_acquire(p->device_bytes, upload_bytes, s, &base, &p->block_bytes, &p->host_block, &p->host_block_bytes);
-  if (rc) { delete p; return rc; }
-  struct { uint8_t* d; uint8_t* data() const { return d; } } blob = {static_cast<uint8_t*>(p->host_block)};
-  memset(blob.data(), 0, upload_bytes);
-  if (p->n_items) memcpy(blob.data() + o_items, p->items.data(), sizeof(DeviceItem) * p->n_items);
-  memcpy(blob.data() + o_cta, cta_item0.data(), sizeof(int32_t) * (n_ctas + 1));
-  if (!visit.empty()) memcpy(blob.data() + o_visit, visit.data(), sizeof(int2) * visit.size());
-  memcpy(blob.data() + o_cdirty, cta_dirty0.data(), sizeof(int32_t) * (n_ctas + 1));
-  if (!dirty.empty()) memcpy(blob.data() + o_dirty, dirty.data(), sizeof(int4) * dirty.size());
+// Assembles the tables in the plan's page-locked buffer, sends them to the device block and fills
+// the cos/sin table there.  The caller has made sure that the buffer's previous copy has completed.
+static int plan_upload(aspd_plan* p, cudaStream_t s) {
+  const aspd::PlanLayout& L = p->layout;
+  const int n_new = p->n_new, d = p->shape.head_dim, n_ctas = p->n_ctas;
+  uint8_t* blob = static_cast<uint8_t*>(p->host_block);
+  memset(blob, 0, L.upload_bytes);
+  if (!p->items.empty()) memcpy(blob + L.o_items, p->items.data(), sizeof(DeviceItem) * p->items.size());
+  memcpy(blob + L.o_cta, p->cta_item0.data(), sizeof(int32_t) * (n_ctas + 1));
+  if (!p->visit.empty()) memcpy(blob + L.o_visit, p->visit.data(), sizeof(int2) * p->visit.size());
+  memcpy(blob + L.o_cdirty, p->cta_dirty0.data(), sizeof(int32_t) * (n_ctas + 1));
+  if (!p->dirty.empty()) memcpy(blob + L.o_dirty, p->dirty.data(), sizeof(int4) * p->dirty.size());
   if (n_new) {
-    memcpy(blob.data() + o_tpage, tok_page.data(), sizeof(int32_t) * n_new);
-    memcpy(blob.data() + o_trow, tok_row.data(), sizeof(int32_t) * n_new);
-    memcpy(blob.data() + o_tpos, pos.data(), sizeof(int32_t) * n_new);
-    memcpy(blob.data() + o_tvis, tok_vis.data(), sizeof(int4) * n_new);
+    memcpy(blob + L.o_tpage, p->tok_page.data(), sizeof(int32_t) * n_new);
+    memcpy(blob + L.o_trow, p->tok_row.data(), sizeof(int32_t) * n_new);
+    memcpy(blob + L.o_tpos, p->q_pos.data(), sizeof(int32_t) * n_new);
+    memcpy(blob + L.o_tvis, p->tok_vis.data(), sizeof(int4) * n_new);
   }
-  if (!row_blocks.empty()) memcpy(blob.data() + o_rb, row_blocks.data(), sizeof(int2) * row_blocks.size());
-  memcpy(blob.data() + o_pbase, part_base.data(), sizeof(int32_t) * part_base.size());
-  double* freq = reinterpret_cast<double*>(blob.data() + o_freq);
-  for (int i = 0; i < d / 2; ++i) freq[i] = pow((double)shape->rope_theta, -2.0 * i / d);
-
-  if (cudaMemcpyAsync(base, blob.data(), upload_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
-    cudaFree(base); cudaFreeHost(p->host_block); delete p; return ASPD_ERR_CUDA;
-  }
+  if (!p->row_blocks.empty()) memcpy(blob + L.o_rb, p->row_blocks.data(), sizeof(int2) * p->row_blocks.size());
+  memcpy(blob + L.o_pbase, p->part_base.data(), sizeof(int32_t) * p->part_base.size());
+  double* freq = reinterpret_cast<double*>(blob + L.o_freq);
+  for (int i = 0; i < d / 2; ++i) freq[i] = pow((double)p->shape.rope_theta, -2.0 * i / d);
+  if (cudaMemcpyAsync(p->device_base, blob, L.upload_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return ASPD_ERR_CUDA;
+  if (p->upload_done) { cudaEventDestroy(p->upload_done); p->upload_done = nullptr; }
   if (cudaEventCreateWithFlags(&p->upload_done, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventRecord(p->upload_done, s) != cudaSuccess) {
     if (p->upload_done) cudaEventDestroy(p->upload_done);
     p->upload_done = nullptr;
     cudaStreamSynchronize(s);                      // no event to tell when the buffer is free again: be done with it now
   }
-  p->streams.push_back(s);
-  // the tables were assembled in the plan's page-locked buffer, which lives as long as the device block
+  if (std::find(p->streams.begin(), p->streams.end(), s) == p->streams.end()) p->streams.push_back(s);
+  // cos/sin of every new token's position (query rotation, fused append): on the device, after the upload
+  return n_new > 0 ? launch_qcs(p, s) : ASPD_OK;
+}
+
+static int plan_to_device(aspd_plan* p, cudaStream_t s) {
+  plan_layout(p, p->tune.updatable ? 1.25 : 1.0, &p->layout);
+  const aspd::PlanLayout& L = p->layout;
+  p->device_bytes = L.device_bytes;
+  void* base = nullptr;
+  int rc = block_acquire(L.device_bytes, L.upload_bytes, s, &base, &p->block_bytes, &p->host_block, &p->host_block_bytes);
+  if (rc) return rc;
   uint8_t* b8 = (uint8_t*)base;
   p->device_base = base;
-  p->dev.items = (const DeviceItem*)(b8 + o_items);
-  p->dev.cta_item0 = (const int32_t*)(b8 + o_cta);
-  p->dev.visit = (const int2*)(b8 + o_visit);
-  p->dev.cta_dirty0 = (const int32_t*)(b8 + o_cdirty);
-  p->dev.dirty = (const int4*)(b8 + o_dirty);
-  p->dev.tok_vis = (const int4*)(b8 + o_tvis);
-  p->dev.row_blocks = (const int2*)(b8 + o_rb);
-
-  p->dev.tok_page = (const int32_t*)(b8 + o_tpage);
-  p->dev.tok_row = (const int32_t*)(b8 + o_trow);
-  p->dev.tok_pos = (const int32_t*)(b8 + o_tpos);
-  p->dev.q_cs = (const float2*)(b8 + o_qcs);
-  p->dev.part_base = (const int32_t*)(b8 + o_pbase);
-  p->dev.inv_freq = (const double*)(b8 + o_freq);
-  p->dev.status = (int32_t*)(b8 + o_status);
+  p->dev.items = (const DeviceItem*)(b8 + L.o_items);
+  p->dev.cta_item0 = (const int32_t*)(b8 + L.o_cta);
+  p->dev.visit = (const int2*)(b8 + L.o_visit);
+  p->dev.cta_dirty0 = (const int32_t*)(b8 + L.o_cdirty);
+  p->dev.dirty = (const int4*)(b8 + L.o_dirty);
+  p->dev.tok_vis = (const int4*)(b8 + L.o_tvis);
+  p->dev.row_blocks = (const int2*)(b8 + L.o_rb);
+  p->dev.tok_page = (const int32_t*)(b8 + L.o_tpage);
+  p->dev.tok_row = (const int32_t*)(b8 + L.o_trow);
+  p->dev.tok_pos = (const int32_t*)(b8 + L.o_tpos);
+  p->dev.q_cs = (const float2*)(b8 + L.o_qcs);
+  p->dev.part_base = (const int32_t*)(b8 + L.o_pbase);
+  p->dev.inv_freq = (const double*)(b8 + L.o_freq);
+  p->dev.status = (int32_t*)(b8 + L.o_status);
   p->dev.work_counter = p->dev.status + 1;
-  p->dev.ws_o = (float*)(b8 + o_wso);
-  p->dev.ws_ml = (float2*)(b8 + o_wsml);
-  p->dev.st_q = b8 + o_stq; p->dev.st_k = b8 + o_stk; p->dev.st_v = b8 + o_stv; p->dev.st_out = b8 + o_sto;
-  p->dev.st_pos = (int32_t*)(b8 + o_stp);
-  // cos/sin of every new token's position (query rotation, fused append): on the device, after the upload
-  if (n_new > 0 && (rc = launch_qcs(p, s)) != ASPD_OK) { cudaFree(base); cudaFreeHost(p->host_block); delete p; return rc; }
-  *plan_out = p;
-  return ASPD_OK;
+  p->dev.ws_o = (float*)(b8 + L.o_wso);
+  p->dev.ws_ml = (float2*)(b8 + L.o_wsml);
+  p->dev.st_q = b8 + L.o_stq; p->dev.st_k = b8 + L.o_stk; p->dev.st_v = b8 + L.o_stv; p->dev.st_out = b8 + L.o_sto;
+  p->dev.st_pos = (int32_t*)(b8 + L.o_stp);
+  rc = plan_upload(p, s);
+  if (rc) {
+    cudaFree(base); cudaFreeHost(p->host_block);
+    p->device_base = nullptr; p->host_block = nullptr;
+  }
+  return rc;
+}
+
+int aspd_plan_update(aspd_plan_t* p, const aspd_request_t* req, const aspd_branch_t* br, const int32_t* page_ids, int n_req,
+                     const int32_t* q_pos, void* stream) {
+  if (!p || p->host_only || !p->device_base) return ASPD_ERR_INVALID_ARG;
+  aspd_tuning_t tune = p->tune;
+  tune.host_only = 1;
+  aspd_plan* t = nullptr;
+  int rc = plan_create_impl(&p->shape, req, br, page_ids, n_req, p->n_pool_pages, p->mode, q_pos, &tune, nullptr, p->sm_count, &t);
+  if (rc) return rc;
+  const aspd::PlanLayout& L = p->layout;
+  if (t->n_new != p->n_new || t->n_ctas != p->n_ctas || t->kernel != p->kernel || t->wide != p->wide || t->dealt != p->dealt ||
+      t->fuse_append != p->fuse_append || t->shared_mask != p->shared_mask || t->kernel != ASPD_KERNEL_MMA ||
+      t->row_blocks.size() != L.n_row_blocks || t->part_base.size() != L.n_part_base ||
+      (t->algorithmic_bytes >= (128LL << 20)) != (p->algorithmic_bytes >= (128LL << 20))) {   // the combine's launch attribute
+    delete t;
+    return ASPD_ERR_UNSUPPORTED;
+  }
+  if (t->items.size() > L.cap_items || t->visit.size() > L.cap_visit || t->dirty.size() > L.cap_dirty ||
+      (size_t)t->n_partials > L.cap_partials) {
+    delete t;
+    return ASPD_ERR_TOO_LARGE;
+  }
+  // the page-locked buffer is written again: its previous copy must be through
+  if (p->upload_done && cudaEventSynchronize(p->upload_done) != cudaSuccess) { delete t; return ASPD_ERR_CUDA; }
+  p->n_req = t->n_req; p->n_items = t->n_items; p->n_partials = t->n_partials; p->n_row_blocks = t->n_row_blocks;
+  p->kv_tokens_read = t->kv_tokens_read; p->algorithmic_bytes = t->algorithmic_bytes;
+  p->items.swap(t->items); p->visit.swap(t->visit); p->tok_vis.swap(t->tok_vis); p->cta_item0.swap(t->cta_item0);
+  p->part_base.swap(t->part_base); p->q_pos.swap(t->q_pos); p->row_blocks.swap(t->row_blocks);
+  p->tok_page.swap(t->tok_page); p->tok_row.swap(t->tok_row); p->cta_dirty0.swap(t->cta_dirty0); p->dirty.swap(t->dirty);
+  delete t;
+  return plan_upload(p, (cudaStream_t)stream);
 }
 
 int aspd_plan_destroy(aspd_plan_t* plan) {
