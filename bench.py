@@ -416,6 +416,42 @@ def run_decode_loop(args):
             if rc:
                 raise SystemExit("bench.py: a step call returned %d" % rc)
         return plan_s
+    if args.loop_graph:
+        # One step captured once; every step re-plans IN PLACE (aspd_plan_update keeps the tables'
+        # addresses) and replays the graph: no kernel launch from the host inside the loop.
+        side = torch.cuda.Stream()
+        torch.cuda.set_stream(side)
+        stream = side.cuda_stream
+        tune_u = B.Tuning(B.KERNEL_AUTO, 0, 0, 0, 1, 0, 1)
+        req0, br0, pages0 = packed[0]
+        if lib.aspd_plan_create(shape_p, req0.ctypes.data, br0.ctypes.data, pages0.ctypes.data, len(req0), wl.n_pool_pages, ph.mode,
+                                None, ctypes.addressof(tune_u), stream, handle_p):
+            raise SystemExit("bench.py: aspd_plan_create failed")
+
+        def one_step():
+            rc = 0
+            for kc, vc, oc in layer_ptrs:
+                rc |= lib.aspd_branch_step(handle, qp, kp, vp, kc, vc, oc, stream)
+            if rc:
+                raise SystemExit("bench.py: a step call returned %d" % rc)
+        one_step()
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            stream = torch.cuda.current_stream().cuda_stream
+            one_step()
+        stream = side.cuda_stream
+
+        def loop():                                  # noqa: F811  (replaces the host-launched loop above)
+            plan_s = 0.0
+            for req, br, pages in packed:
+                t0 = time.perf_counter()
+                rc = lib.aspd_plan_update(handle, req.ctypes.data, br.ctypes.data, pages.ctypes.data, len(req), None, stream)
+                plan_s += time.perf_counter() - t0
+                if rc:
+                    raise SystemExit("bench.py: aspd_plan_update returned %d" % rc)
+                graph.replay()
+            return plan_s
     loop()
     torch.cuda.synchronize()
     sampler = ClockSampler(0)
@@ -441,8 +477,9 @@ def run_decode_loop(args):
         "steps": total_steps, "warmup": n_steps, "ms_per_step": ms / total_steps, "higher_is_better": True, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": "serving-mix, 64 consecutive decoding steps, a new plan every step", "layers": L,
-                   "query_tokens_per_step": n_new, "cuda_graph": False,
-                   "calls_per_step": "aspd_plan_create, %d x aspd_branch_step, aspd_plan_destroy" % L},
+                   "query_tokens_per_step": n_new, "cuda_graph": bool(args.loop_graph),
+                   "calls_per_step": ("aspd_plan_update, replay of the captured step (%d x aspd_branch_step)" % L) if args.loop_graph
+                   else "aspd_plan_create, %d x aspd_branch_step, aspd_plan_destroy" % L},
         "host_ms_per_step": host_s / total_steps * 1e3, "plan_create_call_ms_per_step": plan_s / total_steps * 1e3,
         "plan_create_note": "time inside aspd_plan_create; when the host is ahead of the GPU it includes the wait for a parked block "
                             "whose table upload the GPU has not reached yet (the loop's backpressure)",
@@ -695,6 +732,9 @@ def main():
                     help="call aspd_kv_append and aspd_branch_attn separately instead of aspd_branch_step")
     ap.add_argument("--no-stable-cache", action="store_true", help="create the plan without the stable-cache promise")
     ap.add_argument("--e2e-streams", type=int, default=4, help="plans/streams the layers rotate over in the end-to-end leg")
+    ap.add_argument("--loop-graph", action="store_true",
+                    help="decode-loop: capture the step once and re-plan in place every step (aspd_plan_update) instead of "
+                         "making a new plan and launching from the host")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -656,6 +656,62 @@ def test_plan_per_step_reuses_device_blocks_without_synchronising():
     B.release_cached_memory()
 
 
+def test_plan_update_in_place_keeps_a_captured_graph_valid():
+    """A decode loop over 12 steps: the step (fused append + attention + combine) is captured into a
+    CUDA graph once with an updatable plan; every following step calls aspd_plan_update with the
+    longer branches and replays the graph.  Each step's output equals that of a fresh plan."""
+    import torch
+    E = engine()
+    n_steps = 12
+    prefix, prior = [300, 40, 700], [[20, 9, 131], [5], [64, 3]]
+    wl = W.build_segment_workload("upd", 61, 28, 4, 128, "bf16", 1e6, prefix, [[x + n_steps - 1 for x in p] for p in prior],
+                                  [[1] * len(p) for p in prior])
+    run = E.WorkloadRun(wl)
+    for ph in wl.phases[:-1]:
+        run.step(ph)
+    ph = wl.phases[-1]
+    q, k, v = (E.to_device(x, wl.dtype) for x in (ph.q, ph.k_new, ph.v_new))
+    descs = []
+    for t in range(n_steps):
+        d = {kk: vv.copy() for kk, vv in ph.desc.items()}
+        d["br_kv_len"] = (ph.desc["br_kv_len"] - (n_steps - 1 - t)).astype(np.int32)
+        descs.append(d)
+    k2, v2 = run.cache.k.clone(), run.cache.v.clone()          # a second cache for the fresh plans
+    stream = torch.cuda.Stream()
+    out_g, out_f = torch.zeros_like(q), torch.zeros_like(q)
+    with torch.cuda.stream(stream):
+        # a grid size that stays the same while the lengths grow (a full-size step has the whole GPU at every length)
+        plan = B.Plan(run.shape, descs[0], wl.n_pool_pages, ph.mode, updatable=True, stable_cache=True, stream=stream, n_ctas=8)
+        B.branch_step(plan, q, k, v, run.cache.k, run.cache.v, out_g, stream=stream)     # warm-up outside the capture
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            B.branch_step(plan, q, k, v, run.cache.k, run.cache.v, out_g, stream=stream)
+        for t in range(n_steps):
+            if t > 0:
+                plan.update(descs[t], stream=stream)
+            graph.replay()
+            stream.synchronize()
+            fresh = B.Plan(run.shape, descs[t], wl.n_pool_pages, ph.mode, stream=stream, n_ctas=8)
+            B.branch_step(fresh, q, k, v, k2, v2, out_f, stream=stream)
+            stream.synchronize()
+            assert plan.status(stream) == 0 and fresh.status(stream) == 0
+            np.testing.assert_array_equal(out_g.float().cpu().numpy(), out_f.float().cpu().numpy())
+            fresh.destroy()
+    assert torch.equal(run.cache.k, k2) and torch.equal(run.cache.v, v2)
+    # a step that needs another launch sequence is refused and leaves the plan as it was
+    other = {kk: vv.copy() for kk, vv in descs[-1].items()}
+    other["br_q_len"] = other["br_q_len"].copy(); other["br_q_len"][0] = 0
+    with pytest.raises(B.AspdError) as e:
+        plan.update(other, stream=stream)
+    assert e.value.status == -3                     # ASPD_ERR_UNSUPPORTED
+    with torch.cuda.stream(stream):
+        graph.replay()
+        stream.synchronize()
+    np.testing.assert_array_equal(out_g.float().cpu().numpy(), out_f.float().cpu().numpy())
+    plan.destroy()
+
+
 def test_zero_new_tokens_is_a_no_op():
     E = engine()
     wl = W.build_segment_workload("e", 8, 28, 4, 128, "bf16", 1e6, [20], [[5, 9]], [[1, 1]])
