@@ -739,6 +739,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.op != "step" and int(os.environ.get("RANK", "0")) != 0:
+        return 0          # the side measurements are single-GPU: rank 0 alone runs and prints them
     if args.op == "rerotate":
         return run_rerotate(args)
     if args.op == "serial-chain":
