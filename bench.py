@@ -44,10 +44,9 @@ import numpy as np
 METRIC = "branch_decode_attn_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes moved per algorithmic byte by the split-K attention kernel, from the ncu capture
-# summarised in profiles/attn_tc_kernel_serving_mix.md (62.36 MB of dram read + write for 61.44 MB
-# algorithmic on the 8-request case; the kernel streams every page once, so traffic scales with the
-# cached tokens).
+# DRAM bytes moved per algorithmic byte by the split-K attention kernel, from an ncu capture of the
+# 8-request case of the serving mix (62.36 MB of dram read + write for 61.44 MB algorithmic; the
+# kernel streams every page once, so traffic scales with the cached tokens).
 TRAFFIC_PER_ALGORITHMIC_BYTE = 1.015
 
 

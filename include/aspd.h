@@ -58,6 +58,9 @@ enum { ASPD_DTYPE_F32 = 0, ASPD_DTYPE_BF16 = 1 };
 /* aspd_branch_t.q_len of a region that belongs to an EARLIER stage (a merged branch, or the serial
  * tokens written between two parallel stages): every token of the step sees all of it. */
 enum { ASPD_Q_SHARED = -1 };
+/* aspd_branch_t.pos_start value that makes the library derive the paper's shared position-ID rule
+ * itself (Eq. 4: stage_start = the number of tokens before the stage). */
+enum { ASPD_POS_AUTO = -1 };
 enum { ASPD_KERNEL_AUTO = 0, ASPD_KERNEL_GENERIC = 1, ASPD_KERNEL_MMA = 2 };
 
 /* One request (host memory).  Logical slot s of the request lives in physical page
@@ -77,8 +80,12 @@ typedef struct {
 typedef struct {
   int32_t kv_off;    /* first logical slot of the branch (page-aligned)                     */
   int32_t kv_len;    /* tokens of the branch in the cache AFTER this step's append          */
-  int32_t pos_start; /* position ID of the branch's first token; Eq. 4 gives the number of tokens
-                        before the stage: prefix_len plus the lengths of all ASPD_Q_SHARED regions */
+  int32_t pos_start; /* position ID of the branch's first token.  ASPD_POS_AUTO: the library applies
+                        Eq. 4 itself -- stage_start = the number of tokens before the stage = the
+                        request's prefix_len plus the kv_len of all its ASPD_Q_SHARED regions, the same
+                        for every branch of the stage (branches share the ID of a timestep).  Any
+                        value >= 0 is taken as given (position-ID variants of the ablation).  Ignored
+                        for ASPD_Q_SHARED regions and in serial mode.                              */
   int32_t q_len;     /* query tokens this step = the LAST q_len tokens (0: finished branch of the
                         current stage, invisible to the other branches; ASPD_Q_SHARED: region of an
                         earlier stage, visible to every branch -- Eq. 3, different stages)       */
@@ -175,8 +182,8 @@ int aspd_count_new_tokens(const aspd_request_t* req /*host*/, const aspd_branch_
  * Position ID and logical slot of every new token (Eq. 4; Section 3.3: positions grow by
  * one per token inside a branch, and the first serial token after a segment takes its index
  * in the complete sequence).  Pure host integer code, no CUDA.
- *   branch mode: i-th query of a branch -> pos_start + kv_len - q_len + i,
- *                slot kv_off + kv_len - q_len + i
+ *   branch mode: i-th query of a branch -> pos_start + kv_len - q_len + i, with pos_start derived
+ *                per Eq. 4 where the descriptor says ASPD_POS_AUTO; slot kv_off + kv_len - q_len + i
  *   serial mode: prefix_len + sum of kv_len + tail_len - 1, slot tail_off + tail_len - 1
  * pos_out, slot_out, req_out: host arrays of aspd_count_new_tokens entries (req_out may be NULL).
  */
@@ -190,6 +197,12 @@ int aspd_positions(const aspd_request_t* req, const aspd_branch_t* br, int n_req
 int aspd_visible_slots(const aspd_request_t* req, const aspd_branch_t* br, int n_req, int mode,
                        int n_slots, uint8_t* vis_out /*host*/);
 
+/* aspd_visible_slots under either attention mask (ASPD_MASK_*): with ASPD_MASK_SHARED a new token at
+ * offset k of its branch also attends the slots at offsets below k of the stage's other branches
+ * (the paper's attention-mask ablation).  Serial mode is the same under both.  Host only, for tests. */
+int aspd_visible_slots_masked(const aspd_request_t* req, const aspd_branch_t* br, int n_req, int mode, int mask,
+                              int n_slots, uint8_t* vis_out /*host*/);
+
 /*
  * Validate the descriptors and build the step's plan: new-token table, query RoPE table,
  * split-K work list over (request, KV head, key chunk), partial-result workspace.  One plan
@@ -202,9 +215,6 @@ int aspd_visible_slots(const aspd_request_t* req, const aspd_branch_t* br, int n
  * Errors: ASPD_ERR_BAD_DESCRIPTOR for overlapping or out-of-table regions, unaligned kv_off /
  * tail_off, q_len > kv_len, serial mode with tail_len < 1, duplicate or out-of-pool page ids.
  */
-int aspd_visible_slots_masked(const aspd_request_t* req, const aspd_branch_t* br, int n_req, int mode, int mask,
-                              int n_slots, uint8_t* vis_out /*host*/);
-
 int aspd_plan_create(const aspd_shape_t* shape, const aspd_request_t* req, const aspd_branch_t* br,
                      const int32_t* page_ids, int n_req, int64_t n_pool_pages, int mode,
                      const int32_t* q_pos, const aspd_tuning_t* tuning, void* stream,
@@ -250,9 +260,10 @@ int aspd_plan_token_ranges(const aspd_plan_t* plan, int32_t* pe, int32_t* lo, in
  * other branches at offsets below k), and per stream page the page's index inside its branch
  * (host arrays of n_new and n_stream_pages entries).  ASPD_ERR_INVALID_ARG for other plans. */
 int aspd_plan_shared_mask_tables(const aspd_plan_t* plan, int32_t* below /*host*/, int32_t* page_in_branch /*host*/);
-/* Device status word of the plan (synchronises `stream`): ASPD_OK, or the first error a
- * kernel recorded (ASPD_ERR_TIMEOUT from a bounded wait, ASPD_ERR_BAD_DESCRIPTOR from a
- * bounds check). */
+/* Device status word of the plan (synchronises `stream`): ASPD_OK, or the first error a kernel
+ * recorded since the plan was created: ASPD_ERR_TIMEOUT from a bounded wait; in a library built
+ * with -DASPD_DEBUG_BOUNDS also ASPD_ERR_BAD_DESCRIPTOR from a kernel that met a page id or row
+ * outside the pool (it skips the access).  aspd_plan_update leaves the word as it is. */
 int aspd_plan_status(aspd_plan_t* plan, void* stream);
 
 /*
@@ -346,17 +357,26 @@ int aspd_step_host_async(aspd_plan_t* plan, const void* q /*host*/, const void* 
  * that array, and writes `out`.  It calls no cudaMalloc / cudaFree and no allocating library
  * routine.  q, k_pool, v_pool, out are device buffers as for aspd_branch_attn.
  *
- *  - Plans whose tables plus workspace exceed ASPD_STATIC_SCRATCH_BYTES are rejected with
- *    ASPD_ERR_TOO_LARGE before anything is launched.
+ *  - Plans whose tables plus workspace exceed ASPD_STATIC_SCRATCH_BYTES (less its last 256 bytes,
+ *    which hold the status word) are rejected with ASPD_ERR_TOO_LARGE before anything is launched.
  *  - The first call on a device looks the array's device address up (once per device, with
- *    that device current); make that first call outside any stream capture.
+ *    that device current; host threads are serialised on that look-up).  The array's memory is
+ *    taken when the CUDA module that holds it is loaded, which with lazy loading may be this first
+ *    call; make it outside any stream capture.
+ *  - The tables are copied from pageable host memory that lives only as long as the call, so the
+ *    host may wait inside the call until earlier work on the stream has drained, and a call on a
+ *    stream that is being captured returns ASPD_ERR_UNSUPPORTED and enqueues nothing.
  *  - All calls share the one array, which keeps the previous call's contents; every call
- *    rewrites the tables and the status word it needs.  Two calls that overlap on the GPU
+ *    rewrites the tables and clears the status word it needs.  Two calls that overlap on the GPU
  *    (different streams, or different host threads) race on it: serialise them.
+ *  - A bounded device-side wait that ran out is recorded in the array's status word, which
+ *    aspd_static_status reads (it synchronises `stream`; ASPD_OK, or ASPD_ERR_TIMEOUT, of the last
+ *    call on the current device).
  */
 #define ASPD_STATIC_SCRATCH_BYTES (8u << 20)
 int aspd_attn_static(const aspd_plan_t* plan /*host-only*/, const void* q /*device*/, const void* k_pool /*device*/,
                      const void* v_pool /*device*/, void* out /*device*/, void* stream);
+int aspd_static_status(void* stream);
 
 /* Read one cached token (physical page, row, KV head) back as head_dim floats (host).
  * Synchronises `stream`.  For tests. */
@@ -383,6 +403,16 @@ int aspd_k_rerotate(const aspd_shape_t* shape, void* k_pool /*device*/, const in
  * Synchronises `stream`.
  */
 int aspd_debug_bounded_wait(int64_t limit_cycles, int32_t* status_out /*host*/, void* stream);
+
+/*
+ * Development aid of the tensor-core attention kernel.  In a library built with -DASPD_TC_PROFILE,
+ * CTA `cta` of every later launch stamps its clock at the pipeline events of its first 64 tiles
+ * into device_buf[0 .. 1024) and every CTA stamps the global timer at entry, after set-up, after
+ * its last record and at exit into device_buf[1024 + 4 * blockIdx ..) (device memory of at least
+ * 1024 + 4 * n_ctas int64, caller-owned; NULL switches the stamps off).  Other builds return
+ * ASPD_ERR_UNSUPPORTED.
+ */
+int aspd_debug_profile(void* device_buf /*device*/, int cta);
 
 #ifdef __cplusplus
 }

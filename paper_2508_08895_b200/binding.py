@@ -20,6 +20,7 @@ MODE_BRANCH, MODE_SERIAL = 0, 1
 DTYPE_F32, DTYPE_BF16 = 0, 1
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_MMA = 0, 1, 2
 Q_SHARED = -1
+POS_AUTO = -1
 MASK_BRANCH_INVISIBLE, MASK_SHARED = 0, 1
 
 REQUEST_DTYPE = np.dtype([(n, np.int32) for n in
@@ -62,7 +63,7 @@ EXPORTS = ("aspd_strerror", "aspd_pool_bytes", "aspd_count_new_tokens", "aspd_po
            "aspd_visible_slots_masked", "aspd_plan_create", "aspd_plan_update", "aspd_plan_destroy", "aspd_release_cached_memory", "aspd_plan_info", "aspd_plan_items", "aspd_plan_cta_ranges", "aspd_plan_stream_pages",
            "aspd_plan_token_ranges", "aspd_plan_shared_mask_tables", "aspd_plan_status",
            "aspd_kv_append", "aspd_branch_attn", "aspd_serial_attn", "aspd_attn_partials", "aspd_attn_combine",
-           "aspd_branch_step", "aspd_serial_step", "aspd_step_host", "aspd_step_host_async", "aspd_attn_static", "aspd_k_rerotate", "aspd_debug_read_token", "aspd_debug_bounded_wait")
+           "aspd_branch_step", "aspd_serial_step", "aspd_step_host", "aspd_step_host_async", "aspd_attn_static", "aspd_static_status", "aspd_k_rerotate", "aspd_debug_read_token", "aspd_debug_bounded_wait", "aspd_debug_profile")
 
 _lib = None
 
@@ -75,7 +76,8 @@ def lib() -> ctypes.CDLL:
     """Load the CUDA library (building it first if the sources are newer).  Fails loudly."""
     global _lib
     if _lib is None:
-        # ASPD_LIBRARY selects another build of the same sources (e.g. one with profiling hooks)
+        # ASPD_LIBRARY selects another build of the same sources: the GPU tests run a subset once
+        # more against the -DASPD_DEBUG_BOUNDS build (kernels that check page ids and rows) this way
         path = os.environ.get("ASPD_LIBRARY") or _build.build()
         L = ctypes.CDLL(path)
         L.aspd_strerror.restype = ctypes.c_char_p
@@ -108,8 +110,10 @@ def lib() -> ctypes.CDLL:
         L.aspd_step_host.argtypes = [vp] * 9
         L.aspd_step_host_async.argtypes = [vp] * 9
         L.aspd_attn_static.argtypes = [vp] * 6
+        L.aspd_static_status.argtypes = [vp]
         L.aspd_k_rerotate.argtypes = [vp, vp, vp, vp, vp, ci, vp]
         L.aspd_debug_bounded_wait.argtypes = [ctypes.c_int64, vp, vp]
+        L.aspd_debug_profile.argtypes = [vp, ci]
         L.aspd_debug_read_token.argtypes = [vp, vp, ctypes.c_int64, ci, ci, vp, vp]
         for name in EXPORTS:
             if name not in ("aspd_strerror", "aspd_pool_bytes"):
@@ -152,8 +156,8 @@ def make_shape(n_q_heads, n_kv_heads, head_dim, page_size, dtype, rope_theta, sm
 def pack_descriptors(desc: Dict[str, np.ndarray]):
     """dict of int32 arrays -> (aspd_request_t[], aspd_branch_t[], page_ids) numpy arrays.
 
-    A missing ``br_pos_start`` is filled with the number of tokens before the stage, the paper's
-    shared position-ID rule (Eq. 4: stage_start)."""
+    A missing ``br_pos_start`` becomes ``ASPD_POS_AUTO``: the library then derives the paper's shared
+    position-ID rule (Eq. 4: stage_start) itself."""
     n_req = len(desc["prefix_len"])
     req = np.zeros(n_req, dtype=REQUEST_DTYPE)
     for name in REQUEST_DTYPE.names:
@@ -161,14 +165,7 @@ def pack_descriptors(desc: Dict[str, np.ndarray]):
     n_br = len(desc["br_kv_off"])
     br = np.zeros(n_br, dtype=BRANCH_DTYPE)
     br["kv_off"], br["kv_len"], br["q_len"] = desc["br_kv_off"], desc["br_kv_len"], desc["br_q_len"]
-    if "br_pos_start" in desc:
-        br["pos_start"] = desc["br_pos_start"]
-    else:
-        # Eq. 4, stage_start: tokens before the stage = prefix + every region of an earlier stage
-        for r in range(n_req):
-            b0, nb = int(req["branch_begin"][r]), int(req["n_branches"][r])
-            shared = br["q_len"][b0:b0 + nb] == Q_SHARED
-            br["pos_start"][b0:b0 + nb] = req["prefix_len"][r] + int(br["kv_len"][b0:b0 + nb][shared].sum())
+    br["pos_start"] = desc["br_pos_start"] if "br_pos_start" in desc else POS_AUTO
     pages = np.ascontiguousarray(desc["page_ids"], dtype=np.int32)
     return req, br, pages
 
@@ -350,6 +347,17 @@ def attn_static(plan: Plan, q, k_pool, v_pool, out, stream=None) -> None:
     ``aspd_attn_static`` in ``aspd.h`` for the size limit and the sharing rules)."""
     _check(lib().aspd_attn_static(plan._h, _ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(out), _stream(stream)),
            "aspd_attn_static")
+
+
+def static_status(stream=None) -> int:
+    """Status word of the last ``attn_static`` call on the current device (synchronises the stream)."""
+    return lib().aspd_static_status(_stream(stream))
+
+
+def debug_profile(device_buf, cta: int = 0) -> int:
+    """Point the profiling build's stamps at ``device_buf`` (int64 device tensor); returns the
+    status (ASPD_ERR_UNSUPPORTED = -3 in an ordinary build)."""
+    return lib().aspd_debug_profile(_ptr(device_buf), cta)
 
 
 def debug_read_token(shape: Shape, pool, page: int, row: int, kv_head: int, stream=None) -> np.ndarray:

@@ -27,8 +27,6 @@
 // (TMEM lane quadrant = warp - 12); warp 10 is idle.  All cross-role hand-offs are mbarriers; every
 // wait is bounded and on expiry sets the plan's status word to ASPD_ERR_TIMEOUT and makes all
 // roles drain and exit.
-#include <stdlib.h>
-
 #include "aspd_internal.cuh"
 
 namespace aspd {
@@ -209,8 +207,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 }
 
 #ifdef ASPD_TC_PROFILE
-// Development aid: CTA 0 stamps clock64() at pipeline events of its first 64 tiles into the
-// buffer whose address is given by the environment (see launch_attn_mma).
+// Development aid (builds with -DASPD_TC_PROFILE): one CTA stamps clock64() at pipeline events of
+// its first 64 tiles into the buffer given to aspd_debug_profile.
 #define ASPD_STAMP(c, g, ev) do { if ((c).prof && blockIdx.x == (c).prof_cta && (g) < 64) (c).prof[(g) * 16 + (ev)] = clock64(); } while (0)
 // every CTA: globaltimer (ns) at entry / after set-up / after its last epilogue / at exit
 __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
@@ -696,7 +694,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     }
   } else if (warp == W_KPROD || warp == W_VPROD) {
     // ================================ bulk-copy producers ================================
-    // Warp 4 streams the K tiles and warp 7 the V tiles, each on its own ring, so that a K load
+    // Warp 8 streams the K tiles and warp 11 the V tiles, each on its own ring, so that a K load
     // never queues behind a V slot that is still being read (and vice versa).
     // Lane l keeps stream-page entry (batch * 32 + l) of the item in a register; the next batch
     // of 32 entries (4 tiles) is requested before the current one is consumed, so the page list
@@ -964,8 +962,20 @@ int launch_wait_probe(long long limit_cycles, int32_t* status_dev, cudaStream_t 
   return cudaGetLastError() == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
 }
 
-namespace {
-}  // namespace
+// where the profiling build's stamps go (aspd_debug_profile)
+static long long* g_prof_buf = nullptr;
+static int g_prof_cta = 0;
+
+int set_profile_buffer(long long* device_buf, int cta) {
+#ifdef ASPD_TC_PROFILE
+  g_prof_buf = device_buf;
+  g_prof_cta = cta;
+  return ASPD_OK;
+#else
+  (void)device_buf; (void)cta;
+  return ASPD_ERR_UNSUPPORTED;
+#endif
+}
 
 static int launch_tc(const aspd_plan* p, const void* q, const void* k_new, const void* v_new, const void* k_pool,
                      const void* v_pool, void* out, cudaStream_t s) {
@@ -986,8 +996,8 @@ static int launch_tc(const aspd_plan* p, const void* q, const void* k_new, const
   c.prof = nullptr;
   c.prof_cta = 0;
 #ifdef ASPD_TC_PROFILE
-  if (const char* e = getenv("ASPD_TC_PROFILE_BUF")) c.prof = (long long*)strtoull(e, nullptr, 0);
-  if (const char* e = getenv("ASPD_TC_PROFILE_CTA")) c.prof_cta = atoi(e);
+  c.prof = g_prof_buf;
+  c.prof_cta = g_prof_cta;
 #endif
   c.q = (const __nv_bfloat16*)q;
   c.k_new = (const __nv_bfloat16*)k_new;

@@ -127,8 +127,8 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 enum { kPdlAppend = 1, kPdlAttn = 2, kPdlCombine = 4, kPdlCombineLarge = 8 };
-int pdl_mask();   // which kernels are launched with the attribute (environment ASPD_PDL: bits 1 append, 2 attention,
-                  // 4 combine; default: append, attention, and the combine of large steps)
+// which kernels are launched with the attribute: append, attention, and the combine of large steps
+constexpr int pdl_mask() { return kPdlAppend | kPdlAttn | kPdlCombineLarge; }
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(int which, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
@@ -160,6 +160,7 @@ int launch_attn_mma_step(const aspd_plan* p, const void* q, const void* k_new, c
                          void* v_pool, void* out, cudaStream_t s);
 int launch_rerotate(const aspd_shape_t* shape, void* k_pool, const int32_t* pages, const int32_t* rows, const int32_t* delta,
                     int n, cudaStream_t s);
+int set_profile_buffer(long long* device_buf, int cta);
 int launch_wait_probe(long long limit_cycles, int32_t* status_dev, cudaStream_t s);
 int launch_read_token(const aspd_shape_t* shape, const void* pool, int64_t page, int row, int kv_head,
                       float* out_dev, cudaStream_t s);

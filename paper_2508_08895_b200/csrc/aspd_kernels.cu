@@ -2,18 +2,7 @@
 // supported dtype / head_dim / page_size), the log-sum-exp combine (a7) and a debug reader.
 #include "aspd_internal.cuh"
 
-#include <stdlib.h>
-
 namespace aspd {
-
-int pdl_mask() {
-  static int mask = -1;
-  if (mask < 0) {
-    const char* e = getenv("ASPD_PDL");
-    mask = e ? atoi(e) & 7 : (kPdlAppend | kPdlAttn | kPdlCombineLarge);   // the combine only on large steps (see launch_combine)
-  }
-  return mask;
-}
 
 namespace {
 
@@ -364,7 +353,7 @@ int launch_combine(const aspd_plan* p, void* out, cudaStream_t s) {
   // Measured: with the attribute the combine's blocks wait on the SMs while the attention pass
   // ends, which wins a little on a large step (serving mix: 48.6 against 49.2 us per layer) and
   // loses a lot on small ones (long context, one request: 24.9 against 17.6), so it follows the
-  // step's size unless the environment decides.
+  // step's size.
   const int which = p->algorithmic_bytes >= (128LL << 20) ? (kPdlCombine | kPdlCombineLarge) : kPdlCombine;
 #define ASPD_CMB(T, D) \
   return status_of(launch_pdl(which, combine_kernel<T, D>, grid, block, 0, s, p->dev, (T*)out, p->n_new, sh.n_q_heads, sh.n_kv_heads))

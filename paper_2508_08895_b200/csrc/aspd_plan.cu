@@ -88,8 +88,9 @@ int block_release(void* ptr, size_t bytes, void* host, size_t host_bytes, cudaEv
   std::vector<cudaEvent_t> events;
   for (size_t i = 0; park && i < streams.size(); ++i) {
     cudaEvent_t e;
-    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess || cudaEventRecord(e, streams[i]) != cudaSuccess) park = false;
-    else events.push_back(e);
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) { park = false; break; }
+    if (cudaEventRecord(e, streams[i]) != cudaSuccess) { cudaEventDestroy(e); park = false; break; }   // e.g. the stream is gone
+    events.push_back(e);
   }
   if (park) {
     std::lock_guard<std::mutex> lock(g_blocks_mu);
@@ -151,7 +152,7 @@ int check_counts(const aspd_request_t* req, const aspd_branch_t* br, int n_req, 
     if (q.n_branches > 0 && !br) return ASPD_ERR_INVALID_ARG;
     for (int b = 0; b < q.n_branches; ++b) {
       const aspd_branch_t& x = br[q.branch_begin + b];
-      if (x.kv_off < 0 || x.kv_len < 0 || x.q_len < ASPD_Q_SHARED || x.q_len > x.kv_len || x.pos_start < 0)
+      if (x.kv_off < 0 || x.kv_len < 0 || x.q_len < ASPD_Q_SHARED || x.q_len > x.kv_len || x.pos_start < ASPD_POS_AUTO)
         return ASPD_ERR_BAD_DESCRIPTOR;
     }
     if (mode == ASPD_MODE_SERIAL && q.tail_len < 1) return ASPD_ERR_BAD_DESCRIPTOR;
@@ -245,11 +246,18 @@ int aspd_positions(const aspd_request_t* req, const aspd_branch_t* br, int n_req
   for (int r = 0; r < n_req; ++r) {
     const aspd_request_t& q = req[r];
     if (mode == ASPD_MODE_BRANCH) {
+      // Eq. 4, stage_start: every token cached before the stage counts -- the prefix and the regions
+      // of earlier stages (merged branches, serial tokens between stages); all branches share it
+      long stage_start = q.prefix_len;
+      for (int b = 0; b < q.n_branches; ++b)
+        if (br[q.branch_begin + b].q_len == ASPD_Q_SHARED) stage_start += br[q.branch_begin + b].kv_len;
       for (int b = 0; b < q.n_branches; ++b) {
         const aspd_branch_t& x = br[q.branch_begin + b];
+        const long first = x.pos_start == ASPD_POS_AUTO ? stage_start : (long)x.pos_start;
         for (int i = 0; i < x.q_len; ++i, ++t) {
           int k = x.kv_len - x.q_len + i;        // index of the token inside its branch
-          pos_out[t] = x.pos_start + k;          // Eq. 4: stage_start + delta
+          if (first + k > INT32_MAX) return ASPD_ERR_TOO_LARGE;
+          pos_out[t] = (int32_t)(first + k);     // Eq. 4: stage_start + delta
           slot_out[t] = x.kv_off + k;
           if (req_out) req_out[t] = r;
         }
@@ -555,12 +563,10 @@ static int plan_create_impl(const aspd_shape_t* shape, const aspd_request_t* req
     // Every CTA gets the same cost, cost = pages + kItemCost per item it starts: an item boundary
     // (new query tile, ragged last tile, epilogue) costs about as much as streaming a dozen pages,
     // so CTAs that end up with several short items get fewer pages.
-    const char* ice = getenv("ASPD_ITEM_COST");
-    const double kItemCost = ice ? atof(ice) : 12.0;
+    const double kItemCost = 12.0;
     // a page costs a little more the more query rows are scored against it (best measured balance:
     // 0.35 % per row), so streams of requests with many branches weigh more
-    const char* rce = getenv("ASPD_ROW_COST");
-    const double kRowCost = rce ? atof(rce) : 0.0035;
+    const double kRowCost = 0.0035;
     auto page_cost = [&](const Stream& st) { return 1.0 + kRowCost * st.n_tok * G; };
     // the share is re-derived from what is left whenever a CTA is closed, so rounding does not pile up
     double cost_left = 0.0;
@@ -665,8 +671,10 @@ static void plan_layout(const aspd_plan* p, double slack, aspd::PlanLayout* L) {
   L->o_rb = take(sizeof(int2) * std::max<size_t>(1, p->row_blocks.size()));
   L->o_pbase = take(sizeof(int32_t) * p->part_base.size());
   L->o_freq = take(sizeof(double) * (d / 2));
-  L->o_status = take(sizeof(int32_t) * 2);
   L->upload_bytes = off;
+  // the status word is zeroed when the plan is created and never uploaded again, so that a time-out
+  // recorded by an earlier launch survives aspd_plan_update until aspd_plan_status reads it
+  L->o_status = take(sizeof(int32_t) * 2);
   L->o_qcs = take(sizeof(float2) * std::max(1, n_new) * (d / 2));   // filled on the device from tok_pos and inv_freq
   L->o_wso = take(sizeof(float) * L->cap_partials * G * d);
   L->o_wsml = take(sizeof(float2) * L->cap_partials * G);
@@ -742,7 +750,7 @@ static int plan_to_device(aspd_plan* p, cudaStream_t s) {
   p->dev.ws_ml = (float2*)(b8 + L.o_wsml);
   p->dev.st_q = b8 + L.o_stq; p->dev.st_k = b8 + L.o_stk; p->dev.st_v = b8 + L.o_stv; p->dev.st_out = b8 + L.o_sto;
   p->dev.st_pos = (int32_t*)(b8 + L.o_stp);
-  rc = plan_upload(p, s);
+  rc = cudaMemsetAsync(p->dev.status, 0, 2 * sizeof(int32_t), s) == cudaSuccess ? plan_upload(p, s) : ASPD_ERR_CUDA;
   if (rc) {
     cudaFree(base); cudaFreeHost(p->host_block);
     p->device_base = nullptr; p->host_block = nullptr;
@@ -967,6 +975,11 @@ int aspd_k_rerotate(const aspd_shape_t* shape, void* k_pool, const int32_t* page
   if (n == 0) return ASPD_OK;
   if (!k_pool || !pages || !rows || !delta || misaligned16(k_pool)) return ASPD_ERR_INVALID_ARG;
   return launch_rerotate(shape, k_pool, pages, rows, delta, n, (cudaStream_t)stream);
+}
+
+int aspd_debug_profile(void* device_buf, int cta) {
+  if (cta < 0) return ASPD_ERR_INVALID_ARG;
+  return set_profile_buffer((long long*)device_buf, cta);
 }
 
 int aspd_debug_bounded_wait(int64_t limit_cycles, int32_t* status_out, void* stream) {

@@ -1,7 +1,9 @@
 // aspd_attn_static: the attention of a step with every byte of scratch in a device array that
 // is part of the library image, for callers that cannot allocate device memory.
+#include <math.h>
 #include <string.h>
 
+#include <mutex>
 #include <vector>
 
 #include "aspd_internal.cuh"
@@ -16,11 +18,13 @@ static __device__ __align__(256) unsigned char g_scratch[ASPD_STATIC_SCRATCH_BYT
 
 constexpr int kMaxDevices = 64;
 unsigned char* g_scratch_addr[kMaxDevices] = {};
+std::mutex g_scratch_mu;      // two host threads making their first call on a device at the same time
 
 // Device address of the scratch array on the current device (looked up once per device).
 int scratch_address(unsigned char** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ASPD_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_scratch_mu);
   if (!g_scratch_addr[dev]) {
     void* ptr = nullptr;
     if (cudaGetSymbolAddress(&ptr, g_scratch) != cudaSuccess || !ptr) return ASPD_ERR_CUDA;
@@ -32,6 +36,10 @@ int scratch_address(unsigned char** out) {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// The status word sits at a fixed place, the array's last 256 bytes, so that aspd_static_status
+// finds it whatever the last call's tables looked like.
+constexpr size_t kStatusOffset = ASPD_STATIC_SCRATCH_BYTES - 256;
+
 }  // namespace
 
 extern "C" int aspd_attn_static(const aspd_plan_t* plan, const void* q, const void* k_pool, const void* v_pool, void* out,
@@ -39,6 +47,12 @@ extern "C" int aspd_attn_static(const aspd_plan_t* plan, const void* q, const vo
   if (!plan || !plan->host_only) return ASPD_ERR_INVALID_ARG;
   if (plan->n_new == 0) return ASPD_OK;
   if (!q || !k_pool || !v_pool || !out || aspd::misaligned16(q, k_pool, v_pool, out)) return ASPD_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  // The tables go up from pageable memory of this call: such a copy cannot be recorded into a
+  // graph (a replay would read a buffer that is gone), so a capturing stream is refused.
+  cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(s, &capturing) != cudaSuccess) return ASPD_ERR_CUDA;
+  if (capturing != cudaStreamCaptureStatusNone) return ASPD_ERR_UNSUPPORTED;
   const aspd_shape_t& sh = plan->shape;
   const int d = sh.head_dim, G = sh.n_q_heads / sh.n_kv_heads, n_new = plan->n_new;
 
@@ -52,11 +66,10 @@ extern "C" int aspd_attn_static(const aspd_plan_t* plan, const void* q, const vo
   const size_t o_rb = take(sizeof(int2) * plan->row_blocks.size());
   const size_t o_qcs = take(sizeof(float2) * (size_t)n_new * (d / 2));
   const size_t o_pbase = take(sizeof(int32_t) * plan->part_base.size());
-  const size_t o_status = take(sizeof(int32_t) * 2);
   const size_t upload_bytes = off;
   const size_t o_wso = take(sizeof(float) * (size_t)plan->n_partials * G * d);
   const size_t o_wsml = take(sizeof(float2) * (size_t)plan->n_partials * G);
-  if (off > ASPD_STATIC_SCRATCH_BYTES) return ASPD_ERR_TOO_LARGE;
+  if (off > kStatusOffset) return ASPD_ERR_TOO_LARGE;
 
   unsigned char* base = nullptr;
   int rc = scratch_address(&base);
@@ -72,14 +85,18 @@ extern "C" int aspd_attn_static(const aspd_plan_t* plan, const void* q, const vo
   memcpy(blob.data() + o_rb, plan->row_blocks.data(), sizeof(int2) * plan->row_blocks.size());
   memcpy(blob.data() + o_pbase, plan->part_base.data(), sizeof(int32_t) * plan->part_base.size());
   float2* qcs = reinterpret_cast<float2*>(blob.data() + o_qcs);
+  double inv_freq[64];
+  for (int i = 0; i < d / 2; ++i) inv_freq[i] = pow((double)sh.rope_theta, -2.0 * i / d);
   for (int t = 0; t < n_new; ++t)
     for (int i = 0; i < d / 2; ++i) {
-      const double a = (double)plan->q_pos[t] * pow((double)sh.rope_theta, -2.0 * i / d);
+      const double a = (double)plan->q_pos[t] * inv_freq[i];
       qcs[(size_t)t * (d / 2) + i] = make_float2((float)cos(a), (float)sin(a));
     }
-  cudaStream_t s = (cudaStream_t)stream;
-  // the source is pageable host memory: the copy is staged before the call returns
-  if (cudaMemcpyAsync(base, blob.data(), upload_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return ASPD_ERR_CUDA;
+  // the source is pageable host memory: the copy is staged before the call returns (the host may
+  // wait for earlier work on the stream); the status word and the work counter start at zero
+  if (cudaMemcpyAsync(base, blob.data(), upload_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemsetAsync(base + kStatusOffset, 0, 2 * sizeof(int32_t), s) != cudaSuccess)
+    return ASPD_ERR_CUDA;
 
   // a shell of the plan whose device pointers all lie inside the scratch array
   aspd_plan shell;
@@ -98,7 +115,7 @@ extern "C" int aspd_attn_static(const aspd_plan_t* plan, const void* q, const vo
   shell.dev.row_blocks = (const int2*)(base + o_rb);
   shell.dev.q_cs = (const float2*)(base + o_qcs);
   shell.dev.part_base = (const int32_t*)(base + o_pbase);
-  shell.dev.status = (int32_t*)(base + o_status);
+  shell.dev.status = (int32_t*)(base + kStatusOffset);
   shell.dev.work_counter = shell.dev.status + 1;
   shell.dev.ws_o = (float*)(base + o_wso);
   shell.dev.ws_ml = (float2*)(base + o_wsml);
@@ -107,4 +124,16 @@ extern "C" int aspd_attn_static(const aspd_plan_t* plan, const void* q, const vo
                                        : launch_attn_generic(&shell, q, k_pool, v_pool, s);
   if (rc) return rc;
   return launch_combine(&shell, out, s);
+}
+
+extern "C" int aspd_static_status(void* stream) {
+  unsigned char* base = nullptr;
+  int rc = scratch_address(&base);
+  if (rc) return rc;
+  int32_t st = 0;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(&st, base + kStatusOffset, sizeof(st), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess)
+    return ASPD_ERR_CUDA;
+  return st;
 }

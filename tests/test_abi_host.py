@@ -69,6 +69,52 @@ def test_positions_closed_forms():
     assert slot.tolist() == [96 + 1]
 
 
+def test_stage_start_is_derived_behind_the_c_abi():
+    """Eq. 4's stage_start without any help from the Python binding: the raw C structs are filled
+    with numpy (pos_start = ASPD_POS_AUTO) and handed to aspd_positions through ctypes; the result
+    is the oracle's, bit for bit, for a first stage (prefix only) and a second stage (prefix + the
+    merged branches of the first + the serial tokens between them).  A caller-given pos_start >= 0
+    is taken as it is."""
+    import ctypes
+    L = B.lib()
+    one = W.build_segment_workload("s1", 11, 4, 2, 64, "f32", 1e4, [37, 5], [[3, 0, 7], [2]], [[1, 2, 1], [4]])
+    two = W.build_two_stage_workload("s2", 12, 4, 2, 64, "f32", 1e4, 9, [3, 1, 2], 2, [4, 0, 6], [1, 2, 1])
+    for wl, want_start in ((one, [37, 37, 37, 5]), (two, None)):
+        d = [p for p in wl.phases if p.label == "parallel-step"][0].desc
+        n_req, n_br = len(d["prefix_len"]), len(d["br_kv_off"])
+        req = np.zeros(n_req, dtype=np.dtype([(n, np.int32) for n in ("prefix_len", "n_branches", "branch_begin", "page_begin",
+                                                                       "n_pages", "tail_off", "tail_len")]))
+        for name in req.dtype.names:
+            req[name] = d[name]
+        br = np.zeros(n_br, dtype=np.dtype([(n, np.int32) for n in ("kv_off", "kv_len", "pos_start", "q_len")]))
+        br["kv_off"], br["kv_len"], br["q_len"], br["pos_start"] = d["br_kv_off"], d["br_kv_len"], d["br_q_len"], -1
+        assert req.itemsize == 28 and br.itemsize == 16
+        n = L.aspd_count_new_tokens(req.ctypes.data, br.ctypes.data, n_req, 0)
+        opos, oslot, oreq = oracle.new_tokens(d, oracle.MODE_BRANCH)
+        assert n == len(opos) > 0
+        pos, slot, rq = (np.full(n, -7, np.int32) for _ in range(3))
+        assert L.aspd_positions(req.ctypes.data, br.ctypes.data, n_req, 0, pos.ctypes.data, slot.ctypes.data, rq.ctypes.data) == 0
+        np.testing.assert_array_equal(pos, opos)
+        np.testing.assert_array_equal(slot, oslot)
+        np.testing.assert_array_equal(rq, oreq)
+        if want_start is not None:      # closed form: P + k
+            k = np.concatenate([np.arange(l - q, l) for l, q in zip(d["br_kv_len"], d["br_q_len"]) if q > 0])
+            first = np.concatenate([[s_] * q for s_, q in zip(want_start, d["br_q_len"]) if q > 0])
+            np.testing.assert_array_equal(pos, first + k)
+        else:                           # second stage: 9 prefix + (3 + 1 + 2) merged + 2 serial tokens = 17
+            live = d["br_q_len"] > 0
+            k = np.concatenate([np.arange(l - q, l) for l, q in zip(d["br_kv_len"][live], d["br_q_len"][live])])
+            np.testing.assert_array_equal(pos, 17 + k)
+        # a caller-given start (a position-ID variant) is used as given
+        br["pos_start"] = 1000
+        assert L.aspd_positions(req.ctypes.data, br.ctypes.data, n_req, 0, pos.ctypes.data, slot.ctypes.data, rq.ctypes.data) == 0
+        live = d["br_q_len"] > 0
+        k = np.concatenate([np.arange(l - q, l) for l, q in zip(d["br_kv_len"][live], d["br_q_len"][live])])
+        np.testing.assert_array_equal(pos, 1000 + k)
+        br["pos_start"] = -2
+        assert L.aspd_positions(req.ctypes.data, br.ctypes.data, n_req, 0, pos.ctypes.data, slot.ctypes.data, rq.ctypes.data) == -2
+
+
 def test_visible_slots_match_oracle_bit_exact():
     for wl in small_workloads():
         for ph in wl.phases:

@@ -13,26 +13,14 @@ import oracle
 from oracle.run import OracleRun, run_workload as oracle_run
 from paper_2508_08895_b200 import binding as B, workloads as W
 
-pytestmark = pytest.mark.gpu
+from parity_check import TOL, check, errors
 
-TOL = {"bf16": dict(max_abs=2e-2, mean_abs=2e-3, rel_l2=1e-2), "f32": dict(max_abs=1e-4, mean_abs=1e-5, rel_l2=1e-5)}
+pytestmark = pytest.mark.gpu
 
 
 def engine():
     from paper_2508_08895_b200 import engine as E
     return E
-
-
-def check(gpu, ref, dtype, what=""):
-    gpu = np.asarray(gpu, dtype=np.float64)
-    assert gpu.shape == ref.shape, what
-    assert np.isfinite(gpu).all(), what
-    err = np.abs(gpu - ref)
-    t = TOL[dtype]
-    rel = np.linalg.norm(gpu - ref) / max(np.linalg.norm(ref), 1e-30)
-    assert err.max() <= t["max_abs"], (what, err.max())
-    assert err.mean() <= t["mean_abs"], (what, err.mean())
-    assert rel <= t["rel_l2"], (what, rel)
 
 
 def compare_workload(wl, **kw):
@@ -78,10 +66,18 @@ def test_config3_branch_open_merge_serial(kernel):
     assert len(run.outputs) == 65
     check(run.outputs[0], ref.outputs[0], wl.dtype, "open step (72 queries)")
     check(np.concatenate(run.outputs[1:]), np.concatenate(ref.outputs[1:]), wl.dtype, "64 serial steps")
-    # serial steps only ever wrote the 64 tail rows: everything cached before is bit-identical
+    # The merge moved nothing and the serial steps wrote only tail rows: every page outside the tail
+    # region holds the bytes it held right after the open step, K and V alike.
     import torch
-    changed_k = (run.cache.k != snap[0]).view(-1, 2).any(dim=1).sum().item()
-    assert changed_k <= 64 * wl.Hkv * wl.d
+    d = wl.phases[-1].desc
+    first, last = int(d["tail_off"][0]) // wl.page_size, (int(d["tail_off"][0]) + int(d["tail_len"][0]) - 1) // wl.page_size
+    tail_pages = set(int(x) for x in d["page_ids"][int(d["page_begin"][0]) + first: int(d["page_begin"][0]) + last + 1])
+    assert len(tail_pages) == 4 and int(d["tail_len"][0]) == 64
+    keep = torch.tensor([pg not in tail_pages for pg in range(wl.n_pool_pages)], device=run.cache.k.device)
+    for now, then in ((run.cache.k, snap[0]), (run.cache.v, snap[1])):
+        now, then = now.view(wl.n_pool_pages, -1), then.view(wl.n_pool_pages, -1)
+        assert torch.equal(now[keep], then[keep])
+        assert (now[~keep] != then[~keep]).any()          # the tail pages are the ones that changed
     for (p, s, q), (op, os_, oq) in zip(run.positions, ref.positions):
         np.testing.assert_array_equal(p, op)
     assert run.positions[-1][0].tolist() == [1024 + 72 + 63]
@@ -97,10 +93,36 @@ def test_config5_serving_mix_full_size(kernel):
     """Full size, in the launch configuration the benchmark times (automatic plan)."""
     wl = W.config_serving_mix()
     run, ref = compare_workload(wl, kernel=kernel)
-    # requests with a single branch are plain serial decoding: same result through the serial call
+    # Requests with a single branch are plain serial decoding (N = 1): the same tokens through
+    # aspd_serial_attn over the same cache -- the branch described as the main branch's tail, so the
+    # new token keeps its slot and gets position P + len - 1 either way -- give the same output.
+    import torch
+    E = engine()
     ph = wl.phases[-1]
-    singles = [r for r in range(len(ph.desc["prefix_len"])) if ph.desc["n_branches"][r] == 1]
-    assert singles
+    d = ph.desc
+    singles = [r for r in range(len(d["prefix_len"])) if d["n_branches"][r] == 1 and d["br_q_len"][d["branch_begin"][r]] == 1]
+    assert len(singles) >= 2
+    b_of = [int(d["branch_begin"][r]) for r in singles]
+    sd = {"prefix_len": d["prefix_len"][singles], "n_branches": np.zeros(len(singles), np.int32),
+          "branch_begin": np.zeros(len(singles), np.int32), "page_begin": d["page_begin"][singles], "n_pages": d["n_pages"][singles],
+          "tail_off": d["br_kv_off"][b_of], "tail_len": d["br_kv_len"][b_of],
+          "br_kv_off": np.zeros(0, np.int32), "br_kv_len": np.zeros(0, np.int32), "br_q_len": np.zeros(0, np.int32),
+          "page_ids": d["page_ids"]}
+    sd = {k: np.ascontiguousarray(v, dtype=np.int32) for k, v in sd.items()}
+    pos_b, _, req_b = B.positions(d, W.MODE_BRANCH)
+    rows = [int(np.flatnonzero(req_b == r)[0]) for r in singles]
+    pos_s, slot_s, _ = B.positions(sd, W.MODE_SERIAL)
+    np.testing.assert_array_equal(pos_s, pos_b[rows])
+    plan = B.Plan(run.shape, sd, wl.n_pool_pages, W.MODE_SERIAL, kernel=kernel)
+    q = E.to_device(np.ascontiguousarray(ph.q[rows]), wl.dtype)
+    out = torch.empty_like(q)
+    B.serial_attn(plan, q, run.cache.k, run.cache.v, out)
+    torch.cuda.synchronize()
+    assert plan.status() == 0
+    serial = out.float().cpu().numpy()
+    check(serial, ref.outputs[-1][rows], wl.dtype, "single-branch requests through the serial call")
+    assert np.abs(serial - run.outputs[-1][rows]).max() <= 1e-2
+    plan.destroy()
 
 
 def test_masked_prefill_full_size():
@@ -117,22 +139,31 @@ def test_masked_prefill_full_size():
     assert run.outputs[0].shape[0] == 17069
 
 
-def test_peaked_softmax_variant():
-    """sm_scale x 4: logits ~ N(0, 16), outputs are O(1), so the bounds bite.  The cached keys,
-    the rotated query and the softmax weights fed to the tensor cores are bf16 (relative
-    rounding 2^-9 each) while the oracle keeps everything exact; that perturbs a logit by about
-    4 * 1.6e-3 and an O(1) output by a few 1e-3 on average, a few 1e-2 at the maximum.  The
-    bounds of this variant are derived from that (max-abs 6e-2, mean-abs 4e-3); the relative L2
-    bound stays at 1e-2."""
+# Peaked variant: bounds per kernel, about 1.5 x the errors measured on a B200 (recorded with the
+# derivation in the design notes): the tensor-core path feeds bf16 K', bf16 rotated Q and bf16
+# softmax weights to the MMAs, the generic kernel keeps Q and the weights in fp32.
+PEAKED_TOL = {B.KERNEL_AUTO: dict(max_abs=6e-2, mean_abs=4e-3, rel_l2=1e-2),
+              B.KERNEL_GENERIC: dict(max_abs=6e-2, mean_abs=4e-3, rel_l2=1e-2)}
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_peaked_softmax_variant(kernel, record_property):
+    """sm_scale x 4: logits ~ N(0, 16), outputs are O(1), so the bounds bite.  The cached keys are
+    bf16 on both kernels and, on the tensor-core path, so are the rotated query and the softmax
+    weights (relative rounding 2^-9 each) while the oracle keeps everything exact; that perturbs a
+    logit of standard deviation 4 by several 1e-3 and an O(1) output by a few 1e-3 on average, a few
+    1e-2 at the maximum."""
     wl = W.config_qwen7b_layer()
     wl.sm_scale *= 4.0
     ref = oracle_run(wl)
-    run = engine().run_workload(wl)
+    run = engine().run_workload(wl, kernel=kernel)
     g, r = run.outputs[0].astype(np.float64), ref.outputs[0]
     assert np.abs(r).max() > 0.5
-    err = np.abs(g - r)
-    assert err.max() <= 6e-2 and err.mean() <= 4e-3
-    assert np.linalg.norm(g - r) / np.linalg.norm(r) <= 1e-2
+    mx, mean, rel = errors(g, r)
+    print("peaked variant, kernel %d: max-abs %.3e mean-abs %.3e rel-l2 %.3e" % (kernel, mx, mean, rel))
+    for k, v in (("max_abs", mx), ("mean_abs", mean), ("rel_l2", rel)):
+        record_property(k, v)
+    check(g, r, wl.dtype, "peaked", tol=PEAKED_TOL[kernel])
 
 
 @pytest.mark.parametrize("chunk,n_ctas", [(16, 0), (64, 0), (448, 0), (32768, 0), (16, 3), (0, 1), (48, 37)])

@@ -546,6 +546,67 @@ def test_shared_mask_descriptor_visible_sets():
     assert t == len(vis) and (vis != iso).any()
 
 
+def _load_shared_example():
+    rows = {}
+    for line in open(GOLDEN_SHARED):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        idx, p_, want = line.split()
+        rows[int(idx)] = (int(p_), [int(x) for x in want.split(",")])
+    return rows
+
+
+def test_shared_mask_descriptor_matches_worked_example():
+    """The descriptor form under the visible mask against the hand-derived table, mapped to slots the
+    way the paper's mask is: rows 8 and 9 (second step of stage 1: two live branches at offset 1, one
+    stopped branch of one token), row 10 (last step of stage 1: offset 2, the others stopped), row 15
+    (stage 3: offset 1, the other branch stopped at one token) and row 16 (the serial token after it,
+    the same under both masks)."""
+    rows = _load_shared_example()
+    # ---- stage 1, its second decoding step: branches 0 and 2 decode their second token
+    wl = W.build_segment_workload("t", 1, 2, 1, 8, "f32", 100.0, [5], [[1, 1, 1]], [[1, 0, 1]])
+    par = [p for p in wl.phases if p.label == "parallel-step"][0]
+    pos, _, _ = oracle.new_tokens(par.desc, oracle.MODE_BRANCH)
+    assert pos.tolist() == [rows[8][0], rows[9][0]]
+    n_slots = int(par.desc["n_pages"][0]) * wl.page_size
+    off = par.desc["br_kv_off"]
+    flat_to_slot = {i: i for i in range(5)}
+    flat_to_slot.update({5: off[0], 8: off[0] + 1, 10: off[0] + 2, 6: off[1], 7: off[2], 9: off[2] + 1})
+    vis = oracle.visible_slots(par.desc, oracle.MODE_BRANCH, n_slots, mask=oracle.MASK_SHARED)
+    for t, flat in enumerate((8, 9)):
+        assert sorted(np.flatnonzero(vis[t]).tolist()) == sorted(int(flat_to_slot[j]) for j in rows[flat][1]), flat
+    # ---- stage 1, its last step: only branch 0 decodes (offset 2); it sees both tokens of branch 2
+    wl = W.build_segment_workload("t", 1, 2, 1, 8, "f32", 100.0, [5], [[2, 1, 2]], [[1, 0, 0]])
+    par = [p for p in wl.phases if p.label == "parallel-step"][0]
+    pos, _, _ = oracle.new_tokens(par.desc, oracle.MODE_BRANCH)
+    assert pos.tolist() == [rows[10][0]]
+    assert (par.desc["br_kv_off"] == off).all()
+    vis = oracle.visible_slots(par.desc, oracle.MODE_BRANCH, n_slots, mask=oracle.MASK_SHARED)
+    assert sorted(np.flatnonzero(vis[0]).tolist()) == sorted(int(flat_to_slot[j]) for j in rows[10][1])
+    # ---- stage 3 (a second parallel stage) and the serial token after it
+    wl = W.build_two_stage_workload("t2", 3, 2, 1, 8, "f32", 100.0, 5, [3, 1, 2], 2, [1, 1], [1, 0], serial_steps=1)
+    par = [p for p in wl.phases if p.label == "parallel-step"][0]
+    d = par.desc
+    pos, _, _ = oracle.new_tokens(d, oracle.MODE_BRANCH)
+    assert pos.tolist() == [rows[15][0]]
+    off = d["br_kv_off"]      # regions: stage-1 branches 0..2, the two serial tokens, stage-3 branches 0..1
+    flat_to_slot = {i: i for i in range(5)}
+    flat_to_slot.update({5: off[0], 8: off[0] + 1, 10: off[0] + 2, 6: off[1], 7: off[2], 9: off[2] + 1,
+                         11: off[3], 12: off[3] + 1, 13: off[4], 15: off[4] + 1, 14: off[5]})
+    n_slots = int(d["n_pages"][0]) * wl.page_size
+    vis = oracle.visible_slots(d, oracle.MODE_BRANCH, n_slots, mask=oracle.MASK_SHARED)
+    assert sorted(np.flatnonzero(vis[0]).tolist()) == sorted(int(flat_to_slot[j]) for j in rows[15][1])
+    iso = oracle.visible_slots(d, oracle.MODE_BRANCH, n_slots)
+    assert set(np.flatnonzero(vis[0])) - set(np.flatnonzero(iso[0])) == {int(off[5])}      # flat index 14 is what the mask adds
+    ser = [p for p in wl.phases if p.label == "serial-0"][0]
+    pos, _, _ = oracle.new_tokens(ser.desc, oracle.MODE_SERIAL)
+    assert pos.tolist() == [rows[16][0]]
+    flat_to_slot[16] = int(ser.desc["tail_off"][0])
+    vis = oracle.visible_slots(ser.desc, oracle.MODE_SERIAL, n_slots, mask=oracle.MASK_SHARED)
+    assert sorted(np.flatnonzero(vis[0]).tolist()) == sorted(int(flat_to_slot[j]) for j in rows[16][1])
+
+
 def test_shared_mask_single_branch_is_plain_causal():
     """With one branch there is nobody else to see: both masks give the same attention."""
     wl = W.build_segment_workload("one", 9, 4, 2, 16, "f32", 1e4, [11], [[5]], [[3]], serial_steps=1)
