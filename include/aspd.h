@@ -303,6 +303,12 @@ int aspd_serial_attn(aspd_plan_t* plan, const void* q /*device*/, const void* k_
 int aspd_attn_partials(aspd_plan_t* plan, const void* q /*device*/, const void* k_pool /*device*/,
                        const void* v_pool /*device*/, void* stream);
 int aspd_attn_combine(aspd_plan_t* plan, void* out /*device*/, void* stream);
+/* The first half of aspd_branch_step / aspd_serial_step alone, for plans whose step fuses the append
+ * (aspd_plan_info_t.fused_append = 1 and direct_output = 0): the attention pass that first writes
+ * the step's new K/V rows and then leaves the (max, sum, O) records; aspd_attn_combine completes
+ * it.  ASPD_ERR_UNSUPPORTED for other plans.  For profilers and the benchmark's kernel timing. */
+int aspd_step_partials(aspd_plan_t* plan, const void* q /*device*/, const void* k_new /*device*/,
+                       const void* v_new /*device*/, void* k_pool /*device*/, void* v_pool /*device*/, void* stream);
 
 /*
  * a3 + a4-a7 (or a3 + a9) in one call: the step's new K/V rows are written into the cache by the
@@ -321,8 +327,14 @@ int aspd_serial_step(aspd_plan_t* plan, const void* q /*device*/, const void* k_
 
 /*
  * The whole step (a3-a7 or a3 + a9, by the plan's mode) from HOST buffers: copies q, k_new,
- * v_new, pos to staging memory the plan owns, runs append + attention, copies out back, all
- * on `stream`, then synchronises it.  The pools stay on the device (they are the state).
+ * v_new to staging memory the plan owns, runs the step, copies out back, all on `stream`, then
+ * synchronises it.  The pools stay on the device (they are the state).
+ *   - When pos equals the position IDs the plan derived (aspd_positions, or its q_pos), which is
+ *     compared on the host, the step is aspd_branch_step / aspd_serial_step (new rows written by
+ *     the attention pass where the plan allows) and pos is not copied; otherwise pos goes up too
+ *     and the step is aspd_kv_append with those positions followed by the attention call.
+ *   - When k_new starts where q ends and v_new where k_new ends (one packed host buffer), one copy
+ *     moves all three.
  */
 int aspd_step_host(aspd_plan_t* plan, const void* q /*host*/, const void* k_new /*host*/,
                    const void* v_new /*host*/, const int32_t* pos /*host*/, void* k_pool /*device*/,

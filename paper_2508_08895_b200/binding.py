@@ -62,7 +62,7 @@ class AspdError(RuntimeError):
 EXPORTS = ("aspd_strerror", "aspd_pool_bytes", "aspd_count_new_tokens", "aspd_positions", "aspd_visible_slots",
            "aspd_visible_slots_masked", "aspd_plan_create", "aspd_plan_update", "aspd_plan_destroy", "aspd_release_cached_memory", "aspd_plan_info", "aspd_plan_items", "aspd_plan_cta_ranges", "aspd_plan_stream_pages",
            "aspd_plan_token_ranges", "aspd_plan_shared_mask_tables", "aspd_plan_status",
-           "aspd_kv_append", "aspd_branch_attn", "aspd_serial_attn", "aspd_attn_partials", "aspd_attn_combine",
+           "aspd_kv_append", "aspd_branch_attn", "aspd_serial_attn", "aspd_attn_partials", "aspd_attn_combine", "aspd_step_partials",
            "aspd_branch_step", "aspd_serial_step", "aspd_step_host", "aspd_step_host_async", "aspd_attn_static", "aspd_static_status", "aspd_k_rerotate", "aspd_debug_read_token", "aspd_debug_bounded_wait", "aspd_debug_profile")
 
 _lib = None
@@ -105,6 +105,7 @@ def lib() -> ctypes.CDLL:
         L.aspd_serial_attn.argtypes = [vp] * 6
         L.aspd_attn_partials.argtypes = [vp] * 5
         L.aspd_attn_combine.argtypes = [vp] * 3
+        L.aspd_step_partials.argtypes = [vp] * 7
         L.aspd_branch_step.argtypes = [vp] * 8
         L.aspd_serial_step.argtypes = [vp] * 8
         L.aspd_step_host.argtypes = [vp] * 9
@@ -296,6 +297,11 @@ def attn_partials(plan: Plan, q, k_pool, v_pool, stream=None) -> None:
 
 def attn_combine(plan: Plan, out, stream=None) -> None:
     _check(lib().aspd_attn_combine(plan._h, _ptr(out), _stream(stream)), "aspd_attn_combine")
+
+
+def step_partials(plan: Plan, q, k_new, v_new, k_pool, v_pool, stream=None) -> None:
+    _check(lib().aspd_step_partials(plan._h, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pool), _ptr(v_pool), _stream(stream)),
+           "aspd_step_partials")
 
 
 def branch_step(plan: Plan, q, k_new, v_new, k_pool, v_pool, out, stream=None) -> None:

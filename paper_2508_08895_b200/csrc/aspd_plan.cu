@@ -876,6 +876,16 @@ int aspd_attn_partials(aspd_plan_t* p, const void* q, const void* k_pool, const 
                                       : launch_attn_generic(p, q, k_pool, v_pool, s);
 }
 
+int aspd_step_partials(aspd_plan_t* p, const void* q, const void* k_new, const void* v_new, void* k_pool, void* v_pool,
+                       void* stream) {
+  if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
+  if (p->n_new == 0) return ASPD_OK;
+  if (!q || !k_new || !v_new || !k_pool || !v_pool || misaligned16(q, k_new, v_new, k_pool, v_pool)) return ASPD_ERR_INVALID_ARG;
+  if (!(p->kernel == ASPD_KERNEL_MMA && p->fuse_append) || attn_mma_writes_output(p)) return ASPD_ERR_UNSUPPORTED;
+  note_stream(p, stream);
+  return launch_attn_mma_step(p, q, k_new, v_new, k_pool, v_pool, nullptr, (cudaStream_t)stream);
+}
+
 int aspd_attn_combine(aspd_plan_t* p, void* out, void* stream) {
   if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
   if (p->n_new == 0) return ASPD_OK;
@@ -946,14 +956,29 @@ int aspd_step_host_async(aspd_plan_t* p, const void* q, const void* k_new, const
   const aspd_shape_t& sh = p->shape;
   const size_t es = esize_of(sh.dtype);
   const size_t qb = es * p->n_new * sh.n_q_heads * sh.head_dim, kb = es * p->n_new * sh.n_kv_heads * sh.head_dim;
-  if (cudaMemcpyAsync(p->dev.st_q, q, qb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(p->dev.st_k, k_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(p->dev.st_v, v_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(p->dev.st_pos, pos, sizeof(int32_t) * p->n_new, cudaMemcpyHostToDevice, s) != cudaSuccess)
+  // The staging areas of q, k_new and v_new lie back to back in the plan's block; when the caller's
+  // three buffers do too (one packed host buffer), one copy moves them all.
+  const char* qh = static_cast<const char*>(q);
+  const bool packed = static_cast<const char*>(k_new) == qh + qb && static_cast<const char*>(v_new) == qh + qb + kb &&
+                      static_cast<char*>(p->dev.st_k) == static_cast<char*>(p->dev.st_q) + qb &&
+                      static_cast<char*>(p->dev.st_v) == static_cast<char*>(p->dev.st_q) + qb + kb;
+  if (packed) {
+    if (cudaMemcpyAsync(p->dev.st_q, q, qb + 2 * kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return ASPD_ERR_CUDA;
+  } else if (cudaMemcpyAsync(p->dev.st_q, q, qb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+             cudaMemcpyAsync(p->dev.st_k, k_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+             cudaMemcpyAsync(p->dev.st_v, v_new, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) {
     return ASPD_ERR_CUDA;
-  int rc = launch_append(p, p->dev.st_k, p->dev.st_v, p->dev.st_pos, k_pool, v_pool, s);
-  if (rc) return rc;
-  rc = run_attn(p, p->mode, p->dev.st_q, k_pool, v_pool, p->dev.st_out, stream);
+  }
+  int rc;
+  if (memcmp(pos, p->q_pos.data(), sizeof(int32_t) * p->n_new) == 0) {
+    // the caller's position IDs are the plan's (the usual case): they are on the device already,
+    // and the step may write the new rows inside the attention pass
+    rc = run_step(p, p->mode, p->dev.st_q, p->dev.st_k, p->dev.st_v, k_pool, v_pool, p->dev.st_out, stream);
+  } else {
+    if (cudaMemcpyAsync(p->dev.st_pos, pos, sizeof(int32_t) * p->n_new, cudaMemcpyHostToDevice, s) != cudaSuccess) return ASPD_ERR_CUDA;
+    rc = launch_append(p, p->dev.st_k, p->dev.st_v, p->dev.st_pos, k_pool, v_pool, s);
+    if (rc == ASPD_OK) rc = run_attn(p, p->mode, p->dev.st_q, k_pool, v_pool, p->dev.st_out, stream);
+  }
   if (rc) return rc;
   if (cudaMemcpyAsync(out, p->dev.st_out, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return ASPD_ERR_CUDA;
   return ASPD_OK;

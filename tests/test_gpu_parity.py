@@ -142,8 +142,10 @@ def test_masked_prefill_full_size():
 # Peaked variant: bounds per kernel, about 1.5 x the errors measured on a B200 (recorded with the
 # derivation in the design notes): the tensor-core path feeds bf16 K', bf16 rotated Q and bf16
 # softmax weights to the MMAs, the generic kernel keeps Q and the weights in fp32.
-PEAKED_TOL = {B.KERNEL_AUTO: dict(max_abs=6e-2, mean_abs=4e-3, rel_l2=1e-2),
-              B.KERNEL_GENERIC: dict(max_abs=6e-2, mean_abs=4e-3, rel_l2=1e-2)}
+# Measured: tensor-core kernel max-abs 3.5e-2, mean-abs 2.0e-3, rel-L2 6.0e-3; generic kernel 1.9e-2,
+# 1.5e-3, 4.5e-3.
+PEAKED_TOL = {B.KERNEL_AUTO: dict(max_abs=5.5e-2, mean_abs=3e-3, rel_l2=9e-3),
+              B.KERNEL_GENERIC: dict(max_abs=3e-2, mean_abs=2.4e-3, rel_l2=7e-3)}
 
 
 @pytest.mark.parametrize("kernel", KERNELS)
@@ -331,6 +333,23 @@ def test_step_host_matches_device_path():
     for o in outs:
         np.testing.assert_array_equal(o.float().numpy(), dev)
     assert plan.status() == 0 and plan_b.status() == 0
+    # q, k_new, v_new packed into one host buffer: a single copy carries them
+    packed = torch.cat([q.reshape(-1), k.reshape(-1), v.reshape(-1)]).pin_memory()
+    nq, nk = q.numel(), k.numel()
+    out_p = torch.zeros_like(q).pin_memory()
+    B.step_host(plan, packed[:nq], packed[nq:nq + nk], packed[nq + nk:], pos_h, run.cache.k, run.cache.v, out_p)
+    np.testing.assert_array_equal(out_p.float().numpy(), dev)
+    # position IDs that are not the plan's (a position-ID variant for the keys): they are copied and
+    # the append kernel uses them -- same result as aspd_kv_append + aspd_branch_attn on the device
+    pos5 = np.ascontiguousarray(pos + 5)
+    out_v = torch.zeros_like(q).pin_memory()
+    B.step_host(plan, q, k, v, pos5, run.cache.k, run.cache.v, out_v)
+    out_d = torch.empty_like(q, device="cuda")
+    B.kv_append(plan, k.cuda(), v.cuda(), torch.from_numpy(pos5).cuda(), run.cache.k, run.cache.v)
+    B.branch_attn(plan, q.cuda(), run.cache.k, run.cache.v, out_d)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(out_v.float().numpy(), out_d.float().cpu().numpy())
+    assert np.abs(out_v.float().numpy() - dev).max() > 1e-3
     plan.destroy(); plan_b.destroy()
 
 
