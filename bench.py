@@ -252,17 +252,27 @@ def time_replays(run, reps, warmup=3):
 
 
 def attention_kernel_call(plan, mode, q_d, k_d, v_d, fused):
-    """The call that launches ONLY the attention kernel the step really runs: the fused pass that
-    also writes the new rows (aspd_step_partials), the plain split-K pass (aspd_attn_partials), or,
-    for plans whose kernel writes the output itself, the attention call (a single launch)."""
+    """The call that launches ONLY the attention kernel the step really runs: for plans whose kernel
+    writes the output itself (single-launch plans, plans that deal whole streams) the step or
+    attention call, which is that one launch; otherwise the fused pass that also writes the new rows
+    (aspd_step_partials) or the plain split-K pass (aspd_attn_partials)."""
     from paper_2508_08895_b200 import binding as B, workloads as W
     info = plan.info
-    if info.direct_output:
+    if info.single_launch and fused and info.fused_append:       # the step is this one launch
+        fstep = B.branch_step if mode == W.MODE_BRANCH else B.serial_step
+        return lambda c, o: fstep(plan, q_d, k_d, v_d, c.k, c.v, o)
+    if info.direct_output or info.single_launch:
         attn = B.branch_attn if mode == W.MODE_BRANCH else B.serial_attn
         return lambda c, o: attn(plan, q_d, c.k, c.v, o)
     if fused and info.fused_append:
         return lambda c, o: B.step_partials(plan, q_d, k_d, v_d, c.k, c.v)
     return lambda c, o: B.attn_partials(plan, q_d, c.k, c.v)
+
+
+def launches_per_layer(info, fused):
+    """Kernel launches of one layer's step: the append kernel unless the attention pass writes the
+    new rows itself, the attention pass, the combine unless the attention pass writes the output."""
+    return (0 if (fused and info.fused_append) else 1) + 1 + (0 if (info.direct_output or info.single_launch) else 1)
 
 
 def measure_step_workload(wl, layers, steps, warmup, plan_kw=None, fused=True, use_graph=True, sample_clocks=True, device_index=0):
@@ -328,7 +338,7 @@ def measure_step_workload(wl, layers, steps, warmup, plan_kw=None, fused=True, u
     res = {"layers": L, "query_tokens": int(plan.n_new), "kv_tokens_per_layer": int(info.kv_tokens_read),
            "alg_bytes": int(info.algorithmic_bytes), "step_ms": step_ms, "step_us_per_layer": step_ms / L * 1e3,
            "kernel_us": kernel_ms * 1e3, "kernel_us_isolated": float(np.median(iso)), "clocks": clocks,
-           "launches_per_layer": (2 if (fused and info.fused_append) or info.direct_output else 3), "layers_agree": bool(same),
+           "launches_per_layer": launches_per_layer(info, fused), "layers_agree": bool(same),
            "n_ctas": int(info.n_ctas), "work_items": int(info.n_items), "kernel": {1: "generic", 2: "mma"}[info.kernel],
            "fused_append": bool(info.fused_append), "direct_output": bool(info.direct_output)}
     return res, dict(plan=plan, shape=shape, caches=caches, outs=outs, q_d=q_d, k_d=k_d, v_d=v_d, pos=pos, pos_d=pos_d, ph=ph,
@@ -454,7 +464,8 @@ def measure_serial_chain(args):
             B.kv_append(plan, k_d, v_d, pos_d, c.k, c.v)
         torch.cuda.synchronize()
         plan.destroy()
-    plans = [B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode, stable_cache=True) for ph in serial]
+    combine = {"auto": B.COMBINE_AUTO, "kernel": B.COMBINE_KERNEL, "fused": B.COMBINE_FUSED}[getattr(args, "combine", "auto")]
+    plans = [B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode, stable_cache=True, combine=combine) for ph in serial]
     qkv = [tuple(E.to_device(x, wl.dtype) for x in (ph.q, ph.k_new, ph.v_new)) for ph in serial]
     outs = [torch.empty_like(q) for q, _, _ in qkv]
     alg = float(sum(pl.info.algorithmic_bytes for pl in plans))
@@ -487,7 +498,7 @@ def measure_serial_chain(args):
         raise SystemExit("bench.py: device status")
     peak, peak_kind = measured_peaks()
     gbs = alg * L * reps / (ms * 1e-3) / 1e9
-    launches = sum(2 if pl.info.fused_append else 3 for pl in plans) * L * reps
+    launches = sum(launches_per_layer(pl.info, True) for pl in plans) * L * reps
     line = ({
         "op": "serial-chain", "metric": "serial_decode_steps_per_second", "value": n_serial * reps / (ms * 1e-3), "unit": "steps/s",
         "n_gpus": 1, "steps": reps, "warmup": max(args.warmup, 3), "ms_per_step": ms / reps, "higher_is_better": True,
@@ -628,7 +639,7 @@ def run_decode_loop(args):
         "plan_create_note": "time inside aspd_plan_create; when the host is ahead of the GPU it includes the wait for a parked block "
                             "whose table upload the GPU has not reached yet (the loop's backpressure)",
         "hbm_gbs": gbs, "hbm_frac_of_measured": gbs / peak, "peak_kind": "of " + peak_kind,
-        "gpu_launches": 2 * L * total_steps + total_steps, "clocks": clocks}))
+        "gpu_launches": L * total_steps + total_steps, "clocks": clocks}))
     return 0
 
 
@@ -652,7 +663,8 @@ def run_ours(args):
     fused = not args.separate_append
     # decode loop: a layer's pools are written only by that layer's own step, so the plan may carry
     # the stable-cache promise (the kernel starts fetching before the previous layer's combine ends)
-    plan_kw = dict(kernel=kernel, chunk_tokens=args.chunk, n_ctas=args.ctas, stable_cache=not args.no_stable_cache)
+    plan_kw = dict(kernel=kernel, chunk_tokens=args.chunk, n_ctas=args.ctas, stable_cache=not args.no_stable_cache,
+                   combine={"auto": B.COMBINE_AUTO, "kernel": B.COMBINE_KERNEL, "fused": B.COMBINE_FUSED}[args.combine])
 
     def barrier():
         if world > 1:
@@ -810,9 +822,10 @@ def run_ours(args):
                        "chunk_tokens": info.chunk_tokens, "work_items": info.n_items, "n_ctas": info.n_ctas,
                        "l2": "footprint %.1f GB of distinct K/V pools per step, far above L2" % (alg * L / 1e9),
                        "layers_agree": bool(same), "cuda_graph": not args.no_graph, "stable_cache": not args.no_stable_cache,
-                       "calls_per_layer": (step_name + (" (append fused into the attention pass) -> combine" if info.fused_append
-                                                       else " (append kernel -> attention pass writing the output)" if info.direct_output
-                                                       else " (append kernel -> attention pass -> combine)")) if fused
+                       "launches_per_layer": launches_per_layer(info, fused), "combine": "inside the attention kernel" if info.single_launch
+                       else "none needed" if info.direct_output else "combine kernel",
+                       "calls_per_layer": (step_name + (" (new rows written by the attention pass)" if info.fused_append else " (append kernel, attention pass)")
+                                           + ("" if info.single_launch or info.direct_output else " -> combine kernel")) if fused
                        else "aspd_kv_append -> " + attn_name},
             "hbm_gbs": alg * L * args.steps / (ms * 1e-3) / 1e9,
             "hbm_frac_of_measured": alg * L * args.steps / (ms * 1e-3) / 1e9 / peak,
@@ -836,7 +849,7 @@ def run_ours(args):
                              "layers rotating over %d plans on %d streams, one synchronisation per step" % (n_e, n_e)},
             "single_call_us": {"median": float(np.median(lat)), "best": float(np.min(lat)), "calls": len(lat),
                                "what": "one layer's step call launched from the host, CUDA events around it"},
-            "gpu_launches": (2 if (fused and info.fused_append) or info.direct_output else 3) * L * args.steps,
+            "gpu_launches": launches_per_layer(info, fused) * L * args.steps,
             "clocks": clocks,
         }
         if mhz:
@@ -914,6 +927,8 @@ def main():
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "mma"])
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--ctas", type=int, default=0)
+    ap.add_argument("--combine", default="auto", choices=["auto", "kernel", "fused"],
+                    help="where the split-K records are merged: a combine launch, or inside the attention kernel (one launch per layer)")
     ap.add_argument("--requests", type=int, default=0, help="serving-mix only: number of requests (default 32)")
     ap.add_argument("--cpu-budget", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -117,7 +117,18 @@ typedef struct {
                            stream has finished.  0 (default): full stream ordering for the pools */
   int32_t mask;         /* ASPD_MASK_*: attention mask of a parallel step (default: branch-invisible) */
   int32_t updatable;    /* 1: leave room in the plan's tables (25 %) for aspd_plan_update                */
+  int32_t combine;      /* ASPD_COMBINE_*: where a7 (the merge of a token's split-K records) runs        */
 } aspd_tuning_t;
+
+/* a7 of a stream-K plan of the tensor-core kernel.  KERNEL: the separate combine launch (what AUTO
+ * takes: it measured faster on every workload of the benchmark).  FUSED: one launch per layer --
+ * every CTA counts the records of a (token, KV head) as it stores its own, and the CTA that stores
+ * the last one merges them all, in record order, and writes the output (no CTA ever waits for
+ * another); a key stream that lies inside one CTA is normalised and written by that CTA without
+ * any record.  Both give the same bits.  FUSED is honoured where the plan allows it (not the
+ * generic kernel, which keeps the combine launch, and not plans that deal whole streams, which
+ * need no merge at all); aspd_plan_info_t.single_launch says what the plan does. */
+enum { ASPD_COMBINE_AUTO = 0, ASPD_COMBINE_KERNEL = 1, ASPD_COMBINE_FUSED = 2 };
 
 /* Attention mask of a parallel step.  BRANCH_INVISIBLE is the paper's mask (its Eq. 2-3).  SHARED
  * is the visible mask of its attention-mask ablation, read as "only the order of the position IDs
@@ -143,7 +154,7 @@ typedef struct {
   int32_t part_slot;  /* which partial record of (token, KV head) this item writes           */
   int32_t request;
   int32_t row_block;  /* index of the item's block of query tokens among all blocks of the step */
-  int32_t reserved;
+  int32_t n_parts;    /* items the key stream of (row block, KV head) was cut into = records per row */
 } aspd_item_t;
 
 typedef struct {
@@ -161,7 +172,8 @@ typedef struct {
   int32_t max_rows_per_item;/* query rows (tokens x group heads) an item may carry: 64 or 128       */
   int32_t dealt;            /* 1: whole streams dealt to the CTAs (every row block has a page list of its
                                own, so n_stream_pages counts shared pages once per row block); 0: stream-K cuts */
-  int32_t reserved;
+  int32_t single_launch;    /* 1: the attention kernel merges the split-K records itself (ASPD_COMBINE_FUSED): the
+                               attention and step calls are one launch; 0: a combine launch follows      */
   int64_t workspace_bytes;  /* device memory the plan holds                                 */
   int64_t kv_tokens_read;   /* cached tokens the step must read (each once)                 */
   int64_t algorithmic_bytes;/* K+V of those tokens + q in + out + appended K/V              */
@@ -419,9 +431,11 @@ int aspd_debug_bounded_wait(int64_t limit_cycles, int32_t* status_out /*host*/, 
 /*
  * Development aid of the tensor-core attention kernel.  In a library built with -DASPD_TC_PROFILE,
  * CTA `cta` of every later launch stamps its clock at the pipeline events of its first 64 tiles
- * into device_buf[0 .. 1024) and every CTA stamps the global timer at entry, after set-up, after
- * its last record and at exit into device_buf[1024 + 4 * blockIdx ..) (device memory of at least
- * 1024 + 4 * n_ctas int64, caller-owned; NULL switches the stamps off).  Other builds return
+ * into device_buf[0 .. 1024) and every CTA stamps the global timer (ns) into device_buf[1024 +
+ * 8 * blockIdx ..): at entry, after set-up, after its last record, after the final barrier, then
+ * (plans that merge inside the kernel) records stored / fenced / counted of its last announced
+ * item, and after its merges (device memory of at least 1024 + 8 * n_ctas int64, caller-owned and
+ * zero-filled; NULL switches the stamps off).  Other builds return
  * ASPD_ERR_UNSUPPORTED.
  */
 int aspd_debug_profile(void* device_buf /*device*/, int cta);

@@ -22,13 +22,14 @@ KERNEL_AUTO, KERNEL_GENERIC, KERNEL_MMA = 0, 1, 2
 Q_SHARED = -1
 POS_AUTO = -1
 MASK_BRANCH_INVISIBLE, MASK_SHARED = 0, 1
+COMBINE_AUTO, COMBINE_KERNEL, COMBINE_FUSED = 0, 1, 2
 
 REQUEST_DTYPE = np.dtype([(n, np.int32) for n in
                           ("prefix_len", "n_branches", "branch_begin", "page_begin", "n_pages", "tail_off", "tail_len")])
 BRANCH_DTYPE = np.dtype([(n, np.int32) for n in ("kv_off", "kv_len", "pos_start", "q_len")])
 ITEM_DTYPE = np.dtype([(n, np.int32) for n in
                        ("q_tok0", "n_q_tok", "kv_head", "page0", "n_pages", "key0", "part_slot", "request", "row_block",
-                        "reserved")])
+                        "n_parts")])
 
 
 class Shape(ctypes.Structure):
@@ -40,7 +41,7 @@ class Shape(ctypes.Structure):
 class Tuning(ctypes.Structure):
     _fields_ = [("kernel", ctypes.c_int32), ("chunk_tokens", ctypes.c_int32), ("n_ctas", ctypes.c_int32),
                 ("host_only", ctypes.c_int32), ("stable_cache", ctypes.c_int32), ("mask", ctypes.c_int32),
-                ("updatable", ctypes.c_int32)]
+                ("updatable", ctypes.c_int32), ("combine", ctypes.c_int32)]
 
 
 class PlanInfo(ctypes.Structure):
@@ -48,7 +49,7 @@ class PlanInfo(ctypes.Structure):
                 ("n_stream_pages", ctypes.c_int32), ("kernel", ctypes.c_int32), ("chunk_tokens", ctypes.c_int32),
                 ("n_ctas", ctypes.c_int32), ("fused_append", ctypes.c_int32),
                 ("direct_output", ctypes.c_int32), ("max_rows_per_item", ctypes.c_int32),
-                ("dealt", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("dealt", ctypes.c_int32), ("single_launch", ctypes.c_int32),
                 ("workspace_bytes", ctypes.c_int64), ("kv_tokens_read", ctypes.c_int64),
                 ("algorithmic_bytes", ctypes.c_int64)]
 
@@ -206,10 +207,10 @@ class Plan:
 
     def __init__(self, shape: Shape, desc, n_pool_pages: int, mode: int, q_pos=None, kernel: int = KERNEL_AUTO,
                  chunk_tokens: int = 0, n_ctas: int = 0, host_only: bool = False, stable_cache: bool = False, stream=None,
-                 mask: int = 0, updatable: bool = False):
+                 mask: int = 0, updatable: bool = False, combine: int = COMBINE_AUTO):
         self.shape, self.mode = shape, mode
         req, br, pages = pack_descriptors(desc)
-        tune = Tuning(kernel, chunk_tokens, n_ctas, 1 if host_only else 0, 1 if stable_cache else 0, mask, 1 if updatable else 0)
+        tune = Tuning(kernel, chunk_tokens, n_ctas, 1 if host_only else 0, 1 if stable_cache else 0, mask, 1 if updatable else 0, combine)
         qp = None if q_pos is None else np.ascontiguousarray(q_pos, dtype=np.int32)
         handle = ctypes.c_void_p()
         self._h = None

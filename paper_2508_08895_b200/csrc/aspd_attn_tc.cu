@@ -28,6 +28,7 @@
 // wait is bounded and on expiry sets the plan's status word to ASPD_ERR_TIMEOUT and makes all
 // roles drain and exit.
 #include "aspd_internal.cuh"
+#include "aspd_combine.cuh"
 
 namespace aspd {
 namespace {
@@ -52,6 +53,7 @@ enum Bar { K_FULL = 0, K_EMPTY = 2, V_FULL = 4, V_EMPTY = 6, S_FULL = 8, S_EMPTY
            O_FULL = 14, O_EMPTY = 16, Q_FULL = 18, Q_EMPTY = 20, E_FULL = 22, A_DONE = 24, NUM_BARS = 25 };
 
 constexpr int kItemCache = 10;      // items of a CTA kept in shared memory (more are read from global)
+constexpr int kMergeQueue = 21;     // (token, KV head) pairs whose last record this CTA stored, waiting to be merged
 constexpr int kMaxTokPerItem = 16;  // tokens of a row block whose ranges are cached (n_q_tok is at most 64 / G)
 
 // The wide variant of the kernel (row blocks of up to 128 query rows, no replication) fills all
@@ -69,6 +71,8 @@ struct Misc {
   int4 vis[kItemCache][kMaxTokPerItem]; // its query tokens: no global-load chain at an item boundary
   uint32_t tmem_base;
   int abort_flag;
+  int mq_n;                    // merge queue (plans that merge inside the kernel): filled by the epilogue warps with
+  int mq[kMergeQueue][3];      // (token * n_kv_heads + KV head, first record, number of records)
 };
 static_assert(sizeof(Misc) <= 8192, "Misc must fit into the unused rows of the P tile");
 constexpr size_t kSmemBytes = 7 * kTileBytes + 1024;   // + slack to align the base to 1024
@@ -210,9 +214,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 // Development aid (builds with -DASPD_TC_PROFILE): one CTA stamps clock64() at pipeline events of
 // its first 64 tiles into the buffer given to aspd_debug_profile.
 #define ASPD_STAMP(c, g, ev) do { if ((c).prof && blockIdx.x == (c).prof_cta && (g) < 64) (c).prof[(g) * 16 + (ev)] = clock64(); } while (0)
-// every CTA: globaltimer (ns) at entry / after set-up / after its last epilogue / at exit
+// every CTA: globaltimer (ns) at entry / after set-up / after its last epilogue / after the final barrier; of the last
+// item with records to announce: records stored / fenced / counted; and after the CTA's merges
 __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define ASPD_CTA_STAMP(c, ev) do { if ((c).prof) (c).prof[1024 + blockIdx.x * 4 + (ev)] = gtime(); } while (0)
+#define ASPD_CTA_STAMP(c, ev) do { if ((c).prof) (c).prof[1024 + blockIdx.x * 8 + (ev)] = gtime(); } while (0)
 #else
 #define ASPD_STAMP(c, g, ev) do { } while (0)
 #define ASPD_CTA_STAMP(c, ev) do { } while (0)
@@ -231,7 +236,21 @@ struct Ctx {
   float scale_log2;
   int early_fetch;             // plan promise: pages without new rows are not written by in-flight work
   __nv_bfloat16* out;          // non-null (plans with one item per (token, KV head)): the epilogue writes O / l here
+  __nv_bfloat16* merge_out;    // non-null (single-launch plans): the CTA that stores the last record of a (token, KV
+                               // head) merges all of them into this; streams with a single item are written directly
 };
+
+// Merge the queued (token, KV head) pairs: one warp per (pair, head of the group) at a time, the
+// records in slot order (the combine kernel's arithmetic).  Called by `n_warps` warps that have
+// passed a barrier after the last push; the caller resets the queue behind another barrier.
+__device__ __forceinline__ void drain_merge_queue(const Ctx& c, const Misc* misc, int warp_rank, int n_warps, int lane) {
+  const int G = c.n_q_heads / c.n_kv_heads, n = min(misc->mq_n, kMergeQueue) * G;
+  for (int u = warp_rank; u < n; u += n_warps) {
+    const int idx = misc->mq[u / G][0], g = u % G, tok = idx / c.n_kv_heads, h = idx % c.n_kv_heads;
+    const int p0 = misc->mq[u / G][1], np = misc->mq[u / G][2];
+    combine_row<__nv_bfloat16, 128>(c.pd.ws_o, c.pd.ws_ml, p0, np, G, g, lane, c.merge_out + ((size_t)tok * c.n_q_heads + h * G + g) * 128);
+  }
+}
 
 // Item idx of this CTA (rel = idx - item_begin): from the shared-memory cache when it is there.
 __device__ __forceinline__ DeviceItem get_item(const Ctx& c, const Misc* misc, int idx, int item_begin) {
@@ -644,6 +663,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     const int counts[NUM_BARS] = {1, 1, 1, 1, 1, 1, 1, 1, 1, 1, 256, 256, 256, 1, 1, 1, 128, 128, 128, 128, 1, 1, 256, 256, 128};
     for (int i = 0; i < NUM_BARS; ++i) mbar_init(bars + 8 * i, counts[i]);
     misc->abort_flag = 0;
+    misc->mq_n = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -877,10 +897,16 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
       dead |= !mbar_wait(bars + 8 * (E_FULL + ob), (item_no >> 1) & 1, ab);
       dead |= !mbar_wait(bars + 8 * (O_FULL + ob), (item_no >> 1) & 1, ab);
       tc_fence_after();
+      // where the item's result goes: a record for the merge, or -- when the item is the row's whole key
+      // stream -- the normalised output itself
+      // (the wide variant only serves plans that deal whole streams: always direct, never a merge)
+      const bool merging = !WIDE && c.merge_out != nullptr;
+      const bool direct = c.out != nullptr || (merging && it.n_parts == 1);
+      __nv_bfloat16* const out_base = c.out != nullptr ? c.out : c.merge_out;
       if (ew < R / 32) {
         const int r = et;                          // row of O held by this thread's TMEM lane
         size_t rec = 0;
-        if (r < M && c.out == nullptr) {
+        if (r < M && !direct) {
           const int tok = it.q_tok0 + r / G;
           rec = (size_t)(c.pd.part_base[tok * c.n_kv_heads + it.kv_head] + it.part_slot) * G + r % G;
           float lt = 0.f;
@@ -892,18 +918,18 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
         const uint32_t o_addr = tmem + ((uint32_t)(ew * 32) << 16) + COL_O + ob * 128;
         float inv_l = 0.f;                         // direct output: the item is the row's whole key stream
         __nv_bfloat16* orow = nullptr;
-        if (c.out != nullptr && r < M) {
+        if (direct && r < M) {
           float lt = 0.f;
           for (int jj = 0; jj < KS; ++jj) lt += misc->fin_l[ob][jj * R + r] + misc->fin_l[ob][128 + jj * R + r];
           inv_l = lt > 0.f ? 1.f / lt : 0.f;
-          orow = c.out + ((size_t)(it.q_tok0 + r / G) * c.n_q_heads + it.kv_head * G + r % G) * 128;
+          orow = out_base + ((size_t)(it.q_tok0 + r / G) * c.n_q_heads + it.kv_head * G + r % G) * 128;
         }
 #pragma unroll 1
         for (int q4 = 0; q4 < 4; ++q4) {
           float o[32];
           ASPD_TMEM_LD32(o_addr + q4 * 32, o, 0);
           tmem_wait_ld();
-          if (c.out != nullptr) {
+          if (direct) {
             if (r < M && !dead) {
               uint4* dst = reinterpret_cast<uint4*>(orow + q4 * 32);
 #pragma unroll
@@ -920,6 +946,30 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
       }
       tc_fence_before();
       mbar_arrive(bars + 8 * (O_EMPTY + ob));
+      if (merging && !direct) {
+        // Announce the item's records: every thread's stores are fenced, then one thread per token
+        // counts the record in; the thread that counts the last record of a (token, KV head) queues
+        // the pair for the merge and puts the counter back to zero for the next launch.  Nobody waits.
+        if (et == 0) ASPD_CTA_STAMP(c, 4);
+        __threadfence();
+        if (misc->mq_n + it.n_q_tok > kMergeQueue) {              // no room for this item's pairs: merge what is queued now
+          drain_merge_queue(c, misc, ew, 4, lane);
+          named_sync(2, 128);
+          if (et == 0) misc->mq_n = 0;
+        }
+        named_sync(2, 128);
+        if (et == 0) ASPD_CTA_STAMP(c, 5);
+        if (et < it.n_q_tok && !dead) {
+          const int idx = (it.q_tok0 + et) * c.n_kv_heads + it.kv_head;
+          if (atomicAdd(c.pd.arrive + idx, 1) == it.n_parts - 1) {
+            __threadfence();                                        // the other CTAs' records, before anyone here reads them
+            c.pd.arrive[idx] = 0;
+            const int e = atomicAdd(&misc->mq_n, 1);
+            misc->mq[e][0] = idx; misc->mq[e][1] = c.pd.part_base[idx]; misc->mq[e][2] = it.n_parts;
+          }
+        }
+        if (et == 0) ASPD_CTA_STAMP(c, 6);
+      }
       if (named_sync_or(2, 128, dead || *ab)) break;
     }
     if (et == 0) ASPD_CTA_STAMP(c, 2);
@@ -938,6 +988,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
   }
+  // single-launch plans: the pairs whose last record this CTA stored are merged now, by all warps
+  if (!WIDE && c.merge_out != nullptr && !*ab) drain_merge_queue(c, misc, warp, kThreads / 32, lane);
+  if (tid == 0) ASPD_CTA_STAMP(c, 7);
 }
 
 
@@ -1010,6 +1063,7 @@ static int launch_tc(const aspd_plan* p, const void* q, const void* k_new, const
   c.scale_log2 = sh.sm_scale * kLog2e;
   c.early_fetch = p->stable_cache;
   c.out = p->dealt ? (__nv_bfloat16*)out : nullptr;   // only when every (token, KV head) has a single item
+  c.merge_out = (!p->dealt && p->single_launch) ? (__nv_bfloat16*)out : nullptr;
   const cudaError_t e = p->wide ? launch_pdl(kPdlAttn, attn_tc_kernel<true>, dim3(p->n_ctas), dim3(kThreads), kSmemBytes, s, c)
                                 : launch_pdl(kPdlAttn, attn_tc_kernel<false>, dim3(p->n_ctas), dim3(kThreads), kSmemBytes, s, c);
   return e == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;

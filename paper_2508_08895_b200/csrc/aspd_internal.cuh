@@ -36,7 +36,7 @@ __host__ __device__ inline uint32_t tile_offset(int t, uint32_t b, uint32_t row_
 }
 
 struct DeviceItem {       // mirrors aspd_item_t, 40 bytes
-  int32_t q_tok0, n_q_tok, kv_head, page0, n_pages, key0, part_slot, request, row_block, reserved;
+  int32_t q_tok0, n_q_tok, kv_head, page0, n_pages, key0, part_slot, request, row_block, n_parts;   // n_parts: items its stream was cut into
 };
 
 struct PlanDevice {       // pointers into the plan's single device allocation
@@ -58,6 +58,8 @@ struct PlanDevice {       // pointers into the plan's single device allocation
   float2* ws_ml;               // [n_partials][G] (reference max in log2 units, sum)
   int32_t* status;             // first error recorded by a kernel
   int32_t* work_counter;       // dynamic work-list cursor (reset by its last reader)
+  int32_t* arrive;             // [n_new * n_kv_heads] records of (new token, KV head) stored so far in this launch (plans
+                               // that merge inside the attention kernel; zero between launches)
   // staging for aspd_step_host
   void* st_q; void* st_k; void* st_v; void* st_out; int32_t* st_pos;
 };
@@ -69,7 +71,7 @@ namespace aspd {
 // length-dependent ones have room for.
 struct PlanLayout {
   size_t o_items = 0, o_cta = 0, o_visit = 0, o_cdirty = 0, o_dirty = 0, o_tpage = 0, o_trow = 0, o_tpos = 0, o_tvis = 0,
-         o_rb = 0, o_pbase = 0, o_freq = 0, o_status = 0, upload_bytes = 0, o_qcs = 0, o_wso = 0, o_wsml = 0, o_stq = 0,
+         o_rb = 0, o_pbase = 0, o_freq = 0, o_status = 0, o_arrive = 0, upload_bytes = 0, o_qcs = 0, o_wso = 0, o_wsml = 0, o_stq = 0,
          o_stk = 0, o_stv = 0, o_sto = 0, o_stp = 0, device_bytes = 0;
   size_t cap_items = 0, cap_visit = 0, cap_dirty = 0, cap_partials = 0, n_row_blocks = 0, n_part_base = 0;
 };
@@ -93,6 +95,7 @@ struct aspd_plan {
   int dealt = 0;                   // whole streams dealt to the CTAs in turn (many more streams than CTAs)
   int shared_mask = 0;             // parallel step under the ablation's visible mask
   int wide = 0;                    // dealt plan of the tensor-core kernel: row blocks of up to kMaxRowsWide rows
+  int single_launch = 0;           // stream-K plan of the tensor-core kernel whose last-arriving CTAs merge the records themselves
   int64_t n_pool_pages = 0;
   int64_t kv_tokens_read = 0;
   int64_t algorithmic_bytes = 0;
@@ -151,7 +154,8 @@ int launch_attn_generic(const aspd_plan* p, const void* q, const void* k_pool, c
 // kernel itself when the plan has one item per (token, KV head) (ignored otherwise)
 int launch_attn_mma(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, void* out,
                     cudaStream_t s);
-inline bool attn_mma_writes_output(const aspd_plan* p) { return p->kernel == ASPD_KERNEL_MMA && p->dealt; }
+inline bool attn_mma_direct(const aspd_plan* p) { return p->kernel == ASPD_KERNEL_MMA && p->dealt; }   // one item per (token, KV head)
+inline bool attn_mma_writes_output(const aspd_plan* p) { return attn_mma_direct(p) || (p->kernel == ASPD_KERNEL_MMA && p->single_launch); }
 int launch_combine(const aspd_plan* p, void* out, cudaStream_t s);
 // fills the plan's cos/sin table from its position and frequency tables (plan creation, after the upload)
 int launch_qcs(const aspd_plan* p, cudaStream_t s);

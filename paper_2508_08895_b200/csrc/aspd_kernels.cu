@@ -1,6 +1,7 @@
 // Small kernels: RoPE + paged append (a3), the generic CUDA-core attention kernel (any
 // supported dtype / head_dim / page_size), the log-sum-exp combine (a7) and a debug reader.
 #include "aspd_internal.cuh"
+#include "aspd_combine.cuh"
 
 namespace aspd {
 
@@ -243,7 +244,6 @@ __global__ void __launch_bounds__(128) attn_generic_kernel(PlanDevice pd, const 
 // and their O rows together, so a row with up to eight records costs one memory round trip.
 template <typename T, int D>
 __global__ void combine_kernel(PlanDevice pd, T* __restrict__ out, int n_new, int n_q_heads, int n_kv_heads) {
-  constexpr int EPL = D / 32;
   pdl_launch_dependents();
   const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   const bool active = w < n_new * n_q_heads;
@@ -252,51 +252,7 @@ __global__ void combine_kernel(PlanDevice pd, T* __restrict__ out, int n_new, in
   const int p0 = pd.part_base[tok * n_kv_heads + h], n = pd.part_base[tok * n_kv_heads + h + 1] - p0;
   pdl_wait();
   if (!active) return;
-  float M = -INFINITY, L = 0.f, acc[EPL];
-#pragma unroll
-  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-  for (int b0 = 0; b0 < n; b0 += 8) {
-    const int cnt = min(8, n - b0);
-    float2 ml = make_float2(-INFINITY, 0.f);
-    if (lane < cnt) ml = pd.ws_ml[(size_t)(p0 + b0 + lane) * G + g];
-    float v[8][EPL];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const float* row = pd.ws_o + ((size_t)(p0 + b0 + min(u, cnt - 1)) * G + g) * D + lane * EPL;
-      if constexpr (EPL == 4) {
-        const float4 x = *reinterpret_cast<const float4*>(row);
-        v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
-      } else {
-        const float2 x = *reinterpret_cast<const float2*>(row);
-        v[u][0] = x.x; v[u][1] = x.y;
-      }
-    }
-    float mb = ml.y > 0.f ? ml.x : -INFINITY;     // records of chunks with no visible key have sum 0
-#pragma unroll
-    for (int o = 4; o; o >>= 1) mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, o));
-    mb = __shfl_sync(0xffffffffu, mb, 0);         // maximum over the round's records (lanes 0..7)
-    const float m_new = fmaxf(M, mb);
-    const float alpha = m_new == -INFINITY ? 1.f : exp2f(M - m_new);   // M = -inf: alpha = 0
-    L *= alpha;
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) acc[e] *= alpha;
-    M = m_new;
-    const float wt = (lane < cnt && ml.y > 0.f) ? exp2f(ml.x - M) : 0.f;
-    float lw = ml.y * wt;
-#pragma unroll
-    for (int o = 4; o; o >>= 1) lw += __shfl_xor_sync(0xffffffffu, lw, o);
-    L += __shfl_sync(0xffffffffu, lw, 0);
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const float wi = __shfl_sync(0xffffffffu, wt, u);
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) acc[e] += wi != 0.f ? v[u][e] * wi : 0.f;   // a skipped record may hold anything
-    }
-  }
-  const float inv = 1.f / L;
-  T* dst = out + ((size_t)tok * n_q_heads + hq) * D + lane * EPL;
-#pragma unroll
-  for (int e = 0; e < EPL; ++e) dst[e] = from_f32<T>(acc[e] * inv);
+  combine_row<T, D>(pd.ws_o, pd.ws_ml, p0, n, G, g, lane, out + ((size_t)tok * n_q_heads + hq) * D);
 }
 
 template <typename T>

@@ -342,12 +342,13 @@ static int plan_create_impl(const aspd_shape_t* shape, const aspd_request_t* req
   const int n_new = aspd_count_new_tokens(req, br, n_req, mode);
   if (n_new < 0) return n_new;
 
-  aspd_tuning_t tune = {ASPD_KERNEL_AUTO, 0, 0, 0, 0, ASPD_MASK_BRANCH_INVISIBLE, 0};
+  aspd_tuning_t tune = {ASPD_KERNEL_AUTO, 0, 0, 0, 0, ASPD_MASK_BRANCH_INVISIBLE, 0, ASPD_COMBINE_AUTO};
   if (tuning) tune = *tuning;
   const int ps = shape->page_size, d = shape->head_dim, Hq = shape->n_q_heads, Hkv = shape->n_kv_heads;
   const int G = Hq / Hkv, es = esize_of(shape->dtype);
   if (tune.chunk_tokens < 0 || tune.chunk_tokens % ps || tune.n_ctas < 0) return ASPD_ERR_INVALID_ARG;
   if (tune.mask != ASPD_MASK_BRANCH_INVISIBLE && tune.mask != ASPD_MASK_SHARED) return ASPD_ERR_INVALID_ARG;
+  if (tune.combine != ASPD_COMBINE_AUTO && tune.combine != ASPD_COMBINE_KERNEL && tune.combine != ASPD_COMBINE_FUSED) return ASPD_ERR_INVALID_ARG;
   const bool shared_mask = tune.mask == ASPD_MASK_SHARED && mode == ASPD_MODE_BRANCH;
   const bool mma_ok = shape->dtype == ASPD_DTYPE_BF16 && d == 128 && ps == 16;
   int kernel = tune.kernel;
@@ -553,7 +554,7 @@ static int plan_create_impl(const aspd_shape_t* shape, const aspd_request_t* req
         const Stream& st = streams[si];
         DeviceItem it;
         it.q_tok0 = st.tok0; it.n_q_tok = st.n_tok; it.kv_head = st.head; it.page0 = st.page0; it.n_pages = st.n_pages;
-        it.key0 = 0; it.part_slot = 0; it.request = st.request; it.row_block = st.row_block; it.reserved = 0;
+        it.key0 = 0; it.part_slot = 0; it.request = st.request; it.row_block = st.row_block; it.n_parts = 1;
         p->items.push_back(it);
         for (int i = 0; i < st.n_tok; ++i) n_parts[(size_t)(st.tok0 + i) * Hkv + st.head] = 1;
       }
@@ -581,6 +582,7 @@ static int plan_create_impl(const aspd_shape_t* shape, const aspd_request_t* req
     auto next_cta = [&]() { cta_item0[++cta] = (int)p->items.size(); acc = 0.0; share = share_now(n_ctas - cta); };
     for (const Stream& st : streams) {
       int at = 0, slot = 0;
+      const size_t first_item = p->items.size();
       const double pc = page_cost(st);
       --streams_left;
       while (at < st.n_pages) {
@@ -591,7 +593,7 @@ static int plan_create_impl(const aspd_shape_t* shape, const aspd_request_t* req
         DeviceItem it;
         it.q_tok0 = st.tok0; it.n_q_tok = st.n_tok; it.kv_head = st.head; it.page0 = st.page0 + at;
         it.n_pages = (int)take; it.key0 = at * ps; it.part_slot = slot++; it.request = st.request;
-        it.row_block = st.row_block; it.reserved = 0;
+        it.row_block = st.row_block; it.n_parts = 0;
         p->items.push_back(it);
         at += (int)take;
         cost_left -= pc * take;
@@ -599,6 +601,7 @@ static int plan_create_impl(const aspd_shape_t* shape, const aspd_request_t* req
         if (acc >= share - 0.5 && cta + 1 < n_ctas) next_cta();
       }
       for (int i = 0; i < st.n_tok; ++i) n_parts[(size_t)(st.tok0 + i) * Hkv + st.head] = slot;
+      for (size_t i = first_item; i < p->items.size(); ++i) p->items[i].n_parts = slot;
     }
     while (cta < n_ctas) cta_item0[++cta] = (int)p->items.size();
   }
@@ -624,6 +627,13 @@ static int plan_create_impl(const aspd_shape_t* shape, const aspd_request_t* req
     for (int c = 0; c < n_ctas; ++c) most = std::max(most, cta_dirty0[c + 1] - cta_dirty0[c]);
     p->fuse_append = (most <= 20 && !shared_mask && tok_field_fits) ? 1 : 0;
   }
+  // the merge of a token's records inside the attention kernel: stream-K plans of the tensor-core kernel
+  // Merging inside the attention kernel is an option, not the default.  Measured on every workload of
+  // the benchmark, the CTA that stores a pair's last record is a CTA at the very end of its own work,
+  // so its fence, count and merge (1.5 us + one memory round trip per 16 rows of the pairs it ended
+  // up with; all rows of a stream cut into dozens of parts land on one CTA) lengthen the kernel by
+  // more than the combine launch costs, whose blocks are resident and waiting when the pass ends.
+  p->single_launch = (kernel == ASPD_KERNEL_MMA && !deal_streams && tune.combine == ASPD_COMBINE_FUSED) ? 1 : 0;
   for (size_t i = 0; i < n_parts.size(); ++i) part_base[i + 1] = part_base[i] + n_parts[i];
   p->n_items = (int)p->items.size();
   p->n_partials = part_base[n_parts.size()];
@@ -675,6 +685,7 @@ static void plan_layout(const aspd_plan* p, double slack, aspd::PlanLayout* L) {
   // the status word is zeroed when the plan is created and never uploaded again, so that a time-out
   // recorded by an earlier launch survives aspd_plan_update until aspd_plan_status reads it
   L->o_status = take(sizeof(int32_t) * 2);
+  L->o_arrive = take(sizeof(int32_t) * std::max(1, n_new) * Hkv);   // right behind the status word: cleared with it
   L->o_qcs = take(sizeof(float2) * std::max(1, n_new) * (d / 2));   // filled on the device from tok_pos and inv_freq
   L->o_wso = take(sizeof(float) * L->cap_partials * G * d);
   L->o_wsml = take(sizeof(float2) * L->cap_partials * G);
@@ -746,11 +757,13 @@ static int plan_to_device(aspd_plan* p, cudaStream_t s) {
   p->dev.inv_freq = (const double*)(b8 + L.o_freq);
   p->dev.status = (int32_t*)(b8 + L.o_status);
   p->dev.work_counter = p->dev.status + 1;
+  p->dev.arrive = (int32_t*)(b8 + L.o_arrive);
   p->dev.ws_o = (float*)(b8 + L.o_wso);
   p->dev.ws_ml = (float2*)(b8 + L.o_wsml);
   p->dev.st_q = b8 + L.o_stq; p->dev.st_k = b8 + L.o_stk; p->dev.st_v = b8 + L.o_stv; p->dev.st_out = b8 + L.o_sto;
   p->dev.st_pos = (int32_t*)(b8 + L.o_stp);
-  rc = cudaMemsetAsync(p->dev.status, 0, 2 * sizeof(int32_t), s) == cudaSuccess ? plan_upload(p, s) : ASPD_ERR_CUDA;
+  rc = cudaMemsetAsync(p->dev.status, 0, (L.o_arrive - L.o_status) + sizeof(int32_t) * std::max(1, p->n_new) * p->shape.n_kv_heads, s) == cudaSuccess
+           ? plan_upload(p, s) : ASPD_ERR_CUDA;
   if (rc) {
     cudaFree(base); cudaFreeHost(p->host_block);
     p->device_base = nullptr; p->host_block = nullptr;
@@ -768,7 +781,7 @@ int aspd_plan_update(aspd_plan_t* p, const aspd_request_t* req, const aspd_branc
   if (rc) return rc;
   const aspd::PlanLayout& L = p->layout;
   if (t->n_new != p->n_new || t->n_ctas != p->n_ctas || t->kernel != p->kernel || t->wide != p->wide || t->dealt != p->dealt ||
-      t->fuse_append != p->fuse_append || t->shared_mask != p->shared_mask || t->kernel != ASPD_KERNEL_MMA ||
+      t->fuse_append != p->fuse_append || t->shared_mask != p->shared_mask || t->single_launch != p->single_launch || t->kernel != ASPD_KERNEL_MMA ||
       t->row_blocks.size() != L.n_row_blocks || t->part_base.size() != L.n_part_base ||
       (t->algorithmic_bytes >= (128LL << 20)) != (p->algorithmic_bytes >= (128LL << 20))) {   // the combine's launch attribute
     delete t;
@@ -805,8 +818,8 @@ int aspd_plan_info(const aspd_plan_t* p, aspd_plan_info_t* info) {
   info->n_new = p->n_new; info->n_items = p->n_items; info->n_partials = p->n_partials;
   info->n_stream_pages = (int32_t)p->visit.size(); info->kernel = p->kernel;
   info->chunk_tokens = p->chunk_tokens; info->n_ctas = p->n_ctas; info->fused_append = (p->kernel == ASPD_KERNEL_MMA && p->fuse_append) ? 1 : 0;
-  info->direct_output = attn_mma_writes_output(p) ? 1 : 0; info->max_rows_per_item = p->wide ? kMaxRowsWide : kMaxRowsPerItem;
-  info->dealt = p->dealt; info->reserved = 0;
+  info->direct_output = attn_mma_direct(p) ? 1 : 0; info->max_rows_per_item = p->wide ? kMaxRowsWide : kMaxRowsPerItem;
+  info->dealt = p->dealt; info->single_launch = p->single_launch;
   info->workspace_bytes = (int64_t)p->device_bytes;
   info->kv_tokens_read = p->kv_tokens_read; info->algorithmic_bytes = p->algorithmic_bytes;
   return ASPD_OK;
@@ -881,7 +894,7 @@ int aspd_step_partials(aspd_plan_t* p, const void* q, const void* k_new, const v
   if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
   if (p->n_new == 0) return ASPD_OK;
   if (!q || !k_new || !v_new || !k_pool || !v_pool || misaligned16(q, k_new, v_new, k_pool, v_pool)) return ASPD_ERR_INVALID_ARG;
-  if (!(p->kernel == ASPD_KERNEL_MMA && p->fuse_append) || attn_mma_writes_output(p)) return ASPD_ERR_UNSUPPORTED;
+  if (!(p->kernel == ASPD_KERNEL_MMA && p->fuse_append) || attn_mma_direct(p)) return ASPD_ERR_UNSUPPORTED;
   note_stream(p, stream);
   return launch_attn_mma_step(p, q, k_new, v_new, k_pool, v_pool, nullptr, (cudaStream_t)stream);
 }
@@ -900,7 +913,8 @@ static int run_attn(aspd_plan_t* p, int mode, const void* q, const void* k_pool,
   if (p->n_new == 0) return ASPD_OK;
   if (!q || !k_pool || !v_pool || !out || misaligned16(q, k_pool, v_pool, out)) return ASPD_ERR_INVALID_ARG;
   note_stream(p, stream);
-  // a plan with one item per (token, KV head) needs no records: the kernel normalises and writes the output
+  // a plan with one item per (token, KV head) needs no records: the kernel normalises and writes the output;
+  // a single-launch plan's kernel merges its records itself
   if (attn_mma_writes_output(p)) return launch_attn_mma(p, q, k_pool, v_pool, out, (cudaStream_t)stream);
   int rc = aspd_attn_partials(p, q, k_pool, v_pool, stream);
   if (rc) return rc;

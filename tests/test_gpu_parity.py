@@ -169,12 +169,34 @@ def test_peaked_softmax_variant(kernel, record_property):
 
 
 @pytest.mark.parametrize("chunk,n_ctas", [(16, 0), (64, 0), (448, 0), (32768, 0), (16, 3), (0, 1), (48, 37)])
-@pytest.mark.parametrize("kernel", KERNELS)
-def test_split_k_counts_agree(chunk, n_ctas, kernel):
+@pytest.mark.parametrize("kernel,combine", [(B.KERNEL_GENERIC, B.COMBINE_AUTO), (B.KERNEL_AUTO, B.COMBINE_KERNEL),
+                                            (B.KERNEL_AUTO, B.COMBINE_FUSED)])
+def test_split_k_counts_agree(chunk, n_ctas, kernel, combine):
     """Forced cuts of the key streams (every `chunk` keys) and forced grid sizes: one item per page,
-    hundreds of items per CTA (beyond what a CTA keeps in shared memory), a single CTA."""
+    hundreds of items per CTA (beyond what a CTA keeps in shared memory, and more last records per
+    CTA than its merge queue holds), a single CTA; records merged by the combine kernel or inside the
+    attention kernel."""
     wl = W.config_long_rag(prefix=1024 + 7)
-    compare_workload(wl, kernel=kernel, chunk_tokens=chunk, n_ctas=n_ctas)
+    compare_workload(wl, kernel=kernel, chunk_tokens=chunk, n_ctas=n_ctas, combine=combine)
+
+
+@pytest.mark.parametrize("fused", [False, True])
+def test_merge_inside_the_attention_kernel_gives_the_combine_kernels_bits(fused):
+    """a7 by a combine launch and a7 by the last-arriving CTAs of the attention kernel are the same
+    arithmetic in the same record order: identical outputs, on the serving mix (stream-K cuts), with
+    forced cuts, and on a request whose streams all lie inside one CTA (written without records)."""
+    E = engine()
+    cases = [(W.config_serving_mix(n_req=8), {}), (W.config_serving_mix(n_req=8), dict(chunk_tokens=160, n_ctas=5)),
+             (W.build_segment_workload("one", 31, 28, 4, 128, "bf16", 1e6, [90], [[40, 17]], [[1, 1]], serial_steps=1), {})]
+    for wl, kw in cases:
+        a = E.run_workload(wl, combine=B.COMBINE_KERNEL, fused=fused, **kw)
+        b = E.run_workload(wl, combine=B.COMBINE_FUSED, fused=fused, **kw)
+        assert len(a.outputs) == len(b.outputs) > 0
+        for x, y in zip(a.outputs, b.outputs):
+            np.testing.assert_array_equal(x, y)
+        ref = oracle_run(wl)
+        for x, r in zip(b.outputs, ref.outputs):
+            check(x, r, wl.dtype, wl.name)
 
 
 @pytest.mark.parametrize("kernel", KERNELS)
@@ -441,9 +463,12 @@ def test_position_id_variants(rule, fused):
     assert np.abs(plain.outputs[-1] - ref.outputs[-1]).max() > 1e-3     # the variant really differs from Eq. 4
 
 
-def test_deterministic_across_repeated_launches():
+@pytest.mark.parametrize("combine", [B.COMBINE_KERNEL, B.COMBINE_FUSED])
+def test_deterministic_across_repeated_launches(combine):
     """Repeated launches of the same step give bit-identical outputs (no data race in the
-    warp-specialised pipeline shows up as run-to-run noise)."""
+    warp-specialised pipeline shows up as run-to-run noise), whether a combine launch merges the
+    records or the attention kernel's last-arriving CTAs do (whichever CTA that is, the records are
+    merged in record order)."""
     import torch
     E = engine()
     wl = W.config_serving_mix(n_req=8)
@@ -451,7 +476,8 @@ def test_deterministic_across_repeated_launches():
     for ph in wl.phases[:-1]:
         run.step(ph)
     ph = wl.phases[-1]
-    plan = B.Plan(run.shape, ph.desc, wl.n_pool_pages, ph.mode, stable_cache=True)
+    plan = B.Plan(run.shape, ph.desc, wl.n_pool_pages, ph.mode, stable_cache=True, combine=combine)
+    assert plan.info.single_launch == (1 if combine == B.COMBINE_FUSED else 0)
     q, k, v = (E.to_device(x, wl.dtype) for x in (ph.q, ph.k_new, ph.v_new))
     outs = [torch.empty_like(q) for _ in range(6)]
     first = None

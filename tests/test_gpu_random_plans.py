@@ -48,6 +48,7 @@ def draw_case(n):
         kw["chunk_tokens"] = int(rng.choice([16, 48, 128, 1024]))
     if rng.integers(0, 6) == 0:
         kw["kernel"] = B.KERNEL_GENERIC
+    kw["combine"] = int(np.random.default_rng(991 + n).integers(0, 3))      # drawn apart: the cases above stay what they were
     return wl, kw
 
 
