@@ -382,25 +382,35 @@ def measure_rerotate(args):
     wl = build_workload(args.workload, 0, args.requests)
     shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
     d = wl.phases[-1].desc
-    pages, rows, delta = [], [], []
+    # sequential renumbering of the finished segment: branch b of a request moves, as a whole, by the
+    # number of tokens in the branches before it
+    pages, rows, delta, ranges = [], [], [], []
     for r in range(len(d["prefix_len"])):
-        P = at = int(d["prefix_len"][r])
+        moved = 0
         for b in range(int(d["branch_begin"][r]), int(d["branch_begin"][r]) + int(d["n_branches"][r])):
             k = np.arange(int(d["br_kv_len"][b]))
             s_ = int(d["br_kv_off"][b]) + k
             pages.append(d["page_ids"][int(d["page_begin"][r]) + s_ // wl.page_size]); rows.append(s_ % wl.page_size)
-            delta.append(at - P + 0 * k); at += len(k)        # sequential renumbering: (at + k) - (P + k)
+            delta.append(moved + 0 * k)
+            ranges.append((int(d["page_begin"][r]), int(d["br_kv_off"][b]), len(k), moved))
+            moved += len(k)
     pages, rows, delta = (torch.from_numpy(np.concatenate(x).astype(np.int32)).cuda() for x in (pages, rows, delta))
+    ranges = np.array(ranges, dtype=np.int32)
+    table_d = torch.from_numpy(np.ascontiguousarray(d["page_ids"], dtype=np.int32)).cuda()
+    by_token = bool(getattr(args, "rerotate_by_token", False))
     n = int(pages.numel())
     es = 2 if wl.dtype == "bf16" else 4
-    alg = n * (2 * wl.Hkv * wl.d * es + 12)
+    alg = n * (2 * wl.Hkv * wl.d * es + (12 if by_token else 0))
     L = max(args.layers, int(np.ceil(4 * 126e6 / alg)))
     caches = [E.LayerCache(shape, wl.n_pool_pages) for _ in range(L)]
     fill_caches(wl, shape, caches)
 
     def step():
         for c in caches:
-            B.k_rerotate(shape, c.k, pages, rows, delta)
+            if by_token:
+                B.k_rerotate(shape, c.k, pages, rows, delta)
+            else:
+                B.k_rerotate_ranges(shape, c.k, table_d, ranges)
     for _ in range(2):
         step()
     torch.cuda.synchronize()
@@ -429,9 +439,9 @@ def measure_rerotate(args):
         "config": {"workload": args.workload, "layers": L, "tokens_per_layer": n, "heads": wl.Hkv, "head_dim": wl.d,
                    "l2": "%.1f GB of distinct keys per step" % (alg * L / 1e9)},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_kind": "of " + peak_kind, "kernel": "rerotate_kernel",
+                     "traffic": None, "peak_kind": "of " + peak_kind, "kernel": "rerotate_kernel" if by_token else "rerotate_ranges_kernel",
                      "kernel_us": ms / args.steps / L * 1e3, "algorithmic_bytes_per_launch": alg},
-        "gpu_launches": L * args.steps, "clocks": clocks})
+        "gpu_launches": L * args.steps * (1 if by_token else (len(ranges) + 511) // 512), "clocks": clocks})
 
 
 def run_serial_chain(args):
@@ -940,6 +950,7 @@ def main():
     ap.add_argument("--loop-graph", action="store_true",
                     help="decode-loop: capture the step once and re-plan in place every step (aspd_plan_update) instead of "
                          "making a new plan and launching from the host")
+    ap.add_argument("--rerotate-by-token", action="store_true", help="rerotate: per-token index arrays (aspd_k_rerotate) instead of ranges")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":

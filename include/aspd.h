@@ -420,6 +420,19 @@ int aspd_k_rerotate(const aspd_shape_t* shape, void* k_pool /*device*/, const in
                     const int32_t* rows /*device*/, const int32_t* delta /*device*/, int n, void* stream);
 
 /*
+ * The same for whole ranges of logical slots, which is what Same-Re renumbering moves: range i is
+ * (page-table base, first slot, count, delta) -- `count` consecutive slots from `first` of the
+ * request whose page table starts at page_table[base], all moved by `delta` positions (a finished
+ * branch moves as a whole: delta = the tokens of the branches listed before it).  The kernel
+ * derives page and row itself, so no per-token index arrays exist or are read.
+ *   page_table  device int32, the concatenated page tables (as aspd_plan_create's page_ids)
+ *   ranges      HOST int32[n_ranges][4]; they travel in the launch parameters, 512 per launch
+ * ASPD_ERR_BAD_DESCRIPTOR for a negative base, slot or count.
+ */
+int aspd_k_rerotate_ranges(const aspd_shape_t* shape, void* k_pool /*device*/, const int32_t* page_table /*device*/,
+                           const int32_t* ranges /*host*/, int n_ranges, void* stream);
+
+/*
  * Failure-path check: runs the library's bounded device-side wait on a barrier nobody ever
  * arrives on, with a limit of `limit_cycles` SM clock cycles (at most 4e9).  The kernel gives up
  * when the limit passes and reports ASPD_ERR_TIMEOUT through *status_out (host); the context
@@ -427,6 +440,18 @@ int aspd_k_rerotate(const aspd_shape_t* shape, void* k_pool /*device*/, const in
  * Synchronises `stream`.
  */
 int aspd_debug_bounded_wait(int64_t limit_cycles, int32_t* status_out /*host*/, void* stream);
+
+/*
+ * Checking builds (-DASPD_DEBUG_BOUNDS; python -m paper_2508_08895_b200.build --debug-bounds): the
+ * kernels compare every page id they are about to use with the number of pool pages and every row
+ * with the page size; on a violation they record ASPD_ERR_BAD_DESCRIPTOR in the plan's status word
+ * and leave the access out (a read is redirected to page 0) -- nothing traps or faults.  Plans
+ * the library built never violate (aspd_plan_create validates on the host), so to see the check
+ * work this call LOWERS the page count the kernels of `plan` compare against (n_pages <= the plan's
+ * n_pool_pages; the pools themselves stay as large as they are, so nothing is out of bounds).
+ * Other builds return ASPD_ERR_UNSUPPORTED.
+ */
+int aspd_debug_pool_limit(aspd_plan_t* plan, int64_t n_pages);
 
 /*
  * Development aid of the tensor-core attention kernel.  In a library built with -DASPD_TC_PROFILE,

@@ -64,7 +64,7 @@ EXPORTS = ("aspd_strerror", "aspd_pool_bytes", "aspd_count_new_tokens", "aspd_po
            "aspd_visible_slots_masked", "aspd_plan_create", "aspd_plan_update", "aspd_plan_destroy", "aspd_release_cached_memory", "aspd_plan_info", "aspd_plan_items", "aspd_plan_cta_ranges", "aspd_plan_stream_pages",
            "aspd_plan_token_ranges", "aspd_plan_shared_mask_tables", "aspd_plan_status",
            "aspd_kv_append", "aspd_branch_attn", "aspd_serial_attn", "aspd_attn_partials", "aspd_attn_combine", "aspd_step_partials",
-           "aspd_branch_step", "aspd_serial_step", "aspd_step_host", "aspd_step_host_async", "aspd_attn_static", "aspd_static_status", "aspd_k_rerotate", "aspd_debug_read_token", "aspd_debug_bounded_wait", "aspd_debug_profile")
+           "aspd_branch_step", "aspd_serial_step", "aspd_step_host", "aspd_step_host_async", "aspd_attn_static", "aspd_static_status", "aspd_k_rerotate", "aspd_k_rerotate_ranges", "aspd_debug_read_token", "aspd_debug_bounded_wait", "aspd_debug_profile", "aspd_debug_pool_limit")
 
 _lib = None
 
@@ -114,8 +114,10 @@ def lib() -> ctypes.CDLL:
         L.aspd_attn_static.argtypes = [vp] * 6
         L.aspd_static_status.argtypes = [vp]
         L.aspd_k_rerotate.argtypes = [vp, vp, vp, vp, vp, ci, vp]
+        L.aspd_k_rerotate_ranges.argtypes = [vp, vp, vp, vp, ci, vp]
         L.aspd_debug_bounded_wait.argtypes = [ctypes.c_int64, vp, vp]
         L.aspd_debug_profile.argtypes = [vp, ci]
+        L.aspd_debug_pool_limit.argtypes = [vp, ctypes.c_int64]
         L.aspd_debug_read_token.argtypes = [vp, vp, ctypes.c_int64, ci, ci, vp, vp]
         for name in EXPORTS:
             if name not in ("aspd_strerror", "aspd_pool_bytes"):
@@ -338,6 +340,14 @@ def k_rerotate(shape: Shape, k_pool, pages, rows, delta, stream=None) -> None:
                                  _stream(stream)), "aspd_k_rerotate")
 
 
+def k_rerotate_ranges(shape: Shape, k_pool, page_table, ranges, stream=None) -> None:
+    """Rotate whole slot ranges in place: ``ranges`` is a host int32 array [n][4] of (page-table
+    base, first slot, count, delta), ``page_table`` the device int32 page tables."""
+    ranges = np.ascontiguousarray(ranges, dtype=np.int32).reshape(-1, 4)
+    _check(lib().aspd_k_rerotate_ranges(ctypes.addressof(shape), _ptr(k_pool), _ptr(page_table), _ptr(ranges), len(ranges),
+                                        _stream(stream)), "aspd_k_rerotate_ranges")
+
+
 def debug_bounded_wait(limit_cycles: int, stream=None) -> int:
     """Status a bounded device-side wait reports when nothing ever satisfies it (ASPD_ERR_TIMEOUT)."""
     st = np.zeros(1, dtype=np.int32)
@@ -359,6 +369,12 @@ def attn_static(plan: Plan, q, k_pool, v_pool, out, stream=None) -> None:
 def static_status(stream=None) -> int:
     """Status word of the last ``attn_static`` call on the current device (synchronises the stream)."""
     return lib().aspd_static_status(_stream(stream))
+
+
+def debug_pool_limit(plan: Plan, n_pages: int) -> int:
+    """Lower the page count a checking build's kernels compare page ids against (status; -3 in an
+    ordinary build)."""
+    return lib().aspd_debug_pool_limit(plan._h, int(n_pages))
 
 
 def debug_profile(device_buf, cta: int = 0) -> int:

@@ -10,6 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libaspd.so")
+LIB_DEBUG_BOUNDS = os.path.join(HERE, "libaspd_debug_bounds.so")   # -DASPD_DEBUG_BOUNDS: kernels that check page ids and rows
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -43,5 +44,15 @@ def build(force: bool = False, verbose: bool = False, out: str = LIB, defines=()
     return out
 
 
+def build_debug_bounds(force: bool = False) -> str:
+    """The checking build, beside the product library (the GPU tests run a subset against it)."""
+    if force or not os.path.exists(LIB_DEBUG_BOUNDS) or (os.path.exists(LIB) and os.path.getmtime(LIB_DEBUG_BOUNDS) < os.path.getmtime(LIB)):
+        build(force=True, out=LIB_DEBUG_BOUNDS, defines=["ASPD_DEBUG_BOUNDS"])
+    return LIB_DEBUG_BOUNDS
+
+
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--debug-bounds" in sys.argv:
+        print(build_debug_bounds(force=True))
+    else:
+        print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

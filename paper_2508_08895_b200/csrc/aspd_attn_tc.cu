@@ -606,7 +606,7 @@ __device__ __forceinline__ void append_new_rows(const Ctx& c, int rank, int d0, 
 #pragma unroll
     for (int k = 0; k < 2; ++k) {
       const int u = u0 + k * 128, sub = u % 24;
-      if (u >= n_units) continue;
+      if (u >= n_units || !bounds_ok(c.pd, d[k].x, d[k].w, 16)) continue;
       const size_t tile = ((size_t)d[k].x * c.n_kv_heads + d[k].y) * 4096;
       if (sub < 8) {
         const __nv_bfloat162* a2 = reinterpret_cast<const __nv_bfloat162*>(&a[k]);
@@ -751,6 +751,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
         pg.x = __shfl_sync(0xffffffffu, cur.x, (t & 3) * 8 + (lane & 7));
         pg.y = __shfl_sync(0xffffffffu, cur.y, (t & 3) * 8 + (lane & 7));
         if (lane >= npg) pg = make_int2(0, 0);
+        if (lane < npg && !bounds_ok(c.pd, pg.x, 0, 16)) pg.x = 0;       // checking builds: flagged, page 0 read instead
         if (producer_runs_ahead && !waited && __any_sync(0xffffffffu, ((pg.y >> 8) & 31) != 0)) {
           pdl_wait();                                  // new rows come from the previous kernel (or from this one)
           waited = true;

@@ -62,7 +62,22 @@ struct PlanDevice {       // pointers into the plan's single device allocation
                                // that merge inside the attention kernel; zero between launches)
   // staging for aspd_step_host
   void* st_q; void* st_k; void* st_v; void* st_out; int32_t* st_pos;
+  int32_t pool_limit;          // pages in each pool: what builds with -DASPD_DEBUG_BOUNDS check page ids against
 };
+
+// Builds with -DASPD_DEBUG_BOUNDS: a kernel that meets a page id or row outside the pool records
+// ASPD_ERR_BAD_DESCRIPTOR in the plan's status word and leaves the access out (nothing traps).
+// Host validation makes this unreachable for plans the library built; the check is there for the
+// development of the planner and of the kernels' index arithmetic.
+#ifdef ASPD_DEBUG_BOUNDS
+__device__ __forceinline__ bool bounds_ok(const PlanDevice& pd, int page, int row, int page_size) {
+  if (page >= 0 && page < pd.pool_limit && row >= 0 && row < page_size) return true;
+  atomicCAS(pd.status, 0, (int)ASPD_ERR_BAD_DESCRIPTOR);
+  return false;
+}
+#else
+__device__ __forceinline__ bool bounds_ok(const PlanDevice&, int, int, int) { return true; }
+#endif
 
 }  // namespace aspd
 
@@ -164,6 +179,8 @@ int launch_attn_mma_step(const aspd_plan* p, const void* q, const void* k_new, c
                          void* v_pool, void* out, cudaStream_t s);
 int launch_rerotate(const aspd_shape_t* shape, void* k_pool, const int32_t* pages, const int32_t* rows, const int32_t* delta,
                     int n, cudaStream_t s);
+int launch_rerotate_ranges(const aspd_shape_t* shape, void* k_pool, const int32_t* page_table, const int32_t* ranges, int n_ranges,
+                           cudaStream_t s);
 int set_profile_buffer(long long* device_buf, int cta);
 int launch_wait_probe(long long limit_cycles, int32_t* status_dev, cudaStream_t s);
 int launch_read_token(const aspd_shape_t* shape, const void* pool, int64_t page, int row, int kv_head,

@@ -26,7 +26,7 @@ __global__ void __launch_bounds__(kAppendThreads)
 append_kernel(const T* __restrict__ k_new, const T* __restrict__ v_new, const int32_t* __restrict__ pos,
               const int32_t* __restrict__ tok_page, const int32_t* __restrict__ tok_row,
               const double* __restrict__ inv_freq, T* __restrict__ k_pool, T* __restrict__ v_pool,
-              int n_new, int n_kv_heads, int head_dim, int page_size) {
+              int n_new, int n_kv_heads, int head_dim, int page_size, PlanDevice pd) {
   constexpr int VEC = 16 / sizeof(T);
   pdl_launch_dependents();
   const int half = head_dim / 2, chunks = half / VEC;
@@ -37,7 +37,7 @@ append_kernel(const T* __restrict__ k_new, const T* __restrict__ v_new, const in
 #pragma unroll
   for (int j = 0; j < VEC; ++j) f[j] = inv_freq[c * VEC + j];
   pdl_wait();
-  if (t >= n_new) return;
+  if (t >= n_new || !bounds_ok(pd, tok_page[t], tok_row[t], page_size)) return;
   // angle reduced to [-pi, pi] in fp64, then fp32 sincos: the error stays near 1e-7 rad
   // however large the position is
   float sn[VEC], cs[VEC];
@@ -101,6 +101,38 @@ constexpr int kRerotateThreads = 256;
 struct InvFreq {          // theta^(-2i/d), computed by the host in double; by value in the launch
   double f[64];
 };
+// One thread's share of a token: the 16-byte chunk at o0 and its partner at o1 in every KV head's
+// tile.  The loads of four heads are issued before the first store (the stores go to the same pool,
+// so the compiler would otherwise keep every head's loads behind the previous head's stores).
+template <typename T>
+__device__ __forceinline__ void rotate_token_heads(char* tile, size_t tb, uint32_t o0, uint32_t o1, int n_kv_heads,
+                                                   const float (&sn)[16 / sizeof(T)], const float (&cs)[16 / sizeof(T)]) {
+  constexpr int VEC = 16 / sizeof(T);
+  for (int h0 = 0; h0 < n_kv_heads; h0 += 4) {
+    uint4 u0[4], u1[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int h = min(h0 + k, n_kv_heads - 1);
+      u0[k] = *reinterpret_cast<const uint4*>(tile + h * tb + o0);
+      u1[k] = *reinterpret_cast<const uint4*>(tile + h * tb + o1);
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (h0 + k >= n_kv_heads) break;
+      T* x0 = reinterpret_cast<T*>(&u0[k]);
+      T* x1 = reinterpret_cast<T*>(&u1[k]);
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) {
+        const float a = to_f32(x0[j]), b = to_f32(x1[j]);
+        x0[j] = from_f32<T>(a * cs[j] - b * sn[j]);
+        x1[j] = from_f32<T>(b * cs[j] + a * sn[j]);
+      }
+      *reinterpret_cast<uint4*>(tile + (h0 + k) * tb + o0) = u0[k];
+      *reinterpret_cast<uint4*>(tile + (h0 + k) * tb + o1) = u1[k];
+    }
+  }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kRerotateThreads)
 rerotate_kernel(T* __restrict__ k_pool, const int32_t* __restrict__ pages, const int32_t* __restrict__ rows,
@@ -128,21 +160,89 @@ rerotate_kernel(T* __restrict__ k_pool, const int32_t* __restrict__ pages, const
   const size_t tb = tile_bytes(page_size, head_dim, sizeof(T));
   char* tile = reinterpret_cast<char*>(k_pool) + (size_t)pages[t] * n_kv_heads * tb;
   const uint32_t o0 = tile_offset(rows[t], c * 16, rb), o1 = tile_offset(rows[t], half * sizeof(T) + c * 16, rb);
-#pragma unroll 4
-  for (int h = 0; h < n_kv_heads; ++h) {
-    uint4* p0 = reinterpret_cast<uint4*>(tile + h * tb + o0);
-    uint4* p1 = reinterpret_cast<uint4*>(tile + h * tb + o1);
-    uint4 u0 = *p0, u1 = *p1;
-    T* x0 = reinterpret_cast<T*>(&u0);
-    T* x1 = reinterpret_cast<T*>(&u1);
+  rotate_token_heads<T>(tile, tb, o0, o1, n_kv_heads, sn, cs);
+}
+
+// The same with the tokens given as ranges of logical slots: range i covers `count` consecutive
+// slots from `first` of the request whose page table starts at page_table[base], all moved by the
+// same `delta` (a finished branch that is renumbered moves as a whole).  The kernel derives page
+// and row itself, so no per-token index arrays are read: a block takes one page of one range.
+constexpr int kMaxRanges = 512;         // ranges per launch (they travel in the launch parameters, about 10 KB)
+struct RerotateRanges {
+  int n;
+  int unit0[kMaxRanges + 1];            // first page unit of range i (prefix sum of the pages each range touches)
+  int4 r[kMaxRanges];                   // (page-table base, first slot, count, delta)
+};
+template <typename T>
+__global__ void __launch_bounds__(512)
+rerotate_ranges_kernel(T* __restrict__ k_pool, const int32_t* __restrict__ page_table, const RerotateRanges rr, const InvFreq table,
+                       int n_kv_heads, int head_dim, int page_size) {
+  constexpr int VEC = 16 / sizeof(T);
+  __shared__ float2 cs_sm[64];          // (cos, sin) of the range's delta for every element pair: the same for all tokens of the page
+  pdl_launch_dependents();
+  const int half = head_dim / 2, chunks = half / VEC;
+  const int u = blockIdx.x;
+  int lo = 0, hi = rr.n - 1;            // the range this block's page belongs to: last i with unit0[i] <= u
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (rr.unit0[mid] <= u) lo = mid; else hi = mid - 1;
+  }
+  const int4 rg = rr.r[lo];
+  const int page = rg.y / page_size + (u - rr.unit0[lo]);           // index of the page in the request's table
+  const int tok = threadIdx.x / chunks, c = threadIdx.x % chunks, slot = page * page_size + tok;
+  const bool active = tok < page_size && slot >= rg.y && slot < rg.y + rg.z;
+  // the sines and cosines depend on the launch parameters only: taken before the dependency wait,
+  // i.e. while the previous kernel of the stream is still running
+  if ((int)threadIdx.x < half) {
+    double a = (double)rg.w * table.f[threadIdx.x];
+    a -= rint(a * 0.15915494309189535) * 6.283185307179586;
+    float sn1, cs1;
+    sincosf((float)a, &sn1, &cs1);
+    cs_sm[threadIdx.x] = make_float2(cs1, sn1);
+  }
+  __syncthreads();
+  pdl_wait();
+  const uint32_t rb = head_dim * sizeof(T);
+  const size_t tb = tile_bytes(page_size, head_dim, sizeof(T));
+  char* tile = reinterpret_cast<char*>(k_pool) + (size_t)page_table[rg.x + page] * n_kv_heads * tb;
+  const uint32_t o0 = tile_offset(tok, c * 16, rb), o1 = tile_offset(tok, half * sizeof(T) + c * 16, rb);
+  uint4 u0[4], u1[4];
 #pragma unroll
-    for (int j = 0; j < VEC; ++j) {
-      const float a = to_f32(x0[j]), b = to_f32(x1[j]);
-      x0[j] = from_f32<T>(a * cs[j] - b * sn[j]);
-      x1[j] = from_f32<T>(b * cs[j] + a * sn[j]);
+  for (int k = 0; k < 4; ++k) {
+    u0[k] = make_uint4(0, 0, 0, 0); u1[k] = u0[k];
+    if (active) {
+      const int h = min(k, n_kv_heads - 1);
+      u0[k] = *reinterpret_cast<const uint4*>(tile + h * tb + o0);
+      u1[k] = *reinterpret_cast<const uint4*>(tile + h * tb + o1);
     }
-    *p0 = u0;
-    *p1 = u1;
+  }
+  if (!active) return;
+  float sn[VEC], cs[VEC];
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) { cs[j] = cs_sm[c * VEC + j].x; sn[j] = cs_sm[c * VEC + j].y; }
+  for (int h0 = 0; h0 < n_kv_heads; h0 += 4) {
+    if (h0 > 0) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int h = min(h0 + k, n_kv_heads - 1);
+        u0[k] = *reinterpret_cast<const uint4*>(tile + h * tb + o0);
+        u1[k] = *reinterpret_cast<const uint4*>(tile + h * tb + o1);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (h0 + k >= n_kv_heads) break;
+      T* x0 = reinterpret_cast<T*>(&u0[k]);
+      T* x1 = reinterpret_cast<T*>(&u1[k]);
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) {
+        const float a = to_f32(x0[j]), b = to_f32(x1[j]);
+        x0[j] = from_f32<T>(a * cs[j] - b * sn[j]);
+        x1[j] = from_f32<T>(b * cs[j] + a * sn[j]);
+      }
+      *reinterpret_cast<uint4*>(tile + (h0 + k) * tb + o0) = u0[k];
+      *reinterpret_cast<uint4*>(tile + (h0 + k) * tb + o1) = u1[k];
+    }
   }
 }
 
@@ -188,6 +288,7 @@ __global__ void __launch_bounds__(128) attn_generic_kernel(PlanDevice pd, const 
         const int2 pg = pd.visit[it.page0 + j / page_size];
         const int row = j % page_size, kg = it.key0 + j;
         seen = row < (pg.y & 255) && (kg < vis.x || (kg >= vis.y && kg < vis.z) || (pg.y >> 13) * page_size + row < vis.w);
+        if (seen && !bounds_ok(pd, pg.x, row, page_size)) seen = false;      // checking builds: flagged, key left out
         if (seen) {
           const char* tile = reinterpret_cast<const char*>(k_pool) + ((size_t)pg.x * n_kv_heads + it.kv_head) * tb;
           float dot = 0.f;
@@ -274,10 +375,10 @@ int launch_append(const aspd_plan* p, const void* k_new, const void* v_new, cons
   if (sh.dtype == ASPD_DTYPE_BF16)
     return status_of(launch_pdl(kPdlAppend, append_kernel<__nv_bfloat16>, grid, block, 0, s, (const __nv_bfloat16*)k_new,
                                 (const __nv_bfloat16*)v_new, pos, p->dev.tok_page, p->dev.tok_row, p->dev.inv_freq,
-                                (__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool, p->n_new, sh.n_kv_heads, sh.head_dim, sh.page_size));
+                                (__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool, p->n_new, sh.n_kv_heads, sh.head_dim, sh.page_size, p->dev));
   return status_of(launch_pdl(kPdlAppend, append_kernel<float>, grid, block, 0, s, (const float*)k_new, (const float*)v_new, pos,
                               p->dev.tok_page, p->dev.tok_row, p->dev.inv_freq, (float*)k_pool, (float*)v_pool, p->n_new,
-                              sh.n_kv_heads, sh.head_dim, sh.page_size));
+                              sh.n_kv_heads, sh.head_dim, sh.page_size, p->dev));
 }
 
 int launch_attn_generic(const aspd_plan* p, const void* q, const void* k_pool, const void* v_pool, cudaStream_t s) {
@@ -331,6 +432,36 @@ int launch_rerotate(const aspd_shape_t* sh, void* k_pool, const int32_t* pages, 
                                 delta, table, n, sh->n_kv_heads, sh->head_dim, sh->page_size));
   return status_of(launch_pdl(kPdlAppend, rerotate_kernel<float>, grid, block, 0, s, (float*)k_pool, pages, rows, delta,
                               table, n, sh->n_kv_heads, sh->head_dim, sh->page_size));
+}
+
+int launch_rerotate_ranges(const aspd_shape_t* sh, void* k_pool, const int32_t* page_table, const int32_t* ranges, int n_ranges,
+                           cudaStream_t s) {
+  const int chunks = sh->head_dim / 2 / (16 / esize_of(sh->dtype)), ps = sh->page_size;
+  InvFreq table;
+  for (int i = 0; i < sh->head_dim / 2; ++i) table.f[i] = pow((double)sh->rope_theta, -2.0 * i / (double)sh->head_dim);
+  for (int r0 = 0; r0 < n_ranges; r0 += kMaxRanges) {
+    RerotateRanges rr;
+    rr.n = 0; rr.unit0[0] = 0;
+    for (int i = r0; i < n_ranges && rr.n < kMaxRanges; ++i) {
+      const int32_t* g = ranges + 4 * (size_t)i;
+      if (g[2] <= 0) continue;                                   // an empty range moves nothing
+      const int pages = (g[1] + g[2] - 1) / ps - g[1] / ps + 1;
+      rr.r[rr.n] = make_int4(g[0], g[1], g[2], g[3]);
+      rr.unit0[rr.n + 1] = rr.unit0[rr.n] + pages;
+      ++rr.n;
+    }
+    if (rr.n == 0) continue;
+    const dim3 grid((unsigned)rr.unit0[rr.n]), block((unsigned)(ps * chunks));
+    cudaError_t e;
+    if (sh->dtype == ASPD_DTYPE_BF16)
+      e = launch_pdl(kPdlAppend, rerotate_ranges_kernel<__nv_bfloat16>, grid, block, 0, s, (__nv_bfloat16*)k_pool, page_table, rr, table,
+                     sh->n_kv_heads, sh->head_dim, ps);
+    else
+      e = launch_pdl(kPdlAppend, rerotate_ranges_kernel<float>, grid, block, 0, s, (float*)k_pool, page_table, rr, table, sh->n_kv_heads,
+                     sh->head_dim, ps);
+    if (e != cudaSuccess) return ASPD_ERR_CUDA;
+  }
+  return ASPD_OK;
 }
 
 int launch_read_token(const aspd_shape_t* sh, const void* pool, int64_t page, int row, int kv_head, float* out_dev,

@@ -762,6 +762,7 @@ static int plan_to_device(aspd_plan* p, cudaStream_t s) {
   p->dev.ws_ml = (float2*)(b8 + L.o_wsml);
   p->dev.st_q = b8 + L.o_stq; p->dev.st_k = b8 + L.o_stk; p->dev.st_v = b8 + L.o_stv; p->dev.st_out = b8 + L.o_sto;
   p->dev.st_pos = (int32_t*)(b8 + L.o_stp);
+  p->dev.pool_limit = (int32_t)std::min<int64_t>(p->n_pool_pages, INT32_MAX);
   rc = cudaMemsetAsync(p->dev.status, 0, (L.o_arrive - L.o_status) + sizeof(int32_t) * std::max(1, p->n_new) * p->shape.n_kv_heads, s) == cudaSuccess
            ? plan_upload(p, s) : ASPD_ERR_CUDA;
   if (rc) {
@@ -1014,6 +1015,30 @@ int aspd_k_rerotate(const aspd_shape_t* shape, void* k_pool, const int32_t* page
   if (n == 0) return ASPD_OK;
   if (!k_pool || !pages || !rows || !delta || misaligned16(k_pool)) return ASPD_ERR_INVALID_ARG;
   return launch_rerotate(shape, k_pool, pages, rows, delta, n, (cudaStream_t)stream);
+}
+
+int aspd_k_rerotate_ranges(const aspd_shape_t* shape, void* k_pool, const int32_t* page_table, const int32_t* ranges, int n_ranges,
+                           void* stream) {
+  int rc = check_shape(shape);
+  if (rc) return rc;
+  if (n_ranges < 0) return ASPD_ERR_INVALID_ARG;
+  if (n_ranges == 0) return ASPD_OK;
+  if (!k_pool || !page_table || !ranges || misaligned16(k_pool)) return ASPD_ERR_INVALID_ARG;
+  for (int i = 0; i < n_ranges; ++i) {
+    const int32_t* g = ranges + 4 * (size_t)i;
+    if (g[0] < 0 || g[1] < 0 || g[2] < 0 || (long)g[1] + g[2] > INT32_MAX) return ASPD_ERR_BAD_DESCRIPTOR;
+  }
+  return launch_rerotate_ranges(shape, k_pool, page_table, ranges, n_ranges, (cudaStream_t)stream);
+}
+
+int aspd_debug_pool_limit(aspd_plan_t* p, int64_t n_pages) {
+  if (!p || p->host_only || n_pages < 0 || n_pages > p->n_pool_pages) return ASPD_ERR_INVALID_ARG;
+#ifdef ASPD_DEBUG_BOUNDS
+  p->dev.pool_limit = (int32_t)std::min<int64_t>(n_pages, INT32_MAX);
+  return ASPD_OK;
+#else
+  return ASPD_ERR_UNSUPPORTED;
+#endif
 }
 
 int aspd_debug_profile(void* device_buf, int cta) {

@@ -119,6 +119,7 @@ extern "C" int aspd_attn_static(const aspd_plan_t* plan, const void* q, const vo
   shell.dev.work_counter = shell.dev.status + 1;
   shell.dev.ws_o = (float*)(base + o_wso);
   shell.dev.ws_ml = (float2*)(base + o_wsml);
+  shell.dev.pool_limit = (int32_t)plan->n_pool_pages;
 
   rc = shell.kernel == ASPD_KERNEL_MMA ? launch_attn_mma(&shell, q, k_pool, v_pool, nullptr, s)
                                        : launch_attn_generic(&shell, q, k_pool, v_pool, s);

@@ -31,14 +31,30 @@ def torch_dtype(dtype: str):
 
 
 class LayerCache:
-    """K and V pools of one attention layer (opaque tile format, see ``aspd.h``)."""
+    """K and V pools of one attention layer (opaque tile format, see ``aspd.h``).
+
+    Each pool sits between two guard pages filled with a byte pattern that no kernel may touch;
+    ``canaries_intact()`` tells whether they still hold it (a write one page before or behind a
+    pool shows there)."""
+
+    CANARY = 0xA5
 
     def __init__(self, shape: B.Shape, n_pool_pages: int, device="cuda"):
         nbytes = B.pool_bytes(shape, n_pool_pages)
         if nbytes == 0 and n_pool_pages > 0:
             raise B.AspdError(-3, "aspd_pool_bytes")
-        self.k = torch.zeros(max(nbytes, 16), dtype=torch.uint8, device=device)
-        self.v = torch.zeros(max(nbytes, 16), dtype=torch.uint8, device=device)
+        self._guard = max(B.pool_bytes(shape, 1), 256)
+        self._raw = []
+        for name in ("k", "v"):
+            raw = torch.full((self._guard * 2 + max(nbytes, 16),), self.CANARY, dtype=torch.uint8, device=device)
+            pool = raw[self._guard: self._guard + max(nbytes, 16)]
+            pool.zero_()
+            self._raw.append(raw)
+            setattr(self, name, pool)
+
+    def canaries_intact(self) -> bool:
+        g = self._guard
+        return all(bool((raw[:g] == self.CANARY).all()) and bool((raw[-g:] == self.CANARY).all()) for raw in self._raw)
 
 
 class WorkloadRun:

@@ -32,6 +32,7 @@ def compare_workload(wl, **kw):
     for (p, s, q), (op, os_, oq) in zip(run.positions, ref.positions):
         np.testing.assert_array_equal(p, op)
         np.testing.assert_array_equal(s, os_)
+    assert run.cache.canaries_intact(), "a kernel wrote outside the pools"
     return run, ref
 
 
@@ -583,10 +584,20 @@ def test_rerotation_moves_cached_keys_to_new_positions():
                 delta.append(at - (P + k)); at += 1
         t = lambda x: torch.tensor(x, dtype=torch.int32, device="cuda")
         before = [run.read_token("k", pg, r, 0) for pg, r in zip(pages, rows)]
-        vbefore = run.cache.v.clone()
+        vbefore, kbefore = run.cache.v.clone(), run.cache.k.clone()
         B.k_rerotate(run.shape, run.cache.k, t(pages), t(rows), t(delta))
         torch.cuda.synchronize()
         assert torch.equal(run.cache.v, vbefore)
+        # the same renumbering given as one range per branch (table base, first slot, count, delta): same bytes
+        ranges, before_b = [], 0
+        for b in range(int(d["n_branches"][0])):
+            ranges.append((0, int(d["br_kv_off"][b]), int(d["br_kv_len"][b]), before_b))
+            before_b += int(d["br_kv_len"][b])
+        k2 = kbefore.clone()
+        B.k_rerotate_ranges(run.shape, k2, t(d["page_ids"].tolist()), np.array(ranges + [(0, 5, 0, 99)], dtype=np.int32))
+        torch.cuda.synchronize()
+        assert torch.equal(k2, run.cache.k) and not torch.equal(k2, kbefore)
+        assert run.cache.canaries_intact()
         # Two roundings to the storage dtype: the stored key is off by half an ulp of each element,
         # the rotation mixes the pair (i, i + d/2), and the result is rounded again.
         ulp_half = 2.0 ** -8 if wl.dtype == "bf16" else 4e-6    # bf16: 8 significand bits
@@ -625,7 +636,18 @@ def test_same_re_serial_decoding_after_rerotation():
                 pages.append(int(d["page_ids"][pg0 + s_ // wl.page_size])); rows.append(s_ % wl.page_size)
                 delta.append(at - (P + k)); at += 1
     t = lambda x: torch.tensor(x, dtype=torch.int32, device="cuda")
-    B.k_rerotate(run.shape, run.cache.k, t(pages), t(rows), t(delta))
+    # one range per branch; every request has its own page table inside the concatenated one
+    ranges = []
+    for r in range(len(d["prefix_len"])):
+        moved = 0
+        for b in range(int(d["branch_begin"][r]), int(d["branch_begin"][r]) + int(d["n_branches"][r])):
+            ranges.append((int(d["page_begin"][r]), int(d["br_kv_off"][b]), int(d["br_kv_len"][b]), moved))
+            moved += int(d["br_kv_len"][b])
+    check_k = run.cache.k.clone()
+    B.k_rerotate(run.shape, check_k, t(pages), t(rows), t(delta))
+    B.k_rerotate_ranges(run.shape, run.cache.k, t(d["page_ids"].tolist()), np.array(ranges, dtype=np.int32))
+    torch.cuda.synchronize()
+    assert torch.equal(check_k, run.cache.k)
     for pg, r, dl in zip(pages, rows, delta):
         for h in range(wl.Hkv):
             ref.k_pool[pg, h, r] = oracle.rope(ref.k_pool[pg, h, r], float(dl), wl.theta)

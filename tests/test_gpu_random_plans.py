@@ -62,3 +62,4 @@ def test_random_requests_and_plan_options(block):
         assert len(run.outputs) == len(ref.outputs) and len(ref.outputs) > 0, (n, kw)
         for g, r in zip(run.outputs, ref.outputs):
             check(g, r, wl.dtype, f"case {n} {kw}")
+        assert run.cache.canaries_intact(), (n, kw)
