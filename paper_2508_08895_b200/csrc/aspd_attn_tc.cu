@@ -235,6 +235,7 @@ struct Ctx {
   int n_items, n_q_heads, n_kv_heads;
   float scale_log2;
   int early_fetch;             // plan promise: pages without new rows are not written by in-flight work
+  int stagger_start;           // plans with few tiles per CTA: the first K tile is requested ahead of the other first tiles
   __nv_bfloat16* out;          // non-null (plans with one item per (token, KV head)): the epilogue writes O / l here
   __nv_bfloat16* merge_out;    // non-null (single-launch plans): the CTA that stores the last record of a (token, KV
                                // head) merges all of them into this; streams with a single item are written directly
@@ -645,9 +646,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
   volatile int* ab = &misc->abort_flag;
   if (tid == 0) ASPD_CTA_STAMP(c, 0);
   if (tid == 0) pdl_launch_dependents();
-  const int item_begin = c.pd.cta_item0[blockIdx.x], item_end = c.pd.cta_item0[blockIdx.x + 1];
-  // Plan tables do not depend on earlier kernels of the stream: the first item and, for the
-  // producers, its first batch of page entries are fetched while the CTA is still setting up.
+  const int4 head = c.pd.cta_head[blockIdx.x];
+  const int item_begin = head.x, item_end = head.y;
+  // Plan tables do not depend on earlier kernels of the stream: the CTA's items and, for the
+  // producers, the first batch of page entries (whose place comes with the head entry, so that it
+  // is the second load of the kernel, not the fourth) are fetched while the CTA is still setting up.
+  int2 first_pages = make_int2(0, 0);
+  if ((warp == W_KPROD || warp == W_VPROD) && lane < head.w) first_pages = c.pd.visit[head.z + lane];
   {
     const int n_cached = min(item_end - item_begin, kItemCache);
     for (int e = tid; e < n_cached * (int)(sizeof(DeviceItem) / 4); e += kThreads)
@@ -725,11 +730,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     bool ok = true, appended = false, waited = false;
     // (item, batch of 32 pages) pairs are walked as one sequence: `cur` holds the batch being
     // consumed, `nxt` the one after it, which may already belong to the next item.
-    int2 nxt = make_int2(0, 0);
-    if (item_begin < item_end) {
-      const DeviceItem f = get_item(c, misc, item_begin, item_begin);
-      if (lane < f.n_pages) nxt = c.pd.visit[f.page0 + lane];
-    }
+    int2 nxt = first_pages;
     for (int idx = item_begin; idx < item_end && ok; ++idx) {
       const DeviceItem it = get_item(c, misc, idx, item_begin);
       const int n_tiles = (it.n_pages + 7) >> 3;
@@ -770,6 +771,18 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
         good = __shfl_sync(0xffffffffu, good, 0);
         if (!good) { ok = false; break; }
         if (lane == 0) ASPD_STAMP(c, g, 6 + kv);
+        if (c.stagger_start && g <= 1 && (kv | g) != 0) {
+          // A CTA with only a few tiles: its four first tiles requested at once (as all 148 CTAs do)
+          // would all land together, late.  So the first K tile goes out alone; the first V tile and the
+          // second K tile follow when it has landed, the second V tile when the first has.  Only a
+          // hint about the order: the wait is short and gives up silently.
+          const uint32_t first = bars + 8 * ((kv == 1 && g == 1) ? V_FULL : K_FULL);
+          if (lane == 0) {
+            const long long t0 = clock64();
+            while (!mbar_try(first, 0) && clock64() - t0 < 8000) { }
+          }
+          __syncwarp();
+        }
         if (kv == 0 && lane < 8) misc->nval[g & 3][lane] = pg.y;   // read by the softmax warps of tile g
         __syncwarp();
         if (lane == 0) mbar_expect_tx(full, (uint32_t)npg * 4096u);
@@ -1063,6 +1076,7 @@ static int launch_tc(const aspd_plan* p, const void* q, const void* k_new, const
   c.n_kv_heads = sh.n_kv_heads;
   c.scale_log2 = sh.sm_scale * kLog2e;
   c.early_fetch = p->stable_cache;
+  c.stagger_start = p->stagger_start;
   c.out = p->dealt ? (__nv_bfloat16*)out : nullptr;   // only when every (token, KV head) has a single item
   c.merge_out = (!p->dealt && p->single_launch) ? (__nv_bfloat16*)out : nullptr;
   const cudaError_t e = p->wide ? launch_pdl(kPdlAttn, attn_tc_kernel<true>, dim3(p->n_ctas), dim3(kThreads), kSmemBytes, s, c)

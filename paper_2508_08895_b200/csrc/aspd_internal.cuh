@@ -41,7 +41,8 @@ struct DeviceItem {       // mirrors aspd_item_t, 40 bytes
 
 struct PlanDevice {       // pointers into the plan's single device allocation
   const DeviceItem* items;
-  const int32_t* cta_item0;    // [n_ctas + 1] items of CTA c are [cta_item0[c], cta_item0[c + 1])
+  const int4* cta_head;        // [n_ctas] (first item, end item, page0 and n_pages of the first item): everything a CTA
+                               // needs to request its first pages comes with one load
   const int2* visit;           // key streams, per page to read: (physical page, valid rows | new rows << 8 |
                                // first new token << 13); the new rows are the last valid rows of the page
   const int32_t* cta_dirty0;   // [n_ctas + 1] range of `dirty` that CTA c must write before reading (fused step)
@@ -110,6 +111,7 @@ struct aspd_plan {
   int dealt = 0;                   // whole streams dealt to the CTAs in turn (many more streams than CTAs)
   int shared_mask = 0;             // parallel step under the ablation's visible mask
   int wide = 0;                    // dealt plan of the tensor-core kernel: row blocks of up to kMaxRowsWide rows
+  int stagger_start = 0;           // few tiles per CTA: order the requests of a CTA's first tiles (see the producers)
   int single_launch = 0;           // stream-K plan of the tensor-core kernel whose last-arriving CTAs merge the records themselves
   int64_t n_pool_pages = 0;
   int64_t kv_tokens_read = 0;
@@ -185,6 +187,13 @@ int set_profile_buffer(long long* device_buf, int cta);
 int launch_wait_probe(long long limit_cycles, int32_t* status_dev, cudaStream_t s);
 int launch_read_token(const aspd_shape_t* shape, const void* pool, int64_t page, int row, int kv_head,
                       float* out_dev, cudaStream_t s);
+// the per-CTA head table of the device plan, from the host tables
+inline void fill_cta_head(const aspd_plan* p, int4* dst) {
+  for (int c = 0; c < p->n_ctas; ++c) {
+    const int b = p->cta_item0[c], e = p->cta_item0[c + 1];
+    dst[c] = make_int4(b, e, b < e ? p->items[b].page0 : 0, b < e ? p->items[b].n_pages : 0);
+  }
+}
 inline int esize_of(int dtype) { return dtype == ASPD_DTYPE_BF16 ? 2 : 4; }
 // device buffers are moved in 16-byte pieces: a pointer off that boundary is refused, not dereferenced
 inline bool misaligned16(const void* a, const void* b = nullptr, const void* c = nullptr, const void* d = nullptr,

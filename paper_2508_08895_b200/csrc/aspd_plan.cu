@@ -628,6 +628,7 @@ static int plan_create_impl(const aspd_shape_t* shape, const aspd_request_t* req
     p->fuse_append = (most <= 20 && !shared_mask && tok_field_fits) ? 1 : 0;
   }
   // the merge of a token's records inside the attention kernel: stream-K plans of the tensor-core kernel
+  p->stagger_start = (!deal_streams && total_pages <= 6L * 8 * n_ctas) ? 1 : 0;       // at most six 128-key tiles per CTA
   // Merging inside the attention kernel is an option, not the default.  Measured on every workload of
   // the benchmark, the CTA that stores a pair's last record is a CTA at the very end of its own work,
   // so its fence, count and merge (1.5 us + one memory round trip per 16 rows of the pairs it ended
@@ -670,7 +671,7 @@ static void plan_layout(const aspd_plan* p, double slack, aspd::PlanLayout* L) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   L->o_items = take(sizeof(DeviceItem) * L->cap_items);
-  L->o_cta = take(sizeof(int32_t) * (p->n_ctas + 1));
+  L->o_cta = take(sizeof(int4) * std::max(1, p->n_ctas));
   L->o_visit = take(sizeof(int2) * L->cap_visit);
   L->o_cdirty = take(sizeof(int32_t) * (p->n_ctas + 1));
   L->o_dirty = take(sizeof(int4) * L->cap_dirty);
@@ -706,7 +707,7 @@ static int plan_upload(aspd_plan* p, cudaStream_t s) {
   uint8_t* blob = static_cast<uint8_t*>(p->host_block);
   memset(blob, 0, L.upload_bytes);
   if (!p->items.empty()) memcpy(blob + L.o_items, p->items.data(), sizeof(DeviceItem) * p->items.size());
-  memcpy(blob + L.o_cta, p->cta_item0.data(), sizeof(int32_t) * (n_ctas + 1));
+  fill_cta_head(p, reinterpret_cast<int4*>(blob + L.o_cta));
   if (!p->visit.empty()) memcpy(blob + L.o_visit, p->visit.data(), sizeof(int2) * p->visit.size());
   memcpy(blob + L.o_cdirty, p->cta_dirty0.data(), sizeof(int32_t) * (n_ctas + 1));
   if (!p->dirty.empty()) memcpy(blob + L.o_dirty, p->dirty.data(), sizeof(int4) * p->dirty.size());
@@ -743,7 +744,7 @@ static int plan_to_device(aspd_plan* p, cudaStream_t s) {
   uint8_t* b8 = (uint8_t*)base;
   p->device_base = base;
   p->dev.items = (const DeviceItem*)(b8 + L.o_items);
-  p->dev.cta_item0 = (const int32_t*)(b8 + L.o_cta);
+  p->dev.cta_head = (const int4*)(b8 + L.o_cta);
   p->dev.visit = (const int2*)(b8 + L.o_visit);
   p->dev.cta_dirty0 = (const int32_t*)(b8 + L.o_cdirty);
   p->dev.dirty = (const int4*)(b8 + L.o_dirty);

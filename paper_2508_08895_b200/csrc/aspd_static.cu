@@ -60,7 +60,7 @@ extern "C" int aspd_attn_static(const aspd_plan_t* plan, const void* q, const vo
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   const size_t o_items = take(sizeof(DeviceItem) * plan->items.size());
-  const size_t o_cta = take(sizeof(int32_t) * plan->cta_item0.size());
+  const size_t o_cta = take(sizeof(int4) * (size_t)(plan->n_ctas > 0 ? plan->n_ctas : 1));
   const size_t o_visit = take(sizeof(int2) * plan->visit.size());
   const size_t o_tvis = take(sizeof(int4) * plan->tok_vis.size());
   const size_t o_rb = take(sizeof(int2) * plan->row_blocks.size());
@@ -79,7 +79,7 @@ extern "C" int aspd_attn_static(const aspd_plan_t* plan, const void* q, const vo
   // and the work counter start at zero; the workspace is fully written before it is read)
   std::vector<uint8_t> blob(upload_bytes, 0);
   memcpy(blob.data() + o_items, plan->items.data(), sizeof(DeviceItem) * plan->items.size());
-  memcpy(blob.data() + o_cta, plan->cta_item0.data(), sizeof(int32_t) * plan->cta_item0.size());
+  aspd::fill_cta_head(plan, reinterpret_cast<int4*>(blob.data() + o_cta));
   memcpy(blob.data() + o_visit, plan->visit.data(), sizeof(int2) * plan->visit.size());
   memcpy(blob.data() + o_tvis, plan->tok_vis.data(), sizeof(int4) * plan->tok_vis.size());
   memcpy(blob.data() + o_rb, plan->row_blocks.data(), sizeof(int2) * plan->row_blocks.size());
@@ -109,7 +109,7 @@ extern "C" int aspd_attn_static(const aspd_plan_t* plan, const void* q, const vo
   shell.device_bytes = 0; shell.device_base = nullptr;
   memset(&shell.dev, 0, sizeof(shell.dev));
   shell.dev.items = (const DeviceItem*)(base + o_items);
-  shell.dev.cta_item0 = (const int32_t*)(base + o_cta);
+  shell.dev.cta_head = (const int4*)(base + o_cta);
   shell.dev.visit = (const int2*)(base + o_visit);
   shell.dev.tok_vis = (const int4*)(base + o_tvis);
   shell.dev.row_blocks = (const int2*)(base + o_rb);
