@@ -118,6 +118,10 @@ typedef struct {
   int32_t mask;         /* ASPD_MASK_*: attention mask of a parallel step (default: branch-invisible) */
   int32_t updatable;    /* 1: leave room in the plan's tables (25 %) for aspd_plan_update                */
   int32_t combine;      /* ASPD_COMBINE_*: where a7 (the merge of a token's split-K records) runs        */
+  int32_t wide_rows;    /* plans that deal whole streams to the tensor-core kernel: query rows of a row
+                           block, 128 (one tile) or 256 (two tiles scored against every K/V tile the CTA
+                           fetches); 0 = automatic (256 when a request has more query tokens than one
+                           tile holds)                                                                */
 } aspd_tuning_t;
 
 /* a7 of a stream-K plan of the tensor-core kernel.  KERNEL: the separate combine launch (what AUTO
@@ -146,7 +150,7 @@ enum { ASPD_COMBINE_AUTO = 0, ASPD_COMBINE_KERNEL = 1, ASPD_COMBINE_FUSED = 2 };
  * k / page_size. */
 typedef struct {
   int32_t q_tok0;     /* first new token (step order) of the item's row block               */
-  int32_t n_q_tok;    /* tokens in the block; rows = n_q_tok * (n_q_heads / n_kv_heads) <= 64 */
+  int32_t n_q_tok;    /* tokens in the block; rows = n_q_tok * (n_q_heads / n_kv_heads) <= max_rows_per_item */
   int32_t kv_head;
   int32_t page0;      /* index of the item's first page in the plan's stream-page list       */
   int32_t n_pages;    /* pages of the item                                                   */
@@ -169,7 +173,7 @@ typedef struct {
                                attention pass; 0: they run the append kernel first               */
   int32_t direct_output;    /* 1: one item per (token, KV head) and the attention kernel writes the
                                output itself (no records, no combine launch)                     */
-  int32_t max_rows_per_item;/* query rows (tokens x group heads) an item may carry: 64 or 128       */
+  int32_t max_rows_per_item;/* query rows (tokens x group heads) an item may carry: 64, 128 or 256  */
   int32_t dealt;            /* 1: whole streams dealt to the CTAs (every row block has a page list of its
                                own, so n_stream_pages counts shared pages once per row block); 0: stream-K cuts */
   int32_t single_launch;    /* 1: the attention kernel merges the split-K records itself (ASPD_COMBINE_FUSED): the
@@ -310,7 +314,9 @@ int aspd_serial_attn(aspd_plan_t* plan, const void* q /*device*/, const void* k_
  * The two halves of either attention call, for callers (and profilers) that want them
  * apart: a4-a6, the split-K pass that leaves one un-normalised (max, sum, O) record per work
  * item and query row in the plan's workspace; and a7, the log-sum-exp merge of a token's
- * records into `out`.  aspd_branch_attn / aspd_serial_attn are exactly these two in sequence.
+ * records into `out`.  aspd_branch_attn / aspd_serial_attn are exactly these two in sequence
+ * (plans with 256-row blocks, whose kernel only writes final outputs, return
+ * ASPD_ERR_UNSUPPORTED from aspd_attn_partials).
  */
 int aspd_attn_partials(aspd_plan_t* plan, const void* q /*device*/, const void* k_pool /*device*/,
                        const void* v_pool /*device*/, void* stream);

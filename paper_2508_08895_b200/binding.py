@@ -41,7 +41,7 @@ class Shape(ctypes.Structure):
 class Tuning(ctypes.Structure):
     _fields_ = [("kernel", ctypes.c_int32), ("chunk_tokens", ctypes.c_int32), ("n_ctas", ctypes.c_int32),
                 ("host_only", ctypes.c_int32), ("stable_cache", ctypes.c_int32), ("mask", ctypes.c_int32),
-                ("updatable", ctypes.c_int32), ("combine", ctypes.c_int32)]
+                ("updatable", ctypes.c_int32), ("combine", ctypes.c_int32), ("wide_rows", ctypes.c_int32)]
 
 
 class PlanInfo(ctypes.Structure):
@@ -209,10 +209,10 @@ class Plan:
 
     def __init__(self, shape: Shape, desc, n_pool_pages: int, mode: int, q_pos=None, kernel: int = KERNEL_AUTO,
                  chunk_tokens: int = 0, n_ctas: int = 0, host_only: bool = False, stable_cache: bool = False, stream=None,
-                 mask: int = 0, updatable: bool = False, combine: int = COMBINE_AUTO):
+                 mask: int = 0, updatable: bool = False, combine: int = COMBINE_AUTO, wide_rows: int = 0):
         self.shape, self.mode = shape, mode
         req, br, pages = pack_descriptors(desc)
-        tune = Tuning(kernel, chunk_tokens, n_ctas, 1 if host_only else 0, 1 if stable_cache else 0, mask, 1 if updatable else 0, combine)
+        tune = Tuning(kernel, chunk_tokens, n_ctas, 1 if host_only else 0, 1 if stable_cache else 0, mask, 1 if updatable else 0, combine, wide_rows)
         qp = None if q_pos is None else np.ascontiguousarray(q_pos, dtype=np.int32)
         handle = ctypes.c_void_p()
         self._h = None

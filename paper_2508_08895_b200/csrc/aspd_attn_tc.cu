@@ -27,8 +27,11 @@
 // (TMEM lane quadrant = warp - 12); warp 10 is idle.  All cross-role hand-offs are mbarriers; every
 // wait is bounded and on expiry sets the plan's status word to ASPD_ERR_TIMEOUT and makes all
 // roles drain and exit.
+#include <type_traits>
+
 #include "aspd_internal.cuh"
 #include "aspd_combine.cuh"
+#include "aspd_tc_common.cuh"
 
 namespace aspd {
 namespace {
@@ -40,7 +43,6 @@ constexpr int W_KPROD = 8, W_MMA = 9, W_VPROD = 11, W_EPI = 12;   // warp roles 
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRaise = 8.0f;                 // raise the reference maximum only beyond 2^8
 constexpr float kLower = 32.0f;                // wide variant: lower the initial reference (0) when a row's first keys are below 2^-32
-constexpr long long kWaitCycles = 3000000000LL; // ~1.5 s at 1.9 GHz
 
 constexpr uint32_t kTileBytes = 32768;         // one K, V, Q or P tile: 128 rows x 256 B
 constexpr uint32_t kHalf = 16384;              // second 64-element span of a tile
@@ -79,136 +81,6 @@ constexpr size_t kSmemBytes = 7 * kTileBytes + 1024;   // + slack to align the b
 
 // TMEM columns: S double buffer, O double buffer
 constexpr uint32_t COL_S = 0, COL_O = 256;
-
-// ------------------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait: false means "give up" (time limit hit here or in another role).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          long long limit = kWaitCycles) {
-  if (mbar_try(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-    if (mbar_try(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > limit) { *abort_flag = 1; return false; }
-  }
-}
-__device__ __forceinline__ void bulk_copy(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
-}
-// The same two, executed by a whole warp with warp-uniform operands; lane 0 alone issues.  With
-// uniform control flow around them the descriptors stay in the uniform datapath.
-__device__ __forceinline__ void tc_commit_lane0(uint32_t bar) {
-  asm volatile(
-      "{\n\t.reg .pred e;\n\t.reg .u32 l;\n\t"
-      "mov.u32 l, %%laneid;\n\t"
-      "setp.eq.u32 e, l, 0;\n\t"
-      "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma_lane0(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p, e;\n\t.reg .u32 l;\n\t"
-      "mov.u32 l, %%laneid;\n\t"
-      "setp.eq.u32 e, l, 0;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
-// Barrier among n threads that also ORs a predicate, so that all of them take the same exit.
-__device__ __forceinline__ bool named_sync_or(int id, int n, bool pred) {
-  uint32_t out;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
-      "setp.ne.b32 q, %3, 0;\n\t"
-      "bar.red.or.pred p, %1, %2, q;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(out) : "r"(id), "r"(n), "r"((uint32_t)pred) : "memory");
-  return out != 0;
-}
-
-#define ASPD_R32(v, o) "=f"(v[o + 0]), "=f"(v[o + 1]), "=f"(v[o + 2]), "=f"(v[o + 3]), "=f"(v[o + 4]), "=f"(v[o + 5]),  \
-    "=f"(v[o + 6]), "=f"(v[o + 7]), "=f"(v[o + 8]), "=f"(v[o + 9]), "=f"(v[o + 10]), "=f"(v[o + 11]), "=f"(v[o + 12]),    \
-    "=f"(v[o + 13]), "=f"(v[o + 14]), "=f"(v[o + 15]), "=f"(v[o + 16]), "=f"(v[o + 17]), "=f"(v[o + 18]),                 \
-    "=f"(v[o + 19]), "=f"(v[o + 20]), "=f"(v[o + 21]), "=f"(v[o + 22]), "=f"(v[o + 23]), "=f"(v[o + 24]),                 \
-    "=f"(v[o + 25]), "=f"(v[o + 26]), "=f"(v[o + 27]), "=f"(v[o + 28]), "=f"(v[o + 29]), "=f"(v[o + 30]), "=f"(v[o + 31])
-#define ASPD_W32(v, o) "f"(v[o + 0]), "f"(v[o + 1]), "f"(v[o + 2]), "f"(v[o + 3]), "f"(v[o + 4]), "f"(v[o + 5]),        \
-    "f"(v[o + 6]), "f"(v[o + 7]), "f"(v[o + 8]), "f"(v[o + 9]), "f"(v[o + 10]), "f"(v[o + 11]), "f"(v[o + 12]),           \
-    "f"(v[o + 13]), "f"(v[o + 14]), "f"(v[o + 15]), "f"(v[o + 16]), "f"(v[o + 17]), "f"(v[o + 18]), "f"(v[o + 19]),       \
-    "f"(v[o + 20]), "f"(v[o + 21]), "f"(v[o + 22]), "f"(v[o + 23]), "f"(v[o + 24]), "f"(v[o + 25]), "f"(v[o + 26]),       \
-    "f"(v[o + 27]), "f"(v[o + 28]), "f"(v[o + 29]), "f"(v[o + 30]), "f"(v[o + 31])
-
-// 32 consecutive fp32 columns of this thread's TMEM lane -> v[o .. o+31]
-#define ASPD_TMEM_LD32(taddr, v, o)                                                                               \
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, "  \
-               "%13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, " \
-               "[%32];" : ASPD_R32(v, o) : "r"(taddr) : "memory")
-#define ASPD_TMEM_ST32(taddr, v, o)                                                                               \
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, " \
-               "%12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, "   \
-               "%31};" ::ASPD_W32(v, o), "r"(taddr) : "memory")
-#define ASPD_TMEM_LD16(taddr, v, o)                                                                               \
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, "  \
-               "%13, %14, %15}, [%16];"                                                                          \
-               : "=f"(v[o + 0]), "=f"(v[o + 1]), "=f"(v[o + 2]), "=f"(v[o + 3]), "=f"(v[o + 4]), "=f"(v[o + 5]),  \
-                 "=f"(v[o + 6]), "=f"(v[o + 7]), "=f"(v[o + 8]), "=f"(v[o + 9]), "=f"(v[o + 10]), "=f"(v[o + 11]), \
-                 "=f"(v[o + 12]), "=f"(v[o + 13]), "=f"(v[o + 14]), "=f"(v[o + 15])                               \
-               : "r"(taddr) : "memory")
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
-         (1ull << 46) | (2ull << 61);
-}
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, A K-major.
-__device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
-}
-
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
-  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
-  return *reinterpret_cast<uint32_t*>(&h);
-}
 
 #ifdef ASPD_TC_PROFILE
 // Development aid (builds with -DASPD_TC_PROFILE): one CTA stamps clock64() at pipeline events of
@@ -516,9 +388,10 @@ __device__ __forceinline__ bool softmax_item_wide(const Ctx& c, const DeviceItem
 struct QUnits {
   uint32_t lo[4][4], hi[4][4];   // per unit: the rotated chunk of the first and of the second span, bf16 pairs
 };
-__device__ __forceinline__ void prep_q_compute(const Ctx& c, const DeviceItem& it, int rank, int e0, QUnits& qu) {
+// tile128: the rows always form a 128-row tile of their own (no replication), however few they are
+__device__ __forceinline__ void prep_q_compute(const Ctx& c, const DeviceItem& it, int rank, int e0, QUnits& qu, bool tile128 = false) {
   const int G = c.n_q_heads / c.n_kv_heads;
-  const int M = it.n_q_tok * G, R = M <= 32 ? 32 : (M <= 64 ? 64 : 128);
+  const int M = it.n_q_tok * G, R = tile128 ? 128 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
   uint4 a[4], b[4];
   float4 w[4][4];
 #pragma unroll
@@ -549,9 +422,10 @@ __device__ __forceinline__ void prep_q_compute(const Ctx& c, const DeviceItem& i
     }
   }
 }
-__device__ __forceinline__ void prep_q_store(const Ctx& c, const DeviceItem& it, uint32_t qbuf, int rank, int e0, const QUnits& qu) {
+__device__ __forceinline__ void prep_q_store(const Ctx& c, const DeviceItem& it, uint32_t qbuf, int rank, int e0, const QUnits& qu,
+                                             bool tile128 = false) {
   const int G = c.n_q_heads / c.n_kv_heads;
-  const int M = it.n_q_tok * G, R = M <= 32 ? 32 : (M <= 64 ? 64 : 128), KS = 128 / R;
+  const int M = it.n_q_tok * G, R = tile128 ? 128 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128)), KS = 128 / R;
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
     const int e = e0 + rank + u * 128, r = e >> 3, ch = e & 7;
@@ -1024,14 +898,18 @@ __global__ void wait_probe_kernel(long long limit_cycles, int32_t* status) {
 
 }  // namespace
 
+#include "aspd_attn_tc_w2.cuh"
+
 int launch_wait_probe(long long limit_cycles, int32_t* status_dev, cudaStream_t s) {
   wait_probe_kernel<<<1, 32, 0, s>>>(limit_cycles, status_dev);
   return cudaGetLastError() == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
 }
 
 // where the profiling build's stamps go (aspd_debug_profile)
+#ifdef ASPD_TC_PROFILE
 static long long* g_prof_buf = nullptr;
 static int g_prof_cta = 0;
+#endif
 
 int set_profile_buffer(long long* device_buf, int cta) {
 #ifdef ASPD_TC_PROFILE
@@ -1054,7 +932,8 @@ static int launch_tc(const aspd_plan* p, const void* q, const void* k_new, const
   if (cudaGetDevice(&dev) != cudaSuccess) return ASPD_ERR_CUDA;
   if (dev < 0 || dev >= 64 || !configured[dev]) {
     if (cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
+        cudaFuncSetAttribute(attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_tc_w2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytesW2) != cudaSuccess)
       return ASPD_ERR_CUDA;
     if (dev >= 0 && dev < 64) configured[dev] = true;
   }
@@ -1079,6 +958,11 @@ static int launch_tc(const aspd_plan* p, const void* q, const void* k_new, const
   c.stagger_start = p->stagger_start;
   c.out = p->dealt ? (__nv_bfloat16*)out : nullptr;   // only when every (token, KV head) has a single item
   c.merge_out = (!p->dealt && p->single_launch) ? (__nv_bfloat16*)out : nullptr;
+  if (p->wide == 2) {                       // row blocks of two query tiles: final outputs only
+    if (c.out == nullptr) return ASPD_ERR_UNSUPPORTED;
+    c.k_new = nullptr; c.v_new = nullptr;
+    return launch_pdl(kPdlAttn, attn_tc_w2_kernel, dim3(p->n_ctas), dim3(kThreads), kSmemBytesW2, s, c) == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;
+  }
   const cudaError_t e = p->wide ? launch_pdl(kPdlAttn, attn_tc_kernel<true>, dim3(p->n_ctas), dim3(kThreads), kSmemBytes, s, c)
                                 : launch_pdl(kPdlAttn, attn_tc_kernel<false>, dim3(p->n_ctas), dim3(kThreads), kSmemBytes, s, c);
   return e == cudaSuccess ? ASPD_OK : ASPD_ERR_CUDA;

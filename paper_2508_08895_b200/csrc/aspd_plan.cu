@@ -16,7 +16,6 @@ using namespace aspd;
 
 namespace {
 
-inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // ---- device blocks of destroyed plans are kept for the next plan --------------------------------
@@ -342,12 +341,13 @@ static int plan_create_impl(const aspd_shape_t* shape, const aspd_request_t* req
   const int n_new = aspd_count_new_tokens(req, br, n_req, mode);
   if (n_new < 0) return n_new;
 
-  aspd_tuning_t tune = {ASPD_KERNEL_AUTO, 0, 0, 0, 0, ASPD_MASK_BRANCH_INVISIBLE, 0, ASPD_COMBINE_AUTO};
+  aspd_tuning_t tune = {ASPD_KERNEL_AUTO, 0, 0, 0, 0, ASPD_MASK_BRANCH_INVISIBLE, 0, ASPD_COMBINE_AUTO, 0};
   if (tuning) tune = *tuning;
   const int ps = shape->page_size, d = shape->head_dim, Hq = shape->n_q_heads, Hkv = shape->n_kv_heads;
   const int G = Hq / Hkv, es = esize_of(shape->dtype);
   if (tune.chunk_tokens < 0 || tune.chunk_tokens % ps || tune.n_ctas < 0) return ASPD_ERR_INVALID_ARG;
   if (tune.mask != ASPD_MASK_BRANCH_INVISIBLE && tune.mask != ASPD_MASK_SHARED) return ASPD_ERR_INVALID_ARG;
+  if (tune.wide_rows != 0 && tune.wide_rows != 128 && tune.wide_rows != 256) return ASPD_ERR_INVALID_ARG;
   if (tune.combine != ASPD_COMBINE_AUTO && tune.combine != ASPD_COMBINE_KERNEL && tune.combine != ASPD_COMBINE_FUSED) return ASPD_ERR_INVALID_ARG;
   const bool shared_mask = tune.mask == ASPD_MASK_SHARED && mode == ASPD_MODE_BRANCH;
   const bool mma_ok = shape->dtype == ASPD_DTYPE_BF16 && d == 128 && ps == 16;
@@ -530,7 +530,15 @@ static int plan_create_impl(const aspd_shape_t* shape, const aspd_request_t* req
   p->wide = 0;
   if (deal_streams) {
     p->wide = (kernel == ASPD_KERNEL_MMA && kMaxRowsWide / G > max_tok) ? 1 : 0;
-    const int tok_per_block = p->wide ? kMaxRowsWide / G : max_tok;
+    // A step in which some request has more query tokens than one 128-row tile holds takes row blocks
+    // of two tiles (the two-tile variant of the kernel: both tiles are scored against every K/V tile
+    // the CTA fetches, one softmax group per tile), unless the caller asked for single tiles.
+    if (p->wide && tune.wide_rows != 128) {
+      int most_q = 0;
+      for (const Block& bk : blocks) most_q = std::max(most_q, bk.n_tok);
+      if (most_q > kMaxRowsWide / G || tune.wide_rows == 256) p->wide = 2;
+    }
+    const int tok_per_block = p->wide ? p->wide * (kMaxRowsWide / G) : max_tok;
     build_visit(tok_per_block);
     build_streams(tok_per_block);
   }
@@ -625,7 +633,7 @@ static int plan_create_impl(const aspd_shape_t* shape, const aspd_request_t* req
     // rows per CTA (a branch-open step) the separate append kernel is the faster way
     int most = 0;
     for (int c = 0; c < n_ctas; ++c) most = std::max(most, cta_dirty0[c + 1] - cta_dirty0[c]);
-    p->fuse_append = (most <= 20 && !shared_mask && tok_field_fits) ? 1 : 0;
+    p->fuse_append = (most <= 20 && !shared_mask && tok_field_fits && p->wide != 2) ? 1 : 0;
   }
   // the merge of a token's records inside the attention kernel: stream-K plans of the tensor-core kernel
   p->stagger_start = (!deal_streams && total_pages <= 6L * 8 * n_ctas) ? 1 : 0;       // at most six 128-key tiles per CTA
@@ -820,7 +828,7 @@ int aspd_plan_info(const aspd_plan_t* p, aspd_plan_info_t* info) {
   info->n_new = p->n_new; info->n_items = p->n_items; info->n_partials = p->n_partials;
   info->n_stream_pages = (int32_t)p->visit.size(); info->kernel = p->kernel;
   info->chunk_tokens = p->chunk_tokens; info->n_ctas = p->n_ctas; info->fused_append = (p->kernel == ASPD_KERNEL_MMA && p->fuse_append) ? 1 : 0;
-  info->direct_output = attn_mma_direct(p) ? 1 : 0; info->max_rows_per_item = p->wide ? kMaxRowsWide : kMaxRowsPerItem;
+  info->direct_output = attn_mma_direct(p) ? 1 : 0; info->max_rows_per_item = p->wide ? p->wide * kMaxRowsWide : kMaxRowsPerItem;
   info->dealt = p->dealt; info->single_launch = p->single_launch;
   info->workspace_bytes = (int64_t)p->device_bytes;
   info->kv_tokens_read = p->kv_tokens_read; info->algorithmic_bytes = p->algorithmic_bytes;
@@ -885,6 +893,7 @@ int aspd_attn_partials(aspd_plan_t* p, const void* q, const void* k_pool, const 
   if (!p || p->host_only) return ASPD_ERR_INVALID_ARG;
   if (p->n_new == 0) return ASPD_OK;
   if (!q || !k_pool || !v_pool || misaligned16(q, k_pool, v_pool)) return ASPD_ERR_INVALID_ARG;
+  if (p->wide == 2) return ASPD_ERR_UNSUPPORTED;       // the two-tile variant only writes final outputs
   cudaStream_t s = (cudaStream_t)stream;
   note_stream(p, stream);
   return p->kernel == ASPD_KERNEL_MMA ? launch_attn_mma(p, q, k_pool, v_pool, nullptr, s)

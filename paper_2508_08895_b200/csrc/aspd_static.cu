@@ -121,6 +121,8 @@ extern "C" int aspd_attn_static(const aspd_plan_t* plan, const void* q, const vo
   shell.dev.ws_ml = (float2*)(base + o_wsml);
   shell.dev.pool_limit = (int32_t)plan->n_pool_pages;
 
+  // plans that deal whole streams have one item per (token, KV head): their kernel writes the output
+  if (attn_mma_direct(&shell)) return launch_attn_mma(&shell, q, k_pool, v_pool, out, s);
   rc = shell.kernel == ASPD_KERNEL_MMA ? launch_attn_mma(&shell, q, k_pool, v_pool, nullptr, s)
                                        : launch_attn_generic(&shell, q, k_pool, v_pool, s);
   if (rc) return rc;

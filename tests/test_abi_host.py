@@ -148,7 +148,7 @@ def _check_cover(wl, ph, plan, chunk=0, dealt=False, mask=0):
     slots_seen = {}
     ps = wl.page_size
     for it in plan.items():
-        assert it["n_q_tok"] * wl.G <= (128 if dealt else 64) and it["n_pages"] >= 1 and it["key0"] % ps == 0
+        assert it["n_q_tok"] * wl.G <= (256 if dealt else 64) and it["n_pages"] >= 1 and it["key0"] % ps == 0
         if chunk:
             assert it["n_pages"] * ps <= chunk
         for i in range(int(it["n_q_tok"])):
@@ -212,17 +212,19 @@ def test_shared_mask_plans_cover_the_oracles_visible_sets():
     assert _plan_rc(W.config_tiny(), W.config_tiny().phases[-1].desc, W.config_tiny().phases[-1].mode, mask=7) == -1     # ASPD_ERR_INVALID_ARG
 
 
-@pytest.mark.parametrize("kernel", [B.KERNEL_MMA, B.KERNEL_GENERIC])
-def test_dealt_plan_of_a_step_with_many_query_tokens(kernel):
+@pytest.mark.parametrize("kernel,wide_rows", [(B.KERNEL_MMA, 0), (B.KERNEL_MMA, 128), (B.KERNEL_GENERIC, 0)])
+def test_dealt_plan_of_a_step_with_many_query_tokens(kernel, wide_rows):
     """Many more streams than CTAs: whole streams are dealt out, one record per (token, head);
-    each row block lists the prefix and only the branch pages its tokens see (up to 128 rows
-    for the tensor-core kernel), and the visible sets are still exactly the oracle's."""
+    each row block lists the prefix and only the branch pages its tokens see (up to 256 rows, two
+    query tiles, for the tensor-core kernel, or 128 when asked), and the visible sets are still
+    exactly the oracle's."""
     wl = W.build_segment_workload("deal", 31, 28, 4, 128, "bf16", 1e6, [70, 9, 33], [[0, 17, 5, 2], [3], [0, 0]],
                                   [[40, 25, 31, 1], [21], [2, 50]], serial_steps=0)
     ph = wl.phases[-1]
-    plan = B.Plan(_shape(wl), ph.desc, wl.n_pool_pages, ph.mode, kernel=kernel, n_ctas=6, host_only=True)
+    plan = B.Plan(_shape(wl), ph.desc, wl.n_pool_pages, ph.mode, kernel=kernel, n_ctas=6, host_only=True, wide_rows=wide_rows)
     items = plan.items()
-    assert int(items["n_q_tok"].max()) == (18 if kernel == B.KERNEL_MMA else 9)
+    assert int(items["n_q_tok"].max()) == ((18 if wide_rows == 128 else 36) if kernel == B.KERNEL_MMA else 9)
+    assert plan.info.max_rows_per_item == ((128 if wide_rows == 128 else 256) if kernel == B.KERNEL_MMA else 64)
     assert (items["part_slot"] == 0).all() and (items["key0"] == 0).all()
     seen = _check_cover(wl, ph, plan, dealt=True)
     assert all(len(v) == 1 for v in seen.values())

@@ -134,7 +134,7 @@ def test_masked_prefill_full_size():
     ph = wl.phases[-1]
     shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
     plan = B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode, host_only=True)
-    assert plan.info.direct_output and plan.info.max_rows_per_item == 128 and plan.info.n_ctas == 148
+    assert plan.info.direct_output and plan.info.max_rows_per_item == 256 and plan.info.n_ctas == 148
     plan.destroy()
     run, ref = compare_workload(wl, fused=True, stable_cache=True)
     assert run.outputs[0].shape[0] == 17069
@@ -501,33 +501,52 @@ def test_masked_prefill_of_a_parallel_segment(kernel):
     run, ref = compare_workload(wl, kernel=kernel)
     assert run.outputs[0].shape[0] == 240
     # with few CTAs the plan has many more streams than CTAs and deals whole streams instead of
-    # cutting; the tensor-core kernel then runs its wide variant (row blocks of up to 18 tokens)
+    # cutting; the tensor-core kernel then runs its variants for such plans: row blocks of two
+    # query tiles (up to 36 tokens), or of one tile (18 tokens) when asked
     compare_workload(wl, kernel=kernel, n_ctas=8)
+    compare_workload(wl, kernel=kernel, n_ctas=8, wide_rows=128)
 
 
-def test_wide_row_blocks_mixed_sizes_and_raised_maxima():
-    """The wide variant of the tensor-core kernel on a dealt plan whose row blocks have 1 to 18
-    tokens (7 to 126 rows: all three softmax layouts in one launch, tiles with padding rows,
-    requests whose only visible keys are their own), at the default scale and with logits x 4
-    (the reference maximum of a row is raised many times along its key stream; bounds derived as
-    for the peaked decode variant)."""
+@pytest.mark.parametrize("wide_rows", [128, 256])
+def test_wide_row_blocks_mixed_sizes_and_raised_maxima(wide_rows):
+    """The variants of the tensor-core kernel for dealt plans, on row blocks of 1 to 18 tokens (one
+    query tile: 7 to 126 rows, all three softmax layouts in one launch) or 1 to 36 tokens (two query
+    tiles, the second absent, partly or completely filled), tiles with padding rows, requests
+    whose only visible keys are their own, at the default scale and with logits x 4 (the reference
+    maximum of a row is raised many times along its key stream; bounds derived as for the peaked
+    decode variant)."""
     E = engine()
     wl = W.build_segment_workload("wide", 37, 28, 4, 128, "bf16", 1e6, [700, 33, 0, 129], [[0, 40, 3], [5], [0, 0], [200]],
                                   [[130, 9, 4], [1], [20, 3], [57]], serial_steps=1)
     shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
     ph = [x for x in wl.phases if x.mode == W.MODE_BRANCH and x.q is not None][-1]
-    plan = B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode, n_ctas=5, host_only=True)
+    plan = B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode, n_ctas=5, host_only=True, wide_rows=wide_rows)
     ntok = plan.items()["n_q_tok"]
-    assert ntok.max() == 18 and ntok.min() <= 4 and ((ntok > 4) & (ntok <= 9)).any()
+    if wide_rows == 128:
+        assert ntok.max() == 18 and ntok.min() <= 4 and ((ntok > 4) & (ntok <= 9)).any()
+    else:
+        assert plan.info.max_rows_per_item == 256 and ntok.max() == 36 and ntok.min() == 1 and ((ntok > 18) & (ntok < 36)).any()
     plan.destroy()
-    compare_workload(wl, n_ctas=5)
-    compare_workload(wl, n_ctas=5, fused=True)
+    compare_workload(wl, n_ctas=5, wide_rows=wide_rows)
+    compare_workload(wl, n_ctas=5, fused=True, wide_rows=wide_rows)
     wl.sm_scale *= 4.0
     ref = oracle_run(wl)
-    run = E.run_workload(wl, n_ctas=5)
+    run = E.run_workload(wl, n_ctas=5, wide_rows=wide_rows)
     g, r = run.outputs[0].astype(np.float64), ref.outputs[0]
     err = np.abs(g - r)
     assert err.max() <= 6e-2 and err.mean() <= 4e-3
+    # logits x 16: exponents pass 2^40 along a row's key stream, where the two-tile variant raises its
+    # reference (the one-tile variants raise theirs at 2^8 and did so above already).  The softmax is
+    # close to an argmax here and the bf16 keys decide between near-equal candidates differently from
+    # the oracle's exact ones for some rows, so only gross errors are excluded: finite, a loose mean
+    # bound, and most rows agree closely.
+    wl.sm_scale *= 4.0
+    ref = oracle_run(wl)
+    run = E.run_workload(wl, n_ctas=5, wide_rows=wide_rows)
+    g, r = run.outputs[0].astype(np.float64), ref.outputs[0]
+    err = np.abs(g - r)
+    assert np.isfinite(g).all() and err.mean() <= 3e-2
+    assert (err.reshape(err.shape[0], -1).max(axis=1) <= 0.1).mean() >= 0.8
     assert np.linalg.norm(g - r) / np.linalg.norm(r) <= 1e-2
 
 

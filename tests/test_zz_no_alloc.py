@@ -113,7 +113,7 @@ def test_static_scratch_runs_the_plans_other_regimes():
     run, ph, q, ref = _setup(wl)
     want = ref.float().cpu().numpy()
     wide = B.Plan(run.shape, ph.desc, wl.n_pool_pages, ph.mode, n_ctas=8, host_only=True)
-    assert wide.info.max_rows_per_item == 128
+    assert wide.info.max_rows_per_item == 256
     out = torch.full_like(q, float("nan"))
     B.attn_static(wide, q, run.cache.k, run.cache.v, out)
     torch.cuda.synchronize()
