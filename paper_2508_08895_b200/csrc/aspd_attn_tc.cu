@@ -42,6 +42,7 @@ constexpr int kSoftmaxThreads = 256;           // two warps per TMEM lane quadra
 constexpr int W_KPROD = 8, W_MMA = 9, W_VPROD = 11, W_EPI = 12;   // warp roles (0-7 softmax, 10 idle, 12-15 epilogue)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRaise = 8.0f;                 // raise the reference maximum only beyond 2^8
+constexpr float kLazyLimit = 1099511627776.0f;  // 2^40: a tile's sum of exponentials beyond which the reference is raised
 constexpr float kLower = 32.0f;                // wide variant: lower the initial reference (0) when a row's first keys are below 2^-32
 
 constexpr uint32_t kTileBytes = 32768;         // one K, V, Q or P tile: 128 rows x 256 B
@@ -166,9 +167,49 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
     if constexpr (HC == 32) ASPD_TMEM_LD32(s_addr, s, 0);
     else ASPD_TMEM_LD16(s_addr, s, 0);
     tmem_wait_ld();
-    tc_fence_before();
-    mbar_arrive(bars + 8 * (S_EMPTY + sb));
     if (tid == 0) ASPD_STAMP(c, g, 1);
+    // After an item's first tile the rows have a reference maximum, and a tile's exponentials are
+    // taken against it right away: one pass (mask, packed fp32 pairs, the exponentials), no maximum,
+    // no exchange between the threads of a row.  The reference then stays where it is unless an
+    // exponent passes 2^40, which shows in the sum; the barrier below ORs that over the CTA and the
+    // tile is redone the long way (scores read again from TMEM, row maximum exchanged, reference
+    // raised, O rescaled).  Everything is floating point, so a reference up to 2^40 below a row's
+    // true maximum costs no precision.
+    bool lazy = t > 0;
+    if (lazy) {
+      if (m_ref == -INFINITY) m_ref = 0.f;        // the row has seen nothing so far (l and O are 0): any reference will do
+      float2 lsum = make_float2(0.f, 0.f);
+      const float2 sc2 = make_float2(c.scale_log2, c.scale_log2), nm2 = make_float2(-m_ref, -m_ref);
+#pragma unroll
+      for (int pg = 0; pg < HC / 16; ++pg) {
+        const int ye = misc->nval[g & 3][col0 / 16 + pg], nv = ye & 255;
+        const int kb = it.key0 + t * kTile + col0 + pg * 16;
+        const uint32_t mask = bits_between(0, min(nv, vis.x - kb)) | bits_between(vis.y - kb, min(nv, vis.z - kb)) |
+                              bits_between(0, min(nv, vis.w - (ye >> 13) * 16));
+#pragma unroll
+        for (int i = 0; i < 16; i += 2) {
+          float2 x = __ffma2_rn(make_float2(s[pg * 16 + i], s[pg * 16 + i + 1]), sc2, nm2);
+          if (mask != 0xFFFFu) {
+            x.x = (mask >> i) & 1u ? x.x : -INFINITY;
+            x.y = (mask >> (i + 1)) & 1u ? x.y : -INFINITY;
+          }
+          x.x = ex2(x.x); x.y = ex2(x.y);
+          s[pg * 16 + i] = x.x; s[pg * 16 + i + 1] = x.y;
+          lsum = __fadd2_rn(lsum, x);
+        }
+      }
+      const float tsum = lsum.x + lsum.y;
+      lazy = !named_sync_or(1, kSoftmaxThreads, !(tsum <= kLazyLimit));
+      if (lazy) {
+        l += tsum;
+      } else {                                     // rare: the scores again, then the long way
+        if constexpr (HC == 32) ASPD_TMEM_LD32(s_addr, s, 0);
+        else ASPD_TMEM_LD16(s_addr, s, 0);
+        tmem_wait_ld();
+      }
+    }
+    if (tid == 0) ASPD_STAMP(c, g, 2);
+    if (!lazy) {
     // visibility of my HC keys: valid rows of each page, and the token's ranges [0, pe), [lo, hi)
     float mx = -INFINITY;
 #pragma unroll
@@ -193,7 +234,6 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
     mx *= c.scale_log2;                           // the scale is positive: max commutes with it
     misc->smax[sb][tid] = mx;
     named_sync(1, kSoftmaxThreads);
-    if (tid == 0) ASPD_STAMP(c, g, 2);
     float m_tile = mx;
 #pragma unroll
     for (int jj = 0; jj < KS; ++jj)
@@ -221,15 +261,19 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
       }
     }
     const float nmsafe = m_ref == -INFINITY ? 0.f : -m_ref;
-    float lsum0 = 0.f, lsum1 = 0.f;
+    float2 lsum = make_float2(0.f, 0.f);
+    const float2 sc2 = make_float2(c.scale_log2, c.scale_log2), nm2 = make_float2(nmsafe, nmsafe);
 #pragma unroll
-    for (int i = 0; i < HC; i += 2) {             // p = 2^(s * scale - m): one FFMA, one MUFU
-      s[i] = ex2(fmaf(s[i], c.scale_log2, nmsafe));
-      s[i + 1] = ex2(fmaf(s[i + 1], c.scale_log2, nmsafe));
-      lsum0 += s[i];
-      lsum1 += s[i + 1];
+    for (int i = 0; i < HC; i += 2) {             // p = 2^(s * scale - m): packed fp32 pairs (one FFMA, one FADD per two scores), two MUFU
+      float2 x = __ffma2_rn(make_float2(s[i], s[i + 1]), sc2, nm2);
+      x.x = ex2(x.x); x.y = ex2(x.y);
+      s[i] = x.x; s[i + 1] = x.y;
+      lsum = __fadd2_rn(lsum, x);
     }
-    l += lsum0 + lsum1;
+    l += lsum.x + lsum.y;
+    }
+    tc_fence_before();
+    mbar_arrive(bars + 8 * (S_EMPTY + sb));       // the scores are not needed again
     if (tid == 0) ASPD_STAMP(c, g, 3);
     if (g > 0) dead |= !mbar_wait(bars + 8 * P_EMPTY, (g - 1) & 1, ab);   // P tile is free again
     if (tid == 0) ASPD_STAMP(c, g, 4);
