@@ -26,6 +26,8 @@ constexpr uint32_t W2_OFF_K = 0, W2_OFF_V = 2 * kTileBytes, W2_OFF_Q = 4 * kTile
 constexpr uint32_t kPHalfBytes = 16384;       // 128 rows x 64 keys x 2 B: one 128-byte-swizzle span
 constexpr size_t kSmemBytesW2 = 7 * kTileBytes + 2048 + 1024;   // + Misc + slack to align the base to 1024
 constexpr int kItemCacheW2 = 8;
+constexpr bool kSplitS = true;     // scores of a tile as two MMAs of 64 keys (own columns and barriers each: a half's columns are
+                                   // free again as soon as its pass is final) or one of 128 (measured: 1141 against 1021 us)
 // The reference maximum of a row is raised when an exponent passes 2^40 (everything is floating point,
 // bf16 and fp32 alike, so the distance costs no precision; what must not happen is an overflow, and
 // 2^40 x 2^13 keys x |v| is far from one).  The one-tile variants raise at 2^8.
@@ -86,9 +88,12 @@ __device__ __forceinline__ void softmax_group_w2(const Ctx& c, MiscW2* misc, uin
       for (int h = 0; h < halves; ++h, ++hc) {
         // The scores of the two halves are separate MMAs into separate columns: a half's columns are
         // given back as soon as its pass is final, so its next scores are there before they are needed.
-        dead |= !mbar_wait(bar_sfull + 8 * h, sc[h] & 1, ab);
-        ++sc[h];
-        tc_fence_after();
+        if (kSplitS || h == 0) {
+          dead |= !mbar_wait(bar_sfull + 8 * h, sc[h] & 1, ab);
+          ++sc[h];
+          tc_fence_after();
+        }
+        if (tid == 0) ASPD_STAMP(c, g, 4 * h);
         uint32_t pk[32];
         float tile_sum, tmax;
         // p = 2^(s * scale - ref) for the thread's 64 scores of this half.  The common pass does not
@@ -169,9 +174,13 @@ __device__ __forceinline__ void softmax_group_w2(const Ctx& c, MiscW2* misc, uin
           pass(m_ref, std::false_type());           // the whole warp again (TMEM loads are warp-wide)
         }
         l += tile_sum;
-        tc_fence_before();                          // this half's scores are read: the MMA warp may overwrite them
-        mbar_arrive(bar_sempty + 8 * h);
+        if (kSplitS || h == halves - 1) {           // the scores are read: the MMA warp may overwrite them
+          tc_fence_before();
+          mbar_arrive(bar_sempty + (kSplitS ? 8 * h : 0));
+        }
+        if (tid == 0) ASPD_STAMP(c, g, 4 * h + 1);
         if (hc > 0) dead |= !mbar_wait(bar_pempty, (hc - 1) & 1, ab);   // the P half buffer is free again
+        if (tid == 0) ASPD_STAMP(c, g, 4 * h + 2);
 #pragma unroll
         for (int c8 = 0; c8 < 8; ++c8) {
           const uint32_t addr = pbuf + r * 128 + ((c8 ^ (r & 7)) << 4);
@@ -181,6 +190,7 @@ __device__ __forceinline__ void softmax_group_w2(const Ctx& c, MiscW2* misc, uin
         fence_async_smem();
         tc_fence_before();
         mbar_arrive(bar_pfull);
+        if (tid == 0) ASPD_STAMP(c, g, 4 * h + 3);
       }
     }
     // ---- the row is complete: normalise and store it
@@ -295,6 +305,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_w2_kernel(Ctx c) {
         if (lane == 0) good = mbar_wait(empty, ((g >> 1) & 1) ^ 1, ab) ? 1 : 0;
         good = __shfl_sync(0xffffffffu, good, 0);
         if (!good) { ok = false; break; }
+        if (lane == 0) ASPD_STAMP(c, g, 13 + kv);
         if (kv == 0 && lane < 8) misc->nval[g & 3][lane] = pg.y;   // read by the softmax groups of tile g
         __syncwarp();
         if (lane == 0) mbar_expect_tx(full, (uint32_t)npg * 4096u);
@@ -356,6 +367,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_w2_kernel(Ctx c) {
             }
           }
           tc_commit_lane0(bars_u + 8 * (WP_EMPTY + grp));
+          if (lane == 0 && grp == 0) ASPD_STAMP(c, g, 10 + u.h);
           const bool last_half = u.h == halves - 1;
           if (last_half) {
             tc_commit_lane0(bars_u + 8 * (WV_EMPTY + (g & 1)));
@@ -374,13 +386,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_w2_kernel(Ctx c) {
       // ---- S_grp = Q_grp . K^T for half h of tile t (keys 64 h ... of the tile)
       if (!cs.done && reached(0, cs.idx)) {
         Cur& v = cs;
-        const int g = v.gbase + v.t, sb = g & 1, npg = min(8, v.n_pages - v.t * 8), halves = npg > 4 ? 2 : 1, item_no = v.idx - ib;
+        const int g = v.gbase + v.t, sb = g & 1, npg = min(8, v.n_pages - v.t * 8), halves = (kSplitS && npg > 4) ? 2 : 1, item_no = v.idx - ib;
         const int cnt = v.h ? v.count1 : v.count;
         if ((v.t > 0 || v.h > 0 || ready(bars_u + 8 * WQ_FULL, item_no & 1)) && ready(bars_u + 8 * (WK_FULL + sb), (g >> 1) & 1) &&
             ready(bars_u + 8 * (WS_EMPTY + 2 * grp + v.h), (cnt & 1) ^ 1)) {
           tc_fence_after();
           const uint32_t qbuf = base_u + W2_OFF_Q + grp * kTileBytes, kbuf = base_u + W2_OFF_K + sb * kTileBytes + v.h * 16384;
-          const uint32_t idesc_s = instr_desc((uint32_t)min(4, npg - 4 * v.h) * 16u, 0);
+          const uint32_t idesc_s = instr_desc((uint32_t)(kSplitS ? min(4, npg - 4 * v.h) : npg) * 16u, 0);
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
             const uint64_t a = smem_desc(qbuf + (ks >> 2) * kHalf + (ks & 3) * 32, 16, 1024);
@@ -388,6 +400,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_w2_kernel(Ctx c) {
             tc_mma_lane0(tmem_u + COL_S + grp * 128 + v.h * 64, a, b, idesc_s, ks > 0 ? 1u : 0u);
           }
           tc_commit_lane0(bars_u + 8 * (WS_FULL + 2 * grp + v.h));
+          if (lane == 0 && grp == 0) ASPD_STAMP(c, g, 8 + v.h);
           if (v.h) ++v.count1; else ++v.count;
           if (v.h == halves - 1) {
             tc_commit_lane0(bars_u + 8 * (WK_EMPTY + sb));
