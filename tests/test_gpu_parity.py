@@ -550,6 +550,28 @@ def test_wide_row_blocks_mixed_sizes_and_raised_maxima(wide_rows):
     assert np.linalg.norm(g - r) / np.linalg.norm(r) <= 1e-2
 
 
+@pytest.mark.parametrize("n_ctas", [1, 2, 7])
+def test_two_tile_row_blocks_at_their_edges(n_ctas):
+    """The two-tile variant where its bookkeeping changes: requests with exactly 18, 19, 35, 36, 37 and
+    73 query tokens (a second tile that is absent, holds one token, is one short of full, full; a
+    block boundary crossed by one token; three blocks), an empty prefix, key streams of 1 to 9+
+    pages (tiles whose second half has no keys), and a single CTA that walks more items than it
+    caches in shared memory, so that the second group sits out whole runs of items."""
+    wl = W.build_segment_workload("w2edge", 59, 28, 4, 128, "bf16", 1e6, [0, 3, 70, 129, 16, 250, 40],
+                                  [[0], [1], [0, 0], [5], [0, 2], [0, 9, 0], [0, 0, 0, 0]],
+                                  [[18], [19], [35, 1], [36], [37, 3], [73, 2, 20], [1, 2, 18, 19]], serial_steps=1)
+    shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
+    ph = [x for x in wl.phases if x.mode == W.MODE_BRANCH and x.q is not None][-1]
+    plan = B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode, n_ctas=n_ctas, host_only=True)
+    items = plan.items()
+    assert plan.info.dealt and plan.info.max_rows_per_item == 256 and plan.info.n_ctas == n_ctas
+    assert {4, 18, 19, 23, 36}.issubset(set(int(x) for x in items["n_q_tok"]))
+    assert int(np.diff(plan.cta_ranges()).max()) > 8 or n_ctas > 2
+    plan.destroy()
+    compare_workload(wl, n_ctas=n_ctas)
+    compare_workload(wl, n_ctas=n_ctas, fused=True, stable_cache=True)
+
+
 def test_large_decode_batch_takes_the_dealt_plan():
     """A decode step with many more (request, KV head) streams than CTAs: whole streams are dealt
     out, the append is still fused into the attention launch (few new rows per CTA), the kernel
