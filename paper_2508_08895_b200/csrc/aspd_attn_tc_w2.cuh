@@ -7,15 +7,16 @@
 //     S_j = Q_j . K^T        tcgen05.mma M=128, N=keys, K=128       TMEM columns 128 j
 //     softmax group j        four warps, thread r = row r of tile j: the tile's keys in two halves of
 //                            64, exponentials against the row's reference maximum (raised only when
-//                            an exponent passes 2^8, judged by the thread alone: no exchange), P half
-//                            (128 rows x 64 keys, bf16) to shared memory
-//     O_j += P_j . V         tcgen05.mma M=128, N=128, K=64 per half   TMEM columns 256 + 128 j
+//                            an exponent passes 2^40, judged by the thread alone: no exchange), P half
+//                            (64 keys, bf16) over the first 32 columns of the half's own scores
+//     O_j += P_j . V         tcgen05.mma M=128, N=128, K=64 per half, A operand from tensor memory
+//                            TMEM columns 256 + 128 j
 //
 // so that while one group is in its exponentials the tensor pipe works for the other, and a thread
 // owns its row from the first score to the normalised output (it divides by l and stores the row
 // itself; there are no statistics to hand over).  Each group has an MMA warp with two cursors (S and P.V of the
 // group) and issues whichever has its operands ready.  Warp roles: 0-3 group 0, 4-7 group 1, 8 / 11
-// K / V producers, 9 / 10 MMA issuers of group 0 / 1, 12-15 query preparation.  Single buffers for S, P halves
+// K / V producers, 9 / 10 MMA issuers of group 0 / 1, 12-15 query preparation.  Single buffers for S (by halves)
 // and the query tiles; K and V tiles double-buffered.  All waits are bounded as in the other variants.
 #pragma once
 
@@ -26,6 +27,8 @@ constexpr uint32_t W2_OFF_K = 0, W2_OFF_V = 2 * kTileBytes, W2_OFF_Q = 4 * kTile
 constexpr uint32_t kPHalfBytes = 16384;       // 128 rows x 64 keys x 2 B: one 128-byte-swizzle span
 constexpr size_t kSmemBytesW2 = 7 * kTileBytes + 2048 + 1024;   // + Misc + slack to align the base to 1024
 constexpr int kItemCacheW2 = 8;
+constexpr bool kPInTmem = true;    // P halves go into the first 32 columns of their own score half in tensor memory and are the
+                                   // A operand of P.V from there (no shared-memory round trip); needs kSplitS
 constexpr bool kSplitS = true;     // scores of a tile as two MMAs of 64 keys (own columns and barriers each: a half's columns are
                                    // free again as soon as its pass is final) or one of 128 (measured: 1141 against 1021 us)
 // The reference maximum of a row is raised when an exponent passes 2^40 (everything is floating point,
@@ -36,6 +39,8 @@ constexpr float kRaiseW2 = 40.0f, kRaiseSumW2 = 1099511627776.0f;
 // S_FULL / S_EMPTY: one per (group, half of the tile's keys)
 enum BarW2 { WK_FULL = 0, WK_EMPTY = 2, WV_FULL = 4, WV_EMPTY = 6, WS_FULL = 8, WS_EMPTY = 12, WP_FULL = 16, WP_EMPTY = 18,
              WO_FULL = 20, WQ_FULL = 22, WQ_EMPTY = 23, W2_NUM_BARS = 24 };
+
+static_assert(kSplitS || !kPInTmem, "P in tensor memory lives in its own score half: the scores must be issued by halves");
 
 struct MiscW2 {
   uint64_t bars[W2_NUM_BARS];
@@ -174,20 +179,31 @@ __device__ __forceinline__ void softmax_group_w2(const Ctx& c, MiscW2* misc, uin
           pass(m_ref, std::false_type());           // the whole warp again (TMEM loads are warp-wide)
         }
         l += tile_sum;
-        if (kSplitS || h == halves - 1) {           // the scores are read: the MMA warp may overwrite them
+        if (!kPInTmem && (kSplitS || h == halves - 1)) {   // the scores are read: the MMA warp may overwrite them
           tc_fence_before();
           mbar_arrive(bar_sempty + (kSplitS ? 8 * h : 0));
         }
         if (tid == 0) ASPD_STAMP(c, g, 4 * h + 1);
-        if (hc > 0) dead |= !mbar_wait(bar_pempty, (hc - 1) & 1, ab);   // the P half buffer is free again
-        if (tid == 0) ASPD_STAMP(c, g, 4 * h + 2);
+        if constexpr (kPInTmem) {
+          // the half's P (64 bf16 = 32 columns) over its own scores, which nobody needs any more: the
+          // MMA warp frees these columns for the next tile's scores when this half's P.V is done
+          ASPD_TMEM_ST32U(s_base + h * 64, pk, 0);
+          tmem_wait_st();
+          // one barrier announces both halves in turn, and a parity tells only its two latest phases
+          // apart: the previous half's P.V must have been taken before this half is announced
+          if (hc > 0) dead |= !mbar_wait(bar_pempty, (hc - 1) & 1, ab);
+          if (tid == 0) ASPD_STAMP(c, g, 4 * h + 2);
+        } else {
+          if (hc > 0) dead |= !mbar_wait(bar_pempty, (hc - 1) & 1, ab);   // the P half buffer is free again
+          if (tid == 0) ASPD_STAMP(c, g, 4 * h + 2);
 #pragma unroll
-        for (int c8 = 0; c8 < 8; ++c8) {
-          const uint32_t addr = pbuf + r * 128 + ((c8 ^ (r & 7)) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[c8 * 4 + 0]), "r"(pk[c8 * 4 + 1]),
-                       "r"(pk[c8 * 4 + 2]), "r"(pk[c8 * 4 + 3]) : "memory");
+          for (int c8 = 0; c8 < 8; ++c8) {
+            const uint32_t addr = pbuf + r * 128 + ((c8 ^ (r & 7)) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[c8 * 4 + 0]), "r"(pk[c8 * 4 + 1]),
+                         "r"(pk[c8 * 4 + 2]), "r"(pk[c8 * 4 + 3]) : "memory");
+          }
+          fence_async_smem();
         }
-        fence_async_smem();
         tc_fence_before();
         mbar_arrive(bar_pfull);
         if (tid == 0) ASPD_STAMP(c, g, 4 * h + 3);
@@ -242,7 +258,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_w2_kernel(Ctx c) {
   }
   if (tid == 0) {
     //                               K_FULL K_EMPTY V_FULL V_EMPTY S_FULL(4)   S_EMPTY(4)          P_FULL    P_EMPTY O_FULL Q_FULL Q_EMPTY
-    const int counts[W2_NUM_BARS] = {1, 1,  2, 2,   1, 1,  2, 2,   1, 1, 1, 1,  128, 128, 128, 128, 128, 128, 1, 1,   1, 1,  128,   2};
+    const int se = kPInTmem ? 1 : 128;      // who gives a score half's columns back: the MMA warp's commit, or the 128 threads that read them
+    const int counts[W2_NUM_BARS] = {1, 1,  2, 2,   1, 1,  2, 2,   1, 1, 1, 1,  se, se, se, se, 128, 128, 1, 1,   1, 1,  128,   2};
     for (int i = 0; i < W2_NUM_BARS; ++i) mbar_init(bars + 8 * i, counts[i]);
     misc->abort_flag = 0;
     misc->lead[0] = item_begin; misc->lead[1] = item_begin;
@@ -361,12 +378,18 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_w2_kernel(Ctx c) {
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) {
             if (ks < n) {
-              const uint64_t a = smem_desc(pbuf + ks * 32, 16, 1024);
               const uint64_t b = smem_desc(vbuf + (4 * u.h + ks) * 4096, 1024, 2048);   // 16 keys = one page per k-step
-              tc_mma_lane0(tmem_u + COL_O + grp * 128, a, b, idesc_pv, (u.t > 0 || u.h > 0 || ks > 0) ? 1u : 0u);
+              const uint32_t acc = (u.t > 0 || u.h > 0 || ks > 0) ? 1u : 0u;
+              if constexpr (kPInTmem) {
+                tc_mma_ts_lane0(tmem_u + COL_O + grp * 128, tmem_u + COL_S + grp * 128 + u.h * 64 + ks * 8, b, idesc_pv, acc);
+              } else {
+                const uint64_t a = smem_desc(pbuf + ks * 32, 16, 1024);
+                tc_mma_lane0(tmem_u + COL_O + grp * 128, a, b, idesc_pv, acc);
+              }
             }
           }
           tc_commit_lane0(bars_u + 8 * (WP_EMPTY + grp));
+          if constexpr (kPInTmem) tc_commit_lane0(bars_u + 8 * (WS_EMPTY + 2 * grp + u.h));   // the half's columns are free for the next scores
           if (lane == 0 && grp == 0) ASPD_STAMP(c, g, 10 + u.h);
           const bool last_half = u.h == halves - 1;
           if (last_half) {
