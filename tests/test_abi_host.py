@@ -31,6 +31,18 @@ def test_library_exports_every_declared_symbol():
 def test_struct_sizes_and_strerror():
     assert B.REQUEST_DTYPE.itemsize == 28 and B.BRANCH_DTYPE.itemsize == 16 and B.ITEM_DTYPE.itemsize == 40
     assert ctypes.sizeof(B.Shape) == 28
+    assert ctypes.sizeof(B.Tuning) == 36 and ctypes.sizeof(B.PlanInfo) == 72      # 9 and 12 int32 + 3 int64, as in aspd.h
+    # the header itself, through a C compiler: the binding's structs have the sizes C gives them
+    import subprocess, tempfile
+    src = ('#include <stdio.h>\n#include "aspd.h"\nint main(void) { printf("%zu %zu %zu %zu %zu %zu\\n", sizeof(aspd_request_t), '
+           'sizeof(aspd_branch_t), sizeof(aspd_shape_t), sizeof(aspd_tuning_t), sizeof(aspd_item_t), sizeof(aspd_plan_info_t)); return 0; }\n')
+    with tempfile.TemporaryDirectory() as tmp:
+        open(os.path.join(tmp, "s.c"), "w").write(src)
+        subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), os.path.join(tmp, "s.c"), "-o", os.path.join(tmp, "s")],
+                       check=True)
+        sizes = [int(x) for x in subprocess.run([os.path.join(tmp, "s")], capture_output=True, text=True, check=True).stdout.split()]
+    assert sizes == [B.REQUEST_DTYPE.itemsize, B.BRANCH_DTYPE.itemsize, ctypes.sizeof(B.Shape), ctypes.sizeof(B.Tuning),
+                     B.ITEM_DTYPE.itemsize, ctypes.sizeof(B.PlanInfo)]
     assert B.strerror(0) == "ok"
     for code in range(-7, 0):
         assert B.strerror(code) not in ("ok", "unknown status")
