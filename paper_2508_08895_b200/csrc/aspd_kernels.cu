@@ -409,8 +409,9 @@ int launch_combine(const aspd_plan* p, void* out, cudaStream_t s) {
   const dim3 block(128), grid((warps + 3) / 4);
   // Measured: with the attribute the combine's blocks wait on the SMs while the attention pass
   // ends, which wins a little on a large step (serving mix: 48.6 against 49.2 us per layer) and
-  // loses a lot on small ones (long context, one request: 24.9 against 17.6), so it follows the
-  // step's size.
+  // loses a lot on small ones (long context, one request: 24.9 against 17.6; also with the rows in a
+  // few blocks of 32 warps, so that only a few SMs hold combine blocks: 24.7 against 18.2), so it
+  // follows the step's size.
   const int which = p->algorithmic_bytes >= (128LL << 20) ? (kPdlCombine | kPdlCombineLarge) : kPdlCombine;
 #define ASPD_CMB(T, D) \
   return status_of(launch_pdl(which, combine_kernel<T, D>, grid, block, 0, s, p->dev, (T*)out, p->n_new, sh.n_q_heads, sh.n_kv_heads))
