@@ -7,7 +7,7 @@
 //     S_j = Q_j . K^T        tcgen05.mma M=128, N=keys, K=128       TMEM columns 128 j
 //     softmax group j        four warps, thread r = row r of tile j: the tile's keys in two halves of
 //                            64, exponentials against the row's reference maximum (raised only when
-//                            an exponent passes 2^40, judged by the thread alone: no exchange), P half
+//                            an exponent passes 2^40, decided by the thread alone: no exchange), P half
 //                            (64 keys, bf16) over the first 32 columns of the half's own scores
 //     O_j += P_j . V         tcgen05.mma M=128, N=128, K=64 per half, A operand from tensor memory
 //                            TMEM columns 256 + 128 j

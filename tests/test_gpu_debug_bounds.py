@@ -27,7 +27,7 @@ def _child_env():
 
 
 def test_parity_subset_is_green_on_the_checking_build():
-    """The same parity cases through kernels that check: identical verdicts and a clean status word
+    """The same parity cases through kernels that check: the same outcomes and a clean status word
     (the engine raises on a non-zero status after every step)."""
     sel = "config2 or ragged_edges or second_parallel_stage or shared_mask_variant or fused_step_appends or config4"
     res = subprocess.run([sys.executable, "-m", "pytest", os.path.join(ROOT, "tests", "test_gpu_parity.py"), "-x", "-q", "-m", "gpu",
