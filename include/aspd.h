@@ -122,6 +122,9 @@ typedef struct {
                            block, 128 (one tile) or 256 (two tiles scored against every K/V tile the CTA
                            fetches); 0 = automatic (256 when a request has more query tokens than one
                            tile holds)                                                                */
+  int32_t mma_m;        /* stream-K plans of the tensor-core kernel: M of its MMAs, 128 (the at most 64 query
+                           rows of a row block are replicated to fill 128 accumulator rows) or 64 (half the
+                           tensor work; the accumulators then use 16 lanes of each quadrant); 0 = automatic */
 } aspd_tuning_t;
 
 /* a7 of a stream-K plan of the tensor-core kernel.  KERNEL: the separate combine launch (what AUTO
@@ -178,6 +181,8 @@ typedef struct {
                                own, so n_stream_pages counts shared pages once per row block); 0: stream-K cuts */
   int32_t single_launch;    /* 1: the attention kernel merges the split-K records itself (ASPD_COMBINE_FUSED): the
                                attention and step calls are one launch; 0: a combine launch follows      */
+  int32_t mma_m;            /* M of the tensor-core kernel's MMAs in this plan: 128 or 64 (0: generic kernel) */
+  int32_t reserved;
   int64_t workspace_bytes;  /* device memory the plan holds                                 */
   int64_t kv_tokens_read;   /* cached tokens the step must read (each once)                 */
   int64_t algorithmic_bytes;/* K+V of those tokens + q in + out + appended K/V              */

@@ -41,7 +41,8 @@ class Shape(ctypes.Structure):
 class Tuning(ctypes.Structure):
     _fields_ = [("kernel", ctypes.c_int32), ("chunk_tokens", ctypes.c_int32), ("n_ctas", ctypes.c_int32),
                 ("host_only", ctypes.c_int32), ("stable_cache", ctypes.c_int32), ("mask", ctypes.c_int32),
-                ("updatable", ctypes.c_int32), ("combine", ctypes.c_int32), ("wide_rows", ctypes.c_int32)]
+                ("updatable", ctypes.c_int32), ("combine", ctypes.c_int32), ("wide_rows", ctypes.c_int32),
+                ("mma_m", ctypes.c_int32)]
 
 
 class PlanInfo(ctypes.Structure):
@@ -49,7 +50,7 @@ class PlanInfo(ctypes.Structure):
                 ("n_stream_pages", ctypes.c_int32), ("kernel", ctypes.c_int32), ("chunk_tokens", ctypes.c_int32),
                 ("n_ctas", ctypes.c_int32), ("fused_append", ctypes.c_int32),
                 ("direct_output", ctypes.c_int32), ("max_rows_per_item", ctypes.c_int32),
-                ("dealt", ctypes.c_int32), ("single_launch", ctypes.c_int32),
+                ("dealt", ctypes.c_int32), ("single_launch", ctypes.c_int32), ("mma_m", ctypes.c_int32), ("reserved", ctypes.c_int32),
                 ("workspace_bytes", ctypes.c_int64), ("kv_tokens_read", ctypes.c_int64),
                 ("algorithmic_bytes", ctypes.c_int64)]
 
@@ -209,10 +210,10 @@ class Plan:
 
     def __init__(self, shape: Shape, desc, n_pool_pages: int, mode: int, q_pos=None, kernel: int = KERNEL_AUTO,
                  chunk_tokens: int = 0, n_ctas: int = 0, host_only: bool = False, stable_cache: bool = False, stream=None,
-                 mask: int = 0, updatable: bool = False, combine: int = COMBINE_AUTO, wide_rows: int = 0):
+                 mask: int = 0, updatable: bool = False, combine: int = COMBINE_AUTO, wide_rows: int = 0, mma_m: int = 0):
         self.shape, self.mode = shape, mode
         req, br, pages = pack_descriptors(desc)
-        tune = Tuning(kernel, chunk_tokens, n_ctas, 1 if host_only else 0, 1 if stable_cache else 0, mask, 1 if updatable else 0, combine, wide_rows)
+        tune = Tuning(kernel, chunk_tokens, n_ctas, 1 if host_only else 0, 1 if stable_cache else 0, mask, 1 if updatable else 0, combine, wide_rows, mma_m)
         qp = None if q_pos is None else np.ascontiguousarray(q_pos, dtype=np.int32)
         handle = ctypes.c_void_p()
         self._h = None

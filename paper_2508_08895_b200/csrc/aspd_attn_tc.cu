@@ -108,6 +108,7 @@ struct Ctx {
   int n_items, n_q_heads, n_kv_heads;
   float scale_log2;
   int early_fetch;             // plan promise: pages without new rows are not written by in-flight work
+  int m64;                     // MMAs with M = 64: row blocks of at most 64 rows are not padded to 128 (half the tensor work)
   int stagger_start;           // plans with few tiles per CTA: the first K tile is requested ahead of the other first tiles
   __nv_bfloat16* out;          // non-null (plans with one item per (token, KV head)): the epilogue writes O / l here
   __nv_bfloat16* merge_out;    // non-null (single-launch plans): the CTA that stores the last record of a (token, KV
@@ -298,6 +299,177 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
   return !named_sync_or(1, kSoftmaxThreads, dead || *ab);
 }
 
+// The same role for MMAs with M = 64 (half the tensor work of M = 128 for row blocks of at most 64 rows):
+// the 64 accumulator rows hold the R = 32 or 64 padded query rows KS = 64 / R times, and sit in lanes
+// 0..15 of each 32-lane quadrant (row 16 q + i in lane i of quadrant q).  A warp reads its quadrant's 16
+// lanes with the 16x256b shape, so all 32 threads get data: thread t holds, of every block of 8 columns,
+// columns 2 (t % 4), + 1 of rows 16 q + t / 4 and 16 q + t / 4 + 8.  Warps w and w + 4 again take half of a
+// replica's key range each, so a thread has as many scores per tile as in the M = 128 layout, now of two
+// rows.  P pairs go to shared memory as 4-byte stores (the four threads of a quad fill a 16-byte chunk).
+template <int NC>   // NC = padded row count R
+__device__ __forceinline__ bool softmax_item_m64(const Ctx& c, const DeviceItem& it, Misc* misc, uint32_t bars, uint32_t smem_p,
+                                                 uint32_t tmem, int item_no, int& g) {
+  constexpr int R = NC, KS = 64 / NC, NCOL = 128 / KS, NH = NCOL / 2, NB = NH / 8;   // NB blocks of 8 columns per thread and tile
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int q = warp & 3, half = warp >> 2, cq = lane & 3, g8 = lane >> 2;
+  const int rho_a = 16 * q + g8, rho_b = rho_a + 8;          // accumulator rows of this thread
+  const int j = rho_a / R;                                     // their replica (the same for both: R is a multiple of 16)
+  const int ra = rho_a % R, rb = rho_b % R;                    // the query rows they stand for
+  const int col0 = j * NCOL + half * NH;                       // first tile column (key) of this thread
+  const int G = c.n_q_heads / c.n_kv_heads, M = it.n_q_tok * G;
+  const int n_tiles = (it.n_pages + 7) >> 3;
+  volatile int* ab = &misc->abort_flag;
+  int4 vis_a = make_int4(0, 0, 0, 0), vis_b = vis_a;           // padding rows see nothing
+  if (ra < M) vis_a = (item_no < kItemCache && ra / G < kMaxTokPerItem) ? misc->vis[item_no][ra / G] : c.pd.tok_vis[it.q_tok0 + ra / G];
+  if (rb < M) vis_b = (item_no < kItemCache && rb / G < kMaxTokPerItem) ? misc->vis[item_no][rb / G] : c.pd.tok_vis[it.q_tok0 + rb / G];
+  const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+  const bool o_owner = half == 0 && j == 0;                    // threads whose rows are rows of O
+  const int ob = item_no & 1;
+  float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
+  bool dead = false;
+  for (int t = 0; t < n_tiles; ++t, ++g) {
+    const int sb = g & 1;
+    dead |= !mbar_wait(bars + 8 * (S_FULL + sb), (g >> 1) & 1, ab);
+    tc_fence_after();
+    float s[4 * NB];
+    const uint32_t s_addr = tmem + lane_addr + COL_S + sb * 128 + col0;
+    if constexpr (NB == 8) ASPD_TMEM_LD16x256_X8(s_addr, s);
+    else ASPD_TMEM_LD16x256_X4(s_addr, s);
+    tmem_wait_ld();
+    // 16-bit masks of the pages this thread's columns lie in, per row
+    uint32_t mk_a[NH / 16], mk_b[NH / 16];
+#pragma unroll
+    for (int pg = 0; pg < NH / 16; ++pg) {
+      const int ye = misc->nval[g & 3][col0 / 16 + pg], nv = ye & 255;
+      const int kb = it.key0 + t * kTile + col0 + pg * 16;
+      const int sh = (ye >> 13) * 16;
+      mk_a[pg] = bits_between(0, min(nv, vis_a.x - kb)) | bits_between(vis_a.y - kb, min(nv, vis_a.z - kb)) | bits_between(0, min(nv, vis_a.w - sh));
+      mk_b[pg] = bits_between(0, min(nv, vis_b.x - kb)) | bits_between(vis_b.y - kb, min(nv, vis_b.z - kb)) | bits_between(0, min(nv, vis_b.w - sh));
+    }
+    bool lazy = t > 0;
+    if (lazy) {        // one pass against the rows' references (see softmax_item)
+      if (m_a == -INFINITY) m_a = 0.f;
+      if (m_b == -INFINITY) m_b = 0.f;
+      float2 sum_a = make_float2(0.f, 0.f), sum_b = sum_a;
+      const float2 sc2 = make_float2(c.scale_log2, c.scale_log2), nm_a = make_float2(-m_a, -m_a), nm_b = make_float2(-m_b, -m_b);
+#pragma unroll
+      for (int n = 0; n < NB; ++n) {
+        const int bit = (n & 1) * 8 + 2 * cq;
+        float2 xa = __ffma2_rn(make_float2(s[4 * n], s[4 * n + 1]), sc2, nm_a);
+        float2 xb = __ffma2_rn(make_float2(s[4 * n + 2], s[4 * n + 3]), sc2, nm_b);
+        const uint32_t ma = mk_a[n >> 1] >> bit, mb = mk_b[n >> 1] >> bit;
+        if ((ma & 3u) != 3u) { xa.x = ma & 1u ? xa.x : -INFINITY; xa.y = ma & 2u ? xa.y : -INFINITY; }
+        if ((mb & 3u) != 3u) { xb.x = mb & 1u ? xb.x : -INFINITY; xb.y = mb & 2u ? xb.y : -INFINITY; }
+        xa.x = ex2(xa.x); xa.y = ex2(xa.y); xb.x = ex2(xb.x); xb.y = ex2(xb.y);
+        s[4 * n] = xa.x; s[4 * n + 1] = xa.y; s[4 * n + 2] = xb.x; s[4 * n + 3] = xb.y;
+        sum_a = __fadd2_rn(sum_a, xa);
+        sum_b = __fadd2_rn(sum_b, xb);
+      }
+      const float ta = sum_a.x + sum_a.y, tb = sum_b.x + sum_b.y;
+      lazy = !named_sync_or(1, kSoftmaxThreads, !(ta <= kLazyLimit) || !(tb <= kLazyLimit));
+      if (lazy) {
+        l_a += ta; l_b += tb;
+      } else {                                     // rare: the scores again, then the long way
+        if constexpr (NB == 8) ASPD_TMEM_LD16x256_X8(s_addr, s);
+        else ASPD_TMEM_LD16x256_X4(s_addr, s);
+        tmem_wait_ld();
+      }
+    }
+    if (!lazy) {
+      float mx_a = -INFINITY, mx_b = -INFINITY;
+#pragma unroll
+      for (int n = 0; n < NB; ++n) {
+        const int bit = (n & 1) * 8 + 2 * cq;
+        const uint32_t ma = mk_a[n >> 1] >> bit, mb = mk_b[n >> 1] >> bit;
+        s[4 * n] = ma & 1u ? s[4 * n] : -INFINITY;         s[4 * n + 1] = ma & 2u ? s[4 * n + 1] : -INFINITY;
+        s[4 * n + 2] = mb & 1u ? s[4 * n + 2] : -INFINITY; s[4 * n + 3] = mb & 2u ? s[4 * n + 3] : -INFINITY;
+        mx_a = fmaxf(mx_a, fmaxf(s[4 * n], s[4 * n + 1]));
+        mx_b = fmaxf(mx_b, fmaxf(s[4 * n + 2], s[4 * n + 3]));
+      }
+      // row maxima: over the quad, then (through shared memory) over the two halves and the replicas
+#pragma unroll
+      for (int o = 1; o <= 2; o <<= 1) {
+        mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, o));
+        mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, o));
+      }
+      mx_a *= c.scale_log2; mx_b *= c.scale_log2;          // the scale is positive: max commutes with it
+      if (cq == 0) { misc->smax[sb][half * 64 + rho_a] = mx_a; misc->smax[sb][half * 64 + rho_b] = mx_b; }
+      named_sync(1, kSoftmaxThreads);
+      float t_a = -INFINITY, t_b = -INFINITY;
+#pragma unroll
+      for (int jj = 0; jj < KS; ++jj) {
+        t_a = fmaxf(t_a, fmaxf(misc->smax[sb][jj * R + ra], misc->smax[sb][64 + jj * R + ra]));
+        t_b = fmaxf(t_b, fmaxf(misc->smax[sb][jj * R + rb], misc->smax[sb][64 + jj * R + rb]));
+      }
+      const bool upd_a = t_a > m_a + kRaise, upd_b = t_b > m_b + kRaise;   // also the first finite maximum (m = -inf)
+      float al_a = 1.f, al_b = 1.f;
+      if (upd_a) { al_a = ex2(m_a - t_a); m_a = t_a; }
+      if (upd_b) { al_b = ex2(m_b - t_b); m_b = t_b; }
+      l_a *= al_a; l_b *= al_b;
+      if (t > 0 && o_owner) {                       // the owners of rows 0..R-1 rescale O in TMEM (warp-wide)
+        if (__any_sync(0xffffffffu, upd_a || upd_b)) {
+          dead |= !mbar_wait(bars + 8 * P_EMPTY, (g - 1) & 1, ab);   // PV of the previous tile is done
+          tc_fence_after();
+          const uint32_t o_addr = tmem + lane_addr + COL_O + ob * 128;
+#pragma unroll 1
+          for (int q4 = 0; q4 < 4; ++q4) {
+            float o[16];
+            ASPD_TMEM_LD16x256_X4(o_addr + q4 * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int n = 0; n < 4; ++n) { o[4 * n] *= al_a; o[4 * n + 1] *= al_a; o[4 * n + 2] *= al_b; o[4 * n + 3] *= al_b; }
+            ASPD_TMEM_ST16x256_X4(o_addr + q4 * 32, o);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+        }
+      }
+      const float na = m_a == -INFINITY ? 0.f : -m_a, nb = m_b == -INFINITY ? 0.f : -m_b;
+      float2 sum_a = make_float2(0.f, 0.f), sum_b = sum_a;
+      const float2 sc2 = make_float2(c.scale_log2, c.scale_log2), nm_a = make_float2(na, na), nm_b = make_float2(nb, nb);
+#pragma unroll
+      for (int n = 0; n < NB; ++n) {
+        float2 xa = __ffma2_rn(make_float2(s[4 * n], s[4 * n + 1]), sc2, nm_a);
+        float2 xb = __ffma2_rn(make_float2(s[4 * n + 2], s[4 * n + 3]), sc2, nm_b);
+        xa.x = ex2(xa.x); xa.y = ex2(xa.y); xb.x = ex2(xb.x); xb.y = ex2(xb.y);
+        s[4 * n] = xa.x; s[4 * n + 1] = xa.y; s[4 * n + 2] = xb.x; s[4 * n + 3] = xb.y;
+        sum_a = __fadd2_rn(sum_a, xa);
+        sum_b = __fadd2_rn(sum_b, xb);
+      }
+      l_a += sum_a.x + sum_a.y; l_b += sum_b.x + sum_b.y;
+    }
+    tc_fence_before();
+    mbar_arrive(bars + 8 * (S_EMPTY + sb));       // the scores are not needed again
+    if (g > 0) dead |= !mbar_wait(bars + 8 * P_EMPTY, (g - 1) & 1, ab);   // P tile is free again
+#pragma unroll
+    for (int n = 0; n < NB; ++n) {
+      const int kk = col0 + 8 * n;                 // first key of the 16-byte chunk the quad fills
+      const uint32_t ch = (uint32_t)(kk >> 6) * kHalf + 4u * cq;
+      const uint32_t addr_a = smem_p + ch + ra * 128 + ((((kk & 63) >> 3) ^ (ra & 7)) << 4);
+      const uint32_t addr_b = smem_p + ch + rb * 128 + ((((kk & 63) >> 3) ^ (rb & 7)) << 4);
+      asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr_a), "r"(pack_bf16(s[4 * n], s[4 * n + 1])) : "memory");
+      asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr_b), "r"(pack_bf16(s[4 * n + 2], s[4 * n + 3])) : "memory");
+    }
+    fence_async_smem();
+    tc_fence_before();
+    mbar_arrive(bars + 8 * P_FULL);
+  }
+  // ---- hand the item's statistics to the epilogue warps and move on to the next item
+  dead |= !mbar_wait(bars + 8 * (O_EMPTY + ob), ((item_no >> 1) & 1) ^ 1, ab);   // epilogue of item_no - 2 is done
+#pragma unroll
+  for (int o = 1; o <= 2; o <<= 1) {               // the quad's share of the rows' sums
+    l_a += __shfl_xor_sync(0xffffffffu, l_a, o);
+    l_b += __shfl_xor_sync(0xffffffffu, l_b, o);
+  }
+  if (cq == 0) {
+    if (o_owner) { misc->fin_m[ob][ra] = m_a; misc->fin_m[ob][rb] = m_b; }
+    misc->fin_l[ob][half * 128 + j * R + ra] = l_a;
+    misc->fin_l[ob][half * 128 + j * R + rb] = l_b;
+  }
+  mbar_arrive(bars + 8 * (E_FULL + ob));
+  return !named_sync_or(1, kSoftmaxThreads, dead || *ab);
+}
+
 // Row blocks of 65..128 query rows: every TMEM lane is a row of its own (no replication), thread
 // (half, r) takes columns [64 half, 64 half + 64) of row r in two chunks of 32.  One pass per
 // tile: the exponentials are taken against the current reference maximum while the largest
@@ -469,7 +641,7 @@ __device__ __forceinline__ void prep_q_compute(const Ctx& c, const DeviceItem& i
 __device__ __forceinline__ void prep_q_store(const Ctx& c, const DeviceItem& it, uint32_t qbuf, int rank, int e0, const QUnits& qu,
                                              bool tile128 = false) {
   const int G = c.n_q_heads / c.n_kv_heads;
-  const int M = it.n_q_tok * G, R = tile128 ? 128 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128)), KS = 128 / R;
+  const int M = it.n_q_tok * G, R = tile128 ? 128 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128)), KS = (c.m64 && !tile128 ? 64 : 128) / R;
 #pragma unroll
   for (int u = 0; u < 4; ++u) {
     const int e = e0 + rank + u * 128, r = e >> 3, ch = e & 7;
@@ -630,8 +802,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
            : M <= 64 ? softmax_item<64>(c, it, misc, bars, base + OFF_P, tmem, item_no, g)
                      : softmax_item_wide(c, it, misc, bars, base + OFF_P, tmem, item_no, g);
       } else {
-        ok = M <= 32 ? softmax_item<32>(c, it, misc, bars, base + OFF_P, tmem, item_no, g)
-                     : softmax_item<64>(c, it, misc, bars, base + OFF_P, tmem, item_no, g);
+        if (c.m64)
+          ok = M <= 32 ? softmax_item_m64<32>(c, it, misc, bars, base + OFF_P, tmem, item_no, g)
+                       : softmax_item_m64<64>(c, it, misc, bars, base + OFF_P, tmem, item_no, g);
+        else
+          ok = M <= 32 ? softmax_item<32>(c, it, misc, bars, base + OFF_P, tmem, item_no, g)
+                       : softmax_item<64>(c, it, misc, bars, base + OFF_P, tmem, item_no, g);
       }
       if (!ok) break;
     }
@@ -724,7 +900,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
       struct TileRef { int npg, first, last, qb, ob, item_no; };   // qb: query tile (always 0 in the wide kernel)
       auto q_fill = [](int item_no) { return WIDE ? item_no : item_no >> 1; };   // how often the item's query tile was filled before
       auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(full_mask, mbar_wait(bar, parity, ab)) != 0; };
-      const uint32_t idesc_pv = instr_desc(128, 1);
+      const uint32_t mma_m = c.m64 ? 64u : 128u;
+      const uint32_t idesc_pv = instr_desc(128, 1, mma_m);
       auto issue_s = [&](const TileRef& tr, int g) -> bool {
         const int sb = g & 1;
         if (tr.first && !wait_all(bars_u + 8 * (Q_FULL + tr.qb), q_fill(tr.item_no) & 1)) return false;
@@ -734,7 +911,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
         tc_fence_after();
         if (lane == 0) ASPD_STAMP(c, g, 8);
         const uint32_t qbuf = base_u + OFF_Q + tr.qb * kTileBytes, kbuf = base_u + OFF_K + sb * kTileBytes;
-        const uint32_t idesc_s = instr_desc((uint32_t)tr.npg * 16u, 0);
+        const uint32_t idesc_s = instr_desc((uint32_t)tr.npg * 16u, 0, mma_m);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
           // k-step ks covers head_dim elements [16 ks, 16 ks + 16): span ks / 4, 32 bytes per step
@@ -805,7 +982,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     }
     for (int idx = item_begin; idx < item_end; ++idx, ++item_no) {
       const DeviceItem it = get_item(c, misc, idx, item_begin);
-      const int ob = item_no & 1, M = it.n_q_tok * G, R = M <= 32 ? 32 : (M <= 64 ? 64 : 128), KS = 128 / R;
+      const bool m64 = !WIDE && c.m64;             // M = 64 accumulators: row 16 q + i sits in lane i < 16 of quadrant q
+      const int ob = item_no & 1, M = it.n_q_tok * G, R = M <= 32 ? 32 : (M <= 64 ? 64 : 128), KS = (m64 ? 64 : 128) / R;
       if (idx + 1 < item_end) {                    // the next item's query tile: into the other buffer, or (wide
         const int qn = WIDE ? 0 : (item_no + 1) & 1;   // kernel) into the only one once this item's last S is issued
         const int fills = WIDE ? item_no + 1 : (item_no + 1) >> 1;
@@ -835,8 +1013,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
       const bool merging = !WIDE && c.merge_out != nullptr;
       const bool direct = c.out != nullptr || (merging && it.n_parts == 1);
       __nv_bfloat16* const out_base = c.out != nullptr ? c.out : c.merge_out;
-      if (ew < R / 32) {
-        const int r = et;                          // row of O held by this thread's TMEM lane
+      if (ew < R / (m64 ? 16 : 32)) {
+        const int r = m64 ? ((et & 31) < 16 ? ew * 16 + (et & 31) : 1 << 20) : et;   // row of O held by this thread's TMEM lane
         size_t rec = 0;
         if (r < M && !direct) {
           const int tok = it.q_tok0 + r / G;
@@ -1000,6 +1178,7 @@ static int launch_tc(const aspd_plan* p, const void* q, const void* k_new, const
   c.scale_log2 = sh.sm_scale * kLog2e;
   c.early_fetch = p->stable_cache;
   c.stagger_start = p->stagger_start;
+  c.m64 = (p->m64 && !p->wide && !p->dealt) ? 1 : 0;
   c.out = p->dealt ? (__nv_bfloat16*)out : nullptr;   // only when every (token, KV head) has a single item
   c.merge_out = (!p->dealt && p->single_launch) ? (__nv_bfloat16*)out : nullptr;
   if (p->wide == 2) {                       // row blocks of two query tiles: final outputs only

@@ -111,6 +111,7 @@ struct aspd_plan {
   int dealt = 0;                   // whole streams dealt to the CTAs in turn (many more streams than CTAs)
   int shared_mask = 0;             // parallel step under the ablation's visible mask
   int wide = 0;                    // dealt plan of the tensor-core kernel: row blocks of up to kMaxRowsWide rows
+  int m64 = 0;                     // stream-K plan of the tensor-core kernel whose MMAs take M = 64 (row blocks are at most 64 rows)
   int stagger_start = 0;           // few tiles per CTA: order the requests of a CTA's first tiles (see the producers)
   int single_launch = 0;           // stream-K plan of the tensor-core kernel whose last-arriving CTAs merge the records themselves
   int64_t n_pool_pages = 0;

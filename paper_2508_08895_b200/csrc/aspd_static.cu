@@ -105,7 +105,7 @@ extern "C" int aspd_attn_static(const aspd_plan_t* plan, const void* q, const vo
   shell.chunk_tokens = plan->chunk_tokens; shell.n_ctas = plan->n_ctas; shell.host_only = 0;
   shell.sm_count = plan->sm_count; shell.n_row_blocks = plan->n_row_blocks; shell.stable_cache = 0; shell.fuse_append = 0; shell.n_pool_pages = plan->n_pool_pages;
   shell.kv_tokens_read = plan->kv_tokens_read; shell.algorithmic_bytes = plan->algorithmic_bytes;
-  shell.dealt = plan->dealt; shell.wide = plan->wide; shell.shared_mask = plan->shared_mask;   // which kernel variant the items were made for
+  shell.dealt = plan->dealt; shell.wide = plan->wide; shell.shared_mask = plan->shared_mask; shell.m64 = plan->m64;   // which kernel variant the items were made for
   shell.device_bytes = 0; shell.device_base = nullptr;
   memset(&shell.dev, 0, sizeof(shell.dev));
   shell.dev.items = (const DeviceItem*)(base + o_items);

@@ -146,6 +146,24 @@ __device__ __forceinline__ bool named_sync_or(int id, int n, bool pred) {
                  "=f"(v[o + 6]), "=f"(v[o + 7]), "=f"(v[o + 8]), "=f"(v[o + 9]), "=f"(v[o + 10]), "=f"(v[o + 11]), \
                  "=f"(v[o + 12]), "=f"(v[o + 13]), "=f"(v[o + 14]), "=f"(v[o + 15])                               \
                : "r"(taddr) : "memory")
+// 16 lanes x 256 bits per block, N blocks along the columns: thread t of the warp gets, per block of 8
+// columns, columns 2 (t % 4), + 1 of lane t / 4 (registers 4 n, 4 n + 1) and of lane t / 4 + 8 (4 n + 2,
+// 4 n + 3): the accumulator of an M = 64 MMA keeps 16 rows in lanes 0..15 of each 32-lane quadrant.
+#define ASPD_TMEM_LD16x256_X4(taddr, v)                                                                             \
+  asm volatile("tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, "    \
+               "%13, %14, %15}, [%16];"                                                                            \
+               : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]),    \
+                 "=f"(v[8]), "=f"(v[9]), "=f"(v[10]), "=f"(v[11]), "=f"(v[12]), "=f"(v[13]), "=f"(v[14]), "=f"(v[15]) \
+               : "r"(taddr) : "memory")
+#define ASPD_TMEM_LD16x256_X8(taddr, v)                                                                             \
+  asm volatile("tcgen05.ld.sync.aligned.16x256b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, "    \
+               "%13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, "   \
+               "[%32];" : ASPD_R32(v, 0) : "r"(taddr) : "memory")
+#define ASPD_TMEM_ST16x256_X4(taddr, v)                                                                             \
+  asm volatile("tcgen05.st.sync.aligned.16x256b.x4.b32 [%16], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, "  \
+               "%12, %13, %14, %15};"                                                                              \
+               ::"f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]), "f"(v[8]), \
+                 "f"(v[9]), "f"(v[10]), "f"(v[11]), "f"(v[12]), "f"(v[13]), "f"(v[14]), "f"(v[15]), "r"(taddr) : "memory")
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -154,9 +172,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
          (1ull << 46) | (2ull << 61);
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, A K-major.
-__device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128 (or 64), A K-major.
+__device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t b_mn_major, uint32_t m = 128u) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major << 16) | ((n >> 3) << 17) | ((m >> 4) << 24);
 }
 
 __device__ __forceinline__ float ex2(float x) {

@@ -62,11 +62,12 @@ class WorkloadRun:
 
     def __init__(self, wl: W.Workload, kernel: int = B.KERNEL_AUTO, chunk_tokens: int = 0, n_ctas: int = 0,
                  device="cuda", fused: bool = False, stable_cache: bool = False, mask: int = B.MASK_BRANCH_INVISIBLE,
-                 combine: int = B.COMBINE_AUTO, wide_rows: int = 0):
+                 combine: int = B.COMBINE_AUTO, wide_rows: int = 0, mma_m: int = 0):
         self.wl, self.kernel, self.chunk_tokens, self.n_ctas, self.device = wl, kernel, chunk_tokens, n_ctas, device
         self.mask = mask            # attention mask of the parallel steps (ASPD_MASK_*)
         self.combine = combine      # where the split-K records are merged (ASPD_COMBINE_*)
         self.wide_rows = wide_rows  # rows of a row block in plans that deal whole streams (0 = automatic)
+        self.mma_m = mma_m          # M of the tensor-core kernel's MMAs in stream-K plans (0 = automatic)
         self.stable_cache = stable_cache
         self.fused = fused          # attention phases go through aspd_branch_step / aspd_serial_step
         self.shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
@@ -81,7 +82,7 @@ class WorkloadRun:
         wl = self.wl
         plan = B.Plan(self.shape, ph.desc, wl.n_pool_pages, ph.mode, q_pos=pos_override, kernel=self.kernel,
                       chunk_tokens=self.chunk_tokens, n_ctas=self.n_ctas, stable_cache=self.stable_cache, mask=self.mask,
-                      combine=self.combine, wide_rows=self.wide_rows)
+                      combine=self.combine, wide_rows=self.wide_rows, mma_m=self.mma_m)
         pos, slot, req = B.positions(ph.desc, ph.mode)
         if pos_override is not None:
             pos = np.ascontiguousarray(pos_override, dtype=np.int32)

@@ -31,7 +31,7 @@ def test_library_exports_every_declared_symbol():
 def test_struct_sizes_and_strerror():
     assert B.REQUEST_DTYPE.itemsize == 28 and B.BRANCH_DTYPE.itemsize == 16 and B.ITEM_DTYPE.itemsize == 40
     assert ctypes.sizeof(B.Shape) == 28
-    assert ctypes.sizeof(B.Tuning) == 36 and ctypes.sizeof(B.PlanInfo) == 72      # 9 and 12 int32 + 3 int64, as in aspd.h
+    assert ctypes.sizeof(B.Tuning) == 40 and ctypes.sizeof(B.PlanInfo) == 80      # 10 and 14 int32 + 3 int64, as in aspd.h
     # the header itself, through a C compiler: the binding's structs have the sizes C gives them
     import subprocess, tempfile
     src = ('#include <stdio.h>\n#include "aspd.h"\nint main(void) { printf("%zu %zu %zu %zu %zu %zu\\n", sizeof(aspd_request_t), '

@@ -464,6 +464,43 @@ def test_position_id_variants(rule, fused):
     assert np.abs(plain.outputs[-1] - ref.outputs[-1]).max() > 1e-3     # the variant really differs from Eq. 4
 
 
+@pytest.mark.parametrize("mma_m", [64, 128])
+def test_mma_m_variants_on_the_decode_shapes(mma_m):
+    """The tensor-core kernel's stream-K path with M = 128 MMAs (rows replicated to fill the
+    accumulator) and with M = 64 (half the tensor work, accumulators in 16 lanes of each quadrant,
+    two rows per softmax thread): the serving mix (row blocks of 7 to 56 rows: both padded sizes,
+    one and two replicas), ragged edges, forced cuts with many items per CTA, a single CTA, the
+    visible mask, the fused step, a second stage and serial steps, at the default scale and with
+    logits x 4 (references raised along the stream: the long way of a tile, with O rescaled)."""
+    E = engine()
+    wl = W.config_serving_mix(n_req=12)
+    run, ref = compare_workload(wl, mma_m=mma_m)
+    compare_workload(wl, mma_m=mma_m, fused=True, stable_cache=True)
+    ph = wl.phases[-1]
+    plan = B.Plan(run.shape, ph.desc, wl.n_pool_pages, ph.mode, mma_m=mma_m, host_only=True)
+    assert plan.info.mma_m == mma_m and not plan.info.dealt
+    rows = plan.items()["n_q_tok"] * 7
+    assert (rows <= 32).any() and (rows > 32).any()
+    plan.destroy()
+    rag = W.build_segment_workload("ragged", 77, 28, 4, 128, "bf16", 1e6, [15, 16, 17, 0, 1, 300],
+                                   [[14, 15, 16], [0], [31, 0, 47, 1], [5, 0], [16], [255, 256, 1, 0, 99, 17, 33, 64]],
+                                   [[1, 1, 1], [1], [1, 1, 0, 1], [1, 1], [0], [1] * 8], serial_steps=2)
+    compare_workload(rag, mma_m=mma_m)
+    compare_workload(rag, mma_m=mma_m, mask=B.MASK_SHARED)
+    lr = W.config_long_rag(prefix=1024 + 7)
+    for chunk, n_ctas in ((16, 0), (448, 0), (0, 1), (48, 37)):
+        compare_workload(lr, mma_m=mma_m, chunk_tokens=chunk, n_ctas=n_ctas)
+    two = W.build_two_stage_workload("ts", 61, 28, 4, 128, "bf16", 1e6, 200, [30, 5, 41], 3, [17, 0, 6], [1, 1, 1], serial_steps=2)
+    compare_workload(two, mma_m=mma_m, fused=True)
+    peaked = W.config_qwen7b_layer()
+    peaked.sm_scale *= 4.0
+    ref = oracle_run(peaked)
+    run = E.run_workload(peaked, mma_m=mma_m)
+    check(run.outputs[0], ref.outputs[0], "bf16", "peaked", tol=PEAKED_TOL[B.KERNEL_AUTO])
+    # open step of config 3: 72 query tokens in row blocks of 9 (63 rows), several blocks per request
+    compare_workload(W.config_branch_open(serial_steps=2), mma_m=mma_m)
+
+
 @pytest.mark.parametrize("combine", [B.COMBINE_KERNEL, B.COMBINE_FUSED])
 def test_deterministic_across_repeated_launches(combine):
     """Repeated launches of the same step give bit-identical outputs (no data race in the
