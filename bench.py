@@ -940,7 +940,7 @@ def main():
     ap.add_argument("--ctas", type=int, default=0)
     ap.add_argument("--wide-rows", type=int, default=0, choices=[0, 128, 256],
                     help="plans that deal whole streams: query rows per row block (one or two tiles; 0 = automatic)")
-    ap.add_argument("--mma-m", type=int, default=0, choices=[0, 64, 128], help="stream-K plans: M of the tensor-core kernel's MMAs (0 = automatic)")
+    ap.add_argument("--mma-m", type=int, default=0, choices=[0, 64, 96, 128], help="stream-K plans: M of the tensor-core kernel's MMAs (0 = automatic)")
     ap.add_argument("--combine", default="auto", choices=["auto", "kernel", "fused"],
                     help="where the split-K records are merged: a combine launch, or inside the attention kernel (one launch per layer)")
     ap.add_argument("--requests", type=int, default=0, help="serving-mix only: number of requests (default 32)")

@@ -123,8 +123,9 @@ typedef struct {
                            fetches); 0 = automatic (256 when a request has more query tokens than one
                            tile holds)                                                                */
   int32_t mma_m;        /* stream-K plans of the tensor-core kernel: M of its MMAs, 128 (the at most 64 query
-                           rows of a row block are replicated to fill 128 accumulator rows) or 64 (half the
-                           tensor work; the accumulators then use 16 lanes of each quadrant); 0 = automatic */
+                           rows of a row block are replicated to fill 128 accumulator rows), 64 (half the
+                           tensor work; the accumulators then use 16 lanes of each quadrant) or 96, which
+                           stands for both: scores at M = 128, P.V at M = 64; 0 = automatic (96)        */
 } aspd_tuning_t;
 
 /* a7 of a stream-K plan of the tensor-core kernel.  KERNEL: the separate combine launch (what AUTO
@@ -181,7 +182,8 @@ typedef struct {
                                own, so n_stream_pages counts shared pages once per row block); 0: stream-K cuts */
   int32_t single_launch;    /* 1: the attention kernel merges the split-K records itself (ASPD_COMBINE_FUSED): the
                                attention and step calls are one launch; 0: a combine launch follows      */
-  int32_t mma_m;            /* M of the tensor-core kernel's MMAs in this plan: 128 or 64 (0: generic kernel) */
+  int32_t mma_m;            /* M of the tensor-core kernel's MMAs in this plan: 128, 64 or 96 (see aspd_tuning_t;
+                               0: generic kernel)                                                          */
   int32_t reserved;
   int64_t workspace_bytes;  /* device memory the plan holds                                 */
   int64_t kv_tokens_read;   /* cached tokens the step must read (each once)                 */

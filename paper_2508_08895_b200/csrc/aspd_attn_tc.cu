@@ -109,6 +109,8 @@ struct Ctx {
   float scale_log2;
   int early_fetch;             // plan promise: pages without new rows are not written by in-flight work
   int m64;                     // MMAs with M = 64: row blocks of at most 64 rows are not padded to 128 (half the tensor work)
+  int pv64;                    // only P.V with M = 64 (scores and the softmax layout stay at M = 128): O then sits in 16 lanes
+                               // of each quadrant (at most 64 of the 128 rows of P.V are ever read)
   int stagger_start;           // plans with few tiles per CTA: the first K tile is requested ahead of the other first tiles
   __nv_bfloat16* out;          // non-null (plans with one item per (token, KV head)): the epilogue writes O / l here
   __nv_bfloat16* merge_out;    // non-null (single-launch plans): the CTA that stores the last record of a (token, KV
@@ -243,7 +245,34 @@ __device__ __forceinline__ bool softmax_item(const Ctx& c, const DeviceItem& it,
     float alpha = 1.f;
     if (upd) { alpha = ex2(m_ref - m_tile); m_ref = m_tile; }
     l *= alpha;
-    if (t > 0 && o_owner) {                       // the owners of rows 0..R-1 rescale O in TMEM
+    if (t > 0 && c.pv64) {
+      // O comes from an M = 64 MMA: row 16 q + i sits in lane i of quadrant q, which is not the lane of
+      // the thread that knows the row's factor.  The factors go through shared memory (the other score
+      // buffer's exchange array is free), then warps 0..3 rescale their quadrant's 16 rows.
+      if (j == 0 && half == 0) misc->smax[sb ^ 1][r] = alpha;
+      named_sync(1, kSoftmaxThreads);
+      if (half == 0) {
+        const int lq = tid & 31, rq = (warp & 3) * 16 + (lq & 15);
+        const float a = (lq < 16 && rq < R) ? misc->smax[sb ^ 1][rq] : 1.f;
+        if (__any_sync(0xffffffffu, a != 1.f)) {
+          dead |= !mbar_wait(bars + 8 * P_EMPTY, (g - 1) & 1, ab);   // PV of the previous tile is done
+          tc_fence_after();
+          const uint32_t o_addr = tmem + lane_addr + COL_O + ob * 128;
+#pragma unroll 1
+          for (int q4 = 0; q4 < 4; ++q4) {
+            float o[32];
+            ASPD_TMEM_LD32(o_addr + q4 * 32, o, 0);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] *= a;
+            ASPD_TMEM_ST32(o_addr + q4 * 32, o, 0);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+        }
+      }
+      named_sync(1, kSoftmaxThreads);                // the array is written again in the next long tile
+    } else if (t > 0 && o_owner) {                // the owners of rows 0..R-1 rescale O in TMEM
       if (__any_sync(0xffffffffu, upd)) {
         dead |= !mbar_wait(bars + 8 * P_EMPTY, (g - 1) & 1, ab);   // PV of the previous tile is done
         tc_fence_after();
@@ -901,7 +930,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
       auto q_fill = [](int item_no) { return WIDE ? item_no : item_no >> 1; };   // how often the item's query tile was filled before
       auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(full_mask, mbar_wait(bar, parity, ab)) != 0; };
       const uint32_t mma_m = c.m64 ? 64u : 128u;
-      const uint32_t idesc_pv = instr_desc(128, 1, mma_m);
+      const uint32_t idesc_pv = instr_desc(128, 1, (c.m64 || c.pv64) ? 64u : 128u);
       auto issue_s = [&](const TileRef& tr, int g) -> bool {
         const int sb = g & 1;
         if (tr.first && !wait_all(bars_u + 8 * (Q_FULL + tr.qb), q_fill(tr.item_no) & 1)) return false;
@@ -982,8 +1011,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
     }
     for (int idx = item_begin; idx < item_end; ++idx, ++item_no) {
       const DeviceItem it = get_item(c, misc, idx, item_begin);
-      const bool m64 = !WIDE && c.m64;             // M = 64 accumulators: row 16 q + i sits in lane i < 16 of quadrant q
-      const int ob = item_no & 1, M = it.n_q_tok * G, R = M <= 32 ? 32 : (M <= 64 ? 64 : 128), KS = (m64 ? 64 : 128) / R;
+      const bool m64 = !WIDE && (c.m64 || c.pv64);  // O from an M = 64 MMA: row 16 q + i sits in lane i < 16 of quadrant q
+      const int ob = item_no & 1, M = it.n_q_tok * G, R = M <= 32 ? 32 : (M <= 64 ? 64 : 128),
+                KS = ((!WIDE && c.m64) ? 64 : 128) / R;                // replicas in the softmax threads' layout
       if (idx + 1 < item_end) {                    // the next item's query tile: into the other buffer, or (wide
         const int qn = WIDE ? 0 : (item_no + 1) & 1;   // kernel) into the only one once this item's last S is issued
         const int fills = WIDE ? item_no + 1 : (item_no + 1) >> 1;
@@ -1178,7 +1208,8 @@ static int launch_tc(const aspd_plan* p, const void* q, const void* k_new, const
   c.scale_log2 = sh.sm_scale * kLog2e;
   c.early_fetch = p->stable_cache;
   c.stagger_start = p->stagger_start;
-  c.m64 = (p->m64 && !p->wide && !p->dealt) ? 1 : 0;
+  c.m64 = (p->m64 == 1 && !p->wide && !p->dealt) ? 1 : 0;
+  c.pv64 = (p->m64 == 2 && !p->wide && !p->dealt) ? 1 : 0;
   c.out = p->dealt ? (__nv_bfloat16*)out : nullptr;   // only when every (token, KV head) has a single item
   c.merge_out = (!p->dealt && p->single_launch) ? (__nv_bfloat16*)out : nullptr;
   if (p->wide == 2) {                       // row blocks of two query tiles: final outputs only

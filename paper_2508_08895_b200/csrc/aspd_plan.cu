@@ -348,7 +348,7 @@ static int plan_create_impl(const aspd_shape_t* shape, const aspd_request_t* req
   if (tune.chunk_tokens < 0 || tune.chunk_tokens % ps || tune.n_ctas < 0) return ASPD_ERR_INVALID_ARG;
   if (tune.mask != ASPD_MASK_BRANCH_INVISIBLE && tune.mask != ASPD_MASK_SHARED) return ASPD_ERR_INVALID_ARG;
   if (tune.wide_rows != 0 && tune.wide_rows != 128 && tune.wide_rows != 256) return ASPD_ERR_INVALID_ARG;
-  if (tune.mma_m != 0 && tune.mma_m != 64 && tune.mma_m != 128) return ASPD_ERR_INVALID_ARG;
+  if (tune.mma_m != 0 && tune.mma_m != 64 && tune.mma_m != 96 && tune.mma_m != 128) return ASPD_ERR_INVALID_ARG;
   if (tune.combine != ASPD_COMBINE_AUTO && tune.combine != ASPD_COMBINE_KERNEL && tune.combine != ASPD_COMBINE_FUSED) return ASPD_ERR_INVALID_ARG;
   const bool shared_mask = tune.mask == ASPD_MASK_SHARED && mode == ASPD_MODE_BRANCH;
   const bool mma_ok = shape->dtype == ASPD_DTYPE_BF16 && d == 128 && ps == 16;
@@ -637,7 +637,10 @@ static int plan_create_impl(const aspd_shape_t* shape, const aspd_request_t* req
     p->fuse_append = (most <= 20 && !shared_mask && tok_field_fits && p->wide != 2) ? 1 : 0;
   }
   // the merge of a token's records inside the attention kernel: stream-K plans of the tensor-core kernel
-  p->m64 = (kernel == ASPD_KERNEL_MMA && !deal_streams && tune.mma_m == 64) ? 1 : 0;
+  // 1: both MMAs with M = 64; 2: only P.V (the default: at most 64 of P.V's 128 rows are ever read, a quarter
+  // less tensor work lifts the power-capped clock and the softmax layout, which M = 64 scores would slow
+  // down, stays as it is); 0: both with M = 128
+  p->m64 = (kernel == ASPD_KERNEL_MMA && !deal_streams) ? (tune.mma_m == 64 ? 1 : tune.mma_m == 128 ? 0 : 2) : 0;
   p->stagger_start = (!deal_streams && total_pages <= 6L * 8 * n_ctas) ? 1 : 0;       // at most six 128-key tiles per CTA
   // Merging inside the attention kernel is an option, not the default.  Measured on every workload of
   // the benchmark, the CTA that stores a pair's last record is a CTA at the very end of its own work,
@@ -832,7 +835,7 @@ int aspd_plan_info(const aspd_plan_t* p, aspd_plan_info_t* info) {
   info->chunk_tokens = p->chunk_tokens; info->n_ctas = p->n_ctas; info->fused_append = (p->kernel == ASPD_KERNEL_MMA && p->fuse_append) ? 1 : 0;
   info->direct_output = attn_mma_direct(p) ? 1 : 0; info->max_rows_per_item = p->wide ? p->wide * kMaxRowsWide : kMaxRowsPerItem;
   info->dealt = p->dealt; info->single_launch = p->single_launch;
-  info->mma_m = p->kernel == ASPD_KERNEL_MMA ? (p->m64 ? 64 : 128) : 0; info->reserved = 0;
+  info->mma_m = p->kernel == ASPD_KERNEL_MMA ? (p->m64 == 1 ? 64 : p->m64 == 2 ? 96 : 128) : 0; info->reserved = 0;
   info->workspace_bytes = (int64_t)p->device_bytes;
   info->kv_tokens_read = p->kv_tokens_read; info->algorithmic_bytes = p->algorithmic_bytes;
   return ASPD_OK;

@@ -464,7 +464,7 @@ def test_position_id_variants(rule, fused):
     assert np.abs(plain.outputs[-1] - ref.outputs[-1]).max() > 1e-3     # the variant really differs from Eq. 4
 
 
-@pytest.mark.parametrize("mma_m", [64, 128])
+@pytest.mark.parametrize("mma_m", [64, 96, 128])
 def test_mma_m_variants_on_the_decode_shapes(mma_m):
     """The tensor-core kernel's stream-K path with M = 128 MMAs (rows replicated to fill the
     accumulator) and with M = 64 (half the tensor work, accumulators in 16 lanes of each quadrant,
@@ -497,6 +497,32 @@ def test_mma_m_variants_on_the_decode_shapes(mma_m):
     ref = oracle_run(peaked)
     run = E.run_workload(peaked, mma_m=mma_m)
     check(run.outputs[0], ref.outputs[0], "bf16", "peaked", tol=PEAKED_TOL[B.KERNEL_AUTO])
+    # logits x 16: along a key stream exponents pass 2^40 against the reference of the item's first
+    # tile, so tiles are redone the long way and O is rescaled in tensor memory (in the layout of this
+    # variant's P.V).  The softmax is close to an argmax and bf16 keys decide between near-equal
+    # candidates differently from the oracle's exact ones for some rows: only gross errors are excluded.
+    peaked.sm_scale *= 4.0
+    for wl16 in (peaked, W.config_long_rag(prefix=4096 + 5)):
+        if wl16 is not peaked:
+            wl16.sm_scale *= 16.0
+        ref = oracle_run(wl16)
+        run = E.run_workload(wl16, mma_m=mma_m)
+        g_, r_ = run.outputs[0].astype(np.float64), ref.outputs[0]
+        err = np.abs(g_ - r_)
+        assert np.isfinite(g_).all() and err.mean() <= 3e-2, (wl16.name, err.mean())
+        assert (err.reshape(err.shape[0], -1).max(axis=1) <= 0.1).mean() >= 0.7, wl16.name
+    # A jump built into the keys: from slot 1000 on every key has 96 in the slowest rotary pair's first
+    # element and every query 4 (both exact in bf16, hardly rotated), i.e. logits 49 powers of two
+    # above the earlier ones.  With two CTAs an item has many tiles, the jump falls into a later tile of
+    # one: its sum passes 2^40, the tile is redone the long way, the reference raised and O rescaled.
+    jump = W.config_long_rag(prefix=2048 + 5)
+    for ph in jump.phases:
+        if ph.label == "fill-prefix":
+            ph.k_new[1000:, :, 63] = 96.0
+        if ph.q is not None:
+            ph.q[:, :, 63] = 4.0
+    compare_workload(jump, mma_m=mma_m, n_ctas=2)
+    compare_workload(jump, mma_m=mma_m, n_ctas=2, fused=True)
     # open step of config 3: 72 query tokens in row blocks of 9 (63 rows), several blocks per request
     compare_workload(W.config_branch_open(serial_steps=2), mma_m=mma_m)
 
