@@ -368,8 +368,9 @@ def per_config_entry(res, peak, flops=None, tensor_peak=None):
 
 
 def run_rerotate(args):
-    """--op rerotate: the Same-Re renumbering of a finished segment, aspd_k_rerotate over every
-    branch token of the workload, one launch per layer.  One GPU; prints its own JSON line."""
+    """--op rerotate: the Same-Re renumbering of a finished segment, the keys of every branch token
+    of the workload re-rotated in all layers' pools (one launch for all layers; --rerotate-per-layer
+    and --rerotate-by-token: one call per layer).  One GPU; prints its own JSON line."""
     print(json.dumps(measure_rerotate(args)))
     return 0
 
@@ -405,7 +406,13 @@ def measure_rerotate(args):
     caches = [E.LayerCache(shape, wl.n_pool_pages) for _ in range(L)]
     fill_caches(wl, shape, caches)
 
+    per_layer = by_token or bool(getattr(args, "rerotate_per_layer", False))
+    launches = 1 if by_token else (len(ranges) + 511) // 512
+    launches *= L if per_layer else (L + 63) // 64
+
     def step():
+        if not per_layer:                  # every layer's pool in one launch (64 pools per launch)
+            return B.k_rerotate_ranges_layers(shape, [c.k for c in caches], table_d, ranges)
         for c in caches:
             if by_token:
                 B.k_rerotate(shape, c.k, pages, rows, delta)
@@ -437,11 +444,13 @@ def measure_rerotate(args):
         "unit": "tokens/s", "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
         "higher_is_better": True, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": args.workload, "layers": L, "tokens_per_layer": n, "heads": wl.Hkv, "head_dim": wl.d,
-                   "l2": "%.1f GB of distinct keys per step" % (alg * L / 1e9)},
+                   "call": "aspd_k_rerotate" if by_token else "aspd_k_rerotate_ranges" if per_layer else "aspd_k_rerotate_ranges_layers",
+                   "launches_per_step": launches, "l2": "%.1f GB of distinct keys per step" % (alg * L / 1e9)},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": None, "peak_kind": "of " + peak_kind, "kernel": "rerotate_kernel" if by_token else "rerotate_ranges_kernel",
-                     "kernel_us": ms / args.steps / L * 1e3, "algorithmic_bytes_per_launch": alg},
-        "gpu_launches": L * args.steps * (1 if by_token else (len(ranges) + 511) // 512), "clocks": clocks})
+                     "kernel_us": ms / args.steps / L * 1e3, "algorithmic_bytes_per_launch": alg * L // launches,
+                     "algorithmic_bytes_per_layer": alg},
+        "gpu_launches": launches * args.steps, "clocks": clocks})
 
 
 def run_serial_chain(args):
@@ -916,7 +925,8 @@ def per_config_block(args, peak):
     torch.cuda.empty_cache()
     sub.workload, sub.requests = "serving-mix", 0
     rr = measure_rerotate(sub)
-    out["rerotate"] = {"kernel_us": rr["roofline"]["kernel_us"], "alg_bytes": rr["roofline"]["algorithmic_bytes_per_launch"],
+    out["rerotate"] = {"kernel_us": rr["roofline"]["kernel_us"], "alg_bytes": rr["roofline"]["algorithmic_bytes_per_layer"],
+                       "call": rr["config"]["call"], "launches": rr["config"]["launches_per_step"],
                        "frac": rr["roofline"]["frac"], "bound": "hbm", "tokens_per_layer": rr["config"]["tokens_per_layer"],
                        "layers": rr["config"]["layers"], "sm_mhz": (rr["clocks"] or {}).get("sm_mhz")}
     torch.cuda.empty_cache()
@@ -955,6 +965,8 @@ def main():
                     help="decode-loop: capture the step once and re-plan in place every step (aspd_plan_update) instead of "
                          "making a new plan and launching from the host")
     ap.add_argument("--rerotate-by-token", action="store_true", help="rerotate: per-token index arrays (aspd_k_rerotate) instead of ranges")
+    ap.add_argument("--rerotate-per-layer", action="store_true",
+                    help="rerotate: one aspd_k_rerotate_ranges call per layer instead of all layers in one launch")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -446,6 +446,17 @@ int aspd_k_rerotate_ranges(const aspd_shape_t* shape, void* k_pool /*device*/, c
                            const int32_t* ranges /*host*/, int n_ranges, void* stream);
 
 /*
+ * The same for the K pools of several layers in one launch (a finished segment is renumbered in
+ * every layer of the model at once; the layers share the page tables, so the same slots move in
+ * each).  k_pools: HOST array of n_layers device pointers, read before the call returns; 64 pools
+ * per launch.  Pools must not overlap.  Same results, bit for bit, as n_layers calls of
+ * aspd_k_rerotate_ranges; one launch of n_layers times the blocks instead of n_layers short ones.
+ */
+int aspd_k_rerotate_ranges_layers(const aspd_shape_t* shape, void* const* k_pools /*host array of device pointers*/,
+                                  int n_layers, const int32_t* page_table /*device*/,
+                                  const int32_t* ranges /*host*/, int n_ranges, void* stream);
+
+/*
  * Failure-path check: runs the library's bounded device-side wait on a barrier nobody ever
  * arrives on, with a limit of `limit_cycles` SM clock cycles (at most 4e9).  The kernel gives up
  * when the limit passes and reports ASPD_ERR_TIMEOUT through *status_out (host); the context

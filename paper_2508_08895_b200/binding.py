@@ -65,7 +65,7 @@ EXPORTS = ("aspd_strerror", "aspd_pool_bytes", "aspd_count_new_tokens", "aspd_po
            "aspd_visible_slots_masked", "aspd_plan_create", "aspd_plan_update", "aspd_plan_destroy", "aspd_release_cached_memory", "aspd_plan_info", "aspd_plan_items", "aspd_plan_cta_ranges", "aspd_plan_stream_pages",
            "aspd_plan_token_ranges", "aspd_plan_shared_mask_tables", "aspd_plan_status",
            "aspd_kv_append", "aspd_branch_attn", "aspd_serial_attn", "aspd_attn_partials", "aspd_attn_combine", "aspd_step_partials",
-           "aspd_branch_step", "aspd_serial_step", "aspd_step_host", "aspd_step_host_async", "aspd_attn_static", "aspd_static_status", "aspd_k_rerotate", "aspd_k_rerotate_ranges", "aspd_debug_read_token", "aspd_debug_bounded_wait", "aspd_debug_profile", "aspd_debug_pool_limit")
+           "aspd_branch_step", "aspd_serial_step", "aspd_step_host", "aspd_step_host_async", "aspd_attn_static", "aspd_static_status", "aspd_k_rerotate", "aspd_k_rerotate_ranges", "aspd_k_rerotate_ranges_layers", "aspd_debug_read_token", "aspd_debug_bounded_wait", "aspd_debug_profile", "aspd_debug_pool_limit")
 
 _lib = None
 
@@ -116,6 +116,7 @@ def lib() -> ctypes.CDLL:
         L.aspd_static_status.argtypes = [vp]
         L.aspd_k_rerotate.argtypes = [vp, vp, vp, vp, vp, ci, vp]
         L.aspd_k_rerotate_ranges.argtypes = [vp, vp, vp, vp, ci, vp]
+        L.aspd_k_rerotate_ranges_layers.argtypes = [vp, vp, ci, vp, vp, ci, vp]
         L.aspd_debug_bounded_wait.argtypes = [ctypes.c_int64, vp, vp]
         L.aspd_debug_profile.argtypes = [vp, ci]
         L.aspd_debug_pool_limit.argtypes = [vp, ctypes.c_int64]
@@ -347,6 +348,14 @@ def k_rerotate_ranges(shape: Shape, k_pool, page_table, ranges, stream=None) -> 
     ranges = np.ascontiguousarray(ranges, dtype=np.int32).reshape(-1, 4)
     _check(lib().aspd_k_rerotate_ranges(ctypes.addressof(shape), _ptr(k_pool), _ptr(page_table), _ptr(ranges), len(ranges),
                                         _stream(stream)), "aspd_k_rerotate_ranges")
+
+
+def k_rerotate_ranges_layers(shape: Shape, k_pools, page_table, ranges, stream=None) -> None:
+    """The same for the K pools of several layers (a sequence of device tensors) in one launch."""
+    ranges = np.ascontiguousarray(ranges, dtype=np.int32).reshape(-1, 4)
+    ptrs = (ctypes.c_void_p * len(k_pools))(*[_ptr(k) for k in k_pools])
+    _check(lib().aspd_k_rerotate_ranges_layers(ctypes.addressof(shape), ptrs, len(k_pools), _ptr(page_table), _ptr(ranges),
+                                               len(ranges), _stream(stream)), "aspd_k_rerotate_ranges_layers")
 
 
 def debug_bounded_wait(limit_cycles: int, stream=None) -> int:

@@ -182,8 +182,8 @@ int launch_attn_mma_step(const aspd_plan* p, const void* q, const void* k_new, c
                          void* v_pool, void* out, cudaStream_t s);
 int launch_rerotate(const aspd_shape_t* shape, void* k_pool, const int32_t* pages, const int32_t* rows, const int32_t* delta,
                     int n, cudaStream_t s);
-int launch_rerotate_ranges(const aspd_shape_t* shape, void* k_pool, const int32_t* page_table, const int32_t* ranges, int n_ranges,
-                           cudaStream_t s);
+int launch_rerotate_ranges(const aspd_shape_t* shape, void* const* k_pools, int n_layers, const int32_t* page_table,
+                           const int32_t* ranges, int n_ranges, cudaStream_t s);
 int set_profile_buffer(long long* device_buf, int cta);
 int launch_wait_probe(long long limit_cycles, int32_t* status_dev, cudaStream_t s);
 int launch_read_token(const aspd_shape_t* shape, const void* pool, int64_t page, int row, int kv_head,

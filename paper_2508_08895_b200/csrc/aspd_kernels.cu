@@ -173,10 +173,15 @@ struct RerotateRanges {
   int unit0[kMaxRanges + 1];            // first page unit of range i (prefix sum of the pages each range touches)
   int4 r[kMaxRanges];                   // (page-table base, first slot, count, delta)
 };
+constexpr int kMaxLayerPools = 64;      // K pools (layers) per launch: grid.y, their addresses in the launch parameters
+struct PoolList {
+  void* p[kMaxLayerPools];
+};
 template <typename T>
 __global__ void __launch_bounds__(512)
-rerotate_ranges_kernel(T* __restrict__ k_pool, const int32_t* __restrict__ page_table, const RerotateRanges rr, const InvFreq table,
+rerotate_ranges_kernel(const PoolList pools, const int32_t* __restrict__ page_table, const RerotateRanges rr, const InvFreq table,
                        int n_kv_heads, int head_dim, int page_size) {
+  T* __restrict__ k_pool = static_cast<T*>(pools.p[blockIdx.y]);   // the layers share the page tables, so the same pages move in each
   constexpr int VEC = 16 / sizeof(T);
   __shared__ float2 cs_sm[64];          // (cos, sin) of the range's delta for every element pair: the same for all tokens of the page
   pdl_launch_dependents();
@@ -435,16 +440,16 @@ int launch_rerotate(const aspd_shape_t* sh, void* k_pool, const int32_t* pages, 
                               table, n, sh->n_kv_heads, sh->head_dim, sh->page_size));
 }
 
-int launch_rerotate_ranges(const aspd_shape_t* sh, void* k_pool, const int32_t* page_table, const int32_t* ranges, int n_ranges,
-                           cudaStream_t s) {
+int launch_rerotate_ranges(const aspd_shape_t* sh, void* const* k_pools, int n_layers, const int32_t* page_table,
+                           const int32_t* ranges, int n_ranges, cudaStream_t s) {
   const int chunks = sh->head_dim / 2 / (16 / esize_of(sh->dtype)), ps = sh->page_size;
   InvFreq table;
   for (int i = 0; i < sh->head_dim / 2; ++i) table.f[i] = pow((double)sh->rope_theta, -2.0 * i / (double)sh->head_dim);
-  for (int r0 = 0; r0 < n_ranges; r0 += kMaxRanges) {
+  for (int r0 = 0; r0 < n_ranges;) {
     RerotateRanges rr;
     rr.n = 0; rr.unit0[0] = 0;
-    for (int i = r0; i < n_ranges && rr.n < kMaxRanges; ++i) {
-      const int32_t* g = ranges + 4 * (size_t)i;
+    for (; r0 < n_ranges && rr.n < kMaxRanges; ++r0) {
+      const int32_t* g = ranges + 4 * (size_t)r0;
       if (g[2] <= 0) continue;                                   // an empty range moves nothing
       const int pages = (g[1] + g[2] - 1) / ps - g[1] / ps + 1;
       rr.r[rr.n] = make_int4(g[0], g[1], g[2], g[3]);
@@ -452,15 +457,20 @@ int launch_rerotate_ranges(const aspd_shape_t* sh, void* k_pool, const int32_t* 
       ++rr.n;
     }
     if (rr.n == 0) continue;
-    const dim3 grid((unsigned)rr.unit0[rr.n]), block((unsigned)(ps * chunks));
-    cudaError_t e;
-    if (sh->dtype == ASPD_DTYPE_BF16)
-      e = launch_pdl(kPdlAppend, rerotate_ranges_kernel<__nv_bfloat16>, grid, block, 0, s, (__nv_bfloat16*)k_pool, page_table, rr, table,
-                     sh->n_kv_heads, sh->head_dim, ps);
-    else
-      e = launch_pdl(kPdlAppend, rerotate_ranges_kernel<float>, grid, block, 0, s, (float*)k_pool, page_table, rr, table, sh->n_kv_heads,
-                     sh->head_dim, ps);
-    if (e != cudaSuccess) return ASPD_ERR_CUDA;
+    for (int l0 = 0; l0 < n_layers; l0 += kMaxLayerPools) {
+      PoolList pools;
+      const int nl = std::min(kMaxLayerPools, n_layers - l0);
+      for (int l = 0; l < kMaxLayerPools; ++l) pools.p[l] = k_pools[l0 + std::min(l, nl - 1)];
+      const dim3 grid((unsigned)rr.unit0[rr.n], (unsigned)nl), block((unsigned)(ps * chunks));
+      cudaError_t e;
+      if (sh->dtype == ASPD_DTYPE_BF16)
+        e = launch_pdl(kPdlAppend, rerotate_ranges_kernel<__nv_bfloat16>, grid, block, 0, s, pools, page_table, rr, table, sh->n_kv_heads,
+                       sh->head_dim, ps);
+      else
+        e = launch_pdl(kPdlAppend, rerotate_ranges_kernel<float>, grid, block, 0, s, pools, page_table, rr, table, sh->n_kv_heads,
+                       sh->head_dim, ps);
+      if (e != cudaSuccess) return ASPD_ERR_CUDA;
+    }
   }
   return ASPD_OK;
 }

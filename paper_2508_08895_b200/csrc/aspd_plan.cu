@@ -1037,18 +1037,30 @@ int aspd_k_rerotate(const aspd_shape_t* shape, void* k_pool, const int32_t* page
   return launch_rerotate(shape, k_pool, pages, rows, delta, n, (cudaStream_t)stream);
 }
 
-int aspd_k_rerotate_ranges(const aspd_shape_t* shape, void* k_pool, const int32_t* page_table, const int32_t* ranges, int n_ranges,
-                           void* stream) {
-  int rc = check_shape(shape);
-  if (rc) return rc;
-  if (n_ranges < 0) return ASPD_ERR_INVALID_ARG;
-  if (n_ranges == 0) return ASPD_OK;
-  if (!k_pool || !page_table || !ranges || misaligned16(k_pool)) return ASPD_ERR_INVALID_ARG;
+static int check_ranges(const int32_t* ranges, int n_ranges) {
   for (int i = 0; i < n_ranges; ++i) {
     const int32_t* g = ranges + 4 * (size_t)i;
     if (g[0] < 0 || g[1] < 0 || g[2] < 0 || (long)g[1] + g[2] > INT32_MAX) return ASPD_ERR_BAD_DESCRIPTOR;
   }
-  return launch_rerotate_ranges(shape, k_pool, page_table, ranges, n_ranges, (cudaStream_t)stream);
+  return ASPD_OK;
+}
+
+int aspd_k_rerotate_ranges(const aspd_shape_t* shape, void* k_pool, const int32_t* page_table, const int32_t* ranges, int n_ranges,
+                           void* stream) {
+  return aspd_k_rerotate_ranges_layers(shape, &k_pool, 1, page_table, ranges, n_ranges, stream);
+}
+
+int aspd_k_rerotate_ranges_layers(const aspd_shape_t* shape, void* const* k_pools, int n_layers, const int32_t* page_table,
+                                  const int32_t* ranges, int n_ranges, void* stream) {
+  int rc = check_shape(shape);
+  if (rc) return rc;
+  if (n_ranges < 0 || n_layers < 0) return ASPD_ERR_INVALID_ARG;
+  if (n_ranges == 0 || n_layers == 0) return ASPD_OK;
+  if (!k_pools || !page_table || !ranges) return ASPD_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l)
+    if (!k_pools[l] || misaligned16(k_pools[l])) return ASPD_ERR_INVALID_ARG;
+  if ((rc = check_ranges(ranges, n_ranges))) return rc;
+  return launch_rerotate_ranges(shape, k_pools, n_layers, page_table, ranges, n_ranges, (cudaStream_t)stream);
 }
 
 int aspd_debug_pool_limit(aspd_plan_t* p, int64_t n_pages) {

@@ -748,10 +748,18 @@ def test_same_re_serial_decoding_after_rerotation():
             ranges.append((int(d["page_begin"][r]), int(d["br_kv_off"][b]), int(d["br_kv_len"][b]), moved))
             moved += int(d["br_kv_len"][b])
     check_k = run.cache.k.clone()
+    # three layers' pools (different contents, the same page tables) in one launch against one call each
+    layers = [run.cache.k.clone(), (run.cache.k.float() * 0.5).to(run.cache.k.dtype), run.cache.k.flip(0).contiguous()]
+    singles = [x.clone() for x in layers]
     B.k_rerotate(run.shape, check_k, t(pages), t(rows), t(delta))
     B.k_rerotate_ranges(run.shape, run.cache.k, t(d["page_ids"].tolist()), np.array(ranges, dtype=np.int32))
+    B.k_rerotate_ranges_layers(run.shape, layers, t(d["page_ids"].tolist()), np.array(ranges, dtype=np.int32))
+    for x in singles:
+        B.k_rerotate_ranges(run.shape, x, t(d["page_ids"].tolist()), np.array(ranges, dtype=np.int32))
+    B.k_rerotate_ranges_layers(run.shape, [], t(d["page_ids"].tolist()), np.array(ranges, dtype=np.int32))    # no layer: nothing
     torch.cuda.synchronize()
-    assert torch.equal(check_k, run.cache.k)
+    assert torch.equal(check_k, run.cache.k) and torch.equal(layers[0], check_k)
+    assert all(torch.equal(a, b) for a, b in zip(layers, singles)) and not torch.equal(layers[1], layers[0])
     for pg, r, dl in zip(pages, rows, delta):
         for h in range(wl.Hkv):
             ref.k_pool[pg, h, r] = oracle.rope(ref.k_pool[pg, h, r], float(dl), wl.theta)
