@@ -14,9 +14,11 @@
 //
 // so that while one group is in its exponentials the tensor pipe works for the other, and a thread
 // owns its row from the first score to the normalised output (it divides by l and stores the row
-// itself; there are no statistics to hand over).  Each group has an MMA warp with two cursors (S and P.V of the
-// group) and issues whichever has its operands ready.  Warp roles: 0-3 group 0, 4-7 group 1, 8 / 11
-// K / V producers, 9 / 10 MMA issuers of group 0 / 1, 12-15 query preparation.  Single buffers for S (by halves)
+// itself; there are no statistics to hand over).  Each of the four streams of MMAs (scores and P.V of
+// either group) has a warp of its own that takes its operations in order and waits for each one's
+// operands.  Warp roles: 0-3 group 0, 4-7 group 1, 8 / 11 K / V producers, 9 / 10 P.V issuers of group
+// 0 / 1, 12-15 query preparation, of which 12 / 13 also issue the scores of group 0 / 1 (an item's
+// query tiles are written and its scores issued at different times).  Single buffers for S (by halves)
 // and the query tiles; K and V tiles double-buffered.  All waits are bounded as in the other variants.
 #pragma once
 
@@ -48,7 +50,7 @@ struct MiscW2 {
   DeviceItem items[kItemCacheW2];
   uint32_t tmem_base;
   int abort_flag;
-  int lead[2];                       // items group 0's MMA warp has finished issuing: scores / P.V (read by group 1's)
+  int lead[2];                       // [1]: the item group 0's P.V issuer is at (read by group 1's); [0] unused
 };
 static_assert(sizeof(MiscW2) <= 2048, "MiscW2 must fit behind the tiles");
 
@@ -333,122 +335,85 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_w2_kernel(Ctx c) {
       }
     }
   } else if (warp == W_MMA || warp == W_MMA + 1) {
-    // =================================== MMA issuers ===================================
-    // One warp per group (warps 9 and 10), each with two cursors -- the group's score MMAs and its
-    // P.V MMAs -- that walk the CTA's tiles independently; the warp polls them in turn and issues
-    // whichever has its operands ready (the barriers carry the real dependencies).  All lanes run the
-    // same control flow on the same values (what a barrier says is taken from lane 0); lane 0 issues.
+    // ================================ P.V issuers (warp 9: group 0, warp 10: group 1) ================================
+    // One warp per stream of operations, each with one cursor and a suspending wait for every
+    // operand (all lanes wait, so the warp never diverges; lane 0 issues).  A warp that polled two
+    // cursors (scores and P.V of its group) spent ~1300 cycles per operation on asking, issuing and
+    // committing, beside two softmax warps on its scheduler, and was what bounded the tile period.
     const int grp = warp - W_MMA;
     const uint32_t fm = 0xffffffffu;
     const uint32_t tmem_u = __shfl_sync(fm, tmem, 0), base_u = __shfl_sync(fm, base, 0), bars_u = base_u + W2_OFF_MISC;
     const int ib = __shfl_sync(fm, item_begin, 0), ie = __shfl_sync(fm, item_end, 0);
-    struct Cur { int idx, t, h, n_pages, n_tiles, gbase, count, count1, both; bool done; };   // count1: second halves (score cursor)
-    auto seek = [&](Cur& u) {                      // the next item in which the group has rows
-      while (u.idx < ie) {
-        const DeviceItem it = get_item_w2(c, misc, u.idx, ib);
-        const int n_pages = __shfl_sync(fm, it.n_pages, 0), n_q_tok = __shfl_sync(fm, it.n_q_tok, 0);
-        if (n_q_tok > grp * tpt) { u.n_pages = n_pages; u.n_tiles = (n_pages + 7) >> 3; u.both = n_q_tok > tpt; u.t = 0; u.h = 0; return; }
-        u.gbase += (n_pages + 7) >> 3;
-        ++u.idx;
-      }
-      u.done = true;
-    };
-    auto ready = [&](uint32_t bar, uint32_t parity) { return __shfl_sync(fm, mbar_test(bar, parity) ? 1 : 0, 0) != 0; };   // polled: never suspends
-    auto arrive0 = [&](uint32_t bar) { if (lane == 0) mbar_arrive(bar); };
+    auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(fm, mbar_wait(bar, parity, ab)) != 0; };
     // A parity only tells the two latest phases of a barrier apart.  Group 1 is absent from items with
-    // a single query tile, so its cursors may sit at an item that group 0 has not reached yet and
-    // would then take an older phase of a shared barrier (K, V, Q) for theirs: they hold until group
-    // 0's cursor of the same kind has reached their item (group 0's warp publishes how far it is).
+    // a single query tile, so its cursor may come to an item that group 0 has not reached yet and
+    // would then take an older phase of a V barrier for its own: it holds until group 0's cursor
+    // has reached the item (group 0's warp publishes how far it is).
     volatile int* lead = misc->lead;
-    auto reached = [&](int which, int idx) { return grp == 0 || __shfl_sync(fm, lead[which], 0) >= idx; };
-    Cur cs = {ib, 0, 0, 0, 0, 0, 0, 0, 0, false}, cp = cs;
-    seek(cs); seek(cp);
     const uint32_t idesc_pv = instr_desc(128, 1);
-    long long last_progress = clock64();
-    while (!(cs.done && cp.done)) {
-      bool progressed = false;
-      // ---- O_grp += P_grp . V for half h of tile t
-      if (!cp.done && reached(1, cp.idx)) {
-        Cur& u = cp;
-        const int g = u.gbase + u.t, npg = min(8, u.n_pages - u.t * 8), halves = npg > 4 ? 2 : 1;
-        if (ready(bars_u + 8 * (WP_FULL + grp), u.count & 1) && ready(bars_u + 8 * (WV_FULL + (g & 1)), (g >> 1) & 1)) {
-          tc_fence_after();
-          const uint32_t pbuf = base_u + W2_OFF_P + grp * kPHalfBytes, vbuf = base_u + W2_OFF_V + (g & 1) * kTileBytes;
-          const int n = min(4, npg - 4 * u.h);
+    const uint32_t o_tmem = tmem_u + COL_O + grp * 128, p_tmem = tmem_u + COL_S + grp * 128;
+    int gbase = 0, count = 0;
+    bool ok = true;
+    for (int idx = ib; idx < ie && ok; ++idx) {
+      const DeviceItem it = get_item_w2(c, misc, idx, ib);
+      const int n_pages = __shfl_sync(fm, it.n_pages, 0), n_q_tok = __shfl_sync(fm, it.n_q_tok, 0), n_tiles = (n_pages + 7) >> 3;
+      if (n_q_tok > grp * tpt) {
+        const bool both = n_q_tok > tpt;
+        if (grp == 1) {
+          const long long t0 = clock64();
+          while (ok && __shfl_sync(fm, lead[1], 0) < idx) {
+            __nanosleep(100);
+            if (__shfl_sync(fm, (*ab || clock64() - t0 > kWaitCycles) ? 1 : 0, 0)) { *ab = 1; ok = false; }
+          }
+        }
+        for (int t = 0; t < n_tiles && ok; ++t) {
+          const int g = gbase + t, npg = min(8, n_pages - t * 8), halves = npg > 4 ? 2 : 1;
+          const uint32_t vbuf = base_u + W2_OFF_V + (g & 1) * kTileBytes;
+          for (int h = 0; h < halves && ok; ++h, ++count) {
+            ok = wait_all(bars_u + 8 * (WP_FULL + grp), count & 1) && (h > 0 || wait_all(bars_u + 8 * (WV_FULL + (g & 1)), (g >> 1) & 1));
+            if (!ok) break;
+            tc_fence_after();
+            if (lane == 0 && grp == 0 && h == 0) ASPD_STAMP(c, g, 15);
+            if constexpr (kPInTmem) {        // 16 keys = one page per k-step
+              tc_mma_ts_pv_lane0(o_tmem, p_tmem + h * 64, smem_desc(vbuf + 4 * h * 4096, 1024, 2048), idesc_pv, (t > 0 || h > 0) ? 1u : 0u,
+                                 min(4, npg - 4 * h));
+            } else {
+              const uint32_t pbuf = base_u + W2_OFF_P + grp * kPHalfBytes;
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks) {
-            if (ks < n) {
-              const uint64_t b = smem_desc(vbuf + (4 * u.h + ks) * 4096, 1024, 2048);   // 16 keys = one page per k-step
-              const uint32_t acc = (u.t > 0 || u.h > 0 || ks > 0) ? 1u : 0u;
-              if constexpr (kPInTmem) {
-                tc_mma_ts_lane0(tmem_u + COL_O + grp * 128, tmem_u + COL_S + grp * 128 + u.h * 64 + ks * 8, b, idesc_pv, acc);
-              } else {
-                const uint64_t a = smem_desc(pbuf + ks * 32, 16, 1024);
-                tc_mma_lane0(tmem_u + COL_O + grp * 128, a, b, idesc_pv, acc);
-              }
+              for (int ks = 0; ks < 4; ++ks)
+                if (ks < npg - 4 * h)
+                  tc_mma_lane0(o_tmem, smem_desc(pbuf + ks * 32, 16, 1024), smem_desc(vbuf + (4 * h + ks) * 4096, 1024, 2048), idesc_pv,
+                               (t > 0 || h > 0 || ks > 0) ? 1u : 0u);
+            }
+            tc_commit_lane0(bars_u + 8 * (WP_EMPTY + grp));
+            if constexpr (kPInTmem) tc_commit_lane0(bars_u + 8 * (WS_EMPTY + 2 * grp + h));   // the half's columns are free for the next scores
+            if (lane == 0 && grp == 0) ASPD_STAMP(c, g, 10 + h);
+            if (h == halves - 1) {
+              tc_commit_lane0(bars_u + 8 * (WV_EMPTY + (g & 1)));
+              if (!both && lane == 0) mbar_arrive(bars_u + 8 * (WV_EMPTY + (g & 1)));       // the absent group's share
+              if (t == n_tiles - 1) tc_commit_lane0(bars_u + 8 * (WO_FULL + grp));
             }
           }
-          tc_commit_lane0(bars_u + 8 * (WP_EMPTY + grp));
-          if constexpr (kPInTmem) tc_commit_lane0(bars_u + 8 * (WS_EMPTY + 2 * grp + u.h));   // the half's columns are free for the next scores
-          if (lane == 0 && grp == 0) ASPD_STAMP(c, g, 10 + u.h);
-          const bool last_half = u.h == halves - 1;
-          if (last_half) {
-            tc_commit_lane0(bars_u + 8 * (WV_EMPTY + (g & 1)));
-            if (!u.both) arrive0(bars_u + 8 * (WV_EMPTY + (g & 1)));       // the absent group's share
-            if (u.t == u.n_tiles - 1) tc_commit_lane0(bars_u + 8 * (WO_FULL + grp));
-          }
-          ++u.count;
-          if (!last_half) ++u.h;
-          else {
-            u.h = 0;
-            if (++u.t == u.n_tiles) { u.gbase += u.n_tiles; ++u.idx; seek(u); if (grp == 0 && lane == 0) lead[1] = u.done ? ie : u.idx; }
-          }
-          progressed = true;
         }
+        if (grp == 0 && lane == 0) lead[1] = idx + 1;
       }
-      // ---- S_grp = Q_grp . K^T for half h of tile t (keys 64 h ... of the tile)
-      if (!cs.done && reached(0, cs.idx)) {
-        Cur& v = cs;
-        const int g = v.gbase + v.t, sb = g & 1, npg = min(8, v.n_pages - v.t * 8), halves = (kSplitS && npg > 4) ? 2 : 1, item_no = v.idx - ib;
-        const int cnt = v.h ? v.count1 : v.count;
-        if ((v.t > 0 || v.h > 0 || ready(bars_u + 8 * WQ_FULL, item_no & 1)) && ready(bars_u + 8 * (WK_FULL + sb), (g >> 1) & 1) &&
-            ready(bars_u + 8 * (WS_EMPTY + 2 * grp + v.h), (cnt & 1) ^ 1)) {
-          tc_fence_after();
-          const uint32_t qbuf = base_u + W2_OFF_Q + grp * kTileBytes, kbuf = base_u + W2_OFF_K + sb * kTileBytes + v.h * 16384;
-          const uint32_t idesc_s = instr_desc((uint32_t)(kSplitS ? min(4, npg - 4 * v.h) : npg) * 16u, 0);
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            const uint64_t a = smem_desc(qbuf + (ks >> 2) * kHalf + (ks & 3) * 32, 16, 1024);
-            const uint64_t b = smem_desc(kbuf + (ks >> 2) * 1024 + (ks & 3) * 32, 16, 2048);
-            tc_mma_lane0(tmem_u + COL_S + grp * 128 + v.h * 64, a, b, idesc_s, ks > 0 ? 1u : 0u);
-          }
-          tc_commit_lane0(bars_u + 8 * (WS_FULL + 2 * grp + v.h));
-          if (lane == 0 && grp == 0) ASPD_STAMP(c, g, 8 + v.h);
-          if (v.h) ++v.count1; else ++v.count;
-          if (v.h == halves - 1) {
-            tc_commit_lane0(bars_u + 8 * (WK_EMPTY + sb));
-            if (!v.both) arrive0(bars_u + 8 * (WK_EMPTY + sb));
-            if (v.t == v.n_tiles - 1) {
-              tc_commit_lane0(bars_u + 8 * WQ_EMPTY);
-              if (!v.both) arrive0(bars_u + 8 * WQ_EMPTY);
-            }
-            v.h = 0;
-            if (++v.t == v.n_tiles) { v.gbase += v.n_tiles; ++v.idx; seek(v); if (grp == 0 && lane == 0) lead[0] = v.done ? ie : v.idx; }
-          } else {
-            ++v.h;
-          }
-          progressed = true;
-        }
-      }
-      if (progressed) last_progress = clock64();
-      else if (*ab || clock64() - last_progress > kWaitCycles) { *ab = 1; break; }
+      gbase += n_tiles;
     }
+    if (grp == 0 && lane == 0) lead[1] = ie;
     __syncwarp();
   } else if (warp >= W_EPI) {
-    // ================================ query preparation ================================
-    const int et = tid - W_EPI * 32;
+    // ================== query preparation (warps 12-15) and score issuers (warp 12: group 0, warp 13: group 1) ==================
+    // The query tiles of an item can be written only when the last scores of the previous item have
+    // been issued, and the first scores of an item need its query tiles: the two never overlap, so
+    // two of the preparation warps issue the score MMAs between their preparations (one cursor each,
+    // suspending waits, the tiles of an item in order).
+    const int et = tid - W_EPI * 32, grp = warp - W_EPI;       // grp is a group only for warps 12 and 13
+    const uint32_t fm = 0xffffffffu;
+    const uint32_t tmem_u = __shfl_sync(fm, tmem, 0), base_u = __shfl_sync(fm, base, 0), bars_u = base_u + W2_OFF_MISC;
+    auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(fm, mbar_wait(bar, parity, ab)) != 0; };
+    const uint64_t adesc_q = smem_desc(base_u + W2_OFF_Q + (grp & 1) * kTileBytes, 16, 1024);
     bool dead = false;
-    int item_no = 0;
+    int item_no = 0, gbase = 0, cnt[2] = {0, 0};
     for (int idx = item_begin; idx < item_end; ++idx, ++item_no) {
       const DeviceItem it = get_item_w2(c, misc, idx, item_begin);
       bool waited_q = false;
@@ -471,6 +436,37 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_w2_kernel(Ctx c) {
       fence_async_smem();
       mbar_arrive(bars + 8 * WQ_FULL);
       if (named_sync_or(3, 128, dead || *ab)) break;
+      // ---- S_grp = Q_grp . K^T for the halves of the item's tiles (keys 64 h ... of a tile)
+      const int n_pages = __shfl_sync(fm, it.n_pages, 0), n_q_tok = __shfl_sync(fm, it.n_q_tok, 0), n_tiles = (n_pages + 7) >> 3;
+      if (grp < 2 && n_q_tok > grp * tpt) {
+        const bool both = n_q_tok > tpt;
+        bool ok = wait_all(bars_u + 8 * WQ_FULL, item_no & 1);
+        for (int t = 0; t < n_tiles && ok; ++t) {
+          const int g = gbase + t, sb = g & 1, npg = min(8, n_pages - t * 8), halves = (kSplitS && npg > 4) ? 2 : 1;
+          for (int h = 0; h < halves && ok; ++h) {
+            ok = (h > 0 || wait_all(bars_u + 8 * (WK_FULL + sb), (g >> 1) & 1)) && wait_all(bars_u + 8 * (WS_EMPTY + 2 * grp + h), (cnt[h] & 1) ^ 1);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t kbuf = base_u + W2_OFF_K + sb * kTileBytes + h * 16384;
+            const uint32_t idesc_s = instr_desc((uint32_t)(kSplitS ? min(4, npg - 4 * h) : npg) * 16u, 0);
+            if (lane == 0 && grp == 0 && h == 0) ASPD_STAMP(c, g, 12);
+            tc_mma_ss_k128_lane0<kHalf, 1024>(tmem_u + COL_S + grp * 128 + h * 64, adesc_q, smem_desc(kbuf, 16, 2048), idesc_s);
+            tc_commit_lane0(bars_u + 8 * (WS_FULL + 2 * grp + h));
+            if (lane == 0 && grp == 0) ASPD_STAMP(c, g, 8 + h);
+            ++cnt[h];
+            if (h == halves - 1) {
+              tc_commit_lane0(bars_u + 8 * (WK_EMPTY + sb));
+              if (!both && lane == 0) mbar_arrive(bars_u + 8 * (WK_EMPTY + sb));       // the absent group's share
+              if (t == n_tiles - 1) {
+                tc_commit_lane0(bars_u + 8 * WQ_EMPTY);
+                if (!both && lane == 0) mbar_arrive(bars_u + 8 * WQ_EMPTY);
+              }
+            }
+          }
+        }
+        dead |= !ok;
+      }
+      gbase += n_tiles;
     }
   }
 

@@ -96,6 +96,60 @@ __device__ __forceinline__ void tc_mma_ts_lane0(uint32_t d_tmem, uint32_t a_tmem
       "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
       ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
 }
+// Whole operations in one statement each, so that the issuing warp spends a handful of instructions
+// per MMA (it shares its scheduler with softmax warps; descriptor arithmetic per MMA made an
+// operation of 8 take ~600 cycles to issue).  A descriptor's low bits are the address / 16, so the
+// k-steps are additions to the first descriptor.
+//
+// Eight k-steps of a 128 x N x 128 product with both operands in shared memory (K-major, 128-byte
+// swizzle): k-step ks reads A at +32 (ks % 4) bytes in half ks / 4 (a_half bytes apart), B likewise
+// with halves b_half bytes apart.  Lane 0 issues; the first k-step overwrites the accumulator.
+template <uint32_t A_HALF, uint32_t B_HALF>
+__device__ __forceinline__ void tc_mma_ss_k128_lane0(uint32_t d_tmem, uint64_t a0, uint64_t b0, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred e, z, o;\n\t.reg .u32 l;\n\t.reg .b64 a, b;\n\t"
+      "mov.u32 l, %%laneid;\n\t"
+      "setp.eq.u32 e, l, 0;\n\t"
+      "setp.ne.b32 z, 0, 0;\n\t"
+      "setp.eq.b32 o, 0, 0;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, z;\n\t"
+      "add.s64 a, %1, 2;\n\tadd.s64 b, %2, 2;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, o;\n\t"
+      "add.s64 a, %1, 4;\n\tadd.s64 b, %2, 4;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, o;\n\t"
+      "add.s64 a, %1, 6;\n\tadd.s64 b, %2, 6;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, o;\n\t"
+      "add.s64 a, %1, %4;\n\tadd.s64 b, %2, %5;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, o;\n\t"
+      "add.s64 a, %1, %4 + 2;\n\tadd.s64 b, %2, %5 + 2;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, o;\n\t"
+      "add.s64 a, %1, %4 + 4;\n\tadd.s64 b, %2, %5 + 4;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, o;\n\t"
+      "add.s64 a, %1, %4 + 6;\n\tadd.s64 b, %2, %5 + 6;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, o;\n\t}"
+      ::"r"(d_tmem), "l"(a0), "l"(b0), "r"(idesc), "n"(A_HALF / 16), "n"(B_HALF / 16) : "memory");
+}
+// Up to four k-steps of 16 keys of O += P . V: P (bf16) in tensor memory, 8 columns per k-step; V
+// pages of 4096 bytes in shared memory.  `first_acc` = 0 overwrites the accumulator at the first k-step.
+__device__ __forceinline__ void tc_mma_ts_pv_lane0(uint32_t d_tmem, uint32_t p_tmem, uint64_t v0, uint32_t idesc, uint32_t first_acc, int n) {
+  asm volatile(
+      "{\n\t.reg .pred e, f, o, q;\n\t.reg .u32 l;\n\t.reg .b32 t;\n\t.reg .b64 b;\n\t"
+      "mov.u32 l, %%laneid;\n\t"
+      "setp.eq.u32 e, l, 0;\n\t"
+      "setp.ne.b32 f, %4, 0;\n\t"
+      "setp.eq.b32 o, 0, 0;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, f;\n\t"
+      "setp.gt.and.s32 q, %5, 1, e;\n\t"
+      "add.u32 t, %1, 8;\n\tadd.s64 b, %2, 256;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [t], b, %3, o;\n\t"
+      "setp.gt.and.s32 q, %5, 2, e;\n\t"
+      "add.u32 t, %1, 16;\n\tadd.s64 b, %2, 512;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [t], b, %3, o;\n\t"
+      "setp.gt.and.s32 q, %5, 3, e;\n\t"
+      "add.u32 t, %1, 24;\n\tadd.s64 b, %2, 768;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [t], b, %3, o;\n\t}"
+      ::"r"(d_tmem), "r"(p_tmem), "l"(v0), "r"(idesc), "r"(first_acc), "r"(n) : "memory");
+}
 __device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 // Barrier among n threads that also ORs a predicate, so that all of them take the same exit.
 __device__ __forceinline__ bool named_sync_or(int id, int n, bool pred) {
