@@ -38,9 +38,9 @@ constexpr bool kSplitS = true;     // scores of a tile as two MMAs of 64 keys (o
 // 2^40 x 2^13 keys x |v| is far from one).  The one-tile variants raise at 2^8.
 constexpr float kRaiseW2 = 40.0f, kRaiseSumW2 = 1099511627776.0f;
 
-// S_FULL / S_EMPTY: one per (group, half of the tile's keys)
-enum BarW2 { WK_FULL = 0, WK_EMPTY = 2, WV_FULL = 4, WV_EMPTY = 6, WS_FULL = 8, WS_EMPTY = 12, WP_FULL = 16, WP_EMPTY = 18,
-             WO_FULL = 20, WQ_FULL = 22, WQ_EMPTY = 23, W2_NUM_BARS = 24 };
+// S_FULL / S_EMPTY / P_FULL: one per (group, half of the tile's keys)
+enum BarW2 { WK_FULL = 0, WK_EMPTY = 2, WV_FULL = 4, WV_EMPTY = 6, WS_FULL = 8, WS_EMPTY = 12, WP_FULL = 16, WP_EMPTY = 20,
+             WO_FULL = 22, WQ_FULL = 24, WQ_EMPTY = 25, W2_NUM_BARS = 26 };
 
 static_assert(kSplitS || !kPInTmem, "P in tensor memory lives in its own score half: the scores must be issued by halves");
 
@@ -69,7 +69,7 @@ __device__ __forceinline__ void softmax_group_w2(const Ctx& c, MiscW2* misc, uin
   const uint32_t s_base = tmem + lane_addr + COL_S + grp * 128, o_base = tmem + lane_addr + COL_O + grp * 128;
   const uint32_t pbuf = base + W2_OFF_P + grp * kPHalfBytes;
   const uint32_t bar_sfull = bars + 8 * (WS_FULL + 2 * grp), bar_sempty = bars + 8 * (WS_EMPTY + 2 * grp),   // + 8 h
-                 bar_pfull = bars + 8 * (WP_FULL + grp), bar_pempty = bars + 8 * (WP_EMPTY + grp), bar_ofull = bars + 8 * (WO_FULL + grp);
+                 bar_pfull = bars + 8 * (WP_FULL + 2 * grp), bar_pempty = bars + 8 * (WP_EMPTY + grp), bar_ofull = bars + 8 * (WO_FULL + grp);
   int g = 0;            // tiles of the CTA so far (both groups count the same)
   int sc[2] = {0, 0}, hc = 0, ic = 0;   // this group's score halves (first / second), P halves and items so far
   bool dead = false;
@@ -95,8 +95,8 @@ __device__ __forceinline__ void softmax_group_w2(const Ctx& c, MiscW2* misc, uin
       for (int h = 0; h < halves; ++h, ++hc) {
         // The scores of the two halves are separate MMAs into separate columns: a half's columns are
         // given back as soon as its pass is final, so its next scores are there before they are needed.
+        if (kSplitS && h > 0) dead |= !mbar_wait(bar_sfull + 8 * h, sc[h] & 1, ab);    // h = 0: waited for above
         if (kSplitS || h == 0) {
-          dead |= !mbar_wait(bar_sfull + 8 * h, sc[h] & 1, ab);
           ++sc[h];
           tc_fence_after();
         }
@@ -107,8 +107,13 @@ __device__ __forceinline__ void softmax_group_w2(const Ctx& c, MiscW2* misc, uin
         // track the largest exponent: packed fp32 pairs (one FFMA and one FADD per two scores), the
         // exponentials, the bf16 pairs.  An exponent beyond 2^40 shows in the sum; the tracking pass
         // then (and for rows that have not seen a key yet) finds the maximum.
-        auto pass = [&](float ref, auto track_tag) {
-          constexpr bool TRACK = decltype(track_tag)::value;
+        // Most halves lie wholly inside what every row of the warp may see (the prefix, full pages): the
+        // warp then takes the pass without any mask arithmetic.
+        const int kb0 = it.key0 + t * kTile + h * 64;
+        const bool plain_row = r >= M || (kb0 + 64 <= vis.x && (ye8[h * 4] & 255) + (ye8[h * 4 + 1] & 255) + (ye8[h * 4 + 2] & 255) + (ye8[h * 4 + 3] & 255) == 64);
+        const bool masked = __any_sync(0xffffffffu, !plain_row);
+        auto pass_impl = [&](float ref, auto track_tag, auto masked_tag) {
+          constexpr bool TRACK = decltype(track_tag)::value, MASKED = decltype(masked_tag)::value;
           float mx0 = -INFINITY, mx1 = -INFINITY;
           float2 sum0 = make_float2(0.f, 0.f), sum1 = sum0, sum2 = sum0, sum3 = sum0;
           const float2 sc2 = make_float2(c.scale_log2, c.scale_log2), nb2 = make_float2(-ref, -ref);
@@ -121,12 +126,13 @@ __device__ __forceinline__ void softmax_group_w2(const Ctx& c, MiscW2* misc, uin
             for (int pg = 0; pg < 2; ++pg) {
               const int nv = (h ? ye8[4 + ch * 2 + pg] : ye8[ch * 2 + pg]) & 255;
               const int kb = it.key0 + t * kTile + h * 64 + ch * 32 + pg * 16;
-              const uint32_t mask = bits_between(0, min(nv, vis.x - kb)) | bits_between(vis.y - kb, min(nv, vis.z - kb));
+              uint32_t mask = 0xFFFFu;
+              if constexpr (MASKED) mask = bits_between(0, min(nv, vis.x - kb)) | bits_between(vis.y - kb, min(nv, vis.z - kb));
 #pragma unroll
               for (int i = 0; i < 16; i += 4) {
                 float2 x0 = __ffma2_rn(make_float2(s[pg * 16 + i], s[pg * 16 + i + 1]), sc2, nb2);
                 float2 x1 = __ffma2_rn(make_float2(s[pg * 16 + i + 2], s[pg * 16 + i + 3]), sc2, nb2);
-                if (mask != 0xFFFFu) {
+                if (MASKED && mask != 0xFFFFu) {
                   x0.x = (mask >> i) & 1u ? x0.x : -INFINITY;
                   x0.y = (mask >> (i + 1)) & 1u ? x0.y : -INFINITY;
                   x1.x = (mask >> (i + 2)) & 1u ? x1.x : -INFINITY;
@@ -144,6 +150,10 @@ __device__ __forceinline__ void softmax_group_w2(const Ctx& c, MiscW2* misc, uin
           const float2 st = __fadd2_rn(__fadd2_rn(sum0, sum1), __fadd2_rn(sum2, sum3));
           tile_sum = st.x + st.y;
           tmax = fmaxf(mx0, mx1);
+        };
+        auto pass = [&](float ref, auto track_tag) {
+          if (masked) pass_impl(ref, track_tag, std::true_type());
+          else pass_impl(ref, track_tag, std::false_type());
         };
         const bool need_track = __any_sync(0xffffffffu, !seen);
         if (need_track) pass(m_ref, std::true_type());
@@ -191,9 +201,8 @@ __device__ __forceinline__ void softmax_group_w2(const Ctx& c, MiscW2* misc, uin
           // MMA warp frees these columns for the next tile's scores when this half's P.V is done
           ASPD_TMEM_ST32U(s_base + h * 64, pk, 0);
           tmem_wait_st();
-          // one barrier announces both halves in turn, and a parity tells only its two latest phases
-          // apart: the previous half's P.V must have been taken before this half is announced
-          if (hc > 0) dead |= !mbar_wait(bar_pempty, (hc - 1) & 1, ab);
+          // (each half has its own barrier: the scores that P replaces were issued only after the
+          // half's previous P.V was done, so its previous announcement has been taken)
           if (tid == 0) ASPD_STAMP(c, g, 4 * h + 2);
         } else {
           if (hc > 0) dead |= !mbar_wait(bar_pempty, (hc - 1) & 1, ab);   // the P half buffer is free again
@@ -207,7 +216,7 @@ __device__ __forceinline__ void softmax_group_w2(const Ctx& c, MiscW2* misc, uin
           fence_async_smem();
         }
         tc_fence_before();
-        mbar_arrive(bar_pfull);
+        mbar_arrive(bar_pfull + (kPInTmem ? 8 * h : 0));
         if (tid == 0) ASPD_STAMP(c, g, 4 * h + 3);
       }
     }
@@ -259,9 +268,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_w2_kernel(Ctx c) {
       reinterpret_cast<int*>(misc->items)[e] = reinterpret_cast<const int*>(c.pd.items + item_begin)[e];
   }
   if (tid == 0) {
-    //                               K_FULL K_EMPTY V_FULL V_EMPTY S_FULL(4)   S_EMPTY(4)          P_FULL    P_EMPTY O_FULL Q_FULL Q_EMPTY
+    //                               K_FULL K_EMPTY V_FULL V_EMPTY S_FULL(4)   S_EMPTY(4)          P_FULL(4)           P_EMPTY O_FULL Q_FULL Q_EMPTY
     const int se = kPInTmem ? 1 : 128;      // who gives a score half's columns back: the MMA warp's commit, or the 128 threads that read them
-    const int counts[W2_NUM_BARS] = {1, 1,  2, 2,   1, 1,  2, 2,   1, 1, 1, 1,  se, se, se, se, 128, 128, 1, 1,   1, 1,  128,   2};
+    const int counts[W2_NUM_BARS] = {1, 1,  2, 2,   1, 1,  2, 2,   1, 1, 1, 1,  se, se, se, se, 128, 128, 128, 128, 1, 1,   1, 1,  128,   2};
     for (int i = 0; i < W2_NUM_BARS; ++i) mbar_init(bars + 8 * i, counts[i]);
     misc->abort_flag = 0;
     misc->lead[0] = item_begin; misc->lead[1] = item_begin;
@@ -352,7 +361,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_w2_kernel(Ctx c) {
     volatile int* lead = misc->lead;
     const uint32_t idesc_pv = instr_desc(128, 1);
     const uint32_t o_tmem = tmem_u + COL_O + grp * 128, p_tmem = tmem_u + COL_S + grp * 128;
-    int gbase = 0, count = 0;
+    int gbase = 0, cnt_p[2] = {0, 0};        // P.V operations so far on either half
     bool ok = true;
     for (int idx = ib; idx < ie && ok; ++idx) {
       const DeviceItem it = get_item_w2(c, misc, idx, ib);
@@ -369,8 +378,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_w2_kernel(Ctx c) {
         for (int t = 0; t < n_tiles && ok; ++t) {
           const int g = gbase + t, npg = min(8, n_pages - t * 8), halves = npg > 4 ? 2 : 1;
           const uint32_t vbuf = base_u + W2_OFF_V + (g & 1) * kTileBytes;
-          for (int h = 0; h < halves && ok; ++h, ++count) {
-            ok = wait_all(bars_u + 8 * (WP_FULL + grp), count & 1) && (h > 0 || wait_all(bars_u + 8 * (WV_FULL + (g & 1)), (g >> 1) & 1));
+          for (int h = 0; h < halves && ok; ++h) {
+            const int ph = kPInTmem ? h : 0;
+            ok = wait_all(bars_u + 8 * (WP_FULL + 2 * grp + ph), cnt_p[ph] & 1) && (h > 0 || wait_all(bars_u + 8 * (WV_FULL + (g & 1)), (g >> 1) & 1));
+            ++cnt_p[ph];
             if (!ok) break;
             tc_fence_after();
             if (lane == 0 && grp == 0 && h == 0) ASPD_STAMP(c, g, 15);
