@@ -83,6 +83,7 @@ __device__ __forceinline__ void softmax_group_w2(const Ctx& c, MiscW2* misc, uin
     if (r < M) vis = c.pd.tok_vis[tok];
     float m_ref = 0.f, l = 0.f;                                 // see the one-tile variant: the reference starts at 0
     bool seen = r >= M;                                         // padding rows never need the tracking pass
+    bool warp_seen = false;                                     // all rows of the warp have (kept up in the full path only)
     for (int t = 0; t < n_tiles; ++t, ++g) {
       const int npg = min(8, it.n_pages - t * 8), halves = npg > 4 ? 2 : 1;
       // the tile's page entries, taken when its first scores are there: the ring slot may be rewritten
@@ -155,40 +156,43 @@ __device__ __forceinline__ void softmax_group_w2(const Ctx& c, MiscW2* misc, uin
           if (masked) pass_impl(ref, track_tag, std::true_type());
           else pass_impl(ref, track_tag, std::false_type());
         };
-        const bool need_track = __any_sync(0xffffffffu, !seen);
-        if (need_track) pass(m_ref, std::true_type());
-        else {
+        // The common case -- every row of the warp has seen a key and no exponent passed 2^40 -- is
+        // the plain pass and one vote; everything else goes the full way.
+        bool settled = false;
+        if (warp_seen) {
           pass(m_ref, std::false_type());
           // an exponent beyond 2^40 makes the sum exceed it (the converse is harmless: one more pass)
-          if (__any_sync(0xffffffffu, !(tile_sum <= kRaiseSumW2))) pass(m_ref, std::true_type());
-          else tmax = 0.f;
+          settled = !__any_sync(0xffffffffu, !(tile_sum <= kRaiseSumW2));
         }
-        // move the reference: up when an exponent passed 2^40; down only while the row has not seen a
-        // key yet (l and its row of O are still exactly 0 then, so nothing is rescaled)
-        const bool raise = tmax > kRaiseW2, lower = !seen && tmax < -kLower && tmax > -INFINITY;
-        const bool upd = raise || lower;
-        seen |= tmax > -INFINITY;
-        float alpha = 1.f;
-        if (raise) alpha = ex2(-tmax);
-        if (upd) m_ref += tmax;
-        l *= alpha;
-        const bool any_upd = __any_sync(0xffffffffu, upd);
-        if (any_upd) {
-          if (t > 0 || h > 0) {                     // the rows' O so far is rescaled in TMEM (the warp together)
-            dead |= !mbar_wait(bar_pempty, (hc - 1) & 1, ab);      // the P.V of the previous half is done
-            tc_fence_after();
+        if (!settled) {
+          pass(m_ref, std::true_type());
+          // move the reference: up when an exponent passed 2^40; down only while the row has not seen a
+          // key yet (l and its row of O are still exactly 0 then, so nothing is rescaled)
+          const bool raise = tmax > kRaiseW2, lower = !seen && tmax < -kLower && tmax > -INFINITY;
+          const bool upd = raise || lower;
+          seen |= tmax > -INFINITY;
+          warp_seen = !__any_sync(0xffffffffu, !seen);
+          float alpha = 1.f;
+          if (raise) alpha = ex2(-tmax);
+          if (upd) m_ref += tmax;
+          l *= alpha;
+          if (__any_sync(0xffffffffu, upd)) {
+            if (t > 0 || h > 0) {                     // the rows' O so far is rescaled in TMEM (the warp together)
+              dead |= !mbar_wait(bar_pempty, (hc - 1) & 1, ab);      // the P.V of the previous half is done
+              tc_fence_after();
 #pragma unroll 1
-            for (int q4 = 0; q4 < 4; ++q4) {
-              float o[32];
-              ASPD_TMEM_LD32(o_base + q4 * 32, o, 0);
-              tmem_wait_ld();
+              for (int q4 = 0; q4 < 4; ++q4) {
+                float o[32];
+                ASPD_TMEM_LD32(o_base + q4 * 32, o, 0);
+                tmem_wait_ld();
 #pragma unroll
-              for (int i = 0; i < 32; ++i) o[i] *= alpha;
-              ASPD_TMEM_ST32(o_base + q4 * 32, o, 0);
+                for (int i = 0; i < 32; ++i) o[i] *= alpha;
+                ASPD_TMEM_ST32(o_base + q4 * 32, o, 0);
+              }
+              tmem_wait_st();
             }
-            tmem_wait_st();
+            pass(m_ref, std::false_type());           // the whole warp again (TMEM loads are warp-wide)
           }
-          pass(m_ref, std::false_type());           // the whole warp again (TMEM loads are warp-wide)
         }
         l += tile_sum;
         if (!kPInTmem && (kSplitS || h == halves - 1)) {   // the scores are read: the MMA warp may overwrite them
