@@ -941,13 +941,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
         if (lane == 0) ASPD_STAMP(c, g, 8);
         const uint32_t qbuf = base_u + OFF_Q + tr.qb * kTileBytes, kbuf = base_u + OFF_K + sb * kTileBytes;
         const uint32_t idesc_s = instr_desc((uint32_t)tr.npg * 16u, 0, mma_m);
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          // k-step ks covers head_dim elements [16 ks, 16 ks + 16): span ks / 4, 32 bytes per step
-          const uint64_t a = smem_desc(qbuf + (ks >> 2) * kHalf + (ks & 3) * 32, 16, 1024);
-          const uint64_t b = smem_desc(kbuf + (ks >> 2) * 1024 + (ks & 3) * 32, 16, 2048);
-          tc_mma_lane0(tmem_u + COL_S + sb * 128, a, b, idesc_s, ks > 0 ? 1u : 0u);
-        }
+        // k-step ks covers head_dim elements [16 ks, 16 ks + 16): span ks / 4, 32 bytes per step
+        tc_mma_ss_k128_lane0<kHalf, 1024>(tmem_u + COL_S + sb * 128, smem_desc(qbuf, 16, 1024), smem_desc(kbuf, 16, 2048), idesc_s);
         if (lane == 0) ASPD_STAMP(c, g, 9);
         tc_commit_lane0(bars_u + 8 * (S_FULL + sb));
         tc_commit_lane0(bars_u + 8 * (K_EMPTY + sb));
@@ -962,14 +957,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_tc_kernel(Ctx c) {
         if (tr.first && !wait_all(bars_u + 8 * (O_EMPTY + tr.ob), ((tr.item_no >> 1) & 1) ^ 1)) return false;
         tc_fence_after();
         const uint32_t pbuf = base_u + OFF_P, vbuf = base_u + OFF_V + (g & 1) * kTileBytes;
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          if (ks < tr.npg) {
-            const uint64_t a = smem_desc(pbuf + (ks >> 2) * kHalf + (ks & 3) * 32, 16, 1024);
-            const uint64_t b = smem_desc(vbuf + ks * 4096, 1024, 2048);   // 16 keys = one page per k-step
-            tc_mma_lane0(tmem_u + COL_O + tr.ob * 128, a, b, idesc_pv, (!tr.first || ks > 0) ? 1u : 0u);
-          }
-        }
+        // 16 keys = one page per k-step
+        tc_mma_ss_pv_lane0<kHalf>(tmem_u + COL_O + tr.ob * 128, smem_desc(pbuf, 16, 1024), smem_desc(vbuf, 1024, 2048), idesc_pv,
+                                  tr.first ? 0u : 1u, tr.npg);
         if (lane == 0) ASPD_STAMP(c, g, 12);
         tc_commit_lane0(bars_u + 8 * P_EMPTY);
         tc_commit_lane0(bars_u + 8 * (V_EMPTY + (g & 1)));

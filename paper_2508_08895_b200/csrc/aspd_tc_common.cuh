@@ -150,6 +150,41 @@ __device__ __forceinline__ void tc_mma_ts_pv_lane0(uint32_t d_tmem, uint32_t p_t
       "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [t], b, %3, o;\n\t}"
       ::"r"(d_tmem), "r"(p_tmem), "l"(v0), "r"(idesc), "r"(first_acc), "r"(n) : "memory");
 }
+// Up to eight k-steps of 16 keys of O += P . V with both operands in shared memory: P K-major in two
+// spans of 64 keys (A_HALF bytes apart), V pages of 4096 bytes.  `first_acc` = 0 overwrites the
+// accumulator at the first k-step; k-steps at and beyond n are skipped.
+template <uint32_t A_HALF>
+__device__ __forceinline__ void tc_mma_ss_pv_lane0(uint32_t d_tmem, uint64_t p0, uint64_t v0, uint32_t idesc, uint32_t first_acc, int n) {
+  asm volatile(
+      "{\n\t.reg .pred e, f, o, q;\n\t.reg .u32 l;\n\t.reg .b64 a, b;\n\t"
+      "mov.u32 l, %%laneid;\n\t"
+      "setp.eq.u32 e, l, 0;\n\t"
+      "setp.ne.b32 f, %4, 0;\n\t"
+      "setp.eq.b32 o, 0, 0;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, f;\n\t"
+      "setp.gt.and.s32 q, %5, 1, e;\n\t"
+      "add.s64 a, %1, 2;\n\tadd.s64 b, %2, 256;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, o;\n\t"
+      "setp.gt.and.s32 q, %5, 2, e;\n\t"
+      "add.s64 a, %1, 4;\n\tadd.s64 b, %2, 512;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, o;\n\t"
+      "setp.gt.and.s32 q, %5, 3, e;\n\t"
+      "add.s64 a, %1, 6;\n\tadd.s64 b, %2, 768;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, o;\n\t"
+      "setp.gt.and.s32 q, %5, 4, e;\n\t"
+      "add.s64 a, %1, %6;\n\tadd.s64 b, %2, 1024;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, o;\n\t"
+      "setp.gt.and.s32 q, %5, 5, e;\n\t"
+      "add.s64 a, %1, %6 + 2;\n\tadd.s64 b, %2, 1280;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, o;\n\t"
+      "setp.gt.and.s32 q, %5, 6, e;\n\t"
+      "add.s64 a, %1, %6 + 4;\n\tadd.s64 b, %2, 1536;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, o;\n\t"
+      "setp.gt.and.s32 q, %5, 7, e;\n\t"
+      "add.s64 a, %1, %6 + 6;\n\tadd.s64 b, %2, 1792;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, o;\n\t}"
+      ::"r"(d_tmem), "l"(p0), "l"(v0), "r"(idesc), "r"(first_acc), "r"(n), "n"(A_HALF / 16) : "memory");
+}
 __device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 // Barrier among n threads that also ORs a predicate, so that all of them take the same exit.
 __device__ __forceinline__ bool named_sync_or(int id, int n, bool pred) {
