@@ -14,18 +14,20 @@ template <> __device__ inline __nv_bfloat16 combine_from_f32<__nv_bfloat16>(floa
 // Records p0 .. p0 + n - 1 of KV-head group member g; lane owns D / 32 consecutive output elements.
 // The records are read past L1 (ld.global.cg): inside the attention kernel they were written by
 // other CTAs of the same launch.
-template <typename T, int D>
+// PREFETCH: the next round's records are requested before this round is folded in (same arithmetic in
+// the same order, so the same bits; a row cut into 37 parts then costs about one memory round trip
+// plus five short rounds instead of five round trips).
+template <typename T, int D, bool PREFETCH = false>
 __device__ __forceinline__ void combine_row(const float* __restrict__ ws_o, const float2* __restrict__ ws_ml, int p0, int n, int G,
                                             int g, int lane, T* __restrict__ dst) {
   constexpr int EPL = D / 32;
   float M = -INFINITY, L = 0.f, acc[EPL];
 #pragma unroll
   for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-  for (int b0 = 0; b0 < n; b0 += 8) {
+  auto fetch = [&](int b0, float2& ml, float (&v)[8][EPL]) {
     const int cnt = min(8, n - b0);
-    float2 ml = make_float2(-INFINITY, 0.f);
+    ml = make_float2(-INFINITY, 0.f);
     if (lane < cnt) ml = __ldcg(ws_ml + (size_t)(p0 + b0 + lane) * G + g);
-    float v[8][EPL];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
       const float* row = ws_o + ((size_t)(p0 + b0 + min(u, cnt - 1)) * G + g) * D + lane * EPL;
@@ -36,6 +38,17 @@ __device__ __forceinline__ void combine_row(const float* __restrict__ ws_o, cons
         const float2 x = __ldcg(reinterpret_cast<const float2*>(row));
         v[u][0] = x.x; v[u][1] = x.y;
       }
+    }
+  };
+  float2 ml, ml_next = make_float2(-INFINITY, 0.f);
+  float v[8][EPL], v_next[8][EPL];
+  if (PREFETCH && n > 0) fetch(0, ml, v);
+  for (int b0 = 0; b0 < n; b0 += 8) {
+    const int cnt = min(8, n - b0);
+    if constexpr (PREFETCH) {
+      if (b0 + 8 < n) fetch(b0 + 8, ml_next, v_next);
+    } else {
+      fetch(b0, ml, v);
     }
     float mb = ml.y > 0.f ? ml.x : -INFINITY;     // records of chunks with no visible key have sum 0
 #pragma unroll
@@ -57,6 +70,13 @@ __device__ __forceinline__ void combine_row(const float* __restrict__ ws_o, cons
       const float wi = __shfl_sync(0xffffffffu, wt, u);
 #pragma unroll
       for (int e = 0; e < EPL; ++e) acc[e] += wi != 0.f ? v[u][e] * wi : 0.f;   // a skipped record may hold anything
+    }
+    if constexpr (PREFETCH) {
+      ml = ml_next;
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) v[u][e] = v_next[u][e];
     }
   }
   const float inv = 1.f / L;

@@ -358,7 +358,7 @@ __global__ void combine_kernel(PlanDevice pd, T* __restrict__ out, int n_new, in
   const int p0 = pd.part_base[tok * n_kv_heads + h], n = pd.part_base[tok * n_kv_heads + h + 1] - p0;
   pdl_wait();
   if (!active) return;
-  combine_row<T, D>(pd.ws_o, pd.ws_ml, p0, n, G, g, lane, out + ((size_t)tok * n_q_heads + hq) * D);
+  combine_row<T, D, true>(pd.ws_o, pd.ws_ml, p0, n, G, g, lane, out + ((size_t)tok * n_q_heads + hq) * D);
 }
 
 template <typename T>
