@@ -30,7 +30,7 @@ constexpr uint32_t kPHalfBytes = 16384;       // 128 rows x 64 keys x 2 B: one 1
 constexpr size_t kSmemBytesW2 = 7 * kTileBytes + 2048 + 1024;   // + Misc + slack to align the base to 1024
 constexpr int kItemCacheW2 = 8;
 constexpr bool kPolyExp = true;     // plain pass: a quarter of the exponentials as a cubic on the FMA pipe (10 % fewer cycles per tile;
-                                    // under the power cap 883-888 against 889-898 us on the masked-prefill workload)
+                                    // under the power cap, same box: none 894-899 us, an eighth 881-882, a quarter 873-879, half 923-928)
 constexpr bool kPInTmem = true;    // P halves go into the first 32 columns of their own score half in tensor memory and are the
                                    // A operand of P.V from there (no shared-memory round trip); needs kSplitS
 constexpr bool kSplitS = true;     // scores of a tile as two MMAs of 64 keys (own columns and barriers each: a half's columns are
