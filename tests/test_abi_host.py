@@ -342,6 +342,36 @@ def test_malformed_descriptors_are_rejected_without_launching():
     assert _plan_rc(wl, good, kernel=B.KERNEL_MMA) == -3
 
 
+def test_rerotation_by_ranges_checks_its_arguments_before_any_launch():
+    """aspd_k_rerotate_ranges / _layers validate on the host (nothing here reaches the device): a
+    negative count, base or slot, missing or misaligned pools, a negative layer count; no layer and
+    no range are valid and do nothing."""
+    import ctypes
+    L = B.lib()
+    sh = B.make_shape(28, 4, 128, 16, "bf16", 1e6, 0.088)
+    shp = ctypes.addressof(sh)
+    ranges = np.array([[0, 16, 5, 3]], dtype=np.int32)
+    table = np.zeros(4, dtype=np.int32)
+    fake = ctypes.c_void_p(4096)                     # non-null, 16-byte aligned; never dereferenced on these paths
+    pools = (ctypes.c_void_p * 2)(4096, 8192)
+    rp, tp = ranges.ctypes.data, table.ctypes.data
+    assert L.aspd_k_rerotate_ranges_layers(shp, pools, 0, tp, rp, 1, None) == 0          # no layer
+    assert L.aspd_k_rerotate_ranges_layers(shp, pools, 2, tp, rp, 0, None) == 0          # no range
+    assert L.aspd_k_rerotate_ranges_layers(shp, pools, -1, tp, rp, 1, None) == -1
+    assert L.aspd_k_rerotate_ranges_layers(shp, pools, 2, tp, rp, -1, None) == -1
+    assert L.aspd_k_rerotate_ranges_layers(shp, None, 2, tp, rp, 1, None) == -1
+    assert L.aspd_k_rerotate_ranges_layers(shp, pools, 2, None, rp, 1, None) == -1
+    assert L.aspd_k_rerotate_ranges_layers(shp, (ctypes.c_void_p * 2)(4096, 0), 2, tp, rp, 1, None) == -1     # a missing pool
+    assert L.aspd_k_rerotate_ranges_layers(shp, (ctypes.c_void_p * 2)(4096, 8200), 2, tp, rp, 1, None) == -1  # misaligned
+    assert L.aspd_k_rerotate_ranges(shp, None, tp, rp, 1, None) == -1
+    for bad in ([-1, 16, 5, 3], [0, -16, 5, 3], [0, 16, -5, 3], [0, 2**31 - 4, 8, 3]):
+        r = np.array([[0, 0, 0, 9], bad], dtype=np.int32)
+        assert L.aspd_k_rerotate_ranges_layers(shp, pools, 2, tp, r.ctypes.data, 2, None) == -2
+        assert L.aspd_k_rerotate_ranges(shp, fake, tp, r.ctypes.data, 2, None) == -2
+    bad_shape = B.make_shape(4, 2, 96, 16, "f32", 1e4, 0.1)
+    assert L.aspd_k_rerotate_ranges_layers(ctypes.addressof(bad_shape), pools, 2, tp, rp, 1, None) == -3
+
+
 def test_empty_inputs():
     wl = W.build_segment_workload("e", 8, 4, 2, 64, "f32", 1e4, [20], [[5, 9]], [[1, 1]])
     desc = {k: v.copy() for k, v in wl.phases[-1].desc.items()}
