@@ -635,6 +635,44 @@ def test_two_tile_row_blocks_at_their_edges(n_ctas):
     compare_workload(wl, n_ctas=n_ctas, fused=True, stable_cache=True)
 
 
+def test_two_tile_plain_pass_with_huge_and_tiny_exponents():
+    """The two-tile variant's common pass takes a quarter of its exponentials as a cubic with the
+    exponent bits patched in (keys 6, 7, 14, 15 of every page) and judges an overflow from the sum.
+    Prefix keys scaled by 400 at such places, deep inside the prefix (full, unmasked halves): for some
+    rows their logits are far above 2^127 relative to the reference (the clamp keeps the patched
+    exponent in range, the sum shows the overflow, the reference is raised), for others far below
+    2^-126 (weights that must vanish, not wrap around).  A row whose jump is positive puts nearly
+    all its weight on that key, so the output is close to that key's V row."""
+    E = engine()
+    wl = W.build_segment_workload("w2jump", 67, 28, 4, 128, "bf16", 1e6, [600, 300, 400], [[0, 5], [3], [0]], [[30, 25], [36], [20]])
+    fill = [p for p in wl.phases if p.label == "fill-prefix"][0]
+    # one scaled key per request (two would tie for some rows, and a tie between logits of several
+    # hundred is decided by the bf16 rounding of the cached keys): slots 310 and 150 take the cubic,
+    # slot 305 the special-function unit
+    for slot in (310, 600 + 150, 900 + 305):
+        fill.k_new[slot] *= 400.0
+    shape = B.make_shape(wl.Hq, wl.Hkv, wl.d, wl.page_size, wl.dtype, wl.theta, wl.sm_scale)
+    ph = [x for x in wl.phases if x.label == "parallel-step"][0]
+    plan = B.Plan(shape, ph.desc, wl.n_pool_pages, ph.mode, n_ctas=3, host_only=True)
+    assert plan.info.dealt and plan.info.max_rows_per_item == 256
+    plan.destroy()
+    ref = oracle_run(wl)
+    for n_ctas in (3, 1):
+        run = E.run_workload(wl, n_ctas=n_ctas)
+        g, r = run.outputs[0].astype(np.float64), ref.outputs[0]
+        err = np.abs(g - r)
+        assert np.isfinite(g).all()
+        # A cached key 400 times the usual size carries 400 times the usual rounding error (several
+        # units of its logit), so a row for which the scaled key's logit falls within ten units of its
+        # other keys' largest puts a different weight on it than the oracle does (up to all or none:
+        # errors of the size of a V row).  Those rows are about 1 %.  A wrapped exponent or a missed
+        # overflow spoils the many rows whose scaled key is hundreds of units above or below everything
+        # else (measured with the upper clamp taken out: mean error 1.2e-2 instead of 8e-4, 97.6 %
+        # of the rows within 3e-2 instead of 99.0 %; without the lower clamp: not finite).
+        row_err = err.reshape(-1, err.shape[-1]).max(axis=1)
+        assert (row_err <= 3e-2).mean() >= 0.985 and err.mean() <= 2e-3, ((row_err <= 3e-2).mean(), err.max(), err.mean())
+
+
 def test_large_decode_batch_takes_the_dealt_plan():
     """A decode step with many more (request, KV head) streams than CTAs: whole streams are dealt
     out, the append is still fused into the attention launch (few new rows per CTA), the kernel
