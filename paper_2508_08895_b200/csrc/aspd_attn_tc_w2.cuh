@@ -91,14 +91,22 @@ __device__ __forceinline__ void softmax_group_w2(const Ctx& c, MiscW2* misc, uin
       // the tile's page entries, taken when its first scores are there: the ring slot may be rewritten
       // while this group is still in its pass (the other group, alone in later items, can run several
       // tiles ahead)
-      dead |= !mbar_wait(bar_sfull, sc[0] & 1, ab);
+      if (!mbar_test(bar_sfull, sc[0] & 1)) dead |= !mbar_wait(bar_sfull, sc[0] & 1, ab);
       int ye8[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) ye8[i] = misc->nval[g & 3][i];
+      {
+        const int4 ya = *reinterpret_cast<const int4*>(&misc->nval[g & 3][0]), yb = *reinterpret_cast<const int4*>(&misc->nval[g & 3][4]);
+        ye8[0] = ya.x; ye8[1] = ya.y; ye8[2] = ya.z; ye8[3] = ya.w; ye8[4] = yb.x; ye8[5] = yb.y; ye8[6] = yb.z; ye8[7] = yb.w;
+      }
+      // Most halves lie wholly inside what every row of the warp may see (the prefix, full pages): the
+      // warp then takes the pass without any mask arithmetic.  Both halves' verdicts are taken here.
+      const int kbt = it.key0 + t * kTile;
+      const bool plain0 = r >= M || (kbt + 64 <= vis.x && (ye8[0] & 255) + (ye8[1] & 255) + (ye8[2] & 255) + (ye8[3] & 255) == 64);
+      const bool plain1 = r >= M || (kbt + 128 <= vis.x && (ye8[4] & 255) + (ye8[5] & 255) + (ye8[6] & 255) + (ye8[7] & 255) == 64);
+      const bool masked0 = __any_sync(0xffffffffu, !plain0), masked1 = __any_sync(0xffffffffu, !plain1);
       for (int h = 0; h < halves; ++h, ++hc) {
         // The scores of the two halves are separate MMAs into separate columns: a half's columns are
         // given back as soon as its pass is final, so its next scores are there before they are needed.
-        if (kSplitS && h > 0) dead |= !mbar_wait(bar_sfull + 8 * h, sc[h] & 1, ab);    // h = 0: waited for above
+        if (kSplitS && h > 0 && !mbar_test(bar_sfull + 8 * h, sc[h] & 1)) dead |= !mbar_wait(bar_sfull + 8 * h, sc[h] & 1, ab);    // h = 0: waited for above
         if (kSplitS || h == 0) {
           ++sc[h];
           tc_fence_after();
@@ -110,11 +118,8 @@ __device__ __forceinline__ void softmax_group_w2(const Ctx& c, MiscW2* misc, uin
         // track the largest exponent: packed fp32 pairs (one FFMA and one FADD per two scores), the
         // exponentials, the bf16 pairs.  An exponent beyond 2^40 shows in the sum; the tracking pass
         // then (and for rows that have not seen a key yet) finds the maximum.
-        // Most halves lie wholly inside what every row of the warp may see (the prefix, full pages): the
-        // warp then takes the pass without any mask arithmetic.
-        const int kb0 = it.key0 + t * kTile + h * 64;
-        const bool plain_row = r >= M || (kb0 + 64 <= vis.x && (ye8[h * 4] & 255) + (ye8[h * 4 + 1] & 255) + (ye8[h * 4 + 2] & 255) + (ye8[h * 4 + 3] & 255) == 64);
-        const bool masked = __any_sync(0xffffffffu, !plain_row);
+        const int kb0 = kbt + h * 64;
+        const bool masked = h ? masked1 : masked0;
         auto pass_impl = [&](float ref, auto track_tag, auto masked_tag) {
           constexpr bool TRACK = decltype(track_tag)::value, MASKED = decltype(masked_tag)::value;
           float mx0 = -INFINITY, mx1 = -INFINITY;
