@@ -14,9 +14,9 @@ template <> __device__ inline __nv_bfloat16 combine_from_f32<__nv_bfloat16>(floa
 // Records p0 .. p0 + n - 1 of KV-head group member g; lane owns D / 32 consecutive output elements.
 // The records are read past L1 (ld.global.cg): inside the attention kernel they were written by
 // other CTAs of the same launch.
-// PREFETCH: the next round's records are requested before this round is folded in (same arithmetic in
-// the same order, so the same bits; a row cut into 37 parts then costs about one memory round trip
-// plus five short rounds instead of five round trips).
+// PREFETCH: the next eight records are requested before the current eight are folded in (same
+// arithmetic in the same order, so the same bits; a row cut into 37 parts then costs about one
+// memory round trip plus five short steps instead of five round trips).
 template <typename T, int D, bool PREFETCH = false>
 __device__ __forceinline__ void combine_row(const float* __restrict__ ws_o, const float2* __restrict__ ws_ml, int p0, int n, int G,
                                             int g, int lane, T* __restrict__ dst) {
@@ -53,7 +53,7 @@ __device__ __forceinline__ void combine_row(const float* __restrict__ ws_o, cons
     float mb = ml.y > 0.f ? ml.x : -INFINITY;     // records of chunks with no visible key have sum 0
 #pragma unroll
     for (int o = 4; o; o >>= 1) mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, o));
-    mb = __shfl_sync(0xffffffffu, mb, 0);         // maximum over the round's records (lanes 0..7)
+    mb = __shfl_sync(0xffffffffu, mb, 0);         // maximum over the eight records (lanes 0..7)
     const float m_new = fmaxf(M, mb);
     const float alpha = m_new == -INFINITY ? 1.f : exp2f(M - m_new);   // M = -inf: alpha = 0
     L *= alpha;
