@@ -51,7 +51,25 @@ def build_debug_bounds(force: bool = False) -> str:
     return LIB_DEBUG_BOUNDS
 
 
+def build_probes() -> str:
+    """Stand-alone timing probes of the tensor-core kernels' building blocks (csrc/probes/*.cu -> csrc/probes/bin/)."""
+    out_dir = os.path.join(CSRC, "probes", "bin")
+    os.makedirs(out_dir, exist_ok=True)
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    for src in sorted(glob.glob(os.path.join(CSRC, "probes", "*.cu"))):
+        exe = os.path.join(out_dir, os.path.splitext(os.path.basename(src))[0])
+        cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
+               "-o", exe, src]
+        res = subprocess.run(cmd, capture_output=True, text=True)
+        if res.returncode != 0:
+            raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+    return out_dir
+
+
 if __name__ == "__main__":
+    if "--probes" in sys.argv:
+        print(build_probes())
+        sys.exit(0)
     if "--debug-bounds" in sys.argv:
         print(build_debug_bounds(force=True))
     else:
