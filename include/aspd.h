@@ -440,6 +440,7 @@ int aspd_k_rerotate(const aspd_shape_t* shape, void* k_pool /*device*/, const in
  * derives page and row itself, so no per-token index arrays exist or are read.
  *   page_table  device int32, the concatenated page tables (as aspd_plan_create's page_ids)
  *   ranges      HOST int32[n_ranges][4]; they travel in the launch parameters, 512 per launch
+ * The ranges of one call must not overlap (every key is read and written once, by one block).
  * ASPD_ERR_BAD_DESCRIPTOR for a negative base, slot or count.
  */
 int aspd_k_rerotate_ranges(const aspd_shape_t* shape, void* k_pool /*device*/, const int32_t* page_table /*device*/,

@@ -807,6 +807,32 @@ def test_same_re_serial_decoding_after_rerotation():
         check(got, want, wl.dtype, "same-re serial step")
 
 
+def test_rerotation_by_ranges_in_several_launches():
+    """More ranges than one launch carries (512) and more pools than one launch carries (64): 603
+    single-token ranges over 70 pools in one call give the bits of three whole-branch ranges applied
+    to a pool by itself.  (The ranges of one call must not overlap: every key is read and written once.)"""
+    import torch
+    E = engine()
+    wl = W.build_segment_workload("re-many", 29, 28, 4, 128, "bf16", 1e6, [16], [[200, 200, 200]], [[1, 1, 1]])
+    run = E.run_workload(wl)
+    d = wl.phases[-1].desc
+    t = lambda x: torch.tensor(x, dtype=torch.int32, device="cuda")
+    table = t(d["page_ids"].tolist())
+    whole, moved = [], 0
+    for b in range(3):
+        whole.append((0, int(d["br_kv_off"][b]), int(d["br_kv_len"][b]), moved))
+        moved += int(d["br_kv_len"][b])
+    single = [(base, s0 + i, 1, dl) for (base, s0, n, dl) in whole for i in range(n)]
+    assert len(single) == 603
+    want = run.cache.k.clone()
+    B.k_rerotate_ranges(run.shape, want, table, np.array(whole, dtype=np.int32))
+    pools = [run.cache.k.clone() for _ in range(70)]
+    B.k_rerotate_ranges_layers(run.shape, pools, table, np.array(single, dtype=np.int32))
+    torch.cuda.synchronize()
+    assert not torch.equal(want, run.cache.k)
+    assert all(torch.equal(x, want) for x in pools)
+
+
 @pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("kernel", KERNELS)
 def test_shared_mask_variant(kernel, fused):
