@@ -427,7 +427,7 @@ int aspd_debug_read_token(const aspd_shape_t* shape, const void* pool /*device*/
  * compose, re-rotating the cached keys does the same with one read and one write per key and no
  * model pass.  Token t is row rows[t] of physical page pages[t] (all KV heads); delta[t] may be
  * negative.  pages, rows, delta: device int32[n].  V is untouched.  Each call rounds the keys to
- * the storage dtype once more.
+ * the storage dtype once more.  A token must not be listed twice in one call.
  */
 int aspd_k_rerotate(const aspd_shape_t* shape, void* k_pool /*device*/, const int32_t* pages /*device*/,
                     const int32_t* rows /*device*/, const int32_t* delta /*device*/, int n, void* stream);
